@@ -1,0 +1,305 @@
+"""Pins for the CPU oracle: every check compares it with something other than itself --
+hand-derived values, brute force written independently in numpy/Python, algebraic identities
+the paper states, closed forms and library routines."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+
+
+def _offsets(w):
+    return np.concatenate([[0], np.cumsum(w)]).astype(int)
+
+
+def _rand_ints(rng, shape, lo=-3, hi=3):
+    return rng.integers(lo, hi + 1, size=shape).astype(np.float64)
+
+
+# ---- P7: hand-derived examples (tests/golden/hand_examples.json) ------------------------------
+
+@pytest.mark.parametrize("key", ["typed_q2", "typed_q3"])
+def test_hand_examples_typed(golden, key):
+    g = golden[key]
+    W = np.array(g["W"], dtype=np.float64)
+    x = np.array(g["x"], dtype=np.float64)
+    q = len(x)
+    ones = [1] * q
+    for t, want in enumerate(g["y_by_type"]):
+        for form in ("rows", "alg1"):
+            got = oracle.proj(x[None, :], [t], W, ones, ones, form=form)
+            assert got.tolist() == [list(map(float, want))], (key, t, form)
+    dense = oracle.proj(x[None, :], [0], W, ones, ones, keep=oracle.support(q, "dense"))
+    assert dense.tolist() == [list(map(float, g["dense"]))]
+
+
+def test_hand_example_square(golden):
+    g = golden["square_q2"]
+    A, B, C = (np.array(g[k], dtype=np.float64) for k in "ABC")
+    one = [1, 1]
+    AB = oracle.square(A, B, one, one, one)
+    BC = oracle.square(B, C, one, one, one)
+    assert AB.tolist() == g["A_star_B"]
+    assert BC.tolist() == g["B_star_C"]
+    assert oracle.square(AB, C, one, one, one).tolist() == g["ABC"]
+    assert oracle.square(A, BC, one, one, one).tolist() == g["ABC"]
+
+
+# ---- P1: the six-product rule, term by term ---------------------------------------------------
+
+def test_q2_six_products_term_by_term():
+    """One-hot block probes: X group k and W block (k', j) non-zero. The output block j of a
+    type-t row is non-zero iff k == k' and k in {t, j}; for q=2 exactly A Wa, A Wu, U Wd,
+    V Wa, D Wv, D Wd survive and U Wv, V Wu never appear (Eq. six-product)."""
+    q, s, r = 2, [2, 3], [3, 2]
+    so, ro = _offsets(s), _offsets(r)
+    rng = np.random.default_rng(1)
+    survivors = set()
+    for t, k, kp, j in itertools.product(range(q), repeat=4):
+        X = np.zeros((1, sum(s)))
+        W = np.zeros((sum(s), sum(r)))
+        X[0, so[k]:so[k + 1]] = rng.integers(1, 4, size=s[k])
+        W[so[kp]:so[kp + 1], ro[j]:ro[j + 1]] = rng.integers(1, 4, size=(s[kp], r[j]))
+        Y = oracle.proj(X, [t], W, s, r)
+        nz = bool(np.any(Y != 0))
+        assert nz == (k == kp and k in (t, j)), (t, k, kp, j)
+        if nz:
+            assert np.array_equal(Y, X @ W)
+            outside = np.ones(sum(r), bool)
+            outside[ro[j]:ro[j + 1]] = False
+            assert not np.any(Y[0, outside])
+            survivors.add((t, k, j))
+    # (type, activation group, output group): A=(0,0) U=(0,1) V=(1,0) D=(1,1)
+    assert survivors == {(0, 0, 0), (0, 0, 1), (0, 1, 1), (1, 0, 0), (1, 1, 0), (1, 1, 1)}
+    assert (0, 1, 0) not in survivors and (1, 0, 1) not in survivors  # U Wv and V Wu
+
+
+@pytest.mark.parametrize("q", [3, 4, 5])
+def test_support_probe_general_q(q):
+    keep = oracle.support(q)
+    for i, j, k in itertools.product(range(q), repeat=3):
+        assert bool(keep[i, j, k]) == (k in (i, j))
+
+
+# ---- P2: counts and MAC formulas -------------------------------------------------------------
+
+def test_gemm_counts(golden):
+    for q, n in golden["gemm_counts"]["qq"].items():
+        q = int(q)
+        keep = oracle.support(q)
+        assert oracle.gemm_count(keep) == n == 2 * q * q - q
+        assert all(int(keep[i].sum()) == 2 * q - 1 for i in range(q))
+        assert oracle.gemm_count(oracle.support(q, "dense")) == q ** 3
+    for q, n in golden["gemm_counts"]["q2pow"].items():
+        assert oracle.gemm_count(oracle.support(int(q), "q2pow")) == n
+
+
+def test_mac_formulas():
+    rng = np.random.default_rng(2)
+    for q in (2, 3, 4, 7):
+        s = rng.integers(1, 9, size=q)
+        r = rng.integers(1, 9, size=q)
+        rows = rng.integers(0, 50, size=q)
+        keep = oracle.support(q)
+        d_diag = int((s * r).sum())
+        N = int(r.sum())
+        want = int(rows.sum()) * d_diag + int(sum(rows[i] * s[i] * (N - r[i]) for i in range(q)))
+        assert oracle.macs(keep, s, r, rows) == want  # Eq. rectangular-batch-cost
+    for q in (2, 4, 8, 16):  # equal groups: rho_q = (2q-1)/q^2
+        s, r, rows = [6] * q, [10] * q, [3] * q
+        M, K, N = 3 * q, 6 * q, 10 * q
+        assert oracle.macs(oracle.support(q), s, r, rows) * q * q == (2 * q - 1) * M * K * N
+    # tensor power: ratio (3/4)^L with equal groups and equally frequent types
+    for L in (1, 2, 3):
+        q = 2 ** L
+        m = oracle.macs(oracle.support(q, "q2pow"), [4] * q, [4] * q, [5] * q)
+        assert m * 4 ** L == 3 ** L * (5 * q) * (4 * q) * (4 * q)
+
+
+# ---- P3: dense minus the removed products (brute force, independent numpy) --------------------
+
+@pytest.mark.parametrize("q", [2, 3, 4])
+def test_dense_minus_removed(q):
+    rng = np.random.default_rng(10 + q)
+    s = rng.integers(1, 4, size=q)
+    r = rng.integers(1, 4, size=q)
+    so, ro = _offsets(s), _offsets(r)
+    M = 8
+    X = _rand_ints(rng, (M, s.sum()))
+    W = _rand_ints(rng, (s.sum(), r.sum()))
+    types = rng.integers(0, q, size=M)
+    want = X @ W
+    for b in range(M):
+        for j in range(q):
+            for k in range(q):
+                if k not in (types[b], j):
+                    want[b, ro[j]:ro[j + 1]] -= X[b, so[k]:so[k + 1]] @ W[so[k]:so[k + 1], ro[j]:ro[j + 1]]
+    for form in ("rows", "alg1"):
+        assert np.array_equal(oracle.proj(X, types, W, s, r, form=form), want)
+
+
+def test_pure_python_scalar_loops():
+    """Scalar-level restatement of Eqs. typed-diag/off with explicit Python loops."""
+    rng = np.random.default_rng(5)
+    q, s, r = 3, [2, 1, 3], [1, 2, 2]
+    so, ro = _offsets(s), _offsets(r)
+    X = _rand_ints(rng, (6, 6))
+    W = _rand_ints(rng, (6, 5))
+    types = [0, 1, 2, 2, 1, 0]
+    want = np.zeros((6, 5))
+    for b, i in enumerate(types):
+        for j in range(q):
+            for n in range(ro[j], ro[j + 1]):
+                acc = 0.0
+                for c in range(so[i], so[i + 1]):        # x_i W_ij
+                    acc += X[b, c] * W[c, n]
+                if j != i:
+                    for c in range(so[j], so[j + 1]):    # + x_j W_jj
+                        acc += X[b, c] * W[c, n]
+                want[b, n] = acc
+    assert np.array_equal(oracle.proj(X, types, W, s, r), want)
+
+
+# ---- P4, P5, P8: associativity, unit, edge ideal on integer block arrays ---------------------
+
+def _np_square_star(A, B, q, b):
+    """Independent numpy statement of (d,n)*(d',n') = (dd', dn' + nd') (Appendix A)."""
+    C = np.zeros_like(A)
+    blk = lambda Z, i, j: Z[i * b:(i + 1) * b, j * b:(j + 1) * b]
+    for i in range(q):
+        for j in range(q):
+            if i == j:
+                blk(C, i, i)[:] = blk(A, i, i) @ blk(B, i, i)
+            else:
+                blk(C, i, j)[:] = blk(A, i, i) @ blk(B, i, j) + blk(A, i, j) @ blk(B, j, j)
+    return C
+
+
+@pytest.mark.parametrize("q,b", [(2, 1), (2, 3), (3, 2), (4, 2), (4, 3)])
+def test_associativity_unit_ideal(q, b):
+    rng = np.random.default_rng(100 * q + b)
+    n = q * b
+    w = [b] * q
+    X, Y, Z = (_rand_ints(rng, (n, n), -2, 2) for _ in range(3))
+    star = lambda P, Q: oracle.square(P, Q, w, w, w)
+    assert np.array_equal(star(X, Y), _np_square_star(X, Y, q, b))
+    assert np.array_equal(star(star(X, Y), Z), star(X, star(Y, Z)))
+    E = np.eye(n)
+    assert np.array_equal(star(E, X), X) and np.array_equal(star(X, E), X)
+    # two arrays with zero diagonal blocks multiply to zero (J^2 = 0)
+    mask = np.kron(1 - np.eye(q), np.ones((b, b)))
+    assert not np.any(star(X * mask, Y * mask))
+    # the rule is not ordinary matrix multiplication
+    assert not np.array_equal(star(X, Y), X @ Y)
+
+
+def test_associativity_rectangular_blocks():
+    rng = np.random.default_rng(77)
+    a, c, d, e = [2, 1, 3], [1, 2, 2], [3, 1, 1], [2, 2, 1]
+    X = _rand_ints(rng, (sum(a), sum(c)))
+    Y = _rand_ints(rng, (sum(c), sum(d)))
+    Z = _rand_ints(rng, (sum(d), sum(e)))
+    left = oracle.square(oracle.square(X, Y, a, c, d), Z, a, d, e)
+    right = oracle.square(X, oracle.square(Y, Z, c, d, e), a, c, e)
+    assert np.array_equal(left, right)
+
+
+# ---- P6: typed rows <-> square display, and the composition law ------------------------------
+
+def test_typed_rows_match_square_display():
+    """Row block i of the square product is the typed projection of rows of type i."""
+    rng = np.random.default_rng(8)
+    q, a, c, d = 3, [2, 3, 1], [2, 1, 2], [1, 3, 2]
+    A = _rand_ints(rng, (sum(a), sum(c)))
+    B = _rand_ints(rng, (sum(c), sum(d)))
+    types = np.repeat(np.arange(q), a)
+    assert np.array_equal(oracle.proj(A, types, B, c, d), oracle.square(A, B, a, c, d))
+
+
+def test_composition_law():
+    """Phi_{W2}(Phi_{W1}(X)) = Phi_{W1 * W2}(X) for row-typed X (Eq. association-intro)."""
+    rng = np.random.default_rng(9)
+    q, s, m, r = 3, [2, 1, 2], [1, 3, 2], [2, 2, 1]
+    M = 11
+    X = _rand_ints(rng, (M, sum(s)))
+    W1 = _rand_ints(rng, (sum(s), sum(m)))
+    W2 = _rand_ints(rng, (sum(m), sum(r)))
+    types = rng.integers(0, q, size=M)
+    lhs = oracle.proj(oracle.proj(X, types, W1, s, m), types, W2, m, r)
+    rhs = oracle.proj(X, types, oracle.square(W1, W2, s, m, r), s, r)
+    assert np.array_equal(lhs, rhs)
+
+
+# ---- P9: reductions to library routines and closed forms -------------------------------------
+
+def test_dense_table_and_q1_are_matmul():
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((17, 12))
+    W = rng.standard_normal((12, 10))
+    types = rng.integers(0, 3, size=17)
+    Y = oracle.proj(X, types, W, [3, 4, 5], [2, 5, 3], keep=oracle.support(3, "dense"))
+    np.testing.assert_allclose(Y, X @ W, rtol=1e-13, atol=1e-13)
+    Y1 = oracle.proj(X, np.zeros(17, int), W, [12], [10])
+    np.testing.assert_allclose(Y1, X @ W, rtol=1e-13, atol=1e-13)
+    bias = rng.standard_normal(10)
+    Yb = oracle.proj(X, np.zeros(17, int), W, [12], [10], bias=bias)
+    np.testing.assert_allclose(Yb, X @ W + bias, rtol=1e-13, atol=1e-13)
+
+
+def test_rows_vs_alg1_float():
+    rng = np.random.default_rng(4)
+    q, s, r = 4, [3, 5, 2, 4], [4, 1, 6, 2]
+    X = rng.standard_normal((23, sum(s)))
+    W = rng.standard_normal((sum(s), sum(r)))
+    types = rng.integers(0, q, size=23)
+    np.testing.assert_allclose(oracle.proj(X, types, W, s, r, form="rows"),
+                               oracle.proj(X, types, W, s, r, form="alg1"), rtol=1e-12, atol=1e-12)
+
+
+def test_gelu_closed_form(golden):
+    for z, want in golden["gelu"]["points"]:
+        assert abs(oracle.gelu(z) - want) < 5e-10
+    import math
+    for z in np.linspace(-6, 6, 41):
+        assert abs(oracle.gelu(z) - 0.5 * z * math.erfc(-z / math.sqrt(2))) < 1e-14
+
+
+def test_ffn_composes_projections():
+    rng = np.random.default_rng(6)
+    q, dw, fw = 2, [3, 2], [4, 5]
+    M = 9
+    X = rng.standard_normal((M, 5))
+    Wu = rng.standard_normal((5, 9))
+    Wd = rng.standard_normal((9, 5))
+    bu, bd = rng.standard_normal(9), rng.standard_normal(5)
+    types = rng.integers(0, q, size=M)
+    Y, H = oracle.ffn(X, types, Wu, Wd, dw, fw, b_up=bu, b_down=bd, return_hidden=True)
+    # independent numpy composition using the dense-minus-removed statement for q=2
+    def star2(Xm, Wm, s, r, bias):
+        so, ro = _offsets(s), _offsets(r)
+        out = Xm @ Wm + bias
+        for b, t in enumerate(types):
+            o = 1 - t  # the removed product for a type-t row is x_o W_{o,t}
+            out[b, ro[t]:ro[t + 1]] -= Xm[b, so[o]:so[o + 1]] @ Wm[so[o]:so[o + 1], ro[t]:ro[t + 1]]
+        return out
+    import math
+    Hn = star2(X, Wu, dw, fw, bu)
+    Hn = np.vectorize(lambda z: 0.5 * z * (1 + math.erf(z / math.sqrt(2))))(Hn)
+    np.testing.assert_allclose(H, Hn, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(Y, star2(Hn, Wd, fw, dw, bd), rtol=1e-12, atol=1e-12)
+
+
+def test_bad_type_rejected():
+    with pytest.raises(oracle.OracleError):
+        oracle.proj(np.zeros((2, 2)), [0, 2], np.zeros((2, 2)), [1, 1], [1, 1])
+    with pytest.raises(oracle.OracleError):
+        oracle.proj(np.zeros((2, 2)), [0, -1], np.zeros((2, 2)), [1, 1], [1, 1], form="alg1")
+
+
+def test_empty_and_missing_types():
+    Y = oracle.proj(np.zeros((0, 4)), np.zeros(0, int), np.ones((4, 6)), [2, 2], [3, 3])
+    assert Y.shape == (0, 6)
+    X = np.ones((3, 4))
+    Y = oracle.proj(X, [1, 1, 1], np.ones((4, 6)), [2, 2], [3, 3])  # no type-0 rows at all
+    assert np.array_equal(Y, np.tile([4, 4, 4, 2, 2, 2], (3, 1)).astype(float))
