@@ -1,0 +1,158 @@
+/*
+ * algproj.h -- C ABI of the row-typed associative-algebra projection  Y = X *_q W  for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper, Section "Transformer Projections", Eqs. typed-diag / typed-off, and
+ * Section "Training and Inference", Eq. recursive-row-action, Algorithm 1):
+ *   X is M x K, W is the ordinary K x N weight bank.  Input features are split into q groups
+ *   of widths s[0..q-1] (sum K), output features into q groups of widths r[0..q-1] (sum N);
+ *   W_{kj} = W[S_k, R_j] is the s[k] x r[j] sub-block.  Row b carries a type t_b in [0,q)
+ *   (0-based; the paper counts types from 1).  Its output group j is
+ *        y_j = bias_j + sum_{k in B(t_b, j)} x_k W_{kj},
+ *   where for the paper's complete-graph law Q_q the support set is B(i,j) = {i,j} as a set:
+ *        y_i = x_i W_ii,      y_j = x_i W_ij + x_j W_jj   (j != i).
+ *   For q = 2 this is the six-product rule (Eq. six-product): type-0 rows give
+ *   [A Wa, A Wu + U Wd], type-1 rows give [V Wa + D Wv, D Wd].
+ *
+ * Conventions
+ *   - All matrices are row-major; leading dimensions are in ELEMENTS.
+ *   - Every pointer named X, W, bias, Y, types, workspace is a DEVICE pointer unless the
+ *     function name ends in _host; the caller owns all of them and the stream.
+ *   - W is the canonical bank: no packing or transposition is required.
+ *   - Y is overwritten, never accumulated into (Algorithm 1 starts from Y <- 0).
+ *   - forward calls enqueue work on `stream` and return; they never synchronise with the
+ *     host and never allocate, so they can be captured into a CUDA graph (the captured graph
+ *     bakes in the addresses and M it was captured with).
+ *   - Two forward calls that share a workspace must be ordered on the GPU (same stream or an
+ *     event between them).
+ *   - Nothing aborts, traps or throws across this boundary; every function returns a status.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef ALGPROJ_H_
+#define ALGPROJ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct alg_proj_s *alg_proj_t;
+typedef struct alg_ffn_s *alg_ffn_t;
+
+typedef enum {
+  ALG_OK = 0,
+  ALG_ERR_INVALID_ARG = 1,         /* NULL pointer, q out of range, non-positive width, ...   */
+  ALG_ERR_UNSUPPORTED_SHAPE = 2,   /* legal problem this build has no kernel for              */
+  ALG_ERR_WORKSPACE_TOO_SMALL = 3, /* workspace_bytes below alg_*_workspace_bytes(M)          */
+  ALG_ERR_CUDA = 4,                /* a CUDA runtime/driver call failed                       */
+  ALG_ERR_BAD_TYPE = 5,            /* device saw types[b] outside [0,q); that row of Y is 0   */
+  ALG_ERR_DEVICE_TIMEOUT = 6       /* a bounded device-side wait expired; output is invalid   */
+} alg_status_t;
+
+typedef enum { ALG_F32 = 0, ALG_BF16 = 1 } alg_dtype_t;
+
+/* Which (type i, output group j, input group k) products are kept.
+ * QQ     : the paper's complete-graph law, k in {i,j}  (2q^2-q block GEMMs, Eq. q-rank).
+ * DENSE  : all k -- the ordinary product X W (q^3 block GEMMs); the same-library control.
+ * CUSTOM : caller-supplied keep[(i*q+j)*q+k] bytes (non-zero = kept), e.g. the tensor-power
+ *          law Q_2^{(x)L} of the appendix "The Tensor-Square Candidate". */
+typedef enum { ALG_TABLE_QQ = 0, ALG_TABLE_DENSE = 1, ALG_TABLE_CUSTOM = 2 } alg_table_t;
+
+/* Activation applied to (acc + bias) before the store. GELU_ERF is z/2 (1 + erf(z/sqrt 2)). */
+typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } alg_act_t;
+
+/* EXPLICIT: the caller passes types[M] with every forward call.
+ * CYCLIC  : type of row b is b mod q (the paper's example schedule tau(p) = p mod q for a
+ *           batch whose sequence length is a multiple of q); `types` may be NULL. */
+typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1 } alg_schedule_t;
+
+/* Kernel families, reported by alg_proj_kernel_path(). */
+typedef enum {
+  ALG_PATH_SIMT = 0,    /* fp32-FMA tiles, any widths                                    */
+  ALG_PATH_TCGEN05 = 1, /* bf16 grouped tcgen05 GEMM, TMA-fed, TMEM accumulators         */
+  ALG_PATH_DECODE = 2   /* small-M weight-streaming kernel                               */
+} alg_path_t;
+
+#define ALG_MAX_Q 32
+
+/* ---- projection handle ---------------------------------------------------------------------
+ * alg_proj_create: build the interaction table for q groups (Eqs. q-product-diag/off, or the
+ * DENSE / CUSTOM variants), pick kernels, allocate a few hundred bytes of device metadata on
+ * the CURRENT device.  in_widths = s[q], out_widths = r[q] (host arrays, copied).  dtype is
+ * the element type of X and W (ALG_F32: true fp32 FMAs; ALG_BF16: bf16 operands, fp32
+ * accumulation).  custom_keep is read only for ALG_TABLE_CUSTOM, else pass NULL; every
+ * (i,j) of a custom table must keep at least one k.  1 <= q <= ALG_MAX_Q.
+ * The tensor-core path needs every s[k] to be a multiple of 64 and every r[j] a multiple of
+ * 128; other bf16/fp32 shapes run on the SIMT path.  */
+alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
+                             const int32_t *out_widths, alg_dtype_t dtype, alg_table_t table,
+                             const uint8_t *custom_keep, alg_schedule_t schedule);
+alg_status_t alg_proj_destroy(alg_proj_t h);
+
+/* Bytes of device scratch a forward call with at most max_M rows needs (row permutation,
+ * bucket offsets, tile list, and -- on the tensor-core path -- the type-bucketed copy of X). */
+alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes);
+
+/* Y[M x N] = act( X[M x K] *_q W[K x N] + bias ).
+ * X: dtype of the handle, ldx >= K.  types: int32[M] device (ignored for CYCLIC).
+ * W: dtype of the handle, ldw >= N.  bias: N values of the handle's dtype, or NULL.
+ * Y: y_dtype (ALG_F32 or ALG_BF16, round-to-nearest-even), ldy >= N.
+ * workspace: >= alg_proj_workspace_bytes(h, M), 256-byte aligned.
+ * bf16 pointers and leading dimensions must keep rows 16-byte aligned (multiples of 8
+ * elements).  M = 0 is a successful no-op; a type with no rows is legal.
+ * M <= 64 with bf16 runs the decode kernel, larger M the prefill kernels. */
+alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const int32_t *types,
+                              int64_t M, const void *W, int64_t ldw, const void *bias,
+                              alg_act_t act, void *Y, int64_t ldy, alg_dtype_t y_dtype,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* Number of kept block GEMMs (2q^2-q for QQ, Eq. q-rank). */
+alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n);
+/* Multiply-accumulates of one forward pass with rows_per_type[i] rows of type i
+ * (Eq. rectangular-batch-cost: M D_diag + sum_i M_i s_i (N - r_i) for QQ). Host array in. */
+alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *macs);
+/* Kernel family a forward call with M rows would use. */
+alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path);
+/* Read and clear the handle's device status word (ALG_OK, ALG_ERR_BAD_TYPE or
+ * ALG_ERR_DEVICE_TIMEOUT).  Synchronises `stream` first. */
+alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *status);
+
+/* ---- FFN handle: Y = act(X *_q W_up + b_up) *_q W_down + b_down  ---------------------------
+ * The two-map MLP (g = 1 in Eq. icml-decode-total) with both projections under the same law
+ * and the same row types (the projection is row-local).  d_widths: q groups of d_model,
+ * f_widths: q groups of d_ff.  X: M x D packed (ld = D), W_up: D x F packed, W_down: F x D
+ * packed, Y: M x D packed.  The hidden state H = act(.) is kept in the workspace in the
+ * handle's dtype (bf16: rounded to nearest even), rows in type-bucketed order. */
+alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths,
+                            const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,
+                            const uint8_t *custom_keep, alg_schedule_t schedule);
+alg_status_t alg_ffn_destroy(alg_ffn_t h);
+alg_status_t alg_ffn_workspace_bytes(alg_ffn_t h, int64_t max_M, size_t *bytes);
+alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, int64_t M,
+                             const void *W_up, const void *b_up, const void *W_down,
+                             const void *b_down, alg_act_t act, void *Y, alg_dtype_t y_dtype,
+                             void *workspace, size_t workspace_bytes, void *stream);
+/* Same computation with X, types and Y in HOST memory (pinned memory makes the copies
+ * asynchronous).  Copies X and types to device staging inside the workspace, runs the
+ * forward pass, copies Y back, all on `stream`; returns without synchronising.  Weights and
+ * biases stay device pointers.  Workspace size: alg_ffn_host_workspace_bytes. */
+alg_status_t alg_ffn_host_workspace_bytes(alg_ffn_t h, int64_t max_M, alg_dtype_t y_dtype,
+                                          size_t *bytes);
+alg_status_t alg_ffn_forward_host(alg_ffn_t h, const void *X_host, const int32_t *types_host,
+                                  int64_t M, const void *W_up, const void *b_up,
+                                  const void *W_down, const void *b_down, alg_act_t act,
+                                  void *Y_host, alg_dtype_t y_dtype, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+alg_status_t alg_ffn_macs(alg_ffn_t h, const int64_t *rows_per_type, int64_t *macs);
+alg_status_t alg_ffn_last_status(alg_ffn_t h, void *stream, alg_status_t *status);
+
+const char *alg_status_string(alg_status_t s);
+/* Number of kernels the library has launched in this process (all handles, all streams). */
+int64_t alg_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALGPROJ_H_ */

@@ -1,0 +1,254 @@
+"""Thin ctypes binding over libalgproj.so -- argument marshalling only.
+
+Function names mirror ``include/algproj.h``.  PyTorch appears here solely as the owner of device
+memory and streams: tensors are turned into raw pointers and every step of the path runs inside
+the CUDA library.  There is no CPU or eager fallback; a missing library is an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libalgproj.so")
+
+ALG_OK = 0
+STATUS = {0: "ALG_OK", 1: "ALG_ERR_INVALID_ARG", 2: "ALG_ERR_UNSUPPORTED_SHAPE", 3: "ALG_ERR_WORKSPACE_TOO_SMALL",
+          4: "ALG_ERR_CUDA", 5: "ALG_ERR_BAD_TYPE", 6: "ALG_ERR_DEVICE_TIMEOUT"}
+ALG_F32, ALG_BF16 = 0, 1
+ALG_TABLE_QQ, ALG_TABLE_DENSE, ALG_TABLE_CUSTOM = 0, 1, 2
+ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
+ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC = 0, 1
+ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
+
+_DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
+_TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM}
+_ACTS = {None: ALG_ACT_NONE, "none": ALG_ACT_NONE, "gelu": ALG_ACT_GELU_ERF, "gelu_erf": ALG_ACT_GELU_ERF,
+         "gelu_tanh": ALG_ACT_GELU_TANH}
+_SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC}
+
+EXPORTS = [
+    "alg_proj_create", "alg_proj_destroy", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
+    "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
+    "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
+    "alg_ffn_macs", "alg_ffn_last_status", "alg_status_string", "alg_launch_count",
+]
+
+_lib = None
+
+
+class AlgError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {STATUS.get(code, code)}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """Load libalgproj.so (built by ``python -m paper_2609_32814_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_32814_b200.build`; "
+                "there is no fallback implementation")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        L.alg_proj_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
+        L.alg_proj_destroy.argtypes = [vp]
+        L.alg_proj_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_proj_forward.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp, ctypes.c_size_t, vp]
+        L.alg_proj_gemm_count.argtypes = [vp, ctypes.POINTER(i64)]
+        L.alg_proj_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.alg_proj_kernel_path.argtypes = [vp, i64, ctypes.POINTER(i32)]
+        L.alg_proj_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.alg_ffn_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
+        L.alg_ffn_destroy.argtypes = [vp]
+        L.alg_ffn_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_ffn_forward.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
+        L.alg_ffn_host_workspace_bytes.argtypes = [vp, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_ffn_forward_host.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
+        L.alg_ffn_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.alg_ffn_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.alg_status_string.argtypes = [i32]
+        L.alg_status_string.restype = ctypes.c_char_p
+        L.alg_launch_count.argtypes = []
+        L.alg_launch_count.restype = i64
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != ALG_OK:
+        raise AlgError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _widths(w):
+    arr = (ctypes.c_int32 * len(w))(*[int(v) for v in w])
+    return arr
+
+
+def launch_count() -> int:
+    return int(lib().alg_launch_count())
+
+
+class _Handle:
+    _destroy = None
+
+    def __init__(self):
+        self._h = ctypes.c_void_p()
+        self._ws = None
+
+    def close(self):
+        if self._h:
+            getattr(lib(), self._destroy)(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _workspace(self, nbytes: int, device) -> torch.Tensor:
+        if self._ws is None or self._ws.numel() < nbytes or self._ws.device != device:
+            self._ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+        return self._ws
+
+
+def _keep_arg(table, custom_keep, q):
+    if _TABLES[table] != ALG_TABLE_CUSTOM:
+        return None, None
+    flat = [int(bool(v)) for v in custom_keep.reshape(-1).tolist()]
+    if len(flat) != q * q * q:
+        raise ValueError("custom_keep must hold q*q*q entries")
+    buf = (ctypes.c_uint8 * len(flat))(*flat)
+    return buf, ctypes.cast(buf, ctypes.c_void_p)
+
+
+class Proj(_Handle):
+    """alg_proj_* : Y = act(X *_q W + bias)."""
+    _destroy = "alg_proj_destroy"
+
+    def __init__(self, in_widths, out_widths, dtype="bf16", table="qq", custom_keep=None, schedule="explicit"):
+        super().__init__()
+        self.q = len(in_widths)
+        self.in_widths, self.out_widths = list(in_widths), list(out_widths)
+        self.K, self.N = sum(self.in_widths), sum(self.out_widths)
+        self.dtype = _DTYPES[dtype]
+        self.schedule = _SCHEDS[schedule]
+        buf, keep = _keep_arg(table, custom_keep, self.q)
+        s, r = _widths(in_widths), _widths(out_widths)
+        _check(lib().alg_proj_create(ctypes.byref(self._h), self.q, ctypes.cast(s, ctypes.c_void_p),
+                                     ctypes.cast(r, ctypes.c_void_p), self.dtype, _TABLES[table], keep,
+                                     self.schedule), "alg_proj_create")
+
+    def workspace_bytes(self, max_M: int) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_proj_workspace_bytes(self._h, max_M, ctypes.byref(out)), "alg_proj_workspace_bytes")
+        return out.value
+
+    def forward(self, X, types, W, bias=None, act=None, out=None, out_dtype=None, workspace=None, stream=None):
+        M = X.shape[0]
+        if out is None:
+            out = torch.empty((M, self.N), dtype=out_dtype or X.dtype, device=X.device)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(M), X.device)
+        _check(lib().alg_proj_forward(self._h, _ptr(X), X.stride(0) if M else self.K, _ptr(types), M, _ptr(W),
+                                      W.stride(0), _ptr(bias), _ACTS[act], _ptr(out),
+                                      out.stride(0) if M else self.N, _DTYPES[out.dtype], _ptr(ws), ws.numel(),
+                                      _stream(stream)), "alg_proj_forward")
+        return out
+
+    def gemm_count(self) -> int:
+        n = ctypes.c_int64()
+        _check(lib().alg_proj_gemm_count(self._h, ctypes.byref(n)), "alg_proj_gemm_count")
+        return n.value
+
+    def macs(self, rows_per_type) -> int:
+        rows = (ctypes.c_int64 * self.q)(*[int(v) for v in rows_per_type])
+        out = ctypes.c_int64()
+        _check(lib().alg_proj_macs(self._h, rows, ctypes.byref(out)), "alg_proj_macs")
+        return out.value
+
+    def kernel_path(self, M: int) -> int:
+        p = ctypes.c_int()
+        _check(lib().alg_proj_kernel_path(self._h, M, ctypes.byref(p)), "alg_proj_kernel_path")
+        return p.value
+
+    def last_status(self, stream=None) -> int:
+        s = ctypes.c_int()
+        _check(lib().alg_proj_last_status(self._h, _stream(stream), ctypes.byref(s)), "alg_proj_last_status")
+        return s.value
+
+
+class FFN(_Handle):
+    """alg_ffn_* : Y = act(X *_q W_up + b_up) *_q W_down + b_down."""
+    _destroy = "alg_ffn_destroy"
+
+    def __init__(self, d_widths, f_widths, dtype="bf16", table="qq", custom_keep=None, schedule="explicit"):
+        super().__init__()
+        self.q = len(d_widths)
+        self.D, self.F = sum(d_widths), sum(f_widths)
+        self.dtype = _DTYPES[dtype]
+        self.schedule = _SCHEDS[schedule]
+        buf, keep = _keep_arg(table, custom_keep, self.q)
+        d, f = _widths(d_widths), _widths(f_widths)
+        _check(lib().alg_ffn_create(ctypes.byref(self._h), self.q, ctypes.cast(d, ctypes.c_void_p),
+                                    ctypes.cast(f, ctypes.c_void_p), self.dtype, _TABLES[table], keep, self.schedule),
+               "alg_ffn_create")
+
+    def workspace_bytes(self, max_M: int) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_ffn_workspace_bytes(self._h, max_M, ctypes.byref(out)), "alg_ffn_workspace_bytes")
+        return out.value
+
+    def host_workspace_bytes(self, max_M: int, out_dtype) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_ffn_host_workspace_bytes(self._h, max_M, _DTYPES[out_dtype], ctypes.byref(out)),
+               "alg_ffn_host_workspace_bytes")
+        return out.value
+
+    def forward(self, X, types, W_up, W_down, b_up=None, b_down=None, act="gelu", out=None, out_dtype=None,
+                workspace=None, stream=None):
+        M = X.shape[0]
+        if not (X.is_contiguous() and W_up.is_contiguous() and W_down.is_contiguous()):
+            raise ValueError("alg_ffn_forward takes packed row-major tensors")
+        if out is None:
+            out = torch.empty((M, self.D), dtype=out_dtype or X.dtype, device=X.device)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(M), X.device)
+        _check(lib().alg_ffn_forward(self._h, _ptr(X), _ptr(types), M, _ptr(W_up), _ptr(b_up), _ptr(W_down),
+                                     _ptr(b_down), _ACTS[act], _ptr(out), _DTYPES[out.dtype], _ptr(ws), ws.numel(),
+                                     _stream(stream)), "alg_ffn_forward")
+        return out
+
+    def forward_host(self, X_host, types_host, W_up, W_down, Y_host, b_up=None, b_down=None, act="gelu",
+                     workspace=None, stream=None):
+        """X_host / types_host / Y_host are CPU tensors (pinned for asynchronous copies)."""
+        M = X_host.shape[0]
+        need = self.host_workspace_bytes(M, Y_host.dtype)
+        ws = workspace if workspace is not None else self._workspace(need, W_up.device)
+        _check(lib().alg_ffn_forward_host(self._h, _ptr(X_host), _ptr(types_host), M, _ptr(W_up), _ptr(b_up),
+                                          _ptr(W_down), _ptr(b_down), _ACTS[act], _ptr(Y_host), _DTYPES[Y_host.dtype],
+                                          _ptr(ws), ws.numel(), _stream(stream)), "alg_ffn_forward_host")
+        return Y_host
+
+    def macs(self, rows_per_type) -> int:
+        rows = (ctypes.c_int64 * self.q)(*[int(v) for v in rows_per_type])
+        out = ctypes.c_int64()
+        _check(lib().alg_ffn_macs(self._h, rows, ctypes.byref(out)), "alg_ffn_macs")
+        return out.value
+
+    def last_status(self, stream=None) -> int:
+        s = ctypes.c_int()
+        _check(lib().alg_ffn_last_status(self._h, _stream(stream), ctypes.byref(s)), "alg_ffn_last_status")
+        return s.value

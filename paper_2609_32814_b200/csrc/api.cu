@@ -1,0 +1,495 @@
+// C-ABI entry points: handle creation (interaction-table expansion, kernel selection), argument
+// validation, workspace layout and the launch sequence of one forward pass.
+#include <algorithm>
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace algproj;
+
+namespace algproj {
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace algproj
+
+struct alg_proj_s {
+  int q = 0;
+  int s[kMaxQ] = {0}, r[kMaxQ] = {0};
+  int K = 0, N = 0;
+  alg_dtype_t dtype = ALG_F32;
+  alg_schedule_t sched = ALG_SCHED_EXPLICIT;
+  DevTable tab;             // host copy
+  DevTable *d_tab = nullptr;
+  int *d_status = nullptr;  // owned unless `shared_status`
+  bool shared_status = false;
+  bool tc_ok = false;
+  int tile_n = 0;           // tensor-core tile width
+  int device = 0;
+  int num_sms = 148;
+};
+
+struct alg_ffn_s {
+  alg_proj_s up, down;
+  int D = 0, F = 0;
+};
+
+namespace {
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+int n_col_tiles(const alg_proj_s &p, int tile_n) {
+  int n = 0;
+  for (int j = 0; j < p.q; ++j) n += ceil_div(p.r[j], tile_n);
+  return n;
+}
+
+// Upper bound on the tiles of one list: sum over pairs of ceil(M_i/tm) * ceil(r_j/tn).
+size_t max_tiles(const alg_proj_s &p, int64_t M, int tile_m, int tile_n) {
+  return (size_t)(M / tile_m + p.q + 1) * (size_t)n_col_tiles(p, tile_n);
+}
+
+bool use_tc(const alg_proj_s &p) { return p.dtype == ALG_BF16 && p.tc_ok; }
+int tile_m_of(const alg_proj_s &p) { return use_tc(p) ? kTcTileM : 64; }
+int tile_n_of(const alg_proj_s &p) { return use_tc(p) ? p.tile_n : 64; }
+int elem_bytes(alg_dtype_t d) { return d == ALG_BF16 ? 2 : 4; }
+
+alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t *out_w, alg_dtype_t dtype,
+                       alg_table_t table, const uint8_t *custom, alg_schedule_t sched, int *shared_status) {
+  if (q < 1 || q > kMaxQ || !in_w || !out_w) return ALG_ERR_INVALID_ARG;
+  if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM) return ALG_ERR_INVALID_ARG;
+  if (table == ALG_TABLE_CUSTOM && !custom) return ALG_ERR_INVALID_ARG;
+  if (sched != ALG_SCHED_EXPLICIT && sched != ALG_SCHED_CYCLIC) return ALG_ERR_INVALID_ARG;
+  p.q = q;
+  p.dtype = dtype;
+  p.sched = sched;
+  std::memset(&p.tab, 0, sizeof(p.tab));
+  p.tab.q = q;
+  int64_t K = 0, N = 0;
+  for (int g = 0; g < q; ++g) {
+    if (in_w[g] <= 0 || out_w[g] <= 0) return ALG_ERR_INVALID_ARG;
+    p.s[g] = in_w[g];
+    p.r[g] = out_w[g];
+    p.tab.so[g] = (int)K;
+    p.tab.ro[g] = (int)N;
+    K += in_w[g];
+    N += out_w[g];
+    if (K > (1 << 30) || N > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  }
+  p.tab.so[q] = (int)K;
+  p.tab.ro[q] = (int)N;
+  p.K = (int)K;
+  p.N = (int)N;
+  // support sets B(i,j): Q_q keeps k in {i,j} (Eqs. typed-diag / typed-off)
+  for (int i = 0; i < q; ++i)
+    for (int j = 0; j < q; ++j) {
+      uint32_t m = 0;
+      for (int k = 0; k < q; ++k) {
+        bool keep = table == ALG_TABLE_DENSE  ? true
+                    : table == ALG_TABLE_QQ   ? (k == i || k == j)
+                                              : custom[((size_t)i * q + j) * q + k] != 0;
+        if (keep) m |= 1u << k;
+      }
+      if (m == 0) return ALG_ERR_INVALID_ARG;  // an output block nobody writes
+      p.tab.keep[i * q + j] = m;
+    }
+  // pairs sorted by total K length, longest first (stable)
+  std::vector<std::pair<int, int>> order;  // (-K length, pair)
+  for (int pr = 0; pr < q * q; ++pr) {
+    int len = 0;
+    for (int k = 0; k < q; ++k)
+      if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
+    order.push_back({-len, pr});
+  }
+  std::stable_sort(order.begin(), order.end(),
+                   [](const std::pair<int, int> &x, const std::pair<int, int> &y) { return x.first < y.first; });
+  p.tab.n_pairs = q * q;
+  for (int e = 0; e < q * q; ++e) p.tab.pair_order[e] = order[e].second;
+
+  // tensor-core eligibility: bf16, K groups in 64-steps, N groups in 128-steps
+  p.tc_ok = dtype == ALG_BF16;
+  bool all256 = true;
+  for (int g = 0; g < q; ++g) {
+    if (p.s[g] % kTcBlockK) p.tc_ok = false;
+    if (p.r[g] % 128) p.tc_ok = false;
+    if (p.r[g] % 256) all256 = false;
+  }
+  p.tile_n = all256 ? 256 : 128;
+
+  if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, p.device) != cudaSuccess) return ALG_ERR_CUDA;
+  p.num_sms = prop.multiProcessorCount;
+  if (prop.major != 10) return ALG_ERR_UNSUPPORTED_SHAPE;  // sm_100a code only
+  if (cudaMalloc(&p.d_tab, sizeof(DevTable)) != cudaSuccess) return ALG_ERR_CUDA;
+  if (cudaMemcpy(p.d_tab, &p.tab, sizeof(DevTable), cudaMemcpyHostToDevice) != cudaSuccess) return ALG_ERR_CUDA;
+  if (shared_status) {
+    p.d_status = shared_status;
+    p.shared_status = true;
+  } else {
+    if (cudaMalloc(&p.d_status, sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
+    if (cudaMemset(p.d_status, 0, sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
+  }
+  if (use_tc(p) && tc_init() != cudaSuccess) return ALG_ERR_CUDA;
+  return ALG_OK;
+}
+
+void free_proj(alg_proj_s &p) {
+  if (p.d_tab) cudaFree(p.d_tab);
+  if (p.d_status && !p.shared_status) cudaFree(p.d_status);
+  p.d_tab = nullptr;
+  p.d_status = nullptr;
+}
+
+struct WsLayout {
+  size_t hdr = 0, chunks = 0, perm = 0, tiles0 = 0, tiles1 = 0, xb = 0, h = 0, total = 0;
+};
+
+// `second`: the down projection of an FFN (nullptr for a single projection).
+WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
+  WsLayout L;
+  size_t off = 0;
+  L.hdr = off;
+  off = align_up(off + sizeof(WsHeader));
+  L.chunks = off;
+  off = align_up(off + (size_t)ceil_div((int)(M > 0 ? M : 1), kBucketChunk) * (first.q + 1) * sizeof(int));
+  L.perm = off;
+  off = align_up(off + (size_t)M * sizeof(int));
+  L.tiles0 = off;
+  off = align_up(off + max_tiles(first, M, tile_m_of(first), tile_n_of(first)) * sizeof(TileRec));
+  if (second) {
+    L.tiles1 = off;
+    off = align_up(off + max_tiles(*second, M, tile_m_of(*second), tile_n_of(*second)) * sizeof(TileRec));
+  }
+  if (use_tc(first)) {
+    L.xb = off;
+    off = align_up(off + (size_t)M * first.K * 2, 1024);
+  }
+  if (second) {
+    L.h = off;
+    off = align_up(off + (size_t)M * first.N * elem_bytes(first.dtype), 1024);
+  }
+  L.total = off;
+  return L;
+}
+
+alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG_ERR_CUDA; }
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+ListSpec make_list(const alg_proj_s &p, char *ws, size_t off) {
+  ListSpec ls;
+  ls.tab = p.d_tab;
+  ls.tiles = (TileRec *)(ws + off);
+  ls.tile_m = tile_m_of(p);
+  ls.tile_n = tile_n_of(p);
+  return ls;
+}
+
+alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list, const void *X, int64_t ldx,
+                      bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
+                      int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st) {
+  ProjArgs a;
+  a.tab = p.d_tab;
+  a.hdr = (const WsHeader *)(ws + L.hdr);
+  a.tiles = (const TileRec *)(ws + (list == 0 ? L.tiles0 : L.tiles1));
+  a.list = list;
+  a.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
+  a.W = W;
+  a.ldw = ldw;
+  a.bias = bias;
+  a.act = (int)act;
+  a.Y = Y;
+  a.ldy = ldy;
+  a.y_bf16 = y_dtype == ALG_BF16;
+  a.M = (int)M;
+  a.K = p.K;
+  a.N = p.N;
+  a.status = p.d_status;
+  if (use_tc(p)) {
+    if (x_bucketed) {
+      a.X = X;
+      a.ldx = ldx;
+    } else {
+      cudaError_t e = launch_gather_rows(X, ldx, (const int *)(ws + L.perm), (int)M, p.K, 2, ws + L.xb, st);
+      if (e != cudaSuccess) return ALG_ERR_CUDA;
+      a.X = ws + L.xb;
+      a.ldx = p.K;
+    }
+    a.in_perm = nullptr;
+    return cuda_status(launch_proj_tc(a, p.tile_n, p.num_sms, st));
+  }
+  a.X = X;
+  a.ldx = ldx;
+  a.in_perm = x_bucketed ? nullptr : (const int *)(ws + L.perm);
+  return cuda_status(launch_proj_simt(a, p.dtype == ALG_BF16, st));
+}
+
+}  // namespace
+
+extern "C" {
+
+alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths, const int32_t *out_widths,
+                             alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
+                             alg_schedule_t schedule) {
+  if (!out) return ALG_ERR_INVALID_ARG;
+  *out = nullptr;
+  alg_proj_s *p = new (std::nothrow) alg_proj_s();
+  if (!p) return ALG_ERR_INVALID_ARG;
+  alg_status_t s = init_proj(*p, q, in_widths, out_widths, dtype, table, custom_keep, schedule, nullptr);
+  if (s != ALG_OK) {
+    free_proj(*p);
+    delete p;
+    return s;
+  }
+  *out = p;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_destroy(alg_proj_t h) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  free_proj(*h);
+  delete h;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes) {
+  if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  *bytes = layout(*h, nullptr, max_M).total;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const int32_t *types, int64_t M,
+                              const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y, int64_t ldy,
+                              alg_dtype_t y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+  if (!h || M < 0 || M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (M == 0) return ALG_OK;
+  if (!X || !W || !Y || !workspace) return ALG_ERR_INVALID_ARG;
+  if (h->sched == ALG_SCHED_EXPLICIT && !types) return ALG_ERR_INVALID_ARG;
+  if (ldx < h->K || ldw < h->N || ldy < h->N) return ALG_ERR_INVALID_ARG;
+  if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  if ((int)act < 0 || (int)act > 2) return ALG_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255u) != 0) return ALG_ERR_INVALID_ARG;
+  if (h->dtype == ALG_BF16) {
+    if (!aligned16(X) || !aligned16(W) || ldx % 8 || ldw % 8) return ALG_ERR_INVALID_ARG;
+  }
+  if (!aligned16(Y) || (ldy * elem_bytes(y_dtype)) % 16) return ALG_ERR_INVALID_ARG;
+  const WsLayout L = layout(*h, nullptr, M);
+  if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)workspace;
+
+  BucketArgs b;
+  b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
+  b.M = (int)M;
+  b.q = h->q;
+  b.hdr = (WsHeader *)(ws + L.hdr);
+  b.chunk_counts = (int *)(ws + L.chunks);
+  b.perm = (int *)(ws + L.perm);
+  b.status = h->d_status;
+  b.lists[0] = make_list(*h, ws, L.tiles0);
+  b.lists[1] = b.lists[0];
+  b.n_lists = 1;
+  b.Y = Y;
+  b.ldy = ldy;
+  b.N = h->N;
+  b.y_elem_bytes = elem_bytes(y_dtype);
+  if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  return run_proj(*h, L, ws, 0, X, ldx, false, W, ldw, bias, act, Y, ldy, y_dtype, false, M, st);
+}
+
+alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
+  if (!h || !n) return ALG_ERR_INVALID_ARG;
+  int64_t c = 0;
+  for (int pr = 0; pr < h->q * h->q; ++pr) c += __builtin_popcount(h->tab.keep[pr]);
+  *n = c;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *macs) {
+  if (!h || !rows_per_type || !macs) return ALG_ERR_INVALID_ARG;
+  int64_t total = 0;
+  for (int i = 0; i < h->q; ++i) {
+    if (rows_per_type[i] < 0) return ALG_ERR_INVALID_ARG;
+    for (int j = 0; j < h->q; ++j)
+      for (int k = 0; k < h->q; ++k)
+        if ((h->tab.keep[i * h->q + j] >> k) & 1u) total += rows_per_type[i] * (int64_t)h->s[k] * h->r[j];
+  }
+  *macs = total;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path) {
+  if (!h || !path || M < 0) return ALG_ERR_INVALID_ARG;
+  *path = use_tc(*h) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
+  return ALG_OK;
+}
+
+static alg_status_t read_status(int *d_status, void *stream, alg_status_t *status) {
+  if (!status) return ALG_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int v = 0;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (cudaMemcpy(&v, d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ALG_ERR_CUDA;
+  if (v != 0 && cudaMemset(d_status, 0, sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
+  *status = (alg_status_t)v;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *status) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  return read_status(h->d_status, stream, status);
+}
+
+alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,
+                            alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
+                            alg_schedule_t schedule) {
+  if (!out) return ALG_ERR_INVALID_ARG;
+  *out = nullptr;
+  alg_ffn_s *f = new (std::nothrow) alg_ffn_s();
+  if (!f) return ALG_ERR_INVALID_ARG;
+  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr);
+  if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status);
+  if (s != ALG_OK) {
+    free_proj(f->down);
+    free_proj(f->up);
+    delete f;
+    return s;
+  }
+  f->D = f->up.K;
+  f->F = f->up.N;
+  *out = f;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_destroy(alg_ffn_t h) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  free_proj(h->down);
+  free_proj(h->up);
+  delete h;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_workspace_bytes(alg_ffn_t h, int64_t max_M, size_t *bytes) {
+  if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  *bytes = layout(h->up, &h->down, max_M).total;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, int64_t M, const void *W_up,
+                             const void *b_up, const void *W_down, const void *b_down, alg_act_t act, void *Y,
+                             alg_dtype_t y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+  if (!h || M < 0 || M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (M == 0) return ALG_OK;
+  if (!X || !W_up || !W_down || !Y || !workspace) return ALG_ERR_INVALID_ARG;
+  if (h->up.sched == ALG_SCHED_EXPLICIT && !types) return ALG_ERR_INVALID_ARG;
+  if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  if ((int)act < 0 || (int)act > 2) return ALG_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255u) != 0) return ALG_ERR_INVALID_ARG;
+  const int eb = elem_bytes(h->up.dtype);
+  if (!aligned16(X) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(Y)) return ALG_ERR_INVALID_ARG;
+  if ((h->D * eb) % 16 || (h->F * eb) % 16 || (h->D * elem_bytes(y_dtype)) % 16) return ALG_ERR_INVALID_ARG;
+  const WsLayout L = layout(h->up, &h->down, M);
+  if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)workspace;
+
+  BucketArgs b;
+  b.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;
+  b.M = (int)M;
+  b.q = h->up.q;
+  b.hdr = (WsHeader *)(ws + L.hdr);
+  b.chunk_counts = (int *)(ws + L.chunks);
+  b.perm = (int *)(ws + L.perm);
+  b.status = h->up.d_status;
+  b.lists[0] = make_list(h->up, ws, L.tiles0);
+  b.lists[1] = make_list(h->down, ws, L.tiles1);
+  b.n_lists = 2;
+  b.Y = Y;
+  b.ldy = h->D;
+  b.N = h->D;
+  b.y_elem_bytes = elem_bytes(y_dtype);
+  if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  void *H = ws + L.h;
+  alg_status_t s = run_proj(h->up, L, ws, 0, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st);
+  if (s != ALG_OK) return s;
+  return run_proj(h->down, L, ws, 1, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st);
+}
+
+alg_status_t alg_ffn_host_workspace_bytes(alg_ffn_t h, int64_t max_M, alg_dtype_t y_dtype, size_t *bytes) {
+  if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  size_t dev = layout(h->up, &h->down, max_M).total;
+  size_t x = align_up((size_t)max_M * h->D * elem_bytes(h->up.dtype));
+  size_t t = align_up((size_t)max_M * sizeof(int32_t));
+  size_t y = align_up((size_t)max_M * h->D * elem_bytes(y_dtype));
+  *bytes = align_up(dev) + x + t + y;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_forward_host(alg_ffn_t h, const void *X_host, const int32_t *types_host, int64_t M,
+                                  const void *W_up, const void *b_up, const void *W_down, const void *b_down,
+                                  alg_act_t act, void *Y_host, alg_dtype_t y_dtype, void *workspace,
+                                  size_t workspace_bytes, void *stream) {
+  if (!h || M < 0 || M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (M == 0) return ALG_OK;
+  if (!X_host || !Y_host || !workspace) return ALG_ERR_INVALID_ARG;
+  if (h->up.sched == ALG_SCHED_EXPLICIT && !types_host) return ALG_ERR_INVALID_ARG;
+  if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  size_t need = 0;
+  alg_status_t s = alg_ffn_host_workspace_bytes(h, M, y_dtype, &need);
+  if (s != ALG_OK) return s;
+  if (workspace_bytes < need) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)workspace;
+  const size_t dev = align_up(layout(h->up, &h->down, M).total);
+  const size_t xb = (size_t)M * h->D * elem_bytes(h->up.dtype);
+  const size_t tb = (size_t)M * sizeof(int32_t);
+  const size_t yb = (size_t)M * h->D * elem_bytes(y_dtype);
+  char *dX = ws + dev;
+  char *dT = dX + align_up(xb);
+  char *dY = dT + align_up(tb);
+  if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (types_host && cudaMemcpyAsync(dT, types_host, tb, cudaMemcpyHostToDevice, st) != cudaSuccess) return ALG_ERR_CUDA;
+  s = alg_ffn_forward(h, dX, types_host ? (const int32_t *)dT : nullptr, M, W_up, b_up, W_down, b_down, act, dY,
+                      y_dtype, ws, dev, st);
+  if (s != ALG_OK) return s;
+  if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ALG_ERR_CUDA;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_macs(alg_ffn_t h, const int64_t *rows_per_type, int64_t *macs) {
+  if (!h || !macs) return ALG_ERR_INVALID_ARG;
+  int64_t a = 0, b = 0;
+  alg_status_t s = alg_proj_macs(&h->up, rows_per_type, &a);
+  if (s != ALG_OK) return s;
+  s = alg_proj_macs(&h->down, rows_per_type, &b);
+  if (s != ALG_OK) return s;
+  *macs = a + b;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_last_status(alg_ffn_t h, void *stream, alg_status_t *status) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  return read_status(h->up.d_status, stream, status);
+}
+
+const char *alg_status_string(alg_status_t s) {
+  switch (s) {
+    case ALG_OK: return "ok";
+    case ALG_ERR_INVALID_ARG: return "invalid argument";
+    case ALG_ERR_UNSUPPORTED_SHAPE: return "unsupported shape or device";
+    case ALG_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case ALG_ERR_CUDA: return "CUDA call failed";
+    case ALG_ERR_BAD_TYPE: return "row type outside [0, q)";
+    case ALG_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
+  }
+  return "unknown status";
+}
+
+int64_t alg_launch_count(void) { return algproj::g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,216 @@
+// Row-type bucketing (Algorithm 1, line "I_i <- {b : tau(p_b) = i}") as a stable permutation,
+// plus the device-side tile list of the grouped GEMM.  No host synchronisation anywhere: the
+// row counts per type never leave the device.
+//
+//   kernel 1 (count):   per-chunk histograms; the last CTA to finish scans them into per-chunk
+//                       bases, writes the bucket offsets and emits the tile lists.
+//   kernel 2 (scatter): perm[offset[t] + base[chunk][t] + rank_in_chunk] = row  (stable).
+//   kernel 3 (gather):  Xb[d,:] = X[perm[d],:]  -- every type becomes a contiguous M-slab.
+#include "common.cuh"
+
+namespace algproj {
+
+namespace {
+
+__device__ __forceinline__ int row_type(const BucketArgs &a, int row) {
+  int t = a.types ? a.types[row] : (row % a.q);
+  return (t < 0 || t >= a.q) ? a.q : t;  // pseudo-type q collects out-of-range rows
+}
+
+// Exclusive scan of v over the 256 threads of the CTA; returns the prefix, *total gets the sum.
+__device__ int block_exclusive_scan_256(int v, int *smem_warp /*[8]*/, int *total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += n;
+  }
+  if (lane == 31) smem_warp[warp] = incl;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    int c = smem_warp[w];
+    if (w < warp) base += c;
+    tot += c;
+  }
+  __syncthreads();
+  *total = tot;
+  return base + incl - v;
+}
+
+__device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list, WsHeader *hdr_w,
+                               int *s_prefix /*[kMaxPairs+1]*/, int *s_warp /*[8]*/) {
+  const DevTable *tab = ls.tab;
+  const int q = tab->q, np = tab->n_pairs;
+  // tiles per pair, in the host-chosen order (longest K first)
+  constexpr int kPer = kMaxPairs / 256;  // 4 pairs per thread
+  int local[kPer];
+  int sum = 0;
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    int p = threadIdx.x * kPer + e;
+    int cnt = 0;
+    if (p < np) {
+      int pair = tab->pair_order[p];
+      int i = pair / q, j = pair % q;
+      int rows = hdr->offsets[i + 1] - hdr->offsets[i];
+      int width = tab->ro[j + 1] - tab->ro[j];
+      cnt = ceil_div(rows, ls.tile_m) * ceil_div(width, ls.tile_n);
+    }
+    local[e] = cnt;
+    sum += cnt;
+  }
+  int total;
+  int base = block_exclusive_scan_256(sum, s_warp, &total);
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    int p = threadIdx.x * kPer + e;
+    if (p < kMaxPairs) s_prefix[p] = base;
+    base += local[e];
+  }
+  if (threadIdx.x == 255) s_prefix[kMaxPairs] = total;
+  __syncthreads();
+  for (int e = threadIdx.x; e < total; e += 256) {
+    // last p with s_prefix[p] <= e and a non-empty pair
+    int lo = 0, hi = np;  // invariant: s_prefix[lo] <= e < s_prefix[hi] (s_prefix[np..] == total)
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (s_prefix[mid] <= e) lo = mid; else hi = mid;
+    }
+    int pair = tab->pair_order[lo];
+    int i = pair / q, j = pair % q;
+    int width = tab->ro[j + 1] - tab->ro[j];
+    int n_tiles = ceil_div(width, ls.tile_n);
+    int loc = e - s_prefix[lo];
+    int mt = loc / n_tiles, nt = loc % n_tiles;  // n fastest: neighbours share the A rows
+    int rows = hdr->offsets[i + 1] - hdr->offsets[i];
+    TileRec rec;
+    rec.row0 = hdr->offsets[i] + mt * ls.tile_m;
+    rec.rows = min(ls.tile_m, rows - mt * ls.tile_m);
+    rec.pair = pair;
+    rec.n0 = tab->ro[j] + nt * ls.tile_n;
+    ls.tiles[e] = rec;
+  }
+  if (threadIdx.x == 0) {
+    hdr_w->n_tiles[list] = total;
+    hdr_w->counter[list] = 0;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
+  __shared__ int s_cnt[kMaxQ + 1];
+  __shared__ int s_last;
+  __shared__ int s_prefix[kMaxPairs + 1];
+  __shared__ int s_warp[8];
+  const int tid = threadIdx.x;
+  const int nt = a.q + 1;
+  if (tid < nt) s_cnt[tid] = 0;
+  __syncthreads();
+  const int row = blockIdx.x * kBucketChunk + tid;
+  if (row < a.M) {
+    int t = row_type(a, row);
+    if (t == a.q) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
+    atomicAdd(&s_cnt[t], 1);
+  }
+  __syncthreads();
+  if (tid < nt) a.chunk_counts[blockIdx.x * nt + tid] = s_cnt[tid];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&a.hdr->ticket, 1) == (int)gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // ---- last CTA: per-type exclusive scan over chunks (warp w takes types w, w+8, ...) -------
+  const int lane = tid & 31, warp = tid >> 5;
+  const int n_chunks = gridDim.x;
+  for (int t = warp; t < nt; t += 8) {
+    int carry = 0;
+    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+      int c = c0 + lane;
+      int v = (c < n_chunks) ? __ldcg(&a.chunk_counts[c * nt + t]) : 0;
+      int incl = v;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += n;
+      }
+      if (c < n_chunks) a.chunk_counts[c * nt + t] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_cnt[t] = carry;  // total rows of (pseudo-)type t
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int t = 0; t < nt; ++t) {
+      a.hdr->offsets[t] = run;
+      run += s_cnt[t];
+    }
+    a.hdr->offsets[nt] = run;  // == M
+    a.hdr->ticket = 0;         // ready for the next forward call
+  }
+  __syncthreads();
+  for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, s_prefix, s_warp);
+}
+
+__global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a) {
+  __shared__ int s_wcnt[8][kMaxQ + 1];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nt = a.q + 1;
+  for (int e = tid; e < 8 * (kMaxQ + 1); e += 256) (&s_wcnt[0][0])[e] = 0;
+  __syncthreads();
+  const int row = blockIdx.x * kBucketChunk + tid;
+  const bool live = row < a.M;
+  const int t = live ? row_type(a, row) : -1 - lane;  // dead lanes never match each other
+  const unsigned peers = __match_any_sync(0xffffffffu, t);
+  const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+  if (live && rank_in_warp == 0) s_wcnt[warp][t] = __popc(peers);
+  __syncthreads();
+  if (!live) return;
+  int before = 0;
+  for (int w = 0; w < warp; ++w) before += s_wcnt[w][t];
+  const int dest = a.hdr->offsets[t] + a.chunk_counts[blockIdx.x * nt + t] + before + rank_in_warp;
+  a.perm[dest] = row;
+  if (t == a.q && a.Y) {  // out-of-range type: the row's output is defined to be zero
+    char *y = (char *)a.Y + (size_t)row * a.ldy * a.y_elem_bytes;
+    for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ X, int64_t ldx_v,
+                                                          const int *__restrict__ perm, int M, int vecs,
+                                                          uint4 *__restrict__ Xb) {
+  const int64_t total = (int64_t)M * vecs;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+       e += (int64_t)gridDim.x * blockDim.x) {
+    int d = (int)(e / vecs), v = (int)(e % vecs);
+    Xb[e] = __ldg(&X[(int64_t)perm[d] * ldx_v + v]);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
+  const int n_chunks = ceil_div(a.M, kBucketChunk);
+  bucket_count_kernel<<<n_chunks, 256, 0, st>>>(a);
+  bucket_scatter_kernel<<<n_chunks, 256, 0, st>>>(a);
+  count_launch(2);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int M, int K, int elem_bytes,
+                               void *Xb, cudaStream_t st) {
+  const int vecs = K * elem_bytes / 16;
+  const int64_t total = (int64_t)M * vecs;
+  int grid = (int)((total + 255) / 256);
+  if (grid > 148 * 16) grid = 148 * 16;
+  gather_rows_kernel<<<grid, 256, 0, st>>>((const uint4 *)X, ldx * elem_bytes / 16, perm, M, vecs, (uint4 *)Xb);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+}  // namespace algproj

@@ -1,0 +1,132 @@
+// Shared declarations of the algproj CUDA library (host metadata, device tables, launchers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "algproj.h"
+
+namespace algproj {
+
+constexpr int kMaxQ = ALG_MAX_Q;
+constexpr int kMaxPairs = kMaxQ * kMaxQ;
+constexpr int kBucketChunk = 256;  // rows per CTA of the bucketing kernels
+
+// Interaction table of one projection as the kernels see it (device memory, owned by a handle).
+struct DevTable {
+  int q;
+  int n_pairs;                 // (type i, output group j) pairs with a non-empty support set
+  int so[kMaxQ + 1];           // prefix sums of the input group widths  (S_k = [so[k], so[k+1]))
+  int ro[kMaxQ + 1];           // prefix sums of the output group widths (R_j = [ro[j], ro[j+1]))
+  uint32_t keep[kMaxPairs];    // keep[i*q+j] bit k set  <=>  k in B(i,j)
+  int pair_order[kMaxPairs];   // pairs (i*q+j) sorted by total K length, longest first
+};
+
+// One output tile of the grouped GEMM: rows [row0, row0+rows) of the type-bucketed row order
+// (all of one type), columns [n0, n0+cols) inside one output group.
+struct TileRec {
+  int row0;
+  int rows;
+  int pair;   // i * q + j
+  int n0;     // absolute first column
+};
+
+// Fixed-size header at the start of every workspace.
+struct WsHeader {
+  int offsets[kMaxQ + 2];  // offsets[t] = first bucketed row of type t; [q] = first bad row; [q+1] = M
+  int ticket;              // last-block-done counter of the counting kernel
+  int n_tiles[2];          // tiles in list 0 / 1
+  int counter[2];          // dynamic tile counters of list 0 / 1
+  int pad[25];
+};
+static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
+
+struct ListSpec {
+  const DevTable *tab;
+  TileRec *tiles;
+  int tile_m;
+  int tile_n;
+};
+
+struct BucketArgs {
+  const int32_t *types;  // nullptr => cyclic (row mod q)
+  int M;
+  int q;
+  WsHeader *hdr;
+  int *chunk_counts;     // [n_chunks][q+1]
+  int *perm;             // [M] bucketed position -> original row
+  int *status;           // device status word of the handle
+  ListSpec lists[2];
+  int n_lists;
+  // rows with an out-of-range type get their output row zero-filled here
+  void *Y;
+  int64_t ldy;
+  int N;
+  int y_elem_bytes;
+};
+
+cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st);
+// Xb[d, 0:K] = X[perm[d], 0:K] (16-byte vectors; K*elem_bytes % 16 == 0)
+cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int M, int K,
+                               int elem_bytes, void *Xb, cudaStream_t st);
+
+struct ProjArgs {
+  const DevTable *tab;
+  const WsHeader *hdr;
+  const TileRec *tiles;
+  int list;               // which n_tiles / counter of the header
+  const void *X;          // SIMT: original rows (gathered through perm); tcgen05: bucketed copy
+  int64_t ldx;
+  const int *perm;        // output row scatter: bucketed -> original; nullptr = keep bucketed
+  const int *in_perm;     // SIMT only: input row gather (nullptr = X already bucketed)
+  const void *W;
+  int64_t ldw;
+  const void *bias;
+  int act;
+  void *Y;
+  int64_t ldy;
+  int y_bf16;
+  int M;
+  int K;
+  int N;
+  int *status;
+};
+
+cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
+
+// tcgen05 path. tile_n in {128, 256}.
+constexpr int kTcTileM = 128;
+constexpr int kTcBlockK = 64;
+cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st);
+cudaError_t tc_init();  // resolves the driver entry point for tensor-map encoding
+
+// decode path (M <= 64)
+constexpr int kDecodeMaxM = 64;
+struct DecodeArgs {
+  const DevTable *tab;
+  const void *X;
+  int64_t ldx;
+  const int32_t *types;   // nullptr => cyclic
+  int M;
+  const void *W;
+  int64_t ldw;
+  const void *bias;
+  int act;
+  void *Y;
+  int64_t ldy;
+  int y_bf16;
+  int K;
+  int N;
+  float *partials;        // split-K scratch
+  int *tickets;           // per-strip arrival counters (zero on entry, left zero on exit)
+  int *status;
+};
+size_t decode_workspace_bytes(int K, int N);
+cudaError_t launch_decode(const DecodeArgs &a, int num_sms, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace algproj

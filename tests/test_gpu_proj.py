@@ -1,0 +1,188 @@
+"""GPU parity of alg_proj_forward against the CPU oracle (single projections)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_32814_b200 import binding, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_proj(wl, *, table="qq", custom=None, bias=None, act=None, out_dtype=None, which="up", schedule="explicit",
+              expect_path=None):
+    s, r = (wl.d_widths, wl.f_widths) if which == "up" else (wl.f_widths, wl.d_widths)
+    W = wl.W_up if which == "up" else wl.W_down
+    proj = binding.Proj(s, r, dtype=wl.dtype, table=table, custom_keep=custom, schedule=schedule)
+    if expect_path is not None:
+        assert proj.kernel_path(wl.M) == expect_path
+    X = H.to_dev(wl.X, wl.dtype)
+    Wd = H.to_dev(W, wl.dtype)
+    bd = None if bias is None else H.to_dev(bias, wl.dtype)
+    Y = proj.forward(X, H.dev_types(wl.types), Wd, bias=bd, act=act, out_dtype=out_dtype)
+    assert proj.last_status() == 0
+    return Y, proj
+
+
+# ---- config 1: fp32, true fp32 FMAs ---------------------------------------------------------
+
+def test_cfg1_integer_bit_exact():
+    wl = synth.config1(integer=True)
+    Y, proj = _run_proj(wl, expect_path=binding.ALG_PATH_SIMT)
+    assert proj.gemm_count() == 6
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    got = Y.cpu().numpy()
+    assert got.dtype == np.float32
+    assert np.array_equal(got.view(np.uint32), ref.astype(np.float32).view(np.uint32))
+
+
+def test_cfg1_normal_fp32():
+    wl = synth.config1()
+    Y, _ = _run_proj(wl)
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    got = H.to_np(Y)
+    assert H.rel_fro(got, ref) <= H.F32_REL_FRO
+    assert H.max_abs(got, ref) <= H.F32_MAX_ABS
+
+
+def test_cfg1_dense_table_is_matmul():
+    wl = synth.config1(integer=True)
+    Y, proj = _run_proj(wl, table="dense")
+    assert proj.gemm_count() == 8
+    assert np.array_equal(H.to_np(Y), wl.X.astype(np.float64) @ wl.W_up.astype(np.float64))
+
+
+# ---- SIMT path on awkward shapes (any q, unequal widths, ragged everything) ------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_simt_ragged_unequal_widths(dtype):
+    q, s, r, M = 3, [24, 40, 8], [72, 8, 136], 333
+    rng_types = synth.uniform_types(7, M, q)
+    wl = synth.make_workload("ragged", config=9, variant=1, dtype=dtype, q=q, M=M, D=sum(s), F=sum(r),
+                             types=rng_types, integer=True, with_down=False, d_widths=s, f_widths=r)
+    bias = synth.small_ints(99, (sum(r),))
+    Y, proj = _run_proj(wl, bias=bias, out_dtype=torch.float32, expect_path=binding.ALG_PATH_SIMT)
+    assert proj.gemm_count() == 15
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, s, r, bias=bias)
+    assert np.array_equal(H.to_np(Y), ref)
+
+
+# ---- tensor-core path: integer data is exact in bf16 x bf16 -> fp32 -------------------------
+
+def _tc_workload(q, M, s_w, r_w, types=None, integer=True, seed=1):
+    if types is None:
+        types = synth.uniform_types(1000 + seed, M, q)
+    return synth.make_workload("tc", config=8, variant=seed, dtype="bf16", q=q, M=M, D=s_w * q, F=r_w * q,
+                               types=types, integer=integer, with_down=False)
+
+
+@pytest.mark.parametrize("q,M,s_w,r_w", [
+    (2, 128, 64, 128),     # one tile per pair, one or two k-blocks
+    (2, 300, 128, 256),    # ragged last m-tile, 256-wide tiles
+    (2, 1000, 384, 384),   # 128-wide tiles (384 = 3 x 128), six k-blocks per group
+    (4, 777, 128, 512),    # config-3 group shapes, several types
+    (3, 515, 192, 128),    # non-power-of-two q
+    (1, 200, 256, 256),    # q = 1 degenerates to an ordinary GEMM
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_tc_integer_bit_exact(q, M, s_w, r_w, out_dtype):
+    wl = _tc_workload(q, M, s_w, r_w, seed=q * 10 + M % 7)
+    Y, proj = _run_proj(wl, out_dtype=out_dtype, expect_path=binding.ALG_PATH_TCGEN05)
+    assert proj.gemm_count() == 2 * q * q - q
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    got = H.to_np(Y)
+    bad = np.argwhere(got != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+
+
+def test_tc_missing_type_and_single_row():
+    wl = _tc_workload(2, 1, 128, 128, types=np.array([1], dtype=np.int32))
+    Y, _ = _run_proj(wl, out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+    wl = _tc_workload(4, 260, 64, 128, types=np.full(260, 2, dtype=np.int32))
+    Y, _ = _run_proj(wl, out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+
+
+def test_tc_dense_and_custom_tables():
+    wl = _tc_workload(4, 400, 64, 128, seed=5)
+    Y, proj = _run_proj(wl, table="dense", out_dtype=torch.float32)
+    assert proj.gemm_count() == 64
+    assert np.array_equal(H.to_np(Y), wl.X.astype(np.float64) @ wl.W_up.astype(np.float64))
+    keep = oracle.support(4, "q2pow")  # the tensor-square law: 36 products
+    Y, proj = _run_proj(wl, table="custom", custom=torch.from_numpy(keep), out_dtype=torch.float32)
+    assert proj.gemm_count() == 36
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, keep=keep))
+
+
+def test_tc_bias_and_gelu_normal_data():
+    wl = _tc_workload(2, 700, 384, 256, integer=False, seed=3)
+    bias = synth.bf16_round(synth.normal(5, (wl.F,), 0.5))
+    for act, out_dtype in (("gelu", torch.float32), ("gelu", torch.bfloat16), (None, torch.float32)):
+        Y, _ = _run_proj(wl, bias=bias, act=act, out_dtype=out_dtype)
+        ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, bias=bias)
+        if act:
+            ref = np.vectorize(oracle.gelu)(ref)
+        H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"act={act}")
+
+
+def test_cyclic_schedule_needs_no_types():
+    wl = _tc_workload(2, 513, 128, 128, types=synth.cyclic_types(513, 2))
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), None, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+
+
+def test_strided_operands_and_determinism():
+    wl = _tc_workload(2, 640, 128, 256, seed=11, integer=False)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    Xp = torch.zeros((wl.M, wl.D + 64), dtype=torch.bfloat16, device="cuda")
+    Xp[:, :wl.D] = H.to_dev(wl.X, "bf16")
+    Wp = torch.zeros((wl.D, wl.F + 8), dtype=torch.bfloat16, device="cuda")
+    Wp[:, :wl.F] = H.to_dev(wl.W_up, "bf16")
+    out = torch.full((wl.M, wl.F + 8), 7.0, dtype=torch.float32, device="cuda")
+    t = H.dev_types(wl.types)
+    proj.forward(Xp[:, :wl.D], t, Wp[:, :wl.F], out=out[:, :wl.F])
+    first = out.clone()
+    proj.forward(Xp[:, :wl.D], t, Wp[:, :wl.F], out=out[:, :wl.F])
+    assert torch.equal(first, out)                       # run-to-run bitwise identical
+    assert torch.all(out[:, wl.F:] == 7.0)               # padding columns untouched
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(out[:, :wl.F]), ref, False, "strided")
+
+
+def test_bad_type_sets_status_and_zeroes_row():
+    wl = _tc_workload(2, 300, 64, 128, seed=2)
+    types = wl.types.copy()
+    types[17] = 5
+    types[200] = -1
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(types), H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert proj.last_status() == 5          # ALG_ERR_BAD_TYPE
+    assert proj.last_status() == 0          # reading clears it
+    got = H.to_np(Y)
+    assert not got[17].any() and not got[200].any()
+    good = np.ones(300, bool)
+    good[[17, 200]] = False
+    ref = oracle.proj(wl.X[good], types[good], wl.W_up, wl.d_widths, wl.f_widths)
+    assert np.array_equal(got[good], ref)
+
+
+def test_argument_errors():
+    proj = binding.Proj([128, 128], [128, 128], dtype="bf16")
+    X = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros((256, 256), dtype=torch.bfloat16, device="cuda")
+    t = torch.zeros(4, dtype=torch.int32, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.AlgError) as e:
+        proj.forward(X, t, W, workspace=small)
+    assert e.value.code == 3
+    with pytest.raises(binding.AlgError) as e:
+        proj.forward(X, None, W)            # explicit schedule without types
+    assert e.value.code == 1
+    Y = proj.forward(X[:0], t[:0], W)        # M = 0 is a no-op
+    assert Y.shape == (0, 256)
+    assert proj.macs([3, 5]) == 8 * (2 * 128 * 128) + 3 * 128 * 128 + 5 * 128 * 128
