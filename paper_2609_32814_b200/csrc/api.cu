@@ -155,7 +155,7 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
   L.hdr = off;
   off = align_up(off + sizeof(WsHeader));
   L.chunks = off;
-  off = align_up(off + (size_t)ceil_div((int)(M > 0 ? M : 1), kBucketChunk) * (first.q + 1) * sizeof(int));
+  off = align_up(off + (size_t)kMaxBucketChunks * (first.q + 1) * sizeof(int));
   L.perm = off;
   off = align_up(off + (size_t)M * sizeof(int));
   L.tiles0 = off;
@@ -286,6 +286,7 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
   b.M = (int)M;
   b.q = h->q;
+  b.chunk_rows = bucket_chunk_rows(M);
   b.hdr = (WsHeader *)(ws + L.hdr);
   b.chunk_counts = (int *)(ws + L.chunks);
   b.perm = (int *)(ws + L.perm);
@@ -401,6 +402,7 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   b.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;
   b.M = (int)M;
   b.q = h->up.q;
+  b.chunk_rows = bucket_chunk_rows(M);
   b.hdr = (WsHeader *)(ws + L.hdr);
   b.chunk_counts = (int *)(ws + L.chunks);
   b.perm = (int *)(ws + L.perm);

@@ -2,9 +2,10 @@
 // plus the device-side tile list of the grouped GEMM.  No host synchronisation anywhere: the
 // row counts per type never leave the device.
 //
-//   kernel 1 (count):   per-chunk histograms; the last CTA to finish scans them into per-chunk
-//                       bases, writes the bucket offsets and emits the tile lists.
-//   kernel 2 (scatter): perm[offset[t] + base[chunk][t] + rank_in_chunk] = row  (stable).
+//   kernel 1 (count):   per-chunk histograms (at most 256 chunks).
+//   kernel 2 (scatter): each CTA scans the histograms for the bucket offsets and its own bases,
+//                       then perm[offset[t] + base[t] + rank_in_chunk] = row  (stable); CTA 0
+//                       also emits the tile lists and resets the tile counters.
 //   kernel 3 (gather):  Xb[d,:] = X[perm[d],:]  -- every type becomes a contiguous M-slab.
 #include "common.cuh"
 
@@ -100,84 +101,99 @@ __device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list
   __syncthreads();
 }
 
+// Kernel 1: per-chunk histograms of the row types (pseudo-type q = out of range).
 __global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
   __shared__ int s_cnt[kMaxQ + 1];
-  __shared__ int s_last;
-  __shared__ int s_prefix[kMaxPairs + 1];
-  __shared__ int s_warp[8];
   const int tid = threadIdx.x;
   const int nt = a.q + 1;
   if (tid < nt) s_cnt[tid] = 0;
   __syncthreads();
-  const int row = blockIdx.x * kBucketChunk + tid;
-  if (row < a.M) {
+  const int row_begin = blockIdx.x * a.chunk_rows;
+  const int row_end = min(a.M, row_begin + a.chunk_rows);
+  for (int row = row_begin + tid; row < row_end; row += 256) {
     int t = row_type(a, row);
     if (t == a.q) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
     atomicAdd(&s_cnt[t], 1);
   }
   __syncthreads();
   if (tid < nt) a.chunk_counts[blockIdx.x * nt + tid] = s_cnt[tid];
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&a.hdr->ticket, 1) == (int)gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+}
 
-  // ---- last CTA: per-type exclusive scan over chunks (warp w takes types w, w+8, ...) -------
-  const int lane = tid & 31, warp = tid >> 5;
+// Kernel 2: every CTA scans the (at most 256) chunk histograms to find the bucket offsets and
+// its own base inside each bucket, then places its rows (stable inside a type).  CTA 0 also
+// publishes the offsets and builds the tile lists.
+__global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a) {
+  __shared__ int s_wcnt[8][kMaxQ + 1];
+  __shared__ int s_total[kMaxQ + 1];
+  __shared__ int s_base[kMaxQ + 1];     // rows of this type in earlier chunks (+ earlier sub-blocks)
+  __shared__ int s_offset[kMaxQ + 2];
+  __shared__ int s_prefix[kMaxPairs + 1];
+  __shared__ int s_warp[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nt = a.q + 1;
   const int n_chunks = gridDim.x;
   for (int t = warp; t < nt; t += 8) {
-    int carry = 0;
-    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-      int c = c0 + lane;
-      int v = (c < n_chunks) ? __ldcg(&a.chunk_counts[c * nt + t]) : 0;
-      int incl = v;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += n;
-      }
-      if (c < n_chunks) a.chunk_counts[c * nt + t] = carry + incl - v;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
+    int before = 0, total = 0;
+    for (int c = lane; c < n_chunks; c += 32) {
+      int v = a.chunk_counts[c * nt + t];
+      total += v;
+      if (c < (int)blockIdx.x) before += v;
     }
-    if (lane == 0) s_cnt[t] = carry;  // total rows of (pseudo-)type t
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      before += __shfl_xor_sync(0xffffffffu, before, d);
+      total += __shfl_xor_sync(0xffffffffu, total, d);
+    }
+    if (lane == 0) {
+      s_total[t] = total;
+      s_base[t] = before;
+    }
   }
   __syncthreads();
   if (tid == 0) {
     int run = 0;
     for (int t = 0; t < nt; ++t) {
-      a.hdr->offsets[t] = run;
-      run += s_cnt[t];
+      s_offset[t] = run;
+      run += s_total[t];
     }
-    a.hdr->offsets[nt] = run;  // == M
-    a.hdr->ticket = 0;         // ready for the next forward call
+    s_offset[nt] = run;  // == M
   }
   __syncthreads();
-  for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, s_prefix, s_warp);
-}
 
-__global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a) {
-  __shared__ int s_wcnt[8][kMaxQ + 1];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int nt = a.q + 1;
-  for (int e = tid; e < 8 * (kMaxQ + 1); e += 256) (&s_wcnt[0][0])[e] = 0;
-  __syncthreads();
-  const int row = blockIdx.x * kBucketChunk + tid;
-  const bool live = row < a.M;
-  const int t = live ? row_type(a, row) : -1 - lane;  // dead lanes never match each other
-  const unsigned peers = __match_any_sync(0xffffffffu, t);
-  const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
-  if (live && rank_in_warp == 0) s_wcnt[warp][t] = __popc(peers);
-  __syncthreads();
-  if (!live) return;
-  int before = 0;
-  for (int w = 0; w < warp; ++w) before += s_wcnt[w][t];
-  const int dest = a.hdr->offsets[t] + a.chunk_counts[blockIdx.x * nt + t] + before + rank_in_warp;
-  a.perm[dest] = row;
-  if (t == a.q && a.Y) {  // out-of-range type: the row's output is defined to be zero
-    char *y = (char *)a.Y + (size_t)row * a.ldy * a.y_elem_bytes;
-    for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
+  const int row_begin = blockIdx.x * a.chunk_rows;
+  const int row_end = min(a.M, row_begin + a.chunk_rows);
+  for (int r0 = row_begin; r0 < row_end; r0 += 256) {
+    for (int e = tid; e < 8 * (kMaxQ + 1); e += 256) (&s_wcnt[0][0])[e] = 0;
+    __syncthreads();
+    const int row = r0 + tid;
+    const bool live = row < row_end;
+    const int t = live ? row_type(a, row) : -1 - lane;  // dead lanes never match each other
+    const unsigned peers = __match_any_sync(0xffffffffu, t);
+    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+    if (live && rank_in_warp == 0) s_wcnt[warp][t] = __popc(peers);
+    __syncthreads();
+    if (live) {
+      int before = 0;
+      for (int w = 0; w < warp; ++w) before += s_wcnt[w][t];
+      a.perm[s_offset[t] + s_base[t] + before + rank_in_warp] = row;
+      if (t == a.q && a.Y) {  // out-of-range type: the row's output is defined to be zero
+        char *y = (char *)a.Y + (size_t)row * a.ldy * a.y_elem_bytes;
+        for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
+      }
+    }
+    __syncthreads();
+    if (tid < nt) {
+      int add = 0;
+      for (int w = 0; w < 8; ++w) add += s_wcnt[w][tid];
+      s_base[tid] += add;
+    }
+    __syncthreads();
+  }
+
+  if (blockIdx.x == 0) {
+    for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
+    __syncthreads();
+    for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, s_prefix, s_warp);
   }
 }
 
@@ -195,7 +211,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restric
 }  // namespace
 
 cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
-  const int n_chunks = ceil_div(a.M, kBucketChunk);
+  const int n_chunks = ceil_div(a.M, a.chunk_rows);
   bucket_count_kernel<<<n_chunks, 256, 0, st>>>(a);
   bucket_scatter_kernel<<<n_chunks, 256, 0, st>>>(a);
   count_launch(2);

@@ -11,7 +11,12 @@ namespace algproj {
 
 constexpr int kMaxQ = ALG_MAX_Q;
 constexpr int kMaxPairs = kMaxQ * kMaxQ;
-constexpr int kBucketChunk = 256;  // rows per CTA of the bucketing kernels
+constexpr int kMaxBucketChunks = 256;  // CTAs of the bucketing kernels (each scans all histograms)
+// rows per bucketing CTA: a multiple of 256 that keeps the chunk count <= kMaxBucketChunks
+inline int bucket_chunk_rows(int64_t M) {
+  int64_t iters = (M + 256 * kMaxBucketChunks - 1) / (256 * kMaxBucketChunks);
+  return (int)(256 * (iters > 0 ? iters : 1));
+}
 
 // Interaction table of one projection as the kernels see it (device memory, owned by a handle).
 struct DevTable {
@@ -35,7 +40,7 @@ struct TileRec {
 // Fixed-size header at the start of every workspace.
 struct WsHeader {
   int offsets[kMaxQ + 2];  // offsets[t] = first bucketed row of type t; [q] = first bad row; [q+1] = M
-  int ticket;              // last-block-done counter of the counting kernel
+  int reserved;
   int n_tiles[2];          // tiles in list 0 / 1
   int counter[2];          // dynamic tile counters of list 0 / 1
   int pad[25];
@@ -53,6 +58,7 @@ struct BucketArgs {
   const int32_t *types;  // nullptr => cyclic (row mod q)
   int M;
   int q;
+  int chunk_rows;        // bucket_chunk_rows(M)
   WsHeader *hdr;
   int *chunk_counts;     // [n_chunks][q+1]
   int *perm;             // [M] bucketed position -> original row
