@@ -1,0 +1,163 @@
+"""GPU parity of alg_ffn_forward (up -> GELU -> down) against the fp64 oracle, at the benchmark
+configurations (or the rows the oracle can afford) and on edge cases."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_32814_b200 import binding, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _ffn(wl, table="qq", schedule="explicit", custom=None):
+    return binding.FFN(wl.d_widths, wl.f_widths, dtype=wl.dtype, table=table, schedule=schedule, custom_keep=custom)
+
+
+def _run_ffn(wl, ffn, out_dtype, b_up=None, b_down=None, act="gelu", types=True):
+    X = H.to_dev(wl.X, wl.dtype)
+    Wu, Wd = H.to_dev(wl.W_up, wl.dtype), H.to_dev(wl.W_down, wl.dtype)
+    bu = None if b_up is None else H.to_dev(b_up, wl.dtype)
+    bd = None if b_down is None else H.to_dev(b_down, wl.dtype)
+    Y = ffn.forward(X, H.dev_types(wl.types) if types else None, Wu, Wd, b_up=bu, b_down=bd, act=act,
+                    out_dtype=out_dtype)
+    assert ffn.last_status() == 0
+    return Y
+
+
+def _sample_rows(wl, per_type, seed=0):
+    """first/last rows of every bucket, rows inside the ragged last tile, plus random rows."""
+    rng = np.random.default_rng(seed)
+    rows = []
+    for t in range(wl.q):
+        idx = np.flatnonzero(wl.types == t)
+        if idx.size == 0:
+            continue
+        tail = idx[(idx.size // 128) * 128:]
+        pick = np.concatenate([idx[:2], idx[-2:], tail[:2], rng.choice(idx, size=min(per_type, idx.size), replace=False)])
+        rows.append(pick)
+    return np.unique(np.concatenate(rows))
+
+
+def test_ffn_f32_simt_small():
+    wl = synth.make_workload("ffn32", config=7, variant=1, dtype="f32", q=3, M=200, D=96, F=240,
+                             types=synth.uniform_types(3, 200, 3), x_std=1.0, w_std=0.1)
+    bu, bd = synth.normal(11, (wl.F,), 0.1), synth.normal(12, (wl.D,), 0.1)
+    Y = _run_ffn(wl, _ffn(wl), torch.float32, b_up=bu, b_down=bd)
+    ref = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, b_up=bu, b_down=bd)
+    got = H.to_np(Y)
+    assert H.rel_fro(got, ref) <= 1e-5 and H.max_abs(got, ref) <= 1e-4
+
+
+def test_ffn_integer_identity_activation_bit_exact():
+    """With act = none both projections are exact integer arithmetic through the tensor cores
+    (|H| <= 9*256 stays exactly representable in bf16 only if small: use entries in {-1,0,1})."""
+    wl = synth.make_workload("ffnint", config=7, variant=2, dtype="bf16", q=2, M=600, D=128, F=256,
+                             types=synth.uniform_types(4, 600, 2), integer=True)
+    wl.X = np.sign(wl.X).astype(np.float32)
+    wl.W_up = np.sign(wl.W_up).astype(np.float32) * (np.abs(wl.W_up) > 2)
+    wl.W_down = np.sign(wl.W_down).astype(np.float32)
+    ffn = _ffn(wl)
+    Y = _run_ffn(wl, ffn, torch.float32, act=None)
+    Hh = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    assert np.abs(Hh).max() <= 256  # exactly representable in bf16
+    ref = oracle.proj(Hh, wl.types, wl.W_down, wl.f_widths, wl.d_widths)
+    assert np.array_equal(H.to_np(Y), ref)
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_cfg2_full_every_output(out_dtype):
+    wl = synth.config2()
+    ffn = _ffn(wl)
+    Y = _run_ffn(wl, ffn, out_dtype)
+    rows = np.arange(0, wl.M, 4) if out_dtype == torch.bfloat16 else np.arange(wl.M)
+    ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y)[rows], ref, out_dtype == torch.bfloat16, "cfg2")
+    assert ffn.macs([4096, 4096]) == 2 * 8192 * 768 * 3072 * 3 // 4
+
+
+def test_cfg2_cyclic_schedule_and_dense_control():
+    wl = synth.config2(M=2048)
+    Y = _run_ffn(wl, _ffn(wl, schedule="cyclic"), torch.float32, types=False)
+    ref = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y), ref, False, "cfg2 cyclic")
+    Yd = _run_ffn(wl, _ffn(wl, table="dense"), torch.float32)
+    refd = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=oracle.support(2, "dense"))
+    H.assert_bf16_close(H.to_np(Yd), refd, False, "cfg2 dense control")
+
+
+@pytest.mark.parametrize("q", [4, 8])
+def test_cfg3_full_size_sampled_rows(q):
+    wl = synth.config3(q)
+    ffn = _ffn(wl)
+    Y = _run_ffn(wl, ffn, torch.float32)
+    rows = _sample_rows(wl, 192, seed=q)
+    ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, False, f"cfg3 q={q}")
+    # the square d -> d projection of the same configuration
+    proj = binding.Proj(wl.d_widths, wl.d_widths, dtype="bf16")
+    Wsq = synth.bf16_round(synth.normal(synth.seed_for(3, q) + 9, (wl.D, wl.D), 0.02))
+    Ysq = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(Wsq, "bf16"), out_dtype=torch.float32)
+    refsq = oracle.proj(wl.X[rows], wl.types[rows], Wsq, wl.d_widths, wl.d_widths)
+    H.assert_bf16_close(H.to_np(Ysq[torch.from_numpy(rows).cuda()]), refsq, False, f"cfg3 square q={q}")
+
+
+@pytest.mark.parametrize("M", [1, 8, 32, 64])
+def test_cfg4_decode_shapes(M):
+    wl = synth.config4(M)
+    Y = _run_ffn(wl, _ffn(wl), torch.float32)
+    ref = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y), ref, False, f"cfg4 M={M}")
+    Yb = _run_ffn(wl, _ffn(wl), torch.bfloat16)
+    H.assert_bf16_close(H.to_np(Yb), ref, True, f"cfg4 M={M} bf16 out")
+
+
+@pytest.mark.parametrize("q", [2, 4, 8, 16])
+def test_cfg5_full_size_sampled_rows(q):
+    """Full-size launch (the configuration the benchmark times); the oracle checks every output
+    of >= 64 sampled rows per type, including bucket ends and ragged-tile rows."""
+    wl = synth.config5(q)
+    ffn = _ffn(wl)
+    Y = _run_ffn(wl, ffn, torch.float32)
+    rows = _sample_rows(wl, 64 if q <= 4 else 16, seed=q)
+    ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, False, f"cfg5 q={q}")
+    del Y
+    torch.cuda.empty_cache()
+
+
+def test_ffn_host_entry_point_matches_device_entry_point():
+    wl = synth.config2(M=1024)
+    ffn = _ffn(wl)
+    Yd = _run_ffn(wl, ffn, torch.float32)
+    Xh = torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory()
+    th = torch.from_numpy(wl.types).pin_memory()
+    Yh = torch.empty((wl.M, wl.D), dtype=torch.float32).pin_memory()
+    ffn.forward_host(Xh, th, H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"), Yh)
+    torch.cuda.synchronize()
+    assert torch.equal(Yh, Yd.cpu())
+
+
+def test_ffn_graph_capture_replays():
+    wl = synth.config2(M=1024)
+    ffn = _ffn(wl)
+    X, t = H.to_dev(wl.X, "bf16"), H.dev_types(wl.types)
+    Wu, Wd = H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16")
+    Y = torch.zeros((wl.M, wl.D), dtype=torch.float32, device="cuda")
+    ws = torch.empty(ffn.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
+    ffn.forward(X, t, Wu, Wd, out=Y, workspace=ws)
+    want = Y.clone()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        ffn.forward(X, t, Wu, Wd, out=Y, workspace=ws, stream=s)   # warm-up on the capture stream
+        with torch.cuda.graph(g, stream=s):
+            ffn.forward(X, t, Wu, Wd, out=Y, workspace=ws, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    for _ in range(3):
+        Y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(Y, want)
