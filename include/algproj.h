@@ -145,6 +145,13 @@ alg_status_t alg_ffn_forward_host(alg_ffn_t h, const void *X_host, const int32_t
                                   const void *W_down, const void *b_down, alg_act_t act,
                                   void *Y_host, alg_dtype_t y_dtype, void *workspace,
                                   size_t workspace_bytes, void *stream);
+/* Benchmark aid: when enabled, every alg_ffn_forward on this handle records CUDA events on the
+ * call's stream between its kernels (do not enable while capturing a graph).
+ * alg_ffn_get_timing waits for the most recent call and returns four durations in
+ * milliseconds: [0] row-type bucketing, [1] row gather, [2] up projection (with activation),
+ * [3] down projection. */
+alg_status_t alg_ffn_set_timing(alg_ffn_t h, int enable);
+alg_status_t alg_ffn_get_timing(alg_ffn_t h, float *ms);
 alg_status_t alg_ffn_macs(alg_ffn_t h, const int64_t *rows_per_type, int64_t *macs);
 alg_status_t alg_ffn_last_status(alg_ffn_t h, void *stream, alg_status_t *status);
 

@@ -33,7 +33,7 @@ EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
     "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
-    "alg_ffn_macs", "alg_ffn_last_status", "alg_status_string", "alg_launch_count",
+    "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
 ]
 
 _lib = None
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.alg_ffn_forward_host.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_ffn_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.alg_ffn_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.alg_ffn_set_timing.argtypes = [vp, i32]
+        L.alg_ffn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
         L.alg_status_string.argtypes = [i32]
         L.alg_status_string.restype = ctypes.c_char_p
         L.alg_launch_count.argtypes = []
@@ -241,6 +243,15 @@ class FFN(_Handle):
                                           _ptr(W_down), _ptr(b_down), _ACTS[act], _ptr(Y_host), _DTYPES[Y_host.dtype],
                                           _ptr(ws), ws.numel(), _stream(stream)), "alg_ffn_forward_host")
         return Y_host
+
+    def set_timing(self, enable: bool):
+        _check(lib().alg_ffn_set_timing(self._h, int(enable)), "alg_ffn_set_timing")
+
+    def get_timing(self):
+        """Milliseconds of the last forward call: (bucketing, gather, up projection, down projection)."""
+        ms = (ctypes.c_float * 4)()
+        _check(lib().alg_ffn_get_timing(self._h, ms), "alg_ffn_get_timing")
+        return tuple(float(v) for v in ms)
 
     def macs(self, rows_per_type) -> int:
         rows = (ctypes.c_int64 * self.q)(*[int(v) for v in rows_per_type])

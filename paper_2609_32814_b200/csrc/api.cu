@@ -34,6 +34,8 @@ struct alg_proj_s {
 struct alg_ffn_s {
   alg_proj_s up, down;
   int D = 0, F = 0;
+  bool timing = false;       // record events between the kernels of each forward call
+  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 };
 
 namespace {
@@ -191,7 +193,8 @@ ListSpec make_list(const alg_proj_s &p, char *ws, size_t off) {
 
 alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
-                      int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st) {
+                      int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
+                      cudaEvent_t after_gather = nullptr) {
   ProjArgs a;
   a.tab = p.d_tab;
   a.hdr = (const WsHeader *)(ws + L.hdr);
@@ -219,9 +222,11 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list
       a.X = ws + L.xb;
       a.ldx = p.K;
     }
+    if (after_gather) cudaEventRecord(after_gather, st);
     a.in_perm = nullptr;
     return cuda_status(launch_proj_tc(a, p.tile_n, p.num_sms, st));
   }
+  if (after_gather) cudaEventRecord(after_gather, st);
   a.X = X;
   a.ldx = ldx;
   a.in_perm = x_bucketed ? nullptr : (const int *)(ws + L.perm);
@@ -368,6 +373,8 @@ alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, cons
 
 alg_status_t alg_ffn_destroy(alg_ffn_t h) {
   if (!h) return ALG_ERR_INVALID_ARG;
+  for (int e = 0; e < 5; ++e)
+    if (h->ev[e]) cudaEventDestroy(h->ev[e]);
   free_proj(h->down);
   free_proj(h->up);
   delete h;
@@ -414,11 +421,36 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   b.ldy = h->D;
   b.N = h->D;
   b.y_elem_bytes = elem_bytes(y_dtype);
+  const bool tm = h->timing;
+  if (tm) cudaEventRecord(h->ev[0], st);
   if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;
-  alg_status_t s = run_proj(h->up, L, ws, 0, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st);
+  alg_status_t s = run_proj(h->up, L, ws, 0, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st,
+                            tm ? h->ev[2] : nullptr);
   if (s != ALG_OK) return s;
-  return run_proj(h->down, L, ws, 1, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st);
+  if (tm) cudaEventRecord(h->ev[3], st);
+  s = run_proj(h->down, L, ws, 1, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st);
+  if (tm) cudaEventRecord(h->ev[4], st);
+  return s;
+}
+
+alg_status_t alg_ffn_set_timing(alg_ffn_t h, int enable) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  if (enable && !h->ev[0]) {
+    for (int e = 0; e < 5; ++e)
+      if (cudaEventCreate(&h->ev[e]) != cudaSuccess) return ALG_ERR_CUDA;
+  }
+  h->timing = enable != 0;
+  return ALG_OK;
+}
+
+alg_status_t alg_ffn_get_timing(alg_ffn_t h, float *ms) {
+  if (!h || !ms || !h->ev[0]) return ALG_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(h->ev[4]) != cudaSuccess) return ALG_ERR_CUDA;
+  for (int e = 0; e < 4; ++e)
+    if (cudaEventElapsedTime(&ms[e], h->ev[e], h->ev[e + 1]) != cudaSuccess) return ALG_ERR_CUDA;
+  return ALG_OK;
 }
 
 alg_status_t alg_ffn_host_workspace_bytes(alg_ffn_t h, int64_t max_M, alg_dtype_t y_dtype, size_t *bytes) {
