@@ -108,6 +108,37 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
                               alg_act_t act, void *Y, int64_t ldy, alg_dtype_t y_dtype,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/* alg_proj_forward without a workspace argument and without any allocation.  (The paper has
+ * no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested -- a serving loop whose
+ * memory was handed out once at start-up to a pool it may not grow, a plug-in called from a
+ * host framework that forbids cudaMalloc / cudaFree on its hot path because they synchronise
+ * the whole device, or a caller that simply has no allocator to hand.  Such callers still pass
+ * their own X, types, W, bias and Y; only the scratch (row permutation, bucket offsets, tile
+ * list, type-bucketed copy of X) comes from the library, from a fixed array of
+ * ALG_STATIC_SCRATCH_BYTES that is part of the loaded library image on every GPU and stays
+ * there until the process exits.
+ *
+ * Limits and rules
+ *   - The handle must exist already: create it once at start-up (creation does allocate a few
+ *     hundred bytes).  This call itself performs no cudaMalloc, cudaFree or other allocation.
+ *   - Problems whose scratch need, alg_proj_workspace_bytes(h, M), exceeds
+ *     ALG_STATIC_SCRATCH_BYTES are refused with ALG_ERR_WORKSPACE_TOO_SMALL and nothing is
+ *     launched; use alg_proj_forward with your own workspace for those.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  It keeps whatever the previous call left;
+ *     nothing in it has to start at zero, every call rewrites what it reads.  Two calls that
+ *     overlap on the GPU (different streams without an event between them) race on it and
+ *     give undefined results: order them.
+ * Arguments, layouts and results are otherwise exactly those of alg_proj_forward. */
+#define ALG_STATIC_SCRATCH_BYTES (8u << 20)
+alg_status_t alg_proj_forward_static(alg_proj_t h, const void *X, int64_t ldx,
+                                     const int32_t *types, int64_t M, const void *W, int64_t ldw,
+                                     const void *bias, alg_act_t act, void *Y, int64_t ldy,
+                                     alg_dtype_t y_dtype, void *stream);
+
 /* Number of kept block GEMMs (2q^2-q for QQ, Eq. q-rank). */
 alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n);
 /* Multiply-accumulates of one forward pass with rows_per_type[i] rows of type i

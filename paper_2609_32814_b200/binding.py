@@ -31,7 +31,7 @@ _SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC}
 
 EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
-    "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
+    "alg_proj_forward_static", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
     "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
 ]
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.alg_proj_destroy.argtypes = [vp]
         L.alg_proj_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
         L.alg_proj_forward.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp, ctypes.c_size_t, vp]
+        L.alg_proj_forward_static.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp]
         L.alg_proj_gemm_count.argtypes = [vp, ctypes.POINTER(i64)]
         L.alg_proj_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.alg_proj_kernel_path.argtypes = [vp, i64, ctypes.POINTER(i32)]
@@ -169,6 +170,17 @@ class Proj(_Handle):
                                       W.stride(0), _ptr(bias), _ACTS[act], _ptr(out),
                                       out.stride(0) if M else self.N, _DTYPES[out.dtype], _ptr(ws), ws.numel(),
                                       _stream(stream)), "alg_proj_forward")
+        return out
+
+    def forward_static(self, X, types, W, out, bias=None, act=None, stream=None):
+        """alg_proj_forward_static: same result as forward(), but the scratch is the fixed array
+        inside the library, so nothing is allocated -- `out` must be supplied by the caller, and
+        problems needing more than the built-in scratch raise ALG_ERR_WORKSPACE_TOO_SMALL."""
+        M = X.shape[0]
+        _check(lib().alg_proj_forward_static(self._h, _ptr(X), X.stride(0) if M else self.K, _ptr(types), M,
+                                             _ptr(W), W.stride(0), _ptr(bias), _ACTS[act], _ptr(out),
+                                             out.stride(0) if M else self.N, _DTYPES[out.dtype], _stream(stream)),
+               "alg_proj_forward_static")
         return out
 
     def gemm_count(self) -> int:
