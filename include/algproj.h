@@ -85,7 +85,7 @@ typedef enum {
  * accumulation).  custom_keep is read only for ALG_TABLE_CUSTOM, else pass NULL; every
  * (i,j) of a custom table must keep at least one k.  1 <= q <= ALG_MAX_Q.
  * The tensor-core path needs every s[k] to be a multiple of 64 and every r[j] a multiple of
- * 128; other bf16/fp32 shapes run on the SIMT path.  */
+ * 128 (or of 192); other bf16/fp32 shapes run on the SIMT path.  */
 alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
                              const int32_t *out_widths, alg_dtype_t dtype, alg_table_t table,
                              const uint8_t *custom_keep, alg_schedule_t schedule);

@@ -2,6 +2,7 @@
 // validation, workspace layout and the launch sequence of one forward pass.
 #include <algorithm>
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -26,9 +27,11 @@ struct alg_proj_s {
   int *d_status = nullptr;  // owned unless `shared_status`
   bool shared_status = false;
   bool tc_ok = false;
-  int tile_n = 0;           // tensor-core tile width
+  bool pair_kernel = false; // cta_group::2 kernel (256-row tiles)
+  int tile_n = 0;           // tensor-core tile width of the one-CTA kernel
   int device = 0;
   int num_sms = 148;
+  int n_workers = 1;        // persistent CTAs (or CTA pairs) of the tensor-core kernel
 };
 
 struct alg_ffn_s {
@@ -39,6 +42,9 @@ struct alg_ffn_s {
 };
 
 namespace {
+
+long long *g_trace = nullptr;  // debug timeline buffer of the tensor-core kernel
+int g_trace_cap = 0;
 
 size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
@@ -54,8 +60,8 @@ size_t max_tiles(const alg_proj_s &p, int64_t M, int tile_m, int tile_n) {
 }
 
 bool use_tc(const alg_proj_s &p) { return p.dtype == ALG_BF16 && p.tc_ok; }
-int tile_m_of(const alg_proj_s &p) { return use_tc(p) ? kTcTileM : 64; }
-int tile_n_of(const alg_proj_s &p) { return use_tc(p) ? p.tile_n : 64; }
+int tile_m_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kTc2TileM : kTcTileM; }
+int tile_n_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kTc2TileN : p.tile_n; }
 int elem_bytes(alg_dtype_t d) { return d == ALG_BF16 ? 2 : 4; }
 
 alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t *out_w, alg_dtype_t dtype,
@@ -98,28 +104,52 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
       if (m == 0) return ALG_ERR_INVALID_ARG;  // an output block nobody writes
       p.tab.keep[i * q + j] = m;
     }
-  // pairs sorted by total K length, longest first (stable)
-  std::vector<std::pair<int, int>> order;  // (-K length, pair)
+  // tensor-core eligibility: bf16, K groups in 64-steps, N groups in 128-steps
+  p.tc_ok = dtype == ALG_BF16;
+  bool all256 = true, all192 = true, all128 = true;
+  for (int g = 0; g < q; ++g) {
+    if (p.s[g] % kTcBlockK) p.tc_ok = false;
+    if (p.r[g] % 256) all256 = false;
+    if (p.r[g] % 192) all192 = false;
+    if (p.r[g] % 128) all128 = false;
+  }
+  if (!all256 && !all192 && !all128) p.tc_ok = false;
+  p.tile_n = all256 ? 256 : all192 ? 192 : 128;
+  // CTA-pair kernel whenever every output group splits into 256-wide tiles plus a 128-wide rest
+  // (measured: it wins only when every tile has a long K loop; short loops favour the one-CTA kernel)
+  int min_klen = 1 << 30;
   for (int pr = 0; pr < q * q; ++pr) {
     int len = 0;
     for (int k = 0; k < q; ++k)
       if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
-    order.push_back({-len, pr});
+    min_klen = std::min(min_klen, len);
   }
-  std::stable_sort(order.begin(), order.end(),
-                   [](const std::pair<int, int> &x, const std::pair<int, int> &y) { return x.first < y.first; });
-  p.tab.n_pairs = q * q;
-  for (int e = 0; e < q * q; ++e) p.tab.pair_order[e] = order[e].second;
+  p.pair_kernel = p.tc_ok && all128 && min_klen >= 4096 && std::getenv("ALGPROJ_ONE_CTA") == nullptr;
+  if (std::getenv("ALGPROJ_PAIR") != nullptr) p.pair_kernel = p.tc_ok && all128;
 
-  // tensor-core eligibility: bf16, K groups in 64-steps, N groups in 128-steps
-  p.tc_ok = dtype == ALG_BF16;
-  bool all256 = true;
-  for (int g = 0; g < q; ++g) {
-    if (p.s[g] % kTcBlockK) p.tc_ok = false;
-    if (p.r[g] % 128) p.tc_ok = false;
-    if (p.r[g] % 256) all256 = false;
+  // tile classes sorted by cost = K length x tile width, most expensive first (stable)
+  {
+    const int tn = tile_n_of(p);
+    const bool split = use_tc(p) && p.pair_kernel;
+    std::vector<std::pair<long long, int>> order;  // (-cost, class)
+    for (int pr = 0; pr < q * q; ++pr) {
+      long long len = 0;
+      for (int k = 0; k < q; ++k)
+        if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
+      const int width = p.r[pr % q];
+      if (split) {
+        if (width / tn) order.push_back({-len * tn, pr * 2});
+        if (width % tn) order.push_back({-len * (width % tn), pr * 2 + 1});
+      } else {
+        order.push_back({-len * std::min(tn, width), pr * 2});
+      }
+    }
+    std::stable_sort(order.begin(), order.end(), [](const std::pair<long long, int> &x,
+                                                    const std::pair<long long, int> &y) { return x.first < y.first; });
+    p.tab.n_classes = (int)order.size();
+    for (size_t e = 0; e < order.size(); ++e) p.tab.class_order[e] = order[e].second;
+    p.tab.n_pairs = q * q;
   }
-  p.tile_n = all256 ? 256 : 128;
 
   if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
   cudaDeviceProp prop;
@@ -136,6 +166,10 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     if (cudaMemset(p.d_status, 0, sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
   }
   if (use_tc(p) && tc_init() != cudaSuccess) return ALG_ERR_CUDA;
+  if (use_tc(p)) {
+    p.n_workers = p.pair_kernel ? tc2_max_pairs(p.num_sms) : std::min(p.num_sms, kMaxWorkers);
+    if (p.n_workers < 1) return ALG_ERR_CUDA;
+  }
   return ALG_OK;
 }
 
@@ -188,6 +222,7 @@ ListSpec make_list(const alg_proj_s &p, char *ws, size_t off) {
   ls.tiles = (TileRec *)(ws + off);
   ls.tile_m = tile_m_of(p);
   ls.tile_n = tile_n_of(p);
+  ls.split_rem = use_tc(p) && p.pair_kernel;
   return ls;
 }
 
@@ -200,6 +235,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list
   a.hdr = (const WsHeader *)(ws + L.hdr);
   a.tiles = (const TileRec *)(ws + (list == 0 ? L.tiles0 : L.tiles1));
   a.list = list;
+  a.q = p.q;
   a.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
   a.W = W;
   a.ldw = ldw;
@@ -212,6 +248,9 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list
   a.K = p.K;
   a.N = p.N;
   a.status = p.d_status;
+  a.b_kmajor = std::getenv("ALGPROJ_BT") != nullptr;
+  a.trace = g_trace;
+  a.trace_cap = g_trace_cap;
   if (use_tc(p)) {
     if (x_bucketed) {
       a.X = X;
@@ -224,7 +263,8 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list
     }
     if (after_gather) cudaEventRecord(after_gather, st);
     a.in_perm = nullptr;
-    return cuda_status(launch_proj_tc(a, p.tile_n, p.num_sms, st));
+    if (p.pair_kernel) return cuda_status(launch_proj_tc2(a, p.num_sms, st));
+    return cuda_status(launch_proj_tc(a, p.tile_n, p.n_workers, st));
   }
   if (after_gather) cudaEventRecord(after_gather, st);
   a.X = X;
@@ -522,6 +562,13 @@ const char *alg_status_string(alg_status_t s) {
     case ALG_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
   }
   return "unknown status";
+}
+
+// Internal debug hook (not part of the public header): device buffer of 8*3*cap int64 slots that
+// the first eight CTAs of the tensor-core kernel fill with (clock64 << 8 | tag) records.
+void alg_debug_set_trace(void *device_buffer, int cap) {
+  g_trace = (long long *)device_buffer;
+  g_trace_cap = cap;
 }
 
 int64_t alg_launch_count(void) { return algproj::g_launches.load(std::memory_order_relaxed); }

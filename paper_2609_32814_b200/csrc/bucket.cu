@@ -41,24 +41,38 @@ __device__ int block_exclusive_scan_256(int v, int *smem_warp /*[8]*/, int *tota
   return base + incl - v;
 }
 
-__device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list, WsHeader *hdr_w,
-                               int *s_prefix /*[kMaxPairs+1]*/, int *s_warp /*[8]*/) {
+// Tiles of class `cls` per m-tile, and the geometry of its nt-th tile.
+__device__ __forceinline__ int class_n_tiles(const ListSpec &ls, int cls, int width) {
+  const int w = cls & 1;
+  if (!ls.split_rem) return w == 0 ? ceil_div(width, ls.tile_n) : 0;
+  return w == 0 ? width / ls.tile_n : ((width % ls.tile_n) ? 1 : 0);
+}
+
+struct EmitSmem {
+  int prefix[kMaxClasses + 1];        // tiles before class position c
+  int warp[8];
+};
+
+__device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list, WsHeader *hdr_w, EmitSmem *sm) {
+  int *s_prefix = sm->prefix;
+  int *s_warp = sm->warp;
   const DevTable *tab = ls.tab;
-  const int q = tab->q, np = tab->n_pairs;
-  // tiles per pair, in the host-chosen order (longest K first)
-  constexpr int kPer = kMaxPairs / 256;  // 4 pairs per thread
+  const int q = tab->q, nc = tab->n_classes;
+  // tiles per class, in the host-chosen order (most expensive first)
+  constexpr int kPer = kMaxClasses / 256;  // 8 classes per thread
   int local[kPer];
   int sum = 0;
 #pragma unroll
   for (int e = 0; e < kPer; ++e) {
-    int p = threadIdx.x * kPer + e;
+    int c = threadIdx.x * kPer + e;
     int cnt = 0;
-    if (p < np) {
-      int pair = tab->pair_order[p];
+    if (c < nc) {
+      int cls = tab->class_order[c];
+      int pair = cls >> 1;
       int i = pair / q, j = pair % q;
       int rows = hdr->offsets[i + 1] - hdr->offsets[i];
       int width = tab->ro[j + 1] - tab->ro[j];
-      cnt = ceil_div(rows, ls.tile_m) * ceil_div(width, ls.tile_n);
+      cnt = ceil_div(rows, ls.tile_m) * class_n_tiles(ls, cls, width);
     }
     local[e] = cnt;
     sum += cnt;
@@ -67,31 +81,33 @@ __device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list
   int base = block_exclusive_scan_256(sum, s_warp, &total);
 #pragma unroll
   for (int e = 0; e < kPer; ++e) {
-    int p = threadIdx.x * kPer + e;
-    if (p < kMaxPairs) s_prefix[p] = base;
+    int c = threadIdx.x * kPer + e;
+    s_prefix[c] = base;
     base += local[e];
   }
-  if (threadIdx.x == 255) s_prefix[kMaxPairs] = total;
+  if (threadIdx.x == 255) s_prefix[kMaxClasses] = total;
   __syncthreads();
   for (int e = threadIdx.x; e < total; e += 256) {
-    // last p with s_prefix[p] <= e and a non-empty pair
-    int lo = 0, hi = np;  // invariant: s_prefix[lo] <= e < s_prefix[hi] (s_prefix[np..] == total)
+    // last class c with s_prefix[c] <= e (empty classes share a prefix with their successor)
+    int lo = 0, hi = nc;  // invariant: s_prefix[lo] <= e < s_prefix[hi] (s_prefix[nc..] == total)
     while (hi - lo > 1) {
       int mid = (lo + hi) >> 1;
       if (s_prefix[mid] <= e) lo = mid; else hi = mid;
     }
-    int pair = tab->pair_order[lo];
-    int i = pair / q, j = pair % q;
-    int width = tab->ro[j + 1] - tab->ro[j];
-    int n_tiles = ceil_div(width, ls.tile_n);
-    int loc = e - s_prefix[lo];
-    int mt = loc / n_tiles, nt = loc % n_tiles;  // n fastest: neighbours share the A rows
-    int rows = hdr->offsets[i + 1] - hdr->offsets[i];
+    const int cls = tab->class_order[lo];
+    const int pair = cls >> 1;
+    const int i = pair / q, j = pair % q;
+    const int width = tab->ro[j + 1] - tab->ro[j];
+    const int n_tiles = class_n_tiles(ls, cls, width);
+    const int loc = e - s_prefix[lo];
+    const int mt = loc / n_tiles, nt = loc % n_tiles;  // n fastest: neighbours share the A rows
+    const int rows = hdr->offsets[i + 1] - hdr->offsets[i];
+    const int c0 = (cls & 1) ? (width / ls.tile_n) * ls.tile_n : nt * ls.tile_n;
     TileRec rec;
     rec.row0 = hdr->offsets[i] + mt * ls.tile_m;
     rec.rows = min(ls.tile_m, rows - mt * ls.tile_m);
-    rec.pair = pair;
-    rec.n0 = tab->ro[j] + nt * ls.tile_n;
+    rec.pair = pair | (min(ls.tile_n, width - c0) << 16);
+    rec.n0 = tab->ro[j] + c0;
     ls.tiles[e] = rec;
   }
   if (threadIdx.x == 0) {
@@ -127,8 +143,7 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
   __shared__ int s_total[kMaxQ + 1];
   __shared__ int s_base[kMaxQ + 1];     // rows of this type in earlier chunks (+ earlier sub-blocks)
   __shared__ int s_offset[kMaxQ + 2];
-  __shared__ int s_prefix[kMaxPairs + 1];
-  __shared__ int s_warp[8];
+  __shared__ EmitSmem s_emit;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
   const int n_chunks = gridDim.x;
@@ -193,7 +208,7 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
   if (blockIdx.x == 0) {
     for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
     __syncthreads();
-    for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, s_prefix, s_warp);
+    for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, &s_emit);
   }
 }
 

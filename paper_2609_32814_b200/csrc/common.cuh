@@ -11,6 +11,7 @@ namespace algproj {
 
 constexpr int kMaxQ = ALG_MAX_Q;
 constexpr int kMaxPairs = kMaxQ * kMaxQ;
+constexpr int kMaxClasses = 2 * kMaxPairs;  // per pair: full-width tiles and the remainder tile
 constexpr int kMaxBucketChunks = 256;  // CTAs of the bucketing kernels (each scans all histograms)
 // rows per bucketing CTA: a multiple of 256 that keeps the chunk count <= kMaxBucketChunks
 inline int bucket_chunk_rows(int64_t M) {
@@ -25,7 +26,10 @@ struct DevTable {
   int so[kMaxQ + 1];           // prefix sums of the input group widths  (S_k = [so[k], so[k+1]))
   int ro[kMaxQ + 1];           // prefix sums of the output group widths (R_j = [ro[j], ro[j+1]))
   uint32_t keep[kMaxPairs];    // keep[i*q+j] bit k set  <=>  k in B(i,j)
-  int pair_order[kMaxPairs];   // pairs (i*q+j) sorted by total K length, longest first
+  // Tile classes (pair*2 + w; w = 0: tiles of the full tile width, w = 1: the narrower remainder
+  // tile of the output group), sorted by cost = K length x tile width, most expensive first.
+  int n_classes;
+  int class_order[kMaxClasses];
 };
 
 // One output tile of the grouped GEMM: rows [row0, row0+rows) of the type-bucketed row order
@@ -33,7 +37,7 @@ struct DevTable {
 struct TileRec {
   int row0;
   int rows;
-  int pair;   // i * q + j
+  int pair;   // (i * q + j) | (columns of the tile << 16)
   int n0;     // absolute first column
 };
 
@@ -52,6 +56,7 @@ struct ListSpec {
   TileRec *tiles;
   int tile_m;
   int tile_n;
+  int split_rem;  // 1: full tile_n-wide tiles plus one narrower remainder tile; 0: ceil(width / tile_n) tiles
 };
 
 struct BucketArgs {
@@ -96,15 +101,25 @@ struct ProjArgs {
   int M;
   int K;
   int N;
+  int q;
   int *status;
+  int b_kmajor;           // experiment: B operand given as the transposed bank [N, K]
+  long long *trace;       // debug timeline (nullptr = off)
+  int trace_cap;
 };
 
 cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
 
-// tcgen05 path. tile_n in {128, 256}.
+// tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
+// (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.
 constexpr int kTcTileM = 128;
 constexpr int kTcBlockK = 64;
+constexpr int kTc2TileM = 256;
+constexpr int kTc2TileN = 256;
 cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st);
+cudaError_t launch_proj_tc2(const ProjArgs &a, int num_sms, cudaStream_t st);
+int tc2_max_pairs(int num_sms);  // CTA pairs that can be co-resident (0 on failure)
+constexpr int kMaxWorkers = 256;
 cudaError_t tc_init();  // resolves the driver entry point for tensor-map encoding
 
 // decode path (M <= 64)

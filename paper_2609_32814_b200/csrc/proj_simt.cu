@@ -36,8 +36,9 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
   const int tx = tid & 15, ty = tid >> 4;  // 16 x 16 threads, 4 x 4 outputs each
 
   for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    const TileRec rec = a.tiles[tile];
-    const int i = rec.pair / q, j = rec.pair % q;
+    TileRec rec = a.tiles[tile];
+    rec.pair &= 0xFFFF;
+    const int j = rec.pair % q;
     const int n_valid = min(TN, tab->ro[j + 1] - rec.n0);
     __syncthreads();
     if (tid < TM) {

@@ -1,0 +1,188 @@
+// PTX wrappers and small device helpers shared by the tensor-core kernels (sm_100a only).
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace algproj {
+namespace tc {
+
+constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s at B200 clocks
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
+// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+
+// GELU with the exact (erf) definition, gelu(z) = z * Phi(z).  The lower tail Phi(-u), u >= 0, is
+// evaluated as 2^q(u) with a degree-6 polynomial q fitted to log2(Phi(-u)) on [0, 6] (one ex2 and
+// six FMAs, no branches); |gelu error| < 1e-7 over the whole real line, i.e. fp32 rounding level.
+__device__ __forceinline__ float gelu_erf(float z) {
+  const float u = fminf(fabsf(z), 6.0f);
+  float q = 3.3093889e-05f;
+  q = fmaf(q, u, -7.6922908e-04f);
+  q = fmaf(q, u, 8.0807470e-03f);
+  q = fmaf(q, u, -5.3412151e-02f);
+  q = fmaf(q, u, -4.5877093e-01f);
+  q = fmaf(q, u, -1.1512017f);
+  q = fmaf(q, u, -0.99999309f);
+  float t;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(q));
+  return z * (z < 0.f ? t : 1.0f - t);
+}
+__device__ __forceinline__ float gelu_tanh(float z) {
+  float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+  return 0.5f * z * (1.0f + tanhf(u));
+}
+
+
+// Static schedule: the tile list is sorted most-expensive first; worker c of n takes, in round r,
+// tile r*n + c on even rounds and r*n + (n-1-c) on odd rounds (boustrophedon).  That balances the
+// per-worker cost like a longest-processing-time assignment without inter-CTA traffic, and keeps
+// the workers of one round on neighbouring tiles (same rows or same columns), so the lines one CTA
+// pulls into L2 are the lines its neighbours ask for at the same moment.  (Giving each worker a
+// contiguous run of tiles instead was measured 10-15 % slower: the concurrent working set spreads
+// over the whole problem.)
+__device__ __forceinline__ int snake_tile(int round, int worker, int n_workers) {
+  return round * n_workers + ((round & 1) ? (n_workers - 1 - worker) : worker);
+}
+
+__device__ __forceinline__ TileRec load_tile(const TileRec *tiles, int idx, int end) {
+  TileRec rec;
+  if (idx < end) {
+    const int4 v = __ldg((const int4 *)(tiles + idx));
+    rec.row0 = v.x, rec.rows = v.y, rec.pair = v.z, rec.n0 = v.w;
+  } else {
+    rec.row0 = -1, rec.rows = 0, rec.pair = 0, rec.n0 = 0;
+  }
+  return rec;
+}
+
+// Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
+// it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
+__device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjArgs &a, int64_t out_row, int col) {
+  if (a.bias) {
+    const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
+#pragma unroll
+    for (int x = 0; x < 32; ++x) f[x] += __bfloat162float(__ldg(b + x));
+  }
+  if (a.act == ALG_ACT_GELU_ERF) {
+#pragma unroll
+    for (int x = 0; x < 32; ++x) f[x] = gelu_erf(f[x]);
+  } else if (a.act == ALG_ACT_GELU_TANH) {
+#pragma unroll
+    for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
+  }
+  if (a.y_bf16) {
+    uint32_t w[16];
+#pragma unroll
+    for (int h = 0; h < 16; ++h) {
+      __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * h], f[2 * h + 1]);
+      w[h] = *(uint32_t *)&p;
+    }
+    __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + out_row * a.ldy + col;
+    if ((((uintptr_t)dst) & 31u) == 0) {  // 32-byte stores fill whole sectors
+#pragma unroll
+      for (int g = 0; g < 2; ++g)
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + g * 16), "r"(w[g * 8]),
+                     "r"(w[g * 8 + 1]), "r"(w[g * 8 + 2]), "r"(w[g * 8 + 3]), "r"(w[g * 8 + 4]), "r"(w[g * 8 + 5]),
+                     "r"(w[g * 8 + 6]), "r"(w[g * 8 + 7])
+                     : "memory");
+    } else {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) ((uint4 *)dst)[g] = make_uint4(w[g * 4], w[g * 4 + 1], w[g * 4 + 2], w[g * 4 + 3]);
+    }
+  } else {
+    float *dst = (float *)a.Y + out_row * a.ldy + col;
+    if ((((uintptr_t)dst) & 31u) == 0) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g)
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + g * 8),
+                     "r"(__float_as_uint(f[g * 8])), "r"(__float_as_uint(f[g * 8 + 1])),
+                     "r"(__float_as_uint(f[g * 8 + 2])), "r"(__float_as_uint(f[g * 8 + 3])),
+                     "r"(__float_as_uint(f[g * 8 + 4])), "r"(__float_as_uint(f[g * 8 + 5])),
+                     "r"(__float_as_uint(f[g * 8 + 6])), "r"(__float_as_uint(f[g * 8 + 7]))
+                     : "memory");
+    } else {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) ((float4 *)dst)[g] = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
+    }
+  }
+}
+
+#define ALG_TRACE(role, tag)                                                                        \
+  do {                                                                                              \
+    if (a.trace && blockIdx.x < 8 && tr_n < a.trace_cap)                                            \
+      a.trace[((size_t)blockIdx.x * 3 + (role)) * a.trace_cap + tr_n++] = (clock64() << 8) | (tag); \
+  } while (0)
+
+// Host side: tensor-map encoding through the driver entry point (no link-time libcuda dependency).
+cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,
+                        uint32_t box_inner, uint32_t box_outer);
+
+}  // namespace tc
+}  // namespace algproj

@@ -186,3 +186,20 @@ def test_argument_errors():
     Y = proj.forward(X[:0], t[:0], W)        # M = 0 is a no-op
     assert Y.shape == (0, 256)
     assert proj.macs([3, 5]) == 8 * (2 * 128 * 128) + 3 * 128 * 128 + 5 * 128 * 128
+
+
+def test_gelu_epilogue_accuracy_on_a_dense_grid():
+    """Identity weights turn the projection into a pure epilogue test: Y = gelu(x) in fp32.
+    The kernel's branch-free erf-GELU must match the closed form to fp32 rounding level."""
+    n = 128
+    vals = np.concatenate([np.linspace(-9, 9, 128 * n - 64), [0.0] * 8, [-6.0, 6.0, -40.0, 40.0], np.zeros(52)])
+    X = synth.bf16_round(vals.astype(np.float32).reshape(128, n))
+    proj = binding.Proj([n], [n], dtype="bf16")
+    W = torch.eye(n, dtype=torch.bfloat16, device="cuda")
+    t = torch.zeros(128, dtype=torch.int32, device="cuda")
+    Y = proj.forward(H.to_dev(X, "bf16"), t, W, act="gelu", out_dtype=torch.float32)
+    ref = np.vectorize(oracle.gelu)(X.astype(np.float64))
+    err = np.abs(H.to_np(Y) - ref)
+    assert err.max() <= 4e-7 + 2e-7 * np.abs(ref).max(), err.max()
+    Yt = proj.forward(H.to_dev(X, "bf16"), t, W, act="gelu_tanh", out_dtype=torch.float32)
+    assert np.abs(H.to_np(Yt) - ref).max() <= 2e-3      # the tanh form is a different function
