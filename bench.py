@@ -177,7 +177,10 @@ def main():
     dev = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)
     X, Wu, Wd = dev(wl.X), dev(wl.W_up), dev(wl.W_down)
     types = torch.from_numpy(wl.types).cuda()
-    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    # config 2 fixes the schedule "type = position mod 2": the handle is created with it
+    # (ALG_SCHED_CYCLIC), the per-call types array is then not needed.  The explicit-types path of
+    # the same workload is timed as a side measurement.
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
     ws = torch.empty(ffn.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
     Y = torch.empty((wl.M, wl.D), dtype=torch.bfloat16, device="cuda")
     flops = kept_flops(ffn, wl)
@@ -185,7 +188,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        ffn.forward(X, types, Wu, Wd, act="gelu", out=Y, workspace=ws, stream=stream)
+        ffn.forward(X, None, Wu, Wd, act="gelu", out=Y, workspace=ws, stream=stream)
 
     def barrier():
         if world > 1:
@@ -242,18 +245,17 @@ def main():
 
     # ---- end to end through the host entry point: pinned H2D of X/types, D2H of Y inside the timing ----
     Xh = torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory()
-    th = torch.from_numpy(wl.types).pin_memory()
     Yh = torch.empty((wl.M, wl.D), dtype=torch.bfloat16).pin_memory()
     wsh = torch.empty(ffn.host_workspace_bytes(wl.M, torch.bfloat16), dtype=torch.uint8, device="cuda")
     for _ in range(3):
-        ffn.forward_host(Xh, th, Wu, Wd, Yh, workspace=wsh, stream=stream)
+        ffn.forward_host(Xh, None, Wu, Wd, Yh, workspace=wsh, stream=stream)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_ms = 0.0
     for i in range(args.steps):
         flush.zero_()
         e0.record(stream)
-        ffn.forward_host(Xh, th, Wu, Wd, Yh, workspace=wsh, stream=stream)
+        ffn.forward_host(Xh, None, Wu, Wd, Yh, workspace=wsh, stream=stream)
         e1.record(stream)
         e1.synchronize()
         e2e_ms += e0.elapsed_time(e1)
@@ -262,7 +264,7 @@ def main():
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_ms = float(tt.item())
     e2e = {"value": world * flops * args.steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
-           "h2d_bytes_per_step": int(Xh.numel() * 2 + th.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 2),
+           "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
            "ms_per_step": e2e_ms / args.steps}
 
     extras = {}
@@ -291,19 +293,26 @@ def side_measurements(binding, synth, wl, X, types, Wu, Wd, Y, flush, stream, st
     """Dense same-shape control built in the same library, and the decode-shape weight stream."""
     import torch
     out = {}
-    dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense")
-    wsd = torch.empty(dense.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for _ in range(3):
-        dense.forward(X, types, Wu, Wd, act="gelu", out=Y, workspace=wsd, stream=stream)
-    ms, n = 0.0, 20
-    for _ in range(n):
-        flush.zero_()
-        e0.record(stream)
-        dense.forward(X, types, Wu, Wd, act="gelu", out=Y, workspace=wsd, stream=stream)
-        e1.record(stream)
-        e1.synchronize()
-        ms += e0.elapsed_time(e1)
+
+    def timed(handle, tt, n=20):
+        wsx = torch.empty(handle.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            handle.forward(X, tt, Wu, Wd, act="gelu", out=Y, workspace=wsx, stream=stream)
+        tot = 0.0
+        for _ in range(n):
+            flush.zero_()
+            a0.record(stream)
+            handle.forward(X, tt, Wu, Wd, act="gelu", out=Y, workspace=wsx, stream=stream)
+            a1.record(stream)
+            a1.synchronize()
+            tot += a0.elapsed_time(a1)
+        return tot / n
+
+    out["explicit_types"] = {"ms_per_step": timed(binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16"), types),
+                             "note": "same workload through ALG_SCHED_EXPLICIT (bucketing + row gather kernels run)"}
+    dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule="cyclic")
+    ms, n = timed(dense, None) * 20, 20
     out["vs_dense"] = {"dense_ms_per_step": ms / n, "star_ms_per_step": star_ms, "time_ratio_star_over_dense": star_ms / (ms / n),
                        "control": "same library, ALG_TABLE_DENSE (8 block GEMMs instead of 6)"}
     return out

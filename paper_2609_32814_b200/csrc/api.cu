@@ -48,17 +48,6 @@ int g_trace_cap = 0;
 
 size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
-int n_col_tiles(const alg_proj_s &p, int tile_n) {
-  int n = 0;
-  for (int j = 0; j < p.q; ++j) n += ceil_div(p.r[j], tile_n);
-  return n;
-}
-
-// Upper bound on the tiles of one list: sum over pairs of ceil(M_i/tm) * ceil(r_j/tn).
-size_t max_tiles(const alg_proj_s &p, int64_t M, int tile_m, int tile_n) {
-  return (size_t)(M / tile_m + p.q + 1) * (size_t)n_col_tiles(p, tile_n);
-}
-
 bool use_tc(const alg_proj_s &p) { return p.dtype == ALG_BF16 && p.tc_ok; }
 int tile_m_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kTc2TileM : kTcTileM; }
 int tile_n_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kTc2TileN : p.tile_n; }
@@ -181,7 +170,7 @@ void free_proj(alg_proj_s &p) {
 }
 
 struct WsLayout {
-  size_t hdr = 0, chunks = 0, perm = 0, tiles0 = 0, tiles1 = 0, xb = 0, h = 0, total = 0;
+  size_t hdr = 0, chunks = 0, perm = 0, xb = 0, h = 0, total = 0;
 };
 
 // `second`: the down projection of an FFN (nullptr for a single projection).
@@ -194,12 +183,6 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
   off = align_up(off + (size_t)kMaxBucketChunks * (first.q + 1) * sizeof(int));
   L.perm = off;
   off = align_up(off + (size_t)M * sizeof(int));
-  L.tiles0 = off;
-  off = align_up(off + max_tiles(first, M, tile_m_of(first), tile_n_of(first)) * sizeof(TileRec));
-  if (second) {
-    L.tiles1 = off;
-    off = align_up(off + max_tiles(*second, M, tile_m_of(*second), tile_n_of(*second)) * sizeof(TileRec));
-  }
   if (use_tc(first)) {
     L.xb = off;
     off = align_up(off + (size_t)M * first.K * 2, 1024);
@@ -216,25 +199,18 @@ alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
-ListSpec make_list(const alg_proj_s &p, char *ws, size_t off) {
-  ListSpec ls;
-  ls.tab = p.d_tab;
-  ls.tiles = (TileRec *)(ws + off);
-  ls.tile_m = tile_m_of(p);
-  ls.tile_n = tile_n_of(p);
-  ls.split_rem = use_tc(p) && p.pair_kernel;
-  return ls;
-}
-
-alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list, const void *X, int64_t ldx,
+alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
-                      cudaEvent_t after_gather = nullptr) {
+                      cudaEvent_t after_gather = nullptr, bool cyclic = false) {
   ProjArgs a;
   a.tab = p.d_tab;
-  a.hdr = (const WsHeader *)(ws + L.hdr);
-  a.tiles = (const TileRec *)(ws + (list == 0 ? L.tiles0 : L.tiles1));
-  a.list = list;
+  a.offsets = cyclic ? nullptr : ((const WsHeader *)(ws + L.hdr))->offsets;
+  a.cyclic_rows = cyclic ? (int)(M / p.q) : 0;
+  a.n_classes = p.tab.n_classes;
+  a.geom.tile_m = tile_m_of(p);
+  a.geom.tile_n = tile_n_of(p);
+  a.geom.split_rem = use_tc(p) && p.pair_kernel;
   a.q = p.q;
   a.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
   a.W = W;
@@ -248,11 +224,12 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, int list
   a.K = p.K;
   a.N = p.N;
   a.status = p.d_status;
-  a.b_kmajor = std::getenv("ALGPROJ_BT") != nullptr;
+  a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
+  a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.trace = g_trace;
   a.trace_cap = g_trace_cap;
   if (use_tc(p)) {
-    if (x_bucketed) {
+    if (x_bucketed || cyclic) {
       a.X = X;
       a.ldx = ldx;
     } else {
@@ -336,15 +313,14 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   b.chunk_counts = (int *)(ws + L.chunks);
   b.perm = (int *)(ws + L.perm);
   b.status = h->d_status;
-  b.lists[0] = make_list(*h, ws, L.tiles0);
-  b.lists[1] = b.lists[0];
-  b.n_lists = 1;
   b.Y = Y;
   b.ldy = ldy;
   b.N = h->N;
   b.y_elem_bytes = elem_bytes(y_dtype);
-  if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
-  return run_proj(*h, L, ws, 0, X, ldx, false, W, ldw, bias, act, Y, ldy, y_dtype, false, M, st);
+  // cyclic schedule with equal buckets: no counting, no permutation, no gather
+  const bool cyc = h->sched == ALG_SCHED_CYCLIC && use_tc(*h) && M % h->q == 0;
+  if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  return run_proj(*h, L, ws, X, ldx, false, W, ldw, bias, act, Y, ldy, y_dtype, false, M, st, nullptr, cyc);
 }
 
 alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
@@ -454,23 +430,22 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   b.chunk_counts = (int *)(ws + L.chunks);
   b.perm = (int *)(ws + L.perm);
   b.status = h->up.d_status;
-  b.lists[0] = make_list(h->up, ws, L.tiles0);
-  b.lists[1] = make_list(h->down, ws, L.tiles1);
-  b.n_lists = 2;
   b.Y = Y;
   b.ldy = h->D;
   b.N = h->D;
   b.y_elem_bytes = elem_bytes(y_dtype);
   const bool tm = h->timing;
   if (tm) cudaEventRecord(h->ev[0], st);
-  if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  const bool cyc = h->up.sched == ALG_SCHED_CYCLIC && use_tc(h->up) && use_tc(h->down) && M % h->up.q == 0;
+  if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;
-  alg_status_t s = run_proj(h->up, L, ws, 0, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st,
-                            tm ? h->ev[2] : nullptr);
+  alg_status_t s = run_proj(h->up, L, ws, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st,
+                            tm ? h->ev[2] : nullptr, cyc);
   if (s != ALG_OK) return s;
   if (tm) cudaEventRecord(h->ev[3], st);
-  s = run_proj(h->down, L, ws, 1, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st);
+  s = run_proj(h->down, L, ws, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st,
+               nullptr, cyc);
   if (tm) cudaEventRecord(h->ev[4], st);
   return s;
 }

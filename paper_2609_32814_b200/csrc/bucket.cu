@@ -1,11 +1,11 @@
-// Row-type bucketing (Algorithm 1, line "I_i <- {b : tau(p_b) = i}") as a stable permutation,
-// plus the device-side tile list of the grouped GEMM.  No host synchronisation anywhere: the
-// row counts per type never leave the device.
+// Row-type bucketing (Algorithm 1, line "I_i <- {b : tau(p_b) = i}") as a stable permutation.
+// No host synchronisation anywhere: the row counts per type never leave the device (the GEMM
+// kernels turn the bucket offsets into their tile enumeration themselves).
 //
 //   kernel 1 (count):   per-chunk histograms (at most 256 chunks).
 //   kernel 2 (scatter): each CTA scans the histograms for the bucket offsets and its own bases,
 //                       then perm[offset[t] + base[t] + rank_in_chunk] = row  (stable); CTA 0
-//                       also emits the tile lists and resets the tile counters.
+//                       publishes the bucket offsets.
 //   kernel 3 (gather):  Xb[d,:] = X[perm[d],:]  -- every type becomes a contiguous M-slab.
 #include "common.cuh"
 
@@ -16,105 +16,6 @@ namespace {
 __device__ __forceinline__ int row_type(const BucketArgs &a, int row) {
   int t = a.types ? a.types[row] : (row % a.q);
   return (t < 0 || t >= a.q) ? a.q : t;  // pseudo-type q collects out-of-range rows
-}
-
-// Exclusive scan of v over the 256 threads of the CTA; returns the prefix, *total gets the sum.
-__device__ int block_exclusive_scan_256(int v, int *smem_warp /*[8]*/, int *total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += n;
-  }
-  if (lane == 31) smem_warp[warp] = incl;
-  __syncthreads();
-  int base = 0, tot = 0;
-#pragma unroll
-  for (int w = 0; w < 8; ++w) {
-    int c = smem_warp[w];
-    if (w < warp) base += c;
-    tot += c;
-  }
-  __syncthreads();
-  *total = tot;
-  return base + incl - v;
-}
-
-// Tiles of class `cls` per m-tile, and the geometry of its nt-th tile.
-__device__ __forceinline__ int class_n_tiles(const ListSpec &ls, int cls, int width) {
-  const int w = cls & 1;
-  if (!ls.split_rem) return w == 0 ? ceil_div(width, ls.tile_n) : 0;
-  return w == 0 ? width / ls.tile_n : ((width % ls.tile_n) ? 1 : 0);
-}
-
-struct EmitSmem {
-  int prefix[kMaxClasses + 1];        // tiles before class position c
-  int warp[8];
-};
-
-__device__ void emit_tile_list(const ListSpec &ls, const WsHeader *hdr, int list, WsHeader *hdr_w, EmitSmem *sm) {
-  int *s_prefix = sm->prefix;
-  int *s_warp = sm->warp;
-  const DevTable *tab = ls.tab;
-  const int q = tab->q, nc = tab->n_classes;
-  // tiles per class, in the host-chosen order (most expensive first)
-  constexpr int kPer = kMaxClasses / 256;  // 8 classes per thread
-  int local[kPer];
-  int sum = 0;
-#pragma unroll
-  for (int e = 0; e < kPer; ++e) {
-    int c = threadIdx.x * kPer + e;
-    int cnt = 0;
-    if (c < nc) {
-      int cls = tab->class_order[c];
-      int pair = cls >> 1;
-      int i = pair / q, j = pair % q;
-      int rows = hdr->offsets[i + 1] - hdr->offsets[i];
-      int width = tab->ro[j + 1] - tab->ro[j];
-      cnt = ceil_div(rows, ls.tile_m) * class_n_tiles(ls, cls, width);
-    }
-    local[e] = cnt;
-    sum += cnt;
-  }
-  int total;
-  int base = block_exclusive_scan_256(sum, s_warp, &total);
-#pragma unroll
-  for (int e = 0; e < kPer; ++e) {
-    int c = threadIdx.x * kPer + e;
-    s_prefix[c] = base;
-    base += local[e];
-  }
-  if (threadIdx.x == 255) s_prefix[kMaxClasses] = total;
-  __syncthreads();
-  for (int e = threadIdx.x; e < total; e += 256) {
-    // last class c with s_prefix[c] <= e (empty classes share a prefix with their successor)
-    int lo = 0, hi = nc;  // invariant: s_prefix[lo] <= e < s_prefix[hi] (s_prefix[nc..] == total)
-    while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if (s_prefix[mid] <= e) lo = mid; else hi = mid;
-    }
-    const int cls = tab->class_order[lo];
-    const int pair = cls >> 1;
-    const int i = pair / q, j = pair % q;
-    const int width = tab->ro[j + 1] - tab->ro[j];
-    const int n_tiles = class_n_tiles(ls, cls, width);
-    const int loc = e - s_prefix[lo];
-    const int mt = loc / n_tiles, nt = loc % n_tiles;  // n fastest: neighbours share the A rows
-    const int rows = hdr->offsets[i + 1] - hdr->offsets[i];
-    const int c0 = (cls & 1) ? (width / ls.tile_n) * ls.tile_n : nt * ls.tile_n;
-    TileRec rec;
-    rec.row0 = hdr->offsets[i] + mt * ls.tile_m;
-    rec.rows = min(ls.tile_m, rows - mt * ls.tile_m);
-    rec.pair = pair | (min(ls.tile_n, width - c0) << 16);
-    rec.n0 = tab->ro[j] + c0;
-    ls.tiles[e] = rec;
-  }
-  if (threadIdx.x == 0) {
-    hdr_w->n_tiles[list] = total;
-    hdr_w->counter[list] = 0;
-  }
-  __syncthreads();
 }
 
 // Kernel 1: per-chunk histograms of the row types (pseudo-type q = out of range).
@@ -137,13 +38,12 @@ __global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
 
 // Kernel 2: every CTA scans the (at most 256) chunk histograms to find the bucket offsets and
 // its own base inside each bucket, then places its rows (stable inside a type).  CTA 0 also
-// publishes the offsets and builds the tile lists.
+// publishes the offsets.
 __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a) {
   __shared__ int s_wcnt[8][kMaxQ + 1];
   __shared__ int s_total[kMaxQ + 1];
   __shared__ int s_base[kMaxQ + 1];     // rows of this type in earlier chunks (+ earlier sub-blocks)
   __shared__ int s_offset[kMaxQ + 2];
-  __shared__ EmitSmem s_emit;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
   const int n_chunks = gridDim.x;
@@ -205,11 +105,8 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
     __syncthreads();
   }
 
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0)
     for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
-    __syncthreads();
-    for (int l = 0; l < a.n_lists; ++l) emit_tile_list(a.lists[l], a.hdr, l, a.hdr, &s_emit);
-  }
 }
 
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ X, int64_t ldx_v,

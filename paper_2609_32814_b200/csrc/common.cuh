@@ -44,16 +44,11 @@ struct TileRec {
 // Fixed-size header at the start of every workspace.
 struct WsHeader {
   int offsets[kMaxQ + 2];  // offsets[t] = first bucketed row of type t; [q] = first bad row; [q+1] = M
-  int reserved;
-  int n_tiles[2];          // tiles in list 0 / 1
-  int counter[2];          // dynamic tile counters of list 0 / 1
-  int pad[25];
+  int pad[30];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
 
-struct ListSpec {
-  const DevTable *tab;
-  TileRec *tiles;
+struct TileGeom {
   int tile_m;
   int tile_n;
   int split_rem;  // 1: full tile_n-wide tiles plus one narrower remainder tile; 0: ceil(width / tile_n) tiles
@@ -68,8 +63,6 @@ struct BucketArgs {
   int *chunk_counts;     // [n_chunks][q+1]
   int *perm;             // [M] bucketed position -> original row
   int *status;           // device status word of the handle
-  ListSpec lists[2];
-  int n_lists;
   // rows with an out-of-range type get their output row zero-filled here
   void *Y;
   int64_t ldy;
@@ -84,9 +77,10 @@ cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int 
 
 struct ProjArgs {
   const DevTable *tab;
-  const WsHeader *hdr;
-  const TileRec *tiles;
-  int list;               // which n_tiles / counter of the header
+  const int *offsets;     // device bucket offsets [q+2]; nullptr with the cyclic schedule (equal buckets)
+  int cyclic_rows;        // M/q when offsets == nullptr
+  int n_classes;          // tab->n_classes (host copy, sizes the shared-memory tile map)
+  TileGeom geom;
   const void *X;          // SIMT: original rows (gathered through perm); tcgen05: bucketed copy
   int64_t ldx;
   const int *perm;        // output row scatter: bucketed -> original; nullptr = keep bucketed
@@ -103,7 +97,12 @@ struct ProjArgs {
   int N;
   int q;
   int *status;
-  int b_kmajor;           // experiment: B operand given as the transposed bank [N, K]
+  // Cyclic schedule (type of row b = b mod q, M a multiple of q) needs no permutation: rows of
+  // type i are rows i, i+q, ... .  a_cyclic_rows = M/q makes the A operand a type-strided view of
+  // the original X (3-D tensor map); out_cyclic_rows = M/q makes the epilogue compute
+  // original row = (bucketed row - i*M/q)*q + i.  0 = off.
+  int a_cyclic_rows;
+  int out_cyclic_rows;
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;
 };

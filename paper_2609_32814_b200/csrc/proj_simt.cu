@@ -2,7 +2,7 @@
 // tile of one (row type i, output group j) pair and sums every kept product x_k W_kj
 // (k in B(i,j), Eq. recursive-row-action) in registers before the single store.
 // Serves the fp32 problems and bf16 shapes the tensor-core path does not cover.
-#include "common.cuh"
+#include "tile_map.cuh"
 
 namespace algproj {
 
@@ -27,16 +27,19 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
   __shared__ float As[TK][TM + 1];
   __shared__ float Bs[TK][TN];
   __shared__ int s_rows[TM];
+  __shared__ __align__(16) unsigned char s_map[sizeof(TileMap) + (2 * kMaxClasses + 1) * sizeof(int)];
+  TileMap *tm = reinterpret_cast<TileMap *>(s_map);
   const DevTable *__restrict__ tab = a.tab;
   const int q = tab->q;
-  const int n_tiles = a.hdr->n_tiles[a.list];
+  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  const int n_tiles = tm->total;
   const T *__restrict__ X = (const T *)a.X;
   const T *__restrict__ W = (const T *)a.W;
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;  // 16 x 16 threads, 4 x 4 outputs each
 
   for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    TileRec rec = a.tiles[tile];
+    TileRec rec = tile_map_decode(tm, a.geom, tile);
     rec.pair &= 0xFFFF;
     const int j = rec.pair % q;
     const int n_valid = min(TN, tab->ro[j + 1] - rec.n0);

@@ -61,6 +61,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctl *ctl
   return wait_slow(bar, parity, ctl, status);
 }
 
+constexpr int kSeqCap = 224;  // precomputed tile records per CTA
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 
@@ -73,7 +74,7 @@ struct Cfg {
   static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
   static constexpr int kAccStride = TILE_N <= 128 ? 128 : 256;   // TMEM columns between the two accumulators
   static constexpr int kTmemCols = 2 * kAccStride;
-  static constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + 1024;
+  static constexpr int kFixedSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + kSeqCap * 16 + 16 + 1024;  // + tile map
   static constexpr int kHalf = TILE_N / 2;                        // columns per epilogue warp
   // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N, M=128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
@@ -87,11 +88,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Ctl *ctl = (Ctl *)(smem + C::kStages * C::kStageBytes);
+  TileRec *recs = (TileRec *)(ctl + 1);
+  TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
   const int q = tab->q;
-  const int n_tiles = a.hdr->n_tiles[a.list];
-  int tr_n = 0;
+  [[maybe_unused]] int tr_n = 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -115,6 +117,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x, gridDim.x);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -126,10 +130,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0, round = 0;
       uint32_t phase = 0;
       bool ok = true;
-      TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x, gridDim.x), n_tiles);
+      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
       while (ok && rec.row0 >= 0) {
         ++round;
-        const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x, gridDim.x), n_tiles);  // lands while we issue
         ALG_TRACE(0, 1);
         const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
         for (int k = 0; k < q && ok; ++k) {
@@ -141,7 +144,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t bar = smem_u32(&ctl->full[stage]);
             const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
             mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
-            tma_load_2d(sa, &tmA, bar, k0, rec.row0);
+            if (a.a_cyclic_rows) {
+              const int i = (rec.pair & 0xFFFF) / q;
+              tma_load_3d(sa, &tmA, bar, k0, i, rec.row0 - i * a.a_cyclic_rows);
+            } else {
+              tma_load_2d(sa, &tmA, bar, k0, rec.row0);
+            }
 #pragma unroll
             for (int c = 0; c < TILE_N / 64; ++c)
               tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, rec.n0 + c * 64, k0);
@@ -149,7 +157,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         ALG_TRACE(0, 2);
-        rec = next;
+        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
       }
     }
   } else if (warp == 1) {
@@ -158,10 +166,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0, acc = 0, round = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x, gridDim.x), n_tiles);
+      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
       while (ok && rec.row0 >= 0) {
         ++round;
-        const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x, gridDim.x), n_tiles);
         ALG_TRACE(1, 1);
         ok = wait_bar(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, ctl, a.status);
         if (!ok) break;
@@ -195,7 +202,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_commit(smem_u32(&ctl->tmem_full[acc]));
         ALG_TRACE(1, 4);
         if (++acc == 2) acc = 0, acc_phase ^= 1u;
-        rec = next;
+        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
       }
     }
   } else {
@@ -205,13 +212,19 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = e >> 2;
     int acc = 0, round = 0;
     uint32_t acc_phase = 0;
-    TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x, gridDim.x), n_tiles);
+    TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
     while (rec.row0 >= 0) {
       ++round;
-      const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x, gridDim.x), n_tiles);
       const int r = quad * 32 + lane;
       int64_t out_row = -1;
-      if (r < rec.rows) out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
+      if (r < rec.rows) {
+        if (a.out_cyclic_rows) {
+          const int i = (rec.pair & 0xFFFF) / q;
+          out_row = (int64_t)(rec.row0 + r - i * a.out_cyclic_rows) * q + i;
+        } else {
+          out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
+        }
+      }
       bool ok = wait_bar(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -237,7 +250,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
       if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
-      rec = next;
+      rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
     }
   }
 
@@ -265,16 +278,18 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   using C = Cfg<TILE_N>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  const int smem_bytes = C::kFixedSmemBytes + (int)tile_map_bytes(a.n_classes);
+  if (smem_bytes > 227 * 1024) return cudaErrorInvalidConfiguration;
   CUtensorMap tmA, tmB;
-  cudaError_t e = make_map_2d(&tmA, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, kTcTileM);
+  cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
   e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
   if (e != cudaSuccess) return e;
-  proj_tc_kernel<TILE_N><<<num_sms, kThreads, C::kSmemBytes, st>>>(tmA, tmB, a);
+  proj_tc_kernel<TILE_N><<<num_sms, kThreads, smem_bytes, st>>>(tmA, tmB, a);
   count_launch(1);
   return cudaGetLastError();
 }
@@ -289,6 +304,19 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a) {
+  if (!a.a_cyclic_rows)
+    return make_map_2d(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, kTcTileM);
+  cuuint64_t dims[3] = {(cuuint64_t)a.K, (cuuint64_t)a.q, (cuuint64_t)a.a_cyclic_rows};
+  cuuint64_t strides[2] = {(cuuint64_t)a.ldx * 2, (cuuint64_t)a.ldx * 2 * (cuuint64_t)a.q};
+  cuuint32_t box[3] = {kTcBlockK, 1, kTcTileM};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;

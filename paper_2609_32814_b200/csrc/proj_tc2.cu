@@ -32,6 +32,7 @@ constexpr int kEpiWarps = 8;
 constexpr int kProducerWarpB = 2 + kEpiWarps;   // second TMA producer, after the epilogue warps
 constexpr int kThreads = 32 * (3 + kEpiWarps);
 constexpr int kMaxStages = 7;
+constexpr int kSeqCap = 48;   // precomputed tile records per CTA pair
 constexpr int kABytes = 128 * kTcBlockK * 2;              // 16 KB: this CTA's rows
 constexpr int kBChunkBytes = kTcBlockK * 64 * 2;           // one 64(k) x 64(n) box
 constexpr int kBMaxBytes = kBChunkBytes * (kTc2TileN / 128);  // this CTA's half of the B block: 16 KB
@@ -51,8 +52,13 @@ struct Ctl2 {
   uint32_t keep[1];  // q*q entries follow (the shared-memory request is sized for them)
 };
 constexpr int kMaxSmem = 227 * 1024;
-inline int smem_bytes(int n_stages, int q) { return n_stages * kStageBytes + (int)sizeof(Ctl2) + q * q * 4 + 1024; }
-inline int pick_stages(int q) { return smem_bytes(kMaxStages, q) <= kMaxSmem ? kMaxStages : kMaxStages - 1; }
+inline int smem_bytes(int n_stages, int q, int n_classes) {
+  return n_stages * kStageBytes + (int)sizeof(Ctl2) + q * q * 4 + kSeqCap * 16 + (int)tile_map_bytes(n_classes) + 32 +
+         1024;
+}
+inline int pick_stages(int q, int n_classes) {
+  return smem_bytes(kMaxStages, q, n_classes) <= kMaxSmem ? kMaxStages : kMaxStages - 1;
+}
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -76,6 +82,14 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
           dst),
       "l"(map), "r"(leader_bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0,
+                                                 int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+          dst),
+      "l"(map), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
 __device__ __forceinline__ void tc2_commit_both(uint32_t bar) {
@@ -119,13 +133,15 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int n_stages) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int tab_q = a.q;
   Ctl2 *ctl = (Ctl2 *)(smem + n_stages * kStageBytes);
+  TileRec *recs = (TileRec *)(((uintptr_t)(ctl->keep + tab_q * tab_q) + 15) & ~(uintptr_t)15);
+  TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
-  const int q = tab->q;
+  const int q = tab_q;
   const uint32_t rank = cluster_ctarank();          // 0 = leader
-  const int n_tiles = a.hdr->n_tiles[a.list];
-  int tr_n = 0;
+  [[maybe_unused]] int tr_n = 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -149,6 +165,8 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x >> 1, gridDim.x >> 1);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // the peer's barriers are initialised before anything signals them
@@ -166,10 +184,9 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0, round = 0;
       uint32_t phase = 0;
       bool ok = true;
-      TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
+      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
       while (ok && rec.row0 >= 0) {
         ++round;
-        const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
         if (loads_a) ALG_TRACE(0, 1);
         const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
         const int half_cols = (rec.pair >> 16) >> 1;         // B columns this CTA loads: 128 or 64
@@ -188,9 +205,12 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t bar = own_bar & kPeerMask;
             if (loads_a) {
               if (rank == 0) mbar_expect_tx(own_bar, tx_bytes);
-              tma_load_2d_pair(sa, &tmA, bar, k0, row);
-            } else if (a.b_kmajor) {
-              tma_load_2d_pair(sa + kABytes, &tmB, bar, k0, col);   // one box: half_cols rows of 64 k
+              if (a.a_cyclic_rows) {
+                const int i = (rec.pair & 0xFFFF) / q;
+                tma_load_3d_pair(sa, &tmA, bar, k0, i, row - i * a.a_cyclic_rows);
+              } else {
+                tma_load_2d_pair(sa, &tmA, bar, k0, row);
+              }
             } else {
               for (int c = 0; c < n_chunks; ++c)
                 tma_load_2d_pair(sa + kABytes + c * kBChunkBytes, &tmB, bar, col + c * 64, k0);
@@ -199,7 +219,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
         if (loads_a) ALG_TRACE(0, 2);
-        rec = next;
+        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
       }
     }
   } else if (warp == 1) {
@@ -208,10 +228,9 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0, acc = 0, round = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
+      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
       while (ok && rec.row0 >= 0) {
         ++round;
-        const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
         ALG_TRACE(1, 1);
         ok = wait_bar2(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, ctl, a.status);
         if (!ok) break;
@@ -221,7 +240,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
         const int cols = rec.pair >> 16;
         // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N = cols, M = 256
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | ((a.b_kmajor ? 0u : 1u) << 16) |
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                ((uint32_t)(cols >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
         uint32_t accumulate = 0;
         for (int k = 0; k < q && ok; ++k) {
@@ -234,12 +253,10 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             tc_fence_after();
             const uint32_t sa = smem_u32(smem + stage * kStageBytes);
             const uint64_t da = make_smem_desc(sa, 16, 1024);
-            const uint64_t db = a.b_kmajor ? make_smem_desc(sa + kABytes, 16, 1024)
-                                           : make_smem_desc(sa + kABytes, kBChunkBytes, 1024);
-            const uint64_t db_step = a.b_kmajor ? 2 : 128;
+            const uint64_t db = make_smem_desc(sa + kABytes, kBChunkBytes, 1024);
 #pragma unroll
             for (int kk = 0; kk < kTcBlockK / 16; ++kk) {
-              tc2_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)kk * db_step, idesc, accumulate);
+              tc2_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc, accumulate);
               accumulate = 1;
             }
             tc2_commit_both(smem_u32(&ctl->empty[stage]));
@@ -250,7 +267,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tc2_commit_both(smem_u32(&ctl->tmem_full[acc]));
         ALG_TRACE(1, 4);
         if (++acc == 2) acc = 0, acc_phase ^= 1u;
-        rec = next;
+        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
       }
     }
   } else {
@@ -260,15 +277,21 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int half = e >> 2;
     int acc = 0, round = 0;
     uint32_t acc_phase = 0;
-    TileRec rec = load_tile(a.tiles, snake_tile(0, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
+    TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
     while (rec.row0 >= 0) {
       ++round;
-      const TileRec next = load_tile(a.tiles, snake_tile(round, blockIdx.x >> 1, gridDim.x >> 1), n_tiles);
       const int cols = rec.pair >> 16;
       const int half_cols = cols >> 1;
       const int r = 128 * (int)rank + quad * 32 + lane;   // row inside the 256-row tile
       int64_t out_row = -1;
-      if (r < rec.rows) out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
+      if (r < rec.rows) {
+        if (a.out_cyclic_rows) {
+          const int i = (rec.pair & 0xFFFF) / q;
+          out_row = (int64_t)(rec.row0 + r - i * a.out_cyclic_rows) * q + i;
+        } else {
+          out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
+        }
+      }
       bool ok = wait_bar2(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -297,7 +320,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
-      rec = next;
+      rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
     }
   }
 
@@ -328,7 +351,7 @@ int tc2_max_pairs(int num_sms) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (num_sms / 2));
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem_bytes(kMaxStages - 1, kMaxQ);
+  cfg.dynamicSmemBytes = smem_bytes(kMaxStages - 1, kMaxQ, kMaxClasses);
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, proj_tc2_kernel, &cfg) != cudaSuccess || n < 1) return 0;
   max_pairs = n < num_sms / 2 ? n : num_sms / 2;
@@ -342,16 +365,14 @@ cudaError_t launch_proj_tc2(const ProjArgs &a, int num_sms, cudaStream_t st) {
   const int pairs = tc2_max_pairs(num_sms);
   if (pairs < 1) return cudaErrorInvalidConfiguration;
   const int q = a.q;
-  const int n_stages = pick_stages(q);
+  const int n_stages = pick_stages(q, a.n_classes);
+  if (smem_bytes(n_stages, q, a.n_classes) > kMaxSmem) return cudaErrorInvalidConfiguration;
   CUtensorMap tmA, tmB;
-  e = make_map_2d(&tmA, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, 128);
+  e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
-  if (a.b_kmajor)  // experiment: W holds the transposed bank [N, K]
-    e = make_map_2d(&tmB, a.W, (uint64_t)a.K, (uint64_t)a.N, (uint64_t)a.K * 2, kTcBlockK, 128);
-  else
-    e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
+  e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
   if (e != cudaSuccess) return e;
-  proj_tc2_kernel<<<2 * pairs, kThreads, smem_bytes(n_stages, q), st>>>(tmA, tmB, a, n_stages);
+  proj_tc2_kernel<<<2 * pairs, kThreads, smem_bytes(n_stages, q, a.n_classes), st>>>(tmA, tmB, a, n_stages);
   count_launch(1);
   return cudaGetLastError();
 }

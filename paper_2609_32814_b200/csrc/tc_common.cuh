@@ -3,7 +3,7 @@
 
 #include <cuda.h>
 
-#include "common.cuh"
+#include "tile_map.cuh"
 
 namespace algproj {
 namespace tc {
@@ -37,6 +37,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
       "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+          dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -78,49 +85,40 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
   return d;
 }
 
-// GELU with the exact (erf) definition, gelu(z) = z * Phi(z).  The lower tail Phi(-u), u >= 0, is
-// evaluated as 2^q(u) with a degree-6 polynomial q fitted to log2(Phi(-u)) on [0, 6] (one ex2 and
-// six FMAs, no branches); |gelu error| < 1e-7 over the whole real line, i.e. fp32 rounding level.
-__device__ __forceinline__ float gelu_erf(float z) {
-  const float u = fminf(fabsf(z), 6.0f);
-  float q = 3.3093889e-05f;
-  q = fmaf(q, u, -7.6922908e-04f);
-  q = fmaf(q, u, 8.0807470e-03f);
-  q = fmaf(q, u, -5.3412151e-02f);
-  q = fmaf(q, u, -4.5877093e-01f);
-  q = fmaf(q, u, -1.1512017f);
-  q = fmaf(q, u, -0.99999309f);
-  float t;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(q));
-  return z * (z < 0.f ? t : 1.0f - t);
+// GELU with the exact (erf) definition, gelu(z) = z * Phi(z) = max(z, 0) - |z| * Phi(-|z|).  The
+// lower tail Phi(-u), u >= 0, is evaluated as 2^p(u) with a degree-6 polynomial p fitted to
+// log2(Phi(-u)) on [0, 6] (one ex2, no branches); |gelu error| < 1e-7 over the whole real line,
+// i.e. fp32 rounding level.  Two values are processed at once with the packed fp32x2 FMA of
+// sm_100, which halves the issue slots the epilogue takes from the producer and MMA threads.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ void gelu_erf2(float &z0, float &z1) {
+  const float u0 = fminf(fabsf(z0), 6.0f), u1 = fminf(fabsf(z1), 6.0f);
+  const uint64_t u = pack2(u0, u1);
+  uint64_t p = pack2(3.3093889e-05f, 3.3093889e-05f);
+  p = fma2(p, u, pack2(-7.6922908e-04f, -7.6922908e-04f));
+  p = fma2(p, u, pack2(8.0807470e-03f, 8.0807470e-03f));
+  p = fma2(p, u, pack2(-5.3412151e-02f, -5.3412151e-02f));
+  p = fma2(p, u, pack2(-4.5877093e-01f, -4.5877093e-01f));
+  p = fma2(p, u, pack2(-1.1512017f, -1.1512017f));
+  p = fma2(p, u, pack2(-0.99999309f, -0.99999309f));
+  float t0, t1;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(__uint_as_float((uint32_t)p)));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(__uint_as_float((uint32_t)(p >> 32))));
+  z0 = fmaf(-fabsf(z0), t0, fmaxf(z0, 0.0f));
+  z1 = fmaf(-fabsf(z1), t1, fmaxf(z1, 0.0f));
 }
 __device__ __forceinline__ float gelu_tanh(float z) {
   float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
   return 0.5f * z * (1.0f + tanhf(u));
 }
 
-
-// Static schedule: the tile list is sorted most-expensive first; worker c of n takes, in round r,
-// tile r*n + c on even rounds and r*n + (n-1-c) on odd rounds (boustrophedon).  That balances the
-// per-worker cost like a longest-processing-time assignment without inter-CTA traffic, and keeps
-// the workers of one round on neighbouring tiles (same rows or same columns), so the lines one CTA
-// pulls into L2 are the lines its neighbours ask for at the same moment.  (Giving each worker a
-// contiguous run of tiles instead was measured 10-15 % slower: the concurrent working set spreads
-// over the whole problem.)
-__device__ __forceinline__ int snake_tile(int round, int worker, int n_workers) {
-  return round * n_workers + ((round & 1) ? (n_workers - 1 - worker) : worker);
-}
-
-__device__ __forceinline__ TileRec load_tile(const TileRec *tiles, int idx, int end) {
-  TileRec rec;
-  if (idx < end) {
-    const int4 v = __ldg((const int4 *)(tiles + idx));
-    rec.row0 = v.x, rec.rows = v.y, rec.pair = v.z, rec.n0 = v.w;
-  } else {
-    rec.row0 = -1, rec.rows = 0, rec.pair = 0, rec.n0 = 0;
-  }
-  return rec;
-}
 
 // Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
 // it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
@@ -132,7 +130,7 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
   }
   if (a.act == ALG_ACT_GELU_ERF) {
 #pragma unroll
-    for (int x = 0; x < 32; ++x) f[x] = gelu_erf(f[x]);
+    for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
   } else if (a.act == ALG_ACT_GELU_TANH) {
 #pragma unroll
     for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
@@ -174,15 +172,24 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
   }
 }
 
+#ifdef ALGPROJ_TRACE
 #define ALG_TRACE(role, tag)                                                                        \
   do {                                                                                              \
     if (a.trace && blockIdx.x < 8 && tr_n < a.trace_cap)                                            \
       a.trace[((size_t)blockIdx.x * 3 + (role)) * a.trace_cap + tr_n++] = (clock64() << 8) | (tag); \
   } while (0)
+#else
+#define ALG_TRACE(role, tag) \
+  do {                       \
+  } while (0)
+#endif
 
 // Host side: tensor-map encoding through the driver entry point (no link-time libcuda dependency).
 cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,
                         uint32_t box_inner, uint32_t box_outer);
+// A operand of either kind: plain rows (2-D) or, for the cyclic schedule, the type-strided view
+// {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
+cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);
 
 }  // namespace tc
 }  // namespace algproj
