@@ -3,9 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-One step = one pass of the whole hot path (row-type bucketing, row gather, grouped tcgen05 GEMM
-with fused GELU for the up projection, grouped GEMM with fused row scatter for the down
-projection) over one synthetic batch of the q=2, 768 -> 3072 -> 768, M = 8 x 1024 workload.
+One step = one pass of the whole hot path (grouped tcgen05 GEMM with fused GELU for the up
+projection, grouped GEMM with fused row scatter for the down projection; with explicit row types
+also the bucketing and row-gather kernels) over one synthetic batch of the q=2,
+768 -> 3072 -> 768, M = 8 x 1024 workload.
 Prints ONE JSON line.  FLOPs count only the block GEMMs the rule keeps.
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
@@ -33,10 +34,10 @@ import numpy as np
 WORKLOAD = "cfg2: q=2 FFN 768->3072->768 (GELU), M=8x1024 rows, type = position mod 2, bf16"
 METRIC = "star_q FFN kept-GEMM throughput (prefill)"
 UNIT = "TFLOP/s"
-FLUSH_BYTES = 512 << 20
+N_SETS = 6
 # DRAM traffic of the grouped-GEMM kernels from the ncu capture summarised under profiles/
-# (bytes per launch, up and down projection of this workload); None until captured.
-NCU_TRAFFIC_BYTES = None
+# (bytes of the up launch + the down launch of one step of this workload).
+NCU_TRAFFIC_BYTES = 20.0e6 + 56.8e6  # up + down launch, cold caches (profiles/proj_tc_kernel_cfg2.md)
 
 
 def _peaks():
@@ -49,21 +50,40 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons (NVML, read-only) while the timed region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int):
         self.index, self.samples, self._stop, self._t = index, [], threading.Event(), None
+        self.max_mhz = None
 
     def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                mhz = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+                mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                self.samples.append((float(mhz), int(mask)))
+                self._stop.wait(0.002)
+        except Exception:
+            self._run_smi()
+
+    def _run_smi(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        bits = [0x8, 0x40, 0x20, 0x4]
         while not self._stop.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-i",
+                                      str(self.index)], capture_output=True, text=True, timeout=5).stdout
                 parts = [p.strip() for p in out.strip().split(",")]
                 if len(parts) >= 6:
-                    self.samples.append(parts)
+                    self.max_mhz = float(parts[1])
+                    mask = sum(b for b, v in zip(bits, parts[2:6]) if v.lower().startswith("active"))
+                    self.samples.append((float(parts[0]), mask))
             except Exception:
                 pass
             self._stop.wait(0.05)
@@ -71,6 +91,7 @@ class ClockSampler:
     def __enter__(self):
         self._t = threading.Thread(target=self._run, daemon=True)
         self._t.start()
+        time.sleep(0.02)
         return self
 
     def __exit__(self, *a):
@@ -78,12 +99,12 @@ class ClockSampler:
         self._t.join(timeout=10)
 
     def summary(self):
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.samples)}
+        sm = [s[0] for s in self.samples]
+        mask = 0
+        for s in self.samples:
+            mask |= s[1]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in self.REASONS.items() if mask & b], "samples": len(self.samples)}
 
 
 def kept_flops(ffn, wl) -> int:
@@ -147,8 +168,8 @@ def time_cpu_oracle(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=600)
+    ap.add_argument("--warmup", type=int, default=12)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-control / decode side measurements")
     args = ap.parse_args()
@@ -172,54 +193,61 @@ def main():
     binding.lib()  # fail loudly if the CUDA library is missing
 
     wl = synth.config2()
-    if world > 1:  # each rank draws its own batch of the same shape
-        wl.X = synth.bf16_round(synth.normal(synth.seed_for(2, 50 + rank), wl.X.shape, 1.0))
     dev = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)
-    X, Wu, Wd = dev(wl.X), dev(wl.W_up), dev(wl.W_down)
-    types = torch.from_numpy(wl.types).cuda()
     # config 2 fixes the schedule "type = position mod 2": the handle is created with it
     # (ALG_SCHED_CYCLIC), the per-call types array is then not needed.  The explicit-types path of
     # the same workload is timed as a side measurement.
     ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
-    ws = torch.empty(ffn.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
-    Y = torch.empty((wl.M, wl.D), dtype=torch.bfloat16, device="cuda")
     flops = kept_flops(ffn, wl)
-    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
+    types = torch.from_numpy(wl.types).cuda()
 
-    def step():
-        ffn.forward(X, None, Wu, Wd, act="gelu", out=Y, workspace=ws, stream=stream)
+    # ---- working sets: N_SETS independent copies of (X, W_up, W_down, Y, workspace), ~85 MB each,
+    # used round-robin, so every step reads inputs and weights that have left the 126 MB L2 since
+    # their last use (no explicit flush: a write-flush would leave L2 full of dirty lines whose
+    # write-back the next step then pays for).
+    ws_bytes = ffn.workspace_bytes(wl.M)
+    sets = []
+    for r in range(N_SETS):
+        Xr = synth.bf16_round(synth.normal(synth.seed_for(2, 50 + rank * N_SETS + r), wl.X.shape, 1.0)) if (r or world > 1) else wl.X
+        sets.append({"X": dev(Xr), "Wu": dev(wl.W_up).clone(), "Wd": dev(wl.W_down).clone(),
+                     "Y": torch.empty((wl.M, wl.D), dtype=torch.bfloat16, device="cuda"),
+                     "ws": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")})
+    footprint_mb = N_SETS * (2 * wl.M * wl.D * 2 + 2 * wl.D * wl.F * 2 + ws_bytes) / 1e6
+
+    def step(i, handle=None, tt=None):
+        s_ = sets[i % N_SETS]
+        (handle or ffn).forward(s_["X"], tt, s_["Wu"], s_["Wd"], act="gelu", out=s_["Y"], workspace=s_["ws"], stream=stream)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        flush.zero_()
-        step()
+    def time_steps(n, handle=None, tt=None, first=0):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(n):
+            step(first + i, handle, tt)
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    for i in range(args.warmup):
+        step(i)
     barrier()
     assert ffn.last_status() == 0
 
-    # ---- timed region: K steps, L2 flushed (512 MiB write) before each, CUDA events per step ----
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    # ---- timed region: exactly K steps between two events, barrier + synchronize on both sides ----
     launches0 = binding.launch_count()
     with ClockSampler(local_rank) as clocks:
-        barrier()
-        for i in range(args.steps):
-            flush.zero_()
-            starts[i].record(stream)
-            step()
-            stops[i].record(stream)
-        barrier()
+        total_ms = time_steps(args.steps, first=args.warmup)
     launches = binding.launch_count() - launches0
-    per_step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
-    total_ms = float(sum(per_step_ms))
     if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+        tt_ = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt_, op=dist.ReduceOp.MAX)
+        total_ms = float(tt_.item())
     ms_per_step = total_ms / args.steps
     value = world * flops * args.steps / (total_ms * 1e-3) / 1e12
     assert ffn.last_status() == 0
@@ -228,8 +256,7 @@ def main():
     ffn.set_timing(True)
     kt = np.zeros(4)
     for i in range(args.steps):
-        flush.zero_()
-        step()
+        step(i)
         kt += np.array(ffn.get_timing())
     kt /= args.steps
     ffn.set_timing(False)
@@ -243,40 +270,39 @@ def main():
                 "kernel_ms": {"bucket": float(kt[0]), "gather": float(kt[1]), "up": float(kt[2]), "down": float(kt[3])},
                 "step_frac_of_peak": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
 
-    # ---- end to end through the host entry point: pinned H2D of X/types, D2H of Y inside the timing ----
+    # ---- end to end through the host entry point: pinned H2D of X, D2H of Y inside the timing ----
     Xh = torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory()
     Yh = torch.empty((wl.M, wl.D), dtype=torch.bfloat16).pin_memory()
     wsh = torch.empty(ffn.host_workspace_bytes(wl.M, torch.bfloat16), dtype=torch.uint8, device="cuda")
-    for _ in range(3):
-        ffn.forward_host(Xh, None, Wu, Wd, Yh, workspace=wsh, stream=stream)
+    for i in range(3):
+        ffn.forward_host(Xh, None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], Yh, workspace=wsh, stream=stream)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2e_ms = 0.0
+    e0.record(stream)
     for i in range(args.steps):
-        flush.zero_()
-        e0.record(stream)
-        ffn.forward_host(Xh, None, Wu, Wd, Yh, workspace=wsh, stream=stream)
-        e1.record(stream)
-        e1.synchronize()
-        e2e_ms += e0.elapsed_time(e1)
+        ffn.forward_host(Xh, None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], Yh, workspace=wsh, stream=stream)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
     if world > 1:
-        tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
+        tt_ = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt_, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt_.item())
     e2e = {"value": world * flops * args.steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
            "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
            "ms_per_step": e2e_ms / args.steps}
 
     extras = {}
     if rank == 0 and not args.no_extras:
-        extras = side_measurements(binding, synth, wl, X, types, Wu, Wd, Y, flush, stream, ms_per_step)
+        extras = side_measurements(binding, wl, types, time_steps, ms_per_step)
 
     if rank == 0:
         cpu = time_cpu_oracle(wl) if world >= 1 else None
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "l2": "flushed before every step (512 MiB write, outside the timing)",
+                "config": {"workload": WORKLOAD, "l2": f"{N_SETS} working sets of inputs, weights, outputs and workspace used round-robin "
+                                 f"({footprint_mb:.0f} MB in total, L2 is 126 MB); no data is reused within 5 steps",
                            "rows_per_gpu": wl.M, "parallelism": f"rows sharded over {world} GPU(s), weights replicated"},
                 "tokens_per_s": world * wl.M * args.steps / (total_ms * 1e-3),
                 "kept_gflop_per_step": flops / 1e9,
@@ -289,31 +315,19 @@ def main():
         dist.destroy_process_group()
 
 
-def side_measurements(binding, synth, wl, X, types, Wu, Wd, Y, flush, stream, star_ms):
-    """Dense same-shape control built in the same library, and the decode-shape weight stream."""
-    import torch
+def side_measurements(binding, wl, types, time_steps, star_ms):
+    """The same workload through the explicit-types path, and the dense same-shape control."""
     out = {}
-
-    def timed(handle, tt, n=20):
-        wsx = torch.empty(handle.workspace_bytes(wl.M), dtype=torch.uint8, device="cuda")
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for _ in range(3):
-            handle.forward(X, tt, Wu, Wd, act="gelu", out=Y, workspace=wsx, stream=stream)
-        tot = 0.0
-        for _ in range(n):
-            flush.zero_()
-            a0.record(stream)
-            handle.forward(X, tt, Wu, Wd, act="gelu", out=Y, workspace=wsx, stream=stream)
-            a1.record(stream)
-            a1.synchronize()
-            tot += a0.elapsed_time(a1)
-        return tot / n
-
-    out["explicit_types"] = {"ms_per_step": timed(binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16"), types),
+    n = 24
+    explicit = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    time_steps(6, explicit, types)
+    out["explicit_types"] = {"ms_per_step": time_steps(n, explicit, types) / n,
                              "note": "same workload through ALG_SCHED_EXPLICIT (bucketing + row gather kernels run)"}
     dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule="cyclic")
-    ms, n = timed(dense, None) * 20, 20
-    out["vs_dense"] = {"dense_ms_per_step": ms / n, "star_ms_per_step": star_ms, "time_ratio_star_over_dense": star_ms / (ms / n),
+    time_steps(6, dense)
+    dense_ms = time_steps(n, dense) / n
+    out["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms,
+                       "time_ratio_star_over_dense": star_ms / dense_ms,
                        "control": "same library, ALG_TABLE_DENSE (8 block GEMMs instead of 6)"}
     return out
 

@@ -226,6 +226,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.status = p.d_status;
   a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
+  a.b_3d = 0;
   a.trace = g_trace;
   a.trace_cap = g_trace_cap;
   if (use_tc(p)) {

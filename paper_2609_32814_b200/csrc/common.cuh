@@ -103,6 +103,7 @@ struct ProjArgs {
   // original row = (bucketed row - i*M/q)*q + i.  0 = off.
   int a_cyclic_rows;
   int out_cyclic_rows;
+  int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;
 };

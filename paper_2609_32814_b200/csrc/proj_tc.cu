@@ -20,6 +20,8 @@
 // handle's status word, all roles leave their loops, TMEM is released and the kernel returns.
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
+
 #include "tc_common.cuh"
 
 namespace algproj {
@@ -62,8 +64,12 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctl *ctl
 }
 
 constexpr int kSeqCap = 224;  // precomputed tile records per CTA
-constexpr int kEpiWarps = 8;
-constexpr int kThreads = 32 * (2 + kEpiWarps);
+#ifndef ALGPROJ_EPI_WARPS
+#define ALGPROJ_EPI_WARPS 8
+#endif
+constexpr int kEpiWarps = ALGPROJ_EPI_WARPS;
+constexpr int kProducerWarpB = 2 + kEpiWarps;   // second TMA producer, after the epilogue warps
+constexpr int kThreads = 32 * (3 + kEpiWarps);
 
 template <int TILE_N>
 struct Cfg {
@@ -75,7 +81,7 @@ struct Cfg {
   static constexpr int kAccStride = TILE_N <= 128 ? 128 : 256;   // TMEM columns between the two accumulators
   static constexpr int kTmemCols = 2 * kAccStride;
   static constexpr int kFixedSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + kSeqCap * 16 + 16 + 1024;  // + tile map
-  static constexpr int kHalf = TILE_N / 2;                        // columns per epilogue warp
+  static constexpr int kHalf = TILE_N / (kEpiWarps / 4);          // columns per epilogue warp
   // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N, M=128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                      ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
@@ -124,17 +130,23 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
 
-  if (warp == 0) {
-    // ---------------- TMA producer (one lane) ----------------
+  if (warp == 0 || warp == kProducerWarpB) {
+    // ---------------- TMA producers (one lane each): warp 0 loads A, the last warp loads B ----------------
+    // Issuing a tiled load occupies the thread while the copy engine expands the box; with two
+    // issuing threads a freed stage is refilled sooner, which shortens the
+    // load -> MMA -> free -> load round trip that bounds the bytes in flight.
     if (lane == 0) {
+      const bool loads_a = warp == 0;
       int stage = 0, round = 0;
       uint32_t phase = 0;
       bool ok = true;
       TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
       while (ok && rec.row0 >= 0) {
         ++round;
-        ALG_TRACE(0, 1);
+        if (loads_a) ALG_TRACE(0, 1);
         const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
+        const int type_i = (rec.pair & 0xFFFF) / q;
+        const int a_row = a.a_cyclic_rows ? rec.row0 - type_i * a.a_cyclic_rows : rec.row0;
         for (int k = 0; k < q && ok; ++k) {
           if (!((mask >> k) & 1u)) continue;
           const int k_end = ctl->so[k + 1];
@@ -143,20 +155,21 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!ok) break;
             const uint32_t bar = smem_u32(&ctl->full[stage]);
             const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
-            mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
-            if (a.a_cyclic_rows) {
-              const int i = (rec.pair & 0xFFFF) / q;
-              tma_load_3d(sa, &tmA, bar, k0, i, rec.row0 - i * a.a_cyclic_rows);
+            if (loads_a) {
+              mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+              if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
+              else tma_load_2d(sa, &tmA, bar, k0, a_row);
+            } else if (a.b_3d) {
+              tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, rec.n0 >> 6);  // all 64-column chunks in one box
             } else {
-              tma_load_2d(sa, &tmA, bar, k0, rec.row0);
-            }
 #pragma unroll
-            for (int c = 0; c < TILE_N / 64; ++c)
-              tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, rec.n0 + c * 64, k0);
+              for (int c = 0; c < TILE_N / 64; ++c)
+                tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, rec.n0 + c * 64, k0);
+            }
             if (++stage == C::kStages) stage = 0, phase ^= 1u;
           }
         }
-        ALG_TRACE(0, 2);
+        if (loads_a) ALG_TRACE(0, 2);
         rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
       }
     }
@@ -287,9 +300,13 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   CUtensorMap tmA, tmB;
   cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
-  e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
-  if (e != cudaSuccess) return e;
-  proj_tc_kernel<TILE_N><<<num_sms, kThreads, smem_bytes, st>>>(tmA, tmB, a);
+  ProjArgs b = a;
+  b.b_3d = make_map_b3d(&tmB, a, TILE_N / 64) == cudaSuccess;
+  if (!b.b_3d) {
+    e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
+    if (e != cudaSuccess) return e;
+  }
+  proj_tc_kernel<TILE_N><<<num_sms, kThreads, smem_bytes, st>>>(tmA, tmB, b);
   count_launch(1);
   return cudaGetLastError();
 }
@@ -304,6 +321,21 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// The canonical K x N bank seen as {64 columns, K rows, N/64 column chunks}: one box of
+// 64 x 64 x chunks lands in shared memory chunk-major ([chunk][k][64 n]), which is exactly the
+// MN-major 128-byte-swizzled operand layout, with a single copy instruction per stage.
+cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
+  if (a.N % 64 || std::getenv("ALGPROJ_B2D")) return cudaErrorInvalidValue;
+  cuuint64_t dims[3] = {64, (cuuint64_t)a.K, (cuuint64_t)(a.N / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)a.ldw * 2, 128};
+  cuuint32_t box[3] = {64, kTcBlockK, (cuuint32_t)chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.W), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;

@@ -190,6 +190,7 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
 // A operand of either kind: plain rows (2-D) or, for the cyclic schedule, the type-strided view
 // {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);
+cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks);
 
 }  // namespace tc
 }  // namespace algproj
