@@ -32,6 +32,8 @@ struct alg_proj_s {
   int device = 0;
   int num_sms = 148;
   int n_workers = 1;        // persistent CTAs (or CTA pairs) of the tensor-core kernel
+  bool decode_ok = false;   // the small-M weight-streaming kernel covers this shape
+  DecodePlan decode = {};
 };
 
 struct alg_ffn_s {
@@ -159,6 +161,11 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     p.n_workers = p.pair_kernel ? tc2_max_pairs(p.num_sms) : std::min(p.num_sms, kMaxWorkers);
     if (p.n_workers < 1) return ALG_ERR_CUDA;
   }
+  if (dtype == ALG_BF16 && std::getenv("ALGPROJ_NO_DECODE") == nullptr) {
+    p.decode_ok = decode_plan(q, p.s, p.K, p.N, p.num_sms, &p.decode);
+    for (int g = 0; g < q && p.decode_ok; ++g)
+      if (p.r[g] % p.decode.sn) p.decode_ok = false;
+  }
   return ALG_OK;
 }
 
@@ -251,6 +258,33 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   return cuda_status(launch_proj_simt(a, p.dtype == ALG_BF16, st));
 }
 
+bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && M <= kDecodeMaxM; }
+
+alg_status_t run_decode(const alg_proj_s &p, const void *X, int64_t ldx, const int32_t *types, int64_t M,
+                        const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y, int64_t ldy,
+                        alg_dtype_t y_dtype, cudaStream_t st) {
+  DecodeArgs d;
+  d.tab = p.d_tab;
+  d.X = X;
+  d.ldx = ldx;
+  d.types = p.sched == ALG_SCHED_CYCLIC ? nullptr : types;
+  d.M = (int)M;
+  d.W = W;
+  d.ldw = ldw;
+  d.bias = bias;
+  d.act = (int)act;
+  d.Y = Y;
+  d.ldy = ldy;
+  d.y_bf16 = y_dtype == ALG_BF16;
+  d.K = p.K;
+  d.N = p.N;
+  d.splits = p.decode.splits;
+  d.w_smem_bytes = p.decode.w_smem_bytes;
+  d.x_smem_bytes = p.decode.x_smem_bytes;
+  d.status = p.d_status;
+  return cuda_status(launch_decode(d, p.decode, st));
+}
+
 }  // namespace
 
 extern "C" {
@@ -304,6 +338,7 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
+  if (use_decode(*h, M)) return run_decode(*h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
 
   BucketArgs b;
   b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
@@ -347,7 +382,7 @@ alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *
 
 alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path) {
   if (!h || !path || M < 0) return ALG_ERR_INVALID_ARG;
-  *path = use_tc(*h) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
+  *path = use_decode(*h, M) ? ALG_PATH_DECODE : use_tc(*h) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
   return ALG_OK;
 }
 
@@ -421,6 +456,13 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
+  if (use_decode(h->up, M) && use_decode(h->down, M)) {
+    // decode shapes: no bucketing, H stays in the original row order
+    void *Hd = ws + L.h;
+    alg_status_t sd = run_decode(h->up, X, h->D, types, M, W_up, h->F, b_up, act, Hd, h->F, ALG_BF16, st);
+    if (sd != ALG_OK) return sd;
+    return run_decode(h->down, Hd, h->F, types, M, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, st);
+  }
 
   BucketArgs b;
   b.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;

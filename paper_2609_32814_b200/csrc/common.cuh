@@ -124,11 +124,18 @@ cudaError_t tc_init();  // resolves the driver entry point for tensor-map encodi
 
 // decode path (M <= 64)
 constexpr int kDecodeMaxM = 64;
+struct DecodePlan {
+  int sn;            // strip width in columns (64 or 32)
+  int splits;        // K splits = cluster size (1..8)
+  int w_smem_bytes;  // worst-case weight slice of one CTA
+  int x_smem_bytes;  // worst-case staged X slice
+  int p_smem_bytes;  // partial sums
+};
 struct DecodeArgs {
   const DevTable *tab;
   const void *X;
   int64_t ldx;
-  const int32_t *types;   // nullptr => cyclic
+  const int32_t *types;   // nullptr => cyclic (row mod q)
   int M;
   const void *W;
   int64_t ldw;
@@ -139,12 +146,13 @@ struct DecodeArgs {
   int y_bf16;
   int K;
   int N;
-  float *partials;        // split-K scratch
-  int *tickets;           // per-strip arrival counters (zero on entry, left zero on exit)
+  int splits;
+  int w_smem_bytes;
+  int x_smem_bytes;
   int *status;
 };
-size_t decode_workspace_bytes(int K, int N);
-cudaError_t launch_decode(const DecodeArgs &a, int num_sms, cudaStream_t st);
+bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *plan);
+cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st);
 
 void count_launch(int n = 1);
 
