@@ -329,7 +329,66 @@ def side_measurements(binding, wl, types, time_steps, star_ms):
     out["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms,
                        "time_ratio_star_over_dense": star_ms / dense_ms,
                        "control": "same library, ALG_TABLE_DENSE (8 block GEMMs instead of 6)"}
+    out["decode"] = decode_measurements(binding, wl)
     return out
+
+
+def decode_measurements(binding, wl, layers=64, replays=20):
+    """KV-cached decode shapes (config 4): M new tokens, type = absolute position mod 2.
+    streaming: a CUDA graph of `layers` consecutive FFN layers with distinct weight banks
+    (604 MB, far beyond L2), layer l+1 consuming layer l's output -- GB/s counts the weight
+    blocks some row needs plus X and Y of every projection.  isolated: one FFN per replay."""
+    import torch
+    from paper_2609_32814_b200 import synth
+    peaks = _peaks()
+    D, F = wl.D, wl.F
+    g = torch.Generator(device="cuda").manual_seed(1234)
+    Wu = [(torch.randn((D, F), device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(layers)]
+    Wd = [(torch.randn((F, D), device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(layers)]
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    ws = torch.empty(ffn.workspace_bytes(64), dtype=torch.uint8, device="cuda")
+    res = []
+    stream = torch.cuda.Stream()
+    for M in (1, 8, 32, 64):
+        w4 = synth.config4(M)
+        types = torch.from_numpy(w4.types).cuda()
+        present = len(set(w4.types.tolist()))
+        # weight bytes some row needs: diagonal blocks always, off-diagonal block (k,j) iff type k present
+        frac = 1.0 if present == 2 else 0.75
+        bytes_layer = frac * 2 * D * F * 2 + 2 * M * (D + F) * 2
+        acts = [torch.from_numpy(w4.X).cuda().to(torch.bfloat16)] + \
+               [torch.empty((M, D), dtype=torch.bfloat16, device="cuda") for _ in range(layers)]
+
+        def chain(n):
+            for l in range(n):
+                ffn.forward(acts[l], types, Wu[l], Wd[l], act="gelu", out=acts[l + 1], workspace=ws, stream=stream)
+
+        def graph_time(n, reps):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                chain(n)                      # warm-up outside capture
+                torch.cuda.synchronize()
+                with torch.cuda.graph(gr, stream=stream):
+                    chain(n)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ts = []
+            for _ in range(reps):
+                e0.record()
+                gr.replay()
+                e1.record()
+                e1.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            return float(np.median(ts))
+
+        t_stream = graph_time(layers, replays)
+        t_iso = graph_time(1, replays)
+        gbs = layers * bytes_layer / (t_stream * 1e-3) / 1e9
+        res.append({"M": M, "types_present": present, "needed_mb_per_layer": bytes_layer / 1e6,
+                    "stream_us_per_layer": t_stream * 1e3 / layers, "stream_gbs": gbs,
+                    "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "isolated_warm_us": t_iso * 1e3})
+    assert ffn.last_status() == 0
+    return {"protocol": f"{layers}-layer dependent FFN chain with distinct weights in one CUDA graph, median of {replays} replays",
+            "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res}
 
 
 if __name__ == "__main__":

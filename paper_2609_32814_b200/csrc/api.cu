@@ -279,9 +279,17 @@ alg_status_t run_decode(const alg_proj_s &p, const void *X, int64_t ldx, const i
   d.K = p.K;
   d.N = p.N;
   d.splits = p.decode.splits;
+  d.box_rows = p.decode.box_rows;
   d.w_smem_bytes = p.decode.w_smem_bytes;
   d.x_smem_bytes = p.decode.x_smem_bytes;
   d.status = p.d_status;
+  d.trace = g_trace;
+  d.q = p.q;
+  d.small_q = p.q <= kDecodeParamQ;
+  if (d.small_q) {
+    for (int e = 0; e <= p.q; ++e) d.so[e] = p.tab.so[e], d.ro[e] = p.tab.ro[e];
+    for (int e = 0; e < p.q * p.q; ++e) d.keep[e] = p.tab.keep[e];
+  }
   return cuda_status(launch_decode(d, p.decode, st));
 }
 

@@ -124,9 +124,11 @@ cudaError_t tc_init();  // resolves the driver entry point for tensor-map encodi
 
 // decode path (M <= 64)
 constexpr int kDecodeMaxM = 64;
+constexpr int kDecodeParamQ = 8;   // tables of up to this many groups travel by value in the kernel parameters
 struct DecodePlan {
   int sn;            // strip width in columns (64 or 32)
   int splits;        // K splits = cluster size (1..8)
+  int box_rows;      // rows per TMA box of the weight slice (divides every s[k] / splits, <= 256)
   int w_smem_bytes;  // worst-case weight slice of one CTA
   int x_smem_bytes;  // worst-case staged X slice
   int p_smem_bytes;  // partial sums
@@ -147,9 +149,16 @@ struct DecodeArgs {
   int K;
   int N;
   int splits;
+  int box_rows;
   int w_smem_bytes;
   int x_smem_bytes;
   int *status;
+  long long *trace;       // debug timeline (nullptr = off)
+  int q;
+  int small_q;            // q <= kDecodeParamQ: the table below is valid
+  int so[kDecodeParamQ + 1];
+  int ro[kDecodeParamQ + 1];
+  uint32_t keep[kDecodeParamQ * kDecodeParamQ];
 };
 bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *plan);
 cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st);

@@ -7,34 +7,39 @@
 // nobody needs are skipped (a single row of the Q_2 law touches 3 of the 4 blocks).
 //
 // Decomposition: grid = (N / SN column strips) x (K splits); the `splits` CTAs of a strip form a
-// thread-block cluster.  A CTA copies its slice of the bank (its share of the rows of every
-// needed input group, SN columns wide) into shared memory with 16-byte asynchronous copies that
-// are all in flight at once, stages the matching columns of X (rows that do not use a block are
-// staged as zeros, which is how the row-type rule is applied), multiplies with warp-level
-// mma.sync (bf16 x bf16 -> fp32) and leaves an M x SN partial sum in shared memory.  The cluster
-// then reduces the partial sums through distributed shared memory in a fixed order (deterministic,
+// thread-block cluster.  A CTA fetches its slice of the bank (its share of the rows of every
+// needed input group, SN columns wide) with one or two TMA boxes per group -- issued before it
+// waits for the previous kernel in the stream (programmatic dependent launch), because weights do
+// not depend on it -- stages the matching columns of X with 16-byte asynchronous copies (rows
+// that do not use a block are staged as zeros, which is how the row-type rule is applied),
+// multiplies with warp-level mma.sync (bf16 x bf16 -> fp32), and pushes its partial sums into the
+// shared memory of the CTA that owns the output row (row m belongs to CTA m mod splits).  After
+// one cluster barrier every CTA adds the partial sums of its rows in split order (deterministic,
 // nothing goes through global memory), applies bias / activation and stores Y.
 #include <cuda_runtime.h>
 
-#include "common.cuh"
+#include <cstdlib>
+
+#include "tc_common.cuh"
 
 namespace algproj {
+
+using namespace tc;
 
 namespace {
 
 constexpr int kThreads = 128;
-constexpr int kMaxSeg = kMaxQ;
+constexpr int kMaxBoxRows = 256;
 
 struct Seg {
   int grow0;   // first row of W (= first column of X) of the segment
   int len;     // rows, a multiple of 16
   int loc0;    // first local row inside the CTA's slice
-  unsigned long long rows;  // bit b set: row b of X uses this block
+  uint32_t rows_lo, rows_hi;  // bit b set: row b of X uses this block
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void cp_async_16_zfill(uint32_t dst, const void *src, bool valid) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
@@ -53,8 +58,7 @@ __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t (&r)[2
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -62,12 +66,10 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ float ld_remote_f32(uint32_t local_addr, uint32_t rank) {
+__device__ __forceinline__ void st_remote_f32x2(uint32_t local_addr, uint32_t rank, float x, float y) {
   uint32_t remote;
-  float v;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-  return v;
+  asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote), "f"(x), "f"(y) : "memory");
 }
 __device__ __forceinline__ float act_f(float z, int act) {
   if (act == ALG_ACT_GELU_ERF) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
@@ -78,8 +80,10 @@ __device__ __forceinline__ float act_f(float z, int act) {
   return z;
 }
 
-// Shared-memory images.  W slice: [rows][SN] bf16, 16-byte chunks XOR-swizzled so the 8 rows an
-// ldmatrix touches fall into different banks.  X slice: [m_pad][x_pitch] bf16, swizzled likewise.
+// Shared-memory images.  W slice: [rows][SN] bf16 as the TMA writes it with its 128-byte (SN = 64)
+// or 64-byte (SN = 32) swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7), resp.
+// c ^ ((r >> 1) & 3), so the 8 rows an ldmatrix touches fall into different banks.  X slice:
+// [m_pad][x_pitch] bf16, written by this kernel with the same kind of XOR.
 template <int SN>
 __device__ __forceinline__ uint32_t w_off(int row, int chunk) {
   constexpr int kChunks = SN / 8;
@@ -90,98 +94,151 @@ __device__ __forceinline__ uint32_t x_off(int m, int chunk, int x_pitch_bytes) {
   return (uint32_t)(m * x_pitch_bytes + ((chunk ^ (m & 7)) << 4));
 }
 
+#ifdef ALGPROJ_TRACE
+#define DTR() tr[trn++] = clock64()
+#else
+#define DTR() \
+  do {        \
+  } while (0)
+#endif
+
 template <int SN>
-__global__ void __launch_bounds__(kThreads) decode_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant__ CUtensorMap tmW, const DecodeArgs a) {
   constexpr int NT = SN / 32;          // 8-column n-tiles per warp (4 warps share the strip)
-  constexpr int kWChunks = SN / 8;     // 16-byte chunks per W row
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ Seg s_seg[kMaxSeg];
-  __shared__ int s_nseg, s_rows, s_type[kDecodeMaxM];
-  __shared__ unsigned long long s_bad;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Seg s_seg[kMaxQ];
+  __shared__ int s_nseg, s_rows;
+  __shared__ int s_so[kMaxQ + 1], s_ro[kMaxQ + 1];
+  __shared__ uint32_t s_keep[kMaxPairs];
+  __shared__ uint32_t s_rows32[kMaxQ][2], s_bad32[2];
+  __shared__ __align__(8) uint64_t s_bar;
 
   const DevTable *__restrict__ tab = a.tab;
-  const int q = tab->q;
+  const int q = a.q;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int strip = blockIdx.x, split = blockIdx.y, splits = gridDim.y;
   const int n0 = strip * SN;
   const int M = a.M;
   const int m_tiles = (M + 15) >> 4, m_pad = m_tiles << 4;
+#ifdef ALGPROJ_TRACE
+  long long tr[12];
+  int trn = 0;
+#endif
+  DTR();
 
-  // ---- row types, support of this strip ----
-  if (tid < kDecodeMaxM) {
-    int t = -1;
-    if (tid < M) {
-      t = a.types ? a.types[tid] : (tid % q);
-      if (t < 0 || t >= q) {
-        atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
-        t = -1;
-      }
-    }
-    s_type[tid] = t;
+  // ---- row types, support of this strip (one global round trip, then shared memory only) ----
+  if (a.small_q) {  // table travels in the kernel parameters: no global metadata load at all
+    for (int e = tid; e <= q; e += kThreads) s_so[e] = a.so[e], s_ro[e] = a.ro[e];
+    for (int e = tid; e < q * q; e += kThreads) s_keep[e] = a.keep[e];
+  } else {
+    for (int e = tid; e <= q; e += kThreads) s_so[e] = tab->so[e], s_ro[e] = tab->ro[e];
+    for (int e = tid; e < q * q; e += kThreads) s_keep[e] = tab->keep[e];
   }
-  __syncthreads();
+  int my_type = -1;
+  if (tid < M) {
+    my_type = a.types ? a.types[tid] : (tid % q);
+    if (my_type < 0 || my_type >= q) {
+      atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
+      my_type = -1;
+    }
+  }
   if (tid == 0) {
-    int j = 0;
-    while (j + 1 < q && tab->ro[j + 1] <= n0) ++j;
-    unsigned long long bad = 0;
-    for (int b = 0; b < M; ++b)
-      if (s_type[b] < 0) bad |= 1ull << b;
-    s_bad = bad;
-    int nseg = 0, loc = 0;
-    for (int k = 0; k < q; ++k) {
-      unsigned long long rows = 0;
-      for (int b = 0; b < M; ++b)
-        if (s_type[b] >= 0 && ((tab->keep[s_type[b] * q + j] >> k) & 1u)) rows |= 1ull << b;
-      if (!rows) continue;  // nobody needs W_kj: it is never read
-      const int len = (tab->so[k + 1] - tab->so[k]) / splits;
-      s_seg[nseg].grow0 = tab->so[k] + split * len;
-      s_seg[nseg].len = len;
-      s_seg[nseg].loc0 = loc;
-      s_seg[nseg].rows = rows;
-      loc += len;
-      ++nseg;
-    }
-    s_nseg = nseg;
-    s_rows = loc;
+    mbar_init(smem_u32(&s_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
   }
   __syncthreads();
+  DTR();
+  int j = 0;
+  while (j + 1 < q && s_ro[j + 1] <= n0) ++j;
+  if (tid < kDecodeMaxM) {  // warps 0 and 1: rows 0..63
+    const uint32_t kmask = my_type >= 0 ? s_keep[my_type * q + j] : 0u;  // input groups this row uses for group j
+    const unsigned badv = __ballot_sync(0xffffffffu, tid < M && my_type < 0);
+    if (lane == 0) s_bad32[warp] = badv;
+    for (int k = 0; k < q; ++k) {
+      const unsigned v = __ballot_sync(0xffffffffu, (kmask >> k) & 1u);
+      if (lane == 0) s_rows32[k][warp] = v;
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {  // segment list: lane k owns input group k; prefix of the lengths by shuffles
+    uint32_t lo = 0, hi = 0;
+    int len = 0;
+    if (lane < q) {
+      lo = s_rows32[lane][0], hi = s_rows32[lane][1];
+      if (lo | hi) len = (s_so[lane + 1] - s_so[lane]) / splits;  // nobody needs W_kj -> it is never read
+    }
+    const unsigned have = __ballot_sync(0xffffffffu, len > 0);
+    int incl = len;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += n;
+    }
+    if (len > 0) {
+      const int s = __popc(have & ((1u << lane) - 1u));
+      s_seg[s].grow0 = s_so[lane] + split * len;
+      s_seg[s].len = len;
+      s_seg[s].loc0 = incl - len;
+      s_seg[s].rows_lo = lo, s_seg[s].rows_hi = hi;
+    }
+    if (lane == 31) s_nseg = __popc(have), s_rows = incl;
+  }
+  __syncthreads();
+  DTR();
   const int nseg = s_nseg, rows_cta = s_rows;
   const int x_pitch_bytes = ((rows_cta + 63) & ~63) * 2;  // whole groups of eight 16-byte chunks
-  uint8_t *w_sm = smem;
+  uint8_t *w_sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t *x_sm = w_sm + (size_t)a.w_smem_bytes;
-  float *p_sm = (float *)(x_sm + (size_t)a.x_smem_bytes);   // [m_pad][SN] partial sums
+  float *r_sm = (float *)(x_sm + (size_t)a.x_smem_bytes);   // [splits][rows owned][SN] partial sums of my rows
 
-  // ---- the weight slice: every 16-byte copy in flight at once ----
-  {
-    const __nv_bfloat16 *W = (const __nv_bfloat16 *)a.W;
-    const uint32_t w_base = smem_u32(w_sm);
+  // ---- the weight slice: one TMA box per segment (more when a segment exceeds the box height) ----
+  if (tid == 0) {
+    const uint32_t bar = smem_u32(&s_bar);
+    mbar_expect_tx(bar, (uint32_t)(rows_cta * SN * 2));
     for (int s = 0; s < nseg; ++s) {
       const Seg sg = s_seg[s];
-      const int chunks = sg.len * kWChunks;
-      for (int c = tid; c < chunks; c += kThreads) {
-        const int r = c / kWChunks, ch = c % kWChunks;
-        cp_async_16(w_base + w_off<SN>(sg.loc0 + r, ch), W + (int64_t)(sg.grow0 + r) * a.ldw + n0 + ch * 8);
-      }
+      for (int r0 = 0; r0 < sg.len; r0 += a.box_rows)
+        tma_load_2d(smem_u32(w_sm) + (uint32_t)((sg.loc0 + r0) * SN * 2), &tmW, bar, n0, sg.grow0 + r0);
     }
   }
+  DTR();
+  // The weights do not depend on the previous kernel in the stream, X does: let the next kernel
+  // start its own weight stream now, and wait for the producer of X only here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  DTR();
   // ---- the matching columns of X; rows that do not use a block are staged as zeros ----
   {
     const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
-    const int xchunks = x_pitch_bytes >> 4;
+    const uint32_t x_base = smem_u32(x_sm);
+    // thread -> (row m = tid / 8 + 16 i, chunk ch = tid % 8 + 8 jj): no divisions in the loop
+    const int m_lo = tid >> 3, ch_lo = tid & 7;
     for (int s = 0; s < nseg; ++s) {
       const Seg sg = s_seg[s];
       const int seg_chunks = sg.len >> 3;
-      for (int e = tid; e < m_pad * seg_chunks; e += kThreads) {
-        const int m = e / seg_chunks, ch = e % seg_chunks;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (m < M && ((sg.rows >> m) & 1ull)) v = *(const uint4 *)(X + (int64_t)m * a.ldx + sg.grow0 + ch * 8);
-        *(uint4 *)(x_sm + x_off(m, (sg.loc0 >> 3) + ch, x_pitch_bytes)) = v;
+      for (int m = m_lo; m < m_pad; m += kThreads / 8) {
+        const bool use = m < M && (((m < 32 ? sg.rows_lo : sg.rows_hi) >> (m & 31)) & 1u);
+        const __nv_bfloat16 *src = X + (int64_t)(use ? m : 0) * a.ldx + sg.grow0;
+        for (int ch = ch_lo; ch < seg_chunks; ch += 8)
+          cp_async_16_zfill(x_base + x_off(m, (sg.loc0 >> 3) + ch, x_pitch_bytes), src + ch * 8, use);
       }
     }
-    (void)xchunks;
   }
+  DTR();
   cp_async_wait_all();
+  {  // bounded wait for the weight slice
+    const uint32_t bar = smem_u32(&s_bar);
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, 0)) {
+      if (clock64() - t0 > kTimeoutCycles) {
+        atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+    }
+  }
   __syncthreads();
+  DTR();
 
   // ---- warp-level MMA: warp w owns columns [w * SN/4, +SN/4) of the strip, all rows ----
   float acc[4][NT][4];
@@ -193,72 +250,91 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const DecodeArgs a) {
       for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
   const uint32_t w_base = smem_u32(w_sm), x_base = smem_u32(x_sm);
   const int wcol_chunk = warp * (SN / 32);  // first 16-byte chunk of this warp's columns
+  const int frag_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll 2
   for (int k0 = 0; k0 < rows_cta; k0 += 16) {
-    uint32_t b[NT * 2];
+    uint32_t b[4];
     if (NT == 2) {
-      uint32_t r4[4];
-      const int krow = k0 + (lane & 7) + ((lane >> 3) & 1) * 8;
-      ldmatrix_x4_trans(w_base + w_off<SN>(krow, wcol_chunk + (lane >> 4)), r4);
-      b[0] = r4[0], b[1] = r4[1], b[NT * 2 - 2] = r4[2], b[NT * 2 - 1] = r4[3];
+      ldmatrix_x4_trans(w_base + w_off<SN>(k0 + frag_row, wcol_chunk + (lane >> 4)), b);
     } else {
       uint32_t r2[2];
-      const int krow = k0 + (lane & 7) + ((lane >> 3) & 1) * 8;
-      ldmatrix_x2_trans(w_base + w_off<SN>(krow, wcol_chunk), r2);
-      b[0] = r2[0], b[1] = r2[1];
+      ldmatrix_x2_trans(w_base + w_off<SN>(k0 + frag_row, wcol_chunk), r2);
+      b[0] = r2[0], b[1] = r2[1], b[2] = 0, b[3] = 0;
     }
+    uint32_t af[4][4];
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) {
+    for (int mt = 0; mt < 4; ++mt)
+      if (mt < m_tiles) ldmatrix_x4(x_base + x_off(mt * 16 + frag_row, (k0 >> 3) + (lane >> 4), x_pitch_bytes), af[mt]);
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
       if (mt < m_tiles) {
-        uint32_t af[4];
-        const int m = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        ldmatrix_x4(x_base + x_off(m, (k0 >> 3) + (lane >> 4), x_pitch_bytes), af);
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[mt][nt], af, b[nt * 2], b[nt * 2 + 1]);
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[mt][nt], af[mt], b[nt * 2], b[nt * 2 + 1]);
       }
-    }
   }
-  // ---- partial sums to shared memory ----
+  DTR();
+  // ---- push the partial sums to the owners of the rows: row m -> CTA m % splits, slot m / splits ----
+  const int rows_owned_max = (m_pad + splits - 1) / splits;
   {
+    const uint32_t r_base = smem_u32(r_sm);
     const int g = lane >> 2, t4 = lane & 3;
 #pragma unroll
     for (int mt = 0; mt < 4; ++mt) {
       if (mt < m_tiles) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const int col = warp * (SN / 4) + nt * 8 + t4 * 2;
-          float *p0 = p_sm + (mt * 16 + g) * SN + col;
-          float *p1 = p_sm + (mt * 16 + g + 8) * SN + col;
-          p0[0] = acc[mt][nt][0], p0[1] = acc[mt][nt][1];
-          p1[0] = acc[mt][nt][2], p1[1] = acc[mt][nt][3];
+        for (int h = 0; h < 2; ++h) {
+          const int m = mt * 16 + g + h * 8;
+          const uint32_t owner = (uint32_t)(m % splits);
+          const int slot = m / splits;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const int col = warp * (SN / 4) + nt * 8 + t4 * 2;
+            const uint32_t off = r_base + (uint32_t)(((split * rows_owned_max + slot) * SN + col) * 4);
+            if (splits > 1) st_remote_f32x2(off, owner, acc[mt][nt][h * 2], acc[mt][nt][h * 2 + 1]);
+            else *(float2 *)(r_sm + (slot * SN + col)) = make_float2(acc[mt][nt][h * 2], acc[mt][nt][h * 2 + 1]);
+          }
         }
       }
     }
   }
-  __syncthreads();
-  if (splits > 1) cluster_sync_all();
+  if (splits > 1) cluster_sync_all();  // all partial sums of my rows have arrived; no remote access after this
+  else __syncthreads();
+  DTR();
 
-  // ---- cluster reduction in split order, bias, activation, store ----
-  // element e of the M x SN strip is finished by the CTA with e % splits == split
+  // ---- add the partial sums of my rows in split order, bias, activation, store ----
   {
-    const uint32_t p_base = smem_u32(p_sm);
-    const unsigned long long bad = s_bad;
-    for (int e = split + tid * splits; e < M * SN; e += kThreads * splits) {
-      const int m = e / SN, n = e % SN;
-      float z = 0.f;
-      if (splits > 1) {
-        for (int s = 0; s < splits; ++s) z += ld_remote_f32(p_base + (uint32_t)(m * SN + n) * 4u, (uint32_t)s);
-      } else {
-        z = p_sm[m * SN + n];
+    constexpr int kGroups = SN / 4;
+    const int my_rows = (M - split + splits - 1) / splits;  // rows m = split + splits * slot < M
+    for (int e = tid; e < my_rows * kGroups; e += kThreads) {
+      const int slot = e / kGroups, n = (e % kGroups) * 4;
+      const int m = split + slot * splits;
+      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < splits; ++s) {
+        const float4 p = *(const float4 *)(r_sm + ((s * rows_owned_max + slot) * SN + n));
+        z.x += p.x, z.y += p.y, z.z += p.z, z.w += p.w;
       }
       const int col = n0 + n;
-      if (a.bias) z += __bfloat162float(((const __nv_bfloat16 *)a.bias)[col]);
-      z = act_f(z, a.act);
-      if ((bad >> m) & 1ull) z = 0.f;  // out-of-range type: the row's output is defined to be zero
-      if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[(int64_t)m * a.ldy + col] = __float2bfloat16_rn(z);
-      else ((float *)a.Y)[(int64_t)m * a.ldy + col] = z;
+      const bool bad = ((m < 32 ? s_bad32[0] : s_bad32[1]) >> (m & 31)) & 1u;
+      float v[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if (a.bias) v[c] += __bfloat162float(((const __nv_bfloat16 *)a.bias)[col + c]);
+        v[c] = act_f(v[c], a.act);
+        if (bad) v[c] = 0.f;  // out-of-range type: the row's output is defined to be zero
+      }
+      if (a.y_bf16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
+        *(uint2 *)((__nv_bfloat16 *)a.Y + (int64_t)m * a.ldy + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+      } else {
+        *(float4 *)((float *)a.Y + (int64_t)m * a.ldy + col) = make_float4(v[0], v[1], v[2], v[3]);
+      }
     }
   }
-  if (splits > 1) cluster_sync_all();  // partial sums stay readable until every CTA has finished
+  DTR();
+#ifdef ALGPROJ_TRACE
+  if (a.trace && tid == 0 && blockIdx.x == 3 && blockIdx.y == 0)
+    for (int e = 0; e < trn; ++e) a.trace[e] = tr[e];
+#endif
 }
 
 template <int SN>
@@ -269,19 +345,27 @@ cudaError_t launch_t(const DecodeArgs &a, size_t smem_bytes, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     attr = true;
   }
+  CUtensorMap tmW;
+  cudaError_t e = make_map_2d_sw(&tmW, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, SN, (uint32_t)a.box_rows,
+                                 SN * 2);
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(a.N / SN, a.splits, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 1;
   at[0].val.clusterDim.y = a.splits;
   at[0].val.clusterDim.z = 1;
+  // programmatic dependent launch: this kernel may start while its predecessor in the stream is
+  // still running; it waits (griddepcontrol.wait) before touching anything the predecessor writes
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<SN>, a);
+  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 1 : 2;
+  return cudaLaunchKernelEx(&cfg, decode_kernel<SN>, tmW, a);
 }
 
 }  // namespace
@@ -302,18 +386,28 @@ bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *pla
     if (N % sn) continue;
     for (int sp = 1; sp <= 8; ++sp) {
       if (g % sp) continue;
+      // one TMA box per segment piece: rows per box divide every s[k] / sp, at most 256
+      int box = 0;
+      for (int k = 0; k < q; ++k) {
+        int v = s[k] / sp;
+        int t = box;
+        while (v) { int u = t % v; t = v; v = u; }
+        box = t;
+      }
+      while (box > kMaxBoxRows) box /= 2;
+      if (box % 8) continue;
       const int rows_max = K / sp;  // worst case: every input group needed by the strip
       const size_t w_bytes = (size_t)rows_max * sn * 2;
       const size_t x_bytes = (size_t)kDecodeMaxM * (((rows_max + 63) & ~63) * 2);
-      const size_t p_bytes = (size_t)kDecodeMaxM * sn * 4;
-      if (w_bytes + x_bytes + p_bytes > 190 * 1024) continue;
+      const size_t p_bytes = (size_t)(kDecodeMaxM + 8) * sn * 4;
+      if (w_bytes + x_bytes + p_bytes + 1024 > 190 * 1024) continue;
       const int ctas = (N / sn) * sp;
       // prefer filling the machine, then not overshooting it, then the wider strip
       long long score = ctas >= num_sms ? (1000000 - (ctas - num_sms)) * 4 : (long long)ctas * 4;
       score += (sn == 64) ? 1 : 0;
       if (score > best_score) {
         best_score = score;
-        best.sn = sn, best.splits = sp;
+        best.sn = sn, best.splits = sp, best.box_rows = box;
         best.w_smem_bytes = (int)w_bytes, best.x_smem_bytes = (int)x_bytes, best.p_smem_bytes = (int)p_bytes;
       }
     }
@@ -326,9 +420,10 @@ bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *pla
 cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st) {
   DecodeArgs b = a;
   b.splits = plan.splits;
+  b.box_rows = plan.box_rows;
   b.w_smem_bytes = plan.w_smem_bytes;
   b.x_smem_bytes = plan.x_smem_bytes;
-  const size_t smem = (size_t)plan.w_smem_bytes + plan.x_smem_bytes + plan.p_smem_bytes;
+  const size_t smem = (size_t)plan.w_smem_bytes + plan.x_smem_bytes + plan.p_smem_bytes + 1024;
   cudaError_t e = plan.sn == 64 ? launch_t<64>(b, smem, st) : launch_t<32>(b, smem, st);
   count_launch(1);
   return e;

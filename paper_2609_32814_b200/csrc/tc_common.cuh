@@ -187,6 +187,8 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
 // Host side: tensor-map encoding through the driver entry point (no link-time libcuda dependency).
 cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,
                         uint32_t box_inner, uint32_t box_outer);
+cudaError_t make_map_2d_sw(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,
+                           uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
 // A operand of either kind: plain rows (2-D) or, for the cyclic schedule, the type-strided view
 // {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);
