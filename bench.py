@@ -107,6 +107,29 @@ class ClockSampler:
                 "reasons": [n for b, n in self.REASONS.items() if mask & b], "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Multi-rank timing rule: the job is as slow as its slowest rank (no-op without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_batch_seed(rank: int, world: int, set_index: int) -> int:
+    """Seed of working set `set_index` on `rank`: every rank draws its own rows (rows shard across
+    ranks, weights are replicated); rank 0 of a single-GPU run keeps the parity-test batch."""
+    from paper_2609_32814_b200 import synth
+    return synth.seed_for(2, 50 + rank * N_SETS + set_index)
+
+
+def whole_job_value(flops_per_rank_step: int, world: int, steps: int, total_ms: float) -> float:
+    """Weak scaling: every rank runs the same per-GPU batch; value = work of all ranks / slowest rank's time."""
+    return world * flops_per_rank_step * steps / (total_ms * 1e-3) / 1e12
+
+
 def kept_flops(ffn, wl) -> int:
     rows = np.bincount(wl.types, minlength=wl.q).tolist()
     return 2 * ffn.macs(rows)
@@ -209,7 +232,7 @@ def main():
     ws_bytes = ffn.workspace_bytes(wl.M)
     sets = []
     for r in range(N_SETS):
-        Xr = synth.bf16_round(synth.normal(synth.seed_for(2, 50 + rank * N_SETS + r), wl.X.shape, 1.0)) if (r or world > 1) else wl.X
+        Xr = synth.bf16_round(synth.normal(rank_batch_seed(rank, world, r), wl.X.shape, 1.0)) if (r or world > 1) else wl.X
         sets.append({"X": dev(Xr), "Wu": dev(wl.W_up).clone(), "Wd": dev(wl.W_down).clone(),
                      "Y": torch.empty((wl.M, wl.D), dtype=torch.bfloat16, device="cuda"),
                      "ws": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")})
@@ -244,12 +267,9 @@ def main():
     with ClockSampler(local_rank) as clocks:
         total_ms = time_steps(args.steps, first=args.warmup)
     launches = binding.launch_count() - launches0
-    if world > 1:
-        tt_ = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt_, op=dist.ReduceOp.MAX)
-        total_ms = float(tt_.item())
+    total_ms = max_over_ranks(total_ms, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * flops * args.steps / (total_ms * 1e-3) / 1e12
+    value = whole_job_value(flops, world, args.steps, total_ms)
     assert ffn.last_status() == 0
 
     # ---- per-kernel durations (second pass with events between the kernels) ----
@@ -284,11 +304,8 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tt_ = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt_, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt_.item())
-    e2e = {"value": world * flops * args.steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+    e2e_ms = max_over_ranks(e2e_ms, "cuda")
+    e2e = {"value": whole_job_value(flops, world, args.steps, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
            "ms_per_step": e2e_ms / args.steps}
 
