@@ -215,6 +215,12 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.offsets = cyclic ? nullptr : ((const WsHeader *)(ws + L.hdr))->offsets;
   a.cyclic_rows = cyclic ? (int)(M / p.q) : 0;
   a.n_classes = p.tab.n_classes;
+  a.st.valid = p.q <= kParamQ && p.tab.n_classes <= 2 * kParamQ * kParamQ;
+  if (a.st.valid) {
+    for (int e = 0; e <= p.q; ++e) a.st.so[e] = p.tab.so[e], a.st.ro[e] = p.tab.ro[e];
+    for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = p.tab.keep[e];
+    for (int e = 0; e < p.tab.n_classes; ++e) a.st.class_order[e] = p.tab.class_order[e];
+  }
   a.geom.tile_m = tile_m_of(p);
   a.geom.tile_n = tile_n_of(p);
   a.geom.split_rem = use_tc(p) && p.pair_kernel;

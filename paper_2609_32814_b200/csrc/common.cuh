@@ -75,11 +75,23 @@ cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st);
 cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int M, int K,
                                int elem_bytes, void *Xb, cudaStream_t st);
 
+// Interaction table of a small-q handle, carried by value in the kernel parameters so that a
+// kernel prologue needs no global metadata load.
+constexpr int kParamQ = 8;
+struct SmallTable {
+  int valid;                              // q <= kParamQ and n_classes <= 2 * kParamQ * kParamQ
+  int so[kParamQ + 1];
+  int ro[kParamQ + 1];
+  uint32_t keep[kParamQ * kParamQ];
+  int class_order[2 * kParamQ * kParamQ];
+};
+
 struct ProjArgs {
   const DevTable *tab;
   const int *offsets;     // device bucket offsets [q+2]; nullptr with the cyclic schedule (equal buckets)
   int cyclic_rows;        // M/q when offsets == nullptr
   int n_classes;          // tab->n_classes (host copy, sizes the shared-memory tile map)
+  SmallTable st;          // by-value copy of the table when it is small
   TileGeom geom;
   const void *X;          // SIMT: original rows (gathered through perm); tcgen05: bucketed copy
   int64_t ldx;

@@ -30,8 +30,8 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
   __shared__ __align__(16) unsigned char s_map[sizeof(TileMap) + (2 * kMaxClasses + 1) * sizeof(int)];
   TileMap *tm = reinterpret_cast<TileMap *>(s_map);
   const DevTable *__restrict__ tab = a.tab;
-  const int q = tab->q;
-  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  const int q = a.q;
+  tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
   const int n_tiles = tm->total;
   const T *__restrict__ X = (const T *)a.X;
   const T *__restrict__ W = (const T *)a.W;

@@ -98,7 +98,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
-  const int q = tab->q;
+  const int q = a.q;
   [[maybe_unused]] int tr_n = 0;
 
   if (threadIdx.x == 0) {
@@ -115,15 +115,20 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
   }
-  for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = tab->keep[e];
-  for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = tab->so[e];
+  for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
+  for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"((uint32_t)C::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  // Programmatic dependent launch: everything above touches only this CTA's own state, so it may
+  // run while the previous kernel of the stream is finishing; nothing below (bucket offsets, X, H,
+  // Y) is read or written before that kernel has completed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
   tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x, gridDim.x);
   tc_fence_before();
   __syncthreads();
@@ -306,9 +311,19 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
     if (e != cudaSuccess) return e;
   }
-  proj_tc_kernel<TILE_N><<<num_sms, kThreads, smem_bytes, st>>>(tmA, tmB, b);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(num_sms, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, b);
   count_launch(1);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace

@@ -157,15 +157,15 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
   }
-  for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = tab->keep[e];
-  for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = tab->so[e];
+  for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
+  for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
   if (warp == 1) {  // both CTAs of the pair allocate together, same shared-memory slot
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"((uint32_t)kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
-  tile_map_build(tm, tab, a.offsets, a.cyclic_rows, a.M, a.geom);
+  tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
   tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x >> 1, gridDim.x >> 1);
   tc_fence_before();
   __syncthreads();

@@ -37,17 +37,16 @@ __device__ __forceinline__ int tile_map_n_tiles(const TileGeom &g, int cls, int 
 
 // Called by all threads of the CTA (blockDim.x >= 32).  `offsets` = device bucket offsets, or
 // nullptr for the cyclic schedule with equal buckets of cyclic_rows rows.  Ends with a barrier.
-__device__ inline void tile_map_build(TileMap *tm, const DevTable *tab, const int *offsets, int cyclic_rows, int M,
-                                      const TileGeom &g) {
-  const int q = tab->q, nc = tab->n_classes;
+__device__ inline void tile_map_build(TileMap *tm, const DevTable *tab, const SmallTable &st, int q, int nc,
+                                      const int *offsets, int cyclic_rows, int M, const TileGeom &g) {
   if (threadIdx.x == 0) tm->n_classes = nc, tm->q = q;
   for (int t = threadIdx.x; t <= q + 1; t += blockDim.x)
     tm->offsets[t] = offsets ? offsets[t] : (t <= q ? t * cyclic_rows : M);
-  for (int t = threadIdx.x; t <= q; t += blockDim.x) tm->ro[t] = tab->ro[t];
+  for (int t = threadIdx.x; t <= q; t += blockDim.x) tm->ro[t] = st.valid ? st.ro[t] : tab->ro[t];
   __syncthreads();
   int *cls = tm->cls(), *prefix = tm->prefix();
   for (int c = threadIdx.x; c < nc; c += blockDim.x) {
-    const int id = tab->class_order[c];
+    const int id = st.valid ? st.class_order[c] : tab->class_order[c];
     const int pair = id >> 1, i = pair / q, j = pair % q;
     cls[c] = id;
     prefix[c] = ceil_div(tm->offsets[i + 1] - tm->offsets[i], g.tile_m) * tile_map_n_tiles(g, id, tm->ro[j + 1] - tm->ro[j]);
