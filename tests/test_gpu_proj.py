@@ -84,6 +84,9 @@ def _tc_workload(q, M, s_w, r_w, types=None, integer=True, seed=1):
     (4, 777, 128, 512),    # config-3 group shapes, several types
     (3, 515, 192, 128),    # non-power-of-two q
     (1, 200, 256, 256),    # q = 1 degenerates to an ordinary GEMM
+    (2, 700, 1024, 192),   # long K loops (32 K blocks per off-diagonal tile), 192 columns wide
+    (2, 300, 1024, 256),
+    (1, 520, 1024, 128),
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_tc_integer_bit_exact(q, M, s_w, r_w, out_dtype):
