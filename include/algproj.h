@@ -56,9 +56,12 @@ typedef enum { ALG_F32 = 0, ALG_BF16 = 1 } alg_dtype_t;
 /* Which (type i, output group j, input group k) products are kept.
  * QQ     : the paper's complete-graph law, k in {i,j}  (2q^2-q block GEMMs, Eq. q-rank).
  * DENSE  : all k -- the ordinary product X W (q^3 block GEMMs); the same-library control.
- * CUSTOM : caller-supplied keep[(i*q+j)*q+k] bytes (non-zero = kept), e.g. the tensor-power
- *          law Q_2^{(x)L} of the appendix "The Tensor-Square Candidate". */
-typedef enum { ALG_TABLE_QQ = 0, ALG_TABLE_DENSE = 1, ALG_TABLE_CUSTOM = 2 } alg_table_t;
+ * CUSTOM : caller-supplied keep[(i*q+j)*q+k] bytes (non-zero = kept).
+ * Q2POW  : the tensor power Q_2^{(x)L}, q = 2^L (appendix "The Tensor-Square Candidate", the law
+ *          of the paper's pretraining pilot with L = 2): types and groups are L-bit strings and
+ *          k is kept for (i,j) iff every bit of k equals the matching bit of i or of j
+ *          (6^L block GEMMs; 36 for q = 4; arithmetic fraction (3/4)^L with equal groups). */
+typedef enum { ALG_TABLE_QQ = 0, ALG_TABLE_DENSE = 1, ALG_TABLE_CUSTOM = 2, ALG_TABLE_Q2POW = 3 } alg_table_t;
 
 /* Activation applied to (acc + bias) before the store. GELU_ERF is z/2 (1 + erf(z/sqrt 2)). */
 typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } alg_act_t;

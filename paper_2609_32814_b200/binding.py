@@ -18,13 +18,13 @@ ALG_OK = 0
 STATUS = {0: "ALG_OK", 1: "ALG_ERR_INVALID_ARG", 2: "ALG_ERR_UNSUPPORTED_SHAPE", 3: "ALG_ERR_WORKSPACE_TOO_SMALL",
           4: "ALG_ERR_CUDA", 5: "ALG_ERR_BAD_TYPE", 6: "ALG_ERR_DEVICE_TIMEOUT"}
 ALG_F32, ALG_BF16 = 0, 1
-ALG_TABLE_QQ, ALG_TABLE_DENSE, ALG_TABLE_CUSTOM = 0, 1, 2
+ALG_TABLE_QQ, ALG_TABLE_DENSE, ALG_TABLE_CUSTOM, ALG_TABLE_Q2POW = 0, 1, 2, 3
 ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
 ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC = 0, 1
 ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
 
 _DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
-_TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM}
+_TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM, "q2pow": ALG_TABLE_Q2POW}
 _ACTS = {None: ALG_ACT_NONE, "none": ALG_ACT_NONE, "gelu": ALG_ACT_GELU_ERF, "gelu_erf": ALG_ACT_GELU_ERF,
          "gelu_tanh": ALG_ACT_GELU_TANH}
 _SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC}

@@ -59,7 +59,9 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
                        alg_table_t table, const uint8_t *custom, alg_schedule_t sched, int *shared_status) {
   if (q < 1 || q > kMaxQ || !in_w || !out_w) return ALG_ERR_INVALID_ARG;
   if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
-  if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM) return ALG_ERR_INVALID_ARG;
+  if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM && table != ALG_TABLE_Q2POW)
+    return ALG_ERR_INVALID_ARG;
+  if (table == ALG_TABLE_Q2POW && (q & (q - 1)) != 0) return ALG_ERR_INVALID_ARG;  // q must be a power of two
   if (table == ALG_TABLE_CUSTOM && !custom) return ALG_ERR_INVALID_ARG;
   if (sched != ALG_SCHED_EXPLICIT && sched != ALG_SCHED_CYCLIC) return ALG_ERR_INVALID_ARG;
   p.q = q;
@@ -87,9 +89,11 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     for (int j = 0; j < q; ++j) {
       uint32_t m = 0;
       for (int k = 0; k < q; ++k) {
-        bool keep = table == ALG_TABLE_DENSE  ? true
-                    : table == ALG_TABLE_QQ   ? (k == i || k == j)
-                                              : custom[((size_t)i * q + j) * q + k] != 0;
+        // Q2POW: bits where k differs from i, and bits where k differs from j, must not overlap
+        bool keep = table == ALG_TABLE_DENSE   ? true
+                    : table == ALG_TABLE_QQ    ? (k == i || k == j)
+                    : table == ALG_TABLE_Q2POW ? (((k ^ i) & (k ^ j)) == 0)
+                                               : custom[((size_t)i * q + j) * q + k] != 0;
         if (keep) m |= 1u << k;
       }
       if (m == 0) return ALG_ERR_INVALID_ARG;  // an output block nobody writes

@@ -1,6 +1,6 @@
 """Timing sweep over the benchmark configurations 3 and 5 (and their dense same-shape controls).
 
-    python -m paper_2609_32814_b200.sweep [--configs 3,5] [--reps 10]
+    python -m paper_2609_32814_b200.sweep [--configs 3,5,pilot] [--reps 10]
 
 Prints one JSON line per measured object: the square d->d projection, the up and down projections
 and the whole FFN, each next to the same call with ALG_TABLE_DENSE.  FLOPs count only the block
@@ -45,10 +45,11 @@ def _time(fn, n_sets, reps):
     return e0.elapsed_time(e1) / reps
 
 
-def measure(name, q, M, D, F, seed, reps, want=("up", "down", "ffn")):
+def measure(name, q, M, D, F, seed, reps, want=("up", "down", "ffn"), law="qq", types=None):
     peak_tf, hbm_gbs, src = _peaks()
     g = torch.Generator(device="cuda").manual_seed(seed)
-    types = torch.randint(0, q, (M,), device="cuda", generator=g, dtype=torch.int32)
+    if types is None:
+        types = torch.randint(0, q, (M,), device="cuda", generator=g, dtype=torch.int32)
     counts = torch.bincount(types.long(), minlength=q).tolist()
     dw, fw = [D // q] * q, [F // q] * q
     set_bytes = 2 * (2 * M * D + 2 * D * F + M * F)
@@ -61,7 +62,7 @@ def measure(name, q, M, D, F, seed, reps, want=("up", "down", "ffn")):
     Yd = [torch.empty((M, D), device="cuda", dtype=torch.bfloat16) for _ in range(n_sets)]
     Yf = [torch.empty((M, F), device="cuda", dtype=torch.bfloat16) for _ in range(n_sets)]
     out = []
-    for table in ("qq", "dense"):
+    for table in (law, "dense"):
         objs = {}
         if "square" in want:
             p = binding.Proj(dw, dw, dtype="bf16", table=table)
@@ -93,7 +94,7 @@ def measure(name, q, M, D, F, seed, reps, want=("up", "down", "ffn")):
                         "frac_of_roofline": t_roof / (ms * 1e-3), "peaks": src, "working_sets": n_sets})
     by = {(r["object"], r["table"]): r for r in out}
     for r in out:
-        if r["table"] == "qq":
+        if r["table"] != "dense":
             r["time_vs_dense"] = r["ms"] / by[(r["object"], "dense")]["ms"]
     return out
 
@@ -103,11 +104,19 @@ def main():
     ap.add_argument("--configs", default="3,5")
     ap.add_argument("--reps", type=int, default=10)
     args = ap.parse_args()
-    cfgs = [int(c) for c in args.configs.split(",")]
+    cfgs = [int(c) for c in args.configs.split(",") if c.isdigit()]
     if 3 in cfgs:
         for q in (4, 8):
             for r in measure(f"cfg3-q{q}", q, 16384, q * 128, 4 * q * 128, 300 + q, args.reps, want=("square", "up", "down", "ffn")):
                 print(json.dumps(r), flush=True)
+    if "pilot" in args.configs:
+        # the paper's pilot FFN projections: tensor-square law, D = 768 = 4 x 192, F = 1536 = 4 x 384,
+        # interval schedule floor((p mod 768) / 192), 8 sequences of 1536 tokens
+        from . import synth
+        M = 8 * 1536
+        t = torch.from_numpy(synth.interval_types(M, 4, 768)).cuda()
+        for r in measure("pilot-q2pow", 4, M, 768, 1536, 600, args.reps, law="q2pow", types=t):
+            print(json.dumps(r), flush=True)
     if 5 in cfgs:
         for q in (2, 4, 8, 16):
             for r in measure(f"cfg5-q{q}", q, 32768, 4096, 16384, 500 + q, max(3, args.reps // 2)):

@@ -153,3 +153,17 @@ def config5(q: int, M: int = 32768, D: int = 4096, F: int = 16384, integer: bool
     """scale sweep: 4096 -> 16384, uniform row types."""
     return make_workload(f"cfg5-q{q}", config=5, variant=q * 2 + int(integer), dtype="bf16", q=q, M=M,
                          D=D, F=F, types=uniform_types(seed_for(5, q) + 7, M, q), integer=integer)
+
+
+def interval_types(M: int, q: int, period: int, start: int = 0) -> np.ndarray:
+    """The pilot's schedule: type = floor((position mod period) / (period / q)) -- consecutive
+    intervals of period/q positions share a type."""
+    pos = (np.arange(M, dtype=np.int64) + start) % period
+    return (pos // (period // q)).astype(np.int32)
+
+
+def pilot_ffn(M: int = 4 * 1536, integer: bool = False) -> Workload:
+    """Shape of the paper's ~110M pilot FFN projections: D = 768 split 4 x 192, F = 1536 split
+    4 x 384 (tensor-square law, q = 4), interval schedule with period 768."""
+    return make_workload("pilot", config=6, variant=int(integer), dtype="bf16", q=4, M=M, D=768, F=1536,
+                         types=interval_types(M, 4, 768), integer=integer)

@@ -38,6 +38,9 @@ def test_status_strings_and_argument_errors_need_no_gpu():
     assert L.alg_proj_create(ctypes.byref(h), 2, None, wp, 1, 0, None, 0) == 1    # NULL widths
     assert L.alg_proj_create(ctypes.byref(h), 2, wp, wp, 7, 0, None, 0) == 1      # bad dtype
     assert L.alg_proj_create(ctypes.byref(h), 2, wp, wp, 1, 2, None, 0) == 1      # custom table without keep
+    w3 = (ctypes.c_int32 * 3)(128, 128, 128)
+    w3p = ctypes.cast(w3, ctypes.c_void_p)
+    assert L.alg_proj_create(ctypes.byref(h), 3, w3p, w3p, 1, 3, None, 0) == 1    # tensor-power law needs q = 2^L
     bad = (ctypes.c_int32 * 2)(128, 0)
     assert L.alg_proj_create(ctypes.byref(h), 2, ctypes.cast(bad, ctypes.c_void_p), wp, 1, 0, None, 0) == 1
     assert L.alg_proj_destroy(None) == 1

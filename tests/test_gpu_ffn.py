@@ -179,3 +179,28 @@ def test_cyclic_fast_path_matches_explicit_types(q, M):
     Yp = proj.forward(H.to_dev(wl.X, "bf16"), None, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
     refp = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
     H.assert_bf16_close(H.to_np(Yp), refp, False, f"cyclic proj q={q} M={M}")
+
+
+def test_pilot_tensor_square_law_and_interval_schedule():
+    """The law and shape of the paper's pilot FFN projections: Q_2 (x) Q_2 (36 block products,
+    9/16 of the dense MACs), D = 768 = 4 x 192, F = 1536 = 4 x 384, interval schedule."""
+    wl = synth.pilot_ffn(integer=True)
+    keep = oracle.support(4, "q2pow")
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", table="q2pow")
+    assert proj.gemm_count() == 36
+    counts = np.bincount(wl.types, minlength=4)
+    assert proj.macs(counts.tolist()) * 16 == 9 * wl.M * wl.D * wl.F
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, keep=keep))
+    wl = synth.pilot_ffn()
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="q2pow")
+    Yf = _run_ffn(wl, ffn, torch.float32)
+    rows = _sample_rows(wl, 160, seed=3)
+    ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+    H.assert_bf16_close(H.to_np(Yf[torch.from_numpy(rows).cuda()]), ref, False, "pilot tensor-square FFN")
+    # decode step of the same layer
+    d = synth.pilot_ffn(M=8)
+    d.types = synth.interval_types(8, 4, 768, start=190)      # positions 190..197 straddle a type boundary
+    Yd = _run_ffn(d, ffn, torch.float32)
+    refd = oracle.ffn(d.X, d.types, d.W_up, d.W_down, d.d_widths, d.f_widths, keep=keep)
+    H.assert_bf16_close(H.to_np(Yd), refd, False, "pilot decode")

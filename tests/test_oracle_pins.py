@@ -303,3 +303,20 @@ def test_empty_and_missing_types():
     X = np.ones((3, 4))
     Y = oracle.proj(X, [1, 1, 1], np.ones((4, 6)), [2, 2], [3, 3])  # no type-0 rows at all
     assert np.array_equal(Y, np.tile([4, 4, 4, 2, 2, 2], (3, 1)).astype(float))
+
+
+def test_tensor_power_support_is_kronecker_product_of_q2():
+    """B(alpha, delta) of Q_2^{(x)L} factorises bit by bit into the q=2 rule (appendix on the
+    tensor-square candidate): keep_L[a,d,b] = prod_bits keep_2[a_bit, d_bit, b_bit]."""
+    k2 = oracle.support(2)
+    for L in (1, 2, 3):
+        q = 2 ** L
+        kL = oracle.support(q, "q2pow")
+        for a, d, b in itertools.product(range(q), repeat=3):
+            want = 1
+            for bit in range(L):
+                want *= int(k2[(a >> bit) & 1, (d >> bit) & 1, (b >> bit) & 1])
+            assert int(kL[a, d, b]) == want
+        # per-type product count 3^L, total 6^L; strictly between the direct law and dense for L >= 2
+        assert all(int(kL[a].sum()) == 3 ** L for a in range(q))
+    assert oracle.gemm_count(oracle.support(4, "q2pow")) == 36 > oracle.gemm_count(oracle.support(4)) == 28
