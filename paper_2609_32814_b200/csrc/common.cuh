@@ -115,6 +115,7 @@ struct ProjArgs {
   // original row = (bucketed row - i*M/q)*q + i.  0 = off.
   int a_cyclic_rows;
   int out_cyclic_rows;
+  int dbg;                // experiment switches, honoured only in -DALGPROJ_TRACE builds
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;

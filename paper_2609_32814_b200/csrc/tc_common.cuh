@@ -123,18 +123,31 @@ __device__ __forceinline__ float gelu_tanh(float z) {
 // Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
 // it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
 __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjArgs &a, int64_t out_row, int col) {
+#ifdef ALGPROJ_TRACE
+  if (a.dbg & 4) return;
+#endif
   if (a.bias) {
     const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
 #pragma unroll
     for (int x = 0; x < 32; ++x) f[x] += __bfloat162float(__ldg(b + x));
   }
+#ifdef ALGPROJ_TRACE
+  if (a.act == ALG_ACT_GELU_ERF && !(a.dbg & 2)) {
+#else
   if (a.act == ALG_ACT_GELU_ERF) {
+#endif
 #pragma unroll
     for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
   } else if (a.act == ALG_ACT_GELU_TANH) {
 #pragma unroll
     for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
   }
+#ifdef ALGPROJ_TRACE
+  if (a.dbg & 1) {
+    if (f[0] == 123.456f) ((float *)a.Y)[0] = f[1];
+    return;
+  }
+#endif
   if (a.y_bf16) {
     uint32_t w[16];
 #pragma unroll
