@@ -95,7 +95,8 @@ alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
 alg_status_t alg_proj_destroy(alg_proj_t h);
 
 /* Bytes of device scratch a forward call with at most max_M rows needs (row permutation,
- * bucket offsets, tile list, and -- on the tensor-core path -- the type-bucketed copy of X). */
+ * bucket offsets, and -- on the tensor-core path -- the type-bucketed copy of X).  The contents
+ * need no initialisation. */
 alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes);
 
 /* Y[M x N] = act( X[M x K] *_q W[K x N] + bias ).
@@ -105,7 +106,8 @@ alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes
  * workspace: >= alg_proj_workspace_bytes(h, M), 256-byte aligned.
  * bf16 pointers and leading dimensions must keep rows 16-byte aligned (multiples of 8
  * elements).  M = 0 is a successful no-op; a type with no rows is legal.
- * M <= 64 with bf16 runs the decode kernel, larger M the prefill kernels. */
+ * M <= 64 with bf16 runs the decode kernel (when its per-CTA weight slice fits shared memory),
+ * larger M the prefill kernels. */
 alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const int32_t *types,
                               int64_t M, const void *W, int64_t ldw, const void *bias,
                               alg_act_t act, void *Y, int64_t ldy, alg_dtype_t y_dtype,
@@ -118,8 +120,8 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
  * memory was handed out once at start-up to a pool it may not grow, a plug-in called from a
  * host framework that forbids cudaMalloc / cudaFree on its hot path because they synchronise
  * the whole device, or a caller that simply has no allocator to hand.  Such callers still pass
- * their own X, types, W, bias and Y; only the scratch (row permutation, bucket offsets, tile
- * list, type-bucketed copy of X) comes from the library, from a fixed array of
+ * their own X, types, W, bias and Y; only the scratch (row permutation, bucket offsets,
+ * type-bucketed copy of X) comes from the library, from a fixed array of
  * ALG_STATIC_SCRATCH_BYTES that is part of the loaded library image on every GPU and stays
  * there until the process exits.
  *

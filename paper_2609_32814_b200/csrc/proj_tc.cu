@@ -1,6 +1,6 @@
 // Grouped bf16 GEMM over the interaction table for sm_100a: TMA-fed shared-memory tiles,
-// tcgen05.mma with the accumulator in tensor memory, persistent CTAs walking a device-built
-// tile list in a static boustrophedon order.
+// tcgen05.mma with the accumulator in tensor memory, persistent CTAs walking the tile
+// enumeration (tile_map.cuh) in a static boustrophedon order.
 //
 // One output tile = 128 rows of one row type i  x  TILE_N columns of one output group j.  All
 // kept products of that block (x_k W_kj for k in B(i,j); Eq. recursive-row-action -- for the
@@ -10,9 +10,10 @@
 //
 // Operands: A = type-bucketed rows, K-contiguous (K-major), 128B-swizzled 128x64 tiles.
 //           B = the canonical K x N bank, N-contiguous (MN-major), 64(k) x 64(n) swizzled boxes.
-// Warp roles (320 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocator + MMA
-// issuer (one lane), warps 2..9 = epilogue (TMEM -> registers -> bias / activation -> row
-// scatter to global; two warps per TMEM lane quadrant, each taking half the columns).  The
+// Warp roles (352 threads): warp 0 = TMA producer of A (one lane), warp 10 = TMA producer of B,
+// warp 1 = TMEM allocator + MMA issuer (one lane), warps 2..9 = epilogue (TMEM -> registers ->
+// bias / activation -> row scatter to global; two warps per TMEM lane quadrant, each taking half
+// the columns).  The
 // accumulator is double buffered in TMEM so the epilogue of tile t overlaps the main loop of
 // tile t+1.
 //

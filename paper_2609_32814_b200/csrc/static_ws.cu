@@ -6,8 +6,8 @@
 
 namespace {
 
-// Scratch of every alg_proj_forward_static call on a device: row permutation, bucket offsets,
-// tile list and the type-bucketed copy of X.  Each GPU that loads the library holds these
+// Scratch of every alg_proj_forward_static call on a device: row permutation, bucket offsets
+// and the type-bucketed copy of X.  Each GPU that loads the library holds these
 // 8 MiB until the process exits.
 constexpr size_t kStaticScratchBytes = ALG_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
