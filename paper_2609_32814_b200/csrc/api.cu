@@ -125,24 +125,25 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   // tile classes sorted by cost = K length x tile width, most expensive first (stable)
   {
     const int tn = tile_n_of(p);
-    const bool split = use_tc(p) && p.pair_kernel;
-    std::vector<std::pair<long long, int>> order;  // (-cost, class)
+    struct Item { long long cost; ClassRec rec; };
+    std::vector<Item> order;
     for (int pr = 0; pr < q * q; ++pr) {
       long long len = 0;
       for (int k = 0; k < q; ++k)
         if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
-      const int width = p.r[pr % q];
-      if (split) {
-        if (width / tn) order.push_back({-len * tn, pr * 2});
-        if (width % tn) order.push_back({-len * (width % tn), pr * 2 + 1});
-      } else {
-        order.push_back({-len * std::min(tn, width), pr * 2});
+      const int i = pr / q, j = pr % q, width = p.r[j];
+      for (int t0 = 0; t0 < width / tn; t0 += 4095) {  // n_tiles has 12 bits
+        const int nt = std::min(4095, width / tn - t0);
+        order.push_back({len * tn, ClassRec{(unsigned)i, (unsigned)j, (unsigned)tn, (unsigned)nt, p.tab.ro[j] + t0 * tn}});
       }
+      if (width % tn)
+        order.push_back({len * (width % tn),
+                         ClassRec{(unsigned)i, (unsigned)j, (unsigned)(width % tn), 1u, p.tab.ro[j] + (width / tn) * tn}});
     }
-    std::stable_sort(order.begin(), order.end(), [](const std::pair<long long, int> &x,
-                                                    const std::pair<long long, int> &y) { return x.first < y.first; });
+    if ((int)order.size() > kMaxClasses) return ALG_ERR_INVALID_ARG;
+    std::stable_sort(order.begin(), order.end(), [](const Item &x, const Item &y) { return x.cost > y.cost; });
     p.tab.n_classes = (int)order.size();
-    for (size_t e = 0; e < order.size(); ++e) p.tab.class_order[e] = order[e].second;
+    for (size_t e = 0; e < order.size(); ++e) p.tab.cls[e] = order[e].rec;
     p.tab.n_pairs = q * q;
   }
 
@@ -223,11 +224,10 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   if (a.st.valid) {
     for (int e = 0; e <= p.q; ++e) a.st.so[e] = p.tab.so[e], a.st.ro[e] = p.tab.ro[e];
     for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = p.tab.keep[e];
-    for (int e = 0; e < p.tab.n_classes; ++e) a.st.class_order[e] = p.tab.class_order[e];
+    for (int e = 0; e < p.tab.n_classes; ++e) a.st.cls[e] = p.tab.cls[e];
   }
   a.geom.tile_m = tile_m_of(p);
-  a.geom.tile_n = tile_n_of(p);
-  a.geom.split_rem = use_tc(p) && p.pair_kernel;
+  a.geom.tile_m_log2 = a.geom.tile_m == 256 ? 8 : a.geom.tile_m == 128 ? 7 : 6;
   a.q = p.q;
   a.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
   a.W = W;

@@ -19,6 +19,17 @@ inline int bucket_chunk_rows(int64_t M) {
   return (int)(256 * (iters > 0 ? iters : 1));
 }
 
+// A tile class = all tiles of one (row type i, output group j) pair that have the same width: the
+// full-width tiles of the group, or its single narrower remainder tile.  Everything here is known
+// on the host; only the number of 128- or 256-row tiles of type i depends on the batch.
+struct ClassRec {
+  unsigned i : 5, j : 5;
+  unsigned cols : 10;     // width of every tile of the class
+  unsigned n_tiles : 12;  // tiles of this class per m-tile (wider groups are cut into several classes)
+  int col0;               // absolute first column of the class's first tile
+};
+static_assert(sizeof(ClassRec) == 8 && kMaxQ <= 32, "ClassRec packs a type index into 5 bits");
+
 // Interaction table of one projection as the kernels see it (device memory, owned by a handle).
 struct DevTable {
   int q;
@@ -26,10 +37,9 @@ struct DevTable {
   int so[kMaxQ + 1];           // prefix sums of the input group widths  (S_k = [so[k], so[k+1]))
   int ro[kMaxQ + 1];           // prefix sums of the output group widths (R_j = [ro[j], ro[j+1]))
   uint32_t keep[kMaxPairs];    // keep[i*q+j] bit k set  <=>  k in B(i,j)
-  // Tile classes (pair*2 + w; w = 0: tiles of the full tile width, w = 1: the narrower remainder
-  // tile of the output group), sorted by cost = K length x tile width, most expensive first.
+  // Tile classes, sorted by cost = K length x tile width, most expensive first (see ClassRec).
   int n_classes;
-  int class_order[kMaxClasses];
+  ClassRec cls[kMaxClasses];
 };
 
 // One output tile of the grouped GEMM: rows [row0, row0+rows) of the type-bucketed row order
@@ -49,9 +59,8 @@ struct WsHeader {
 static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
 
 struct TileGeom {
-  int tile_m;
-  int tile_n;
-  int split_rem;  // 1: full tile_n-wide tiles plus one narrower remainder tile; 0: ceil(width / tile_n) tiles
+  int tile_m;        // rows per tile (a power of two)
+  int tile_m_log2;
 };
 
 struct BucketArgs {
@@ -83,7 +92,7 @@ struct SmallTable {
   int so[kParamQ + 1];
   int ro[kParamQ + 1];
   uint32_t keep[kParamQ * kParamQ];
-  int class_order[2 * kParamQ * kParamQ];
+  ClassRec cls[2 * kParamQ * kParamQ];
 };
 
 struct ProjArgs {

@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
   __shared__ float As[TK][TM + 1];
   __shared__ float Bs[TK][TN];
   __shared__ int s_rows[TM];
-  __shared__ __align__(16) unsigned char s_map[sizeof(TileMap) + (2 * kMaxClasses + 1) * sizeof(int)];
+  extern __shared__ __align__(16) unsigned char s_map[];  // tile_map_bytes(n_classes)
   TileMap *tm = reinterpret_cast<TileMap *>(s_map);
   const DevTable *__restrict__ tab = a.tab;
   const int q = a.q;
@@ -115,8 +115,15 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
 
 cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st) {
   const int grid = 148 * 4;
-  if (in_bf16) proj_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
-  else proj_simt_kernel<float><<<grid, 256, 0, st>>>(a);
+  const size_t map_bytes = tile_map_bytes(a.n_classes);
+  static bool attr = false;
+  if (!attr) {
+    cudaFuncSetAttribute(proj_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    cudaFuncSetAttribute(proj_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    attr = true;
+  }
+  if (in_bf16) proj_simt_kernel<__nv_bfloat16><<<grid, 256, map_bytes, st>>>(a);
+  else proj_simt_kernel<float><<<grid, 256, map_bytes, st>>>(a);
   count_launch(1);
   return cudaGetLastError();
 }

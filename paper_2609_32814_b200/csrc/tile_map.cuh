@@ -1,13 +1,12 @@
 // Tile enumeration of the grouped GEMM, computed inside the GEMM kernels.
 //
-// Every CTA builds, once at start-up and in shared memory, the prefix table "tiles before tile
-// class c" from the bucket offsets (row counts per type, which only exist on the device) and the
-// handle's class order (most expensive class first), and then decodes tile indices on the fly.
-// No tile list is ever written to global memory and no extra kernel is needed to produce one.
-//
-// A tile class is (pair (i,j), w): w = 0 -> tiles of the full tile width inside output group j,
-// w = 1 -> the narrower remainder tile of that group (only when the kernel splits remainders).
-// Inside a class tiles are ordered m-tile major, n-tile fastest, so neighbours share their rows.
+// Tile classes (ClassRec: pair (i,j), tiles per m-tile, first column, tile width; 8 bytes) are fixed per
+// handle and sorted on the host, most expensive first.  Only the number of m-tiles of every row
+// type depends on the batch: each CTA turns the bucket offsets (device memory, or arithmetic for
+// the cyclic schedule) into the prefix table "tiles before class c" in shared memory and decodes
+// tile indices with one binary search and one division.  No tile list is ever written to global
+// memory and no extra kernel is needed to produce one.  Inside a class tiles are ordered m-tile
+// major, n-tile fastest, so neighbours share their rows.
 #pragma once
 
 #include "common.cuh"
@@ -18,21 +17,16 @@ struct TileMap {
   int n_classes;
   int total;                       // number of tiles
   int q;
+  int pad_[3];
   int offsets[kMaxQ + 2];          // bucket offsets (first bucketed row of each type)
-  int ro[kMaxQ + 1];               // output group offsets
-  // followed in shared memory by: int cls[n_classes]; int prefix[n_classes + 1];
-  __device__ __forceinline__ int *cls() { return reinterpret_cast<int *>(this + 1); }
-  __device__ __forceinline__ int *prefix() { return cls() + n_classes; }
+  // followed in shared memory by: ClassRec cls[n_classes]; int prefix[n_classes + 1];
+  __device__ __forceinline__ ClassRec *cls() { return reinterpret_cast<ClassRec *>(this + 1); }
+  __device__ __forceinline__ int *prefix() { return reinterpret_cast<int *>(cls() + n_classes); }
 };
+static_assert(sizeof(TileMap) % 16 == 0, "class records stay 16-byte aligned behind the header");
 
 __host__ __device__ inline size_t tile_map_bytes(int n_classes) {
-  return sizeof(TileMap) + (size_t)(2 * n_classes + 1) * sizeof(int);
-}
-
-__device__ __forceinline__ int tile_map_n_tiles(const TileGeom &g, int cls, int width) {
-  const int w = cls & 1;
-  if (!g.split_rem) return w == 0 ? ceil_div(width, g.tile_n) : 0;
-  return w == 0 ? width / g.tile_n : ((width % g.tile_n) ? 1 : 0);
+  return sizeof(TileMap) + (size_t)n_classes * sizeof(ClassRec) + (size_t)(n_classes + 1) * sizeof(int);
 }
 
 // Called by all threads of the CTA (blockDim.x >= 32).  `offsets` = device bucket offsets, or
@@ -42,14 +36,14 @@ __device__ inline void tile_map_build(TileMap *tm, const DevTable *tab, const Sm
   if (threadIdx.x == 0) tm->n_classes = nc, tm->q = q;
   for (int t = threadIdx.x; t <= q + 1; t += blockDim.x)
     tm->offsets[t] = offsets ? offsets[t] : (t <= q ? t * cyclic_rows : M);
-  for (int t = threadIdx.x; t <= q; t += blockDim.x) tm->ro[t] = st.valid ? st.ro[t] : tab->ro[t];
   __syncthreads();
-  int *cls = tm->cls(), *prefix = tm->prefix();
+  ClassRec *cls = tm->cls();
+  int *prefix = tm->prefix();
   for (int c = threadIdx.x; c < nc; c += blockDim.x) {
-    const int id = st.valid ? st.class_order[c] : tab->class_order[c];
-    const int pair = id >> 1, i = pair / q, j = pair % q;
-    cls[c] = id;
-    prefix[c] = ceil_div(tm->offsets[i + 1] - tm->offsets[i], g.tile_m) * tile_map_n_tiles(g, id, tm->ro[j + 1] - tm->ro[j]);
+    const ClassRec r = st.valid ? st.cls[c] : tab->cls[c];
+    cls[c] = r;
+    const int rows = tm->offsets[r.i + 1] - tm->offsets[r.i];
+    prefix[c] = ((rows + g.tile_m - 1) >> g.tile_m_log2) * (int)r.n_tiles;
   }
   __syncthreads();
   if (threadIdx.x < 32) {  // exclusive scan of the counts by one warp
@@ -86,18 +80,14 @@ __device__ __forceinline__ TileRec tile_map_decode(TileMap *tm, const TileGeom &
     const int mid = (lo + hi) >> 1;
     if (prefix[mid] <= idx) lo = mid; else hi = mid;
   }
-  const int id = tm->cls()[lo];
-  const int q = tm->q, pair = id >> 1, i = pair / q, j = pair % q;
-  const int width = tm->ro[j + 1] - tm->ro[j];
-  const int n_tiles = tile_map_n_tiles(g, id, width);
+  const ClassRec r = tm->cls()[lo];
   const int loc = idx - prefix[lo];
-  const int mt = loc / n_tiles, nt = loc % n_tiles;
-  const int rows = tm->offsets[i + 1] - tm->offsets[i];
-  const int c0 = (g.split_rem && (id & 1)) ? (width / g.tile_n) * g.tile_n : nt * g.tile_n;
-  rec.row0 = tm->offsets[i] + mt * g.tile_m;
-  rec.rows = min(g.tile_m, rows - mt * g.tile_m);
-  rec.pair = pair | (min(g.tile_n, width - c0) << 16);
-  rec.n0 = tm->ro[j] + c0;
+  const int ntl = (int)r.n_tiles, mt = loc / ntl, nt = loc - mt * ntl;
+  const int rows = tm->offsets[r.i + 1] - tm->offsets[r.i];
+  rec.row0 = tm->offsets[r.i] + (mt << g.tile_m_log2);
+  rec.rows = min(g.tile_m, rows - (mt << g.tile_m_log2));
+  rec.pair = ((int)r.i * tm->q + (int)r.j) | ((int)r.cols << 16);
+  rec.n0 = r.col0 + nt * (int)r.cols;
   return rec;
 }
 
@@ -109,21 +99,22 @@ __device__ __forceinline__ TileRec tile_map_decode(TileMap *tm, const TileGeom &
 // (Giving each worker a contiguous run of tiles instead was measured 10-15 % slower: the
 // concurrent working set then spreads over the whole problem.)
 //
-// The tile sequence of one persistent worker, decoded once by all threads of the CTA so that the
-// single-thread roles (TMA producer, MMA issuer) only read a 16-byte record per tile: their
-// instruction streams share a scheduler with busy epilogue warps, which makes scalar work in them
-// several times more expensive than it looks.  Rounds beyond `cap` are decoded on the fly.
+// The tile sequence of one persistent worker is decoded once by the threads of the CTA (one round
+// per thread), so that the single-thread roles (TMA producer, MMA issuer) only read a 16-byte
+// record per tile.  Rounds beyond `cap` are decoded on the fly.
 __device__ __forceinline__ int snake_index(int round, int worker, int n_workers) {
   return round * n_workers + ((round & 1) ? (n_workers - 1 - worker) : worker);
 }
 __device__ inline void tile_seq_build(TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int worker,
                                       int n_workers) {
-  for (int r = threadIdx.x; r < cap; r += blockDim.x) recs[r] = tile_map_decode(tm, g, snake_index(r, worker, n_workers));
+  // rounds this worker can have at all: ceil(total / n_workers)
+  const int rounds = min(cap, (tm->total + n_workers - 1) / n_workers + 1);
+  for (int r = threadIdx.x; r < rounds; r += blockDim.x) recs[r] = tile_map_decode(tm, g, snake_index(r, worker, n_workers));
   __syncthreads();
 }
 __device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int round,
                                                 int worker, int n_workers) {
-  if (round < cap) return recs[round];
+  if (round < cap && round <= (tm->total + n_workers - 1) / n_workers) return recs[round];
   return tile_map_decode(tm, g, snake_index(round, worker, n_workers));
 }
 
