@@ -244,6 +244,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.b_3d = 0;
+  a.y_tma = 0;
   a.dbg = std::getenv("ALGPROJ_DBG") ? atoi(std::getenv("ALGPROJ_DBG")) : 0;
   a.trace = g_trace;
   a.trace_cap = g_trace_cap;

@@ -125,7 +125,8 @@ struct ProjArgs {
   int a_cyclic_rows;
   int out_cyclic_rows;
   int dbg;                // experiment switches, honoured only in -DALGPROJ_TRACE builds
-  int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
+  int b_3d;
+  int y_tma;          // 0: direct stores; 2 / 3: tiled stores through a 2-D / 3-D (cyclic) map of Y               // B tensor map is the 3-D chunked view (one copy per stage)
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;
 };

@@ -22,6 +22,7 @@
 #include <cudaTypedefs.h>
 
 #include <cstdlib>
+#include <cstring>
 
 #include "tc_common.cuh"
 
@@ -41,6 +42,7 @@ struct Ctl {
   // interaction table, copied once per CTA so no role waits on global metadata at a tile start
   int so[kMaxQ + 1];
   uint32_t keep[kMaxPairs];
+  uint16_t nkb[kMaxPairs];  // K blocks per tile of a pair
 };
 
 // Bounded wait. Returns false when the CTA is aborting.
@@ -63,7 +65,6 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctl *ctl
   if (mbar_try_wait(bar, parity)) return true;
   return wait_slow(bar, parity, ctl, status);
 }
-
 constexpr int kSeqCap = 224;  // precomputed tile records per CTA
 #ifndef ALGPROJ_EPI_WARPS
 #define ALGPROJ_EPI_WARPS 8
@@ -82,6 +83,7 @@ struct Cfg {
   static constexpr int kAccStride = TILE_N <= 128 ? 128 : 256;   // TMEM columns between the two accumulators
   static constexpr int kTmemCols = 2 * kAccStride;
   static constexpr int kFixedSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + kSeqCap * 16 + 16 + 1024;  // + tile map
+  static constexpr int kStoreBufBytes = 32 * 64;                  // per epilogue warp: 32 rows x 32 bf16 columns
   static constexpr int kHalf = TILE_N / (kEpiWarps / 4);          // columns per epilogue warp
   // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N, M=128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
@@ -90,17 +92,28 @@ struct Cfg {
 
 template <int TILE_N>
 __global__ void __launch_bounds__(kThreads, 1)
-proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
+proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmY, const ProjArgs a) {
   using C = Cfg<TILE_N>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  Ctl *ctl = (Ctl *)(smem + C::kStages * C::kStageBytes);
+  // optional staging buffers of the epilogue warps (tiled stores) sit between the stages and the control block
+  uint8_t *store_buf = smem + C::kStages * C::kStageBytes;
+  Ctl *ctl = (Ctl *)(store_buf + (a.y_tma ? kEpiWarps * C::kStoreBufBytes : 0));
   TileRec *recs = (TileRec *)(ctl + 1);
   TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
   const int q = a.q;
   [[maybe_unused]] int tr_n = 0;
+#ifdef ALGPROJ_TRACE
+  if (a.trace && threadIdx.x == 0) {  // whole-CTA window: global timer and SM clock at entry
+    unsigned long long gt;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 0] = (long long)gt;
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 2] = clock64();
+  }
+#endif
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -115,9 +128,17 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    if (a.y_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmY) : "memory");
   }
   for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
   for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
+  for (int e = threadIdx.x; e < q * q; e += kThreads) {
+    const uint32_t mask = a.st.valid ? a.st.keep[e] : tab->keep[e];
+    int n = 0;
+    for (int k = 0; k < q; ++k)
+      if ((mask >> k) & 1u) n += ((a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k])) / kTcBlockK;
+    ctl->nkb[e] = (uint16_t)n;
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"((uint32_t)C::kTmemCols)
@@ -130,99 +151,128 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
-  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x, gridDim.x);
+  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x, gridDim.x, ctl->nkb);  // (tile_map_build has synchronised ctl->nkb)
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
 
+  // The producer and MMA roles run warp-uniformly: all 32 lanes execute the loops and the waits,
+  // and one elected lane issues the copy / MMA / commit instructions.  In a single-lane
+  // (divergent) branch the compiler has to stage every operand of those instructions through
+  // vector registers, which costs the issuing thread ~500 cycles per K block -- the whole budget
+  // of a 128x256x64 block -- against ~290 cycles when the operands live in uniform registers.
+  // Loop bounds read from shared memory are broadcast with a shuffle so that they count as
+  // warp-uniform.
   if (warp == 0 || warp == kProducerWarpB) {
-    // ---------------- TMA producers (one lane each): warp 0 loads A, the last warp loads B ----------------
+    // ---------------- TMA producers: warp 0 loads A, the last warp loads B ----------------
     // Issuing a tiled load occupies the thread while the copy engine expands the box; with two
-    // issuing threads a freed stage is refilled sooner, which shortens the
+    // issuing warps a freed stage is refilled sooner, which shortens the
     // load -> MMA -> free -> load round trip that bounds the bytes in flight.
-    if (lane == 0) {
-      const bool loads_a = warp == 0;
-      int stage = 0, round = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
-      while (ok && rec.row0 >= 0) {
-        ++round;
-        if (loads_a) ALG_TRACE(0, 1);
-        const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
-        const int type_i = (rec.pair & 0xFFFF) / q;
-        const int a_row = a.a_cyclic_rows ? rec.row0 - type_i * a.a_cyclic_rows : rec.row0;
-        for (int k = 0; k < q && ok; ++k) {
-          if (!((mask >> k) & 1u)) continue;
-          const int k_end = ctl->so[k + 1];
-          for (int k0 = ctl->so[k]; k0 < k_end; k0 += kTcBlockK) {
-            ok = wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, a.status);
-            if (!ok) break;
-            const uint32_t bar = smem_u32(&ctl->full[stage]);
-            const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
+    const bool loads_a = warp == 0;
+    int stage = 0, round = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    const uint32_t smem0 = smem_u32(smem);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
+    while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
+      ++round;
+      if (loads_a && lane == 0) ALG_TRACE(0, 1);
+      const int pair = __shfl_sync(0xffffffffu, rec.pair & 0xFFFF, 0);
+      const int row0 = __shfl_sync(0xffffffffu, rec.row0, 0);
+      const int n0 = __shfl_sync(0xffffffffu, rec.n0, 0);
+      const uint32_t mask = __shfl_sync(0xffffffffu, ctl->keep[pair], 0);
+      const int type_i = pair / q;
+      const int a_row = a.a_cyclic_rows ? row0 - type_i * a.a_cyclic_rows : row0;
+      for (int k = 0; k < q && ok; ++k) {
+        if (!((mask >> k) & 1u)) continue;
+        const int k_begin = __shfl_sync(0xffffffffu, ctl->so[k], 0);
+        const int k_end = __shfl_sync(0xffffffffu, ctl->so[k + 1], 0);
+        for (int k0 = k_begin; k0 < k_end; k0 += kTcBlockK) {
+          ok = __all_sync(0xffffffffu, wait_bar(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, a.status));
+          if (!ok) break;
+          const uint32_t bar = full0 + 8u * (uint32_t)stage;
+          const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
+          if (elect_one()) {
+#ifdef ALGPROJ_TRACE
+            if (a.dbg & 24) {  // timing experiments: 8 = no A loads, 16 = no B loads (results are wrong)
+              if (loads_a) {
+                const uint32_t bytes = ((a.dbg & 8) ? 0u : (uint32_t)C::kABytes) + ((a.dbg & 16) ? 0u : (uint32_t)C::kBBytes);
+                if (bytes) mbar_expect_tx(bar, bytes); else mbar_arrive(bar);
+                if (!(a.dbg & 8)) {
+                  if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
+                  else tma_load_2d(sa, &tmA, bar, k0, a_row);
+                }
+              } else if (!(a.dbg & 16)) {
+                tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
+              }
+            } else
+#endif
             if (loads_a) {
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
               else tma_load_2d(sa, &tmA, bar, k0, a_row);
             } else if (a.b_3d) {
-              tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, rec.n0 >> 6);  // all 64-column chunks in one box
+              tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);  // all 64-column chunks in one box
             } else {
 #pragma unroll
               for (int c = 0; c < TILE_N / 64; ++c)
-                tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, rec.n0 + c * 64, k0);
+                tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, n0 + c * 64, k0);
             }
-            if (++stage == C::kStages) stage = 0, phase ^= 1u;
           }
+          __syncwarp();
+          if (++stage == C::kStages) stage = 0, phase ^= 1u;
         }
-        if (loads_a) ALG_TRACE(0, 2);
-        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
       }
+      if (loads_a && lane == 0) ALG_TRACE(0, 2);
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x, gridDim.x, ctl->nkb);
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer (one lane) ----------------
-    if (lane == 0) {
-      int stage = 0, acc = 0, round = 0;
-      uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
-      while (ok && rec.row0 >= 0) {
-        ++round;
-        ALG_TRACE(1, 1);
-        ok = wait_bar(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, ctl, a.status);
+    // ---------------- MMA issuer ----------------
+    int stage = 0, acc = 0, round = 0;
+    uint32_t phase = 0, acc_phase = 0;
+    bool ok = true;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
+    const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, 1024);
+    const uint64_t db0 = make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
+    while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
+      ++round;
+      if (lane == 0) ALG_TRACE(1, 1);
+      // All kept products of the block run back to back into one accumulator, so this warp only
+      // needs their total number of K blocks (upper half of rec.rows).
+      const int n_kb = __shfl_sync(0xffffffffu, (int)((uint32_t)rec.rows >> 16), 0);
+      ok = __all_sync(0xffffffffu, wait_bar(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
+      if (!ok) break;
+      if (lane == 0) ALG_TRACE(1, 2);
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * C::kAccStride);
+      for (int kb = 0; kb < n_kb; ++kb) {
+        ok = __all_sync(0xffffffffu, wait_bar(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
         if (!ok) break;
-        ALG_TRACE(1, 2);
+        if (kb == 0 && lane == 0) ALG_TRACE(1, 3);
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * C::kAccStride);
-        const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
-        uint32_t accumulate = 0;
-        for (int k = 0; k < q && ok; ++k) {
-          if (!((mask >> k) & 1u)) continue;
-          const int n_kb = (ctl->so[k + 1] - ctl->so[k]) / kTcBlockK;
-          for (int kb = 0; kb < n_kb; ++kb) {
-            ok = wait_bar(smem_u32(&ctl->full[stage]), phase, ctl, a.status);
-            if (!ok) break;
-            if (!accumulate) ALG_TRACE(1, 3);
-            tc_fence_after();
-            const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
-            const uint64_t da = make_smem_desc(sa, 16, 1024);
-            const uint64_t db = make_smem_desc(sa + C::kABytes, C::kBChunkBytes, 1024);
+        const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        if (elect_one()) {
+          // A: 16 k-elements = 32 bytes inside the swizzle atom; B: 16 k-rows = two 8-row groups
+          tc_mma_bf16(d_tmem, da, db, C::kIdesc, kb ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < kTcBlockK / 16; ++kk) {
-              // A: 16 k-elements = 32 bytes inside the swizzle atom; B: 16 k-rows = two 8-row groups
-              tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), C::kIdesc, accumulate);
-              accumulate = 1;
-            }
-            tc_commit(smem_u32(&ctl->empty[stage]));
-            if (++stage == C::kStages) stage = 0, phase ^= 1u;
-          }
+          for (int kk = 1; kk < kTcBlockK / 16; ++kk)
+            tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), C::kIdesc, 1u);
+          tc_commit(empty0 + 8u * (uint32_t)stage);
         }
-        if (!ok) break;
-        tc_commit(smem_u32(&ctl->tmem_full[acc]));
-        ALG_TRACE(1, 4);
-        if (++acc == 2) acc = 0, acc_phase ^= 1u;
-        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
+        __syncwarp();
+        if (++stage == C::kStages) stage = 0, phase ^= 1u;
       }
+      if (!ok) break;
+      if (elect_one()) tc_commit(tfull0 + 8u * (uint32_t)acc);
+      __syncwarp();
+      if (lane == 0) ALG_TRACE(1, 4);
+      if (++acc == 2) acc = 0, acc_phase ^= 1u;
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x, gridDim.x, ctl->nkb);
     }
   } else {
     // ---------------- epilogue: warp e handles TMEM lanes [32*(warp%4), +32), column half e/4 ----
@@ -231,12 +281,13 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = e >> 2;
     int acc = 0, round = 0;
     uint32_t acc_phase = 0;
-    TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x, gridDim.x);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
     while (rec.row0 >= 0) {
       ++round;
       const int r = quad * 32 + lane;
       int64_t out_row = -1;
-      if (r < rec.rows) {
+      const int tile_rows = rec.rows & 0xFFFF;
+      if (r < tile_rows) {
         if (a.out_cyclic_rows) {
           const int i = (rec.pair & 0xFFFF) / q;
           out_row = (int64_t)(rec.row0 + r - i * a.out_cyclic_rows) * q + i;
@@ -252,6 +303,44 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t taddr =
           tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * C::kAccStride + half * C::kHalf);
       const int col_base = rec.n0 + half * C::kHalf;
+      // Tiled stores when this warp's 32 rows are all rows of the tile and the output is
+      // contiguous or cyclic: the bf16 row segments go through a 2 KB staging buffer (64-byte
+      // swizzle, conflict-free 16-byte writes) and leave as one bulk tensor store per 32 x 32
+      // block, instead of 64 sector requests from the load/store unit.
+      const bool staged = a.y_tma && quad * 32 + 32 <= tile_rows;
+      if (staged) {
+        const uint32_t buf = smem_u32(store_buf + e * C::kStoreBufBytes);
+        const uint32_t my_row = buf + (uint32_t)lane * 64u;
+        const uint32_t sw = (uint32_t)((lane >> 1) & 3);
+        const int type_i = (rec.pair & 0xFFFF) / q;
+        const int y_row = rec.row0 + quad * 32 - (a.y_tma == 3 ? type_i * a.out_cyclic_rows : 0);
+#pragma unroll 1
+        for (int c0 = 0; c0 < C::kHalf; c0 += 32) {
+          uint32_t v[32];
+          tc_ld_32x32(taddr + (uint32_t)c0, v);
+          tc_wait_ld();
+          float f[32];
+#pragma unroll
+          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          finish_32(f, a, col_base + c0);
+          uint32_t w[16];
+          pack_bf16_32(f, w);
+          if (lane == 0) tma_store_wait_read();  // the previous block has left the buffer
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((((uint32_t)g) ^ sw) << 4)), "r"(w[g * 4]),
+                         "r"(w[g * 4 + 1]), "r"(w[g * 4 + 2]), "r"(w[g * 4 + 3])
+                         : "memory");
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (a.y_tma == 3) tma_store_3d(buf, &tmY, col_base + c0, type_i, y_row);
+            else tma_store_2d(buf, &tmY, col_base + c0, y_row);
+            tma_store_commit();
+          }
+        }
+      } else {
 #pragma unroll 1
       for (int c0 = 0; c0 < C::kHalf; c0 += 32) {
         uint32_t v[32];
@@ -264,16 +353,18 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           finish_and_store_32(f, a, out_row, col_base + c0);
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
       if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
-      rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x, gridDim.x);
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x, gridDim.x, ctl->nkb);
     }
   }
 
   // ---------------- teardown ----------------
+  if (a.y_tma && warp >= 2 && warp < 2 + kEpiWarps && lane == 0) tma_store_wait_all();
   __syncwarp();
   if (ctl->abort_flag) {
     // give copies that are still in flight time to land before shared memory is released
@@ -283,6 +374,14 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
+#ifdef ALGPROJ_TRACE
+  if (a.trace && threadIdx.x == 0) {
+    unsigned long long gt;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 1] = (long long)gt;
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 3] = clock64();
+  }
+#endif
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
@@ -301,9 +400,9 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int smem_bytes = C::kFixedSmemBytes + (int)tile_map_bytes(a.n_classes);
+  int smem_bytes = C::kFixedSmemBytes + (int)tile_map_bytes(a.n_classes);
   if (smem_bytes > 227 * 1024) return cudaErrorInvalidConfiguration;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmY;
   cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
   ProjArgs b = a;
@@ -311,6 +410,13 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   if (!b.b_3d) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
     if (e != cudaSuccess) return e;
+  }
+  b.y_tma = 0;
+  std::memset(&tmY, 0, sizeof(tmY));
+  if (smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && !std::getenv("ALGPROJ_NO_TMA_STORE") &&
+      make_map_y(&tmY, a) == cudaSuccess) {
+    b.y_tma = a.out_cyclic_rows ? 3 : 2;
+    smem_bytes += kEpiWarps * C::kStoreBufBytes;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(num_sms, 1, 1);
@@ -322,7 +428,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, tmY, b);
   count_launch(1);
   return e;
 }
@@ -372,6 +478,28 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.W), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t make_map_y(CUtensorMap *map, const ProjArgs &a) {
+  if (!a.y_bf16 || a.perm || ((uintptr_t)a.Y & 15u) || (a.ldy * 2) % 16 || a.N % 32) return cudaErrorInvalidValue;
+  cudaError_t e0 = tc_init();
+  if (e0 != cudaSuccess) return e0;
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r;
+  if (a.out_cyclic_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)a.N, (cuuint64_t)a.q, (cuuint64_t)a.out_cyclic_rows};
+    cuuint64_t strides[2] = {(cuuint64_t)a.ldy * 2, (cuuint64_t)a.ldy * 2 * (cuuint64_t)a.q};
+    cuuint32_t box[3] = {32, 1, 32};
+    r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, a.Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
+    cuuint64_t strides[1] = {(cuuint64_t)a.ldy * 2};
+    cuuint32_t box[2] = {32, 32};
+    r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 

@@ -184,7 +184,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0, round = 0;
       uint32_t phase = 0;
       bool ok = true;
-      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
+      TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
       while (ok && rec.row0 >= 0) {
         ++round;
         if (loads_a) ALG_TRACE(0, 1);
@@ -219,7 +219,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
         if (loads_a) ALG_TRACE(0, 2);
-        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
+        rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
       }
     }
   } else if (warp == 1) {
@@ -228,7 +228,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int stage = 0, acc = 0, round = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
+      TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
       while (ok && rec.row0 >= 0) {
         ++round;
         ALG_TRACE(1, 1);
@@ -267,7 +267,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tc2_commit_both(smem_u32(&ctl->tmem_full[acc]));
         ALG_TRACE(1, 4);
         if (++acc == 2) acc = 0, acc_phase ^= 1u;
-        rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
+        rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
       }
     }
   } else {
@@ -277,7 +277,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int half = e >> 2;
     int acc = 0, round = 0;
     uint32_t acc_phase = 0;
-    TileRec rec = tile_seq_get(recs, kSeqCap, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
     while (rec.row0 >= 0) {
       ++round;
       const int cols = rec.pair >> 16;
@@ -320,7 +320,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
-      rec = tile_seq_get(recs, kSeqCap, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
     }
   }
 

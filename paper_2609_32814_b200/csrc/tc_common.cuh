@@ -46,6 +46,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
       "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// One lane of the (converged) warp; the choice is uniform-friendly, unlike `lane == 0`.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -73,6 +83,22 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Tiled stores shared -> global (bulk async group of the issuing thread).
+__device__ __forceinline__ void tma_store_2d(uint32_t src_smem, const CUtensorMap *map, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src_smem),
+               "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(uint32_t src_smem, const CUtensorMap *map, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map),
+               "r"(src_smem), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
 // offsets (all >> 4), descriptor version 1, 128-byte swizzle.
@@ -120,12 +146,8 @@ __device__ __forceinline__ float gelu_tanh(float z) {
 }
 
 
-// Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
-// it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
-__device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjArgs &a, int64_t out_row, int col) {
-#ifdef ALGPROJ_TRACE
-  if (a.dbg & 4) return;
-#endif
+// Bias and activation on one row segment of 32 fp32 accumulator values.
+__device__ __forceinline__ void finish_32(float (&f)[32], const ProjArgs &a, int col) {
   if (a.bias) {
     const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
 #pragma unroll
@@ -142,6 +164,22 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
 #pragma unroll
     for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
   }
+}
+__device__ __forceinline__ void pack_bf16_32(const float (&f)[32], uint32_t (&w)[16]) {
+#pragma unroll
+  for (int h = 0; h < 16; ++h) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * h], f[2 * h + 1]);
+    w[h] = *(uint32_t *)&p;
+  }
+}
+
+// Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
+// it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
+__device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjArgs &a, int64_t out_row, int col) {
+#ifdef ALGPROJ_TRACE
+  if (a.dbg & 4) return;
+#endif
+  finish_32(f, a, col);
 #ifdef ALGPROJ_TRACE
   if (a.dbg & 1) {
     if (f[0] == 123.456f) ((float *)a.Y)[0] = f[1];
@@ -150,11 +188,7 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
 #endif
   if (a.y_bf16) {
     uint32_t w[16];
-#pragma unroll
-    for (int h = 0; h < 16; ++h) {
-      __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * h], f[2 * h + 1]);
-      w[h] = *(uint32_t *)&p;
-    }
+    pack_bf16_32(f, w);
     __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + out_row * a.ldy + col;
     if ((((uintptr_t)dst) & 31u) == 0) {  // 32-byte stores fill whole sectors
 #pragma unroll
@@ -206,6 +240,9 @@ cudaError_t make_map_2d_sw(CUtensorMap *map, const void *base, uint64_t inner, u
 // {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);
 cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks);
+// Output as the target of tiled stores of 32 columns x 32 rows (64-byte swizzle): plain rows, or
+// the type-strided view {N, q, M/q} for the cyclic schedule.  Fails when Y is not eligible.
+cudaError_t make_map_y(CUtensorMap *map, const ProjArgs &a);
 
 }  // namespace tc
 }  // namespace algproj

@@ -17,7 +17,8 @@ struct TileMap {
   int n_classes;
   int total;                       // number of tiles
   int q;
-  int pad_[3];
+  int seq_rounds;                  // tile records precomputed for this worker (the last one is the end marker)
+  int pad_[2];
   int offsets[kMaxQ + 2];          // bucket offsets (first bucketed row of each type)
   // followed in shared memory by: ClassRec cls[n_classes]; int prefix[n_classes + 1];
   __device__ __forceinline__ ClassRec *cls() { return reinterpret_cast<ClassRec *>(this + 1); }
@@ -105,17 +106,26 @@ __device__ __forceinline__ TileRec tile_map_decode(TileMap *tm, const TileGeom &
 __device__ __forceinline__ int snake_index(int round, int worker, int n_workers) {
   return round * n_workers + ((round & 1) ? (n_workers - 1 - worker) : worker);
 }
-__device__ inline void tile_seq_build(TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int worker,
-                                      int n_workers) {
-  // rounds this worker can have at all: ceil(total / n_workers)
+// `nkb_of_pair` (optional, shared memory): number of K blocks of the tiles of a pair; it is packed
+// into the upper half of TileRec::rows so that the MMA thread needs nothing but the record.
+__device__ __forceinline__ TileRec tile_seq_decode(TileMap *tm, const TileGeom &g, int round, int worker, int n_workers,
+                                                   const uint16_t *nkb_of_pair) {
+  TileRec rec = tile_map_decode(tm, g, snake_index(round, worker, n_workers));
+  if (nkb_of_pair && rec.row0 >= 0) rec.rows |= (int)nkb_of_pair[rec.pair & 0xFFFF] << 16;
+  return rec;
+}
+__device__ inline void tile_seq_build(TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int worker, int n_workers,
+                                      const uint16_t *nkb_of_pair = nullptr) {
+  // rounds this worker can have at all: ceil(total / n_workers), plus one record that marks the end
   const int rounds = min(cap, (tm->total + n_workers - 1) / n_workers + 1);
-  for (int r = threadIdx.x; r < rounds; r += blockDim.x) recs[r] = tile_map_decode(tm, g, snake_index(r, worker, n_workers));
+  if (threadIdx.x == 0) tm->seq_rounds = rounds;
+  for (int r = threadIdx.x; r < rounds; r += blockDim.x) recs[r] = tile_seq_decode(tm, g, r, worker, n_workers, nkb_of_pair);
   __syncthreads();
 }
-__device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int round,
-                                                int worker, int n_workers) {
-  if (round < cap && round <= (tm->total + n_workers - 1) / n_workers) return recs[round];
-  return tile_map_decode(tm, g, snake_index(round, worker, n_workers));
+__device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, TileMap *tm, const TileGeom &g, int round, int worker,
+                                                int n_workers, const uint16_t *nkb_of_pair = nullptr) {
+  if (round < tm->seq_rounds) return recs[round];
+  return tile_seq_decode(tm, g, round, worker, n_workers, nkb_of_pair);
 }
 
 }  // namespace algproj
