@@ -229,7 +229,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.geom.tile_m = tile_m_of(p);
   a.geom.tile_m_log2 = a.geom.tile_m == 256 ? 8 : a.geom.tile_m == 128 ? 7 : 6;
   a.q = p.q;
-  a.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
+  a.perm = (y_bucketed || cyclic) ? nullptr : (const int *)(ws + L.perm);  // cyclic outputs are addressed by arithmetic
   a.W = W;
   a.ldw = ldw;
   a.bias = bias;
