@@ -228,6 +228,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   }
   a.geom.tile_m = tile_m_of(p);
   a.geom.tile_m_log2 = a.geom.tile_m == 256 ? 8 : a.geom.tile_m == 128 ? 7 : 6;
+  a.geom.alternate = std::getenv("ALGPROJ_ALTERNATE") ? atoi(std::getenv("ALGPROJ_ALTERNATE")) : 0;
   a.q = p.q;
   a.perm = (y_bucketed || cyclic) ? nullptr : (const int *)(ws + L.perm);  // cyclic outputs are addressed by arithmetic
   a.W = W;
@@ -244,7 +245,7 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.b_3d = 0;
-  a.y_tma = 0;
+  a.y_staged = 0;
   a.dbg = std::getenv("ALGPROJ_DBG") ? atoi(std::getenv("ALGPROJ_DBG")) : 0;
   a.trace = g_trace;
   a.trace_cap = g_trace_cap;

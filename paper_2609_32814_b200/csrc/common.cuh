@@ -61,6 +61,7 @@ static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
 struct TileGeom {
   int tile_m;        // rows per tile (a power of two)
   int tile_m_log2;
+  int alternate;     // 1: a worker takes its tiles alternately from the expensive and the cheap end
 };
 
 struct BucketArgs {
@@ -126,7 +127,7 @@ struct ProjArgs {
   int out_cyclic_rows;
   int dbg;                // experiment switches, honoured only in -DALGPROJ_TRACE builds
   int b_3d;
-  int y_tma;          // 0: direct stores; 2 / 3: tiled stores through a 2-D / 3-D (cyclic) map of Y               // B tensor map is the 3-D chunked view (one copy per stage)
+  int y_staged;       // 1: the epilogue transposes bf16 results through shared memory for coalesced stores               // B tensor map is the 3-D chunked view (one copy per stage)
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;
 };

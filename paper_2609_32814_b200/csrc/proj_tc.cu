@@ -92,14 +92,13 @@ struct Cfg {
 
 template <int TILE_N>
 __global__ void __launch_bounds__(kThreads, 1)
-proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmY, const ProjArgs a) {
+proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
   using C = Cfg<TILE_N>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  // optional staging buffers of the epilogue warps (tiled stores) sit between the stages and the control block
+  // optional staging buffers of the epilogue warps sit between the stages and the control block
   uint8_t *store_buf = smem + C::kStages * C::kStageBytes;
-  Ctl *ctl = (Ctl *)(store_buf + (a.y_tma ? kEpiWarps * C::kStoreBufBytes : 0));
+  Ctl *ctl = (Ctl *)(store_buf + (a.y_staged ? kEpiWarps * C::kStoreBufBytes : 0));
   TileRec *recs = (TileRec *)(ctl + 1);
   TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -128,7 +127,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-    if (a.y_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmY) : "memory");
   }
   for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
   for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
@@ -303,42 +301,57 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t taddr =
           tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * C::kAccStride + half * C::kHalf);
       const int col_base = rec.n0 + half * C::kHalf;
-      // Tiled stores when this warp's 32 rows are all rows of the tile and the output is
-      // contiguous or cyclic: the bf16 row segments go through a 2 KB staging buffer (64-byte
-      // swizzle, conflict-free 16-byte writes) and leave as one bulk tensor store per 32 x 32
-      // block, instead of 64 sector requests from the load/store unit.
-      const bool staged = a.y_tma && quad * 32 + 32 <= tile_rows;
-      if (staged) {
-        const uint32_t buf = smem_u32(store_buf + e * C::kStoreBufBytes);
-        const uint32_t my_row = buf + (uint32_t)lane * 64u;
+      // bf16 outputs are transposed through a 2 KB staging buffer per warp: every lane writes its
+      // own row segment (64 bytes, 16-byte pieces XOR-swizzled so that the writes and the reads
+      // below are bank-conflict free), then four lanes together store one row segment, so one
+      // store instruction covers 8 rows x 64 contiguous bytes (8 cache lines) instead of 32
+      // lines with one sector each.  Works for every output addressing (bucketed, cyclic,
+      // permuted) and for partial tiles.
+      if (a.y_staged) {
+        uint8_t *buf = store_buf + e * C::kStoreBufBytes;
+        const uint32_t my_row = smem_u32(buf) + (uint32_t)lane * 64u;
         const uint32_t sw = (uint32_t)((lane >> 1) & 3);
-        const int type_i = (rec.pair & 0xFFFF) / q;
-        const int y_row = rec.row0 + quad * 32 - (a.y_tma == 3 ? type_i * a.out_cyclic_rows : 0);
+        const int sub = lane >> 2, piece = lane & 3;   // row within a group of 8, 16-byte piece of the segment
+        // destination rows of the four row groups this lane stores for (-1: beyond the tile)
+        int64_t dst_row[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 8 + sub);
+        const uint32_t rd_base = smem_u32(buf) + (uint32_t)sub * 64u;
 #pragma unroll 1
         for (int c0 = 0; c0 < C::kHalf; c0 += 32) {
           uint32_t v[32];
           tc_ld_32x32(taddr + (uint32_t)c0, v);
           tc_wait_ld();
+          if (e == 0 && lane == 0) ALG_TRACE(2, 3);
           float f[32];
 #pragma unroll
           for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
           finish_32(f, a, col_base + c0);
           uint32_t w[16];
           pack_bf16_32(f, w);
-          if (lane == 0) tma_store_wait_read();  // the previous block has left the buffer
-          __syncwarp();
+          if (e == 0 && lane == 0) ALG_TRACE(2, 4);
+          __syncwarp();  // the previous chunk has been read out of the buffer
 #pragma unroll
           for (int g = 0; g < 4; ++g)
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((((uint32_t)g) ^ sw) << 4)), "r"(w[g * 4]),
                          "r"(w[g * 4 + 1]), "r"(w[g * 4 + 2]), "r"(w[g * 4 + 3])
                          : "memory");
-          fence_async_smem();
           __syncwarp();
-          if (lane == 0) {
-            if (a.y_tma == 3) tma_store_3d(buf, &tmY, col_base + c0, type_i, y_row);
-            else tma_store_2d(buf, &tmY, col_base + c0, y_row);
-            tma_store_commit();
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int r = g * 8 + sub;                       // row of the chunk
+            const uint32_t rsw = (uint32_t)((r >> 1) & 3);
+            uint4 val;
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                         : "r"(rd_base + (uint32_t)g * 512u + ((((uint32_t)piece) ^ rsw) << 4)));
+#ifdef ALGPROJ_TRACE
+            if ((a.dbg & 1) && val.x != 0x12345678u) continue;   // timing experiment: no global stores
+#endif
+            if (dst_row[g] >= 0)
+              *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col_base + c0 + piece * 8) = val;
           }
+          if (e == 0 && lane == 0) ALG_TRACE(2, 5);
         }
       } else {
 #pragma unroll 1
@@ -364,7 +377,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 
   // ---------------- teardown ----------------
-  if (a.y_tma && warp >= 2 && warp < 2 + kEpiWarps && lane == 0) tma_store_wait_all();
   __syncwarp();
   if (ctl->abort_flag) {
     // give copies that are still in flight time to land before shared memory is released
@@ -402,7 +414,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   }
   int smem_bytes = C::kFixedSmemBytes + (int)tile_map_bytes(a.n_classes);
   if (smem_bytes > 227 * 1024) return cudaErrorInvalidConfiguration;
-  CUtensorMap tmA, tmB, tmY;
+  CUtensorMap tmA, tmB;
   cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
   ProjArgs b = a;
@@ -411,13 +423,10 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
     if (e != cudaSuccess) return e;
   }
-  b.y_tma = 0;
-  std::memset(&tmY, 0, sizeof(tmY));
-  if (smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && !std::getenv("ALGPROJ_NO_TMA_STORE") &&
-      make_map_y(&tmY, a) == cudaSuccess) {
-    b.y_tma = a.out_cyclic_rows ? 3 : 2;
-    smem_bytes += kEpiWarps * C::kStoreBufBytes;
-  }
+  // staging buffers for the transposing epilogue, when they fit and the output rows are 16-byte aligned
+  b.y_staged = a.y_bf16 && smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && ((uintptr_t)a.Y & 15u) == 0 &&
+               (a.ldy * 2) % 16 == 0 && !std::getenv("ALGPROJ_NO_STAGED_STORE");
+  if (b.y_staged) smem_bytes += kEpiWarps * C::kStoreBufBytes;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(num_sms, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -428,7 +437,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, tmY, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, b);
   count_launch(1);
   return e;
 }
@@ -478,28 +487,6 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.W), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
-}
-
-cudaError_t make_map_y(CUtensorMap *map, const ProjArgs &a) {
-  if (!a.y_bf16 || a.perm || ((uintptr_t)a.Y & 15u) || (a.ldy * 2) % 16 || a.N % 32) return cudaErrorInvalidValue;
-  cudaError_t e0 = tc_init();
-  if (e0 != cudaSuccess) return e0;
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r;
-  if (a.out_cyclic_rows) {
-    cuuint64_t dims[3] = {(cuuint64_t)a.N, (cuuint64_t)a.q, (cuuint64_t)a.out_cyclic_rows};
-    cuuint64_t strides[2] = {(cuuint64_t)a.ldy * 2, (cuuint64_t)a.ldy * 2 * (cuuint64_t)a.q};
-    cuuint32_t box[3] = {32, 1, 32};
-    r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, a.Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  } else {
-    cuuint64_t dims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
-    cuuint64_t strides[1] = {(cuuint64_t)a.ldy * 2};
-    cuuint32_t box[2] = {32, 32};
-    r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  }
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 

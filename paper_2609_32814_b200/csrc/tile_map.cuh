@@ -18,7 +18,8 @@ struct TileMap {
   int total;                       // number of tiles
   int q;
   int seq_rounds;                  // tile records precomputed for this worker (the last one is the end marker)
-  int pad_[2];
+  int seq_valid;                   // tiles this worker owns
+  int pad_[1];
   int offsets[kMaxQ + 2];          // bucket offsets (first bucketed row of each type)
   // followed in shared memory by: ClassRec cls[n_classes]; int prefix[n_classes + 1];
   __device__ __forceinline__ ClassRec *cls() { return reinterpret_cast<ClassRec *>(this + 1); }
@@ -108,17 +109,33 @@ __device__ __forceinline__ int snake_index(int round, int worker, int n_workers)
 }
 // `nkb_of_pair` (optional, shared memory): number of K blocks of the tiles of a pair; it is packed
 // into the upper half of TileRec::rows so that the MMA thread needs nothing but the record.
-__device__ __forceinline__ TileRec tile_seq_decode(TileMap *tm, const TileGeom &g, int round, int worker, int n_workers,
+// Processing order of a worker's own tiles: its share of the cost-sorted enumeration is taken
+// alternately from the expensive and from the cheap end (1st, last, 2nd, last but one, ...).  A
+// tile's epilogue costs the same whatever its K length, so a run of short-K tiles is bound by
+// the epilogue while a run of long-K tiles leaves the epilogue warps idle; alternating lets the
+// epilogue of one kind overlap the main loop of the other.  All workers apply the same
+// permutation to the round index, so the workers of a round still sit on neighbouring tiles.
+__device__ __forceinline__ TileRec tile_seq_decode(TileMap *tm, const TileGeom &g, int pos, int worker, int n_workers,
                                                    const uint16_t *nkb_of_pair) {
-  TileRec rec = tile_map_decode(tm, g, snake_index(round, worker, n_workers));
+  const int n = tm->seq_valid;
+  TileRec rec;
+  if (pos >= n) {
+    rec.row0 = -1, rec.rows = 0, rec.pair = 0, rec.n0 = 0;
+    return rec;
+  }
+  const int round = !g.alternate ? pos : (pos & 1) ? n - 1 - (pos >> 1) : (pos >> 1);
+  rec = tile_map_decode(tm, g, snake_index(round, worker, n_workers));
   if (nkb_of_pair && rec.row0 >= 0) rec.rows |= (int)nkb_of_pair[rec.pair & 0xFFFF] << 16;
   return rec;
 }
 __device__ inline void tile_seq_build(TileRec *recs, int cap, TileMap *tm, const TileGeom &g, int worker, int n_workers,
                                       const uint16_t *nkb_of_pair = nullptr) {
   // rounds this worker can have at all: ceil(total / n_workers), plus one record that marks the end
-  const int rounds = min(cap, (tm->total + n_workers - 1) / n_workers + 1);
-  if (threadIdx.x == 0) tm->seq_rounds = rounds;
+  const int all_rounds = (tm->total + n_workers - 1) / n_workers;
+  const int valid = all_rounds == 0 ? 0 : all_rounds - 1 + (snake_index(all_rounds - 1, worker, n_workers) < tm->total);
+  const int rounds = min(cap, valid + 1);
+  if (threadIdx.x == 0) tm->seq_rounds = rounds, tm->seq_valid = valid;
+  __syncthreads();
   for (int r = threadIdx.x; r < rounds; r += blockDim.x) recs[r] = tile_seq_decode(tm, g, r, worker, n_workers, nkb_of_pair);
   __syncthreads();
 }
