@@ -34,6 +34,11 @@ struct alg_proj_s {
   int n_workers = 1;        // persistent CTAs (or CTA pairs) of the tensor-core kernel
   bool decode_ok = false;   // the small-M weight-streaming kernel covers this shape
   DecodePlan decode = {};
+  // cyclic schedule: per-worker tile sequences for the last M seen, planned on the host
+  TileRec *d_plan = nullptr, *h_plan = nullptr;  // n_workers x plan_stride records (device / pinned host)
+  int plan_stride = 0, plan_rounds = 0;
+  int64_t plan_M = -1;
+  int plan_alternate = 0;
 };
 
 struct alg_ffn_s {
@@ -166,6 +171,12 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     p.n_workers = p.pair_kernel ? tc2_max_pairs(p.num_sms) : std::min(p.num_sms, kMaxWorkers);
     if (p.n_workers < 1) return ALG_ERR_CUDA;
   }
+  if (use_tc(p) && sched == ALG_SCHED_CYCLIC && std::getenv("ALGPROJ_NO_PLAN") == nullptr) {
+    p.plan_stride = p.pair_kernel ? kTc2SeqCap : kTcSeqCap;
+    const size_t bytes = (size_t)p.n_workers * p.plan_stride * sizeof(TileRec);
+    if (cudaMalloc(&p.d_plan, bytes) != cudaSuccess) return ALG_ERR_CUDA;
+    if (cudaMallocHost(&p.h_plan, bytes) != cudaSuccess) return ALG_ERR_CUDA;
+  }
   if (dtype == ALG_BF16 && std::getenv("ALGPROJ_NO_DECODE") == nullptr) {
     p.decode_ok = decode_plan(q, p.s, p.K, p.N, p.num_sms, &p.decode);
     for (int g = 0; g < q && p.decode_ok; ++g)
@@ -175,6 +186,9 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
 }
 
 void free_proj(alg_proj_s &p) {
+  if (p.d_plan) cudaFree(p.d_plan);
+  if (p.h_plan) cudaFreeHost(p.h_plan);
+  p.d_plan = p.h_plan = nullptr;
   if (p.d_tab) cudaFree(p.d_tab);
   if (p.d_status && !p.shared_status) cudaFree(p.d_status);
   p.d_tab = nullptr;
@@ -209,9 +223,67 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
 
 alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG_ERR_CUDA; }
 
+// Host twin of the in-kernel tile enumeration for the cyclic schedule (equal buckets of M/q rows):
+// cost-sorted classes, m-tile major inside a class, boustrophedon assignment of tile indices to
+// workers, optional alternation of expensive and cheap tiles inside a worker.  Fills p.h_plan and
+// copies it to the device on `st`; returns false when the sequences do not fit the plan stride
+// (the kernels then plan for themselves).
+bool prepare_cyclic_plan(alg_proj_s &p, int64_t M, int alternate, cudaStream_t st) {
+  if (!p.d_plan) return false;
+  if (p.plan_M == M && p.plan_alternate == alternate) return p.plan_rounds > 0;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return false;
+  const int q = p.q, nc = p.tab.n_classes, tile_m = tile_m_of(p), nw = p.n_workers, stride = p.plan_stride;
+  const int bucket = (int)(M / q);
+  const int m_tiles = (bucket + tile_m - 1) / tile_m;
+  std::vector<long long> prefix(nc + 1, 0);
+  for (int c = 0; c < nc; ++c) prefix[c + 1] = prefix[c] + (long long)m_tiles * p.tab.cls[c].n_tiles;
+  const long long total = prefix[nc];
+  const long long all_rounds = (total + nw - 1) / nw;
+  p.plan_M = M;
+  p.plan_alternate = alternate;
+  p.plan_rounds = 0;
+  if (all_rounds + 1 > stride) return false;
+  std::vector<int> nkb(q * q, 0);
+  for (int pr = 0; pr < q * q; ++pr)
+    for (int k = 0; k < q; ++k)
+      if ((p.tab.keep[pr] >> k) & 1u) nkb[pr] += p.s[k] / kTcBlockK;
+  auto snake = [&](long long round, int w) { return round * nw + ((round & 1) ? (nw - 1 - w) : w); };
+  const int rounds = (int)all_rounds + 1;
+  for (int w = 0; w < nw; ++w) {
+    const int valid = all_rounds == 0 ? 0 : (int)all_rounds - 1 + (snake(all_rounds - 1, w) < total ? 1 : 0);
+    for (int pos = 0; pos < rounds; ++pos) {
+      TileRec rec;
+      rec.row0 = -1, rec.rows = 0, rec.pair = 0, rec.n0 = 0;
+      if (pos < valid) {
+        const int round = !alternate ? pos : (pos & 1) ? valid - 1 - (pos >> 1) : (pos >> 1);
+        const long long idx = snake(round, w);
+        int c = (int)(std::upper_bound(prefix.begin(), prefix.end(), idx) - prefix.begin()) - 1;
+        const ClassRec &r = p.tab.cls[c];
+        const int loc = (int)(idx - prefix[c]), ntl = (int)r.n_tiles, mt = loc / ntl, nt = loc - mt * ntl;
+        rec.row0 = (int)r.i * bucket + mt * tile_m;
+        rec.rows = std::min(tile_m, bucket - mt * tile_m) | (nkb[(int)r.i * q + (int)r.j] << 16);
+        rec.pair = ((int)r.i * q + (int)r.j) | ((int)r.cols << 16);
+        rec.n0 = r.col0 + nt * (int)r.cols;
+      }
+      p.h_plan[(size_t)w * stride + pos] = rec;
+    }
+  }
+  // the pinned buffer is rewritten only when M changes: wait for the copy, so that no copy of an
+  // older plan can still be reading it then
+  if (cudaMemcpyAsync(p.d_plan, p.h_plan, (size_t)nw * stride * sizeof(TileRec), cudaMemcpyHostToDevice, st) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    p.plan_M = -1;
+    return false;
+  }
+  p.plan_rounds = rounds;
+  return true;
+}
+
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
-alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
+alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
                       cudaEvent_t after_gather = nullptr, bool cyclic = false) {
@@ -246,6 +318,13 @@ alg_status_t run_proj(const alg_proj_s &p, const WsLayout &L, char *ws, const vo
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.b_3d = 0;
   a.y_staged = 0;
+  a.plan = nullptr;
+  a.plan_stride = a.plan_rounds = 0;
+  if (cyclic && prepare_cyclic_plan(p, M, a.geom.alternate, st)) {
+    a.plan = p.d_plan;
+    a.plan_stride = p.plan_stride;
+    a.plan_rounds = p.plan_rounds;
+  }
   a.dbg = std::getenv("ALGPROJ_DBG") ? atoi(std::getenv("ALGPROJ_DBG")) : 0;
   a.trace = g_trace;
   a.trace_cap = g_trace_cap;

@@ -126,8 +126,13 @@ struct ProjArgs {
   int a_cyclic_rows;
   int out_cyclic_rows;
   int dbg;                // experiment switches, honoured only in -DALGPROJ_TRACE builds
-  int b_3d;
-  int y_staged;       // 1: the epilogue transposes bf16 results through shared memory for coalesced stores               // B tensor map is the 3-D chunked view (one copy per stage)
+  int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
+  int y_staged;           // 1: the epilogue transposes bf16 results through shared memory for coalesced stores
+  // Cyclic schedule: the tile sequences of all workers depend only on (handle, M) and are planned
+  // once on the host; worker w reads plan[w * plan_stride .. + plan_rounds) (the last record of
+  // every worker is the end marker).  nullptr: every CTA plans for itself.
+  const TileRec *plan;
+  int plan_stride, plan_rounds;
   long long *trace;       // debug timeline (nullptr = off)
   int trace_cap;
 };
@@ -136,6 +141,7 @@ cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
 
 // tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
 // (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.
+constexpr int kTcSeqCap = 224, kTc2SeqCap = 48;  // precomputed tile records per worker
 constexpr int kTcTileM = 128;
 constexpr int kTcBlockK = 64;
 constexpr int kTc2TileM = 256;

@@ -65,7 +65,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctl *ctl
   if (mbar_try_wait(bar, parity)) return true;
   return wait_slow(bar, parity, ctl, status);
 }
-constexpr int kSeqCap = 224;  // precomputed tile records per CTA
+constexpr int kSeqCap = kTcSeqCap;  // precomputed tile records per CTA
 #ifndef ALGPROJ_EPI_WARPS
 #define ALGPROJ_EPI_WARPS 8
 #endif
@@ -114,29 +114,38 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 #endif
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), 1);
-      mbar_init(smem_u32(&ctl->empty[s]), 1);
+  if (threadIdx.x == 0) ALG_TRACE(0, 20);
+  if (warp == 0) {  // one barrier per lane
+    if (lane < C::kStages) {
+      mbar_init(smem_u32(&ctl->full[lane]), 1);
+      mbar_init(smem_u32(&ctl->empty[lane]), 1);
+    } else if (lane < C::kStages + 2) {
+      mbar_init(smem_u32(&ctl->tmem_full[lane - C::kStages]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[lane - C::kStages]), kEpiWarps);
+    } else if (lane == 31) {
+      ctl->abort_flag = 0;
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[b]), kEpiWarps);
-    }
-    ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+  } else if (warp == 3) {
+    // The table copies below run in different warps so that their first-touch misses (kernel
+    // parameters, table in global memory) overlap instead of adding up.
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    for (int e = lane; e < q * q; e += 32) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
+  } else if (warp == 4) {
+    for (int e = lane; e <= q; e += 32) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
+  } else if (warp == 5) {
+    for (int e = lane; e < q * q; e += 32) {
+      const uint32_t mask = a.st.valid ? a.st.keep[e] : tab->keep[e];
+      int n = 0;
+      for (int k = 0; k < q; ++k)
+        if ((mask >> k) & 1u) n += ((a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k])) / kTcBlockK;
+      ctl->nkb[e] = (uint16_t)n;   // for tile records decoded after the precomputed ones
+    }
   }
-  for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
-  for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
-  for (int e = threadIdx.x; e < q * q; e += kThreads) {
-    const uint32_t mask = a.st.valid ? a.st.keep[e] : tab->keep[e];
-    int n = 0;
-    for (int k = 0; k < q; ++k)
-      if ((mask >> k) & 1u) n += ((a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k])) / kTcBlockK;
-    ctl->nkb[e] = (uint16_t)n;
-  }
+  if (threadIdx.x == 0) ALG_TRACE(0, 21);
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"((uint32_t)C::kTmemCols)
@@ -147,9 +156,19 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // run while the previous kernel of the stream is finishing; nothing below (bucket offsets, X, H,
   // Y) is read or written before that kernel has completed.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (warp == 2) {
+    // one warp plans this CTA's work while the others set up barriers and tensor memory
+    if (a.plan) {  // cyclic schedule: planned on the host, once per (handle, M)
+      for (int r = lane; r < a.plan_rounds; r += 32) recs[r] = a.plan[(size_t)blockIdx.x * a.plan_stride + r];
+      if (lane == 0) tm->seq_rounds = a.plan_rounds, tm->seq_valid = a.plan_rounds, tm->total = 0;
+    } else {
+      if (a.offsets) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
+      tile_plan_warp(tm, recs, kSeqCap, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom, blockIdx.x,
+                     gridDim.x, kTcBlockK);
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
-  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x, gridDim.x, ctl->nkb);  // (tile_map_build has synchronised ctl->nkb)
+  if (threadIdx.x == 0) ALG_TRACE(0, 24);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();

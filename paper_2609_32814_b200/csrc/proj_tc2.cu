@@ -32,7 +32,7 @@ constexpr int kEpiWarps = 8;
 constexpr int kProducerWarpB = 2 + kEpiWarps;   // second TMA producer, after the epilogue warps
 constexpr int kThreads = 32 * (3 + kEpiWarps);
 constexpr int kMaxStages = 7;
-constexpr int kSeqCap = 48;   // precomputed tile records per CTA pair
+constexpr int kSeqCap = kTc2SeqCap;   // precomputed tile records per CTA pair
 constexpr int kABytes = 128 * kTcBlockK * 2;              // 16 KB: this CTA's rows
 constexpr int kBChunkBytes = kTcBlockK * 64 * 2;           // one 64(k) x 64(n) box
 constexpr int kBMaxBytes = kBChunkBytes * (kTc2TileN / 128);  // this CTA's half of the B block: 16 KB
@@ -49,11 +49,11 @@ struct Ctl2 {
   uint32_t tmem_base;
   volatile int abort_flag;
   int so[kMaxQ + 1];
-  uint32_t keep[1];  // q*q entries follow (the shared-memory request is sized for them)
+  uint32_t keep[1];  // q*q entries follow, then q*q uint16 K-block counts (the request is sized for them)
 };
 constexpr int kMaxSmem = 227 * 1024;
 inline int smem_bytes(int n_stages, int q, int n_classes) {
-  return n_stages * kStageBytes + (int)sizeof(Ctl2) + q * q * 4 + kSeqCap * 16 + (int)tile_map_bytes(n_classes) + 32 +
+  return n_stages * kStageBytes + (int)sizeof(Ctl2) + q * q * 6 + 16 + kSeqCap * 16 + (int)tile_map_bytes(n_classes) + 32 +
          1024;
 }
 inline int pick_stages(int q, int n_classes) {
@@ -135,13 +135,22 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int tab_q = a.q;
   Ctl2 *ctl = (Ctl2 *)(smem + n_stages * kStageBytes);
-  TileRec *recs = (TileRec *)(((uintptr_t)(ctl->keep + tab_q * tab_q) + 15) & ~(uintptr_t)15);
+  uint16_t *nkb = (uint16_t *)(ctl->keep + tab_q * tab_q);
+  TileRec *recs = (TileRec *)(((uintptr_t)(nkb + tab_q * tab_q) + 15) & ~(uintptr_t)15);
   TileMap *tm = (TileMap *)(recs + kSeqCap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
   const int q = tab_q;
   const uint32_t rank = cluster_ctarank();          // 0 = leader
   [[maybe_unused]] int tr_n = 0;
+#ifdef ALGPROJ_TRACE
+  if (a.trace && threadIdx.x == 0) {  // whole-CTA window: global timer and SM clock at entry
+    unsigned long long gt;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 0] = (long long)gt;
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 2] = clock64();
+  }
+#endif
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -159,115 +168,130 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
   for (int e = threadIdx.x; e < q * q; e += kThreads) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
   for (int e = threadIdx.x; e <= q; e += kThreads) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
+  for (int e = threadIdx.x; e < q * q; e += kThreads) {
+    const uint32_t mask = a.st.valid ? a.st.keep[e] : tab->keep[e];
+    int n = 0;
+    for (int k = 0; k < q; ++k)
+      if ((mask >> k) & 1u) n += (a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k]) / kTcBlockK;
+    nkb[e] = (uint16_t)n;
+  }
   if (warp == 1) {  // both CTAs of the pair allocate together, same shared-memory slot
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"((uint32_t)kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  // Programmatic dependent launch: everything above touches only this CTA's own state.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   tile_map_build(tm, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom);
-  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x >> 1, gridDim.x >> 1);
+  tile_seq_build(recs, kSeqCap, tm, a.geom, blockIdx.x >> 1, gridDim.x >> 1, nkb);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
 
+  // Producer and MMA roles run warp-uniformly (all lanes execute loops and waits, one elected lane
+  // issues), so that the operands of the copy / MMA / commit instructions stay in uniform
+  // registers; loop bounds read from shared memory are broadcast with a shuffle.
   if (warp == 0 || warp == kProducerWarpB) {
-    // ---------------- TMA producers (one lane each, both CTAs) ----------------
-    // Issuing a tiled load occupies the thread while the copy engine expands the box, so the A
-    // block and the B half of a stage are issued by two threads in different warps: a freed
-    // stage is refilled sooner, which shortens the load -> MMA -> free -> load round trip that
-    // bounds the bytes in flight.
-    if (lane == 0) {
-      const bool loads_a = warp == 0;
-      int stage = 0, round = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
-      while (ok && rec.row0 >= 0) {
-        ++round;
-        if (loads_a) ALG_TRACE(0, 1);
-        const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
-        const int half_cols = (rec.pair >> 16) >> 1;         // B columns this CTA loads: 128 or 64
-        const int n_chunks = half_cols >> 6;
-        const uint32_t tx_bytes = 2u * (uint32_t)(kABytes + n_chunks * kBChunkBytes);
-        const int row = rec.row0 + 128 * (int)rank;
-        const int col = rec.n0 + (int)rank * half_cols;
-        for (int k = 0; k < q && ok; ++k) {
-          if (!((mask >> k) & 1u)) continue;
-          const int k_end = ctl->so[k + 1];
-          for (int k0 = ctl->so[k]; k0 < k_end; k0 += kTcBlockK) {
-            ok = wait_bar2(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, a.status);
-            if (!ok) break;
-            const uint32_t own_bar = smem_u32(&ctl->full[stage]);
-            const uint32_t sa = smem_u32(smem + stage * kStageBytes);
-            const uint32_t bar = own_bar & kPeerMask;
+    // ---------------- TMA producers (both CTAs): warp 0 loads A, the last warp loads the B half ------
+    const bool loads_a = warp == 0;
+    int stage = 0, round = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    const uint32_t smem0 = smem_u32(smem);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1, nkb);
+    while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
+      ++round;
+      if (loads_a && lane == 0) ALG_TRACE(0, 1);
+      const int pair = __shfl_sync(0xffffffffu, rec.pair & 0xFFFF, 0);
+      const int cols = __shfl_sync(0xffffffffu, rec.pair >> 16, 0);
+      const int row0 = __shfl_sync(0xffffffffu, rec.row0, 0);
+      const int n0 = __shfl_sync(0xffffffffu, rec.n0, 0);
+      const uint32_t mask = __shfl_sync(0xffffffffu, ctl->keep[pair], 0);
+      const int half_cols = cols >> 1;                       // B columns this CTA loads: 128 or 64
+      const int n_chunks = half_cols >> 6;
+      const uint32_t tx_bytes = 2u * (uint32_t)(kABytes + n_chunks * kBChunkBytes);
+      const int type_i = pair / q;
+      const int row = row0 + 128 * (int)rank - (a.a_cyclic_rows ? type_i * a.a_cyclic_rows : 0);
+      const int col = n0 + (int)rank * half_cols;
+      for (int k = 0; k < q && ok; ++k) {
+        if (!((mask >> k) & 1u)) continue;
+        const int k_begin = __shfl_sync(0xffffffffu, ctl->so[k], 0);
+        const int k_end = __shfl_sync(0xffffffffu, ctl->so[k + 1], 0);
+        for (int k0 = k_begin; k0 < k_end; k0 += kTcBlockK) {
+          ok = __all_sync(0xffffffffu, wait_bar2(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, a.status));
+          if (!ok) break;
+          const uint32_t own_bar = full0 + 8u * (uint32_t)stage;
+          const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)kStageBytes;
+          const uint32_t bar = own_bar & kPeerMask;
+          if (elect_one()) {
             if (loads_a) {
               if (rank == 0) mbar_expect_tx(own_bar, tx_bytes);
-              if (a.a_cyclic_rows) {
-                const int i = (rec.pair & 0xFFFF) / q;
-                tma_load_3d_pair(sa, &tmA, bar, k0, i, row - i * a.a_cyclic_rows);
-              } else {
-                tma_load_2d_pair(sa, &tmA, bar, k0, row);
-              }
+              if (a.a_cyclic_rows) tma_load_3d_pair(sa, &tmA, bar, k0, type_i, row);
+              else tma_load_2d_pair(sa, &tmA, bar, k0, row);
             } else {
               for (int c = 0; c < n_chunks; ++c)
                 tma_load_2d_pair(sa + kABytes + c * kBChunkBytes, &tmB, bar, col + c * 64, k0);
             }
-            if (++stage == n_stages) stage = 0, phase ^= 1u;
           }
+          __syncwarp();
+          if (++stage == n_stages) stage = 0, phase ^= 1u;
         }
-        if (loads_a) ALG_TRACE(0, 2);
-        rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
       }
+      if (loads_a && lane == 0) ALG_TRACE(0, 2);
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1, nkb);
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer (one lane of the leader CTA) ----------------
-    if (lane == 0 && rank == 0) {
+    // ---------------- MMA issuer (leader CTA) ----------------
+    if (rank == 0) {
       int stage = 0, acc = 0, round = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
-      while (ok && rec.row0 >= 0) {
+      const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+      const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
+      const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, 1024);
+      const uint64_t db0 = make_smem_desc(smem_u32(smem) + kABytes, kBChunkBytes, 1024);
+      TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1, nkb);
+      while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
         ++round;
-        ALG_TRACE(1, 1);
-        ok = wait_bar2(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, ctl, a.status);
+        if (lane == 0) ALG_TRACE(1, 1);
+        const int n_kb = __shfl_sync(0xffffffffu, (int)((uint32_t)rec.rows >> 16), 0);
+        const int cols = __shfl_sync(0xffffffffu, rec.pair >> 16, 0);
+        ok = __all_sync(0xffffffffu, wait_bar2(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
         if (!ok) break;
-        ALG_TRACE(1, 2);
+        if (lane == 0) ALG_TRACE(1, 2);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
-        const uint32_t mask = ctl->keep[rec.pair & 0xFFFF];
-        const int cols = rec.pair >> 16;
         // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N = cols, M = 256
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                ((uint32_t)(cols >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-        uint32_t accumulate = 0;
-        for (int k = 0; k < q && ok; ++k) {
-          if (!((mask >> k) & 1u)) continue;
-          const int n_kb = (ctl->so[k + 1] - ctl->so[k]) / kTcBlockK;
-          for (int kb = 0; kb < n_kb; ++kb) {
-            ok = wait_bar2(smem_u32(&ctl->full[stage]), phase, ctl, a.status);
-            if (!ok) break;
-            if (!accumulate) ALG_TRACE(1, 3);
-            tc_fence_after();
-            const uint32_t sa = smem_u32(smem + stage * kStageBytes);
-            const uint64_t da = make_smem_desc(sa, 16, 1024);
-            const uint64_t db = make_smem_desc(sa + kABytes, kBChunkBytes, 1024);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          ok = __all_sync(0xffffffffu, wait_bar2(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
+          if (!ok) break;
+          if (kb == 0 && lane == 0) ALG_TRACE(1, 3);
+          tc_fence_after();
+          const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(kStageBytes >> 4));
+          const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(kStageBytes >> 4));
+          if (elect_one()) {
+            tc2_mma_bf16(d_tmem, da, db, idesc, kb ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < kTcBlockK / 16; ++kk) {
-              tc2_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc, accumulate);
-              accumulate = 1;
-            }
-            tc2_commit_both(smem_u32(&ctl->empty[stage]));
-            if (++stage == n_stages) stage = 0, phase ^= 1u;
+            for (int kk = 1; kk < kTcBlockK / 16; ++kk)
+              tc2_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc, 1u);
+            tc2_commit_both(empty0 + 8u * (uint32_t)stage);
           }
+          __syncwarp();
+          if (++stage == n_stages) stage = 0, phase ^= 1u;
         }
         if (!ok) break;
-        tc2_commit_both(smem_u32(&ctl->tmem_full[acc]));
-        ALG_TRACE(1, 4);
+        if (elect_one()) tc2_commit_both(tfull0 + 8u * (uint32_t)acc);
+        __syncwarp();
+        if (lane == 0) ALG_TRACE(1, 4);
         if (++acc == 2) acc = 0, acc_phase ^= 1u;
-        rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
+        rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1, nkb);
       }
     }
   } else {
@@ -277,14 +301,14 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int half = e >> 2;
     int acc = 0, round = 0;
     uint32_t acc_phase = 0;
-    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1);
+    TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x >> 1, gridDim.x >> 1, nkb);
     while (rec.row0 >= 0) {
       ++round;
       const int cols = rec.pair >> 16;
       const int half_cols = cols >> 1;
       const int r = 128 * (int)rank + quad * 32 + lane;   // row inside the 256-row tile
       int64_t out_row = -1;
-      if (r < rec.rows) {
+      if (r < (rec.rows & 0xFFFF)) {
         if (a.out_cyclic_rows) {
           const int i = (rec.pair & 0xFFFF) / q;
           out_row = (int64_t)(rec.row0 + r - i * a.out_cyclic_rows) * q + i;
@@ -320,7 +344,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
-      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1);
+      rec = tile_seq_get(recs, tm, a.geom, round, blockIdx.x >> 1, gridDim.x >> 1, nkb);
     }
   }
 
@@ -334,6 +358,14 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // neither CTA leaves while its peer may still signal or read its shared memory
+#ifdef ALGPROJ_TRACE
+  if (a.trace && threadIdx.x == 0) {
+    unsigned long long gt;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 1] = (long long)gt;
+    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 3] = clock64();
+  }
+#endif
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
@@ -372,9 +404,19 @@ cudaError_t launch_proj_tc2(const ProjArgs &a, int num_sms, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
   if (e != cudaSuccess) return e;
-  proj_tc2_kernel<<<2 * pairs, kThreads, smem_bytes(n_stages, q, a.n_classes), st>>>(tmA, tmB, a, n_stages);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes(n_stages, q, a.n_classes);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
+  e = cudaLaunchKernelEx(&cfg, proj_tc2_kernel, tmA, tmB, a, n_stages);
   count_launch(1);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace algproj

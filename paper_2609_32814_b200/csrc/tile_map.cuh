@@ -145,4 +145,56 @@ __device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, TileMap *tm
   return tile_seq_decode(tm, g, round, worker, n_workers, nkb_of_pair);
 }
 
+// The whole plan of one worker -- class prefix table and its own tile sequence, K-block counts
+// included -- built by ONE warp with warp-level synchronisation only, so that the other warps of
+// the CTA can set up barriers and tensor memory meanwhile and a single CTA barrier ends the
+// prologue.  `keep` / `so` are read from the by-value table when it is valid, else from `tab`.
+__device__ inline void tile_plan_warp(TileMap *tm, TileRec *recs, int cap, const DevTable *tab, const SmallTable &st,
+                                      int q, int nc, const int *offsets, int cyclic_rows, int M, const TileGeom &g,
+                                      int worker, int n_workers, int k_block) {
+  const int lane = threadIdx.x & 31;
+  if (lane == 0) tm->n_classes = nc, tm->q = q;
+  for (int t = lane; t <= q + 1; t += 32) tm->offsets[t] = offsets ? offsets[t] : (t <= q ? t * cyclic_rows : M);
+  __syncwarp();
+  ClassRec *cls = tm->cls();
+  int *prefix = tm->prefix();
+  int carry = 0;
+  for (int c0 = 0; c0 < nc; c0 += 32) {
+    const int c = c0 + lane;
+    int v = 0;
+    if (c < nc) {
+      const ClassRec r = st.valid ? st.cls[c] : tab->cls[c];
+      cls[c] = r;
+      const int rows = tm->offsets[r.i + 1] - tm->offsets[r.i];
+      v = ((rows + g.tile_m - 1) >> g.tile_m_log2) * (int)r.n_tiles;
+    }
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += n;
+    }
+    if (c < nc) prefix[c] = carry + incl - v;
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  const int total = carry;
+  const int all_rounds = (total + n_workers - 1) / n_workers;
+  const int valid = all_rounds == 0 ? 0 : all_rounds - 1 + (snake_index(all_rounds - 1, worker, n_workers) < total);
+  const int rounds = min(cap, valid + 1);
+  if (lane == 0) prefix[nc] = total, tm->total = total, tm->seq_rounds = rounds, tm->seq_valid = valid;
+  __syncwarp();
+  for (int r = lane; r < rounds; r += 32) {
+    TileRec rec = tile_seq_decode(tm, g, r, worker, n_workers, nullptr);
+    if (rec.row0 >= 0) {
+      const int pr = rec.pair & 0xFFFF;
+      const uint32_t mask = st.valid ? st.keep[pr] : tab->keep[pr];
+      int n = 0;
+      for (int k = 0; k < q; ++k)
+        if ((mask >> k) & 1u) n += (st.valid ? st.so[k + 1] - st.so[k] : tab->so[k + 1] - tab->so[k]) / k_block;
+      rec.rows |= n << 16;
+    }
+    recs[r] = rec;
+  }
+}
+
 }  // namespace algproj
