@@ -68,7 +68,15 @@ typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } a
 
 /* EXPLICIT: the caller passes types[M] with every forward call.
  * CYCLIC  : type of row b is b mod q (the paper's example schedule tau(p) = p mod q for a
- *           batch whose sequence length is a multiple of q); `types` may be NULL. */
+ *           batch whose sequence length is a multiple of q); `types` may be NULL.
+ *           With q | M the tensor-core path needs no permutation, and the tile sequences of its
+ *           persistent CTAs depend only on (handle, M): they are planned on the host at the
+ *           first forward call with a given M and kept in device memory the handle owns (sized
+ *           at create; forward allocates nothing).  That first call copies the plan on `stream`
+ *           and waits for the copy; later calls with the same M do not synchronise.  If a new M
+ *           is first seen while `stream` is being captured, the kernels plan for themselves
+ *           instead (same result).  Calls on one handle share the plan: do not run forward
+ *           calls with different M on the same handle concurrently. */
 typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1 } alg_schedule_t;
 
 /* Kernel families, reported by alg_proj_kernel_path(). */

@@ -181,6 +181,38 @@ def test_cyclic_fast_path_matches_explicit_types(q, M):
     H.assert_bf16_close(H.to_np(Yp), refp, False, f"cyclic proj q={q} M={M}")
 
 
+def test_cyclic_plan_follows_M_and_stream_capture():
+    """The cyclic schedule's tile sequences are planned on the host once per (handle, M).  One handle
+    must give the explicit-types result for M1, then M2, then M1 again; and a first call with a new
+    M inside stream capture (where the host cannot re-plan) must fall back to in-kernel planning."""
+    q = 2
+    cyc = binding.Proj([128] * q, [256] * q, dtype="bf16", schedule="cyclic")
+    exp = binding.Proj([128] * q, [256] * q, dtype="bf16")
+    W = H.to_dev(synth.normal(31, (128 * q, 256 * q), 0.05), "bf16")
+
+    def pair(M, seed):
+        X = H.to_dev(synth.normal(seed, (M, 128 * q), 1.0), "bf16")
+        t = H.dev_types(synth.cyclic_types(M, q))
+        return X, exp.forward(X, t, W, act="gelu")
+
+    for M, seed in ((1024, 1), (2560, 2), (1024, 3), (770, 4)):
+        X, want = pair(M, seed)
+        assert torch.equal(cyc.forward(X, None, W, act="gelu"), want), M
+    X, want = pair(1536, 5)                     # new M, first seen while capturing
+    Y = torch.empty_like(want)
+    ws = torch.empty(cyc.workspace_bytes(1536), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            cyc.forward(X, None, W, act="gelu", out=Y, workspace=ws, stream=stream)
+    Y.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(Y, want) and cyc.last_status() == 0
+    assert torch.equal(cyc.forward(X, None, W, act="gelu"), want)   # planned on the host now
+
+
 def test_pilot_tensor_square_law_and_interval_schedule():
     """The law and shape of the paper's pilot FFN projections: Q_2 (x) Q_2 (36 block products,
     9/16 of the dense MACs), D = 768 = 4 x 192, F = 1536 = 4 x 384, interval schedule."""
