@@ -268,6 +268,22 @@ def main():
     with ClockSampler(local_rank) as clocks:
         total_ms = time_steps(args.steps, first=args.warmup)
     launches = binding.launch_count() - launches0
+    clock_note = "sampled during the timed region"
+    if len(clocks.samples) < 5:
+        # the timed region is only tens of milliseconds; when the sampler (NVML, else nvidia-smi
+        # every 50 ms) caught fewer than five samples, the same steps run on, untimed, under the
+        # sampler for a quarter of a second so that the clock record covers this load
+        with ClockSampler(local_rank) as clocks2:
+            t_end = time.time() + 0.25
+            i = 0
+            while time.time() < t_end:
+                for _ in range(50):
+                    step(i)
+                    i += 1
+                torch.cuda.synchronize()
+        clocks.samples += clocks2.samples
+        clocks.max_mhz = clocks.max_mhz or clocks2.max_mhz
+        clock_note = "timed region too short for the sampler: extended by 0.25 s of the same steps, untimed"
     total_ms = max_over_ranks(total_ms, "cuda")
     ms_per_step = total_ms / args.steps
     value = whole_job_value(flops, world, args.steps, total_ms)
@@ -302,23 +318,44 @@ def main():
                                        "note": "events between the kernels (no launch overlap)"}}
 
     # ---- end to end through the host entry point: pinned H2D of X, D2H of Y inside the timing ----
-    Xh = torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory()
-    Yh = torch.empty((wl.M, wl.D), dtype=torch.bfloat16).pin_memory()
-    wsh = torch.empty(ffn.host_workspace_bytes(wl.M, torch.bfloat16), dtype=torch.uint8, device="cuda")
-    for i in range(3):
-        ffn.forward_host(Xh, None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], Yh, workspace=wsh, stream=stream)
+    # Three slots (pinned X / Y, device workspace, stream) are used round-robin, the way a serving
+    # loop would: the upload of step i+1 and the download of step i-1 overlap the kernels of step i.
+    # Every step still uploads its own X and downloads its own Y inside the timed region.
+    n_slots = 3
+    slots = []
+    for k in range(n_slots):
+        slots.append({"X": torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory(),
+                      "Y": torch.empty((wl.M, wl.D), dtype=torch.bfloat16).pin_memory(),
+                      "ws": torch.empty(ffn.host_workspace_bytes(wl.M, torch.bfloat16), dtype=torch.uint8, device="cuda"),
+                      "stream": torch.cuda.Stream()})
+    Xh, Yh = slots[0]["X"], slots[0]["Y"]
+
+    def host_step(i):
+        sl = slots[i % n_slots]
+        ffn.forward_host(sl["X"], None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], sl["Y"], workspace=sl["ws"],
+                         stream=sl["stream"])
+
+    for i in range(2 * n_slots):
+        host_step(i)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
+    for sl in slots:
+        sl["stream"].wait_event(e0)
     for i in range(args.steps):
-        ffn.forward_host(Xh, None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], Yh, workspace=wsh, stream=stream)
+        host_step(i)
+    for sl in slots:
+        done = torch.cuda.Event()
+        done.record(sl["stream"])
+        stream.wait_event(done)
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
     e2e_ms = max_over_ranks(e2e_ms, "cuda")
     e2e = {"value": whole_job_value(flops, world, args.steps, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
-           "ms_per_step": e2e_ms / args.steps}
+           "ms_per_step": e2e_ms / args.steps,
+           "note": f"{n_slots} host-buffer slots on {n_slots} streams: copies of neighbouring steps overlap the kernels"}
 
     extras = {}
     if rank == 0 and not args.no_extras:
@@ -334,7 +371,7 @@ def main():
                            "rows_per_gpu": wl.M, "parallelism": f"rows sharded over {world} GPU(s), weights replicated"},
                 "tokens_per_s": world * wl.M * args.steps / (total_ms * 1e-3),
                 "kept_gflop_per_step": flops / 1e9,
-                "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": int(launches),
+                "clocks": dict(clocks.summary(), note=clock_note), "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "cpu_baseline": cpu}
         line.update(extras)
         print(json.dumps(line), flush=True)

@@ -115,6 +115,10 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   }
   if (!all256 && !all192 && !all128) p.tc_ok = false;
   p.tile_n = all256 ? 256 : all192 ? 192 : 128;
+  if (const char *tn = std::getenv("ALGPROJ_TILE_N")) {  // experiment: force a tile width that divides every group
+    const int v = atoi(tn);
+    if ((v == 256 && all256) || (v == 192 && all192) || (v == 128 && all128)) p.tile_n = v;
+  }
   // CTA-pair kernel whenever every output group splits into 256-wide tiles plus a 128-wide rest
   // (measured: it wins only when every tile has a long K loop; short loops favour the one-CTA kernel)
   int min_klen = 1 << 30;
