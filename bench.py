@@ -37,7 +37,7 @@ UNIT = "TFLOP/s"
 N_SETS = 6
 # DRAM traffic of the grouped-GEMM kernels from the ncu capture summarised under profiles/
 # (bytes of the up launch + the down launch of one step of this workload).
-NCU_TRAFFIC_BYTES = 20.0e6 + 56.8e6  # up + down launch, cold caches (profiles/proj_tc_kernel_cfg2.md)
+NCU_TRAFFIC_BYTES = 19.2e6 + 57.0e6  # up + down launch, cold caches (profiles/proj_tc_kernel_cfg2.md)
 
 
 def _peaks():
