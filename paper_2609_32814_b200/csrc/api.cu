@@ -2,6 +2,7 @@
 // validation, workspace layout and the launch sequence of one forward pass.
 #include <algorithm>
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -46,6 +47,13 @@ struct alg_ffn_s {
   int D = 0, F = 0;
   bool timing = false;       // record events between the kernels of each forward call
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  // one-kernel FFN (cyclic schedule, bf16, q <= 8): host plan for the last M seen
+  bool fused_ok = false;
+  TileRec *d_fplan = nullptr, *h_fplan = nullptr;
+  TileExt *d_fext = nullptr, *h_fext = nullptr;
+  unsigned long long *d_counters = nullptr;
+  int fused_workers = 0, fused_rounds = 0, fused_blocks = 0, fused_target = 0;
+  int64_t fused_M = -1;
 };
 
 namespace {
@@ -523,14 +531,215 @@ alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, cons
   }
   f->D = f->up.K;
   f->F = f->up.N;
+  // one-kernel FFN: cyclic schedule, bf16 tensor path, tables by value (q <= 8), hidden groups in
+  // 256-column tiles, output groups in 256-, 192- or 128-column tiles
+  constexpr int kMaxFusedBlocks = 4096;
+  bool fused = schedule == ALG_SCHED_CYCLIC && use_tc(f->up) && use_tc(f->down) && q <= kParamQ &&
+               std::getenv("ALGPROJ_FUSED") != nullptr;
+  for (int g = 0; g < q && fused; ++g) fused = f_widths[g] % 256 == 0 && (d_widths[g] % 128 == 0 || d_widths[g] % 192 == 0);
+  if (fused) {
+    f->fused_workers = std::min(f->up.num_sms, kMaxWorkers);
+    const size_t n = (size_t)f->fused_workers * kFfnSeqCap;
+    fused = cudaMalloc(&f->d_fplan, n * sizeof(TileRec)) == cudaSuccess &&
+            cudaMallocHost(&f->h_fplan, n * sizeof(TileRec)) == cudaSuccess &&
+            cudaMalloc(&f->d_fext, n * sizeof(TileExt)) == cudaSuccess &&
+            cudaMallocHost(&f->h_fext, n * sizeof(TileExt)) == cudaSuccess &&
+            cudaMalloc(&f->d_counters, (kMaxFusedBlocks + 1) * sizeof(unsigned long long)) == cudaSuccess &&
+            cudaMemset(f->d_counters, 0, (kMaxFusedBlocks + 1) * sizeof(unsigned long long)) == cudaSuccess;
+  }
+  f->fused_ok = fused;
   *out = f;
   return ALG_OK;
 }
+
+namespace {
+
+// Host plan of the one-kernel FFN for M rows (cyclic schedule: q equal buckets of M/q rows).
+// Up tiles: row block (type i, m-tile) x hidden group j x 256-column tile; down tiles: the same row
+// block x output group j x column tiles (192 wide when that divides the group and 256 does not,
+// else 256 wide plus one of 128).  Built as a simulated timeline (costs in cycles from device
+// timelines); a list that is valid in one timeline cannot deadlock: a wait cycle would need two
+// down tiles that each start before the other.  Returns false when the plan does not fit (the
+// caller then runs the two projections as two kernels).
+bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
+  if (!h.fused_ok) return false;
+  if (h.fused_M == M) return h.fused_rounds > 0;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return false;
+  h.fused_M = M;
+  h.fused_rounds = 0;
+  const alg_proj_s &up = h.up, &dn = h.down;
+  const int q = up.q, nw = h.fused_workers;
+  const int bucket = (int)(M / q), m_tiles = (bucket + kTcTileM - 1) / kTcTileM, n_blocks = q * m_tiles;
+  if (n_blocks > 4096) return false;
+  auto nkb_of = [&](const alg_proj_s &p, int i, int j) {
+    int n = 0;
+    for (int k = 0; k < q; ++k)
+      if ((p.tab.keep[i * q + j] >> k) & 1u) n += p.s[k] / kTcBlockK;
+    return n;
+  };
+  struct Item { TileRec rec; TileExt ext; double cost; int block; };
+  auto make = [&](const alg_proj_s &p, int i, int mt, int j, int col0, int cols, bool down) {
+    Item it;
+    const int nkb = nkb_of(p, i, j);
+    it.rec.row0 = i * bucket + mt * kTcTileM;
+    it.rec.rows = std::min(kTcTileM, bucket - mt * kTcTileM) | (nkb << 16);
+    it.rec.pair = (i * q + j) | (cols << 16);
+    it.rec.n0 = col0;
+    it.block = i * m_tiles + mt;
+    it.ext.dep = down ? it.block : -1;
+    it.ext.sig = down ? -1 : it.block;
+    // cycles: a K block beside a running epilogue, the GELU epilogue as a floor, fixed hand-over
+    it.cost = down ? nkb * (cols == 256 ? 509.0 : cols == 192 ? 467.0 : 460.0) + 2000.0
+                   : std::max(nkb * 640.0, 5300.0) + 700.0;
+    return it;
+  };
+  int ups_per_block = 0;
+  for (int j = 0; j < q; ++j) ups_per_block += up.r[j] / 256;
+  std::vector<Item> ups, downs;
+  for (int mt = 0; mt < m_tiles; ++mt)
+    for (int i = 0; i < q; ++i) {
+      for (int j = 0; j < q; ++j)
+        for (int t = 0; t < up.r[j] / 256; ++t) ups.push_back(make(up, i, mt, j, up.tab.ro[j] + t * 256, 256, false));
+      for (int j = 0; j < q; ++j) {
+        const int width = dn.r[j];
+        if (width % 256 && width % 192 == 0) {
+          for (int t = 0; t < width / 192; ++t) downs.push_back(make(dn, i, mt, j, dn.tab.ro[j] + t * 192, 192, true));
+        } else {
+          for (int t = 0; t < width / 256; ++t) downs.push_back(make(dn, i, mt, j, dn.tab.ro[j] + t * 256, 256, true));
+          if (width % 256) downs.push_back(make(dn, i, mt, j, dn.tab.ro[j] + (width / 256) * 256, 128, true));
+        }
+      }
+    }
+  // 1. which worker runs how much: longest-processing-time over ALL tiles (the down tiles are the
+  //    long ones and go first; the up tiles follow row block by row block as the fine filler)
+  std::vector<double> load(nw, 0.0);
+  std::vector<std::vector<Item>> my_ups(nw), my_downs(nw);
+  auto least = [&]() { return (int)(std::min_element(load.begin(), load.end()) - load.begin()); };
+  std::vector<int> order(downs.size());
+  for (size_t e = 0; e < downs.size(); ++e) order[e] = (int)e;
+  std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return downs[x].cost > downs[y].cost; });
+  for (int e : order) {
+    const int w = least();
+    load[w] += downs[e].cost;
+    my_downs[w].push_back(downs[e]);
+  }
+  for (const Item &it : ups) {
+    const int w = least();
+    load[w] += it.cost;
+    my_ups[w].push_back(it);
+  }
+  // 2. simulated timeline of the up tiles: every worker runs its own first, in row-block order
+  std::vector<std::vector<Item>> seq(nw);
+  std::vector<double> free_at(nw, 5000.0), block_done(n_blocks, 0.0);
+  const double kHandOver = 6000.0;  // last epilogue of the block, signal, counter poll
+  for (int w = 0; w < nw; ++w)
+    for (const Item &it : my_ups[w]) {
+      free_at[w] += it.cost;
+      block_done[it.block] = std::max(block_done[it.block], free_at[w]);
+      seq[w].push_back(it);
+    }
+  // 3. which down tile exactly: step 1 fixed how many tiles of which length a worker runs; tiles
+  //    of equal length are interchangeable.  Event-driven: whenever a worker becomes free it takes,
+  //    among the remaining tiles of the length it is due to run (longest first), the one whose
+  //    row block completed LAST among those already complete (best fit: early row blocks stay
+  //    available for workers that become free early), else the one that completes first.
+  {
+    std::vector<char> taken(downs.size(), 0);
+    std::vector<size_t> next_slot(nw, 0);
+    for (int w = 0; w < nw; ++w)
+      std::stable_sort(my_downs[w].begin(), my_downs[w].end(), [](const Item &x, const Item &y) { return x.cost > y.cost; });
+    size_t left = downs.size();
+    while (left > 0) {
+      int w = -1;
+      for (int v = 0; v < nw; ++v)
+        if (next_slot[v] < my_downs[v].size() && (w < 0 || free_at[v] < free_at[w])) w = v;
+      if (w < 0) break;
+      const double want = my_downs[w][next_slot[w]].cost;
+      int best = -1;
+      for (size_t e = 0; e < downs.size(); ++e) {
+        if (taken[e] || downs[e].cost != want) continue;
+        if (best < 0) { best = (int)e; continue; }
+        const double rb = block_done[downs[best].block] + kHandOver, re = block_done[downs[e].block] + kHandOver;
+        const bool b_ok = rb <= free_at[w], e_ok = re <= free_at[w];
+        if (e_ok && (!b_ok || re > rb)) best = (int)e;          // latest among the ready ones
+        else if (!e_ok && !b_ok && re < rb) best = (int)e;      // nothing ready: the first to become ready
+      }
+      taken[best] = 1;
+      --left;
+      ++next_slot[w];
+      free_at[w] = std::max(free_at[w], block_done[downs[best].block] + kHandOver) + downs[best].cost;
+      seq[w].push_back(downs[best]);
+    }
+  }
+  size_t rounds = 0;
+  for (int w = 0; w < nw; ++w) rounds = std::max(rounds, seq[w].size());
+  rounds += 1;
+  if ((int)rounds > kFfnSeqCap) return false;
+  if (const char *dump = std::getenv("ALGPROJ_PLAN_DUMP")) {
+    for (int w = 0; w < nw; w += (dump[0] == 'a' ? 1 : 20)) {
+      fprintf(stderr, "worker %d (model end %.0f):", w, free_at[w]);
+      for (const Item &it : seq[w])
+        fprintf(stderr, " %c%d/%d(k%d,c%d)", it.ext.dep >= 0 ? 'D' : 'U', it.block, it.ext.dep >= 0 ? (int)block_done[it.block] : 0,
+                it.rec.rows >> 16, it.rec.pair >> 16);
+      fprintf(stderr, "\n");
+    }
+  }
+  TileRec end;
+  end.row0 = -1, end.rows = 0, end.pair = 0, end.n0 = 0;
+  const TileExt none = {-1, -1};
+  for (int w = 0; w < nw; ++w)
+    for (size_t pos = 0; pos < (size_t)kFfnSeqCap; ++pos) {
+      h.h_fplan[(size_t)w * kFfnSeqCap + pos] = pos < seq[w].size() ? seq[w][pos].rec : end;
+      h.h_fext[(size_t)w * kFfnSeqCap + pos] = pos < seq[w].size() ? seq[w][pos].ext : none;
+    }
+  const size_t n = (size_t)nw * kFfnSeqCap;
+  if (cudaMemcpyAsync(h.d_fplan, h.h_fplan, n * sizeof(TileRec), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h.d_fext, h.h_fext, n * sizeof(TileExt), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    h.fused_M = -1;
+    return false;
+  }
+  h.fused_rounds = (int)rounds;
+  h.fused_blocks = n_blocks;
+  h.fused_target = ups_per_block;
+  return true;
+}
+
+// Argument block of one projection as the fused kernel needs it (tables by value).
+void fill_fused_proj(ProjArgs &a, const alg_proj_s &p, const void *X, int64_t ldx, const void *W, int64_t ldw,
+                     const void *bias, alg_act_t act, void *Y, int64_t ldy, alg_dtype_t y_dtype, int64_t M,
+                     int a_cyclic_rows, int out_cyclic_rows) {
+  std::memset(&a, 0, sizeof(a));
+  a.tab = p.d_tab;
+  a.n_classes = p.tab.n_classes;
+  a.st.valid = 1;
+  for (int e = 0; e <= p.q; ++e) a.st.so[e] = p.tab.so[e], a.st.ro[e] = p.tab.ro[e];
+  for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = p.tab.keep[e];
+  a.q = p.q;
+  a.X = X, a.ldx = ldx, a.W = W, a.ldw = ldw, a.bias = bias, a.act = (int)act;
+  a.Y = Y, a.ldy = ldy, a.y_bf16 = y_dtype == ALG_BF16;
+  a.M = (int)M, a.K = p.K, a.N = p.N;
+  a.status = p.d_status;
+  a.a_cyclic_rows = a_cyclic_rows;
+  a.out_cyclic_rows = out_cyclic_rows;
+  a.cyclic_rows = (int)(M / p.q);
+  a.dbg = std::getenv("ALGPROJ_DBG") ? atoi(std::getenv("ALGPROJ_DBG")) : 0;
+  a.trace = g_trace;
+  a.trace_cap = g_trace_cap;
+}
+
+}  // namespace
 
 alg_status_t alg_ffn_destroy(alg_ffn_t h) {
   if (!h) return ALG_ERR_INVALID_ARG;
   for (int e = 0; e < 5; ++e)
     if (h->ev[e]) cudaEventDestroy(h->ev[e]);
+  if (h->d_fplan) cudaFree(h->d_fplan);
+  if (h->h_fplan) cudaFreeHost(h->h_fplan);
+  if (h->d_fext) cudaFree(h->d_fext);
+  if (h->h_fext) cudaFreeHost(h->h_fext);
+  if (h->d_counters) cudaFree(h->d_counters);
   free_proj(h->down);
   free_proj(h->up);
   delete h;
@@ -584,6 +793,22 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   const bool tm = h->timing;
   if (tm) cudaEventRecord(h->ev[0], st);
   const bool cyc = h->up.sched == ALG_SCHED_CYCLIC && use_tc(h->up) && use_tc(h->down) && M % h->up.q == 0;
+  if (cyc && !tm && aligned16(ws + L.h) && prepare_fused_plan(*h, M, st)) {
+    // both projections in one persistent kernel
+    FfnArgs fa;
+    void *Hf = ws + L.h;
+    const int rows = (int)(M / h->up.q);
+    fill_fused_proj(fa.p[0], h->up, X, h->D, W_up, h->F, b_up, act, Hf, h->F, ALG_BF16, M, rows, 0);
+    fill_fused_proj(fa.p[1], h->down, Hf, h->F, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, M, 0, rows);
+    fa.plan = h->d_fplan;
+    fa.ext = h->d_fext;
+    fa.plan_stride = kFfnSeqCap;
+    fa.plan_rounds = h->fused_rounds;
+    fa.counters = h->d_counters;
+    fa.n_blocks = h->fused_blocks;
+    fa.target = (unsigned long long)h->fused_target;
+    return cuda_status(launch_ffn_tc(fa, h->fused_workers, st));
+  }
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;

@@ -139,6 +139,25 @@ struct ProjArgs {
 
 cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
 
+// Fused two-projection FFN kernel (ffn_tc.cu).  Extension of a tile record: an up tile carries the
+// counter it reports to (`sig`, -1 for down tiles), a down tile the counter it waits for (`dep`).
+struct TileExt {
+  int dep;
+  int sig;
+};
+constexpr int kFfnSeqCap = 160;  // tile records per CTA
+struct FfnArgs {
+  ProjArgs p[2];                 // [0] up (X -> H, activation), [1] down (H -> Y); tables by value (q <= 8)
+  const TileRec *plan;           // [n_workers][plan_stride] records, the last of a worker is the end marker
+  const TileExt *ext;            // parallel to plan
+  int plan_stride, plan_rounds;
+  unsigned long long *counters;  // one per 128-row block of H: up tiles finished so far; [n_blocks] = CTAs that have left
+  int n_blocks;
+  unsigned long long target;     // up tiles per row block: the value a counter must reach before the block is read
+                                 // (the last CTA to leave clears the counters, so the value is the same every launch)
+};
+cudaError_t launch_ffn_tc(const FfnArgs &a, int n_workers, cudaStream_t st);
+
 // tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
 // (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.
 constexpr int kTcSeqCap = 224, kTc2SeqCap = 48;  // precomputed tile records per worker

@@ -213,6 +213,46 @@ def test_cyclic_plan_follows_M_and_stream_capture():
     assert torch.equal(cyc.forward(X, None, W, act="gelu"), want)   # planned on the host now
 
 
+@pytest.mark.parametrize("q,M,D,F", [(2, 8192, 768, 3072), (2, 848, 256, 512), (4, 2056, 512, 1024)])
+def test_one_kernel_ffn_matches_two_kernel_ffn(q, M, D, F, monkeypatch):
+    """Cyclic schedule: the FFN runs as one persistent kernel whose down tiles wait for the row
+    blocks of H they read.  Same tiles, same K order, so the result must equal the two-kernel path
+    bit for bit (bf16 and fp32 outputs, with biases), also when replayed from a CUDA graph (the
+    kernel clears its own dependency counters), and must pass the oracle tolerance."""
+    wl = synth.make_workload("fused", config=8, variant=q * 100000 + M, dtype="bf16", q=q, M=M, D=D, F=F,
+                             types=synth.cyclic_types(M, q))
+    bu, bd = synth.normal(41, (wl.F,), 0.1), synth.normal(42, (wl.D,), 0.1)
+    monkeypatch.setenv("ALGPROJ_NO_FUSED", "1")
+    two = _ffn(wl, schedule="cyclic")
+    Y2 = _run_ffn(wl, two, torch.float32, b_up=bu, b_down=bd, types=False)
+    Y2b = _run_ffn(wl, two, torch.bfloat16, b_up=bu, b_down=bd, types=False)
+    monkeypatch.delenv("ALGPROJ_NO_FUSED")
+    one = _ffn(wl, schedule="cyclic")
+    launches = binding.launch_count()
+    Y1 = _run_ffn(wl, one, torch.float32, b_up=bu, b_down=bd, types=False)
+    assert binding.launch_count() - launches == 1          # one kernel
+    Y1b = _run_ffn(wl, one, torch.bfloat16, b_up=bu, b_down=bd, types=False)
+    assert torch.equal(Y1, Y2) and torch.equal(Y1b, Y2b)
+    ref = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, b_up=bu, b_down=bd)
+    H.assert_bf16_close(H.to_np(Y1), ref, False, f"one-kernel FFN q={q} M={M}")
+    # graph replay: the same launch twice
+    X = H.to_dev(wl.X, "bf16")
+    Wu, Wd = H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16")
+    bud, bdd = H.to_dev(bu, "bf16"), H.to_dev(bd, "bf16")
+    Y = torch.empty_like(Y1)
+    ws = torch.empty(one.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            one.forward(X, None, Wu, Wd, b_up=bud, b_down=bdd, act="gelu", out=Y, workspace=ws, stream=stream)
+    for _ in range(3):
+        Y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(Y, Y1) and one.last_status() == 0
+
+
 def test_pilot_tensor_square_law_and_interval_schedule():
     """The law and shape of the paper's pilot FFN projections: Q_2 (x) Q_2 (36 block products,
     9/16 of the dense MACs), D = 768 = 4 x 192, F = 1536 = 4 x 384, interval schedule."""
