@@ -215,18 +215,18 @@ def test_cyclic_plan_follows_M_and_stream_capture():
 
 @pytest.mark.parametrize("q,M,D,F", [(2, 8192, 768, 3072), (2, 848, 256, 512), (4, 2056, 512, 1024)])
 def test_one_kernel_ffn_matches_two_kernel_ffn(q, M, D, F, monkeypatch):
-    """Cyclic schedule: the FFN runs as one persistent kernel whose down tiles wait for the row
-    blocks of H they read.  Same tiles, same K order, so the result must equal the two-kernel path
+    """Cyclic schedule, opt-in (ALGPROJ_FUSED=1 at handle creation): the FFN runs as one persistent
+    kernel whose down tiles wait for the row blocks of H they read.  Same tiles, same K order, so the result must equal the two-kernel path
     bit for bit (bf16 and fp32 outputs, with biases), also when replayed from a CUDA graph (the
     kernel clears its own dependency counters), and must pass the oracle tolerance."""
     wl = synth.make_workload("fused", config=8, variant=q * 100000 + M, dtype="bf16", q=q, M=M, D=D, F=F,
                              types=synth.cyclic_types(M, q))
     bu, bd = synth.normal(41, (wl.F,), 0.1), synth.normal(42, (wl.D,), 0.1)
-    monkeypatch.setenv("ALGPROJ_NO_FUSED", "1")
+    monkeypatch.delenv("ALGPROJ_FUSED", raising=False)
     two = _ffn(wl, schedule="cyclic")
     Y2 = _run_ffn(wl, two, torch.float32, b_up=bu, b_down=bd, types=False)
     Y2b = _run_ffn(wl, two, torch.bfloat16, b_up=bu, b_down=bd, types=False)
-    monkeypatch.delenv("ALGPROJ_NO_FUSED")
+    monkeypatch.setenv("ALGPROJ_FUSED", "1")      # read when the handle is created
     one = _ffn(wl, schedule="cyclic")
     launches = binding.launch_count()
     Y1 = _run_ffn(wl, one, torch.float32, b_up=bu, b_down=bd, types=False)
