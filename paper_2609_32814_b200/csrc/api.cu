@@ -571,14 +571,14 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
   const alg_proj_s &up = h.up, &dn = h.down;
   const int q = up.q, nw = h.fused_workers;
   const int bucket = (int)(M / q), m_tiles = (bucket + kTcTileM - 1) / kTcTileM, n_blocks = q * m_tiles;
-  if (n_blocks > 4096) return false;
+  if (n_blocks * q > 4096) return false;
   auto nkb_of = [&](const alg_proj_s &p, int i, int j) {
     int n = 0;
     for (int k = 0; k < q; ++k)
       if ((p.tab.keep[i * q + j] >> k) & 1u) n += p.s[k] / kTcBlockK;
     return n;
   };
-  struct Item { TileRec rec; TileExt ext; double cost; int block; };
+  struct Item { TileRec rec; TileExt ext; double cost; int block; int group; uint32_t mask; };
   auto make = [&](const alg_proj_s &p, int i, int mt, int j, int col0, int cols, bool down) {
     Item it;
     const int nkb = nkb_of(p, i, j);
@@ -587,15 +587,15 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
     it.rec.pair = (i * q + j) | (cols << 16);
     it.rec.n0 = col0;
     it.block = i * m_tiles + mt;
+    it.group = j;
+    it.mask = p.tab.keep[i * q + j];
     it.ext.dep = down ? it.block : -1;
-    it.ext.sig = down ? -1 : it.block;
+    it.ext.sig = down ? -1 : it.block * q + j;   // an up tile completes part of hidden group j of its row block
     // cycles: a K block beside a running epilogue, the GELU epilogue as a floor, fixed hand-over
     it.cost = down ? nkb * (cols == 256 ? 509.0 : cols == 192 ? 467.0 : 460.0) + 2000.0
                    : std::max(nkb * 640.0, 5300.0) + 700.0;
     return it;
   };
-  int ups_per_block = 0;
-  for (int j = 0; j < q; ++j) ups_per_block += up.r[j] / 256;
   std::vector<Item> ups, downs;
   for (int mt = 0; mt < m_tiles; ++mt)
     for (int i = 0; i < q; ++i) {
@@ -631,14 +631,28 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
   }
   // 2. simulated timeline of the up tiles: every worker runs its own first, in row-block order
   std::vector<std::vector<Item>> seq(nw);
-  std::vector<double> free_at(nw, 5000.0), block_done(n_blocks, 0.0);
-  const double kHandOver = 6000.0;  // last epilogue of the block, signal, counter poll
+  std::vector<double> free_at(nw, 5000.0), part_done((size_t)n_blocks * q, 0.0);
+  const double kHandOver = 6000.0;  // last epilogue of the part, signal, counter poll
   for (int w = 0; w < nw; ++w)
     for (const Item &it : my_ups[w]) {
       free_at[w] += it.cost;
-      block_done[it.block] = std::max(block_done[it.block], free_at[w]);
+      double &d = part_done[(size_t)it.block * q + it.group];
+      d = std::max(d, free_at[w]);
       seq[w].push_back(it);
     }
+  // earliest start of a down tile: its first kept hidden group must be complete, a later one by the
+  // time the K loop reaches it
+  auto ready_at = [&](const Item &it) {
+    double start = 0.0, before = 0.0;
+    for (int k = 0; k < q; ++k) {
+      if (!((it.mask >> k) & 1u)) continue;
+      start = std::max(start, part_done[(size_t)it.block * q + k] + kHandOver - before);
+      before += (dn.s[k] / kTcBlockK) * 467.0;
+    }
+    return start;
+  };
+  std::vector<double> block_done(downs.size(), 0.0);   // per down tile: when it may start
+  for (size_t e = 0; e < downs.size(); ++e) block_done[e] = ready_at(downs[e]) - kHandOver;
   // 3. which down tile exactly: step 1 fixed how many tiles of which length a worker runs; tiles
   //    of equal length are interchangeable.  Event-driven: whenever a worker becomes free it takes,
   //    among the remaining tiles of the length it is due to run (longest first), the one whose
@@ -660,7 +674,7 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
       for (size_t e = 0; e < downs.size(); ++e) {
         if (taken[e] || downs[e].cost != want) continue;
         if (best < 0) { best = (int)e; continue; }
-        const double rb = block_done[downs[best].block] + kHandOver, re = block_done[downs[e].block] + kHandOver;
+        const double rb = block_done[best] + kHandOver, re = block_done[e] + kHandOver;
         const bool b_ok = rb <= free_at[w], e_ok = re <= free_at[w];
         if (e_ok && (!b_ok || re > rb)) best = (int)e;          // latest among the ready ones
         else if (!e_ok && !b_ok && re < rb) best = (int)e;      // nothing ready: the first to become ready
@@ -668,7 +682,7 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
       taken[best] = 1;
       --left;
       ++next_slot[w];
-      free_at[w] = std::max(free_at[w], block_done[downs[best].block] + kHandOver) + downs[best].cost;
+      free_at[w] = std::max(free_at[w], block_done[best] + kHandOver) + downs[best].cost;
       seq[w].push_back(downs[best]);
     }
   }
@@ -680,8 +694,7 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
     for (int w = 0; w < nw; w += (dump[0] == 'a' ? 1 : 20)) {
       fprintf(stderr, "worker %d (model end %.0f):", w, free_at[w]);
       for (const Item &it : seq[w])
-        fprintf(stderr, " %c%d/%d(k%d,c%d)", it.ext.dep >= 0 ? 'D' : 'U', it.block, it.ext.dep >= 0 ? (int)block_done[it.block] : 0,
-                it.rec.rows >> 16, it.rec.pair >> 16);
+        fprintf(stderr, " %c%d(k%d,c%d)", it.ext.dep >= 0 ? 'D' : 'U', it.block, it.rec.rows >> 16, it.rec.pair >> 16);
       fprintf(stderr, "\n");
     }
   }
@@ -701,8 +714,7 @@ bool prepare_fused_plan(alg_ffn_s &h, int64_t M, cudaStream_t st) {
     return false;
   }
   h.fused_rounds = (int)rounds;
-  h.fused_blocks = n_blocks;
-  h.fused_target = ups_per_block;
+  h.fused_blocks = n_blocks * q;
   return true;
 }
 
@@ -805,8 +817,8 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
     fa.plan_stride = kFfnSeqCap;
     fa.plan_rounds = h->fused_rounds;
     fa.counters = h->d_counters;
-    fa.n_blocks = h->fused_blocks;
-    fa.target = (unsigned long long)h->fused_target;
+    fa.n_counters = h->fused_blocks;
+    for (int g = 0; g < kParamQ; ++g) fa.target[g] = g < h->up.q ? h->up.r[g] / 256 : 0;
     return cuda_status(launch_ffn_tc(fa, h->fused_workers, st));
   }
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;

@@ -151,10 +151,12 @@ struct FfnArgs {
   const TileRec *plan;           // [n_workers][plan_stride] records, the last of a worker is the end marker
   const TileExt *ext;            // parallel to plan
   int plan_stride, plan_rounds;
-  unsigned long long *counters;  // one per 128-row block of H: up tiles finished so far; [n_blocks] = CTAs that have left
-  int n_blocks;
-  unsigned long long target;     // up tiles per row block: the value a counter must reach before the block is read
-                                 // (the last CTA to leave clears the counters, so the value is the same every launch)
+  // one counter per (128-row block of H, hidden group): up tiles of that part finished so far;
+  // counters[n_counters] = CTAs that have left (the last one clears everything for the next launch)
+  unsigned long long *counters;
+  int n_counters;
+  int target[kParamQ];           // up tiles per (row block, hidden group g): the value the counter must reach
+                                 // before a down tile reads hidden group g of the block
 };
 cudaError_t launch_ffn_tc(const FfnArgs &a, int n_workers, cudaStream_t st);
 

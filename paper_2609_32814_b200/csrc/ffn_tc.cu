@@ -7,11 +7,12 @@
 // work (last epilogue, prologue, first operands from DRAM) and the down projection has only 1.7
 // tiles per CTA to balance.  Here every CTA walks one host-planned list that holds up tiles and
 // down tiles:
-//   * an up tile (128 rows of one type x 256 hidden columns) ends with its rows of H stored in
-//     bucketed order; a signal warp then publishes it: device-scope fence + one atomic add on the
-//     counter of the tile's row block;
-//   * a down tile (the same 128 rows x 256, 192 or 128 output columns) may start once the counter of
-//     its row block has reached the number of up tiles of that block; its A operand is H.
+//   * an up tile (128 rows of one type x 256 columns of one hidden group) ends with its rows of H
+//     stored in bucketed order; a signal warp then publishes it: device-scope fence + one atomic
+//     add on the counter of (row block, hidden group);
+//   * a down tile (the same 128 rows x 256, 192 or 128 output columns) reads H one kept hidden
+//     group after the other; before the loads of a group it waits until that group's counter has
+//     reached the number of up tiles of the group.
 // The planner (api.cu) list-schedules the tiles on the host: up tiles first, row block by row
 // block, then down tiles longest first as they become ready, in a simulated timeline; a list that
 // is valid in a simulated timeline cannot deadlock (a wait cycle would need two down tiles that
@@ -176,33 +177,36 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_up, const __grid_constant_
       const int a_row = a.a_cyclic_rows ? row0 - type_i * a.a_cyclic_rows : row0;
       const uint32_t tx_bytes = (uint32_t)(kABytes + (cols >> 6) * kBChunkBytes);
       if (loads_a && lane == 0) FTRACE(0, down ? 5 : 1);
-      if (down && loads_a) {
-        // the rows of H this tile reads must be complete: wait for the row block's counter
-        if (lane == 0) {
-          const unsigned long long *cnt = fa.counters + dep;
-          const long long t0 = clock64();
-          unsigned long long seen;
-          while (true) {
-            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(cnt) : "memory");
-            if (seen >= fa.target) break;
-            __nanosleep(100);
-            if (ctl->abort_flag || clock64() - t0 > kTimeoutCycles) {
-              ctl->abort_flag = 1;
-              atomicExch(status, (int)ALG_ERR_DEVICE_TIMEOUT);
-              ok = false;
-              break;
-            }
-          }
-          // H was written through the generic proxy by other SMs and is read by the copy engine
-          asm volatile("fence.proxy.async;" ::: "memory");
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane == 0) FTRACE(0, 6);
-      }
       for (int k = 0; k < q && ok; ++k) {
         if (!((mask >> k) & 1u)) continue;
         const int k_begin = a.st.so[k], k_end = a.st.so[k + 1];
+        if (down && loads_a) {
+          // hidden group k of these rows of H must be complete: wait for the counter of (row block, k).
+          // The other kept group of the tile is awaited only when the K loop reaches it, so its
+          // hand-over hides behind the MMAs of this one.
+          if (lane == 0) {
+            const unsigned long long *cnt = fa.counters + (size_t)dep * q + k;
+            const unsigned long long need = (unsigned long long)fa.target[k];
+            const long long t0 = clock64();
+            unsigned long long seen;
+            while (true) {
+              asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(cnt) : "memory");
+              if (seen >= need) break;
+              __nanosleep(100);
+              if (ctl->abort_flag || clock64() - t0 > kTimeoutCycles) {
+                ctl->abort_flag = 1;
+                atomicExch(status, (int)ALG_ERR_DEVICE_TIMEOUT);
+                ok = false;
+                break;
+              }
+            }
+            // H was written through the generic proxy by other SMs and is read by the copy engine
+            asm volatile("fence.proxy.async;" ::: "memory");
+            FTRACE(0, 6);
+          }
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
         for (int k0 = k_begin; k0 < k_end; k0 += kTcBlockK) {
           ok = __all_sync(0xffffffffu, wait_bar(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, status));
           if (!ok) break;
@@ -416,9 +420,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_up, const __grid_constant_
   // this kernel has completed), so a launch recorded in a CUDA graph replays correctly.
   if (threadIdx.x == 0) {
     __threadfence();
-    const unsigned long long left = atomicAdd(fa.counters + fa.n_blocks, 1ull);
+    const unsigned long long left = atomicAdd(fa.counters + fa.n_counters, 1ull);
     if (left == (unsigned long long)gridDim.x - 1) {
-      for (int b = 0; b <= fa.n_blocks; ++b) fa.counters[b] = 0;
+      for (int b = 0; b <= fa.n_counters; ++b) fa.counters[b] = 0;
       __threadfence();
     }
   }
