@@ -128,22 +128,64 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_fused_kernel(const Bucke
   const int row_begin = blockIdx.x * kFusedThreads;
   int before = 0, all = 0;
   const int n_super = (a.M + 511) >> 9;
-  for (int sb = warp; sb < n_super; sb += 32) {
-    int tt[16];
+  if (nt <= 8) {
+    // q + 1 <= 8 kinds: every lane keeps its own histogram packed in two 64-bit words (16 bits per
+    // kind; a lane sees at most 16 rows per pass and a warp total stays below 2^16), so a pass
+    // costs two instructions per row and one shuffle reduction instead of (q+1) ballots per row
+    unsigned long long all_lo = 0, all_hi = 0, bef_lo = 0, bef_hi = 0;
+    for (int sb = warp; sb < n_super; sb += 32) {
+      int tt[16];
 #pragma unroll
-    for (int u = 0; u < 16; ++u) {
-      const int row = sb * 512 + u * 32 + lane;
-      tt[u] = row < a.M ? row_type(a, row) : -1;
-    }
-    int mine = 0;
-#pragma unroll
-    for (int u = 0; u < 16; ++u)
-      for (int k = 0; k < nt; ++k) {
-        const unsigned b = __ballot_sync(0xffffffffu, tt[u] == k);
-        if (lane == k) mine += __popc(b);
+      for (int u = 0; u < 16; ++u) {
+        const int row = sb * 512 + u * 32 + lane;
+        tt[u] = row < a.M ? row_type(a, row) : -1;
       }
-    all += mine;
-    if (sb * 512 < row_begin) before += mine;
+      unsigned long long lo = 0, hi = 0;
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        const unsigned long long one = tt[u] < 0 ? 0ull : 1ull << ((tt[u] & 3) * 16);
+        if (tt[u] < 4) lo += one; else hi += one;
+      }
+      all_lo += lo, all_hi += hi;
+      if (sb * 512 < row_begin) bef_lo += lo, bef_hi += hi;
+      if (((sb / 32) & 63) == 63) {  // fold into the 32-bit counters before a 16-bit field can overflow
+        for (int d = 16; d > 0; d >>= 1) {
+          all_lo += __shfl_xor_sync(0xffffffffu, all_lo, d), all_hi += __shfl_xor_sync(0xffffffffu, all_hi, d);
+          bef_lo += __shfl_xor_sync(0xffffffffu, bef_lo, d), bef_hi += __shfl_xor_sync(0xffffffffu, bef_hi, d);
+        }
+        if (lane < nt) {
+          all += (int)(((lane < 4 ? all_lo : all_hi) >> ((lane & 3) * 16)) & 0xFFFF);
+          before += (int)(((lane < 4 ? bef_lo : bef_hi) >> ((lane & 3) * 16)) & 0xFFFF);
+        }
+        all_lo = all_hi = bef_lo = bef_hi = 0;
+      }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+      all_lo += __shfl_xor_sync(0xffffffffu, all_lo, d), all_hi += __shfl_xor_sync(0xffffffffu, all_hi, d);
+      bef_lo += __shfl_xor_sync(0xffffffffu, bef_lo, d), bef_hi += __shfl_xor_sync(0xffffffffu, bef_hi, d);
+    }
+    if (lane < nt) {
+      all += (int)(((lane < 4 ? all_lo : all_hi) >> ((lane & 3) * 16)) & 0xFFFF);
+      before += (int)(((lane < 4 ? bef_lo : bef_hi) >> ((lane & 3) * 16)) & 0xFFFF);
+    }
+  } else {
+    for (int sb = warp; sb < n_super; sb += 32) {
+      int tt[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        const int row = sb * 512 + u * 32 + lane;
+        tt[u] = row < a.M ? row_type(a, row) : -1;
+      }
+      int mine = 0;
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        for (int k = 0; k < nt; ++k) {
+          const unsigned b = __ballot_sync(0xffffffffu, tt[u] == k);
+          if (lane == k) mine += __popc(b);
+        }
+      all += mine;
+      if (sb * 512 < row_begin) before += mine;
+    }
   }
   if (lane < nt) s_before[warp][lane] = before, s_all[warp][lane] = all;
   for (int e = tid; e < 32 * (kMaxQ + 1); e += kFusedThreads) (&s_wcnt[0][0])[e] = 0;
