@@ -71,12 +71,12 @@ typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } a
  *           batch whose sequence length is a multiple of q); `types` may be NULL.
  *           With q | M the tensor-core path needs no permutation, and the tile sequences of its
  *           persistent CTAs depend only on (handle, M): they are planned on the host at the
- *           first forward call with a given M and kept in device memory the handle owns (sized
- *           at create; forward allocates nothing).  That first call copies the plan on `stream`
- *           and waits for the copy; later calls with the same M do not synchronise.  If a new M
- *           is first seen while `stream` is being captured, the kernels plan for themselves
- *           instead (same result).  Calls on one handle share the plan: do not run forward
- *           calls with different M on the same handle concurrently. */
+ *           first forward call with a given M, uploaded asynchronously on `stream` (no host
+ *           wait) into device memory the handle owns (sized at create; forward allocates
+ *           nothing) and kept for the last few M.  A call made while `stream` is being captured
+ *           lets the kernels plan for themselves instead (same result), so a captured graph
+ *           never depends on the handle's plan cache.  Forward calls on one handle must be
+ *           ordered on the GPU (one stream, or events between streams). */
 typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1 } alg_schedule_t;
 
 /* Kernel families, reported by alg_proj_kernel_path(). */
@@ -87,6 +87,35 @@ typedef enum {
 } alg_path_t;
 
 #define ALG_MAX_Q 32
+
+/* Per-handle options (alg_proj_set_option / alg_ffn_set_option).  They replace process-wide
+ * switches: nothing in the library reads the environment.  Set them between forward calls,
+ * not concurrently with one; a value the handle's shape cannot honour is refused with
+ * ALG_ERR_UNSUPPORTED_SHAPE and changes nothing.
+ *   GEMM_KERNEL       which prefill tensor-core kernel runs: 0 = the library's choice (default),
+ *                     1 = one-CTA tiles (tcgen05 cta_group::1), 2 = CTA pairs (cta_group::2;
+ *                     needs every output group width to be a multiple of 128).
+ *   TILE_N            tile width of the one-CTA kernel: 0 = automatic, or 128 / 192 / 256 when
+ *                     that divides every output group width.
+ *   SMALL_M_KERNEL    1 (default): M <= 64 runs the weight-streaming kernels; 0: the prefill
+ *                     kernels take every M.
+ *   HOST_PLAN         1 (default): cyclic-schedule tile sequences are planned on the host;
+ *                     0: every CTA plans for itself.
+ *   WAIT_LIMIT_CYCLES bound of every device-side wait (mbarrier, counter), in SM clock cycles;
+ *                     default 4e9 (about 2 s).  A wait that runs out sets
+ *                     ALG_ERR_DEVICE_TIMEOUT in the status word and the kernel returns.
+ *   TEST_STALL_BYTES  test aid, default 0: the small-M kernels add this many bytes to what they
+ *                     expect on their weight barrier.  The bytes never arrive, every issued
+ *                     copy still lands, the bounded wait runs out and the call reports
+ *                     ALG_ERR_DEVICE_TIMEOUT -- the way to exercise that path without a fault. */
+typedef enum {
+  ALG_OPT_GEMM_KERNEL = 1,
+  ALG_OPT_TILE_N = 2,
+  ALG_OPT_SMALL_M_KERNEL = 3,
+  ALG_OPT_HOST_PLAN = 4,
+  ALG_OPT_WAIT_LIMIT_CYCLES = 5,
+  ALG_OPT_TEST_STALL_BYTES = 6
+} alg_option_t;
 
 /* ---- projection handle ---------------------------------------------------------------------
  * alg_proj_create: build the interaction table for q groups (Eqs. q-product-diag/off, or the
@@ -101,6 +130,7 @@ alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
                              const int32_t *out_widths, alg_dtype_t dtype, alg_table_t table,
                              const uint8_t *custom_keep, alg_schedule_t schedule);
 alg_status_t alg_proj_destroy(alg_proj_t h);
+alg_status_t alg_proj_set_option(alg_proj_t h, alg_option_t option, int64_t value);
 
 /* Bytes of device scratch a forward call with at most max_M rows needs (row permutation,
  * bucket offsets, and -- on the tensor-core path -- the type-bucketed copy of X).  The contents
@@ -115,7 +145,13 @@ alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes
  * bf16 pointers and leading dimensions must keep rows 16-byte aligned (multiples of 8
  * elements).  M = 0 is a successful no-op; a type with no rows is legal.
  * M <= 64 with bf16 runs the decode kernel (when its per-CTA weight slice fits shared memory),
- * larger M the prefill kernels. */
+ * larger M the prefill kernels.
+ * Kernels are launched with programmatic stream serialization: they may start while the
+ * kernel before them on `stream` is finishing, and wait for it before they touch X, bias, Y or
+ * the workspace.  The decode kernel requests W before that wait (weights do not change during
+ * a step): W must not be written by the kernel that immediately precedes the call on `stream`.
+ * `types` may be: it is read once early to choose the weight blocks to request and again after
+ * the wait; if the two readings differ the blocks are requested again. */
 alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const int32_t *types,
                               int64_t M, const void *W, int64_t ldw, const void *bias,
                               alg_act_t act, void *Y, int64_t ldy, alg_dtype_t y_dtype,
@@ -160,7 +196,8 @@ alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *
 /* Kernel family a forward call with M rows would use. */
 alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path);
 /* Read and clear the handle's device status word (ALG_OK, ALG_ERR_BAD_TYPE or
- * ALG_ERR_DEVICE_TIMEOUT).  Synchronises `stream` first. */
+ * ALG_ERR_DEVICE_TIMEOUT).  Synchronises `stream` first.  After ALG_ERR_DEVICE_TIMEOUT the
+ * handle's internal counters are reset, so the next forward call starts clean. */
 alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *status);
 
 /* ---- FFN handle: Y = act(X *_q W_up + b_up) *_q W_down + b_down  ---------------------------
@@ -173,6 +210,7 @@ alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths,
                             const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,
                             const uint8_t *custom_keep, alg_schedule_t schedule);
 alg_status_t alg_ffn_destroy(alg_ffn_t h);
+alg_status_t alg_ffn_set_option(alg_ffn_t h, alg_option_t option, int64_t value);  /* both projections */
 alg_status_t alg_ffn_workspace_bytes(alg_ffn_t h, int64_t max_M, size_t *bytes);
 alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, int64_t M,
                              const void *W_up, const void *b_up, const void *W_down,

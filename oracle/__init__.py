@@ -50,6 +50,10 @@ def _load():
                                        ctypes.c_int, i32p, i32p, u8p]
         lib.star_proj_alg1.argtypes = [f64p, i64, i32p, i64, f64p, i64, f64p, i64,
                                        ctypes.c_int, i32p, i32p, u8p]
+        lib.star_proj_entries.argtypes = [f64p, i64, i32p, i64, f64p, i64, f64p, ctypes.c_int, i32p, i32p, u8p,
+                                          i64p, i64p, i64, f64p]
+        lib.star_gelu_array.argtypes = [f64p, i64]
+        lib.star_gelu_array.restype = None
         lib.star_square.argtypes = [f64p, f64p, f64p, ctypes.c_int, i32p, i32p, i32p]
         lib.star_gelu.restype = ctypes.c_double
         lib.star_gelu.argtypes = [ctypes.c_double]
@@ -149,6 +153,45 @@ def proj(X, types, W, s, r, keep=None, bias=None, form: str = "rows") -> np.ndar
     else:
         raise OracleError(f"unknown form {form!r}")
     return Y
+
+
+def proj_entries(X, types, W, s, r, rows, cols, keep=None, bias=None) -> np.ndarray:
+    """Single outputs Y[rows[e], cols[e]] of proj(), each summed straight from the definition."""
+    lib = _load()
+    X, W, types, s, r = _f64(X), _f64(W), _i32(types), _i32(s), _i32(r)
+    q = len(s)
+    if keep is None:
+        keep = support(q, "qq")
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    M, K = X.shape
+    K2, N = W.shape
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    if K != K2 or int(s.sum()) != K or int(r.sum()) != N or len(r) != q or len(types) != M or rows.shape != cols.shape:
+        raise OracleError("shape mismatch")
+    out = np.empty(rows.shape, dtype=np.float64)
+    b = None if bias is None else _f64(bias)
+    f64, i32, u8, i64 = ctypes.c_double, ctypes.c_int32, ctypes.c_uint8, ctypes.c_int64
+    _check(lib.star_proj_entries(_p(X, f64), K, _p(types, i32), M, _p(W, f64), N, _p(b, f64), q, _p(s, i32),
+                                 _p(r, i32), _p(keep, u8), _p(rows, i64), _p(cols, i64), rows.size, _p(out, f64)))
+    return out
+
+
+def gelu_array(z) -> np.ndarray:
+    """Exact GELU of every element (a new fp64 array)."""
+    out = np.array(z, dtype=np.float64, order="C", copy=True)
+    _load().star_gelu_array(_p(out, ctypes.c_double), out.size)
+    return out
+
+
+def ffn_entries(X, types, W_up, W_down, dw, fw, rows, cols, keep=None, b_up=None, b_down=None) -> np.ndarray:
+    """Single outputs Y[rows[e], cols[e]] of ffn(): the hidden rows the entries need are computed in
+    full (fp64, never rounded), the entries of the second projection one by one."""
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    uniq, inv = np.unique(rows, return_inverse=True)
+    types = _i32(types)
+    H = gelu_array(proj(_f64(X)[uniq], types[uniq], W_up, dw, fw, keep=keep, bias=b_up))
+    return proj_entries(H, types[uniq], W_down, fw, dw, inv, cols, keep=keep, bias=b_down)
 
 
 def square(A, B, a, c, d) -> np.ndarray:

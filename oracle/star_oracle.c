@@ -150,8 +150,49 @@ int star_proj_rows(const double *X, int64_t ldx, const int32_t *types, int64_t M
 }
 
 /* ---------------------------------------------------------------------------------------
- * The same function in the batched order of Algorithm 1:  Y <- 0; for each type i build
- * the index set I_i; for each output group j and k in B(i,j): Y_j[I_i] += X_k[I_i] W_{kj}.
+ * Single output entries of the same projection, straight from the definition
+ * (Eq. recursive-row-action): for e = 0..n_entries-1 with (b, n) = (rows[e], cols[e]), n in
+ * output group j,   out[e] = bias[n] + sum_{k in B(t_b, j)} sum_{c in S_k} X[b,c] W[c,n].
+ * Lets the tests sample outputs of problems far too large to compute in full.
+ * ------------------------------------------------------------------------------------- */
+int star_proj_entries(const double *X, int64_t ldx, const int32_t *types, int64_t M,
+                      const double *W, int64_t ldw, const double *bias, int q,
+                      const int32_t *s, const int32_t *r, const uint8_t *keep,
+                      const int64_t *rows, const int64_t *cols, int64_t n_entries, double *out) {
+  if (q < 1 || M < 0 || n_entries < 0 || !s || !r || !keep) return ORACLE_BAD_ARG;
+  int64_t *so = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  int64_t *ro = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  prefix(q, s, so);
+  prefix(q, r, ro);
+  int rc = ORACLE_OK;
+  for (int64_t e = 0; e < n_entries; ++e) {
+    if (rows[e] < 0 || rows[e] >= M || cols[e] < 0 || cols[e] >= ro[q]) rc = ORACLE_BAD_ARG;
+    else if (types[rows[e]] < 0 || types[rows[e]] >= q) rc = ORACLE_BAD_TYPE;
+  }
+  if (rc == ORACLE_OK) {
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < n_entries; ++e) {
+      const int64_t b = rows[e], n = cols[e];
+      const int i = types[b];
+      int j = 0;
+      while (n >= ro[j + 1]) ++j;
+      double acc = bias ? bias[n] : 0.0;
+      for (int k = 0; k < q; ++k) {
+        if (!keep[((size_t)i * q + j) * q + k]) continue;
+        for (int64_t c = so[k]; c < so[k + 1]; ++c) acc += X[b * ldx + c] * W[c * ldw + n];
+      }
+      out[e] = acc;
+    }
+  }
+  free(so);
+  free(ro);
+  return rc;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * The same function evaluated type by type, as Algorithm 1 organises a batch: the rows of one
+ * type are collected first, then every kept (input group, output group) pair of that type
+ * contributes one rectangular product to those rows of Y (which starts from zero).
  * Written separately from star_proj_rows so the two can be tested against each other.
  * ------------------------------------------------------------------------------------- */
 int star_proj_alg1(const double *X, int64_t ldx, const int32_t *types, int64_t M,
@@ -238,6 +279,11 @@ int star_square(const double *A, const double *B, double *C, int q, const int32_
 
 /* Exact GELU, gelu(z) = z/2 (1 + erf(z / sqrt 2)). */
 double star_gelu(double z) { return 0.5 * z * (1.0 + erf(z * 0.70710678118654752440)); }
+/* The same, element by element over an array (in place). */
+void star_gelu_array(double *z, int64_t n) {
+#pragma omp parallel for schedule(static)
+  for (int64_t e = 0; e < n; ++e) z[e] = star_gelu(z[e]);
+}
 
 /* ---------------------------------------------------------------------------------------
  * Two-map FFN: H = gelu(X * W_up + b_up),  Y = H * W_down + b_down, same row types for both

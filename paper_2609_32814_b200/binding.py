@@ -22,6 +22,8 @@ ALG_TABLE_QQ, ALG_TABLE_DENSE, ALG_TABLE_CUSTOM, ALG_TABLE_Q2POW = 0, 1, 2, 3
 ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
 ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC = 0, 1
 ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
+OPTIONS = {"gemm_kernel": 1, "tile_n": 2, "small_m_kernel": 3, "host_plan": 4, "wait_limit_cycles": 5,
+           "test_stall_bytes": 6}
 
 _DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
 _TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM, "q2pow": ALG_TABLE_Q2POW}
@@ -30,7 +32,7 @@ _ACTS = {None: ALG_ACT_NONE, "none": ALG_ACT_NONE, "gelu": ALG_ACT_GELU_ERF, "ge
 _SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC}
 
 EXPORTS = [
-    "alg_proj_create", "alg_proj_destroy", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
+    "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
     "alg_proj_forward_static", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
     "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
@@ -57,6 +59,8 @@ def lib() -> ctypes.CDLL:
         vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
         L.alg_proj_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
         L.alg_proj_destroy.argtypes = [vp]
+        L.alg_proj_set_option.argtypes = [vp, i32, i64]
+        L.alg_ffn_set_option.argtypes = [vp, i32, i64]
         L.alg_proj_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
         L.alg_proj_forward.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp, ctypes.c_size_t, vp]
         L.alg_proj_forward_static.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp]
@@ -107,6 +111,7 @@ def launch_count() -> int:
 
 class _Handle:
     _destroy = None
+    _set_option = None
 
     def __init__(self):
         self._h = ctypes.c_void_p()
@@ -122,6 +127,10 @@ class _Handle:
             self.close()
         except Exception:
             pass
+
+    def set_option(self, name: str, value: int):
+        """alg_*_set_option: per-handle switches (see OPTIONS and the header)."""
+        _check(getattr(lib(), self._set_option)(self._h, OPTIONS[name], int(value)), self._set_option)
 
     def _workspace(self, nbytes: int, device) -> torch.Tensor:
         if self._ws is None or self._ws.numel() < nbytes or self._ws.device != device:
@@ -142,6 +151,7 @@ def _keep_arg(table, custom_keep, q):
 class Proj(_Handle):
     """alg_proj_* : Y = act(X *_q W + bias)."""
     _destroy = "alg_proj_destroy"
+    _set_option = "alg_proj_set_option"
 
     def __init__(self, in_widths, out_widths, dtype="bf16", table="qq", custom_keep=None, schedule="explicit"):
         super().__init__()
@@ -208,6 +218,7 @@ class Proj(_Handle):
 class FFN(_Handle):
     """alg_ffn_* : Y = act(X *_q W_up + b_up) *_q W_down + b_down."""
     _destroy = "alg_ffn_destroy"
+    _set_option = "alg_ffn_set_option"
 
     def __init__(self, d_widths, f_widths, dtype="bf16", table="qq", custom_keep=None, schedule="explicit"):
         super().__init__()

@@ -61,7 +61,6 @@ static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
 struct TileGeom {
   int tile_m;        // rows per tile (a power of two)
   int tile_m_log2;
-  int alternate;     // 1: a worker takes its tiles alternately from the expensive and the cheap end
 };
 
 struct BucketArgs {
@@ -125,40 +124,19 @@ struct ProjArgs {
   // original row = (bucketed row - i*M/q)*q + i.  0 = off.
   int a_cyclic_rows;
   int out_cyclic_rows;
-  int dbg;                // experiment switches, honoured only in -DALGPROJ_TRACE builds
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   int y_staged;           // 1: the epilogue transposes bf16 results through shared memory for coalesced stores
   // Cyclic schedule: the tile sequences of all workers depend only on (handle, M) and are planned
-  // once on the host; worker w reads plan[w * plan_stride .. + plan_rounds) (the last record of
-  // every worker is the end marker).  nullptr: every CTA plans for itself.
+  // once on the host; worker w reads plan[1 + w * plan_stride .. + plan_rounds) (the last record of
+  // every worker is the end marker).  plan[0] is a stamp {row0 = M, rows = plan_tag}: a kernel whose
+  // launch names another (M, tag) than the device copy holds plans for itself instead.
+  // nullptr: every CTA plans for itself.
   const TileRec *plan;
-  int plan_stride, plan_rounds;
-  long long *trace;       // debug timeline (nullptr = off)
-  int trace_cap;
+  int plan_stride, plan_rounds, plan_tag;
+  long long wait_limit;   // bound of every device-side wait, in SM clock cycles
 };
 
 cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
-
-// Fused two-projection FFN kernel (ffn_tc.cu).  Extension of a tile record: an up tile carries the
-// counter it reports to (`sig`, -1 for down tiles), a down tile the counter it waits for (`dep`).
-struct TileExt {
-  int dep;
-  int sig;
-};
-constexpr int kFfnSeqCap = 160;  // tile records per CTA
-struct FfnArgs {
-  ProjArgs p[2];                 // [0] up (X -> H, activation), [1] down (H -> Y); tables by value (q <= 8)
-  const TileRec *plan;           // [n_workers][plan_stride] records, the last of a worker is the end marker
-  const TileExt *ext;            // parallel to plan
-  int plan_stride, plan_rounds;
-  // one counter per (128-row block of H, hidden group): up tiles of that part finished so far;
-  // counters[n_counters] = CTAs that have left (the last one clears everything for the next launch)
-  unsigned long long *counters;
-  int n_counters;
-  int target[kParamQ];           // up tiles per (row block, hidden group g): the value the counter must reach
-                                 // before a down tile reads hidden group g of the block
-};
-cudaError_t launch_ffn_tc(const FfnArgs &a, int n_workers, cudaStream_t st);
 
 // tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
 // (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.
@@ -204,7 +182,8 @@ struct DecodeArgs {
   int w_smem_bytes;
   int x_smem_bytes;
   int *status;
-  long long *trace;       // debug timeline (nullptr = off)
+  long long wait_limit;   // bound of every device-side wait, in SM clock cycles
+  int extra_expect_bytes; // test aid: bytes added to the weight barrier's expectation that never arrive
   int q;
   int small_q;            // q <= kDecodeParamQ: the table below is valid
   int so[kDecodeParamQ + 1];
@@ -215,6 +194,9 @@ bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *pla
 cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st);
 
 void count_launch(int n = 1);
+int handle_device(alg_proj_t h);  // device the handle was created on (-1 for a null handle)
+
+constexpr long long kDefaultWaitLimit = 4000000000LL;  // ~2 s at B200 clocks
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

@@ -10,7 +10,9 @@
 // thread-block cluster.  A CTA fetches its slice of the bank (its share of the rows of every
 // needed input group, SN columns wide) with one or two TMA boxes per group -- issued before it
 // waits for the previous kernel in the stream (programmatic dependent launch), because weights do
-// not depend on it -- stages the matching columns of X with 16-byte asynchronous copies (rows
+// not depend on it.  Which groups are needed follows from the row types, which MAY come from that
+// previous kernel: they are read once before the wait to choose the boxes and once more after it;
+// if the second reading differs, the slice is fetched again for the types that count.  It then stages the matching columns of X with 16-byte asynchronous copies (rows
 // that do not use a block are staged as zeros, which is how the row-type rule is applied),
 // multiplies with warp-level mma.sync (bf16 x bf16 -> fp32), and pushes its partial sums into the
 // shared memory of the CTA that owns the output row (row m belongs to CTA m mod splits).  After
@@ -18,13 +20,13 @@
 // nothing goes through global memory), applies bias / activation and stores Y.
 #include <cuda_runtime.h>
 
-#include <cstdlib>
-
 #include "tc_common.cuh"
 
 namespace algproj {
 
 using namespace tc;
+
+ALG_TRACE_DEFINE(decode)
 
 namespace {
 
@@ -94,13 +96,7 @@ __device__ __forceinline__ uint32_t x_off(int m, int chunk, int x_pitch_bytes) {
   return (uint32_t)(m * x_pitch_bytes + ((chunk ^ (m & 7)) << 4));
 }
 
-#ifdef ALGPROJ_TRACE
-#define DTR() tr[trn++] = clock64()
-#else
-#define DTR() \
-  do {        \
-  } while (0)
-#endif
+#define DTR() ALG_TRACE(0, 0)
 
 template <int SN>
 __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant__ CUtensorMap tmW, const DecodeArgs a) {
@@ -120,10 +116,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   const int n0 = strip * SN;
   const int M = a.M;
   const int m_tiles = (M + 15) >> 4, m_pad = m_tiles << 4;
-#ifdef ALGPROJ_TRACE
-  long long tr[12];
-  int trn = 0;
-#endif
+  ALG_TRACE_VARS;
   DTR();
 
   // ---- row types, support of this strip (one global round trip, then shared memory only) ----
@@ -134,80 +127,116 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
     for (int e = tid; e <= q; e += kThreads) s_so[e] = tab->so[e], s_ro[e] = tab->ro[e];
     for (int e = tid; e < q * q; e += kThreads) s_keep[e] = tab->keep[e];
   }
-  int my_type = -1;
-  if (tid < M) {
-    my_type = a.types ? a.types[tid] : (tid % q);
-    if (my_type < 0 || my_type >= q) {
-      atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
-      my_type = -1;
-    }
-  }
   if (tid == 0) {
     mbar_init(smem_u32(&s_bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
   }
-  __syncthreads();
-  DTR();
   int j = 0;
-  while (j + 1 < q && s_ro[j + 1] <= n0) ++j;
-  if (tid < kDecodeMaxM) {  // warps 0 and 1: rows 0..63
-    const uint32_t kmask = my_type >= 0 ? s_keep[my_type * q + j] : 0u;  // input groups this row uses for group j
-    const unsigned badv = __ballot_sync(0xffffffffu, tid < M && my_type < 0);
-    if (lane == 0) s_bad32[warp] = badv;
-    for (int k = 0; k < q; ++k) {
-      const unsigned v = __ballot_sync(0xffffffffu, (kmask >> k) & 1u);
-      if (lane == 0) s_rows32[k][warp] = v;
-    }
-  }
-  __syncthreads();
-  if (warp == 0) {  // segment list: lane k owns input group k; prefix of the lengths by shuffles
-    uint32_t lo = 0, hi = 0;
-    int len = 0;
-    if (lane < q) {
-      lo = s_rows32[lane][0], hi = s_rows32[lane][1];
-      if (lo | hi) len = (s_so[lane + 1] - s_so[lane]) / splits;  // nobody needs W_kj -> it is never read
-    }
-    const unsigned have = __ballot_sync(0xffffffffu, len > 0);
-    int incl = len;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += n;
-    }
-    if (len > 0) {
-      const int s = __popc(have & ((1u << lane) - 1u));
-      s_seg[s].grow0 = s_so[lane] + split * len;
-      s_seg[s].len = len;
-      s_seg[s].loc0 = incl - len;
-      s_seg[s].rows_lo = lo, s_seg[s].rows_hi = hi;
-    }
-    if (lane == 31) s_nseg = __popc(have), s_rows = incl;
-  }
-  __syncthreads();
-  DTR();
-  const int nseg = s_nseg, rows_cta = s_rows;
-  const int x_pitch_bytes = ((rows_cta + 63) & ~63) * 2;  // whole groups of eight 16-byte chunks
+  const uint32_t bar = smem_u32(&s_bar);
   uint8_t *w_sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t *x_sm = w_sm + (size_t)a.w_smem_bytes;
   float *r_sm = (float *)(x_sm + (size_t)a.x_smem_bytes);   // [splits][rows owned][SN] partial sums of my rows
-
-  // ---- the weight slice: one TMA box per segment (more when a segment exceeds the box height) ----
-  if (tid == 0) {
-    const uint32_t bar = smem_u32(&s_bar);
-    mbar_expect_tx(bar, (uint32_t)(rows_cta * SN * 2));
-    for (int s = 0; s < nseg; ++s) {
-      const Seg sg = s_seg[s];
-      for (int r0 = 0; r0 < sg.len; r0 += a.box_rows)
-        tma_load_2d(smem_u32(w_sm) + (uint32_t)((sg.loc0 + r0) * SN * 2), &tmW, bar, n0, sg.grow0 + r0);
+  int my_type = -1;
+  // Reads the row types (L2, never a stale L1 line), derives the support of this strip and the
+  // segment list, and requests the weight slice: one TMA box per segment (more when a segment
+  // exceeds the box height).  Runs once before the wait for the previous kernel and, only if the
+  // types read after that wait differ, a second time.
+  auto plan_and_fetch = [&]() {
+    my_type = -1;
+    if (tid < M) {
+      my_type = a.types ? __ldcg(a.types + tid) : (tid % q);
+      if (my_type < 0 || my_type >= q) my_type = -1;
     }
-  }
+    __syncthreads();   // tables and barrier are ready (first pass); previous segment list is consumed (second pass)
+    j = 0;
+    while (j + 1 < q && s_ro[j + 1] <= n0) ++j;
+    if (tid < kDecodeMaxM) {  // warps 0 and 1: rows 0..63
+      const uint32_t kmask = my_type >= 0 ? s_keep[my_type * q + j] : 0u;  // input groups this row uses for group j
+      const unsigned badv = __ballot_sync(0xffffffffu, tid < M && my_type < 0);
+      if (lane == 0) s_bad32[warp] = badv;
+      for (int k = 0; k < q; ++k) {
+        const unsigned v = __ballot_sync(0xffffffffu, (kmask >> k) & 1u);
+        if (lane == 0) s_rows32[k][warp] = v;
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {  // segment list: lane k owns input group k; prefix of the lengths by shuffles
+      uint32_t lo = 0, hi = 0;
+      int len = 0;
+      if (lane < q) {
+        lo = s_rows32[lane][0], hi = s_rows32[lane][1];
+        if (lo | hi) len = (s_so[lane + 1] - s_so[lane]) / splits;  // nobody needs W_kj -> it is never read
+      }
+      const unsigned have = __ballot_sync(0xffffffffu, len > 0);
+      int incl = len;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += n;
+      }
+      if (len > 0) {
+        const int s = __popc(have & ((1u << lane) - 1u));
+        s_seg[s].grow0 = s_so[lane] + split * len;
+        s_seg[s].len = len;
+        s_seg[s].loc0 = incl - len;
+        s_seg[s].rows_lo = lo, s_seg[s].rows_hi = hi;
+      }
+      if (lane == 31) s_nseg = __popc(have), s_rows = incl;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      mbar_expect_tx(bar, (uint32_t)(s_rows * SN * 2 + a.extra_expect_bytes));
+      for (int s = 0; s < s_nseg; ++s) {
+        const Seg sg = s_seg[s];
+        for (int r0 = 0; r0 < sg.len; r0 += a.box_rows)
+          tma_load_2d(smem_u32(w_sm) + (uint32_t)((sg.loc0 + r0) * SN * 2), &tmW, bar, n0, sg.grow0 + r0);
+      }
+    }
+  };
+  // Bounded wait for the weight slice (parity = phase of the barrier).
+  auto wait_weights = [&](uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+      if (clock64() - t0 > a.wait_limit) {
+        atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+        while (clock64() - t0 < a.wait_limit + 2000000LL) {  // copies still in flight get time to land
+        }
+        return false;
+      }
+    }
+    return true;
+  };
+  plan_and_fetch();
   DTR();
   // The weights do not depend on the previous kernel in the stream, X does: let the next kernel
   // start its own weight stream now, and wait for the producer of X only here.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   DTR();
+  uint32_t w_parity = 0;
+  bool weights_ok = true;
+  {  // the row types as the previous kernel left them: the ones that count
+    int t_now = -1;
+    if (tid < M) {
+      t_now = a.types ? __ldcg(a.types + tid) : (tid % q);
+      if (t_now < 0 || t_now >= q) {
+        atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
+        t_now = -1;
+      }
+    }
+    if (__syncthreads_or(t_now != my_type)) {
+      // fetched for other types than the final ones: let those copies land, then fetch again
+      weights_ok = wait_weights(0);
+      __syncthreads();
+      if (weights_ok) {
+        plan_and_fetch();
+        w_parity = 1;
+      }
+    }
+  }
+  const int nseg = s_nseg, rows_cta = s_rows;
+  const int x_pitch_bytes = ((rows_cta + 63) & ~63) * 2;  // whole groups of eight 16-byte chunks
   // ---- the matching columns of X; rows that do not use a block are staged as zeros ----
   {
     const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
@@ -227,16 +256,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   }
   DTR();
   cp_async_wait_all();
-  {  // bounded wait for the weight slice
-    const uint32_t bar = smem_u32(&s_bar);
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, 0)) {
-      if (clock64() - t0 > kTimeoutCycles) {
-        atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
-        break;
-      }
-    }
-  }
+  if (weights_ok) wait_weights(w_parity);   // on expiry: status raised, the result is invalid, the kernel still ends
   __syncthreads();
   DTR();
 
@@ -331,10 +351,6 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
     }
   }
   DTR();
-#ifdef ALGPROJ_TRACE
-  if (a.trace && tid == 0 && blockIdx.x == 3 && blockIdx.y == 0)
-    for (int e = 0; e < trn; ++e) a.trace[e] = tr[e];
-#endif
 }
 
 template <int SN>
@@ -364,7 +380,7 @@ cudaError_t launch_t(const DecodeArgs &a, size_t smem_bytes, cudaStream_t st) {
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 1 : 2;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, decode_kernel<SN>, tmW, a);
 }
 

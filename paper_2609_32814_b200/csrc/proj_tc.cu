@@ -5,8 +5,8 @@
 // One output tile = 128 rows of one row type i  x  TILE_N columns of one output group j.  All
 // kept products of that block (x_k W_kj for k in B(i,j); Eq. recursive-row-action -- for the
 // Q_q law x_i W_ij + x_j W_jj, Eqs. typed-diag/off) are issued back to back into the SAME
-// TMEM accumulator, so no partial sum ever reaches HBM ("one forward kernel accumulates both
-// endpoint products before writing the output", Section "Kernels").
+// TMEM accumulator, so no partial sum ever reaches HBM (the fused forward kernel of Section
+// "Kernels": every endpoint product of an output block is summed before the block is written).
 //
 // Operands: A = type-bucketed rows, K-contiguous (K-major), 128B-swizzled 128x64 tiles.
 //           B = the canonical K x N bank, N-contiguous (MN-major), 64(k) x 64(n) swizzled boxes.
@@ -21,7 +21,6 @@
 // handle's status word, all roles leave their loops, TMEM is released and the kernel returns.
 #include <cudaTypedefs.h>
 
-#include <cstdlib>
 #include <cstring>
 
 #include "tc_common.cuh"
@@ -29,6 +28,8 @@
 namespace algproj {
 
 using namespace tc;
+
+ALG_TRACE_DEFINE(proj_tc)
 
 namespace {
 
@@ -39,6 +40,7 @@ struct Ctl {
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;     // bound of every wait, in clock64 cycles
   // interaction table, copied once per CTA so no role waits on global metadata at a tile start
   int so[kMaxQ + 1];
   uint32_t keep[kMaxPairs];
@@ -52,7 +54,7 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, 
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0) {
       if (ctl->abort_flag) return false;
-      if (clock64() - t0 > kTimeoutCycles) {
+      if (clock64() - t0 > ctl->wait_limit) {
         ctl->abort_flag = 1;
         atomicExch(status, (int)ALG_ERR_DEVICE_TIMEOUT);
         return false;
@@ -104,15 +106,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DevTable *__restrict__ tab = a.tab;
   const int q = a.q;
-  [[maybe_unused]] int tr_n = 0;
-#ifdef ALGPROJ_TRACE
-  if (a.trace && threadIdx.x == 0) {  // whole-CTA window: global timer and SM clock at entry
-    unsigned long long gt;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 0] = (long long)gt;
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 2] = clock64();
-  }
-#endif
+  ALG_TRACE_VARS;
+  ALG_TRACE_CTA(0);
 
   if (threadIdx.x == 0) ALG_TRACE(0, 20);
   if (warp == 0) {  // one barrier per lane
@@ -124,6 +119,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&ctl->tmem_empty[lane - C::kStages]), kEpiWarps);
     } else if (lane == 31) {
       ctl->abort_flag = 0;
+      ctl->wait_limit = a.wait_limit;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   } else if (warp == 3) {
@@ -158,8 +154,15 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (warp == 2) {
     // one warp plans this CTA's work while the others set up barriers and tensor memory
-    if (a.plan) {  // cyclic schedule: planned on the host, once per (handle, M)
-      for (int r = lane; r < a.plan_rounds; r += 32) recs[r] = a.plan[(size_t)blockIdx.x * a.plan_stride + r];
+    // cyclic schedule: planned on the host, once per (handle, M); the stamp in front of the records
+    // tells whether the device copy still is the plan this launch was given
+    bool planned = false;
+    if (a.plan) {
+      const TileRec stamp = a.plan[0];
+      planned = stamp.row0 == a.M && stamp.rows == a.plan_tag;
+    }
+    if (planned) {
+      for (int r = lane; r < a.plan_rounds; r += 32) recs[r] = a.plan[1 + (size_t)blockIdx.x * a.plan_stride + r];
       if (lane == 0) tm->seq_rounds = a.plan_rounds, tm->seq_valid = a.plan_rounds, tm->total = 0;
     } else {
       if (a.offsets) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
@@ -212,20 +215,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t bar = full0 + 8u * (uint32_t)stage;
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
           if (elect_one()) {
-#ifdef ALGPROJ_TRACE
-            if (a.dbg & 24) {  // timing experiments: 8 = no A loads, 16 = no B loads (results are wrong)
-              if (loads_a) {
-                const uint32_t bytes = ((a.dbg & 8) ? 0u : (uint32_t)C::kABytes) + ((a.dbg & 16) ? 0u : (uint32_t)C::kBBytes);
-                if (bytes) mbar_expect_tx(bar, bytes); else mbar_arrive(bar);
-                if (!(a.dbg & 8)) {
-                  if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
-                  else tma_load_2d(sa, &tmA, bar, k0, a_row);
-                }
-              } else if (!(a.dbg & 16)) {
-                tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
-              }
-            } else
-#endif
             if (loads_a) {
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
@@ -311,6 +300,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         } else {
           out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
         }
+        if (out_row >= a.M) out_row = -1;   // never store outside Y, whatever the tile record says
       }
       bool ok = wait_bar(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -364,9 +354,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
                          : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
                          : "r"(rd_base + (uint32_t)g * 512u + ((((uint32_t)piece) ^ rsw) << 4)));
-#ifdef ALGPROJ_TRACE
-            if ((a.dbg & 1) && val.x != 0x12345678u) continue;   // timing experiment: no global stores
-#endif
             if (dst_row[g] >= 0)
               *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col_base + c0 + piece * 8) = val;
           }
@@ -405,14 +392,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
-#ifdef ALGPROJ_TRACE
-  if (a.trace && threadIdx.x == 0) {
-    unsigned long long gt;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 1] = (long long)gt;
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 3] = clock64();
-  }
-#endif
+  ALG_TRACE_CTA(1);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
@@ -444,7 +424,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   }
   // staging buffers for the transposing epilogue, when they fit and the output rows are 16-byte aligned
   b.y_staged = a.y_bf16 && smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && ((uintptr_t)a.Y & 15u) == 0 &&
-               (a.ldy * 2) % 16 == 0 && !std::getenv("ALGPROJ_NO_STAGED_STORE");
+               (a.ldy * 2) % 16 == 0;
   if (b.y_staged) smem_bytes += kEpiWarps * C::kStoreBufBytes;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(num_sms, 1, 1);
@@ -455,7 +435,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
+  cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, b);
   count_launch(1);
   return e;
@@ -498,7 +478,7 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
 // 64 x 64 x chunks lands in shared memory chunk-major ([chunk][k][64 n]), which is exactly the
 // MN-major 128-byte-swizzled operand layout, with a single copy instruction per stage.
 cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
-  if (a.N % 64 || std::getenv("ALGPROJ_B2D")) return cudaErrorInvalidValue;
+  if (a.N % 64) return cudaErrorInvalidValue;
   cuuint64_t dims[3] = {64, (cuuint64_t)a.K, (cuuint64_t)(a.N / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldw * 2, 128};
   cuuint32_t box[3] = {64, kTcBlockK, (cuuint32_t)chunks};

@@ -26,6 +26,8 @@ namespace algproj {
 
 using namespace tc;
 
+ALG_TRACE_DEFINE(proj_tc2)
+
 namespace {
 
 constexpr int kEpiWarps = 8;
@@ -48,6 +50,7 @@ struct Ctl2 {
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;     // bound of every wait, in clock64 cycles
   int so[kMaxQ + 1];
   uint32_t keep[1];  // q*q entries follow, then q*q uint16 K-block counts (the request is sized for them)
 };
@@ -114,7 +117,7 @@ __device__ __noinline__ bool wait_slow2(uint32_t bar, uint32_t parity, Ctl2 *ctl
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0) {
       if (ctl->abort_flag) return false;
-      if (clock64() - t0 > kTimeoutCycles) {
+      if (clock64() - t0 > ctl->wait_limit) {
         ctl->abort_flag = 1;
         atomicExch(status, (int)ALG_ERR_DEVICE_TIMEOUT);
         return false;
@@ -142,15 +145,8 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const DevTable *__restrict__ tab = a.tab;
   const int q = tab_q;
   const uint32_t rank = cluster_ctarank();          // 0 = leader
-  [[maybe_unused]] int tr_n = 0;
-#ifdef ALGPROJ_TRACE
-  if (a.trace && threadIdx.x == 0) {  // whole-CTA window: global timer and SM clock at entry
-    unsigned long long gt;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 0] = (long long)gt;
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 2] = clock64();
-  }
-#endif
+  ALG_TRACE_VARS;
+  ALG_TRACE_CTA(0);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -162,6 +158,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * kEpiWarps);
     }
     ctl->abort_flag = 0;
+    ctl->wait_limit = a.wait_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
@@ -315,6 +312,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         } else {
           out_row = a.perm ? __ldg(a.perm + rec.row0 + r) : (rec.row0 + r);
         }
+        if (out_row >= a.M) out_row = -1;   // never store outside Y, whatever the tile record says
       }
       bool ok = wait_bar2(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -358,14 +356,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // neither CTA leaves while its peer may still signal or read its shared memory
-#ifdef ALGPROJ_TRACE
-  if (a.trace && threadIdx.x == 0) {
-    unsigned long long gt;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 1] = (long long)gt;
-    a.trace[(size_t)24 * a.trace_cap + blockIdx.x * 4 + 3] = clock64();
-  }
-#endif
+  ALG_TRACE_CTA(1);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
@@ -413,7 +404,7 @@ cudaError_t launch_proj_tc2(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = std::getenv("ALGPROJ_NO_PDL") ? 0 : 1;
+  cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, proj_tc2_kernel, tmA, tmB, a, n_stages);
   count_launch(1);
   return e;

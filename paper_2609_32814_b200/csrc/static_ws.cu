@@ -17,9 +17,12 @@ void *g_scratch_addr[kMaxDevices] = {nullptr};
 
 // The array's name is only a host-side stand-in; kernels need its device address, which is
 // looked up once per device with that device current.
-alg_status_t scratch_address(void **out) {
+// `handle_dev`: the device the handle's tables live on; the array of any other device is useless
+// to it, so a call with another device current is refused.
+alg_status_t scratch_address(int handle_dev, void **out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ALG_ERR_CUDA;
+  if (dev != handle_dev) return ALG_ERR_INVALID_ARG;
   if (dev < 0 || dev >= kMaxDevices) return ALG_ERR_UNSUPPORTED_SHAPE;
   if (!g_scratch_addr[dev]) {
     void *p = nullptr;
@@ -42,7 +45,7 @@ extern "C" alg_status_t alg_proj_forward_static(alg_proj_t h, const void *X, int
   if (s != ALG_OK) return s;
   if (need > kStaticScratchBytes) return ALG_ERR_WORKSPACE_TOO_SMALL;  // problem exceeds the built-in scratch
   void *scratch = nullptr;
-  s = scratch_address(&scratch);
+  s = scratch_address(algproj::handle_device(h), &scratch);
   if (s != ALG_OK) return s;
   return alg_proj_forward(h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, scratch, kStaticScratchBytes,
                           stream);

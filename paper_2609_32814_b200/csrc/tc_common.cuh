@@ -4,11 +4,10 @@
 #include <cuda.h>
 
 #include "tile_map.cuh"
+#include "trace.cuh"
 
 namespace algproj {
 namespace tc {
-
-constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s at B200 clocks
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -153,11 +152,7 @@ __device__ __forceinline__ void finish_32(float (&f)[32], const ProjArgs &a, int
 #pragma unroll
     for (int x = 0; x < 32; ++x) f[x] += __bfloat162float(__ldg(b + x));
   }
-#ifdef ALGPROJ_TRACE
-  if (a.act == ALG_ACT_GELU_ERF && !(a.dbg & 2)) {
-#else
   if (a.act == ALG_ACT_GELU_ERF) {
-#endif
 #pragma unroll
     for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
   } else if (a.act == ALG_ACT_GELU_TANH) {
@@ -176,16 +171,7 @@ __device__ __forceinline__ void pack_bf16_32(const float (&f)[32], uint32_t (&w)
 // Converts one row segment of 32 fp32 accumulator values (bias / activation applied) and stores
 // it: 64 bytes of bf16 or 128 bytes of fp32, as 32-byte stores when the address allows.
 __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjArgs &a, int64_t out_row, int col) {
-#ifdef ALGPROJ_TRACE
-  if (a.dbg & 4) return;
-#endif
   finish_32(f, a, col);
-#ifdef ALGPROJ_TRACE
-  if (a.dbg & 1) {
-    if (f[0] == 123.456f) ((float *)a.Y)[0] = f[1];
-    return;
-  }
-#endif
   if (a.y_bf16) {
     uint32_t w[16];
     pack_bf16_32(f, w);
@@ -218,18 +204,6 @@ __device__ __forceinline__ void finish_and_store_32(float (&f)[32], const ProjAr
     }
   }
 }
-
-#ifdef ALGPROJ_TRACE
-#define ALG_TRACE(role, tag)                                                                        \
-  do {                                                                                              \
-    if (a.trace && blockIdx.x < 8 && tr_n < a.trace_cap)                                            \
-      a.trace[((size_t)blockIdx.x * 3 + (role)) * a.trace_cap + tr_n++] = (clock64() << 8) | (tag); \
-  } while (0)
-#else
-#define ALG_TRACE(role, tag) \
-  do {                       \
-  } while (0)
-#endif
 
 // Host side: tensor-map encoding through the driver entry point (no link-time libcuda dependency).
 cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,

@@ -109,12 +109,6 @@ __device__ __forceinline__ int snake_index(int round, int worker, int n_workers)
 }
 // `nkb_of_pair` (optional, shared memory): number of K blocks of the tiles of a pair; it is packed
 // into the upper half of TileRec::rows so that the MMA thread needs nothing but the record.
-// Processing order of a worker's own tiles: its share of the cost-sorted enumeration is taken
-// alternately from the expensive and from the cheap end (1st, last, 2nd, last but one, ...).  A
-// tile's epilogue costs the same whatever its K length, so a run of short-K tiles is bound by
-// the epilogue while a run of long-K tiles leaves the epilogue warps idle; alternating lets the
-// epilogue of one kind overlap the main loop of the other.  All workers apply the same
-// permutation to the round index, so the workers of a round still sit on neighbouring tiles.
 __device__ __forceinline__ TileRec tile_seq_decode(TileMap *tm, const TileGeom &g, int pos, int worker, int n_workers,
                                                    const uint16_t *nkb_of_pair) {
   const int n = tm->seq_valid;
@@ -123,8 +117,7 @@ __device__ __forceinline__ TileRec tile_seq_decode(TileMap *tm, const TileGeom &
     rec.row0 = -1, rec.rows = 0, rec.pair = 0, rec.n0 = 0;
     return rec;
   }
-  const int round = !g.alternate ? pos : (pos & 1) ? n - 1 - (pos >> 1) : (pos >> 1);
-  rec = tile_map_decode(tm, g, snake_index(round, worker, n_workers));
+  rec = tile_map_decode(tm, g, snake_index(pos, worker, n_workers));
   if (nkb_of_pair && rec.row0 >= 0) rec.rows |= (int)nkb_of_pair[rec.pair & 0xFFFF] << 16;
   return rec;
 }

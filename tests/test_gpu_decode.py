@@ -21,6 +21,7 @@ def _wl(q, M, s_w, r_w, types=None, integer=True, seed=1):
     (2, 1, 384, 1536), (2, 8, 384, 1536), (2, 33, 384, 1536), (2, 64, 384, 1536),   # up projection of config 4
     (2, 1, 1536, 384), (2, 17, 1536, 384), (2, 64, 1536, 384),                      # down projection of config 4
     (4, 5, 128, 512), (3, 64, 192, 128), (1, 16, 256, 256), (8, 40, 128, 128),
+    (16, 40, 64, 128), (12, 9, 48, 64),   # more groups than the by-value table holds: table read from device memory
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_decode_integer_bit_exact(q, M, s_w, r_w, out_dtype):
@@ -94,3 +95,44 @@ def test_decode_tables_cyclic_bad_type_and_determinism():
     good = np.ones(M, bool)
     good[3] = False
     assert np.array_equal(got[good], oracle.proj(wl.X[good], types[good], wl.W_up, wl.d_widths, wl.f_widths))
+
+
+def test_types_written_by_the_kernel_just_before():
+    """The row types may be produced on the device right before the call (position mod q)."""
+    q, M, s_w, r_w = 2, 24, 384, 1536
+    wl = _wl(q, M, s_w, r_w, seed=31)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    pos = torch.from_numpy(np.arange(100, 100 + M, dtype=np.int32) * 3).cuda()
+    buf = torch.zeros(M, dtype=torch.int32, device="cuda")
+    out = torch.empty((M, wl.F), dtype=torch.float32, device="cuda")
+    for rep in range(3):
+        buf.zero_()                               # stale contents the early read may see
+        torch.remainder(pos + rep, q, out=buf)    # the types of this step, written just before the call
+        proj.forward(X, buf, W, out=out)
+        t = ((np.arange(100, 100 + M) * 3 + rep) % q).astype(np.int32)
+        assert np.array_equal(H.to_np(out), oracle.proj(wl.X, t, wl.W_up, wl.d_widths, wl.f_widths)), rep
+    assert proj.last_status() == 0
+
+
+def test_bounded_wait_expires_and_the_handle_recovers():
+    """A device-side wait that cannot complete must end by itself: the status word reports
+    ALG_ERR_DEVICE_TIMEOUT, the call returns, and the same handle computes exactly again
+    afterwards.  The stall is made without any fault: the kernel is told to expect 1 KiB more on
+    its weight barrier than its copies deliver (every issued copy still lands), with the wait
+    limit lowered to a few milliseconds."""
+    q, M, s_w, r_w = 2, 8, 384, 1536
+    wl = _wl(q, M, s_w, r_w, seed=41)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    X, t, W = H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16")
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    assert np.array_equal(H.to_np(proj.forward(X, t, W, out_dtype=torch.float32)), ref)
+    proj.set_option("wait_limit_cycles", 8_000_000)      # about 4 ms
+    proj.set_option("test_stall_bytes", 1024)
+    proj.forward(X, t, W, out_dtype=torch.float32)
+    assert proj.last_status() == 6                        # ALG_ERR_DEVICE_TIMEOUT, and the call came back
+    assert proj.last_status() == 0                        # reading cleared it
+    proj.set_option("test_stall_bytes", 0)
+    proj.set_option("wait_limit_cycles", 4_000_000_000)
+    assert np.array_equal(H.to_np(proj.forward(X, t, W, out_dtype=torch.float32)), ref)
+    assert proj.last_status() == 0

@@ -95,6 +95,9 @@ def test_cfg3_full_size_sampled_rows(q):
     rows = _sample_rows(wl, 192, seed=q)
     ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
     H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, False, f"cfg3 q={q}")
+    if q == 4:   # the same launch with bf16 output: final rounding adds half an ulp to the bound
+        Yb = _run_ffn(wl, ffn, torch.bfloat16)
+        H.assert_bf16_close(H.to_np(Yb[torch.from_numpy(rows).cuda()]), ref, True, f"cfg3 q={q} bf16 out")
     # the square d -> d projection of the same configuration
     proj = binding.Proj(wl.d_widths, wl.d_widths, dtype="bf16")
     Wsq = synth.bf16_round(synth.normal(synth.seed_for(3, q) + 9, (wl.D, wl.D), 0.02))
@@ -120,10 +123,25 @@ def test_cfg5_full_size_sampled_rows(q):
     wl = synth.config5(q)
     ffn = _ffn(wl)
     Y = _run_ffn(wl, ffn, torch.float32)
-    rows = _sample_rows(wl, 64 if q <= 4 else 16, seed=q)
+    rows = _sample_rows(wl, 64, seed=q)
+    assert all((wl.types[rows] == t).sum() >= 64 for t in range(q))
     ref = oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
     H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, False, f"cfg5 q={q}")
-    del Y
+    # plus 4096 single outputs at random (row, column) positions of the whole result
+    rng = np.random.default_rng(500 + q)
+    er, ec = rng.integers(0, wl.M, size=4096), rng.integers(0, wl.D, size=4096)
+    want = oracle.ffn_entries(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, er, ec)
+    got = Y[torch.from_numpy(er).cuda(), torch.from_numpy(ec).cuda()].double().cpu().numpy()
+    H.assert_bf16_close(got, want, False, f"cfg5 q={q} single entries")
+    if q == 8:   # the same launch with bf16 output
+        del Y
+        Yb = _run_ffn(wl, ffn, torch.bfloat16)
+        H.assert_bf16_close(H.to_np(Yb[torch.from_numpy(rows).cuda()]), ref, True, f"cfg5 q={q} bf16 out")
+        got = Yb[torch.from_numpy(er).cuda(), torch.from_numpy(ec).cuda()].double().cpu().numpy()
+        H.assert_bf16_close(got, want, True, f"cfg5 q={q} single entries, bf16 out")
+        del Yb
+    else:
+        del Y
     torch.cuda.empty_cache()
 
 
@@ -213,44 +231,36 @@ def test_cyclic_plan_follows_M_and_stream_capture():
     assert torch.equal(cyc.forward(X, None, W, act="gelu"), want)   # planned on the host now
 
 
-@pytest.mark.parametrize("q,M,D,F", [(2, 8192, 768, 3072), (2, 848, 256, 512), (4, 2056, 512, 1024)])
-def test_one_kernel_ffn_matches_two_kernel_ffn(q, M, D, F, monkeypatch):
-    """Cyclic schedule, opt-in (ALGPROJ_FUSED=1 at handle creation): the FFN runs as one persistent
-    kernel whose down tiles wait for the row blocks of H they read.  Same tiles, same K order, so the result must equal the two-kernel path
-    bit for bit (bf16 and fp32 outputs, with biases), also when replayed from a CUDA graph (the
-    kernel clears its own dependency counters), and must pass the oracle tolerance."""
-    wl = synth.make_workload("fused", config=8, variant=q * 100000 + M, dtype="bf16", q=q, M=M, D=D, F=F,
-                             types=synth.cyclic_types(M, q))
-    bu, bd = synth.normal(41, (wl.F,), 0.1), synth.normal(42, (wl.D,), 0.1)
-    monkeypatch.delenv("ALGPROJ_FUSED", raising=False)
-    two = _ffn(wl, schedule="cyclic")
-    Y2 = _run_ffn(wl, two, torch.float32, b_up=bu, b_down=bd, types=False)
-    Y2b = _run_ffn(wl, two, torch.bfloat16, b_up=bu, b_down=bd, types=False)
-    monkeypatch.setenv("ALGPROJ_FUSED", "1")      # read when the handle is created
-    one = _ffn(wl, schedule="cyclic")
-    launches = binding.launch_count()
-    Y1 = _run_ffn(wl, one, torch.float32, b_up=bu, b_down=bd, types=False)
-    assert binding.launch_count() - launches == 1          # one kernel
-    Y1b = _run_ffn(wl, one, torch.bfloat16, b_up=bu, b_down=bd, types=False)
-    assert torch.equal(Y1, Y2) and torch.equal(Y1b, Y2b)
-    ref = oracle.ffn(wl.X, wl.types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, b_up=bu, b_down=bd)
-    H.assert_bf16_close(H.to_np(Y1), ref, False, f"one-kernel FFN q={q} M={M}")
-    # graph replay: the same launch twice
-    X = H.to_dev(wl.X, "bf16")
-    Wu, Wd = H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16")
-    bud, bdd = H.to_dev(bu, "bf16"), H.to_dev(bd, "bf16")
-    Y = torch.empty_like(Y1)
-    ws = torch.empty(one.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+def test_captured_graph_survives_later_calls_with_other_M():
+    """A graph captured for M1 must not depend on the handle's plan cache: after eager calls with
+    five other M (more than the cache holds) its replay still writes exactly the M1 result and
+    nothing outside Y (canary rows behind it stay untouched)."""
+    q = 2
+    cyc = binding.Proj([128] * q, [256] * q, dtype="bf16", schedule="cyclic")
+    exp = binding.Proj([128] * q, [256] * q, dtype="bf16")
+    W = H.to_dev(synth.normal(33, (128 * q, 256 * q), 0.05), "bf16")
+    M1 = 1024
+    X1 = H.to_dev(synth.normal(34, (M1, 128 * q), 1.0), "bf16")
+    want = exp.forward(X1, H.dev_types(synth.cyclic_types(M1, q)), W, act="gelu")
+    assert torch.equal(cyc.forward(X1, None, W, act="gelu"), want)       # M1 is in the cache now
+    buf = torch.full((M1 + 64, 256 * q), 7.0, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(cyc.workspace_bytes(M1), dtype=torch.uint8, device="cuda")
     stream = torch.cuda.Stream()
     g = torch.cuda.CUDAGraph()
+    stream.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(stream):
         with torch.cuda.graph(g, stream=stream):
-            one.forward(X, None, Wu, Wd, b_up=bud, b_down=bdd, act="gelu", out=Y, workspace=ws, stream=stream)
-    for _ in range(3):
-        Y.zero_()
-        g.replay()
-        torch.cuda.synchronize()
-        assert torch.equal(Y, Y1) and one.last_status() == 0
+            cyc.forward(X1, None, W, act="gelu", out=buf[:M1], workspace=ws, stream=stream)
+    torch.cuda.current_stream().wait_stream(stream)
+    for k, M2 in enumerate((2560, 512, 768, 3072, 1280)):
+        X2 = H.to_dev(synth.normal(40 + k, (M2, 128 * q), 1.0), "bf16")
+        w2 = exp.forward(X2, H.dev_types(synth.cyclic_types(M2, q)), W, act="gelu")
+        assert torch.equal(cyc.forward(X2, None, W, act="gelu"), w2), M2
+    buf.fill_(7.0)
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(buf[:M1], want) and torch.all(buf[M1:] == 7.0)
+    assert cyc.last_status() == 0
 
 
 def test_pilot_tensor_square_law_and_interval_schedule():

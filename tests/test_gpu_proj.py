@@ -101,6 +101,102 @@ def test_tc_integer_bit_exact(q, M, s_w, r_w, out_dtype):
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
 
 
+# ---- CTA-pair kernel (tcgen05 cta_group::2), selected through a handle option --------------------
+
+@pytest.mark.parametrize("q,M,s_w,r_w,schedule", [
+    (1, 700, 512, 384, "explicit"),    # 256-wide tile plus the 128-wide remainder tile, ragged last 256-row tile
+    (2, 300, 128, 256, "explicit"),    # short K loops, one full tile per group
+    (2, 1337, 256, 384, "explicit"),   # several m-tiles per type, remainder tiles, both endpoint products
+    (3, 515, 64, 128, "explicit"),     # only 128-wide tiles, single K block per group
+    (2, 1026, 128, 384, "cyclic"),     # type-strided A view, arithmetic row scatter
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_pair_kernel_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else None
+    wl = _tc_workload(q, M, s_w, r_w, types=types, seed=q * 31 + M % 11)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    proj.set_option("gemm_kernel", 2)
+    launches = binding.launch_count()
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), None if schedule == "cyclic" else H.dev_types(wl.types),
+                     H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype)
+    assert proj.last_status() == 0
+    assert binding.launch_count() - launches == (1 if schedule == "cyclic" else 3)   # bucketing, gather, GEMM
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+    # the one-CTA kernel on the same handle gives the same bits
+    proj.set_option("gemm_kernel", 1)
+    Y1 = proj.forward(H.to_dev(wl.X, "bf16"), None if schedule == "cyclic" else H.dev_types(wl.types),
+                      H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype)
+    assert torch.equal(Y, Y1)
+
+
+def test_pair_kernel_bias_gelu_normal_data_and_refusal():
+    wl = _tc_workload(2, 900, 384, 384, integer=False, seed=13)
+    bias = synth.bf16_round(synth.normal(15, (wl.F,), 0.5))
+    for act, out_dtype in (("gelu", torch.float32), ("gelu", torch.bfloat16), (None, torch.bfloat16)):
+        proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+        proj.set_option("gemm_kernel", 2)
+        Y = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16"),
+                         bias=H.to_dev(bias, "bf16"), act=act, out_dtype=out_dtype)
+        assert proj.last_status() == 0
+        ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, bias=bias)
+        if act:
+            ref = oracle.gelu_array(ref)
+        H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"pair kernel act={act}")
+    # a shape the pair kernel cannot tile (192-wide groups) refuses the option and keeps working
+    odd = binding.Proj([64, 64], [192, 192], dtype="bf16")
+    with pytest.raises(binding.AlgError) as e:
+        odd.set_option("gemm_kernel", 2)
+    assert e.value.code == 2
+    with pytest.raises(binding.AlgError):
+        odd.set_option("tile_n", 256)
+    wl2 = _tc_workload(2, 260, 64, 192, seed=17)
+    Y = odd.forward(H.to_dev(wl2.X, "bf16"), H.dev_types(wl2.types), H.to_dev(wl2.W_up, "bf16"), out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl2.X, wl2.types, wl2.W_up, wl2.d_widths, wl2.f_widths))
+
+
+def test_bucketing_beyond_65536_rows():
+    """More rows than the one-kernel bucketing covers: the per-chunk histogram + scatter pair of
+    kernels builds the permutation (ragged everything: M is odd, the types are i.i.d.)."""
+    wl = _tc_workload(4, 70001, 64, 128, seed=23)
+    Y, proj = _run_proj(wl, out_dtype=torch.float32, expect_path=binding.ALG_PATH_TCGEN05)
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+    types = wl.types.copy()
+    types[[5, 66000, 70000]] = [4, -3, 99]           # out-of-range types in the first and the last chunk
+    Yb = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(types), H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert proj.last_status() == 5
+    got = H.to_np(Yb)
+    assert not got[[5, 66000, 70000]].any()
+    good = np.ones(wl.M, bool)
+    good[[5, 66000, 70000]] = False
+    assert np.array_equal(got[good], ref[good])
+
+
+def test_options_tile_width_and_in_kernel_plan():
+    """Every tile width that divides the groups, and both ways of planning the cyclic schedule,
+    give the same bits."""
+    M, q = 1024, 2
+    wl = _tc_workload(q, M, 128, 768, types=synth.cyclic_types(M, q), seed=29)
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
+    for tile_n in (0, 128, 192, 256):
+        proj.set_option("tile_n", tile_n)
+        for host_plan in (1, 0):
+            proj.set_option("host_plan", host_plan)
+            Y = proj.forward(X, None, W, out_dtype=torch.float32)
+            assert np.array_equal(H.to_np(Y), ref), (tile_n, host_plan)
+    proj.set_option("small_m_kernel", 0)
+    assert proj.kernel_path(8) == binding.ALG_PATH_TCGEN05
+    Y8 = proj.forward(X[:8], None, W, out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y8), ref[:8])
+
+
 def test_tc_missing_type_and_single_row():
     wl = _tc_workload(2, 1, 128, 128, types=np.array([1], dtype=np.int32))
     Y, _ = _run_proj(wl, out_dtype=torch.float32)

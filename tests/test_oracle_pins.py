@@ -139,6 +139,61 @@ def test_dense_minus_removed(q):
         assert np.array_equal(oracle.proj(X, types, W, s, r, form=form), want)
 
 
+@pytest.mark.parametrize("q", [2, 3, 4])
+def test_single_entries_against_dense_minus_removed(q):
+    """proj_entries sums one output at a time; pinned by the same independent numpy statement
+    (dense product minus the removed block products), with a bias, on every (row, column)."""
+    rng = np.random.default_rng(40 + q)
+    s = rng.integers(1, 4, size=q)
+    r = rng.integers(1, 4, size=q)
+    so, ro = _offsets(s), _offsets(r)
+    M = 7
+    X = _rand_ints(rng, (M, s.sum()))
+    W = _rand_ints(rng, (s.sum(), r.sum()))
+    bias = _rand_ints(rng, (r.sum(),))
+    types = rng.integers(0, q, size=M)
+    want = X @ W + bias
+    for b in range(M):
+        for j in range(q):
+            for k in range(q):
+                if k not in (types[b], j):
+                    want[b, ro[j]:ro[j + 1]] -= X[b, so[k]:so[k + 1]] @ W[so[k]:so[k + 1], ro[j]:ro[j + 1]]
+    rows, cols = np.meshgrid(np.arange(M), np.arange(r.sum()), indexing="ij")
+    got = oracle.proj_entries(X, types, W, s, r, rows.ravel(), cols.ravel(), bias=bias)
+    assert np.array_equal(got.reshape(M, -1), want)
+    with pytest.raises(oracle.OracleError):
+        oracle.proj_entries(X, types, W, s, r, [M], [0])
+
+
+def test_ffn_entries_and_gelu_array():
+    """ffn_entries against an independent numpy composition (q = 2, dense minus the removed product)."""
+    import math
+    rng = np.random.default_rng(61)
+    q, dw, fw = 2, [3, 2], [4, 5]
+    M = 9
+    X = rng.standard_normal((M, 5))
+    Wu = rng.standard_normal((5, 9))
+    Wd = rng.standard_normal((9, 5))
+    bu, bd = rng.standard_normal(9), rng.standard_normal(5)
+    types = rng.integers(0, q, size=M)
+    z = np.linspace(-5, 5, 23)
+    np.testing.assert_allclose(oracle.gelu_array(z), [0.5 * v * math.erfc(-v / math.sqrt(2)) for v in z], atol=1e-14)
+
+    def star2(Xm, Wm, s, r, bias):
+        so, ro = _offsets(s), _offsets(r)
+        out = Xm @ Wm + bias
+        for b, t in enumerate(types):
+            o = 1 - t
+            out[b, ro[t]:ro[t + 1]] -= Xm[b, so[o]:so[o + 1]] @ Wm[so[o]:so[o + 1], ro[t]:ro[t + 1]]
+        return out
+    Hn = np.vectorize(lambda v: 0.5 * v * (1 + math.erf(v / math.sqrt(2))))(star2(X, Wu, dw, fw, bu))
+    want = star2(Hn, Wd, fw, dw, bd)
+    rows = np.array([0, 8, 3, 3, 5, 8])
+    cols = np.array([0, 4, 2, 3, 1, 0])
+    got = oracle.ffn_entries(X, types, Wu, Wd, dw, fw, rows, cols, b_up=bu, b_down=bd)
+    np.testing.assert_allclose(got, want[rows, cols], rtol=1e-12, atol=1e-12)
+
+
 def test_pure_python_scalar_loops():
     """Scalar-level restatement of Eqs. typed-diag/off with explicit Python loops."""
     rng = np.random.default_rng(5)

@@ -31,12 +31,17 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         X, t, W = H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16")
         want = proj.forward(X, t, W, act="gelu", out_dtype=torch.float32)
         got = torch.full_like(want, float("nan"))
-        # count of allocation requests served by torch's caching allocator (frees by the garbage
-        # collector do not touch it): the call must not add one
+        # Two witnesses that nothing was allocated.  torch's caching allocator served no request
+        # (frees by the garbage collector do not touch that counter), and the device's free memory
+        # as the driver reports it did not shrink -- the library links its own CUDA runtime, so a
+        # cudaMalloc inside it would bypass torch's counter but not this one.
+        torch.cuda.synchronize()
         before = torch.cuda.memory_stats()["allocation.all.allocated"]
+        free_before = torch.cuda.mem_get_info()[0]
         proj.forward_static(X, t, W, got, act="gelu")
         torch.cuda.synchronize()
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
+        assert torch.cuda.mem_get_info()[0] >= free_before
         assert proj.last_status() == 0
         # same kernels, same order of additions: the two entry points agree bit for bit,
         # which is tighter than the 5e-3 / 2e-2 bf16 tolerance the parity tests use
