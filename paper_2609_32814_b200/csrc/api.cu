@@ -60,6 +60,10 @@ struct alg_ffn_s {
   int D = 0, F = 0;
   bool timing = false;       // record events between the kernels of each forward call
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  // decode step of the whole FFN in one launch (M <= kFfnDecodeMaxM)
+  bool fd_ok = false;
+  FfnDecodePlan fd = {};
+  unsigned int *d_counters = nullptr;
 };
 
 namespace {
@@ -634,6 +638,10 @@ alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, cons
   }
   f->D = f->up.K;
   f->F = f->up.N;
+  if (dtype == ALG_BF16 && ffn_decode_plan(q, f->up.s, f->down.s, f->D, f->F, f->up.num_sms, &f->fd)) {
+    f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
+               cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
+  }
   *out = f;
   return ALG_OK;
 }
@@ -642,6 +650,7 @@ alg_status_t alg_ffn_destroy(alg_ffn_t h) {
   if (!h) return ALG_ERR_INVALID_ARG;
   for (int e = 0; e < 5; ++e)
     if (h->ev[e]) cudaEventDestroy(h->ev[e]);
+  if (h->d_counters) cudaFree(h->d_counters);
   free_proj(h->down);
   free_proj(h->up);
   delete h;
@@ -671,6 +680,32 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
+  if (h->fd_ok && h->up.opt_small_m && M <= kFfnDecodeMaxM && !h->timing) {
+    // decode step in one launch: both projections, H exchanged through L2 inside the kernel
+    const alg_proj_s &u = h->up;
+    FfnDecodeArgs d = {};
+    d.X = X;
+    d.types = u.sched == ALG_SCHED_CYCLIC ? nullptr : types;
+    d.M = (int)M;
+    d.W_up = W_up, d.W_down = W_down;
+    d.b_up = b_up, d.b_down = b_down;
+    d.act = (int)act;
+    d.H = ws + L.h;
+    d.Y = Y;
+    d.y_bf16 = y_dtype == ALG_BF16;
+    d.D = h->D, d.F = h->F, d.q = u.q;
+    d.counters = h->d_counters;
+    d.status = u.d_status;
+    d.wait_limit = u.wait_limit;
+    d.extra_expect_bytes = u.test_extra_expect;
+    d.tab_up = u.d_tab, d.tab_dn = h->down.d_tab;
+    d.small_q = u.q <= kDecodeParamQ;
+    if (d.small_q) {
+      for (int e = 0; e <= u.q; ++e) d.so_d[e] = u.tab.so[e], d.so_f[e] = h->down.tab.so[e];
+      for (int e = 0; e < u.q * u.q; ++e) d.keep[e] = u.tab.keep[e];
+    }
+    return cuda_status(launch_ffn_decode(d, h->fd, st));
+  }
   if (use_decode(h->up, M) && use_decode(h->down, M)) {
     // decode shapes: no bucketing, H stays in the original row order
     void *Hd = ws + L.h;
@@ -781,7 +816,11 @@ alg_status_t alg_ffn_macs(alg_ffn_t h, const int64_t *rows_per_type, int64_t *ma
 
 alg_status_t alg_ffn_last_status(alg_ffn_t h, void *stream, alg_status_t *status) {
   if (!h) return ALG_ERR_INVALID_ARG;
-  return read_status(h->up.d_status, stream, status);
+  alg_status_t s = read_status(h->up.d_status, stream, status);
+  // a launch that gave up may have left the exchange counters of the one-launch decode step half way
+  if (s == ALG_OK && *status != ALG_OK && h->d_counters)
+    s = cuda_status(cudaMemset(h->d_counters, 0, 2 * sizeof(unsigned int)));
+  return s;
 }
 
 const char *alg_status_string(alg_status_t s) {

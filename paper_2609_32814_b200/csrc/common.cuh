@@ -193,6 +193,39 @@ struct DecodeArgs {
 bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *plan);
 cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st);
 
+// decode step of the whole FFN in one launch (ffn_decode.cu), M <= kFfnDecodeMaxM
+constexpr int kFfnDecodeMaxM = 16;
+struct FfnDecodePlan {
+  int su, sd;          // columns of the hidden state / of the output one CTA owns (multiples of 8)
+  int n_up, n_dn;      // CTAs with an up strip / a down strip
+  int wd_bytes, wu_bytes, stage_bytes, p_bytes, ctl_bytes;  // shared-memory regions
+};
+struct FfnDecodeArgs {
+  const void *X;          // [M][D] bf16, packed
+  const int32_t *types;   // nullptr => cyclic (row mod q)
+  int M;
+  const void *W_up, *W_down;   // canonical banks, packed: [D][F] and [F][D]
+  const void *b_up, *b_down;
+  int act;
+  void *H;                // [M][F] bf16 scratch in global memory
+  void *Y;                // [M][D]
+  int y_bf16;
+  int D, F, q;
+  int su, sd, n_up, n_dn;
+  int off_wu, off_stage, off_p, off_ctl;   // shared-memory offsets (the W_down slice sits at 0)
+  int kc_up, kc_dn, m_pad;                 // K-chunk lengths of the staged activations; staged rows (8 or 16)
+  unsigned int *counters;                  // [0] producers arrived, [1] consumers past the wait; zero between launches
+  int *status;
+  long long wait_limit;
+  int extra_expect_bytes;
+  const DevTable *tab_up, *tab_dn;         // tables in device memory (q > kDecodeParamQ)
+  int small_q;
+  int so_d[kDecodeParamQ + 1], so_f[kDecodeParamQ + 1];
+  uint32_t keep[kDecodeParamQ * kDecodeParamQ];
+};
+bool ffn_decode_plan(int q, const int *dw, const int *fw, int D, int F, int num_sms, FfnDecodePlan *plan);
+cudaError_t launch_ffn_decode(const FfnDecodeArgs &a, const FfnDecodePlan &plan, cudaStream_t st);
+
 void count_launch(int n = 1);
 int handle_device(alg_proj_t h);  // device the handle was created on (-1 for a null handle)
 

@@ -37,8 +37,28 @@
     }                                                                                               \
   } while (0)
 
+// Append-only log shared by all launches: record = {tag, globaltimer, clock64}; the cursor sits at
+// buffer slot 24 * cap + 2048, the records follow it.  CTA 0 / thread 0 only.
+#define ALG_TRACE_SEQ(tag)                                                                          \
+  do {                                                                                              \
+    if (alg_trace_buf && blockIdx.x == 0 && threadIdx.x == 0) {                                     \
+      long long *base_ = alg_trace_buf + (size_t)24 * alg_trace_cap + 2048;                         \
+      const unsigned long long i_ = atomicAdd((unsigned long long *)base_, 1ull);                   \
+      if (i_ < 4096) {                                                                              \
+        unsigned long long gt_;                                                                     \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_));                                     \
+        base_[1 + 3 * i_] = (tag);                                                                  \
+        base_[2 + 3 * i_] = (long long)gt_;                                                         \
+        base_[3 + 3 * i_] = clock64();                                                              \
+      }                                                                                             \
+    }                                                                                               \
+  } while (0)
+
 #else
 
+#define ALG_TRACE_SEQ(tag) \
+  do {                     \
+  } while (0)
 #define ALG_TRACE_DEFINE(name)
 #define ALG_TRACE_VARS \
   do {                 \

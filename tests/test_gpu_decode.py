@@ -136,3 +136,166 @@ def test_bounded_wait_expires_and_the_handle_recovers():
     proj.set_option("wait_limit_cycles", 4_000_000_000)
     assert np.array_equal(H.to_np(proj.forward(X, t, W, out_dtype=torch.float32)), ref)
     assert proj.last_status() == 0
+
+
+# ---- the decode step of the whole FFN in one launch (M <= 16) -----------------------------------
+
+def _ffn_int_workload(q, M, D, F, types=None, seed=1):
+    """Integer FFN problem whose hidden state stays exactly representable in bf16 (entries of X and
+    W_down in {-1,0,1}, W_up sparse), so that with act = none both projections are exact."""
+    if types is None:
+        types = synth.uniform_types(4000 + seed, M, q)
+    wl = synth.make_workload("ffndec", config=4, variant=700 + seed, dtype="bf16", q=q, M=M, D=D, F=F, types=types,
+                             integer=True)
+    wl.X = np.sign(wl.X).astype(np.float32)
+    wl.W_up = (np.sign(wl.W_up) * (np.abs(wl.W_up) > 2)).astype(np.float32)
+    wl.W_down = np.sign(wl.W_down).astype(np.float32)
+    return wl
+
+
+def _ffn_int_ref(wl, keep=None, b_up=None, b_down=None):
+    Hh = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, keep=keep, bias=b_up)
+    assert np.abs(Hh).max() <= 256          # exactly representable in bf16
+    return oracle.proj(Hh, wl.types, wl.W_down, wl.f_widths, wl.d_widths, keep=keep, bias=b_down)
+
+
+@pytest.mark.parametrize("q,M,D,F", [
+    (2, 1, 768, 3072), (2, 3, 768, 3072), (2, 8, 768, 3072), (2, 9, 768, 3072), (2, 16, 768, 3072),   # config 4
+    (4, 5, 512, 2048), (3, 16, 192, 384), (1, 7, 256, 512), (8, 12, 512, 1024),
+    (16, 11, 1024, 2048),      # table read from device memory
+    (2, 16, 96, 160),          # widths that are no multiples of 64: ragged last K chunk
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_ffn_decode_one_launch_integer_bit_exact(q, M, D, F, out_dtype):
+    wl = _ffn_int_workload(q, M, D, F, seed=q * 50 + M)
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    bu = synth.small_ints(71, (F,), -2, 2)
+    bd = synth.small_ints(72, (D,), -2, 2)
+    args = (H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"))
+    launches = binding.launch_count()
+    Y = ffn.forward(*args, b_up=H.to_dev(bu, "bf16"), b_down=H.to_dev(bd, "bf16"), act=None, out_dtype=out_dtype)
+    assert binding.launch_count() - launches == 1          # one kernel for the whole FFN
+    assert ffn.last_status() == 0
+    ref = _ffn_int_ref(wl, b_up=bu, b_down=bd)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5].tolist()}"
+    # the two-kernel path of the same handle gives the same bits
+    ffn.set_option("small_m_kernel", 0)
+    Y2 = ffn.forward(*args, b_up=H.to_dev(bu, "bf16"), b_down=H.to_dev(bd, "bf16"), act=None, out_dtype=out_dtype)
+    assert np.array_equal(H.to_np(Y2), ref)
+
+
+def test_ffn_decode_skips_blocks_no_row_needs():
+    """All rows of type 0: W_10 of both banks is used by nobody.  Poisoned with NaN it must stay
+    unread; the same for type 1 and W_01."""
+    q, M, D, F = 2, 6, 768, 3072
+    for t in (0, 1):
+        wl = _ffn_int_workload(q, M, D, F, types=np.full(M, t, dtype=np.int32), seed=90 + t)
+        Wu, Wd = wl.W_up.copy(), wl.W_down.copy()
+        o = 1 - t   # block (o, t): input group o, output group t is needed only by rows of type o
+        Wu[o * 384:(o + 1) * 384, t * 1536:(t + 1) * 1536] = np.nan
+        Wd[o * 1536:(o + 1) * 1536, t * 384:(t + 1) * 384] = np.nan
+        ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+        Y = ffn.forward(H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(Wu, "bf16"), H.to_dev(Wd, "bf16"),
+                        act=None, out_dtype=torch.float32)
+        assert np.array_equal(H.to_np(Y), _ffn_int_ref(wl)), t
+
+
+def test_ffn_decode_tables_cyclic_bad_type_gelu():
+    q, M, D, F = 4, 13, 512, 1024
+    wl = _ffn_int_workload(q, M, D, F, seed=7)
+    X, Wu, Wd = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16")
+    for table in ("dense", "q2pow"):
+        keep = oracle.support(q, table)
+        ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table=table)
+        Y = ffn.forward(X, H.dev_types(wl.types), Wu, Wd, act=None, out_dtype=torch.float32)
+        assert np.array_equal(H.to_np(Y), _ffn_int_ref(wl, keep=keep)), table
+    cyc = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
+    wc = _ffn_int_workload(q, M, D, F, types=synth.cyclic_types(M, q), seed=7)
+    Y = cyc.forward(X, None, Wu, Wd, act=None, out_dtype=torch.float32)
+    assert np.array_equal(H.to_np(Y), _ffn_int_ref(wc))
+    # out-of-range types: status, zero rows, the other rows exact; bitwise repeatable
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    types = wl.types.copy()
+    types[[2, 12]] = [7, -1]
+    Y1 = ffn.forward(X, H.dev_types(types), Wu, Wd, act=None, out_dtype=torch.float32)
+    assert ffn.last_status() == 5
+    Y2 = ffn.forward(X, H.dev_types(types), Wu, Wd, act=None, out_dtype=torch.float32)
+    assert torch.equal(Y1, Y2)
+    got = H.to_np(Y1)
+    assert not got[[2, 12]].any()
+    good = np.ones(M, bool)
+    good[[2, 12]] = False
+    assert np.array_equal(got[good], _ffn_int_ref(wl)[good])
+    # real-valued data with GELU and biases against the fp64 oracle
+    w = synth.make_workload("ffndec-n", config=4, variant=777, dtype="bf16", q=2, M=16, D=768, F=3072,
+                            types=synth.decode_types(5, 16, 2))
+    bu, bd = synth.bf16_round(synth.normal(8, (w.F,), 0.2)), synth.bf16_round(synth.normal(9, (w.D,), 0.2))
+    f2 = binding.FFN(w.d_widths, w.f_widths, dtype="bf16")
+    Yn = f2.forward(H.to_dev(w.X, "bf16"), H.dev_types(w.types), H.to_dev(w.W_up, "bf16"), H.to_dev(w.W_down, "bf16"),
+                    b_up=H.to_dev(bu, "bf16"), b_down=H.to_dev(bd, "bf16"), act="gelu", out_dtype=torch.float32)
+    ref = oracle.ffn(w.X, w.types, w.W_up, w.W_down, w.d_widths, w.f_widths, b_up=bu, b_down=bd)
+    H.assert_bf16_close(H.to_np(Yn), ref, False, "one-launch decode FFN")
+
+
+def test_ffn_decode_chain_in_a_graph_replays():
+    """Six dependent layers (distinct weights, layer l+1 reads layer l's output) captured in one
+    CUDA graph, as the streaming benchmark does: consecutive launches overlap through programmatic
+    dependent launch and share the handle's exchange counters.  Every replay must reproduce, bit
+    for bit, the result of running the layers one at a time with a device synchronisation between
+    them; that result is checked against the oracle layer by layer."""
+    q, M, D, F, L = 2, 8, 768, 3072, 6
+    wl = synth.config4(M)
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    t = H.dev_types(wl.types)
+    Wu_h = [synth.bf16_round(synth.normal(100 + l, (D, F), 0.02)) for l in range(L)]
+    Wd_h = [synth.bf16_round(synth.normal(200 + l, (F, D), 0.02)) for l in range(L)]
+    Wu, Wd = [H.to_dev(w, "bf16") for w in Wu_h], [H.to_dev(w, "bf16") for w in Wd_h]
+    acts = [H.to_dev(wl.X, "bf16")] + [torch.zeros((M, D), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    ws = torch.empty(ffn.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    want = [acts[0]]
+    for l in range(L):       # one layer at a time
+        want.append(ffn.forward(want[l], t, Wu[l], Wd[l], act="gelu", workspace=ws))
+        torch.cuda.synchronize()
+        ref = oracle.ffn(H.to_np(want[l]), wl.types, Wu_h[l], Wd_h[l], wl.d_widths, wl.f_widths)
+        H.assert_bf16_close(H.to_np(want[l + 1]), ref, True, f"layer {l}")
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        for l in range(L):   # back to back, overlapping
+            ffn.forward(acts[l], t, Wu[l], Wd[l], act="gelu", out=acts[l + 1], workspace=ws, stream=stream)
+        stream.synchronize()
+        for l in range(L):
+            assert torch.equal(acts[l + 1], want[l + 1]), f"eager layer {l}"
+        with torch.cuda.graph(g, stream=stream):
+            for l in range(L):
+                ffn.forward(acts[l], t, Wu[l], Wd[l], act="gelu", out=acts[l + 1], workspace=ws, stream=stream)
+    for rep in range(4):
+        for l in range(L):
+            acts[l + 1].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for l in range(L):
+            assert torch.equal(acts[l + 1], want[l + 1]), f"replay {rep} layer {l}"
+    assert ffn.last_status() == 0
+
+
+def test_ffn_decode_bounded_waits_expire_and_the_handle_recovers():
+    q, M, D, F = 2, 4, 768, 3072
+    wl = _ffn_int_workload(q, M, D, F, seed=55)
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    args = (H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"))
+    ref = _ffn_int_ref(wl)
+    assert np.array_equal(H.to_np(ffn.forward(*args, act=None, out_dtype=torch.float32)), ref)
+    ffn.set_option("wait_limit_cycles", 6_000_000)       # about 3 ms per wait
+    ffn.set_option("test_stall_bytes", 512)
+    ffn.forward(*args, act=None, out_dtype=torch.float32)
+    assert ffn.last_status() == 6                         # the weight barrier and then the exchange gave up
+    ffn.set_option("test_stall_bytes", 0)
+    ffn.set_option("wait_limit_cycles", 4_000_000_000)
+    for _ in range(2):                                    # counters were reset with the status
+        assert np.array_equal(H.to_np(ffn.forward(*args, act=None, out_dtype=torch.float32)), ref)
+    assert ffn.last_status() == 0
