@@ -1,13 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the row-typed star_q FFN forward pass (up -> GELU -> down) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
-One step = one pass of the whole hot path (grouped tcgen05 GEMM with fused GELU for the up
-projection, grouped GEMM with fused row scatter for the down projection; with explicit row types
-also the bucketing and row-gather kernels) over one synthetic batch of the q=2,
-768 -> 3072 -> 768, M = 8 x 1024 workload.
-Prints ONE JSON line.  FLOPs count only the block GEMMs the rule keeps.
+One step = one pass of the whole hot path over one synthetic batch: grouped tcgen05 GEMM with
+fused GELU for the up projection, grouped GEMM with fused row scatter for the down projection;
+with explicit row types also the bucketing and row-gather kernels.  Prints ONE JSON line.  FLOPs
+count only the block GEMMs the rule keeps.
+
+--config selects the workload (default 2, the q=2 768 -> 3072 -> 768 FFN at M = 8 x 1024 rows):
+    2                  q=2 FFN of the ~110M model, type = position mod 2 (cyclic schedule)
+    3q4 3q8            general q, groups of 128 / 512, M = 16384, i.i.d. row types
+    4                  KV-cached decode step, M in {1, 8, 32, 64}: 64-layer dependent FFN chain
+    5q2 5q4 5q8 5q16   scale sweep 4096 -> 16384 -> 4096, M = 32768, i.i.d. row types
+    pilot              tensor-square law Q_2 (x) Q_2 at the paper's pilot shape (768 -> 1536 -> 768)
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
 rank runs the same per-GPU batch (weak scaling), time = max over ranks.
@@ -19,6 +25,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -31,13 +38,32 @@ if ROOT not in sys.path:
 
 import numpy as np
 
-WORKLOAD = "cfg2: q=2 FFN 768->3072->768 (GELU), M=8x1024 rows, type = position mod 2, bf16"
 METRIC = "star_q FFN kept-GEMM throughput (prefill)"
 UNIT = "TFLOP/s"
-N_SETS = 6
-# DRAM traffic of the grouped-GEMM kernels from the ncu capture summarised under profiles/
-# (bytes of the up launch + the down launch of one step of this workload).
-NCU_TRAFFIC_BYTES = 19.2e6 + 57.0e6  # up + down launch, cold caches (profiles/proj_tc_kernel_cfg2.md)
+N_SETS = 6            # working sets of configuration 2
+L2_BYTES = 126e6
+
+CONFIGS = {
+    "2": dict(q=2, D=768, F=3072, M=8192, law="qq", schedule="cyclic",
+              label="cfg2: q=2 FFN 768->3072->768 (GELU), M=8x1024 rows, type = position mod 2, bf16"),
+    "3q4": dict(q=4, D=512, F=2048, M=16384, law="qq", schedule="explicit",
+                label="cfg3: q=4 FFN 512->2048->512 (groups of 128 / 512), M=16384 rows, i.i.d. row types, bf16"),
+    "3q8": dict(q=8, D=1024, F=4096, M=16384, law="qq", schedule="explicit",
+                label="cfg3: q=8 FFN 1024->4096->1024 (groups of 128 / 512), M=16384 rows, i.i.d. row types, bf16"),
+    "5q2": dict(q=2, D=4096, F=16384, M=32768, law="qq", schedule="explicit",
+                label="cfg5: q=2 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
+    "5q4": dict(q=4, D=4096, F=16384, M=32768, law="qq", schedule="explicit",
+                label="cfg5: q=4 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
+    "5q8": dict(q=8, D=4096, F=16384, M=32768, law="qq", schedule="explicit",
+                label="cfg5: q=8 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
+    "5q16": dict(q=16, D=4096, F=16384, M=32768, law="qq", schedule="explicit",
+                 label="cfg5: q=16 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
+    "pilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="explicit",
+                  label="pilot: Q_2 (x) Q_2 FFN 768->1536->768 (4 x 192 / 4 x 384), M=8x1536 rows, interval schedule, bf16"),
+    "4": dict(q=2, D=768, F=3072, M=64, law="qq", schedule="explicit",
+              label="cfg4: KV-cached decode step, q=2 FFN 768->3072->768, M in {1,8,32,64}, type = position mod 2, bf16"),
+}
+WORKLOAD = CONFIGS["2"]["label"]
 
 
 def _peaks():
@@ -51,12 +77,19 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons (NVML, read-only) while the timed region runs."""
+    """Samples SM clock and throttle reasons (NVML, read-only) while the timed region runs.
+    Sampling starts with the context; only samples taken after arm() -- called once the first
+    launch of the timed region is enqueued -- count."""
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int):
         self.index, self.samples, self._stop, self._t = index, [], threading.Event(), None
         self.max_mhz = None
+        self.t_arm = None
+
+    def arm(self):
+        if self.t_arm is None:
+            self.t_arm = time.time()
 
     def _run(self):
         try:
@@ -67,8 +100,8 @@ class ClockSampler:
             while not self._stop.is_set():
                 mhz = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
                 mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
-                self.samples.append((float(mhz), int(mask)))
-                self._stop.wait(0.002)
+                self.samples.append((float(mhz), int(mask), time.time()))
+                self._stop.wait(0.001)
         except Exception:
             self._run_smi()
 
@@ -84,7 +117,7 @@ class ClockSampler:
                 if len(parts) >= 6:
                     self.max_mhz = float(parts[1])
                     mask = sum(b for b, v in zip(bits, parts[2:6]) if v.lower().startswith("active"))
-                    self.samples.append((float(parts[0]), mask))
+                    self.samples.append((float(parts[0]), mask, time.time()))
             except Exception:
                 pass
             self._stop.wait(0.05)
@@ -92,20 +125,23 @@ class ClockSampler:
     def __enter__(self):
         self._t = threading.Thread(target=self._run, daemon=True)
         self._t.start()
-        time.sleep(0.02)
         return self
 
     def __exit__(self, *a):
         self._stop.set()
         self._t.join(timeout=10)
 
+    def armed_samples(self):
+        return [s for s in self.samples if self.t_arm is not None and s[2] >= self.t_arm]
+
     def summary(self):
-        sm = [s[0] for s in self.samples]
+        live = self.armed_samples()
+        sm = [s[0] for s in live]
         mask = 0
-        for s in self.samples:
+        for s in live:
             mask |= s[1]
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
-                "reasons": [n for b, n in self.REASONS.items() if mask & b], "samples": len(self.samples)}
+                "reasons": [n for b, n in self.REASONS.items() if mask & b], "samples": len(live)}
 
 
 def max_over_ranks(value: float, device=None) -> float:
@@ -131,73 +167,92 @@ def whole_job_value(flops_per_rank_step: int, world: int, steps: int, total_ms: 
     return world * flops_per_rank_step * steps / (total_ms * 1e-3) / 1e12
 
 
-def kept_flops(ffn, wl) -> int:
-    rows = np.bincount(wl.types, minlength=wl.q).tolist()
-    return 2 * ffn.macs(rows)
+def make_workload(name: str):
+    """The synthetic problem of a configuration (host arrays; the parity tests use the same generators)."""
+    from paper_2609_32814_b200 import synth
+    if name == "2":
+        return synth.config2()
+    if name in ("3q4", "3q8"):
+        return synth.config3(CONFIGS[name]["q"])
+    if name.startswith("5q"):
+        return synth.config5(CONFIGS[name]["q"])
+    if name == "pilot":
+        return synth.pilot_ffn(M=CONFIGS[name]["M"])
+    if name == "4":
+        return synth.config4(64)
+    raise ValueError(name)
+
+
+def oracle_sample(name: str, wl, budget_macs: float = 2.0e11):
+    """Rows of the workload the CPU oracle is timed on: evenly spaced, about `budget_macs` of work."""
+    import oracle
+    cfg = CONFIGS[name]
+    keep = oracle.support(wl.q, cfg["law"])
+    per_row = (oracle.macs(keep, wl.d_widths, wl.f_widths, np.ones(wl.q, dtype=np.int64)) +
+               oracle.macs(keep, wl.f_widths, wl.d_widths, np.ones(wl.q, dtype=np.int64))) / wl.q
+    n = int(min(wl.M, max(16, 2 ** int(math.log2(max(16.0, budget_macs / per_row))))))
+    rows = np.arange(0, wl.M, max(1, wl.M // n))[:n]
+    counts = np.bincount(wl.types[rows], minlength=wl.q)
+    flops = 2 * (oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + oracle.macs(keep, wl.f_widths, wl.d_widths, counts))
+    return rows, keep, flops
 
 
 def run_reference(args):
     """The oracle as it stands, on the host cores, on a row sample of the same workload."""
     import oracle
-    from paper_2609_32814_b200 import synth
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = synth.config2()
-    sample_rows = 1024
-    rows = np.arange(0, wl.M, wl.M // sample_rows)
+    wl = make_workload(args.config)
+    rows, keep, flops = oracle_sample(args.config, wl, 1.0e11)
     X, t = wl.X[rows], wl.types[rows]
-    keep = oracle.support(wl.q)
-    counts = np.bincount(t, minlength=wl.q)
-    flops = 2 * (oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + oracle.macs(keep, wl.f_widths, wl.d_widths, counts))
     for _ in range(args.warmup):
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
     dt = (time.perf_counter() - t0) / args.steps
     val = flops / dt / 1e12
-    sample = f"{sample_rows} of {wl.M} rows per step (every {wl.M // sample_rows}th row), all outputs, fp64"
+    sample = f"{len(rows)} of {wl.M} rows per step (evenly spaced), all outputs, fp64"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": CONFIGS[args.config]["label"], "sample": sample},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def time_cpu_oracle(wl):
+def time_cpu_oracle(name, wl):
     import oracle
-    sample_rows = 2048
-    rows = np.arange(0, wl.M, wl.M // sample_rows)
+    rows, keep, flops = oracle_sample(name, wl)
     X, t = wl.X[rows], wl.types[rows]
-    keep = oracle.support(wl.q)
-    counts = np.bincount(t, minlength=wl.q)
-    flops = 2 * (oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + oracle.macs(keep, wl.f_widths, wl.d_widths, counts))
     best = None
     t_all = time.perf_counter()
     for _ in range(3):
         t0 = time.perf_counter()
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
         if time.perf_counter() - t_all > 25:
             break
     return {"value": flops / best / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"{sample_rows} of {wl.M} rows (every {wl.M // sample_rows}th), all outputs, best of <=3, "
-                      f"{best:.2f} s per pass"}
+            "sample": f"{len(rows)} of {wl.M} rows (evenly spaced), all outputs, best of <=3, {best:.2f} s per pass"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=600)
+    ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=12)
+    ap.add_argument("--config", default="2", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the dense-control / decode side measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the dense-control / explicit-types / decode side measurements")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.steps is None:
+        args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "4": 20}.get(args.config, 20) if args.impl == "ours" else 3
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else min(args.warmup, 1)
     if args.impl == "reference":
         run_reference(args)
         return
@@ -205,7 +260,7 @@ def main():
     import torch
     import torch.distributed as dist
 
-    from paper_2609_32814_b200 import binding, synth
+    from paper_2609_32814_b200 import binding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -215,32 +270,56 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     binding.lib()  # fail loudly if the CUDA library is missing
+    ctx = {"world": world, "rank": rank, "local_rank": local_rank, "dist": dist, "torch": torch, "binding": binding}
+    line = run_decode(args, ctx) if args.config == "4" else run_prefill(args, ctx)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
 
-    wl = synth.config2()
+
+def run_prefill(args, ctx):
+    torch, binding, dist = ctx["torch"], ctx["binding"], ctx["dist"]
+    world, rank, local_rank = ctx["world"], ctx["rank"], ctx["local_rank"]
+    from paper_2609_32814_b200 import synth
+    name, cfg = args.config, CONFIGS[args.config]
+    wl = make_workload(name)
     dev = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)
-    # config 2 fixes the schedule "type = position mod 2": the handle is created with it
-    # (ALG_SCHED_CYCLIC), the per-call types array is then not needed.  The explicit-types path of
-    # the same workload is timed as a side measurement.
-    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
-    flops = kept_flops(ffn, wl)
+    # configuration 2 fixes the schedule "type = position mod 2": its handle is created with that
+    # schedule (the per-call types array is then not needed); the explicit-types path of the same
+    # workload is timed as a side measurement.  The other configurations draw i.i.d. row types.
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"], schedule=cfg["schedule"])
+    counts = np.bincount(wl.types, minlength=wl.q).tolist()
+    flops = 2 * ffn.macs(counts)
     stream = torch.cuda.current_stream()
     types = torch.from_numpy(wl.types).cuda()
+    call_types = None if cfg["schedule"] == "cyclic" else types
+    M, D, F = wl.M, wl.D, wl.F
 
-    # ---- working sets: N_SETS independent copies of (X, W_up, W_down, Y, workspace), ~85 MB each,
-    # used round-robin, so every step reads inputs and weights that have left the 126 MB L2 since
-    # their last use (no explicit flush: a write-flush would leave L2 full of dirty lines whose
-    # write-back the next step then pays for).
-    ws_bytes = ffn.workspace_bytes(wl.M)
+    # ---- working sets: independent copies of (X, W_up, W_down, Y, workspace) used round-robin, so
+    # every step reads inputs and weights that have left the 126 MB L2 since their last use (no
+    # explicit flush: a write-flush would leave L2 full of dirty lines whose write-back the next
+    # step then pays for).  A set larger than twice the L2 needs no second one.
+    ws_bytes = ffn.workspace_bytes(M)
+    set_bytes = 2 * M * D * 2 + 2 * D * F * 2 + ws_bytes
+    n_sets = N_SETS if name == "2" else (1 if set_bytes > 2 * L2_BYTES else int(min(6, max(2, math.ceil(4 * L2_BYTES / set_bytes)))))
     sets = []
-    for r in range(N_SETS):
-        Xr = synth.bf16_round(synth.normal(rank_batch_seed(rank, world, r), wl.X.shape, 1.0)) if (r or world > 1) else wl.X
-        sets.append({"X": dev(Xr), "Wu": dev(wl.W_up).clone(), "Wd": dev(wl.W_down).clone(),
-                     "Y": torch.empty((wl.M, wl.D), dtype=torch.bfloat16, device="cuda"),
+    for r in range(n_sets):
+        if r == 0 and world == 1:
+            Xr = dev(wl.X)
+        elif name == "2":
+            Xr = dev(synth.bf16_round(synth.normal(rank_batch_seed(rank, world, r), wl.X.shape, 1.0)))
+        else:
+            g = torch.Generator(device="cuda").manual_seed(synth.seed_for(9, rank * 16 + r))
+            Xr = torch.randn((M, D), device="cuda", generator=g).to(torch.bfloat16)
+        sets.append({"X": Xr, "Wu": dev(wl.W_up).clone(), "Wd": dev(wl.W_down).clone(),
+                     "Y": torch.empty((M, D), dtype=torch.bfloat16, device="cuda"),
                      "ws": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")})
-    footprint_mb = N_SETS * (2 * wl.M * wl.D * 2 + 2 * wl.D * wl.F * 2 + ws_bytes) / 1e6
+    footprint_mb = n_sets * set_bytes / 1e6
 
-    def step(i, handle=None, tt=None):
-        s_ = sets[i % N_SETS]
+    def step(i, handle=None, tt=call_types):
+        s_ = sets[i % n_sets]
         (handle or ffn).forward(s_["X"], tt, s_["Wu"], s_["Wd"], act="gelu", out=s_["Y"], workspace=s_["ws"], stream=stream)
 
     def barrier():
@@ -248,12 +327,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def time_steps(n, handle=None, tt=None, first=0):
+    def time_steps(n, handle=None, tt=call_types, first=0, clocks=None):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
         for i in range(n):
             step(first + i, handle, tt)
+            if clocks is not None and i == 0:
+                clocks.arm()      # samples count from the moment the first launch is enqueued
         e1.record(stream)
         barrier()
         return e0.elapsed_time(e1)
@@ -266,24 +347,25 @@ def main():
     # ---- timed region: exactly K steps between two events, barrier + synchronize on both sides ----
     launches0 = binding.launch_count()
     with ClockSampler(local_rank) as clocks:
-        total_ms = time_steps(args.steps, first=args.warmup)
+        total_ms = time_steps(args.steps, first=args.warmup, clocks=clocks)
     launches = binding.launch_count() - launches0
     clock_note = "sampled during the timed region"
-    if len(clocks.samples) < 5:
-        # the timed region is only tens of milliseconds; when the sampler (NVML, else nvidia-smi
-        # every 50 ms) caught fewer than five samples, the same steps run on, untimed, under the
+    if len(clocks.armed_samples()) < 5:
+        # the timed region is too short for five samples: the same steps run on, untimed, under the
         # sampler for a quarter of a second so that the clock record covers this load
         with ClockSampler(local_rank) as clocks2:
             t_end = time.time() + 0.25
             i = 0
             while time.time() < t_end:
-                for _ in range(50):
+                for _ in range(20):
                     step(i)
                     i += 1
+                clocks2.arm()
                 torch.cuda.synchronize()
-        clocks.samples += clocks2.samples
+        clocks.samples = clocks.armed_samples() + clocks2.armed_samples()
+        clocks.t_arm = min([s[2] for s in clocks.samples], default=None)
         clocks.max_mhz = clocks.max_mhz or clocks2.max_mhz
-        clock_note = "timed region too short for the sampler: extended by 0.25 s of the same steps, untimed"
+        clock_note = "timed region too short for five samples: extended by 0.25 s of the same steps, untimed"
     total_ms = max_over_ranks(total_ms, "cuda")
     ms_per_step = total_ms / args.steps
     value = whole_job_value(flops, world, args.steps, total_ms)
@@ -292,48 +374,60 @@ def main():
     # ---- per-kernel durations (second pass with events between the kernels) ----
     ffn.set_timing(True)
     kt = np.zeros(4)
-    for i in range(args.steps):
+    n_kt = min(args.steps, 100)
+    for i in range(n_kt):
         step(i)
         kt += np.array(ffn.get_timing())
-    kt /= args.steps
+    kt /= n_kt
     ffn.set_timing(False)
-    peaks = _peaks()
-    # The timed region holds nothing but launches of the dominant kernel (two per step: up and
-    # down projection, overlapping at their edges through programmatic dependent launch), so its
-    # average launch duration is the event time of the region / launches, and
-    # achieved = algorithmic FLOPs of a launch / that duration = FLOPs of the region / its time.
-    avg_launch_ms = total_ms / max(1, launches // max(1, world))
-    achieved = flops * args.steps / (total_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "proj_tc_kernel (two launches per step: up with GELU, down with row scatter)",
-                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "peak_source": f"{peaks['source']} (burst)",
-                "frac_of_sustained_peak": (achieved / peaks["bf16_tflops_sustained"]) if peaks["bf16_tflops_sustained"] else None,
-                "sustained_peak": peaks["bf16_tflops_sustained"],
-                "peak_note": "600 back-to-back steps (~34 ms) run before the power cap bites, like the burst measurement of "
-                             "the peak, so the burst figure is the denominator; --steps 4000 (0.25 s, sw_power_cap active) "
-                             "measured 928 TFLOP/s = 0.68 of the sustained peak",
-                "traffic": NCU_TRAFFIC_BYTES / 2, "traffic_note": "mean DRAM bytes per launch, ncu, cold caches",
-                "avg_launch_ms": avg_launch_ms, "algorithmic_gflop_per_launch": flops / 2 / 1e9,
-                "algorithmic_mb_per_launch": (wl.M * wl.D + wl.D * wl.F + wl.M * wl.F) * 2 / 1e6,
-                "isolated_kernel_ms": {"up": float(kt[2]), "down": float(kt[3]),
-                                       "note": "events between the kernels (no launch overlap)"}}
 
-    # ---- end to end through the host entry point: pinned H2D of X, D2H of Y inside the timing ----
+    # ---- roofline: the slower of (kept FLOPs at the bf16 peak) and (algorithmic bytes at the HBM rate) ----
+    peaks = _peaks()
+    region_s = total_ms * 1e-3
+    burst = region_s < 0.1       # a region this short runs at burst clocks, like the burst measurement of the peak
+    peak_tf = peaks["bf16_tflops"] if burst or not peaks["bf16_tflops_sustained"] else peaks["bf16_tflops_sustained"]
+    bytes_proj = (M * D + D * F + M * F) * 2          # one projection: activations in, weights, activations out
+    bytes_step = 2 * bytes_proj                       # H is written by the up kernel and read by the down kernel
+    t_tensor, t_hbm = flops / (peak_tf * 1e12), bytes_step / (peaks["hbm_gbs"] * 1e9)
+    gemm_launches = 2 * args.steps                    # the dominant kernel runs twice per step
+    avg_launch_ms = total_ms / gemm_launches
+    kernel = "proj_tc_kernel (two launches per step: up with GELU, down with row scatter)"
+    if t_tensor >= t_hbm:
+        achieved = flops * args.steps / region_s / 1e12
+        roofline = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": achieved / peak_tf,
+                    "peak_source": f"{peaks['source']} ({'burst' if peak_tf == peaks['bf16_tflops'] else 'sustained'})",
+                    "peak_note": f"timed region of {args.steps} steps = {region_s * 1e3:.1f} ms: "
+                                 + ("shorter than 0.1 s, runs at burst clocks like the burst measurement of the peak"
+                                    if burst else "long enough for the power cap, compared with the sustained peak"),
+                    "algorithmic_gflop_per_launch": flops / 2 / 1e9}
+    else:
+        achieved = bytes_step * args.steps / region_s / 1e9
+        roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                    "tensor_time_us": t_tensor * 1e6, "hbm_time_us": t_hbm * 1e6}
+    roofline.update({"traffic": None, "traffic_note": "no ncu capture of this kernel version is tied to this line",
+                     "avg_launch_ms": avg_launch_ms, "algorithmic_mb_per_launch": bytes_proj / 1e6,
+                     "isolated_kernel_ms": {"bucketing": float(kt[0]), "gather": float(kt[1]), "up": float(kt[2]),
+                                            "down": float(kt[3]), "note": "events between the kernels (no launch overlap)"}})
+
+    # ---- end to end through the host entry point: pinned H2D of X (and types), D2H of Y inside the timing ----
     # Three slots (pinned X / Y, device workspace, stream) are used round-robin, the way a serving
     # loop would: the upload of step i+1 and the download of step i-1 overlap the kernels of step i.
     # Every step still uploads its own X and downloads its own Y inside the timed region.
     n_slots = 3
+    e2e_steps = args.steps if name == "2" else min(args.steps, 12)
     slots = []
     for k in range(n_slots):
         slots.append({"X": torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory(),
-                      "Y": torch.empty((wl.M, wl.D), dtype=torch.bfloat16).pin_memory(),
-                      "ws": torch.empty(ffn.host_workspace_bytes(wl.M, torch.bfloat16), dtype=torch.uint8, device="cuda"),
+                      "t": None if call_types is None else torch.from_numpy(wl.types).pin_memory(),
+                      "Y": torch.empty((M, D), dtype=torch.bfloat16).pin_memory(),
+                      "ws": torch.empty(ffn.host_workspace_bytes(M, torch.bfloat16), dtype=torch.uint8, device="cuda"),
                       "stream": torch.cuda.Stream()})
-    Xh, Yh = slots[0]["X"], slots[0]["Y"]
 
     def host_step(i):
         sl = slots[i % n_slots]
-        ffn.forward_host(sl["X"], None, sets[i % N_SETS]["Wu"], sets[i % N_SETS]["Wd"], sl["Y"], workspace=sl["ws"],
+        ffn.forward_host(sl["X"], sl["t"], sets[i % n_sets]["Wu"], sets[i % n_sets]["Wd"], sl["Y"], workspace=sl["ws"],
                          stream=sl["stream"])
 
     for i in range(2 * n_slots):
@@ -343,7 +437,7 @@ def main():
     e0.record(stream)
     for sl in slots:
         sl["stream"].wait_event(e0)
-    for i in range(args.steps):
+    for i in range(e2e_steps):
         host_step(i)
     for sl in slots:
         done = torch.cuda.Event()
@@ -351,70 +445,70 @@ def main():
         stream.wait_event(done)
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = max_over_ranks(e2e_ms, "cuda")
-    e2e = {"value": whole_job_value(flops, world, args.steps, e2e_ms), "unit": UNIT,
-           "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
-           "ms_per_step": e2e_ms / args.steps,
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), "cuda")
+    h2d = int(M * D * 2 + (0 if call_types is None else M * 4))
+    e2e = {"value": whole_job_value(flops, world, e2e_steps, e2e_ms), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": int(M * D * 2), "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
            "note": f"{n_slots} host-buffer slots on {n_slots} streams: copies of neighbouring steps overlap the kernels"}
+    del slots
 
     extras = {}
     if rank == 0 and not args.no_extras:
-        extras = side_measurements(binding, wl, types, time_steps, ms_per_step)
+        n = min(24, args.steps)
+        dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule=cfg["schedule"])
+        time_steps(min(6, n), dense)
+        dense_ms = time_steps(n, dense) / n
+        star_ms = time_steps(n) / n
+        extras["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms,
+                              "time_ratio_star_over_dense": star_ms / dense_ms,
+                              "control": "same library, ALG_TABLE_DENSE, same schedule, measured back to back with the star_q run",
+                              "ideal_ratio": flops / (2.0 * 2 * M * D * F)}
+        del dense
+        if name == "2":
+            explicit = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+            time_steps(6, explicit, types)
+            ex_ms = time_steps(n, explicit, types) / n
+            extras["explicit_types"] = {"ms_per_step": ex_ms, "frac_of_roofline": (flops / (ex_ms * 1e-3) / 1e12) / peak_tf,
+                                        "note": "same workload through ALG_SCHED_EXPLICIT (bucketing + row gather kernels run)"}
+            del explicit
+            extras["decode"] = decode_measurements(binding)
 
-    if rank == 0:
-        cpu = time_cpu_oracle(wl) if world >= 1 else None
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "l2": f"{N_SETS} working sets of inputs, weights, outputs and workspace used round-robin "
-                                 f"({footprint_mb:.0f} MB in total, L2 is 126 MB); no data is reused within 5 steps",
-                           "rows_per_gpu": wl.M, "parallelism": f"rows sharded over {world} GPU(s), weights replicated"},
-                "tokens_per_s": world * wl.M * args.steps / (total_ms * 1e-3),
-                "kept_gflop_per_step": flops / 1e9,
-                "clocks": dict(clocks.summary(), note=clock_note), "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "cpu_baseline": cpu}
-        line.update(extras)
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
-
-
-def side_measurements(binding, wl, types, time_steps, star_ms):
-    """The same workload through the explicit-types path, and the dense same-shape control."""
-    out = {}
-    n = 24
-    explicit = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
-    time_steps(6, explicit, types)
-    out["explicit_types"] = {"ms_per_step": time_steps(n, explicit, types) / n,
-                             "note": "same workload through ALG_SCHED_EXPLICIT (bucketing + row gather kernels run)"}
-    dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule="cyclic")
-    time_steps(6, dense)
-    dense_ms = time_steps(n, dense) / n
-    out["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms,
-                       "time_ratio_star_over_dense": star_ms / dense_ms,
-                       "control": "same library, ALG_TABLE_DENSE (8 block GEMMs instead of 6)"}
-    out["decode"] = decode_measurements(binding, wl)
-    return out
+    cpu = time_cpu_oracle(name, wl) if rank == 0 else None
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg["label"],
+                       "l2": (f"{n_sets} working sets of inputs, weights, outputs and workspace used round-robin "
+                              f"({footprint_mb:.0f} MB in total, L2 is 126 MB)" if n_sets > 1 else
+                              f"one working set of {footprint_mb:.0f} MB, several times the 126 MB L2"),
+                       "rows_per_gpu": M, "rows_per_type": counts, "schedule": cfg["schedule"], "law": cfg["law"],
+                       "parallelism": f"rows sharded over {world} GPU(s), weights replicated"},
+            "tokens_per_s": world * M * args.steps / region_s,
+            "kept_gflop_per_step": flops / 1e9,
+            "clocks": dict(clocks.summary(), note=clock_note), "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu}
+    line.update(extras)
+    return line
 
 
-def decode_measurements(binding, wl, layers=64, replays=20):
-    """KV-cached decode shapes (config 4): M new tokens, type = absolute position mod 2.
+def decode_measurements(binding, layers=64, replays=20):
+    """KV-cached decode shapes (configuration 4): M new tokens, type = absolute position mod 2.
     streaming: a CUDA graph of `layers` consecutive FFN layers with distinct weight banks
     (604 MB, far beyond L2), layer l+1 consuming layer l's output -- GB/s counts the weight
     blocks some row needs plus X and Y of every projection.  isolated: one FFN per replay."""
     import torch
     from paper_2609_32814_b200 import synth
     peaks = _peaks()
-    D, F = wl.D, wl.F
+    cfg = CONFIGS["4"]
+    D, F, q = cfg["D"], cfg["F"], cfg["q"]
     g = torch.Generator(device="cuda").manual_seed(1234)
     Wu = [(torch.randn((D, F), device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(layers)]
     Wd = [(torch.randn((F, D), device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(layers)]
-    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    ffn = binding.FFN([D // q] * q, [F // q] * q, dtype="bf16")
     ws = torch.empty(ffn.workspace_bytes(64), dtype=torch.uint8, device="cuda")
     res = []
     stream = torch.cuda.Stream()
+    launches0 = binding.launch_count()
     for M in (1, 8, 32, 64):
         w4 = synth.config4(M)
         types = torch.from_numpy(w4.types).cuda()
@@ -446,15 +540,45 @@ def decode_measurements(binding, wl, layers=64, replays=20):
                 ts.append(e0.elapsed_time(e1))
             return float(np.median(ts))
 
+        l0 = binding.launch_count()
+        chain(1)
+        per_layer_launches = binding.launch_count() - l0
         t_stream = graph_time(layers, replays)
         t_iso = graph_time(1, replays)
         gbs = layers * bytes_layer / (t_stream * 1e-3) / 1e9
         res.append({"M": M, "types_present": present, "needed_mb_per_layer": bytes_layer / 1e6,
+                    "launches_per_layer": per_layer_launches,
                     "stream_us_per_layer": t_stream * 1e3 / layers, "stream_gbs": gbs,
-                    "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "isolated_warm_us": t_iso * 1e3})
+                    "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": gbs / peaks["hbm_gbs"]},
+                    "isolated_warm_us": t_iso * 1e3})
     assert ffn.last_status() == 0
     return {"protocol": f"{layers}-layer dependent FFN chain with distinct weights in one CUDA graph, median of {replays} replays",
-            "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res}
+            "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res,
+            "launches": binding.launch_count() - launches0}
+
+
+def run_decode(args, ctx):
+    """--config 4: the decode chain is the step; value = needed bytes per second at M = 8."""
+    torch, binding = ctx["torch"], ctx["binding"]
+    world, rank, local_rank = ctx["world"], ctx["rank"], ctx["local_rank"]
+    with ClockSampler(local_rank) as clocks:
+        clocks.arm()
+        dec = decode_measurements(binding, replays=max(3, args.steps))
+    head = [r for r in dec["results"] if r["M"] == 8][0]
+    wl = make_workload("4")
+    cpu = time_cpu_oracle("4", wl) if rank == 0 else None
+    return {"metric": "star_q FFN decode: needed weight and activation bytes per second (64-layer dependent chain)",
+            "value": world * head["stream_gbs"], "unit": "GB/s", "n_gpus": world, "steps": max(3, args.steps), "warmup": args.warmup,
+            "ms_per_step": head["stream_us_per_layer"] * 64 / 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": CONFIGS["4"]["label"], "step": "one replay of the 64-layer chain at M = 8; the other M are in `decode`",
+                       "l2": "64 distinct weight banks, 604 MB in total, L2 is 126 MB"},
+            "clocks": dict(clocks.summary(), note="sampled over the whole decode measurement"),
+            "e2e": {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                    "note": "a decode step keeps its activations on the device; no host entry point is timed"},
+            "gpu_launches": int(dec["launches"]), "roofline": dict(head["roofline"], kernel="ffn_decode_kernel", traffic=None),
+            "cpu_baseline": cpu, "decode": dec}
 
 
 if __name__ == "__main__":

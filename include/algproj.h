@@ -93,8 +93,10 @@ typedef enum {
  * not concurrently with one; a value the handle's shape cannot honour is refused with
  * ALG_ERR_UNSUPPORTED_SHAPE and changes nothing.
  *   GEMM_KERNEL       which prefill tensor-core kernel runs: 0 = the library's choice (default),
- *                     1 = one-CTA tiles (tcgen05 cta_group::1), 2 = CTA pairs (cta_group::2;
- *                     needs every output group width to be a multiple of 128).
+ *                     1 = one-CTA 128-row tiles (tcgen05 cta_group::1), 2 = CTA pairs
+ *                     (cta_group::2), 3 = one-CTA 256-row x 128-column tiles (two accumulators
+ *                     per tile, each B block feeds two MMAs).  2 and 3 need every output group
+ *                     width to be a multiple of 128.
  *   TILE_N            tile width of the one-CTA kernel: 0 = automatic, or 128 / 192 / 256 when
  *                     that divides every output group width.
  *   SMALL_M_KERNEL    1 (default): M <= 64 runs the weight-streaming kernels; 0: the prefill

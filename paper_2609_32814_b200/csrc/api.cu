@@ -39,6 +39,12 @@ struct alg_proj_s {
   bool tc_ok = false;
   bool pair_kernel = false; // cta_group::2 kernel (256-row tiles)
   int tile_n = 0;           // tensor-core tile width of the one-CTA kernel
+  // one-CTA kernel with 256-row x 128-column tiles (two accumulators per tile): taken when every
+  // row type has enough rows to fill such tiles.  Its tile classes (128 columns wide) live in
+  // `tab_tall` when the regular tile width is not 128.
+  bool tall_ok = false;
+  DevTable tab_tall;
+  DevTable *d_tab_tall = nullptr;
   int device = 0;
   int num_sms = 148;
   int n_workers = 1;        // persistent CTAs (or CTA pairs) of the tensor-core kernel
@@ -77,6 +83,33 @@ int tile_m_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kT
 int tile_n_of(const alg_proj_s &p) { return !use_tc(p) ? 64 : p.pair_kernel ? kTc2TileN : p.tile_n; }
 int elem_bytes(alg_dtype_t d) { return d == ALG_BF16 ? 2 : 4; }
 
+// Tile classes of a projection for tiles `tn` columns wide, sorted by cost = K length x tile width,
+// most expensive first (stable).
+alg_status_t build_classes(const alg_proj_s &p, int tn, DevTable &tab) {
+  const int q = p.q;
+  struct Item { long long cost; ClassRec rec; };
+  std::vector<Item> order;
+  for (int pr = 0; pr < q * q; ++pr) {
+    long long len = 0;
+    for (int k = 0; k < q; ++k)
+      if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
+    const int i = pr / q, j = pr % q, width = p.r[j];
+    for (int t0 = 0; t0 < width / tn; t0 += 4095) {  // n_tiles has 12 bits
+      const int nt = std::min(4095, width / tn - t0);
+      order.push_back({len * tn, ClassRec{(unsigned)i, (unsigned)j, (unsigned)tn, (unsigned)nt, p.tab.ro[j] + t0 * tn}});
+    }
+    if (width % tn)
+      order.push_back({len * (width % tn),
+                       ClassRec{(unsigned)i, (unsigned)j, (unsigned)(width % tn), 1u, p.tab.ro[j] + (width / tn) * tn}});
+  }
+  if ((int)order.size() > kMaxClasses) return ALG_ERR_INVALID_ARG;
+  std::stable_sort(order.begin(), order.end(), [](const Item &x, const Item &y) { return x.cost > y.cost; });
+  tab.n_classes = (int)order.size();
+  for (size_t e = 0; e < order.size(); ++e) tab.cls[e] = order[e].rec;
+  tab.n_pairs = q * q;
+  return ALG_OK;
+}
+
 // Kernel selection and the tile classes that follow from it.  Runs at handle creation and again
 // when an option that changes the selection is set.
 alg_status_t configure_kernels(alg_proj_s &p) {
@@ -113,29 +146,20 @@ alg_status_t configure_kernels(alg_proj_s &p) {
     p.pair_kernel = true;
   }
 
-  // tile classes sorted by cost = K length x tile width, most expensive first (stable)
-  {
-    const int tn = tile_n_of(p);
-    struct Item { long long cost; ClassRec rec; };
-    std::vector<Item> order;
-    for (int pr = 0; pr < q * q; ++pr) {
-      long long len = 0;
-      for (int k = 0; k < q; ++k)
-        if ((p.tab.keep[pr] >> k) & 1u) len += p.s[k];
-      const int i = pr / q, j = pr % q, width = p.r[j];
-      for (int t0 = 0; t0 < width / tn; t0 += 4095) {  // n_tiles has 12 bits
-        const int nt = std::min(4095, width / tn - t0);
-        order.push_back({len * tn, ClassRec{(unsigned)i, (unsigned)j, (unsigned)tn, (unsigned)nt, p.tab.ro[j] + t0 * tn}});
-      }
-      if (width % tn)
-        order.push_back({len * (width % tn),
-                         ClassRec{(unsigned)i, (unsigned)j, (unsigned)(width % tn), 1u, p.tab.ro[j] + (width / tn) * tn}});
-    }
-    if ((int)order.size() > kMaxClasses) return ALG_ERR_INVALID_ARG;
-    std::stable_sort(order.begin(), order.end(), [](const Item &x, const Item &y) { return x.cost > y.cost; });
-    p.tab.n_classes = (int)order.size();
-    for (size_t e = 0; e < order.size(); ++e) p.tab.cls[e] = order[e].rec;
-    p.tab.n_pairs = q * q;
+  alg_status_t bs = build_classes(p, tile_n_of(p), p.tab);
+  if (bs != ALG_OK) return bs;
+  // 256-row tiles: one-CTA kernel, 128-column tiles must divide every output group, and wider
+  // tiles (which reuse A as well) must not be available
+  p.tall_ok = p.tc_ok && !p.pair_kernel && all128 && !all256 && p.opt_tile_n == 0 && p.opt_kernel != 1;
+  if (p.opt_kernel == 3) {
+    if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
+    p.pair_kernel = false;
+    p.tall_ok = true;
+  }
+  if (p.tall_ok) {
+    p.tab_tall = p.tab;
+    bs = build_classes(p, 128, p.tab_tall);
+    if (bs != ALG_OK) return bs;
   }
 
   return ALG_OK;
@@ -203,6 +227,8 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   if (prop.major != 10) return ALG_ERR_UNSUPPORTED_SHAPE;  // sm_100a code only
   if (cudaMalloc(&p.d_tab, sizeof(DevTable)) != cudaSuccess) return ALG_ERR_CUDA;
   if (cudaMemcpy(p.d_tab, &p.tab, sizeof(DevTable), cudaMemcpyHostToDevice) != cudaSuccess) return ALG_ERR_CUDA;
+  if (cudaMalloc(&p.d_tab_tall, sizeof(DevTable)) != cudaSuccess) return ALG_ERR_CUDA;
+  if (cudaMemcpy(p.d_tab_tall, &p.tab_tall, sizeof(DevTable), cudaMemcpyHostToDevice) != cudaSuccess) return ALG_ERR_CUDA;
   if (shared_status) {
     p.d_status = shared_status;
     p.shared_status = true;
@@ -240,6 +266,8 @@ void free_proj(alg_proj_s &p) {
     sl = PlanSlot();
   }
   if (p.d_tab) cudaFree(p.d_tab);
+  if (p.d_tab_tall) cudaFree(p.d_tab_tall);
+  p.d_tab_tall = nullptr;
   if (p.d_status && !p.shared_status) cudaFree(p.d_status);
   p.d_tab = nullptr;
   p.d_status = nullptr;
@@ -273,6 +301,19 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
 
 alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG_ERR_CUDA; }
 
+// Tiling of one forward call on the tensor-core path.
+struct TcChoice {
+  int tile_m, tile_n;
+  const DevTable *tab;   // host copy with the tile classes of this tiling
+  const DevTable *d_tab;
+};
+// 256-row tiles pay when every row type fills several of them (a ragged last tile then wastes
+// little); with explicit types the rows per type are not known on the host: assume an even mix.
+TcChoice choose_tiling(const alg_proj_s &p, int64_t M) {
+  if (p.tall_ok && (p.opt_kernel == 3 || M / p.q >= 1024)) return {256, 128, &p.tab_tall, p.d_tab_tall};
+  return {tile_m_of(p), tile_n_of(p), &p.tab, p.d_tab};
+}
+
 // Host twin of the in-kernel tile enumeration for the cyclic schedule (equal buckets of M/q rows):
 // cost-sorted classes, m-tile major inside a class, boustrophedon assignment of tile indices to
 // workers.  The plans of the last few M are cached in device memory the handle owns.  A new plan is
@@ -282,7 +323,7 @@ alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG
 // plan for themselves, with the same result -- while `st` is being captured (a captured launch must
 // not depend on handle state that later calls rewrite), when every slot's last upload is still in
 // flight, or when the sequences do not fit.
-const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, int64_t M, cudaStream_t st) {
+const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, const TcChoice &tc, int64_t M, cudaStream_t st) {
   if (!p.opt_host_plan || p.pair_kernel || !p.plan[0].d) return nullptr;
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return nullptr;
@@ -301,11 +342,12 @@ const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, int64_t M, cudaStream_t st) {
     if (!slot || sl.last_use < slot->last_use) slot = &sl;
   }
   if (!slot) return nullptr;
-  const int q = p.q, nc = p.tab.n_classes, tile_m = tile_m_of(p), nw = p.n_workers, stride = p.plan_stride;
+  const DevTable &tab = *tc.tab;
+  const int q = p.q, nc = tab.n_classes, tile_m = tc.tile_m, nw = p.n_workers, stride = p.plan_stride;
   const int bucket = (int)(M / q);
   const int m_tiles = (bucket + tile_m - 1) / tile_m;
   std::vector<long long> prefix(nc + 1, 0);
-  for (int c = 0; c < nc; ++c) prefix[c + 1] = prefix[c] + (long long)m_tiles * p.tab.cls[c].n_tiles;
+  for (int c = 0; c < nc; ++c) prefix[c + 1] = prefix[c] + (long long)m_tiles * tab.cls[c].n_tiles;
   const long long total = prefix[nc];
   const long long all_rounds = (total + nw - 1) / nw;
   slot->M = M;
@@ -330,7 +372,7 @@ const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, int64_t M, cudaStream_t st) {
       if (pos < valid) {
         const long long idx = snake(pos, w);
         int c = (int)(std::upper_bound(prefix.begin(), prefix.end(), idx) - prefix.begin()) - 1;
-        const ClassRec &r = p.tab.cls[c];
+        const ClassRec &r = tab.cls[c];
         const int loc = (int)(idx - prefix[c]), ntl = (int)r.n_tiles, mt = loc / ntl, nt = loc - mt * ntl;
         rec.row0 = (int)r.i * bucket + mt * tile_m;
         rec.rows = std::min(tile_m, bucket - mt * tile_m) | (nkb[(int)r.i * q + (int)r.j] << 16);
@@ -357,17 +399,19 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
                       cudaEvent_t after_gather = nullptr, bool cyclic = false) {
   ProjArgs a;
-  a.tab = p.d_tab;
+  const TcChoice tc = choose_tiling(p, M);
+  const DevTable &tab = *tc.tab;
+  a.tab = tc.d_tab;
   a.offsets = cyclic ? nullptr : ((const WsHeader *)(ws + L.hdr))->offsets;
   a.cyclic_rows = cyclic ? (int)(M / p.q) : 0;
-  a.n_classes = p.tab.n_classes;
-  a.st.valid = p.q <= kParamQ && p.tab.n_classes <= 2 * kParamQ * kParamQ;
+  a.n_classes = tab.n_classes;
+  a.st.valid = p.q <= kParamQ && tab.n_classes <= 2 * kParamQ * kParamQ;
   if (a.st.valid) {
-    for (int e = 0; e <= p.q; ++e) a.st.so[e] = p.tab.so[e], a.st.ro[e] = p.tab.ro[e];
-    for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = p.tab.keep[e];
-    for (int e = 0; e < p.tab.n_classes; ++e) a.st.cls[e] = p.tab.cls[e];
+    for (int e = 0; e <= p.q; ++e) a.st.so[e] = tab.so[e], a.st.ro[e] = tab.ro[e];
+    for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = tab.keep[e];
+    for (int e = 0; e < tab.n_classes; ++e) a.st.cls[e] = tab.cls[e];
   }
-  a.geom.tile_m = tile_m_of(p);
+  a.geom.tile_m = tc.tile_m;
   a.geom.tile_m_log2 = a.geom.tile_m == 256 ? 8 : a.geom.tile_m == 128 ? 7 : 6;
   a.q = p.q;
   a.perm = (y_bucketed || cyclic) ? nullptr : (const int *)(ws + L.perm);  // cyclic outputs are addressed by arithmetic
@@ -385,12 +429,13 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.b_3d = 0;
+  a.a_box_256 = 0;
   a.y_staged = 0;
   a.plan = nullptr;
   a.plan_stride = a.plan_rounds = a.plan_tag = 0;
   a.wait_limit = p.wait_limit;
   if (cyclic) {
-    if (const PlanSlot *sl = prepare_cyclic_plan(p, M, st)) {
+    if (const PlanSlot *sl = prepare_cyclic_plan(p, tc, M, st)) {
       a.plan = sl->d;
       a.plan_stride = p.plan_stride;
       a.plan_rounds = sl->rounds;
@@ -410,7 +455,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     if (after_gather) cudaEventRecord(after_gather, st);
     a.in_perm = nullptr;
     if (p.pair_kernel) return cuda_status(launch_proj_tc2(a, p.num_sms, st));
-    return cuda_status(launch_proj_tc(a, p.tile_n, p.n_workers, st));
+    return cuda_status(launch_proj_tc(a, tc.tile_n, p.n_workers, st));
   }
   if (after_gather) cudaEventRecord(after_gather, st);
   a.X = X;
@@ -487,7 +532,7 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
   switch (option) {
     case ALG_OPT_GEMM_KERNEL:
     case ALG_OPT_TILE_N: {
-      if (option == ALG_OPT_GEMM_KERNEL && (value < 0 || value > 2)) return ALG_ERR_INVALID_ARG;
+      if (option == ALG_OPT_GEMM_KERNEL && (value < 0 || value > 3)) return ALG_ERR_INVALID_ARG;
       if (option == ALG_OPT_TILE_N && value != 0 && value != 128 && value != 192 && value != 256) return ALG_ERR_INVALID_ARG;
       const int old_kernel = p.opt_kernel, old_tile = p.opt_tile_n;
       (option == ALG_OPT_GEMM_KERNEL ? p.opt_kernel : p.opt_tile_n) = (int)value;
@@ -504,7 +549,8 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
       if (cudaGetDevice(&dev) != cudaSuccess || dev != p.device) return ALG_ERR_INVALID_ARG;
       // the device copy of the table may still be read by kernels in flight
       if (cudaDeviceSynchronize() != cudaSuccess) return ALG_ERR_CUDA;
-      return cuda_status(cudaMemcpy(p.d_tab, &p.tab, sizeof(DevTable), cudaMemcpyHostToDevice));
+      if (cudaMemcpy(p.d_tab, &p.tab, sizeof(DevTable), cudaMemcpyHostToDevice) != cudaSuccess) return ALG_ERR_CUDA;
+      return cuda_status(cudaMemcpy(p.d_tab_tall, &p.tab_tall, sizeof(DevTable), cudaMemcpyHostToDevice));
     }
     case ALG_OPT_SMALL_M_KERNEL: p.opt_small_m = value != 0; return ALG_OK;
     case ALG_OPT_HOST_PLAN: p.opt_host_plan = value != 0; return ALG_OK;

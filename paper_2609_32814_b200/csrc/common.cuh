@@ -125,6 +125,7 @@ struct ProjArgs {
   int a_cyclic_rows;
   int out_cyclic_rows;
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
+  int a_box_256;          // A tensor map carries 256-row boxes (one-CTA kernel with 256-row tiles)
   int y_staged;           // 1: the epilogue transposes bf16 results through shared memory for coalesced stores
   // Cyclic schedule: the tile sequences of all workers depend only on (handle, M) and are planned
   // once on the host; worker w reads plan[1 + w * plan_stride .. + plan_rounds) (the last record of

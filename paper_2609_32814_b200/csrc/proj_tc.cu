@@ -75,27 +75,38 @@ constexpr int kEpiWarps = ALGPROJ_EPI_WARPS;
 constexpr int kProducerWarpB = 2 + kEpiWarps;   // second TMA producer, after the epilogue warps
 constexpr int kThreads = 32 * (3 + kEpiWarps);
 
-template <int TILE_N>
+// TILE_M = 128: one accumulator of 128 rows x TILE_N columns per tile.
+// TILE_M = 256: two accumulators (rows 0..127 and 128..255) side by side in tensor memory; every
+// 64-deep B block is fetched once and used by two M = 128 MMAs, which cuts the operand bytes per
+// multiply-accumulate by a quarter against a 128 x 192 tile -- the layout for projections with a
+// long reduction and narrow output groups (TILE_N = 128 only, so that two tiles still fit the
+// 512 columns and the epilogue of one tile overlaps the main loop of the next).
+template <int TILE_N, int TILE_M>
 struct Cfg {
-  static constexpr int kABytes = kTcTileM * kTcBlockK * 2;      // 16 KB
+  static constexpr int kHalves = TILE_M / 128;                  // accumulators (MMAs per K step) of a tile
+  static constexpr int kABytes = TILE_M * kTcBlockK * 2;        // 16 KB per 128 rows
   static constexpr int kBChunkBytes = kTcBlockK * 64 * 2;       // one 64(k) x 64(n) box: 8 KB
   static constexpr int kBBytes = kBChunkBytes * (TILE_N / 64);
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
-  static constexpr int kAccStride = TILE_N <= 128 ? 128 : 256;   // TMEM columns between the two accumulators
+  static constexpr int kAccStride = TILE_N * kHalves <= 128 ? 128 : 256;   // TMEM columns between the two tile buffers
   static constexpr int kTmemCols = 2 * kAccStride;
   static constexpr int kFixedSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + kSeqCap * 16 + 16 + 1024;  // + tile map
   static constexpr int kStoreBufBytes = 32 * 64;                  // per epilogue warp: 32 rows x 32 bf16 columns
-  static constexpr int kHalf = TILE_N / (kEpiWarps / 4);          // columns per epilogue warp
+  // an epilogue warp takes 32 rows x kHalf columns: half of the columns of the one accumulator, or
+  // all columns of one of the two accumulators
+  static constexpr int kHalf = TILE_N * kHalves / (kEpiWarps / 4);
   // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N, M=128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                     ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
+                                     ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  static_assert(TILE_M == 128 || (TILE_M == 256 && TILE_N == 128), "256-row tiles are 128 columns wide");
+  static_assert(kHalves == 1 || kEpiWarps == 8, "two accumulators need one epilogue warp group each");
 };
 
-template <int TILE_N>
+template <int TILE_N, int TILE_M>
 __global__ void __launch_bounds__(kThreads, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
-  using C = Cfg<TILE_N>;
+  using C = Cfg<TILE_N, TILE_M>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   // optional staging buffers of the epilogue warps sit between the stages and the control block
@@ -107,7 +118,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const DevTable *__restrict__ tab = a.tab;
   const int q = a.q;
   ALG_TRACE_VARS;
-  ALG_TRACE_CTA(0);
+  ALG_TRACE_CTA(0, a.act ? 0 : 1);
 
   if (threadIdx.x == 0) ALG_TRACE(0, 20);
   if (warp == 0) {  // one barrier per lane
@@ -263,11 +274,15 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         if (elect_one()) {
-          // A: 16 k-elements = 32 bytes inside the swizzle atom; B: 16 k-rows = two 8-row groups
-          tc_mma_bf16(d_tmem, da, db, C::kIdesc, kb ? 1u : 0u);
+          // A: 16 k-elements = 32 bytes inside the swizzle atom; B: 16 k-rows = two 8-row groups;
+          // the second 128 rows of a 256-row tile sit 16 KB further in the stage and accumulate
+          // TILE_N columns further in tensor memory
 #pragma unroll
-          for (int kk = 1; kk < kTcBlockK / 16; ++kk)
-            tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), C::kIdesc, 1u);
+          for (int kk = 0; kk < kTcBlockK / 16; ++kk)
+#pragma unroll
+            for (int h = 0; h < C::kHalves; ++h)
+              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * 1024), db + (uint64_t)(kk * 128),
+                          C::kIdesc, (kb | kk) ? 1u : 0u);
           tc_commit(empty0 + 8u * (uint32_t)stage);
         }
         __syncwarp();
@@ -290,7 +305,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
     while (rec.row0 >= 0) {
       ++round;
-      const int r = quad * 32 + lane;
+      const int r = (C::kHalves == 2 ? half * 128 : 0) + quad * 32 + lane;   // row of the tile this lane holds
       int64_t out_row = -1;
       const int tile_rows = rec.rows & 0xFFFF;
       if (r < tile_rows) {
@@ -309,7 +324,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after();
       const uint32_t taddr =
           tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * C::kAccStride + half * C::kHalf);
-      const int col_base = rec.n0 + half * C::kHalf;
+      const int col_base = rec.n0 + (C::kHalves == 2 ? 0 : half * C::kHalf);
       // bf16 outputs are transposed through a 2 KB staging buffer per warp: every lane writes its
       // own row segment (64 bytes, 16-byte pieces XOR-swizzled so that the writes and the reads
       // below are bank-conflict free), then four lanes together store one row segment, so one
@@ -392,7 +407,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
-  ALG_TRACE_CTA(1);
+  ALG_TRACE_CTA(1, a.act ? 0 : 1);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
@@ -402,12 +417,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
-template <int TILE_N>
+template <int TILE_N, int TILE_M>
 cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
-  using C = Cfg<TILE_N>;
+  using C = Cfg<TILE_N, TILE_M>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -436,7 +451,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M>, tmA, tmB, b);
   count_launch(1);
   return e;
 }
@@ -490,11 +505,12 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
 }
 
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a) {
+  const uint32_t box_rows = a.geom.tile_m == 256 && a.a_box_256 ? 256u : 128u;
   if (!a.a_cyclic_rows)
-    return make_map_2d(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, kTcTileM);
+    return make_map_2d(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, box_rows);
   cuuint64_t dims[3] = {(cuuint64_t)a.K, (cuuint64_t)a.q, (cuuint64_t)a.a_cyclic_rows};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldx * 2, (cuuint64_t)a.ldx * 2 * (cuuint64_t)a.q};
-  cuuint32_t box[3] = {kTcBlockK, 1, kTcTileM};
+  cuuint32_t box[3] = {kTcBlockK, 1, box_rows};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -518,9 +534,15 @@ cudaError_t tc_init() {
 cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st) {
   cudaError_t e = tc_init();
   if (e != cudaSuccess) return e;
-  if (tile_n == 256) return launch_t<256>(a, num_sms, st);
-  if (tile_n == 192) return launch_t<192>(a, num_sms, st);
-  if (tile_n == 128) return launch_t<128>(a, num_sms, st);
+  if (a.geom.tile_m == 256) {
+    if (tile_n != 128) return cudaErrorInvalidValue;
+    ProjArgs b = a;
+    b.a_box_256 = 1;   // one box brings all 256 rows of a stage
+    return launch_t<128, 256>(b, num_sms, st);
+  }
+  if (tile_n == 256) return launch_t<256, 128>(a, num_sms, st);
+  if (tile_n == 192) return launch_t<192, 128>(a, num_sms, st);
+  if (tile_n == 128) return launch_t<128, 128>(a, num_sms, st);
   return cudaErrorInvalidValue;
 }
 

@@ -146,7 +146,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int q = tab_q;
   const uint32_t rank = cluster_ctarank();          // 0 = leader
   ALG_TRACE_VARS;
-  ALG_TRACE_CTA(0);
+  ALG_TRACE_CTA(0, a.act ? 0 : 1);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -356,7 +356,7 @@ proj_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // neither CTA leaves while its peer may still signal or read its shared memory
-  ALG_TRACE_CTA(1);
+  ALG_TRACE_CTA(1, a.act ? 0 : 1);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)

@@ -5,7 +5,8 @@
 // A traced build gives every translation unit that says ALG_TRACE_DEFINE(name) a buffer pointer
 // in device memory and an exported setter  alg_trace_set_<name>(void *device_buffer, int cap):
 // the buffer holds [slot][cap] int64 records (clock64 << 8 | tag), slot = CTA * 3 + role for the
-// first eight CTAs, followed by per-CTA {globaltimer, clock64} pairs at entry and exit.
+// first eight CTAs, followed by per-CTA {globaltimer, clock64} pairs at entry and exit (two sets of
+// 256 CTAs x 4 slots), followed at slot 24 * cap + 2048 by an append-only log.
 #pragma once
 
 #ifdef ALGPROJ_TRACE
@@ -26,14 +27,15 @@
     if (alg_trace_buf && blockIdx.x < 8 && tr_n < alg_trace_cap)                                    \
       alg_trace_buf[((size_t)blockIdx.x * 3 + (role)) * alg_trace_cap + tr_n++] = (clock64() << 8) | (tag); \
   } while (0)
-// whole-CTA window: which = 0 at entry, 1 at exit
-#define ALG_TRACE_CTA(which)                                                                        \
+// whole-CTA window: which = 0 at entry, 1 at exit; `set` (0 or 1) keeps two kernels of a step apart
+#define ALG_TRACE_CTA(which, set)                                                                   \
   do {                                                                                              \
     if (alg_trace_buf && threadIdx.x == 0) {                                                        \
       unsigned long long gt_;                                                                       \
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_));                                       \
-      alg_trace_buf[(size_t)24 * alg_trace_cap + blockIdx.x * 4 + (which)] = (long long)gt_;        \
-      alg_trace_buf[(size_t)24 * alg_trace_cap + blockIdx.x * 4 + 2 + (which)] = clock64();         \
+      long long *w_ = alg_trace_buf + (size_t)24 * alg_trace_cap + (set) * 1024 + blockIdx.x * 4;   \
+      w_[(which)] = (long long)gt_;                                                                 \
+      w_[2 + (which)] = clock64();                                                                  \
     }                                                                                               \
   } while (0)
 
@@ -66,8 +68,8 @@
 #define ALG_TRACE(role, tag) \
   do {                       \
   } while (0)
-#define ALG_TRACE_CTA(which) \
-  do {                       \
+#define ALG_TRACE_CTA(which, set) \
+  do {                            \
   } while (0)
 
 #endif

@@ -133,6 +133,49 @@ def test_pair_kernel_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
     assert torch.equal(Y, Y1)
 
 
+# ---- one-CTA kernel with 256-row tiles (two accumulators per tile) -------------------------------
+
+@pytest.mark.parametrize("q,M,s_w,r_w,schedule", [
+    (1, 700, 512, 384, "explicit"),    # ragged last 256-row tile, three column tiles
+    (2, 300, 128, 128, "explicit"),    # buckets smaller than one tile
+    (2, 1337, 256, 384, "explicit"),   # several tiles per type, both endpoint products
+    (3, 515, 64, 128, "explicit"),
+    (2, 1026, 128, 384, "cyclic"),     # type-strided A view with 256-row boxes, arithmetic row scatter
+    (4, 4096, 64, 128, "cyclic"),      # 1024 rows per type: the library picks this tiling by itself
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_tall_tiles_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else None
+    wl = _tc_workload(q, M, s_w, r_w, types=types, seed=q * 37 + M % 13)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    if M < 4096:
+        proj.set_option("gemm_kernel", 3)
+    t = None if schedule == "cyclic" else H.dev_types(wl.types)
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype)
+    assert proj.last_status() == 0
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+    proj.set_option("gemm_kernel", 1)      # 128-row tiles on the same handle: same bits
+    assert torch.equal(Y, proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype))
+
+
+def test_tall_tiles_bias_gelu_normal_data():
+    wl = _tc_workload(2, 2500, 384, 384, integer=False, seed=19)
+    bias = synth.bf16_round(synth.normal(21, (wl.F,), 0.5))
+    for act, out_dtype in (("gelu", torch.float32), ("gelu", torch.bfloat16), (None, torch.bfloat16)):
+        proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")   # 1250 rows per type: 256-row tiles by default
+        Y = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16"),
+                         bias=H.to_dev(bias, "bf16"), act=act, out_dtype=out_dtype)
+        assert proj.last_status() == 0
+        ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, bias=bias)
+        if act:
+            ref = oracle.gelu_array(ref)
+        H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"256-row tiles act={act}")
+
+
 def test_pair_kernel_bias_gelu_normal_data_and_refusal():
     wl = _tc_workload(2, 900, 384, 384, integer=False, seed=13)
     bias = synth.bf16_round(synth.normal(15, (wl.F,), 0.5))
