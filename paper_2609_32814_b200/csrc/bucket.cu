@@ -1,8 +1,9 @@
-// Row-type bucketing (Algorithm 1, line "I_i <- {b : tau(p_b) = i}") as a stable permutation.
-// No host synchronisation anywhere: the row counts per type never leave the device (the GEMM
-// kernels turn the bucket offsets into their tile enumeration themselves).
+// Row-type bucketing: the index sets I_i of Algorithm 1 (all rows of type i), built as one stable
+// permutation.  No host synchronisation anywhere: the row counts per type never leave the device
+// (the GEMM kernels turn the bucket offsets into their tile enumeration themselves).
 //
-//   M <= 65536: one kernel; every CTA counts the rows before its chunk and overall by itself.
+//   M <= 65536: one kernel of M/1024 CTAs: each histograms its own 1024 rows, publishes the counts,
+//               meets the others at a counter (bounded wait) and places its rows.
 //   larger M:
 //   kernel 1 (count):   per-chunk histograms (at most 256 chunks).
 //   kernel 2 (scatter): each CTA scans the histograms for the bucket offsets and its own bases,
@@ -111,112 +112,91 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
     for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
 }
 
-// One-kernel variant for M <= 65536: every CTA (1024 threads, 1024 rows) reads all row types itself
-// (at most 256 KB from L2) and counts, per type, the rows before its own chunk and the rows overall;
-// no histogram array, no second launch.  A warp takes 512 rows at a time with sixteen independent
-// loads per lane in flight; the counts live in registers: lane t of every warp owns type t
-// (pseudo-type q = out of range), fed by one warp ballot per type and 32 rows.
+// One-pass variant for M <= 65536 (at most 64 CTAs of 1024 threads, one row per thread): every row
+// type is read exactly once.  A CTA ranks its rows inside their type (warp match + per-warp counts),
+// publishes its per-type counts, arrives on a counter and waits (bounded) until every CTA has;
+// then it sums the counts of all chunks (bucket offsets) and of the chunks before it (its base)
+// and writes perm.  All CTAs are resident together: the grid is far smaller than the machine, and
+// the kernel launched after it starts only once every CTA of this one has.  The last CTA past the
+// wait clears the counter for the next launch.
 constexpr int kFusedThreads = 1024;
-__global__ void __launch_bounds__(kFusedThreads) bucket_fused_kernel(const BucketArgs a) {
-  __shared__ int s_before[32][kMaxQ + 1], s_all[32][kMaxQ + 1];
-  __shared__ int s_wcnt[32][kMaxQ + 1];
+__global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const BucketArgs a) {
+  __shared__ int s_wcnt[32][kMaxQ + 1];   // rows of type t in warp w; then exclusive prefix over the warps
   __shared__ int s_base[kMaxQ + 1], s_offset[kMaxQ + 2];
+  __shared__ int s_go;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
+  const int n_chunks = gridDim.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the row types may come from the previous kernel
-  const int row_begin = blockIdx.x * kFusedThreads;
-  int before = 0, all = 0;
-  const int n_super = (a.M + 511) >> 9;
-  if (nt <= 8) {
-    // q + 1 <= 8 kinds: every lane keeps its own histogram packed in two 64-bit words (16 bits per
-    // kind; a lane sees at most 16 rows per pass and a warp total stays below 2^16), so a pass
-    // costs two instructions per row and one shuffle reduction instead of (q+1) ballots per row
-    unsigned long long all_lo = 0, all_hi = 0, bef_lo = 0, bef_hi = 0;
-    for (int sb = warp; sb < n_super; sb += 32) {
-      int tt[16];
-#pragma unroll
-      for (int u = 0; u < 16; ++u) {
-        const int row = sb * 512 + u * 32 + lane;
-        tt[u] = row < a.M ? row_type(a, row) : -1;
-      }
-      unsigned long long lo = 0, hi = 0;
-#pragma unroll
-      for (int u = 0; u < 16; ++u) {
-        const unsigned long long one = tt[u] < 0 ? 0ull : 1ull << ((tt[u] & 3) * 16);
-        if (tt[u] < 4) lo += one; else hi += one;
-      }
-      all_lo += lo, all_hi += hi;
-      if (sb * 512 < row_begin) bef_lo += lo, bef_hi += hi;
-      if (((sb / 32) & 63) == 63) {  // fold into the 32-bit counters before a 16-bit field can overflow
-        for (int d = 16; d > 0; d >>= 1) {
-          all_lo += __shfl_xor_sync(0xffffffffu, all_lo, d), all_hi += __shfl_xor_sync(0xffffffffu, all_hi, d);
-          bef_lo += __shfl_xor_sync(0xffffffffu, bef_lo, d), bef_hi += __shfl_xor_sync(0xffffffffu, bef_hi, d);
-        }
-        if (lane < nt) {
-          all += (int)(((lane < 4 ? all_lo : all_hi) >> ((lane & 3) * 16)) & 0xFFFF);
-          before += (int)(((lane < 4 ? bef_lo : bef_hi) >> ((lane & 3) * 16)) & 0xFFFF);
-        }
-        all_lo = all_hi = bef_lo = bef_hi = 0;
-      }
-    }
-    for (int d = 16; d > 0; d >>= 1) {
-      all_lo += __shfl_xor_sync(0xffffffffu, all_lo, d), all_hi += __shfl_xor_sync(0xffffffffu, all_hi, d);
-      bef_lo += __shfl_xor_sync(0xffffffffu, bef_lo, d), bef_hi += __shfl_xor_sync(0xffffffffu, bef_hi, d);
-    }
-    if (lane < nt) {
-      all += (int)(((lane < 4 ? all_lo : all_hi) >> ((lane & 3) * 16)) & 0xFFFF);
-      before += (int)(((lane < 4 ? bef_lo : bef_hi) >> ((lane & 3) * 16)) & 0xFFFF);
-    }
-  } else {
-    for (int sb = warp; sb < n_super; sb += 32) {
-      int tt[16];
-#pragma unroll
-      for (int u = 0; u < 16; ++u) {
-        const int row = sb * 512 + u * 32 + lane;
-        tt[u] = row < a.M ? row_type(a, row) : -1;
-      }
-      int mine = 0;
-#pragma unroll
-      for (int u = 0; u < 16; ++u)
-        for (int k = 0; k < nt; ++k) {
-          const unsigned b = __ballot_sync(0xffffffffu, tt[u] == k);
-          if (lane == k) mine += __popc(b);
-        }
-      all += mine;
-      if (sb * 512 < row_begin) before += mine;
-    }
-  }
-  if (lane < nt) s_before[warp][lane] = before, s_all[warp][lane] = all;
   for (int e = tid; e < 32 * (kMaxQ + 1); e += kFusedThreads) (&s_wcnt[0][0])[e] = 0;
-  __syncthreads();
-  if (tid < nt) {
-    int bsum = 0, asum = 0;
-    for (int w = 0; w < 32; ++w) bsum += s_before[w][tid], asum += s_all[w][tid];
-    s_base[tid] = bsum;
-    s_all[0][tid] = asum;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int run = 0;
-    for (int t = 0; t < nt; ++t) {
-      s_offset[t] = run;
-      run += s_all[0][t];
-    }
-    s_offset[nt] = run;  // == M
-  }
-  const int row = row_begin + tid;
+  const int row = blockIdx.x * kFusedThreads + tid;
   const bool live = row < a.M;
   const int t = live ? row_type(a, row) : -1 - lane;  // dead lanes never match each other
   if (live && t == a.q) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
   const unsigned peers = __match_any_sync(0xffffffffu, t);
   const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+  __syncthreads();
   if (live && rank_in_warp == 0) s_wcnt[warp][t] = __popc(peers);
   __syncthreads();
+  if (tid < nt) {   // exclusive prefix over the warps; the total goes to global memory
+    int run = 0;
+    for (int w = 0; w < 32; ++w) {
+      const int v = s_wcnt[w][tid];
+      s_wcnt[w][tid] = run;
+      run += v;
+    }
+    a.chunk_counts[blockIdx.x * nt + tid] = run;
+    __threadfence();
+  }
+  __syncthreads();
+  if (tid == 0) {
+    atomicAdd(a.sync, 1u);
+    const long long t0 = clock64();
+    int go = 1;
+    unsigned v;
+    do {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.sync) : "memory");
+      if (v < (unsigned)n_chunks && clock64() - t0 > a.wait_limit) {
+        atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+        go = 0;
+        break;
+      }
+    } while (v < (unsigned)n_chunks);
+    s_go = go;
+  }
+  __syncthreads();
+  if (!s_go) return;
+  if (tid == 0 && atomicAdd(a.sync + 1, 1u) == (unsigned)(n_chunks - 1)) a.sync[0] = 0u, a.sync[1] = 0u;
+  if (warp < 2) {   // lanes over the chunks (at most 64), one type after the other
+    for (int ty = warp; ty < nt; ty += 2) {
+      int before = 0, total = 0;
+      for (int c = lane; c < n_chunks; c += 32) {
+        const int v = __ldcg(a.chunk_counts + c * nt + ty);
+        total += v;
+        if (c < (int)blockIdx.x) before += v;
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, d);
+        total += __shfl_xor_sync(0xffffffffu, total, d);
+      }
+      if (lane == 0) s_base[ty] = before, s_offset[ty] = total;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {   // bucket offsets: exclusive prefix of the totals over the types
+    int run = 0;
+    for (int ty = 0; ty < nt; ++ty) {
+      const int v = s_offset[ty];
+      s_offset[ty] = run;
+      run += v;
+    }
+    s_offset[nt] = run;  // == M
+  }
+  __syncthreads();
   if (live) {
-    int bw = 0;
-    for (int w = 0; w < warp; ++w) bw += s_wcnt[w][t];
-    a.perm[s_offset[t] + s_base[t] + bw + rank_in_warp] = row;
+    a.perm[s_offset[t] + s_base[t] + s_wcnt[warp][t] + rank_in_warp] = row;
     if (t == a.q && a.Y) {  // out-of-range type: the row's output is defined to be zero
       char *y = (char *)a.Y + (size_t)row * a.ldy * a.y_elem_bytes;
       for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
@@ -269,9 +249,9 @@ cudaError_t launch_pdl(void (*kernel)(Args...), int grid, int block, cudaStream_
 }  // namespace
 
 cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
-  if (a.M <= 65536) {  // one kernel: every CTA counts for itself
+  if (a.M <= 65536 && a.sync) {  // one kernel, every row type read once
     count_launch(1);
-    return launch_pdl(bucket_fused_kernel, ceil_div(a.M, kFusedThreads), kFusedThreads, st, a);
+    return launch_pdl(bucket_onepass_kernel, ceil_div(a.M, kFusedThreads), kFusedThreads, st, a);
   }
   const int n_chunks = ceil_div(a.M, a.chunk_rows);
   bucket_count_kernel<<<n_chunks, 256, 0, st>>>(a);

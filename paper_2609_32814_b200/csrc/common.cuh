@@ -72,6 +72,8 @@ struct BucketArgs {
   int *chunk_counts;     // [n_chunks][q+1]
   int *perm;             // [M] bucketed position -> original row
   int *status;           // device status word of the handle
+  unsigned int *sync;    // two counters of the handle (zero between launches) for the one-kernel variant
+  long long wait_limit;  // bound of its wait, in SM clock cycles
   // rows with an out-of-range type get their output row zero-filled here
   void *Y;
   int64_t ldy;
