@@ -59,6 +59,10 @@ def _load():
         lib.star_gelu.argtypes = [ctypes.c_double]
         lib.star_ffn.argtypes = [f64p, i32p, i64, f64p, f64p, f64p, f64p, f64p, f64p,
                                  ctypes.c_int, i32p, i32p, u8p]
+        lib.star_silu.restype = ctypes.c_double
+        lib.star_silu.argtypes = [ctypes.c_double]
+        lib.star_ffn_swiglu.argtypes = [f64p, i32p, i64, f64p, f64p, f64p, f64p, f64p, f64p, f64p,
+                                        ctypes.c_int, i32p, i32p, u8p]
         _lib = lib
     return _lib
 
@@ -230,4 +234,29 @@ def ffn(X, types, W_up, W_down, dw, fw, keep=None, b_up=None, b_down=None, retur
     f64, i32, u8 = ctypes.c_double, ctypes.c_int32, ctypes.c_uint8
     _check(lib.star_ffn(_p(X, f64), _p(types, i32), M, _p(W_up, f64), _p(bu, f64), _p(W_down, f64),
                         _p(bd, f64), _p(H, f64), _p(Y, f64), q, _p(dw, i32), _p(fw, i32), _p(keep, u8)))
+    return (Y, H) if return_hidden else Y
+
+
+def silu(g: float) -> float:
+    return float(_load().star_silu(float(g)))
+
+
+def ffn_swiglu(X, types, W_gate, W_up, W_down, dw, fw, keep=None, return_hidden=False):
+    """Y = (silu(X *_q W_gate) .* (X *_q W_up)) *_q W_down, hidden state kept in fp64, no biases."""
+    lib = _load()
+    X, W_gate, W_up, W_down = _f64(X), _f64(W_gate), _f64(W_up), _f64(W_down)
+    types, dw, fw = _i32(types), _i32(dw), _i32(fw)
+    q = len(dw)
+    if keep is None:
+        keep = support(q, "qq")
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    M, D = X.shape
+    F = int(fw.sum())
+    if int(dw.sum()) != D or W_gate.shape != (D, F) or W_up.shape != (D, F) or W_down.shape != (F, D) or len(types) != M:
+        raise OracleError("shape mismatch")
+    G, U, H = (np.empty((M, F), dtype=np.float64) for _ in range(3))
+    Y = np.empty((M, D), dtype=np.float64)
+    f64, i32, u8 = ctypes.c_double, ctypes.c_int32, ctypes.c_uint8
+    _check(lib.star_ffn_swiglu(_p(X, f64), _p(types, i32), M, _p(W_gate, f64), _p(W_up, f64), _p(W_down, f64),
+                               _p(G, f64), _p(U, f64), _p(H, f64), _p(Y, f64), q, _p(dw, i32), _p(fw, i32), _p(keep, u8)))
     return (Y, H) if return_hidden else Y

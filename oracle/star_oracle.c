@@ -15,9 +15,11 @@
  * Pins (all in tests/test_oracle_pins.py): hand-derived scalar examples, the six-product
  * rule term by term, dense-minus-removed brute force, associativity/unit/edge-ideal on
  * integer block arrays, the 2q^2-q count and the MAC formulas, q=1 / dense table against
- * numpy.matmul, GELU against closed-form values.
+ * numpy.matmul, GELU and SiLU against closed-form values, the gated FFN against an
+ * independent numpy composition.
  * Parity unpinned by the paper: the FFN-level choices (erf-GELU, bias added before the
- * activation) come from the benchmark specification, not from a printed value.
+ * activation) come from the benchmark specification, not from a printed value; SwiGLU is
+ * named by the paper without its formula (the standard one is taken).
  *
  * Build: gcc -O2 -fopenmp -shared -fPIC star_oracle.c -o libstar_oracle.so -lm
  */
@@ -301,4 +303,30 @@ int star_ffn(const double *X, const int32_t *types, int64_t M, const double *W_u
 #pragma omp parallel for schedule(static)
   for (int64_t e = 0; e < M * F; ++e) H[e] = star_gelu(H[e]);
   return star_proj_rows(H, F, types, M, W_down, D, b_down, Y, D, q, fw, dw, keep);
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Gated FFN (SwiGLU), the FFN of the paper's pretraining pilot (Section "Projection Shapes":
+ * two D x F weights and one F x D weight, the same row law on each; Appendix "Experimental
+ * Details": bias-free SwiGLU):
+ *     G = X * W_gate,   U = X * W_up,   H = silu(G) .* U,   Y = H * W_down,
+ * silu(g) = g / (1 + exp(-g)), all three projections under the same support and row types,
+ * H kept in fp64 (never rounded).  G, U (M x F each) and H are caller-provided scratch.
+ * Parity unpinned by the paper: it names SwiGLU without writing the formula; the standard
+ * definition is taken.
+ * ------------------------------------------------------------------------------------- */
+double star_silu(double g) { return g / (1.0 + exp(-g)); }
+
+int star_ffn_swiglu(const double *X, const int32_t *types, int64_t M, const double *W_gate,
+                    const double *W_up, const double *W_down, double *G, double *U, double *H,
+                    double *Y, int q, const int32_t *dw, const int32_t *fw, const uint8_t *keep) {
+  int64_t D = 0, F = 0;
+  for (int g = 0; g < q; ++g) { D += dw[g]; F += fw[g]; }
+  int rc = star_proj_rows(X, D, types, M, W_gate, F, NULL, G, F, q, dw, fw, keep);
+  if (rc) return rc;
+  rc = star_proj_rows(X, D, types, M, W_up, F, NULL, U, F, q, dw, fw, keep);
+  if (rc) return rc;
+#pragma omp parallel for schedule(static)
+  for (int64_t e = 0; e < M * F; ++e) H[e] = star_silu(G[e]) * U[e];
+  return star_proj_rows(H, F, types, M, W_down, D, NULL, Y, D, q, fw, dw, keep);
 }

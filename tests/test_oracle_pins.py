@@ -345,6 +345,60 @@ def test_ffn_composes_projections():
     np.testing.assert_allclose(Y, star2(Hn, Wd, fw, dw, bd), rtol=1e-12, atol=1e-12)
 
 
+def test_silu_closed_form(golden):
+    import math
+    for z, want in golden["silu"]["points"]:
+        assert abs(oracle.silu(z) - want) < 1e-12
+    for z in np.linspace(-8, 8, 33):
+        assert abs(oracle.silu(z) - z * 0.5 * (1.0 + math.tanh(0.5 * z))) < 1e-13      # z * sigmoid(z), another form
+
+
+def test_gated_ffn_composes_three_projections():
+    """SwiGLU FFN against an independent numpy composition (q = 2: dense minus the removed product;
+    q = 4 tensor-square law: per-row sums written from the bit rule)."""
+    rng = np.random.default_rng(7)
+    q, dw, fw = 2, [3, 2], [4, 5]
+    M = 9
+    X = rng.standard_normal((M, 5))
+    Wg, Wu = rng.standard_normal((5, 9)), rng.standard_normal((5, 9))
+    Wd = rng.standard_normal((9, 5))
+    types = rng.integers(0, q, size=M)
+
+    def star2(Xm, Wm, s, r):
+        so, ro = _offsets(s), _offsets(r)
+        out = Xm @ Wm
+        for b, t in enumerate(types):
+            o = 1 - t
+            out[b, ro[t]:ro[t + 1]] -= Xm[b, so[o]:so[o + 1]] @ Wm[so[o]:so[o + 1], ro[t]:ro[t + 1]]
+        return out
+    G, U = star2(X, Wg, dw, fw), star2(X, Wu, dw, fw)
+    Hn = G / (1.0 + np.exp(-G)) * U
+    Y, Hh = oracle.ffn_swiglu(X, types, Wg, Wu, Wd, dw, fw, return_hidden=True)
+    np.testing.assert_allclose(Hh, Hn, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(Y, star2(Hn, Wd, fw, dw), rtol=1e-12, atol=1e-12)
+    # tensor-square law, q = 4: group beta enters output group delta of a type-alpha row iff every
+    # bit of beta equals that bit of alpha or of delta
+    q, dw, fw = 4, [2, 1, 2, 1], [1, 2, 1, 2]
+    X = rng.standard_normal((6, 6))
+    Wg, Wu, Wd = rng.standard_normal((6, 6)), rng.standard_normal((6, 6)), rng.standard_normal((6, 6))
+    types = np.array([0, 1, 2, 3, 2, 1])
+    keep = oracle.support(4, "q2pow")
+
+    def star_pow(Xm, Wm, s, r):
+        so, ro = _offsets(s), _offsets(r)
+        out = np.zeros((Xm.shape[0], ro[-1]))
+        for b, al in enumerate(types):
+            for de in range(4):
+                for be in range(4):
+                    if all(((be >> k) & 1) in (((al >> k) & 1), ((de >> k) & 1)) for k in range(2)):
+                        out[b, ro[de]:ro[de + 1]] += Xm[b, so[be]:so[be + 1]] @ Wm[so[be]:so[be + 1], ro[de]:ro[de + 1]]
+        return out
+    G, U = star_pow(X, Wg, dw, fw), star_pow(X, Wu, dw, fw)
+    Hn = G / (1.0 + np.exp(-G)) * U
+    np.testing.assert_allclose(oracle.ffn_swiglu(X, types, Wg, Wu, Wd, dw, fw, keep=keep), star_pow(Hn, Wd, fw, dw),
+                               rtol=1e-12, atol=1e-12)
+
+
 def test_bad_type_rejected():
     with pytest.raises(oracle.OracleError):
         oracle.proj(np.zeros((2, 2)), [0, 2], np.zeros((2, 2)), [1, 1], [1, 1])
