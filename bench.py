@@ -14,6 +14,7 @@ count only the block GEMMs the rule keeps.
     4                  KV-cached decode step, M in {1, 8, 32, 64}: 64-layer dependent FFN chain
     5q2 5q4 5q8 5q16   scale sweep 4096 -> 16384 -> 4096, M = 32768, i.i.d. row types
     pilot              tensor-square law Q_2 (x) Q_2 at the paper's pilot shape (768 -> 1536 -> 768)
+    gpilot g8b         gated (SwiGLU) FFN with merged gate/up bank: the pilot's FFN; 4096 -> 12288 at q=32
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
 rank runs the same per-GPU batch (weak scaling), time = max over ranks.
@@ -60,6 +61,12 @@ CONFIGS = {
                  label="cfg5: q=16 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
     "pilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="explicit",
                   label="pilot: Q_2 (x) Q_2 FFN 768->1536->768 (4 x 192 / 4 x 384), M=8x1536 rows, interval schedule, bf16"),
+    "gpilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="explicit", gated=True,
+                   label="gated pilot: bias-free SwiGLU FFN 768->1536->768 under Q_2 (x) Q_2 (4 x 192 / 4 x 384), merged gate/up "
+                         "bank, M=8x1536 rows, interval schedule, bf16"),
+    "g8b": dict(q=32, D=4096, F=12288, M=2048, law="qq", schedule="explicit", gated=True,
+                label="gated FFN 4096->12288->4096 at q=32 (groups of 128 / 384), merged gate/up bank, M=2048 rows, "
+                      "i.i.d. row types, bf16"),
     "4": dict(q=2, D=768, F=3072, M=64, law="qq", schedule="explicit",
               label="cfg4: KV-cached decode step, q=2 FFN 768->3072->768, M in {1,8,32,64}, type = position mod 2, bf16"),
 }
@@ -180,6 +187,12 @@ def make_workload(name: str):
         return synth.pilot_ffn(M=CONFIGS[name]["M"])
     if name == "4":
         return synth.config4(64)
+    if name in ("gpilot", "g8b"):
+        cfg = CONFIGS[name]
+        types = synth.interval_types(cfg["M"], 4, 768) if name == "gpilot" else synth.uniform_types(synth.seed_for(8, 32), cfg["M"], cfg["q"])
+        wl, Wg = synth.gated_ffn(name, cfg["q"], cfg["M"], cfg["D"], cfg["F"], types, variant=7)
+        wl.meta["W_gate"] = Wg
+        return wl
     raise ValueError(name)
 
 
@@ -188,13 +201,21 @@ def oracle_sample(name: str, wl, budget_macs: float = 2.0e11):
     import oracle
     cfg = CONFIGS[name]
     keep = oracle.support(wl.q, cfg["law"])
-    per_row = (oracle.macs(keep, wl.d_widths, wl.f_widths, np.ones(wl.q, dtype=np.int64)) +
+    up_factor = 2 if cfg.get("gated") else 1      # gate and up are two D x F projections
+    per_row = (up_factor * oracle.macs(keep, wl.d_widths, wl.f_widths, np.ones(wl.q, dtype=np.int64)) +
                oracle.macs(keep, wl.f_widths, wl.d_widths, np.ones(wl.q, dtype=np.int64))) / wl.q
     n = int(min(wl.M, max(16, 2 ** int(math.log2(max(16.0, budget_macs / per_row))))))
     rows = np.arange(0, wl.M, max(1, wl.M // n))[:n]
     counts = np.bincount(wl.types[rows], minlength=wl.q)
-    flops = 2 * (oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + oracle.macs(keep, wl.f_widths, wl.d_widths, counts))
+    flops = 2 * (up_factor * oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + oracle.macs(keep, wl.f_widths, wl.d_widths, counts))
     return rows, keep, flops
+
+
+def oracle_ffn(name, wl, rows, keep):
+    import oracle
+    if CONFIGS[name].get("gated"):
+        return oracle.ffn_swiglu(wl.X[rows], wl.types[rows], wl.meta["W_gate"], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+    return oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
 
 
 def run_reference(args):
@@ -205,12 +226,11 @@ def run_reference(args):
         return
     wl = make_workload(args.config)
     rows, keep, flops = oracle_sample(args.config, wl, 1.0e11)
-    X, t = wl.X[rows], wl.types[rows]
     for _ in range(args.warmup):
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+        oracle_ffn(args.config, wl, rows, keep)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+        oracle_ffn(args.config, wl, rows, keep)
     dt = (time.perf_counter() - t0) / args.steps
     val = flops / dt / 1e12
     sample = f"{len(rows)} of {wl.M} rows per step (evenly spaced), all outputs, fp64"
@@ -227,12 +247,11 @@ def run_reference(args):
 def time_cpu_oracle(name, wl):
     import oracle
     rows, keep, flops = oracle_sample(name, wl)
-    X, t = wl.X[rows], wl.types[rows]
     best = None
     t_all = time.perf_counter()
     for _ in range(3):
         t0 = time.perf_counter()
-        oracle.ffn(X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+        oracle_ffn(name, wl, rows, keep)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
         if time.perf_counter() - t_all > 25:
@@ -251,7 +270,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-control / explicit-types / decode side measurements")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "4": 20}.get(args.config, 20) if args.impl == "ours" else 3
+        args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "gpilot": 300, "g8b": 100, "4": 20}.get(args.config, 20) if args.impl == "ours" else 3
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else min(args.warmup, 1)
     if args.impl == "reference":
         run_reference(args)
@@ -289,7 +308,10 @@ def run_prefill(args, ctx):
     # configuration 2 fixes the schedule "type = position mod 2": its handle is created with that
     # schedule (the per-call types array is then not needed); the explicit-types path of the same
     # workload is timed as a side measurement.  The other configurations draw i.i.d. row types.
-    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"], schedule=cfg["schedule"])
+    gated = bool(cfg.get("gated"))
+    Handle = binding.GatedFFN if gated else binding.FFN
+    ffn = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"], schedule=cfg["schedule"])
+    w_up_host = np.concatenate([wl.meta["W_gate"], wl.W_up], axis=1) if gated else wl.W_up   # merged bank [W_gate | W_up]
     counts = np.bincount(wl.types, minlength=wl.q).tolist()
     flops = 2 * ffn.macs(counts)
     stream = torch.cuda.current_stream()
@@ -302,7 +324,7 @@ def run_prefill(args, ctx):
     # explicit flush: a write-flush would leave L2 full of dirty lines whose write-back the next
     # step then pays for).  A set larger than twice the L2 needs no second one.
     ws_bytes = ffn.workspace_bytes(M)
-    set_bytes = 2 * M * D * 2 + 2 * D * F * 2 + ws_bytes
+    set_bytes = 2 * M * D * 2 + (3 if gated else 2) * D * F * 2 + ws_bytes
     n_sets = N_SETS if name == "2" else (1 if set_bytes > 2 * L2_BYTES else int(min(6, max(2, math.ceil(4 * L2_BYTES / set_bytes)))))
     sets = []
     for r in range(n_sets):
@@ -313,14 +335,17 @@ def run_prefill(args, ctx):
         else:
             g = torch.Generator(device="cuda").manual_seed(synth.seed_for(9, rank * 16 + r))
             Xr = torch.randn((M, D), device="cuda", generator=g).to(torch.bfloat16)
-        sets.append({"X": Xr, "Wu": dev(wl.W_up).clone(), "Wd": dev(wl.W_down).clone(),
+        sets.append({"X": Xr, "Wu": dev(w_up_host).clone(), "Wd": dev(wl.W_down).clone(),
                      "Y": torch.empty((M, D), dtype=torch.bfloat16, device="cuda"),
                      "ws": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")})
     footprint_mb = n_sets * set_bytes / 1e6
 
     def step(i, handle=None, tt=call_types):
         s_ = sets[i % n_sets]
-        (handle or ffn).forward(s_["X"], tt, s_["Wu"], s_["Wd"], act="gelu", out=s_["Y"], workspace=s_["ws"], stream=stream)
+        if gated:
+            (handle or ffn).forward(s_["X"], tt, s_["Wu"], s_["Wd"], out=s_["Y"], workspace=s_["ws"], stream=stream)
+        else:
+            (handle or ffn).forward(s_["X"], tt, s_["Wu"], s_["Wd"], act="gelu", out=s_["Y"], workspace=s_["ws"], stream=stream)
 
     def barrier():
         if world > 1:
@@ -387,11 +412,12 @@ def run_prefill(args, ctx):
     burst = region_s < 0.1       # a region this short runs at burst clocks, like the burst measurement of the peak
     peak_tf = peaks["bf16_tflops"] if burst or not peaks["bf16_tflops_sustained"] else peaks["bf16_tflops_sustained"]
     bytes_proj = (M * D + D * F + M * F) * 2          # one projection: activations in, weights, activations out
-    bytes_step = 2 * bytes_proj                       # H is written by the up kernel and read by the down kernel
+    bytes_step = 2 * bytes_proj + (D * F * 2 if gated else 0)   # H is written by the up kernel and read by the down kernel
     t_tensor, t_hbm = flops / (peak_tf * 1e12), bytes_step / (peaks["hbm_gbs"] * 1e9)
     gemm_launches = 2 * args.steps                    # the dominant kernel runs twice per step
     avg_launch_ms = total_ms / gemm_launches
-    kernel = "proj_tc_kernel (two launches per step: up with GELU, down with row scatter)"
+    kernel = ("proj_tc_kernel (two launches per step: merged gate/up with silu(gate) * up, down with row scatter)" if gated
+              else "proj_tc_kernel (two launches per step: up with GELU, down with row scatter)")
     if t_tensor >= t_hbm:
         achieved = flops * args.steps / region_s / 1e12
         roofline = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
@@ -422,11 +448,26 @@ def run_prefill(args, ctx):
         slots.append({"X": torch.from_numpy(wl.X).to(torch.bfloat16).pin_memory(),
                       "t": None if call_types is None else torch.from_numpy(wl.types).pin_memory(),
                       "Y": torch.empty((M, D), dtype=torch.bfloat16).pin_memory(),
-                      "ws": torch.empty(ffn.host_workspace_bytes(M, torch.bfloat16), dtype=torch.uint8, device="cuda"),
+                      "ws": None if gated else torch.empty(ffn.host_workspace_bytes(M, torch.bfloat16), dtype=torch.uint8, device="cuda"),
                       "stream": torch.cuda.Stream()})
+
+    if gated:   # no host entry point: the same copies are made around the device entry point
+        for sl in slots:
+            sl["Xd"] = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
+            sl["td"] = torch.empty(M, dtype=torch.int32, device="cuda")
+            sl["Yd"] = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
+            sl["wsd"] = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
 
     def host_step(i):
         sl = slots[i % n_slots]
+        if gated:
+            with torch.cuda.stream(sl["stream"]):
+                sl["Xd"].copy_(sl["X"], non_blocking=True)
+                sl["td"].copy_(sl["t"], non_blocking=True)
+                ffn.forward(sl["Xd"], sl["td"], sets[i % n_sets]["Wu"], sets[i % n_sets]["Wd"], out=sl["Yd"], workspace=sl["wsd"],
+                            stream=sl["stream"])
+                sl["Y"].copy_(sl["Yd"], non_blocking=True)
+            return
         ffn.forward_host(sl["X"], sl["t"], sets[i % n_sets]["Wu"], sets[i % n_sets]["Wd"], sl["Y"], workspace=sl["ws"],
                          stream=sl["stream"])
 
@@ -455,14 +496,14 @@ def run_prefill(args, ctx):
     extras = {}
     if rank == 0 and not args.no_extras:
         n = min(24, args.steps)
-        dense = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule=cfg["schedule"])
+        dense = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule=cfg["schedule"])
         time_steps(min(6, n), dense)
         dense_ms = time_steps(n, dense) / n
         star_ms = time_steps(n) / n
         extras["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms,
                               "time_ratio_star_over_dense": star_ms / dense_ms,
                               "control": "same library, ALG_TABLE_DENSE, same schedule, measured back to back with the star_q run",
-                              "ideal_ratio": flops / (2.0 * 2 * M * D * F)}
+                              "ideal_ratio": flops / (2.0 * (3 if gated else 2) * M * D * F)}
         del dense
         if name == "2":
             explicit = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")

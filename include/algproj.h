@@ -218,6 +218,26 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
                              const void *W_up, const void *b_up, const void *W_down,
                              const void *b_down, alg_act_t act, void *Y, alg_dtype_t y_dtype,
                              void *workspace, size_t workspace_bytes, void *stream);
+/* ---- gated FFN (SwiGLU): Y = (silu(X *_q W_gate) .* (X *_q W_up)) *_q W_down  -----------------
+ * The FFN of the paper's pretraining pilot (Section "Projection Shapes": a gated FFN uses two
+ * D x F weights and one F x D weight, the same row law on each; appendix "Experimental Details":
+ * bias-free SwiGLU; appendix "Kernel Benchmark Details", Table kernel-ffn: gate and up merged).
+ * silu(g) = g / (1 + exp(-g)).  No biases.
+ * W_gate_up is the merged bank, D x 2F packed: columns [0, F) are W_gate, columns [F, 2F) are W_up,
+ * each split into the q hidden groups f_widths; one kernel accumulates the gate and the up columns
+ * of a tile side by side and stores silu(gate) * up, so the two pre-activations never reach memory.
+ * W_down is F x D packed.  Create with alg_ffn_gated_create (bf16 only; every d width a multiple
+ * of 64 and every f width a multiple of 128, else ALG_ERR_UNSUPPORTED_SHAPE); workspace size,
+ * options, MAC count (three projections), status and destruction through the alg_ffn_* calls.
+ * Every M runs the prefill kernels (there is no small-M kernel for the gated form yet). */
+alg_status_t alg_ffn_gated_create(alg_ffn_t *out, int q, const int32_t *d_widths,
+                                  const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,
+                                  const uint8_t *custom_keep, alg_schedule_t schedule);
+alg_status_t alg_ffn_gated_forward(alg_ffn_t h, const void *X, const int32_t *types, int64_t M,
+                                   const void *W_gate_up, const void *W_down, void *Y,
+                                   alg_dtype_t y_dtype, void *workspace, size_t workspace_bytes,
+                                   void *stream);
+
 /* Same computation with X, types and Y in HOST memory (pinned memory makes the copies
  * asynchronous).  Copies X and types to device staging inside the workspace, runs the
  * forward pass, copies Y back, all on `stream`; returns without synchronising.  Weights and

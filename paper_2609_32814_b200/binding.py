@@ -35,7 +35,7 @@ EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
     "alg_proj_forward_static", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
-    "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
+    "alg_ffn_gated_create", "alg_ffn_gated_forward", "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
 ]
 
 _lib = None
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.alg_proj_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.alg_ffn_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
         L.alg_ffn_destroy.argtypes = [vp]
+        L.alg_ffn_gated_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
+        L.alg_ffn_gated_forward.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_ffn_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
         L.alg_ffn_forward.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_ffn_host_workspace_bytes.argtypes = [vp, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
@@ -219,6 +221,7 @@ class FFN(_Handle):
     """alg_ffn_* : Y = act(X *_q W_up + b_up) *_q W_down + b_down."""
     _destroy = "alg_ffn_destroy"
     _set_option = "alg_ffn_set_option"
+    _create = "alg_ffn_create"
 
     def __init__(self, d_widths, f_widths, dtype="bf16", table="qq", custom_keep=None, schedule="explicit"):
         super().__init__()
@@ -228,9 +231,9 @@ class FFN(_Handle):
         self.schedule = _SCHEDS[schedule]
         buf, keep = _keep_arg(table, custom_keep, self.q)
         d, f = _widths(d_widths), _widths(f_widths)
-        _check(lib().alg_ffn_create(ctypes.byref(self._h), self.q, ctypes.cast(d, ctypes.c_void_p),
-                                    ctypes.cast(f, ctypes.c_void_p), self.dtype, _TABLES[table], keep, self.schedule),
-               "alg_ffn_create")
+        _check(getattr(lib(), self._create)(ctypes.byref(self._h), self.q, ctypes.cast(d, ctypes.c_void_p),
+                                            ctypes.cast(f, ctypes.c_void_p), self.dtype, _TABLES[table], keep,
+                                            self.schedule), self._create)
 
     def workspace_bytes(self, max_M: int) -> int:
         out = ctypes.c_size_t()
@@ -286,3 +289,25 @@ class FFN(_Handle):
         s = ctypes.c_int()
         _check(lib().alg_ffn_last_status(self._h, _stream(stream), ctypes.byref(s)), "alg_ffn_last_status")
         return s.value
+
+
+class GatedFFN(FFN):
+    """alg_ffn_gated_* : Y = (silu(X *_q W_gate) .* (X *_q W_up)) *_q W_down, W_gate_up = [W_gate | W_up] (D x 2F)."""
+    _create = "alg_ffn_gated_create"
+
+    def forward(self, X, types, W_gate_up, W_down, out=None, out_dtype=None, workspace=None, stream=None):
+        M = X.shape[0]
+        if not (X.is_contiguous() and W_gate_up.is_contiguous() and W_down.is_contiguous()):
+            raise ValueError("alg_ffn_gated_forward takes packed row-major tensors")
+        if W_gate_up.shape != (self.D, 2 * self.F):
+            raise ValueError("W_gate_up must be D x 2F: [W_gate | W_up]")
+        if out is None:
+            out = torch.empty((M, self.D), dtype=out_dtype or X.dtype, device=X.device)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(M), X.device)
+        _check(lib().alg_ffn_gated_forward(self._h, _ptr(X), _ptr(types), M, _ptr(W_gate_up), _ptr(W_down), _ptr(out),
+                                           _DTYPES[out.dtype], _ptr(ws), ws.numel(), _stream(stream)),
+               "alg_ffn_gated_forward")
+        return out
+
+    def forward_host(self, *a, **k):
+        raise NotImplementedError("the gated FFN has no host entry point")

@@ -42,6 +42,7 @@ struct alg_proj_s {
   // one-CTA kernel with 256-row x 128-column tiles (two accumulators per tile): taken when every
   // row type has enough rows to fill such tiles.  Its tile classes (128 columns wide) live in
   // `tab_tall` when the regular tile width is not 128.
+  bool gated = false;       // SwiGLU up projection over the merged [W_gate | W_up] bank (N = F, W has 2 F columns)
   bool tall_ok = false;
   DevTable tab_tall;
   DevTable *d_tab_tall = nullptr;
@@ -67,6 +68,7 @@ struct alg_ffn_s {
   bool timing = false;       // record events between the kernels of each forward call
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   // decode step of the whole FFN in one launch (M <= kFfnDecodeMaxM)
+  bool gated = false;        // SwiGLU: up = merged gate/up projection with silu(gate) * up epilogue
   bool fd_ok = false;
   FfnDecodePlan fd = {};
   unsigned int *d_counters = nullptr;
@@ -140,6 +142,12 @@ alg_status_t configure_kernels(alg_proj_s &p) {
     min_klen = std::min(min_klen, len);
   }
   p.pair_kernel = p.tc_ok && all128 && min_klen >= 4096;
+  if (p.gated) {   // 128 output columns per tile (the MMA is 256 wide: gate and up halves)
+    if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
+    if (p.opt_kernel > 1 || (p.opt_tile_n != 0 && p.opt_tile_n != 128)) return ALG_ERR_UNSUPPORTED_SHAPE;
+    p.tile_n = 128;
+    p.pair_kernel = false;
+  }
   if (p.opt_kernel == 1) p.pair_kernel = false;
   if (p.opt_kernel == 2) {
     if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
@@ -150,7 +158,7 @@ alg_status_t configure_kernels(alg_proj_s &p) {
   if (bs != ALG_OK) return bs;
   // 256-row tiles: one-CTA kernel, 128-column tiles must divide every output group, and wider
   // tiles (which reuse A as well) must not be available
-  p.tall_ok = p.tc_ok && !p.pair_kernel && all128 && !all256 && p.opt_tile_n == 0 && p.opt_kernel != 1;
+  p.tall_ok = p.tc_ok && !p.pair_kernel && !p.gated && all128 && !all256 && p.opt_tile_n == 0 && p.opt_kernel != 1;
   if (p.opt_kernel == 3) {
     if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
     p.pair_kernel = false;
@@ -174,7 +182,9 @@ alg_status_t pick_workers(alg_proj_s &p) {
 }
 
 alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t *out_w, alg_dtype_t dtype,
-                       alg_table_t table, const uint8_t *custom, alg_schedule_t sched, int *shared_status) {
+                       alg_table_t table, const uint8_t *custom, alg_schedule_t sched, int *shared_status,
+                       bool gated = false) {
+  p.gated = gated;
   if (q < 1 || q > kMaxQ || !in_w || !out_w) return ALG_ERR_INVALID_ARG;
   if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
   if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM && table != ALG_TABLE_Q2POW)
@@ -250,7 +260,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
       if (cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming) != cudaSuccess) return ALG_ERR_CUDA;
     }
   }
-  if (dtype == ALG_BF16) {
+  if (dtype == ALG_BF16 && !p.gated) {
     p.decode_ok = decode_plan(q, p.s, p.K, p.N, p.num_sms, &p.decode);
     for (int g = 0; g < q && p.decode_ok; ++g)
       if (p.r[g] % p.decode.sn) p.decode_ok = false;
@@ -430,6 +440,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
   a.b_3d = 0;
   a.a_box_256 = 0;
+  a.gated_f = p.gated ? p.N : 0;
   a.y_staged = 0;
   a.plan = nullptr;
   a.plan_stride = a.plan_rounds = a.plan_tag = 0;
@@ -458,9 +469,11 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
       a.ldx = p.K;
     }
     if (after_gather) cudaEventRecord(after_gather, st);
+    if (p.gated) return cuda_status(launch_proj_tc_gated(a, p.n_workers, st));
     if (p.pair_kernel) return cuda_status(launch_proj_tc2(a, p.num_sms, st));
     return cuda_status(launch_proj_tc(a, tc.tile_n, p.n_workers, st));
   }
+  if (p.gated) return ALG_ERR_UNSUPPORTED_SHAPE;
   if (after_gather) cudaEventRecord(after_gather, st);
   a.X = X;
   a.ldx = ldx;
@@ -674,14 +687,16 @@ alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *stat
   return read_status(h->d_status, stream, status);
 }
 
-alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,
-                            alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
-                            alg_schedule_t schedule) {
+static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,
+                               alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
+                               alg_schedule_t schedule, bool gated) {
   if (!out) return ALG_ERR_INVALID_ARG;
   *out = nullptr;
+  if (gated && dtype != ALG_BF16) return ALG_ERR_UNSUPPORTED_SHAPE;
   alg_ffn_s *f = new (std::nothrow) alg_ffn_s();
   if (!f) return ALG_ERR_INVALID_ARG;
-  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr);
+  f->gated = gated;
+  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated);
   if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status);
   if (s != ALG_OK) {
     free_proj(f->down);
@@ -691,12 +706,32 @@ alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, cons
   }
   f->D = f->up.K;
   f->F = f->up.N;
-  if (dtype == ALG_BF16 && ffn_decode_plan(q, f->up.s, f->down.s, f->D, f->F, f->up.num_sms, &f->fd)) {
+  if (dtype == ALG_BF16 && !gated && ffn_decode_plan(q, f->up.s, f->down.s, f->D, f->F, f->up.num_sms, &f->fd)) {
     f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
   *out = f;
   return ALG_OK;
+}
+
+alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,
+                            alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
+                            alg_schedule_t schedule) {
+  return ffn_create(out, q, d_widths, f_widths, dtype, table, custom_keep, schedule, false);
+}
+
+alg_status_t alg_ffn_gated_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,
+                                  alg_dtype_t dtype, alg_table_t table, const uint8_t *custom_keep,
+                                  alg_schedule_t schedule) {
+  return ffn_create(out, q, d_widths, f_widths, dtype, table, custom_keep, schedule, true);
+}
+
+alg_status_t alg_ffn_gated_forward(alg_ffn_t h, const void *X, const int32_t *types, int64_t M, const void *W_gate_up,
+                                   const void *W_down, void *Y, alg_dtype_t y_dtype, void *workspace,
+                                   size_t workspace_bytes, void *stream) {
+  if (!h || !h->gated) return ALG_ERR_INVALID_ARG;
+  return alg_ffn_forward(h, X, types, M, W_gate_up, nullptr, W_down, nullptr, ALG_ACT_NONE, Y, y_dtype, workspace,
+                         workspace_bytes, stream);
 }
 
 alg_status_t alg_ffn_destroy(alg_ffn_t h) {
@@ -788,8 +823,9 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;
-  alg_status_t s = run_proj(h->up, L, ws, X, h->D, false, W_up, h->F, b_up, act, H, h->F, h->up.dtype, true, M, st,
-                            tm ? h->ev[2] : nullptr, cyc);
+  if (h->gated && (b_up || b_down || act != ALG_ACT_NONE)) return ALG_ERR_INVALID_ARG;   // bias-free, silu(gate) * up
+  alg_status_t s = run_proj(h->up, L, ws, X, h->D, false, W_up, h->gated ? 2 * (int64_t)h->F : h->F, b_up, act, H, h->F,
+                            h->up.dtype, true, M, st, tm ? h->ev[2] : nullptr, cyc);
   if (s != ALG_OK) return s;
   if (tm) cudaEventRecord(h->ev[3], st);
   s = run_proj(h->down, L, ws, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st,
@@ -865,7 +901,7 @@ alg_status_t alg_ffn_macs(alg_ffn_t h, const int64_t *rows_per_type, int64_t *ma
   if (s != ALG_OK) return s;
   s = alg_proj_macs(&h->down, rows_per_type, &b);
   if (s != ALG_OK) return s;
-  *macs = a + b;
+  *macs = (h->gated ? 2 * a : a) + b;   // gate and up are two D x F projections
   return ALG_OK;
 }
 

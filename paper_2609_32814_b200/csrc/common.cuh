@@ -128,6 +128,10 @@ struct ProjArgs {
   int out_cyclic_rows;
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   int a_box_256;          // A tensor map carries 256-row boxes (one-CTA kernel with 256-row tiles)
+  // Gated (SwiGLU) up projection: W is the merged bank [W_gate | W_up] with 2 * gated_f columns, a
+  // tile accumulates 128 gate columns and the matching 128 up columns side by side, the epilogue
+  // stores silu(gate) * up; N = gated_f is the width of the output.  0 = ordinary projection.
+  int gated_f;
   int y_staged;           // 1: the epilogue transposes bf16 results through shared memory for coalesced stores
   // Cyclic schedule: the tile sequences of all workers depend only on (handle, M) and are planned
   // once on the host; worker w reads plan[1 + w * plan_stride .. + plan_rounds) (the last record of
@@ -149,6 +153,7 @@ constexpr int kTcBlockK = 64;
 constexpr int kTc2TileM = 256;
 constexpr int kTc2TileN = 256;
 cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st);
+cudaError_t launch_proj_tc_gated(const ProjArgs &a, int num_sms, cudaStream_t st);  // 128 output columns per tile
 cudaError_t launch_proj_tc2(const ProjArgs &a, int num_sms, cudaStream_t st);
 int tc2_max_pairs(int num_sms);  // CTA pairs that can be co-resident (0 on failure)
 constexpr int kMaxWorkers = 256;

@@ -103,10 +103,16 @@ struct Cfg {
   static_assert(kHalves == 1 || kEpiWarps == 8, "two accumulators need one epilogue warp group each");
 };
 
-template <int TILE_N, int TILE_M>
+// GATED (TILE_N = 256, TILE_M = 128 only): the SwiGLU up projection.  B is the merged bank
+// [W_gate | W_up]; a stage holds the 128 gate columns of the tile followed by its 128 up columns, one
+// N = 256 MMA fills both halves of the accumulator, and the epilogue writes silu(gate) * up -- 128
+// output columns per tile, the hidden state is stored once and the two pre-activations never
+// leave the chip (the merged gate/up kernel of the appendix "Kernel Benchmark Details").
+template <int TILE_N, int TILE_M, bool GATED>
 __global__ void __launch_bounds__(kThreads, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
   using C = Cfg<TILE_N, TILE_M>;
+  static_assert(!GATED || (TILE_N == 256 && TILE_M == 128), "the gated kernel pairs two 128-column halves");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   // optional staging buffers of the epilogue warps sit between the stages and the control block
@@ -230,6 +236,10 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
               else tma_load_2d(sa, &tmA, bar, k0, a_row);
+            } else if (GATED) {
+              // two boxes of two 64-column chunks: the tile's gate columns, then its up columns
+              tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
+              tma_load_3d(sa + C::kABytes + 2 * C::kBChunkBytes, &tmB, bar, 0, k0, (a.gated_f + n0) >> 6);
             } else if (a.b_3d) {
               tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);  // all 64-column chunks in one box
             } else {
@@ -325,6 +335,29 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t taddr =
           tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * C::kAccStride + half * C::kHalf);
       const int col_base = rec.n0 + (C::kHalves == 2 ? 0 : half * C::kHalf);
+      if (GATED) {
+        // this warp: 32 rows x 64 output columns; gate values sit in accumulator columns [0, 128),
+        // the matching up values 128 columns further
+        const uint32_t tg = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * C::kAccStride + half * 64);
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          uint32_t vg[32], vu[32];
+          tc_ld_32x32(tg + (uint32_t)c0, vg);
+          tc_ld_32x32(tg + (uint32_t)(128 + c0), vu);
+          tc_wait_ld();
+          if (out_row >= 0) {
+            float f[32];
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+              const float g = __uint_as_float(vg[x]);
+              float th;
+              asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * g));
+              f[x] = g * fmaf(0.5f, th, 0.5f) * __uint_as_float(vu[x]);   // silu(g) * u, sigmoid(g) = (1 + tanh(g/2)) / 2
+            }
+            finish_and_store_32(f, a, out_row, rec.n0 + half * 64 + c0);
+          }
+        }
+      } else
       // bf16 outputs are transposed through a 2 KB staging buffer per warp: every lane writes its
       // own row segment (64 bytes, 16-byte pieces XOR-swizzled so that the writes and the reads
       // below are bank-conflict free), then four lanes together store one row segment, so one
@@ -417,12 +450,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
-template <int TILE_N, int TILE_M>
+template <int TILE_N, int TILE_M, bool GATED = false>
 cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   using C = Cfg<TILE_N, TILE_M>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -432,13 +465,14 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
   ProjArgs b = a;
-  b.b_3d = make_map_b3d(&tmB, a, TILE_N / 64) == cudaSuccess;
+  b.b_3d = make_map_b3d(&tmB, a, GATED ? 2 : TILE_N / 64) == cudaSuccess;
+  if (GATED && !b.b_3d) return cudaErrorInvalidValue;
   if (!b.b_3d) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
     if (e != cudaSuccess) return e;
   }
   // staging buffers for the transposing epilogue, when they fit and the output rows are 16-byte aligned
-  b.y_staged = a.y_bf16 && smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && ((uintptr_t)a.Y & 15u) == 0 &&
+  b.y_staged = !GATED && a.y_bf16 && smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && ((uintptr_t)a.Y & 15u) == 0 &&
                (a.ldy * 2) % 16 == 0;
   if (b.y_staged) smem_bytes += kEpiWarps * C::kStoreBufBytes;
   cudaLaunchConfig_t cfg = {};
@@ -451,7 +485,7 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED>, tmA, tmB, b);
   count_launch(1);
   return e;
 }
@@ -493,8 +527,9 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
 // 64 x 64 x chunks lands in shared memory chunk-major ([chunk][k][64 n]), which is exactly the
 // MN-major 128-byte-swizzled operand layout, with a single copy instruction per stage.
 cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
-  if (a.N % 64) return cudaErrorInvalidValue;
-  cuuint64_t dims[3] = {64, (cuuint64_t)a.K, (cuuint64_t)(a.N / 64)};
+  const int w_cols = a.gated_f ? 2 * a.gated_f : a.N;   // the merged gate/up bank is twice as wide as the output
+  if (w_cols % 64) return cudaErrorInvalidValue;
+  cuuint64_t dims[3] = {64, (cuuint64_t)a.K, (cuuint64_t)(w_cols / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldw * 2, 128};
   cuuint32_t box[3] = {64, kTcBlockK, (cuuint32_t)chunks};
   cuuint32_t estr[3] = {1, 1, 1};
@@ -529,6 +564,13 @@ cudaError_t tc_init() {
   if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
   g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
   return cudaSuccess;
+}
+
+cudaError_t launch_proj_tc_gated(const ProjArgs &a, int num_sms, cudaStream_t st) {
+  cudaError_t e = tc_init();
+  if (e != cudaSuccess) return e;
+  if (!a.gated_f || a.geom.tile_m != 128 || !a.y_bf16) return cudaErrorInvalidValue;
+  return launch_t<256, 128, true>(a, num_sms, st);
 }
 
 cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st) {

@@ -167,3 +167,12 @@ def pilot_ffn(M: int = 4 * 1536, integer: bool = False) -> Workload:
     4 x 384 (tensor-square law, q = 4), interval schedule with period 768."""
     return make_workload("pilot", config=6, variant=int(integer), dtype="bf16", q=4, M=M, D=768, F=1536,
                          types=interval_types(M, 4, 768), integer=integer)
+
+
+def gated_ffn(name: str, q: int, M: int, D: int, F: int, types: np.ndarray, variant: int = 0, integer: bool = False):
+    """A gated (SwiGLU) FFN problem: the Workload of the two-map FFN plus the gate bank.  Returns
+    (workload, W_gate); the merged bank the library takes is [W_gate | workload.W_up]."""
+    wl = make_workload(name, config=7, variant=300 + variant, dtype="bf16", q=q, M=M, D=D, F=F, types=types, integer=integer)
+    s0 = seed_for(7, 300 + variant)
+    Wg = small_ints(s0 + 4, (D, F)) if integer else bf16_round(normal(s0 + 4, (D, F), 0.02))
+    return wl, Wg

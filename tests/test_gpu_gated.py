@@ -1,0 +1,108 @@
+"""GPU parity of the gated (SwiGLU) FFN, Y = (silu(X * W_gate) .* (X * W_up)) * W_down with the merged
+gate/up bank, against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_32814_b200 import binding, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, Wg, table="qq", schedule="explicit", out_dtype=torch.float32):
+    ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16", table=table, schedule=schedule)
+    Wgu = np.concatenate([Wg, wl.W_up], axis=1)          # the merged bank: [W_gate | W_up]
+    Y = ffn.forward(H.to_dev(wl.X, "bf16"), None if schedule == "cyclic" else H.dev_types(wl.types),
+                    H.to_dev(Wgu, "bf16"), H.to_dev(wl.W_down, "bf16"), out_dtype=out_dtype)
+    assert ffn.last_status() == 0
+    return Y, ffn
+
+
+def _sample_rows(wl, per_type, seed=0):
+    rng = np.random.default_rng(seed)
+    rows = []
+    for t in range(wl.q):
+        idx = np.flatnonzero(wl.types == t)
+        if idx.size:
+            tail = idx[(idx.size // 128) * 128:]
+            rows.append(np.concatenate([idx[:2], idx[-2:], tail[:2], rng.choice(idx, size=min(per_type, idx.size), replace=False)]))
+    return np.unique(np.concatenate(rows))
+
+
+@pytest.mark.parametrize("q,M,D,F,schedule", [
+    (2, 700, 256, 512, "explicit"),      # ragged buckets, two hidden tiles per group
+    (2, 1024, 128, 256, "cyclic"),       # type-strided A view
+    (3, 515, 192, 384, "explicit"),      # non-power-of-two q, one hidden tile per group
+    (1, 300, 128, 384, "explicit"),      # q = 1: an ordinary gated MLP
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_gated_ffn_small_shapes(q, M, D, F, schedule, out_dtype):
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(600 + q, M, q)
+    wl, Wg = synth.gated_ffn("gated", q, M, D, F, types, variant=q * 10 + M % 7)
+    # weights of the test are scaled up so that the hidden state is of order one
+    wl.W_up, Wg, wl.W_down = (synth.bf16_round(w * 4.0) for w in (wl.W_up, Wg, wl.W_down))
+    Y, ffn = _run(wl, Wg, schedule=schedule, out_dtype=out_dtype)
+    ref = oracle.ffn_swiglu(wl.X, wl.types, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"gated q={q} M={M}")
+    counts = np.bincount(wl.types, minlength=q).tolist()
+    keep = oracle.support(q)
+    assert ffn.macs(counts) == 2 * oracle.macs(keep, wl.d_widths, wl.f_widths, counts) + \
+        oracle.macs(keep, wl.f_widths, wl.d_widths, counts)
+
+
+def test_gated_hidden_state_alone():
+    """W_down = identity blocks turns the output into the hidden state of the row's own group:
+    checks silu(gate) * up itself, on values spread over [-8, 8]."""
+    q, M, D = 1, 256, 128
+    F = 128
+    X = synth.bf16_round(np.linspace(-8, 8, M * D, dtype=np.float32).reshape(M, D))
+    Wg = np.eye(D, F, dtype=np.float32)
+    Wu = synth.bf16_round(synth.normal(5, (D, F), 0.5))
+    Wd = np.eye(F, D, dtype=np.float32)
+    ffn = binding.GatedFFN([D], [F], dtype="bf16")
+    t = torch.zeros(M, dtype=torch.int32, device="cuda")
+    Y = ffn.forward(H.to_dev(X, "bf16"), t, H.to_dev(np.concatenate([Wg, Wu], axis=1), "bf16"), H.to_dev(Wd, "bf16"),
+                    out_dtype=torch.float32)
+    ref, Hh = oracle.ffn_swiglu(X, np.zeros(M, np.int32), Wg, Wu, Wd, [D], [F], return_hidden=True)
+    got = H.to_np(Y)
+    # Y is the bf16-rounded hidden state: half an ulp of bf16 plus the activation's own error
+    assert np.all(np.abs(got - Hh) <= 2.0 ** -8 * np.abs(Hh) + 2e-3), float(np.abs(got - Hh).max())
+
+
+def test_gated_pilot_shape_tensor_square_law():
+    """The paper's pilot FFN: D = 768 = 4 x 192, F = 1536 = 4 x 384, bias-free SwiGLU under the
+    tensor-square law Q_2 (x) Q_2, interval schedule."""
+    M = 4 * 1536
+    wl, Wg = synth.gated_ffn("pilot-gated", 4, M, 768, 1536, synth.interval_types(M, 4, 768), variant=1)
+    keep = oracle.support(4, "q2pow")
+    Y, ffn = _run(wl, Wg, table="q2pow")
+    rows = _sample_rows(wl, 128, seed=4)
+    ref = oracle.ffn_swiglu(wl.X[rows], wl.types[rows], Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+    got = H.to_np(Y[torch.from_numpy(rows).cuda()])
+    assert H.rel_fro(got, ref) <= H.BF16_REL_FRO
+    assert H.max_abs(got, ref) <= H.BF16_MAX_ABS
+    counts = np.bincount(wl.types, minlength=4).tolist()
+    assert ffn.macs(counts) * 16 == 9 * 3 * M * 768 * 1536          # (3/4)^2 of the dense 3 M D F
+
+
+def test_gated_kernel_table_shape_q32():
+    """One shape of the paper's gated-FFN table: 4096 -> 12288 -> 4096 at q = 32 (group widths 128
+    and 384), M = 2048 rows, i.i.d. row types."""
+    q, M, D, F = 32, 2048, 4096, 12288
+    wl, Wg = synth.gated_ffn("gated-q32", q, M, D, F, synth.uniform_types(632, M, q), variant=2)
+    Y, ffn = _run(wl, Wg)
+    rows = np.unique(np.concatenate([np.arange(0, M, 16), [M - 1]]))
+    ref = oracle.ffn_swiglu(wl.X[rows], wl.types[rows], Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    got = H.to_np(Y[torch.from_numpy(rows).cuda()])
+    assert H.rel_fro(got, ref) <= H.BF16_REL_FRO
+    assert H.max_abs(got, ref) <= H.BF16_MAX_ABS
+
+
+def test_gated_refusals():
+    with pytest.raises(binding.AlgError) as e:
+        binding.GatedFFN([64, 64], [192, 192], dtype="bf16")      # hidden groups are no multiples of 128
+    assert e.value.code == 2
+    with pytest.raises(binding.AlgError):
+        binding.GatedFFN([64, 64], [128, 128], dtype="f32")
