@@ -59,6 +59,8 @@ def _load():
         lib.star_gelu.argtypes = [ctypes.c_double]
         lib.star_ffn.argtypes = [f64p, i32p, i64, f64p, f64p, f64p, f64p, f64p, f64p,
                                  ctypes.c_int, i32p, i32p, u8p]
+        lib.star_proj_vjp_x.argtypes = [f64p, i64, i32p, i64, f64p, i64, f64p, i64, ctypes.c_int, i32p, i32p, u8p]
+        lib.star_proj_vjp_w.argtypes = [f64p, i64, f64p, i64, i32p, i64, f64p, i64, ctypes.c_int, i32p, i32p, u8p]
         lib.star_silu.restype = ctypes.c_double
         lib.star_silu.argtypes = [ctypes.c_double]
         lib.star_ffn_swiglu.argtypes = [f64p, i32p, i64, f64p, f64p, f64p, f64p, f64p, f64p, f64p,
@@ -260,3 +262,37 @@ def ffn_swiglu(X, types, W_gate, W_up, W_down, dw, fw, keep=None, return_hidden=
     _check(lib.star_ffn_swiglu(_p(X, f64), _p(types, i32), M, _p(W_gate, f64), _p(W_up, f64), _p(W_down, f64),
                                _p(G, f64), _p(U, f64), _p(H, f64), _p(Y, f64), q, _p(dw, i32), _p(fw, i32), _p(keep, u8)))
     return (Y, H) if return_hidden else Y
+
+
+def proj_vjp_x(G, types, W, s, r, keep=None) -> np.ndarray:
+    """dX of Y = X *_q W for the output gradient G (M x N): same block support as the forward pass."""
+    lib = _load()
+    G, W, types, s, r = _f64(G), _f64(W), _i32(types), _i32(s), _i32(r)
+    q = len(s)
+    keep = np.ascontiguousarray(support(q, "qq") if keep is None else keep, dtype=np.uint8)
+    M, N = G.shape
+    K = int(s.sum())
+    if W.shape != (K, N) or int(r.sum()) != N or len(types) != M:
+        raise OracleError("shape mismatch")
+    dX = np.empty((M, K), dtype=np.float64)
+    f64, i32, u8 = ctypes.c_double, ctypes.c_int32, ctypes.c_uint8
+    _check(lib.star_proj_vjp_x(_p(G, f64), N, _p(types, i32), M, _p(W, f64), N, _p(dX, f64), K, q, _p(s, i32),
+                               _p(r, i32), _p(keep, u8)))
+    return dX
+
+
+def proj_vjp_w(X, G, types, s, r, keep=None) -> np.ndarray:
+    """dW of Y = X *_q W for the output gradient G: blocks no row reaches are zero."""
+    lib = _load()
+    X, G, types, s, r = _f64(X), _f64(G), _i32(types), _i32(s), _i32(r)
+    q = len(s)
+    keep = np.ascontiguousarray(support(q, "qq") if keep is None else keep, dtype=np.uint8)
+    M, K = X.shape
+    N = int(r.sum())
+    if G.shape != (M, N) or int(s.sum()) != K or len(types) != M:
+        raise OracleError("shape mismatch")
+    dW = np.empty((K, N), dtype=np.float64)
+    f64, i32, u8 = ctypes.c_double, ctypes.c_int32, ctypes.c_uint8
+    _check(lib.star_proj_vjp_w(_p(X, f64), K, _p(G, f64), N, _p(types, i32), M, _p(dW, f64), N, q, _p(s, i32),
+                               _p(r, i32), _p(keep, u8)))
+    return dW

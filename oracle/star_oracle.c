@@ -16,7 +16,8 @@
  * rule term by term, dense-minus-removed brute force, associativity/unit/edge-ideal on
  * integer block arrays, the 2q^2-q count and the MAC formulas, q=1 / dense table against
  * numpy.matmul, GELU and SiLU against closed-form values, the gated FFN against an
- * independent numpy composition.
+ * independent numpy composition, the two gradient maps against the displayed per-type equations
+ * and against the adjoint identities <X * W, G> = <X, dX(G)> = <W, dW(X, G)>.
  * Parity unpinned by the paper: the FFN-level choices (erf-GELU, bias added before the
  * activation) come from the benchmark specification, not from a printed value; SwiGLU is
  * named by the paper without its formula (the standard one is taken).
@@ -329,4 +330,73 @@ int star_ffn_swiglu(const double *X, const int32_t *types, int64_t M, const doub
 #pragma omp parallel for schedule(static)
   for (int64_t e = 0; e < M * F; ++e) H[e] = star_silu(G[e]) * U[e];
   return star_proj_rows(H, F, types, M, W_down, D, NULL, Y, D, q, fw, dw, keep);
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Vector-Jacobian products of the row-typed projection (Appendix "Vector-Jacobian Products",
+ * Eqs. vjp-xi ... vjp-wjj, written for a general support set): with G the gradient with respect
+ * to Y,
+ *     dX[b, S_k]   = sum_{j : k in B(t_b, j)} G[b, R_j] W[S_k, R_j]^T
+ *     dW[S_k, R_j] = sum_{b : k in B(t_b, j)} X[b, S_k]^T G[b, R_j].
+ * Both keep exactly the block support of the forward table; blocks of dW no row reaches stay 0.
+ * ------------------------------------------------------------------------------------- */
+int star_proj_vjp_x(const double *G, int64_t ldg, const int32_t *types, int64_t M, const double *W,
+                    int64_t ldw, double *dX, int64_t lddx, int q, const int32_t *s,
+                    const int32_t *r, const uint8_t *keep) {
+  if (q < 1 || M < 0 || !s || !r || !keep) return ORACLE_BAD_ARG;
+  int64_t *so = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  int64_t *ro = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  prefix(q, s, so);
+  prefix(q, r, ro);
+  int bad = 0;
+  for (int64_t b = 0; b < M; ++b)
+    if (types[b] < 0 || types[b] >= q) bad = 1;
+  if (!bad) {
+#pragma omp parallel for schedule(static)
+    for (int64_t b = 0; b < M; ++b) {
+      const int i = types[b];
+      for (int k = 0; k < q; ++k)
+        for (int64_t c = so[k]; c < so[k + 1]; ++c) {
+          double acc = 0.0;
+          for (int j = 0; j < q; ++j) {
+            if (!keep[((size_t)i * q + j) * q + k]) continue;
+            for (int64_t n = ro[j]; n < ro[j + 1]; ++n) acc += G[b * ldg + n] * W[c * ldw + n];
+          }
+          dX[b * lddx + c] = acc;
+        }
+    }
+  }
+  free(so);
+  free(ro);
+  return bad ? ORACLE_BAD_TYPE : ORACLE_OK;
+}
+
+int star_proj_vjp_w(const double *X, int64_t ldx, const double *G, int64_t ldg,
+                    const int32_t *types, int64_t M, double *dW, int64_t lddw, int q,
+                    const int32_t *s, const int32_t *r, const uint8_t *keep) {
+  if (q < 1 || M < 0 || !s || !r || !keep) return ORACLE_BAD_ARG;
+  int64_t *so = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  int64_t *ro = (int64_t *)malloc(sizeof(int64_t) * (q + 1));
+  prefix(q, s, so);
+  prefix(q, r, ro);
+  int bad = 0;
+  for (int64_t b = 0; b < M; ++b)
+    if (types[b] < 0 || types[b] >= q) bad = 1;
+  if (!bad) {
+#pragma omp parallel for schedule(static)
+    for (int64_t c = 0; c < so[q]; ++c) {
+      int k = 0;
+      while (c >= so[k + 1]) ++k;
+      for (int j = 0; j < q; ++j)
+        for (int64_t n = ro[j]; n < ro[j + 1]; ++n) {
+          double acc = 0.0;
+          for (int64_t b = 0; b < M; ++b)
+            if (keep[((size_t)types[b] * q + j) * q + k]) acc += X[b * ldx + c] * G[b * ldg + n];
+          dW[c * lddw + n] = acc;
+        }
+    }
+  }
+  free(so);
+  free(ro);
+  return bad ? ORACLE_BAD_TYPE : ORACLE_OK;
 }

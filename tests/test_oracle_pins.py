@@ -399,6 +399,65 @@ def test_gated_ffn_composes_three_projections():
                                rtol=1e-12, atol=1e-12)
 
 
+@pytest.mark.parametrize("q", [2, 3, 4])
+def test_vjp_against_the_displayed_per_type_equations(q):
+    """Eqs. vjp-xi ... vjp-wjj, typed out per token of type i in numpy (integers: exact)."""
+    rng = np.random.default_rng(70 + q)
+    s = rng.integers(1, 4, size=q)
+    r = rng.integers(1, 4, size=q)
+    so, ro = _offsets(s), _offsets(r)
+    M = 11
+    X = _rand_ints(rng, (M, s.sum()))
+    W = _rand_ints(rng, (s.sum(), r.sum()))
+    G = _rand_ints(rng, (M, r.sum()))
+    types = rng.integers(0, q, size=M)
+    dX, dW = np.zeros_like(X), np.zeros_like(W)
+    blk = lambda A, a, b, ao, bo: A[ao[a]:ao[a + 1], bo[b]:bo[b + 1]]
+    for b in range(M):
+        i = types[b]
+        x = lambda k: X[b, so[k]:so[k + 1]]
+        g = lambda j: G[b, ro[j]:ro[j + 1]]
+        dX[b, so[i]:so[i + 1]] += g(i) @ blk(W, i, i, so, ro).T + sum(g(j) @ blk(W, i, j, so, ro).T for j in range(q) if j != i)
+        dW[so[i]:so[i + 1], ro[i]:ro[i + 1]] += np.outer(x(i), g(i))
+        for j in range(q):
+            if j == i:
+                continue
+            dX[b, so[j]:so[j + 1]] += g(j) @ blk(W, j, j, so, ro).T
+            dW[so[i]:so[i + 1], ro[j]:ro[j + 1]] += np.outer(x(i), g(j))
+            dW[so[j]:so[j + 1], ro[j]:ro[j + 1]] += np.outer(x(j), g(j))
+    assert np.array_equal(oracle.proj_vjp_x(G, types, W, s, r), dX)
+    assert np.array_equal(oracle.proj_vjp_w(X, G, types, s, r), dW)
+
+
+@pytest.mark.parametrize("law,q", [("qq", 3), ("q2pow", 4), ("dense", 2)])
+def test_vjp_adjoint_identities(law, q):
+    """The projection is bilinear in (X, W): <X * W, G> = <X, dX(G)> = <W, dW(X, G)>, exactly on integers,
+    for every support set; a missing type leaves its private blocks of dW at zero."""
+    rng = np.random.default_rng(80 + q)
+    s = rng.integers(1, 4, size=q)
+    r = rng.integers(1, 4, size=q)
+    so, ro = _offsets(s), _offsets(r)
+    keep = oracle.support(q, law)
+    M = 13
+    X = _rand_ints(rng, (M, s.sum()))
+    W = _rand_ints(rng, (s.sum(), r.sum()))
+    G = _rand_ints(rng, (M, r.sum()))
+    types = rng.integers(0, q - 1, size=M) if q > 1 else np.zeros(M, int)     # the last type is absent
+    Y = oracle.proj(X, types, W, s, r, keep=keep)
+    dX = oracle.proj_vjp_x(G, types, W, s, r, keep=keep)
+    dW = oracle.proj_vjp_w(X, G, types, s, r, keep=keep)
+    assert np.sum(Y * G) == np.sum(X * dX) == np.sum(W * dW)
+    if law == "qq":   # W_{q-1, j} (j != q-1) is used by rows of type q-1 only
+        assert not dW[so[q - 1]:so[q], :ro[q - 1]].any()
+    # second probe with one-hot gradients pins single entries, not only the sum
+    for (b, n) in [(0, 0), (M - 1, int(r.sum()) - 1), (5, int(ro[1]))]:
+        E = np.zeros_like(G)
+        E[b, n] = 1.0
+        assert np.array_equal(oracle.proj_vjp_x(E, types, W, s, r, keep=keep)[b],
+                              np.array([(oracle.proj(np.eye(1, int(s.sum()), c), [types[b]], W, s, r, keep=keep))[0, n]
+                                        for c in range(int(s.sum()))]))
+
+
 def test_bad_type_rejected():
     with pytest.raises(oracle.OracleError):
         oracle.proj(np.zeros((2, 2)), [0, 2], np.zeros((2, 2)), [1, 1], [1, 1])
