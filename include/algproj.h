@@ -40,6 +40,7 @@ extern "C" {
 
 typedef struct alg_proj_s *alg_proj_t;
 typedef struct alg_ffn_s *alg_ffn_t;
+typedef struct alg_proj_grad_s *alg_proj_grad_t;
 
 typedef enum {
   ALG_OK = 0,
@@ -237,6 +238,40 @@ alg_status_t alg_ffn_gated_forward(alg_ffn_t h, const void *X, const int32_t *ty
                                    const void *W_gate_up, const void *W_down, void *Y,
                                    alg_dtype_t y_dtype, void *workspace, size_t workspace_bytes,
                                    void *stream);
+
+/* ---- gradient maps of the projection (training) ------------------------------------------------
+ * Appendix "Vector-Jacobian Products", Eqs. vjp-xi ... vjp-wjj: with G the gradient with respect to
+ * Y = X *_q W,
+ *     dX[b, S_k]   = sum_{j : k in B(t_b, j)} G[b, R_j] W[S_k, R_j]^T
+ *     dW[S_k, R_j] = sum_{b : k in B(t_b, j)} X[b, S_k]^T G[b, R_j].
+ * Both keep exactly the block support of the forward table, so each costs the forward MACs
+ * (Section "Scaling and Practical Implementation"); every output element has one owner (no atomics,
+ * bitwise repeatable).  bf16 operands, fp32 accumulation; dX / dW in x_dtype / w_dtype.
+ * A gradient handle is created with the parameters of the forward projection it belongs to
+ * (in_widths = s[q] of X, out_widths = r[q] of Y).  dW runs on the tensor-core path only: every r
+ * must be a multiple of 128 (or of 192), else ALG_ERR_UNSUPPORTED_SHAPE; dX needs every r to be a
+ * multiple of 64 and every s a multiple of 128 (or 192) for that path and otherwise runs on the
+ * SIMT kernel.  A custom table must give every weight block at least one row type that uses it.
+ *   grad_input : W is the forward bank (K x N, ldw >= N), used transposed in place.
+ *   grad_weight: dW (K x N, lddw >= N) is overwritten, never accumulated into; blocks whose row
+ *                types are absent from the batch come out zero.  Internally the rows are bucketed
+ *                by type, X is copied transposed and G bucketed (both padded per bucket to a
+ *                multiple of 64 rows with zeros), and one grouped GEMM reduces over the buckets.
+ * Workspace: alg_proj_grad_workspace_bytes(h, M), 256-byte aligned, no initialisation needed. */
+alg_status_t alg_proj_grad_create(alg_proj_grad_t *out, int q, const int32_t *in_widths,
+                                  const int32_t *out_widths, alg_table_t table,
+                                  const uint8_t *custom_keep, alg_schedule_t schedule);
+alg_status_t alg_proj_grad_destroy(alg_proj_grad_t h);
+alg_status_t alg_proj_grad_workspace_bytes(alg_proj_grad_t h, int64_t max_M, size_t *bytes);
+alg_status_t alg_proj_grad_input(alg_proj_grad_t h, const void *G, int64_t ldg, const int32_t *types,
+                                 int64_t M, const void *W, int64_t ldw, void *dX, int64_t lddx,
+                                 alg_dtype_t x_dtype, void *workspace, size_t workspace_bytes,
+                                 void *stream);
+alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx, const void *G,
+                                  int64_t ldg, const int32_t *types, int64_t M, void *dW,
+                                  int64_t lddw, alg_dtype_t w_dtype, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+alg_status_t alg_proj_grad_last_status(alg_proj_grad_t h, void *stream, alg_status_t *status);
 
 /* Same computation with X, types and Y in HOST memory (pinned memory makes the copies
  * asynchronous).  Copies X and types to device staging inside the workspace, runs the

@@ -35,7 +35,8 @@ EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
     "alg_proj_forward_static", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
-    "alg_ffn_gated_create", "alg_ffn_gated_forward", "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
+    "alg_ffn_gated_create", "alg_ffn_gated_forward", "alg_proj_grad_create", "alg_proj_grad_destroy",
+    "alg_proj_grad_workspace_bytes", "alg_proj_grad_input", "alg_proj_grad_weight", "alg_proj_grad_last_status", "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
 ]
 
 _lib = None
@@ -70,6 +71,12 @@ def lib() -> ctypes.CDLL:
         L.alg_proj_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.alg_ffn_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
         L.alg_ffn_destroy.argtypes = [vp]
+        L.alg_proj_grad_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, vp, i32]
+        L.alg_proj_grad_destroy.argtypes = [vp]
+        L.alg_proj_grad_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_proj_grad_input.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i64, i32, vp, ctypes.c_size_t, vp]
+        L.alg_proj_grad_weight.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i64, i32, vp, ctypes.c_size_t, vp]
+        L.alg_proj_grad_last_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.alg_ffn_gated_create.argtypes = [ctypes.POINTER(vp), i32, vp, vp, i32, i32, vp, i32]
         L.alg_ffn_gated_forward.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_ffn_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
@@ -311,3 +318,49 @@ class GatedFFN(FFN):
 
     def forward_host(self, *a, **k):
         raise NotImplementedError("the gated FFN has no host entry point")
+
+
+class ProjGrad(_Handle):
+    """alg_proj_grad_* : the two gradient maps of Y = X *_q W (dX from G and W, dW from X and G)."""
+    _destroy = "alg_proj_grad_destroy"
+
+    def __init__(self, in_widths, out_widths, table="qq", custom_keep=None, schedule="explicit"):
+        super().__init__()
+        self.q = len(in_widths)
+        self.K, self.N = sum(in_widths), sum(out_widths)
+        self.schedule = _SCHEDS[schedule]
+        buf, keep = _keep_arg(table, custom_keep, self.q)
+        s, r = _widths(in_widths), _widths(out_widths)
+        _check(lib().alg_proj_grad_create(ctypes.byref(self._h), self.q, ctypes.cast(s, ctypes.c_void_p),
+                                          ctypes.cast(r, ctypes.c_void_p), _TABLES[table], keep, self.schedule),
+               "alg_proj_grad_create")
+
+    def workspace_bytes(self, max_M: int) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_proj_grad_workspace_bytes(self._h, max_M, ctypes.byref(out)), "alg_proj_grad_workspace_bytes")
+        return out.value
+
+    def grad_input(self, G, types, W, out=None, out_dtype=None, workspace=None, stream=None):
+        M = G.shape[0]
+        if out is None:
+            out = torch.empty((M, self.K), dtype=out_dtype or G.dtype, device=G.device)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(M), G.device)
+        _check(lib().alg_proj_grad_input(self._h, _ptr(G), G.stride(0) if M else self.N, _ptr(types), M, _ptr(W), W.stride(0),
+                                         _ptr(out), out.stride(0) if M else self.K, _DTYPES[out.dtype], _ptr(ws), ws.numel(),
+                                         _stream(stream)), "alg_proj_grad_input")
+        return out
+
+    def grad_weight(self, X, G, types, out=None, out_dtype=torch.float32, workspace=None, stream=None):
+        M = X.shape[0]
+        if out is None:
+            out = torch.empty((self.K, self.N), dtype=out_dtype, device=X.device)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(M), X.device)
+        _check(lib().alg_proj_grad_weight(self._h, _ptr(X), X.stride(0) if M else self.K, _ptr(G), G.stride(0) if M else self.N,
+                                          _ptr(types), M, _ptr(out), out.stride(0), _DTYPES[out.dtype], _ptr(ws), ws.numel(),
+                                          _stream(stream)), "alg_proj_grad_weight")
+        return out
+
+    def last_status(self, stream=None) -> int:
+        s = ctypes.c_int()
+        _check(lib().alg_proj_grad_last_status(self._h, _stream(stream), ctypes.byref(s)), "alg_proj_grad_last_status")
+        return s.value

@@ -43,6 +43,8 @@ struct alg_proj_s {
   // row type has enough rows to fill such tiles.  Its tile classes (128 columns wide) live in
   // `tab_tall` when the regular tile width is not 128.
   bool gated = false;       // SwiGLU up projection over the merged [W_gate | W_up] bank (N = F, W has 2 F columns)
+  bool w_kmajor = false;    // input-gradient pass: W (N x K here) is used transposed
+  bool dyn_segments = false;  // weight-gradient pass: the reduction segments are the padded row buckets of the call
   bool tall_ok = false;
   DevTable tab_tall;
   DevTable *d_tab_tall = nullptr;
@@ -72,6 +74,15 @@ struct alg_ffn_s {
   bool fd_ok = false;
   FfnDecodePlan fd = {};
   unsigned int *d_counters = nullptr;
+};
+
+// Both gradient maps of one forward projection (s[q] -> r[q]).
+struct alg_proj_grad_s {
+  alg_proj_s dx;   // G (M x N) -> dX (M x K): groups swapped, support transposed, W used transposed
+  alg_proj_s dw;   // rows = the K input features typed by their group, reduction over the padded row buckets
+  int q = 0, K = 0, N = 0;
+  alg_schedule_t sched = ALG_SCHED_EXPLICIT;
+  int *d_feat_offsets = nullptr;   // [q+2] offsets of the feature groups: the "row buckets" of the dW problem
 };
 
 namespace {
@@ -148,6 +159,7 @@ alg_status_t configure_kernels(alg_proj_s &p) {
     p.tile_n = 128;
     p.pair_kernel = false;
   }
+  if (p.w_kmajor || p.dyn_segments) p.pair_kernel = false;   // the gradient passes run on the one-CTA kernel
   if (p.opt_kernel == 1) p.pair_kernel = false;
   if (p.opt_kernel == 2) {
     if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
@@ -260,7 +272,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
       if (cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming) != cudaSuccess) return ALG_ERR_CUDA;
     }
   }
-  if (dtype == ALG_BF16 && !p.gated) {
+  if (dtype == ALG_BF16 && !p.gated && !p.w_kmajor && !p.dyn_segments) {
     p.decode_ok = decode_plan(q, p.s, p.K, p.N, p.num_sms, &p.decode);
     for (int g = 0; g < q && p.decode_ok; ++g)
       if (p.r[g] % p.decode.sn) p.decode_ok = false;
@@ -441,6 +453,8 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.b_3d = 0;
   a.a_box_256 = 0;
   a.gated_f = p.gated ? p.N : 0;
+  a.w_kmajor = p.w_kmajor ? 1 : 0;
+  a.dyn_so = nullptr;
   a.y_staged = 0;
   a.plan = nullptr;
   a.plan_stride = a.plan_rounds = a.plan_tag = 0;
@@ -608,7 +622,7 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   if (M == 0) return ALG_OK;
   if (!X || !W || !Y || !workspace) return ALG_ERR_INVALID_ARG;
   if (h->sched == ALG_SCHED_EXPLICIT && !types) return ALG_ERR_INVALID_ARG;
-  if (ldx < h->K || ldw < h->N || ldy < h->N) return ALG_ERR_INVALID_ARG;
+  if (ldx < h->K || ldw < (h->w_kmajor ? h->K : h->N) || ldy < h->N) return ALG_ERR_INVALID_ARG;
   if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
   if ((int)act < 0 || (int)act > 2) return ALG_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255u) != 0) return ALG_ERR_INVALID_ARG;
@@ -685,6 +699,214 @@ static alg_status_t read_status(int *d_status, void *stream, alg_status_t *statu
 alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *status) {
   if (!h) return ALG_ERR_INVALID_ARG;
   return read_status(h->d_status, stream, status);
+}
+
+// ---- gradient maps (Appendix "Vector-Jacobian Products") ------------------------------------------
+
+static alg_status_t support_of(int q, alg_table_t table, const uint8_t *custom, std::vector<uint8_t> &keep) {
+  if (q < 1 || q > kMaxQ) return ALG_ERR_INVALID_ARG;
+  if (table == ALG_TABLE_Q2POW && (q & (q - 1)) != 0) return ALG_ERR_INVALID_ARG;
+  if (table == ALG_TABLE_CUSTOM && !custom) return ALG_ERR_INVALID_ARG;
+  keep.assign((size_t)q * q * q, 0);
+  for (int i = 0; i < q; ++i)
+    for (int j = 0; j < q; ++j)
+      for (int k = 0; k < q; ++k)
+        keep[((size_t)i * q + j) * q + k] = table == ALG_TABLE_DENSE   ? 1
+                                            : table == ALG_TABLE_QQ    ? (k == i || k == j)
+                                            : table == ALG_TABLE_Q2POW ? (((k ^ i) & (k ^ j)) == 0)
+                                                                       : custom[((size_t)i * q + j) * q + k] != 0;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_grad_create(alg_proj_grad_t *out, int q, const int32_t *in_widths, const int32_t *out_widths,
+                                  alg_table_t table, const uint8_t *custom_keep, alg_schedule_t schedule) {
+  if (!out) return ALG_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!in_widths || !out_widths) return ALG_ERR_INVALID_ARG;
+  if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM && table != ALG_TABLE_Q2POW)
+    return ALG_ERR_INVALID_ARG;
+  std::vector<uint8_t> keep;
+  alg_status_t s = support_of(q, table, custom_keep, keep);
+  if (s != ALG_OK) return s;
+  // dX: type i, output group k (of X), reduction over the output groups j with k in B(i,j)
+  // dW: "row type" = feature group k, output group j, reduction over the row types i with k in B(i,j)
+  std::vector<uint8_t> keep_dx((size_t)q * q * q), keep_dw((size_t)q * q * q);
+  for (int i = 0; i < q; ++i)
+    for (int j = 0; j < q; ++j)
+      for (int k = 0; k < q; ++k) {
+        keep_dx[((size_t)i * q + k) * q + j] = keep[((size_t)i * q + j) * q + k];
+        keep_dw[((size_t)k * q + j) * q + i] = keep[((size_t)i * q + j) * q + k];
+      }
+  alg_proj_grad_s *g = new (std::nothrow) alg_proj_grad_s();
+  if (!g) return ALG_ERR_INVALID_ARG;
+  g->q = q;
+  g->sched = schedule;
+  g->dx.w_kmajor = true;
+  s = init_proj(g->dx, q, out_widths, in_widths, ALG_BF16, ALG_TABLE_CUSTOM, keep_dx.data(), schedule, nullptr);
+  if (s == ALG_OK) {
+    int32_t seg[kMaxQ];
+    for (int e = 0; e < q; ++e) seg[e] = kTcBlockK;   // placeholders: the segments of a call are its padded row buckets
+    g->dw.dyn_segments = true;
+    s = init_proj(g->dw, q, seg, out_widths, ALG_BF16, ALG_TABLE_CUSTOM, keep_dw.data(), ALG_SCHED_EXPLICIT, g->dx.d_status);
+    if (s == ALG_ERR_INVALID_ARG) s = ALG_ERR_UNSUPPORTED_SHAPE;   // a weight block no row type ever uses
+  }
+  if (s == ALG_OK && !(use_tc(g->dw) && g->dw.tc_ok)) s = ALG_ERR_UNSUPPORTED_SHAPE;   // dW has no SIMT path
+  if (s == ALG_OK) {
+    g->K = g->dx.N, g->N = g->dx.K;
+    int offs[kMaxQ + 2];
+    for (int e = 0; e <= q; ++e) offs[e] = g->dx.tab.ro[e];   // feature-group offsets
+    offs[q + 1] = g->K;
+    if (cudaMalloc(&g->d_feat_offsets, (q + 2) * sizeof(int)) != cudaSuccess ||
+        cudaMemcpy(g->d_feat_offsets, offs, (q + 2) * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+      s = ALG_ERR_CUDA;
+  }
+  if (s != ALG_OK) {
+    if (g->d_feat_offsets) cudaFree(g->d_feat_offsets);
+    free_proj(g->dw);
+    free_proj(g->dx);
+    delete g;
+    return s;
+  }
+  *out = g;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_grad_destroy(alg_proj_grad_t h) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  if (h->d_feat_offsets) cudaFree(h->d_feat_offsets);
+  free_proj(h->dw);
+  free_proj(h->dx);
+  delete h;
+  return ALG_OK;
+}
+
+namespace {
+int padded_rows(const alg_proj_grad_s &g, int64_t M) { return (int)((M + 63) / 64 * 64) + 64 * g.q; }
+struct GradLayout {
+  size_t hdr, chunks, perm, xt, gp, total;
+};
+GradLayout grad_layout(const alg_proj_grad_s &g, int64_t M) {
+  GradLayout L;
+  size_t off = 0;
+  L.hdr = off;
+  off = align_up(off + sizeof(WsHeader));
+  L.chunks = off;
+  off = align_up(off + (size_t)kMaxBucketChunks * (g.q + 1) * sizeof(int));
+  L.perm = off;
+  off = align_up(off + (size_t)M * sizeof(int));
+  const size_t mp = (size_t)padded_rows(g, M);
+  L.xt = off;
+  off = align_up(off + mp * g.K * 2, 1024);
+  L.gp = off;
+  off = align_up(off + mp * g.N * 2, 1024);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+alg_status_t alg_proj_grad_workspace_bytes(alg_proj_grad_t h, int64_t max_M, size_t *bytes) {
+  if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  *bytes = std::max(layout(h->dx, nullptr, max_M).total, grad_layout(*h, max_M).total);
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_grad_input(alg_proj_grad_t h, const void *G, int64_t ldg, const int32_t *types, int64_t M,
+                                 const void *W, int64_t ldw, void *dX, int64_t lddx, alg_dtype_t x_dtype, void *workspace,
+                                 size_t workspace_bytes, void *stream) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  return alg_proj_forward(&h->dx, G, ldg, types, M, W, ldw, nullptr, ALG_ACT_NONE, dX, lddx, x_dtype, workspace,
+                          workspace_bytes, stream);
+}
+
+alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx, const void *G, int64_t ldg,
+                                  const int32_t *types, int64_t M, void *dW, int64_t lddw, alg_dtype_t w_dtype,
+                                  void *workspace, size_t workspace_bytes, void *stream) {
+  if (!h || M < 0 || M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (!X || !G || !dW || !workspace) return ALG_ERR_INVALID_ARG;
+  if (h->sched == ALG_SCHED_EXPLICIT && !types && M > 0) return ALG_ERR_INVALID_ARG;
+  if (ldx < h->K || ldg < h->N || lddw < h->N) return ALG_ERR_INVALID_ARG;
+  if (w_dtype != ALG_F32 && w_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(G) || !aligned16(dW) || ldx % 8 || ldg % 8 || (lddw * elem_bytes(w_dtype)) % 16)
+    return ALG_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255u) != 0) return ALG_ERR_INVALID_ARG;
+  const GradLayout L = grad_layout(*h, M);
+  if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)workspace;
+  alg_proj_s &p = h->dw;
+  const int mp = padded_rows(*h, M);
+  WsHeader *hdr = (WsHeader *)(ws + L.hdr);
+  // 1. row buckets of this batch (also for the cyclic schedule: the copies below need the permutation)
+  BucketArgs b;
+  b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
+  b.M = (int)M;
+  b.q = h->q;
+  b.chunk_rows = bucket_chunk_rows(M);
+  b.hdr = hdr;
+  b.chunk_counts = (int *)(ws + L.chunks);
+  b.perm = (int *)(ws + L.perm);
+  b.status = p.d_status;
+  b.sync = (unsigned int *)(p.d_status + 2);
+  b.wait_limit = p.wait_limit;
+  b.Y = nullptr;   // nothing to zero: a row with an out-of-range type simply contributes to no block
+  b.ldy = 0, b.N = 0, b.y_elem_bytes = 0;
+  if (M > 0 && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (M == 0) {   // no rows: every block of dW is zero
+    return cuda_status(cudaMemset2DAsync(dW, (size_t)lddw * elem_bytes(w_dtype), 0, (size_t)h->N * elem_bytes(w_dtype),
+                                         (size_t)h->K, st));
+  }
+  // 2. padded, bucketed copies: X transposed (K x m_pad), G as it is (m_pad x N); pad rows are zero
+  if (launch_gather_transpose_padded(X, ldx, hdr, b.perm, h->q, mp, h->K, ws + L.xt, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (launch_gather_rows_padded(G, ldg, hdr, b.perm, h->q, mp, h->N, ws + L.gp, st) != cudaSuccess) return ALG_ERR_CUDA;
+  // 3. the grouped GEMM: rows = input features (type = their group), reduction over the padded buckets
+  ProjArgs a;
+  const TcChoice tc = {tile_m_of(p), tile_n_of(p), &p.tab, p.d_tab};
+  const DevTable &tab = p.tab;
+  a.tab = tc.d_tab;
+  a.offsets = h->d_feat_offsets;
+  a.cyclic_rows = 0;
+  a.n_classes = tab.n_classes;
+  a.st.valid = p.q <= kParamQ && tab.n_classes <= 2 * kParamQ * kParamQ;
+  if (a.st.valid) {
+    for (int e = 0; e <= p.q; ++e) a.st.so[e] = tab.so[e], a.st.ro[e] = tab.ro[e];
+    for (int e = 0; e < p.q * p.q; ++e) a.st.keep[e] = tab.keep[e];
+    for (int e = 0; e < tab.n_classes; ++e) a.st.cls[e] = tab.cls[e];
+  }
+  a.geom.tile_m = tc.tile_m;
+  a.geom.tile_m_log2 = 7;
+  a.q = p.q;
+  a.perm = nullptr;
+  a.in_perm = nullptr;
+  a.X = ws + L.xt;
+  a.ldx = mp;
+  a.W = ws + L.gp;
+  a.ldw = h->N;
+  a.bias = nullptr;
+  a.act = (int)ALG_ACT_NONE;
+  a.Y = dW;
+  a.ldy = lddw;
+  a.y_bf16 = w_dtype == ALG_BF16;
+  a.M = h->K;          // rows of this GEMM = input features
+  a.K = mp;            // reduction = padded rows of the batch
+  a.N = h->N;
+  a.status = p.d_status;
+  a.a_cyclic_rows = 0;
+  a.out_cyclic_rows = 0;
+  a.b_3d = 0;
+  a.a_box_256 = 0;
+  a.gated_f = 0;
+  a.w_kmajor = 0;
+  a.dyn_so = hdr->pad_offsets;
+  a.y_staged = 0;
+  a.plan = nullptr;
+  a.plan_stride = a.plan_rounds = a.plan_tag = 0;
+  a.wait_limit = p.wait_limit;
+  return cuda_status(launch_proj_tc(a, tc.tile_n, p.n_workers, st));
+}
+
+alg_status_t alg_proj_grad_last_status(alg_proj_grad_t h, void *stream, alg_status_t *status) {
+  if (!h) return ALG_ERR_INVALID_ARG;
+  return read_status(h->dx.d_status, stream, status);
 }
 
 static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, const int32_t *f_widths,

@@ -21,6 +21,16 @@ __device__ __forceinline__ int row_type(const BucketArgs &a, int row) {
   return (t < 0 || t >= a.q) ? a.q : t;  // pseudo-type q collects out-of-range rows
 }
 
+// offsets of the same buckets when each is padded to a multiple of 64 rows
+__device__ __forceinline__ void write_pad_offsets(WsHeader *hdr, const int *offset, int q) {
+  int run = 0;
+  for (int t = 0; t < q; ++t) {
+    hdr->pad_offsets[t] = run;
+    run += (offset[t + 1] - offset[t] + 63) & ~63;
+  }
+  hdr->pad_offsets[q] = run;
+}
+
 // Kernel 1: per-chunk histograms of the row types (pseudo-type q = out of range).
 __global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
   __shared__ int s_cnt[kMaxQ + 1];
@@ -108,8 +118,10 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
     __syncthreads();
   }
 
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0) {
     for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
+    if (tid == 0) write_pad_offsets(a.hdr, s_offset, a.q);
+  }
 }
 
 // One-pass variant for M <= 65536 (at most 64 CTAs of 1024 threads, one row per thread): every row
@@ -202,8 +214,10 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
       for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
     }
   }
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0) {
     for (int t2 = tid; t2 <= nt; t2 += kFusedThreads) a.hdr->offsets[t2] = s_offset[t2];
+    if (tid == 0) write_pad_offsets(a.hdr, s_offset, a.q);
+  }
 }
 
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ X, int64_t ldx_v,
@@ -226,6 +240,63 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restric
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         if (v0 + u * 32 < vecs) dst[v0 + u * 32] = r[u];
+    }
+  }
+}
+
+// padded row p -> original row (or -1 for a pad row / beyond the last bucket)
+__device__ __forceinline__ int padded_source_row(const WsHeader *hdr, const int *perm, int q, int p) {
+  int t = 0;
+  while (t + 1 < q && hdr->pad_offsets[t + 1] <= p) ++t;
+  const int rank = p - hdr->pad_offsets[t];
+  const int rows = hdr->offsets[t + 1] - hdr->offsets[t];
+  return (p < hdr->pad_offsets[q] && rank < rows) ? perm[hdr->offsets[t] + rank] : -1;
+}
+
+__global__ void __launch_bounds__(256) gather_rows_padded_kernel(const uint4 *__restrict__ G, int64_t ldg_v,
+                                                                 const WsHeader *__restrict__ hdr,
+                                                                 const int *__restrict__ perm, int q, int m_pad, int vecs,
+                                                                 uint4 *__restrict__ Gp) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // perm and the offsets come from the bucketing kernel
+  const int lane = threadIdx.x & 31;
+  const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int n_warps = (gridDim.x * blockDim.x) >> 5;
+  for (int p = warp_global; p < m_pad; p += n_warps) {
+    const int src_row = padded_source_row(hdr, perm, q, p);
+    uint4 *dst = Gp + (int64_t)p * vecs;
+    for (int v0 = lane; v0 < vecs; v0 += 32) dst[v0] = src_row >= 0 ? __ldg(G + (int64_t)src_row * ldg_v + v0) : make_uint4(0, 0, 0, 0);
+  }
+}
+
+// XpT[c, p] = X[source(p), c]: 64 padded rows x 64 columns per CTA through shared memory, so that both the
+// reads (along c) and the writes (along p) are contiguous.
+__global__ void __launch_bounds__(256) gather_transpose_padded_kernel(const __nv_bfloat16 *__restrict__ X, int64_t ldx,
+                                                                      const WsHeader *__restrict__ hdr,
+                                                                      const int *__restrict__ perm, int q, int m_pad, int K,
+                                                                      __nv_bfloat16 *__restrict__ XpT) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  __shared__ int s_src[64];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int p0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+  const int tid = threadIdx.x;
+  if (tid < 64) s_src[tid] = p0 + tid < m_pad ? padded_source_row(hdr, perm, q, p0 + tid) : -1;
+  __syncthreads();
+  for (int e = tid; e < 64 * 32; e += 256) {   // 64 rows x 32 column pairs
+    const int r = e >> 5, cp = (e & 31) * 2;
+    const int src_row = s_src[r];
+    __nv_bfloat162 v = __floats2bfloat162_rn(0.f, 0.f);
+    if (src_row >= 0 && c0 + cp < K) v = *(const __nv_bfloat162 *)(X + (int64_t)src_row * ldx + c0 + cp);
+    tile[r][cp] = v.x, tile[r][cp + 1] = v.y;
+  }
+  __syncthreads();
+  for (int e = tid; e < 64 * 32; e += 256) {   // 64 columns x 32 row pairs
+    const int c = e >> 5, rp = (e & 31) * 2;
+    if (c0 + c < K && p0 + rp < m_pad) {
+      __nv_bfloat162 v;
+      v.x = tile[rp][c], v.y = tile[rp + 1][c];
+      *(__nv_bfloat162 *)(XpT + (int64_t)(c0 + c) * m_pad + p0 + rp) = v;
     }
   }
 }
@@ -268,6 +339,32 @@ cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int 
   count_launch(1);
   return launch_pdl(gather_rows_kernel, grid, 256, st, (const uint4 *)X, (int64_t)(ldx * elem_bytes / 16), perm, M, vecs,
                     (uint4 *)Xb);
+}
+
+cudaError_t launch_gather_rows_padded(const void *G, int64_t ldg, const WsHeader *hdr, const int *perm, int q, int m_pad,
+                                      int N, void *Gp, cudaStream_t st) {
+  const int vecs = N * 2 / 16;
+  int grid = ceil_div(m_pad, 8);
+  if (grid > 148 * 8) grid = 148 * 8;
+  count_launch(1);
+  return launch_pdl(gather_rows_padded_kernel, grid, 256, st, (const uint4 *)G, (int64_t)(ldg * 2 / 16), hdr, perm, q, m_pad,
+                    vecs, (uint4 *)Gp);
+}
+
+cudaError_t launch_gather_transpose_padded(const void *X, int64_t ldx, const WsHeader *hdr, const int *perm, int q,
+                                           int m_pad, int K, void *XpT, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ceil_div(m_pad, 64), ceil_div(K, 64), 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  count_launch(1);
+  return cudaLaunchKernelEx(&cfg, gather_transpose_padded_kernel, (const __nv_bfloat16 *)X, ldx, hdr, perm, q, m_pad, K,
+                            (__nv_bfloat16 *)XpT);
 }
 
 }  // namespace algproj

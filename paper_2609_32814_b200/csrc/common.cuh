@@ -54,9 +54,12 @@ struct TileRec {
 // Fixed-size header at the start of every workspace.
 struct WsHeader {
   int offsets[kMaxQ + 2];  // offsets[t] = first bucketed row of type t; [q] = first bad row; [q+1] = M
-  int pad[30];
+  // the same buckets with every bucket padded to a multiple of 64 rows (weight-gradient pass):
+  // pad_offsets[t] = first padded row of type t, [q] = end of the last bucket
+  int pad_offsets[kMaxQ + 1];
 };
-static_assert(sizeof(WsHeader) == 256, "workspace header is one 256-byte line");
+static_assert(kMaxQ + 2 + kMaxQ + 1 <= 72, "workspace header layout");
+static_assert(sizeof(WsHeader) <= 512, "workspace header stays within its slot");
 
 struct TileGeom {
   int tile_m;        // rows per tile (a power of two)
@@ -85,6 +88,13 @@ cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st);
 // Xb[d, 0:K] = X[perm[d], 0:K] (16-byte vectors; K*elem_bytes % 16 == 0)
 cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int M, int K,
                                int elem_bytes, void *Xb, cudaStream_t st);
+// Weight-gradient pass (bf16): bucketed copies with every bucket padded to a multiple of 64 rows, pad
+// rows zero.  Gp[p, 0:N] = G[perm[..], 0:N] for the padded row p;  XpT[c, p] = X[perm[..], c]
+// (transposed: K x m_pad, leading dimension m_pad).  m_pad >= padded total (hdr->pad_offsets[q]).
+cudaError_t launch_gather_rows_padded(const void *G, int64_t ldg, const WsHeader *hdr, const int *perm, int q, int m_pad,
+                                      int N, void *Gp, cudaStream_t st);
+cudaError_t launch_gather_transpose_padded(const void *X, int64_t ldx, const WsHeader *hdr, const int *perm, int q,
+                                           int m_pad, int K, void *XpT, cudaStream_t st);
 
 // Interaction table of a small-q handle, carried by value in the kernel parameters so that a
 // kernel prologue needs no global metadata load.
@@ -128,6 +138,11 @@ struct ProjArgs {
   int out_cyclic_rows;
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   int a_box_256;          // A tensor map carries 256-row boxes (one-CTA kernel with 256-row tiles)
+  // Gradient passes.  w_kmajor: W is used transposed (B operand K-major; dX = G W^T): the reduction
+  // runs over the COLUMNS of W, the output columns are its rows.  dyn_so: the q+1 offsets of the
+  // reduction segments come from device memory (padded row buckets; dW = X^T G reduces over rows).
+  int w_kmajor;
+  const int *dyn_so;
   // Gated (SwiGLU) up projection: W is the merged bank [W_gate | W_up] with 2 * gated_f columns, a
   // tile accumulates 128 gate columns and the matching 128 up columns side by side, the epilogue
   // stores silu(gate) * up; N = gated_f is the width of the output.  0 = ordinary projection.

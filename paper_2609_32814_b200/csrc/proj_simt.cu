@@ -71,7 +71,8 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const ProjArgs a) {
           As[kk][r] = v;
           int kb = idx >> 6, c = idx & 63;
           float w = 0.f;
-          if (k0 + kb < k_end && c < n_valid) w = to_f32(W[(int64_t)(k0 + kb) * a.ldw + rec.n0 + c]);
+          if (k0 + kb < k_end && c < n_valid)
+            w = to_f32(a.w_kmajor ? W[(int64_t)(rec.n0 + c) * a.ldw + k0 + kb] : W[(int64_t)(k0 + kb) * a.ldw + rec.n0 + c]);
           Bs[kb][c] = w;
         }
         __syncthreads();

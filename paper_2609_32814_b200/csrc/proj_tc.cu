@@ -148,13 +148,17 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int e = lane; e < q * q; e += 32) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
   } else if (warp == 4) {
-    for (int e = lane; e <= q; e += 32) ctl->so[e] = a.st.valid ? a.st.so[e] : tab->so[e];
+    if (a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");   // segment offsets written by the bucketing kernel
+    for (int e = lane; e <= q; e += 32) ctl->so[e] = a.dyn_so ? a.dyn_so[e] : a.st.valid ? a.st.so[e] : tab->so[e];
   } else if (warp == 5) {
+    if (a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int e = lane; e < q * q; e += 32) {
       const uint32_t mask = a.st.valid ? a.st.keep[e] : tab->keep[e];
       int n = 0;
       for (int k = 0; k < q; ++k)
-        if ((mask >> k) & 1u) n += ((a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k])) / kTcBlockK;
+        if ((mask >> k) & 1u)
+          n += (a.dyn_so ? a.dyn_so[k + 1] - a.dyn_so[k] : a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k]) /
+               kTcBlockK;
       ctl->nkb[e] = (uint16_t)n;   // for tile records decoded after the precomputed ones
     }
   }
@@ -182,9 +186,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int r = lane; r < a.plan_rounds; r += 32) recs[r] = a.plan[1 + (size_t)blockIdx.x * a.plan_stride + r];
       if (lane == 0) tm->seq_rounds = a.plan_rounds, tm->seq_valid = a.plan_rounds, tm->total = 0;
     } else {
-      if (a.offsets) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
+      if (a.offsets || a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
       tile_plan_warp(tm, recs, kSeqCap, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom, blockIdx.x,
-                     gridDim.x, kTcBlockK);
+                     gridDim.x, kTcBlockK, a.dyn_so);
     }
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -236,6 +240,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
               else tma_load_2d(sa, &tmA, bar, k0, a_row);
+            } else if (a.w_kmajor) {
+              // W used transposed: TILE_N rows of W (the output columns) x 64 of its columns (the reduction)
+              tma_load_2d(sa + C::kABytes, &tmB, bar, k0, n0);
             } else if (GATED) {
               // two boxes of two 64-column chunks: the tile's gate columns, then its up columns
               tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
@@ -263,7 +270,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
     const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, 1024);
-    const uint64_t db0 = make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
+    // B: the canonical bank lands MN-major (64-column chunks 8 KB apart, 16 k-rows = two 8-row groups
+    // = 128 descriptor units per K step); used transposed it lands K-major like A (32 bytes per K step)
+    const uint64_t db0 = a.w_kmajor ? make_smem_desc(smem_u32(smem) + C::kABytes, 16, 1024)
+                                    : make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
+    const uint32_t idesc = a.w_kmajor ? (C::kIdesc & ~(1u << 16)) : C::kIdesc;
+    const uint64_t db_step = a.w_kmajor ? 2 : 128;
     TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
     while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
       ++round;
@@ -291,8 +303,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kk = 0; kk < kTcBlockK / 16; ++kk)
 #pragma unroll
             for (int h = 0; h < C::kHalves; ++h)
-              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * 1024), db + (uint64_t)(kk * 128),
-                          C::kIdesc, (kb | kk) ? 1u : 0u);
+              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * 1024), db + (uint64_t)kk * db_step,
+                          idesc, (kb | kk) ? 1u : 0u);
           tc_commit(empty0 + 8u * (uint32_t)stage);
         }
         __syncwarp();
@@ -318,6 +330,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int r = (C::kHalves == 2 ? half * 128 : 0) + quad * 32 + lane;   // row of the tile this lane holds
       int64_t out_row = -1;
       const int tile_rows = rec.rows & 0xFFFF;
+      // a tile without any K block (weight-gradient pass, row type absent from the batch): nothing was
+      // accumulated, its result is zero
+      const bool empty_tile = ((uint32_t)rec.rows >> 16) == 0u;
       if (r < tile_rows) {
         if (a.out_cyclic_rows) {
           const int i = (rec.pair & 0xFFFF) / q;
@@ -382,7 +397,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (e == 0 && lane == 0) ALG_TRACE(2, 3);
           float f[32];
 #pragma unroll
-          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          for (int x = 0; x < 32; ++x) f[x] = empty_tile ? 0.f : __uint_as_float(v[x]);
           finish_32(f, a, col_base + c0);
           uint32_t w[16];
           pack_bf16_32(f, w);
@@ -416,7 +431,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (out_row >= 0) {
           float f[32];
 #pragma unroll
-          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          for (int x = 0; x < 32; ++x) f[x] = empty_tile ? 0.f : __uint_as_float(v[x]);
           finish_and_store_32(f, a, out_row, col_base + c0);
         }
       }
@@ -465,9 +480,16 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   cudaError_t e = make_map_a(&tmA, a);
   if (e != cudaSuccess) return e;
   ProjArgs b = a;
-  b.b_3d = make_map_b3d(&tmB, a, GATED ? 2 : TILE_N / 64) == cudaSuccess;
+  if (a.w_kmajor) {   // W is N x K here (rows = output columns, contiguous along the reduction): boxes of 64 x TILE_N
+    if (GATED) return cudaErrorInvalidValue;
+    b.b_3d = 0;
+    e = make_map_2d(&tmB, a.W, (uint64_t)a.K, (uint64_t)a.N, (uint64_t)a.ldw * 2, kTcBlockK, TILE_N);
+    if (e != cudaSuccess) return e;
+  } else {
+    b.b_3d = make_map_b3d(&tmB, a, GATED ? 2 : TILE_N / 64) == cudaSuccess;
+  }
   if (GATED && !b.b_3d) return cudaErrorInvalidValue;
-  if (!b.b_3d) {
+  if (!b.b_3d && !a.w_kmajor) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
     if (e != cudaSuccess) return e;
   }

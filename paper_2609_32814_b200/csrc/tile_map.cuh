@@ -142,9 +142,11 @@ __device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, TileMap *tm
 // included -- built by ONE warp with warp-level synchronisation only, so that the other warps of
 // the CTA can set up barriers and tensor memory meanwhile and a single CTA barrier ends the
 // prologue.  `keep` / `so` are read from the by-value table when it is valid, else from `tab`.
+// `dyn_so` (optional, device memory): offsets of the reduction segments when they are not the
+// table's (weight-gradient pass: padded row buckets).
 __device__ inline void tile_plan_warp(TileMap *tm, TileRec *recs, int cap, const DevTable *tab, const SmallTable &st,
                                       int q, int nc, const int *offsets, int cyclic_rows, int M, const TileGeom &g,
-                                      int worker, int n_workers, int k_block) {
+                                      int worker, int n_workers, int k_block, const int *dyn_so = nullptr) {
   const int lane = threadIdx.x & 31;
   if (lane == 0) tm->n_classes = nc, tm->q = q;
   for (int t = lane; t <= q + 1; t += 32) tm->offsets[t] = offsets ? offsets[t] : (t <= q ? t * cyclic_rows : M);
@@ -183,7 +185,8 @@ __device__ inline void tile_plan_warp(TileMap *tm, TileRec *recs, int cap, const
       const uint32_t mask = st.valid ? st.keep[pr] : tab->keep[pr];
       int n = 0;
       for (int k = 0; k < q; ++k)
-        if ((mask >> k) & 1u) n += (st.valid ? st.so[k + 1] - st.so[k] : tab->so[k + 1] - tab->so[k]) / k_block;
+        if ((mask >> k) & 1u)
+          n += (dyn_so ? dyn_so[k + 1] - dyn_so[k] : st.valid ? st.so[k + 1] - st.so[k] : tab->so[k + 1] - tab->so[k]) / k_block;
       rec.rows |= n << 16;
     }
     recs[r] = rec;
