@@ -15,6 +15,7 @@ count only the block GEMMs the rule keeps.
     5q2 5q4 5q8 5q16   scale sweep 4096 -> 16384 -> 4096, M = 32768, i.i.d. row types
     pilot              tensor-square law Q_2 (x) Q_2 at the paper's pilot shape (768 -> 1536 -> 768)
     gpilot g8b         gated (SwiGLU) FFN with merged gate/up bank: the pilot's FFN; 4096 -> 12288 at q=32
+    train2 train8b     forward + both gradient maps of one projection (768 -> 3072 at q=2; 4096 -> 12288 at q=32)
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
 rank runs the same per-GPU batch (weak scaling), time = max over ranks.
@@ -67,6 +68,12 @@ CONFIGS = {
     "g8b": dict(q=32, D=4096, F=12288, M=2048, law="qq", schedule="explicit", gated=True,
                 label="gated FFN 4096->12288->4096 at q=32 (groups of 128 / 384), merged gate/up bank, M=2048 rows, "
                       "i.i.d. row types, bf16"),
+    "train2": dict(q=2, D=768, F=3072, M=8192, law="qq", schedule="cyclic", train=True,
+                   label="training step of one projection: forward + dX + dW of the cfg2 up projection 768->3072, q=2, M=8192 rows, "
+                         "type = position mod 2, bf16"),
+    "train8b": dict(q=32, D=4096, F=12288, M=2048, law="qq", schedule="explicit", train=True,
+                    label="training step of one projection: forward + dX + dW of 4096->12288 at q=32 (groups of 128 / 384), "
+                          "M=2048 rows, i.i.d. row types, bf16"),
     "4": dict(q=2, D=768, F=3072, M=64, law="qq", schedule="explicit",
               label="cfg4: KV-cached decode step, q=2 FFN 768->3072->768, M in {1,8,32,64}, type = position mod 2, bf16"),
 }
@@ -270,7 +277,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-control / explicit-types / decode side measurements")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "gpilot": 300, "g8b": 100, "4": 20}.get(args.config, 20) if args.impl == "ours" else 3
+        args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "gpilot": 300, "g8b": 100, "4": 20, "train2": 200,
+                      "train8b": 100}.get(args.config, 20) if args.impl == "ours" else 3
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else min(args.warmup, 1)
     if args.impl == "reference":
         run_reference(args)
@@ -290,7 +298,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     binding.lib()  # fail loudly if the CUDA library is missing
     ctx = {"world": world, "rank": rank, "local_rank": local_rank, "dist": dist, "torch": torch, "binding": binding}
-    line = run_decode(args, ctx) if args.config == "4" else run_prefill(args, ctx)
+    line = run_decode(args, ctx) if args.config == "4" else run_train(args, ctx) if CONFIGS[args.config].get("train") else run_prefill(args, ctx)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -530,6 +538,129 @@ def run_prefill(args, ctx):
             "roofline": roofline, "cpu_baseline": cpu}
     line.update(extras)
     return line
+
+
+def run_train(args, ctx):
+    """--config train*: a step = forward, input gradient and weight gradient of ONE projection (the
+    matrix products of a training step, three times the forward MACs)."""
+    torch, binding = ctx["torch"], ctx["binding"]
+    world, rank, local_rank = ctx["world"], ctx["rank"], ctx["local_rank"]
+    from paper_2609_32814_b200 import synth
+    import oracle
+    name, cfg = args.config, CONFIGS[args.config]
+    q, M, D, F = cfg["q"], cfg["M"], cfg["D"], cfg["F"]
+    dw_, fw_ = [D // q] * q, [F // q] * q
+    types_h = synth.cyclic_types(M, q, period=1024) if cfg["schedule"] == "cyclic" else synth.uniform_types(synth.seed_for(8, 41), M, q)
+    counts = np.bincount(types_h, minlength=q).tolist()
+    Xh = synth.bf16_round(synth.normal(synth.seed_for(8, 42), (M, D), 1.0))
+    Wh = synth.bf16_round(synth.normal(synth.seed_for(8, 43), (D, F), 0.02))
+    Gh = synth.bf16_round(synth.normal(synth.seed_for(8, 44), (M, F), 1.0))
+    dev = lambda a_: torch.from_numpy(a_).cuda().to(torch.bfloat16)
+    stream = torch.cuda.current_stream()
+    tt = None if cfg["schedule"] == "cyclic" else torch.from_numpy(types_h).cuda()
+
+    def handles(table):
+        return (binding.Proj(dw_, fw_, dtype="bf16", table=table, schedule=cfg["schedule"]),
+                binding.ProjGrad(dw_, fw_, table=table, schedule=cfg["schedule"]))
+    fwd, grad = handles(cfg["law"])
+    flops = 3 * 2 * fwd.macs(counts)
+    set_bytes = (2 * M * D + 2 * D * F + 2 * M * F) * 2 + D * F * 4
+    n_sets = 1 if set_bytes > 2 * L2_BYTES else int(min(6, max(2, math.ceil(4 * L2_BYTES / set_bytes))))
+    sets = []
+    for r in range(n_sets):
+        sets.append({"X": dev(Xh).clone(), "W": dev(Wh).clone(), "G": dev(Gh).clone(),
+                     "Y": torch.empty((M, F), dtype=torch.bfloat16, device="cuda"),
+                     "dX": torch.empty((M, D), dtype=torch.bfloat16, device="cuda"),
+                     "dW": torch.empty((D, F), dtype=torch.float32, device="cuda"),
+                     "ws": torch.empty(max(fwd.workspace_bytes(M), grad.workspace_bytes(M)), dtype=torch.uint8, device="cuda")})
+
+    def step(i, f=fwd, g=grad):
+        s_ = sets[i % n_sets]
+        f.forward(s_["X"], tt, s_["W"], out=s_["Y"], workspace=s_["ws"], stream=stream)
+        g.grad_input(s_["G"], tt, s_["W"], out=s_["dX"], workspace=s_["ws"], stream=stream)
+        g.grad_weight(s_["X"], s_["G"], tt, out=s_["dW"], workspace=s_["ws"], stream=stream)
+
+    def time_steps(n, f=fwd, g=grad, clocks=None):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(n):
+            step(i, f, g)
+            if clocks is not None and i == 0:
+                clocks.arm()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert fwd.last_status() == 0 and grad.last_status() == 0
+    launches0 = binding.launch_count()
+    with ClockSampler(local_rank) as clocks:
+        total_ms = time_steps(args.steps, clocks=clocks)
+    launches = binding.launch_count() - launches0
+    total_ms = max_over_ranks(total_ms, "cuda")
+    # the three parts on their own
+    parts = {}
+    for key, fn in (("forward", lambda s_: fwd.forward(s_["X"], tt, s_["W"], out=s_["Y"], workspace=s_["ws"], stream=stream)),
+                    ("grad_input", lambda s_: grad.grad_input(s_["G"], tt, s_["W"], out=s_["dX"], workspace=s_["ws"], stream=stream)),
+                    ("grad_weight", lambda s_: grad.grad_weight(s_["X"], s_["G"], tt, out=s_["dW"], workspace=s_["ws"], stream=stream))):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(min(args.steps, 50)):
+            fn(sets[i % n_sets])
+        e1.record(stream)
+        torch.cuda.synchronize()
+        parts[key + "_ms"] = e0.elapsed_time(e1) / min(args.steps, 50)
+    peaks = _peaks()
+    region_s = total_ms * 1e-3
+    peak_tf = peaks["bf16_tflops"] if region_s < 0.1 or not peaks["bf16_tflops_sustained"] else peaks["bf16_tflops_sustained"]
+    bytes_step = (3 * M * D + 2 * D * F + 3 * M * F) * 2 + D * F * 4    # X, W, Y | G, W, dX | X, G, dW (fp32)
+    t_tensor, t_hbm = flops / (peak_tf * 1e12), bytes_step / (peaks["hbm_gbs"] * 1e9)
+    value = whole_job_value(flops, world, args.steps, total_ms)
+    if t_tensor >= t_hbm:
+        roofline = {"bound": "tensor", "achieved": value / world, "peak": peak_tf, "unit": "TFLOP/s", "frac": value / world / peak_tf,
+                    "peak_source": f"{peaks['source']} ({'burst' if peak_tf == peaks['bf16_tflops'] else 'sustained'})"}
+    else:
+        gbs = bytes_step * args.steps / region_s / 1e9
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                    "peak_source": peaks["source"], "tensor_time_us": t_tensor * 1e6, "hbm_time_us": t_hbm * 1e6}
+    roofline.update({"kernel": "proj_tc_kernel (forward, dX with W used transposed, dW over padded row buckets)", "traffic": None,
+                     "parts": parts})
+    extras = {}
+    if rank == 0 and not args.no_extras:
+        fd, gd = handles("dense")
+        time_steps(3, fd, gd)
+        n = min(24, args.steps)
+        dense_ms = time_steps(n, fd, gd) / n
+        star_ms = time_steps(n) / n
+        extras["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": star_ms, "time_ratio_star_over_dense": star_ms / dense_ms,
+                              "control": "same library, ALG_TABLE_DENSE", "ideal_ratio": flops / (3.0 * 2 * M * D * F)}
+    # CPU baseline: the oracle's forward and both gradient maps on evenly spaced rows
+    cpu = None
+    if rank == 0:
+        keep = oracle.support(q, cfg["law"])
+        n = int(min(M, max(16, 2 ** int(math.log2(max(16.0, 6e10 / (3.0 * D * F)))))))
+        rows = np.arange(0, M, max(1, M // n))[:n]
+        t0 = time.perf_counter()
+        oracle.proj(Xh[rows], types_h[rows], Wh, dw_, fw_, keep=keep)
+        oracle.proj_vjp_x(Gh[rows], types_h[rows], Wh, dw_, fw_, keep=keep)
+        oracle.proj_vjp_w(Xh[rows], Gh[rows], types_h[rows], dw_, fw_, keep=keep)
+        dt = time.perf_counter() - t0
+        c = np.bincount(types_h[rows], minlength=q)
+        cpu = {"value": 3 * 2 * oracle.macs(keep, dw_, fw_, c) / dt / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+               "sample": f"{len(rows)} of {M} rows (evenly spaced), forward + dX + dW, {dt:.2f} s"}
+    return {"metric": "star_q projection training step (forward + dX + dW), kept-GEMM throughput", "value": value, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg["label"], "rows_per_type": counts,
+                       "l2": f"{n_sets} working set(s) of {set_bytes / 1e6:.0f} MB used round-robin, L2 is 126 MB"},
+            "clocks": dict(clocks.summary(), note="sampled during the timed region"),
+            "e2e": {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                    "note": "gradients stay on the device in a training step; no host entry point is timed"},
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras}
 
 
 def decode_measurements(binding, layers=64, replays=20):

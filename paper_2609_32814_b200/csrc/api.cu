@@ -751,6 +751,17 @@ alg_status_t alg_proj_grad_create(alg_proj_grad_t *out, int q, const int32_t *in
     if (s == ALG_ERR_INVALID_ARG) s = ALG_ERR_UNSUPPORTED_SHAPE;   // a weight block no row type ever uses
   }
   if (s == ALG_OK && !(use_tc(g->dw) && g->dw.tc_ok)) s = ALG_ERR_UNSUPPORTED_SHAPE;   // dW has no SIMT path
+  if (s == ALG_OK && g->dw.tile_n > 128) {
+    // dW has as many tiles as the weight bank has 128 x tile_n blocks, whatever the batch: when wide tiles
+    // leave SMs without work, 128-column tiles (twice as many) are the better trade
+    long long tiles = 0;
+    bool all128 = true;
+    for (int e = 0; e < q; ++e) {
+      tiles += (long long)((in_widths[e] + 127) / 128) * (g->dx.K / g->dw.tile_n);
+      if (out_widths[e] % 128) all128 = false;
+    }
+    if (all128 && tiles < g->dw.num_sms) s = set_option(g->dw, ALG_OPT_TILE_N, 128);
+  }
   if (s == ALG_OK) {
     g->K = g->dx.N, g->N = g->dx.K;
     int offs[kMaxQ + 2];
