@@ -394,14 +394,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           uint32_t v[32];
           tc_ld_32x32(taddr + (uint32_t)c0, v);
           tc_wait_ld();
-          if (e == 0 && lane == 0) ALG_TRACE(2, 3);
           float f[32];
 #pragma unroll
           for (int x = 0; x < 32; ++x) f[x] = empty_tile ? 0.f : __uint_as_float(v[x]);
           finish_32(f, a, col_base + c0);
           uint32_t w[16];
           pack_bf16_32(f, w);
-          if (e == 0 && lane == 0) ALG_TRACE(2, 4);
           __syncwarp();  // the previous chunk has been read out of the buffer
 #pragma unroll
           for (int g = 0; g < 4; ++g)
@@ -420,7 +418,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (dst_row[g] >= 0)
               *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col_base + c0 + piece * 8) = val;
           }
-          if (e == 0 && lane == 0) ALG_TRACE(2, 5);
         }
       } else {
 #pragma unroll 1
