@@ -179,7 +179,9 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
  *     ALG_STATIC_SCRATCH_BYTES are refused with ALG_ERR_WORKSPACE_TOO_SMALL and nothing is
  *     launched; use alg_proj_forward with your own workspace for those.
  *   - The first call on each device looks up the device address of the array (with that device
- *     current).  Make that first call outside any stream capture.
+ *     current); with lazy module loading that is also when the driver places the array, so
+ *     the device's free memory drops by its size once, during that call and never after.
+ *     Make that first call at start-up, outside any stream capture.
  *   - All calls on one device share the one array.  It keeps whatever the previous call left;
  *     nothing in it has to start at zero, every call rewrites what it reads.  Two calls that
  *     overlap on the GPU (different streams without an event between them) race on it and

@@ -458,6 +458,26 @@ def test_vjp_adjoint_identities(law, q):
                                         for c in range(int(s.sum()))]))
 
 
+def test_vjp_dense_table_is_the_matmul_transpose_pair():
+    """With every block kept the projection is X @ W, so its gradient maps are G @ W^T and X^T @ G; a one-hot
+    weight perturbation pins single entries of dW for the Q_q law (the map is linear in W)."""
+    rng = np.random.default_rng(91)
+    s, r = np.array([2, 1, 3]), np.array([1, 2, 2])
+    M = 9
+    X = _rand_ints(rng, (M, s.sum()))
+    W = _rand_ints(rng, (s.sum(), r.sum()))
+    G = _rand_ints(rng, (M, r.sum()))
+    types = rng.integers(0, 3, size=M)
+    keep = oracle.support(3, "dense")
+    assert np.array_equal(oracle.proj_vjp_x(G, types, W, s, r, keep=keep), G @ W.T)
+    assert np.array_equal(oracle.proj_vjp_w(X, G, types, s, r, keep=keep), X.T @ G)
+    dW = oracle.proj_vjp_w(X, G, types, s, r)
+    for (k, n) in [(0, 0), (int(s.sum()) - 1, int(r.sum()) - 1), (2, 1), (3, 0)]:
+        E = np.zeros_like(W)
+        E[k, n] = 1.0
+        assert dW[k, n] == np.sum(oracle.proj(X, types, E, s, r) * G)
+
+
 def test_bad_type_rejected():
     with pytest.raises(oracle.OracleError):
         oracle.proj(np.zeros((2, 2)), [0, 2], np.zeros((2, 2)), [1, 1], [1, 1])
