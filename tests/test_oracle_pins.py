@@ -82,6 +82,30 @@ def test_support_probe_general_q(q):
         assert bool(keep[i, j, k]) == (k in (i, j))
 
 
+def test_large_algebra_rows_against_the_two_stage_form():
+    """Fixed-block regime (q in the hundreds, blocks off the tile grid): the per-row equation equals the
+    two-stage form of Section "Kernels" -- the block-diagonal map x_j W_jj for every row, then x_i W_ij
+    for the off-diagonal groups of a type-i row -- written here with numpy slices; counts follow Eq. q-rank."""
+    q, s, r, M = 72, 3, 5, 40
+    rng = np.random.default_rng(72)
+    X = _rand_ints(rng, (M, q * s))
+    W = _rand_ints(rng, (q * s, q * r))
+    types = rng.integers(0, q, size=M)
+    Y = np.zeros((M, q * r))
+    for j in range(q):                                   # stage 1: diagonal blocks, all rows
+        Y[:, j * r:(j + 1) * r] = X[:, j * s:(j + 1) * s] @ W[j * s:(j + 1) * s, j * r:(j + 1) * r]
+    for b in range(M):                                   # stage 2: the row panel of the row's own type
+        i = types[b]
+        panel = X[b, i * s:(i + 1) * s] @ W[i * s:(i + 1) * s, :]
+        panel[i * r:(i + 1) * r] = 0                     # B(i,i) = {i}: counted once, in stage 1
+        Y[b] += panel
+    assert np.array_equal(oracle.proj(X, types, W, [s] * q, [r] * q), Y)
+    keep = oracle.support(q)
+    assert oracle.gemm_count(keep) == 2 * q * q - q
+    rows = np.bincount(types, minlength=q)
+    assert oracle.macs(keep, [s] * q, [r] * q, rows) == M * (2 * q - 1) * s * r
+
+
 # ---- P2: counts and MAC formulas -------------------------------------------------------------
 
 def test_gemm_counts(golden):
