@@ -77,8 +77,12 @@ typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } a
  *           nothing) and kept for the last few M.  A call made while `stream` is being captured
  *           lets the kernels plan for themselves instead (same result), so a captured graph
  *           never depends on the handle's plan cache.  Forward calls on one handle must be
- *           ordered on the GPU (one stream, or events between streams). */
-typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1 } alg_schedule_t;
+ *           ordered on the GPU (one stream, or events between streams).
+ * INTERVAL: type of row b is b / (M/q), q | M: the rows of a type are contiguous -- the typing of
+ *           the square product A * B of two algebra elements (Eqs. q-product-diag/off), where
+ *           the rows of block row i of A carry type i; `types` may be NULL.  No permutation and
+ *           no copy of X.  Large-algebra path only (see alg_proj_create). */
+typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1, ALG_SCHED_INTERVAL = 2 } alg_schedule_t;
 
 /* Kernel families, reported by alg_proj_kernel_path(). */
 typedef enum {
@@ -87,7 +91,8 @@ typedef enum {
   ALG_PATH_DECODE = 2   /* small-M weight-streaming kernel                               */
 } alg_path_t;
 
-#define ALG_MAX_Q 32
+#define ALG_MAX_Q 32        /* general interaction tables (32-bit keep masks) */
+#define ALG_MAX_Q_LARGE 256 /* complete-graph law Q_q with equal group widths: the large-algebra path */
 
 /* Per-handle options (alg_proj_set_option / alg_ffn_set_option).  They replace process-wide
  * switches: nothing in the library reads the environment.  Set them between forward calls,
@@ -100,6 +105,9 @@ typedef enum {
  *                     width to be a multiple of 128.
  *   TILE_N            tile width of the one-CTA kernel: 0 = automatic, or 128 / 192 / 256 when
  *                     that divides every output group width.
+ *   STAGE_K           reduction depth of one pipeline stage of the one-CTA GEMM kernel: 0 =
+ *                     automatic, 32 (eight stages of 24 KB) or 64 (four stages of 48 KB).  Results
+ *                     are identical; only the operand pipeline differs.
  *   SMALL_M_KERNEL    1 (default): M <= 64 runs the weight-streaming kernels; 0: the prefill
  *                     kernels take every M.
  *   HOST_PLAN         1 (default): cyclic-schedule tile sequences are planned on the host;
@@ -117,7 +125,8 @@ typedef enum {
   ALG_OPT_SMALL_M_KERNEL = 3,
   ALG_OPT_HOST_PLAN = 4,
   ALG_OPT_WAIT_LIMIT_CYCLES = 5,
-  ALG_OPT_TEST_STALL_BYTES = 6
+  ALG_OPT_TEST_STALL_BYTES = 6,
+  ALG_OPT_STAGE_K = 7
 } alg_option_t;
 
 /* ---- projection handle ---------------------------------------------------------------------
@@ -128,7 +137,21 @@ typedef enum {
  * accumulation).  custom_keep is read only for ALG_TABLE_CUSTOM, else pass NULL; every
  * (i,j) of a custom table must keep at least one k.  1 <= q <= ALG_MAX_Q.
  * The tensor-core path needs every s[k] to be a multiple of 64 and every r[j] a multiple of
- * 128 (or of 192); other bf16/fp32 shapes run on the SIMT path.  */
+ * 128 (or of 192); other bf16/fp32 shapes run on the SIMT path, except:
+ *
+ * Large-algebra path (the fixed-block regime of Section "Kernel Benchmarks" and of the appendix
+ * "Large Projections and Square Products": q = n / b grows with the matrix, blocks such as
+ * 160 x 800 or 40 x 200 that are no multiple of the GPU tile).  Taken for ALG_TABLE_QQ with
+ * bf16 operands and EQUAL group widths s, r that are multiples of 8, when q > ALG_MAX_Q (up to
+ * ALG_MAX_Q_LARGE), when the widths do not fit the ordinary tensor-core path, or when the
+ * schedule is INTERVAL.  Same tcgen05 pipeline; tiles are enumerated by arithmetic (type-major,
+ * so a row panel W[S_i, :] is streamed once), the operands are fetched through per-group tensor
+ * maps whose out-of-range elements read as zero (a group narrower than the 32- or 64-deep
+ * pipeline stage, or a last column tile narrower than the tile, costs arithmetic on zeros but
+ * no extra bytes), and stores are masked at 8-column granularity.  With q > ALG_MAX_Q only the
+ * CYCLIC and INTERVAL schedules (q | M) are available; fp32 operands, other tables, unequal or
+ * odd widths with q > ALG_MAX_Q are refused with ALG_ERR_UNSUPPORTED_SHAPE.  The FFN and gradient
+ * handles do not take this path.  */
 alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
                              const int32_t *out_widths, alg_dtype_t dtype, alg_table_t table,
                              const uint8_t *custom_keep, alg_schedule_t schedule);

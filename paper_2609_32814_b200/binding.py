@@ -20,16 +20,16 @@ STATUS = {0: "ALG_OK", 1: "ALG_ERR_INVALID_ARG", 2: "ALG_ERR_UNSUPPORTED_SHAPE",
 ALG_F32, ALG_BF16 = 0, 1
 ALG_TABLE_QQ, ALG_TABLE_DENSE, ALG_TABLE_CUSTOM, ALG_TABLE_Q2POW = 0, 1, 2, 3
 ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
-ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC = 0, 1
+ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC, ALG_SCHED_INTERVAL = 0, 1, 2
 ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
 OPTIONS = {"gemm_kernel": 1, "tile_n": 2, "small_m_kernel": 3, "host_plan": 4, "wait_limit_cycles": 5,
-           "test_stall_bytes": 6}
+           "test_stall_bytes": 6, "stage_k": 7}
 
 _DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
 _TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM, "q2pow": ALG_TABLE_Q2POW}
 _ACTS = {None: ALG_ACT_NONE, "none": ALG_ACT_NONE, "gelu": ALG_ACT_GELU_ERF, "gelu_erf": ALG_ACT_GELU_ERF,
          "gelu_tanh": ALG_ACT_GELU_TANH}
-_SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC}
+_SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC, "interval": ALG_SCHED_INTERVAL}
 
 EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",

@@ -26,7 +26,15 @@ struct PlanSlot {
 };
 constexpr int kPlanSlots = 4;
 
+// Large-algebra path (proj_big.cu): complete-graph law, equal group widths, q up to kBigMaxQ.
+struct BigPlan {
+  bool on = false;
+  int s = 0, r = 0;       // width of every input / output group
+  int tile_n = 0, nt_n = 0, block_k = 0;
+};
+
 struct alg_proj_s {
+  BigPlan big;
   int q = 0;
   int s[kMaxQ] = {0}, r[kMaxQ] = {0};
   int K = 0, N = 0;
@@ -54,7 +62,7 @@ struct alg_proj_s {
   bool decode_ok = false;   // the small-M weight-streaming kernel covers this shape
   DecodePlan decode = {};
   // options (alg_proj_set_option)
-  int opt_kernel = 0, opt_tile_n = 0;
+  int opt_kernel = 0, opt_tile_n = 0, opt_stage_k = 0;
   bool opt_small_m = true, opt_host_plan = true;
   long long wait_limit = kDefaultWaitLimit;
   int test_extra_expect = 0;
@@ -193,17 +201,58 @@ alg_status_t pick_workers(alg_proj_s &p) {
   return ALG_OK;
 }
 
+// Tiling of the large-algebra kernel: as few column tiles per output group as 256-wide tiles allow, the
+// tile just wide enough (multiple of 16); 64-deep stages when the group width is a multiple of 64.
+void plan_big(alg_proj_s &p, int s, int r) {
+  p.big.on = true;
+  p.big.s = s, p.big.r = r;
+  p.big.nt_n = (r + 255) / 256;
+  p.big.tile_n = ((r + p.big.nt_n - 1) / p.big.nt_n + 15) / 16 * 16;
+  p.big.nt_n = (r + p.big.tile_n - 1) / p.big.tile_n;
+  p.big.block_k = s % 64 == 0 ? 64 : 32;
+}
+
+// Handle of the large-algebra path only (q > kMaxQ or the interval schedule): no interaction table.
+alg_status_t init_big(alg_proj_s &p, int q, int s, int r, alg_schedule_t sched) {
+  p.q = q;
+  p.dtype = ALG_BF16;
+  p.sched = sched;
+  p.K = q * s;
+  p.N = q * r;
+  plan_big(p, s, r);
+  if (q <= kMaxQ)
+    for (int g = 0; g < q; ++g) p.s[g] = s, p.r[g] = r;
+  if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, p.device) != cudaSuccess) return ALG_ERR_CUDA;
+  p.num_sms = prop.multiProcessorCount;
+  if (prop.major != 10) return ALG_ERR_UNSUPPORTED_SHAPE;
+  if (cudaMalloc(&p.d_status, 4 * sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
+  if (cudaMemset(p.d_status, 0, 4 * sizeof(int)) != cudaSuccess) return ALG_ERR_CUDA;
+  if (tc_init() != cudaSuccess) return ALG_ERR_CUDA;
+  return ALG_OK;
+}
+
 alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t *out_w, alg_dtype_t dtype,
                        alg_table_t table, const uint8_t *custom, alg_schedule_t sched, int *shared_status,
-                       bool gated = false) {
+                       bool gated = false, bool allow_big = false) {
   p.gated = gated;
-  if (q < 1 || q > kMaxQ || !in_w || !out_w) return ALG_ERR_INVALID_ARG;
+  if (q < 1 || q > kBigMaxQ || !in_w || !out_w) return ALG_ERR_INVALID_ARG;
+  if (sched != ALG_SCHED_EXPLICIT && sched != ALG_SCHED_CYCLIC && sched != ALG_SCHED_INTERVAL) return ALG_ERR_INVALID_ARG;
+  // large-algebra path: Q_q law, bf16, equal widths in multiples of 8
+  bool big_fits = allow_big && table == ALG_TABLE_QQ && dtype == ALG_BF16 && in_w[0] > 0 && out_w[0] > 0 &&
+                  in_w[0] % 8 == 0 && out_w[0] % 8 == 0;
+  for (int g = 1; g < q && big_fits; ++g) big_fits = in_w[g] == in_w[0] && out_w[g] == out_w[0];
+  if (q > kMaxQ || sched == ALG_SCHED_INTERVAL) {
+    if (!big_fits || (int64_t)q * in_w[0] > (1 << 30) || (int64_t)q * out_w[0] > (1 << 30)) return ALG_ERR_UNSUPPORTED_SHAPE;
+    if (q > kMaxQ && sched == ALG_SCHED_EXPLICIT) return ALG_ERR_UNSUPPORTED_SHAPE;
+    return init_big(p, q, in_w[0], out_w[0], sched);
+  }
   if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
   if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM && table != ALG_TABLE_Q2POW)
     return ALG_ERR_INVALID_ARG;
   if (table == ALG_TABLE_Q2POW && (q & (q - 1)) != 0) return ALG_ERR_INVALID_ARG;  // q must be a power of two
   if (table == ALG_TABLE_CUSTOM && !custom) return ALG_ERR_INVALID_ARG;
-  if (sched != ALG_SCHED_EXPLICIT && sched != ALG_SCHED_CYCLIC) return ALG_ERR_INVALID_ARG;
   p.q = q;
   p.dtype = dtype;
   p.sched = sched;
@@ -241,6 +290,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     }
   alg_status_t cs = configure_kernels(p);
   if (cs != ALG_OK) return cs;
+  if (big_fits && !p.tc_ok) plan_big(p, in_w[0], out_w[0]);   // widths the table-driven tensor path does not take
 
   if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
   cudaDeviceProp prop;
@@ -309,7 +359,7 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
   off = align_up(off + (size_t)kMaxBucketChunks * (first.q + 1) * sizeof(int));
   L.perm = off;
   off = align_up(off + (size_t)M * sizeof(int));
-  if (use_tc(first)) {
+  if (use_tc(first) || first.big.on) {
     L.xb = off;
     off = align_up(off + (size_t)M * first.K * 2, 1024);
   }
@@ -322,6 +372,9 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
 }
 
 alg_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? ALG_OK : ALG_ERR_CUDA; }
+
+// Reduction depth of a pipeline stage of the one-CTA GEMM kernel (the CTA-pair kernel has its own, 64).
+int block_k_of(const alg_proj_s &p) { return p.pair_kernel ? kTcBlockK : p.opt_stage_k ? p.opt_stage_k : kDefaultStageK; }
 
 // Tiling of one forward call on the tensor-core path.
 struct TcChoice {
@@ -379,7 +432,7 @@ const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, const TcChoice &tc, int64_t M
   std::vector<int> nkb(q * q, 0);
   for (int pr = 0; pr < q * q; ++pr)
     for (int k = 0; k < q; ++k)
-      if ((p.tab.keep[pr] >> k) & 1u) nkb[pr] += p.s[k] / kTcBlockK;
+      if ((p.tab.keep[pr] >> k) & 1u) nkb[pr] += p.s[k] / block_k_of(p);
   auto snake = [&](long long round, int w) { return round * nw + ((round & 1) ? (nw - 1 - w) : w); };
   const int rounds = (int)all_rounds + 1;
   slot->tag = g_plan_tag.fetch_add(1, std::memory_order_relaxed);
@@ -455,6 +508,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.gated_f = p.gated ? p.N : 0;
   a.w_kmajor = p.w_kmajor ? 1 : 0;
   a.dyn_so = nullptr;
+  a.block_k = block_k_of(p);
   a.y_staged = 0;
   a.plan = nullptr;
   a.plan_stride = a.plan_rounds = a.plan_tag = 0;
@@ -496,6 +550,57 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
 }
 
 bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && p.opt_small_m && M <= kDecodeMaxM; }
+
+// Forward call on the large-algebra path.  Equal buckets (cyclic or interval schedule, q | M) need no
+// pre-kernel at all; explicit types (q <= kMaxQ) go through bucketing and the row gather first.
+alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx, const int32_t *types,
+                     int64_t M, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y, int64_t ldy,
+                     alg_dtype_t y_dtype, cudaStream_t st) {
+  BigArgs a;
+  a.X = X, a.ldx = ldx;
+  a.W = W, a.ldw = ldw;
+  a.bias = bias;
+  a.act = (int)act;
+  a.Y = Y, a.ldy = ldy;
+  a.y_bf16 = y_dtype == ALG_BF16;
+  a.M = (int)M, a.q = p.q;
+  a.s = p.big.s, a.r = p.big.r;
+  a.tile_n = p.big.tile_n, a.nt_n = p.big.nt_n;
+  a.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;   // 64-deep stages only when they divide the group width
+  a.offsets = nullptr, a.perm = nullptr;
+  a.rows_per_type = 0;
+  a.status = p.d_status;
+  a.wait_limit = p.wait_limit;
+  const bool equal = p.sched != ALG_SCHED_EXPLICIT && M % p.q == 0;
+  if (equal) {
+    a.sched = p.sched == ALG_SCHED_INTERVAL ? 1 : 2;
+    a.rows_per_type = (int)(M / p.q);
+  } else {
+    if (p.sched == ALG_SCHED_INTERVAL || p.q > kMaxQ) return ALG_ERR_INVALID_ARG;   // these need q | M
+    BucketArgs b;
+    b.types = p.sched == ALG_SCHED_CYCLIC ? nullptr : types;
+    b.M = (int)M;
+    b.q = p.q;
+    b.chunk_rows = bucket_chunk_rows(M);
+    b.hdr = (WsHeader *)(ws + L.hdr);
+    b.chunk_counts = (int *)(ws + L.chunks);
+    b.perm = (int *)(ws + L.perm);
+    b.status = p.d_status;
+    b.sync = (unsigned int *)(p.d_status + 2);
+    b.wait_limit = p.wait_limit;
+    b.Y = Y;
+    b.ldy = ldy;
+    b.N = p.N;
+    b.y_elem_bytes = elem_bytes(y_dtype);
+    if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+    if (launch_gather_rows(X, ldx, b.perm, (int)M, p.K, 2, ws + L.xb, st) != cudaSuccess) return ALG_ERR_CUDA;
+    a.sched = 0;
+    a.X = ws + L.xb, a.ldx = p.K;
+    a.offsets = b.hdr->offsets;
+    a.perm = b.perm;
+  }
+  return cuda_status(launch_proj_big(a, p.num_sms, st));
+}
 
 alg_status_t run_decode(const alg_proj_s &p, const void *X, int64_t ldx, const int32_t *types, int64_t M,
                         const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y, int64_t ldy,
@@ -542,7 +647,7 @@ alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths, c
   *out = nullptr;
   alg_proj_s *p = new (std::nothrow) alg_proj_s();
   if (!p) return ALG_ERR_INVALID_ARG;
-  alg_status_t s = init_proj(*p, q, in_widths, out_widths, dtype, table, custom_keep, schedule, nullptr);
+  alg_status_t s = init_proj(*p, q, in_widths, out_widths, dtype, table, custom_keep, schedule, nullptr, false, true);
   if (s != ALG_OK) {
     free_proj(*p);
     delete p;
@@ -560,9 +665,11 @@ alg_status_t alg_proj_destroy(alg_proj_t h) {
 }
 
 static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value) {
+  const bool no_table = p.q > kMaxQ || p.sched == ALG_SCHED_INTERVAL;   // large-algebra handles have one kernel
   switch (option) {
     case ALG_OPT_GEMM_KERNEL:
     case ALG_OPT_TILE_N: {
+      if (no_table) return value == 0 ? ALG_OK : ALG_ERR_UNSUPPORTED_SHAPE;
       if (option == ALG_OPT_GEMM_KERNEL && (value < 0 || value > 3)) return ALG_ERR_INVALID_ARG;
       if (option == ALG_OPT_TILE_N && value != 0 && value != 128 && value != 192 && value != 256) return ALG_ERR_INVALID_ARG;
       const int old_kernel = p.opt_kernel, old_tile = p.opt_tile_n;
@@ -583,6 +690,11 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
       if (cudaMemcpy(p.d_tab, &p.tab, sizeof(DevTable), cudaMemcpyHostToDevice) != cudaSuccess) return ALG_ERR_CUDA;
       return cuda_status(cudaMemcpy(p.d_tab_tall, &p.tab_tall, sizeof(DevTable), cudaMemcpyHostToDevice));
     }
+    case ALG_OPT_STAGE_K:
+      if (value != 0 && value != 32 && value != 64) return ALG_ERR_INVALID_ARG;
+      p.opt_stage_k = (int)value;
+      for (PlanSlot &sl : p.plan) sl.M = -1;  // cached plans count K blocks of the old depth
+      return ALG_OK;
     case ALG_OPT_SMALL_M_KERNEL: p.opt_small_m = value != 0; return ALG_OK;
     case ALG_OPT_HOST_PLAN: p.opt_host_plan = value != 0; return ALG_OK;
     case ALG_OPT_WAIT_LIMIT_CYCLES:
@@ -635,6 +747,7 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
   if (use_decode(*h, M)) return run_decode(*h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
+  if (h->big.on) return run_big(*h, L, ws, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
 
   BucketArgs b;
   b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
@@ -660,7 +773,8 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
 alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
   if (!h || !n) return ALG_ERR_INVALID_ARG;
   int64_t c = 0;
-  for (int pr = 0; pr < h->q * h->q; ++pr) c += __builtin_popcount(h->tab.keep[pr]);
+  if (h->q > kMaxQ || h->sched == ALG_SCHED_INTERVAL) c = 2 * (int64_t)h->q * h->q - h->q;   // no table: Q_q law (Eq. q-rank)
+  else for (int pr = 0; pr < h->q * h->q; ++pr) c += __builtin_popcount(h->tab.keep[pr]);
   *n = c;
   return ALG_OK;
 }
@@ -668,6 +782,14 @@ alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
 alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *macs) {
   if (!h || !rows_per_type || !macs) return ALG_ERR_INVALID_ARG;
   int64_t total = 0;
+  if (h->q > kMaxQ || h->sched == ALG_SCHED_INTERVAL) {   // no table: one product on the diagonal, two elsewhere
+    for (int i = 0; i < h->q; ++i) {
+      if (rows_per_type[i] < 0) return ALG_ERR_INVALID_ARG;
+      total += rows_per_type[i] * (2 * (int64_t)h->q - 1) * h->big.s * h->big.r;
+    }
+    *macs = total;
+    return ALG_OK;
+  }
   for (int i = 0; i < h->q; ++i) {
     if (rows_per_type[i] < 0) return ALG_ERR_INVALID_ARG;
     for (int j = 0; j < h->q; ++j)
@@ -680,7 +802,7 @@ alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *
 
 alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path) {
   if (!h || !path || M < 0) return ALG_ERR_INVALID_ARG;
-  *path = use_decode(*h, M) ? ALG_PATH_DECODE : use_tc(*h) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
+  *path = use_decode(*h, M) ? ALG_PATH_DECODE : (use_tc(*h) || h->big.on) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
   return ALG_OK;
 }
 
@@ -908,6 +1030,7 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   a.gated_f = 0;
   a.w_kmajor = 0;
   a.dyn_so = hdr->pad_offsets;
+  a.block_k = block_k_of(p);
   a.y_staged = 0;
   a.plan = nullptr;
   a.plan_stride = a.plan_rounds = a.plan_tag = 0;

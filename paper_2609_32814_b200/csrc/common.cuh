@@ -147,6 +147,7 @@ struct ProjArgs {
   // tile accumulates 128 gate columns and the matching 128 up columns side by side, the epilogue
   // stores silu(gate) * up; N = gated_f is the width of the output.  0 = ordinary projection.
   int gated_f;
+  int block_k;            // reduction depth of one pipeline stage of the one-CTA kernel: 64 or 32
   int y_staged;           // 1: the epilogue transposes bf16 results through shared memory for coalesced stores
   // Cyclic schedule: the tile sequences of all workers depend only on (handle, M) and are planned
   // once on the host; worker w reads plan[1 + w * plan_stride .. + plan_rounds) (the last record of
@@ -160,11 +161,39 @@ struct ProjArgs {
 
 cudaError_t launch_proj_simt(const ProjArgs &a, bool in_bf16, cudaStream_t st);
 
+// Large-algebra path: complete-graph law with q equal groups, q up to kBigMaxQ, group widths that
+// need not be multiples of the tile (proj_big.cu).
+constexpr int kBigMaxQ = ALG_MAX_Q_LARGE;
+struct BigArgs {
+  const void *X;          // bf16; sched 0: type-bucketed copy, else the caller's rows
+  int64_t ldx;
+  const void *W;          // bf16 K x N bank
+  int64_t ldw;
+  const void *bias;       // bf16[N] or nullptr
+  int act;
+  void *Y;
+  int64_t ldy;
+  int y_bf16;
+  int M, q;
+  int s, r;               // width of every input / output group (multiples of 8)
+  int tile_n;             // columns per tile: multiple of 16, <= 256
+  int nt_n;               // column tiles per output group = ceil(r / tile_n)
+  int block_k;            // 64 or 32: reduction depth of a pipeline stage
+  int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
+  const int *offsets;     // sched 0: device bucket offsets [q + 1]
+  const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)
+  int rows_per_type;      // sched 1, 2: M / q
+  int *status;
+  long long wait_limit;
+};
+cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st);
+
 // tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
 // (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.
 constexpr int kTcSeqCap = 224, kTc2SeqCap = 48;  // precomputed tile records per worker
 constexpr int kTcTileM = 128;
 constexpr int kTcBlockK = 64;
+constexpr int kDefaultStageK = 64;   // stage depth of the one-CTA GEMM kernel unless a handle asks otherwise
 constexpr int kTc2TileM = 256;
 constexpr int kTc2TileN = 256;
 cudaError_t launch_proj_tc(const ProjArgs &a, int tile_n, int num_sms, cudaStream_t st);

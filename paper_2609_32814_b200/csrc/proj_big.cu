@@ -1,0 +1,450 @@
+// Large-algebra grouped GEMM for sm_100a: the complete-graph law Q_q with q equal groups, q up to
+// 256, and group widths that need not be multiples of the GPU tile (the fixed-block regime of
+// Section "Kernel Benchmarks" and the appendix "Large Projections and Square Products": blocks such
+// as 160 x 800, 80 x 400, 40 x 200, or b x b blocks with q = n / b).
+//
+// One output tile = up to 128 rows of one row type i  x  tile_n columns of one output group j.  Its
+// reduction is x_i W_ij + x_j W_jj (Eqs. typed-diag / typed-off; one product when i = j), both
+// summed in the same TMEM accumulator -- the paper's two stages (diagonal maps for all rows, then
+// the type-dependent maps) become two reduction segments of one tile, so Y is written exactly once
+// and never read.
+//
+// What differs from the table-driven kernel (proj_tc.cu):
+//  * No interaction table and no tile classes: with 65536 (type, group) pairs neither fits shared
+//    memory.  Tile t is decoded by arithmetic, type-major: all tiles of type i are consecutive, so
+//    the row panel W[S_i, :] -- which only type-i rows use -- streams from HBM once while the
+//    q diagonal blocks stay in L2; inside a type the m-tile index runs fastest (CTAs working side by
+//    side share their B blocks), then the column tile, then the output group.
+//  * Operands come through PER-GROUP tensor maps: X as {s, q, rows} (or {s, q, q, M/q} for the
+//    cyclic schedule), W as {N, s, q}.  Coordinates past a group's width (or past N) read as
+//    zero, so a group that is narrower than the pipeline stage, and a last column tile narrower
+//    than tile_n, are padded for free: extra multiply-adds on zeros, no extra bytes, no repacked
+//    copies of X or W.  Everything stays 16-byte aligned because widths are multiples of 8.
+//  * The MMA width is a launch parameter (tile_n, a multiple of 16), stores are masked per 8
+//    columns.
+// Warp roles as in proj_tc.cu: warp 0 = TMA producer of A, warp 10 = TMA producer of B, warp 1 =
+// TMEM allocator + MMA issuer, warps 2..9 = epilogue (TMEM lane quadrant = warp % 4; the two warps
+// of a quadrant alternate over the 32-column chunks).  Double-buffered accumulator; every wait is
+// bounded and ends in ALG_ERR_DEVICE_TIMEOUT.
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+
+#include "tc_common.cuh"
+
+namespace algproj {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kThreads = 352;
+constexpr int kEpiWarps = 8;
+constexpr int kProducerWarpB = 10;
+constexpr int kStoreBufBytes = 32 * 64;   // per epilogue warp: 32 rows x 32 bf16 columns
+
+struct Ctl {
+  uint64_t full[12];
+  uint64_t empty[12];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  volatile int abort_flag;
+  long long wait_limit;
+  int total;                    // tiles of the launch
+  int off[kBigMaxQ + 1];        // sched 0: first bucketed row of every type
+  int pre[kBigMaxQ + 1];        // sched 0: tiles before type i
+};
+
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (ctl->abort_flag) return false;
+      if (clock64() - t0 > ctl->wait_limit) {
+        ctl->abort_flag = 1;
+        atomicExch(status, (int)ALG_ERR_DEVICE_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_slow(bar, parity, ctl, status);
+}
+
+template <int TILE_N, int BK>
+struct Cfg {
+  static constexpr int kABytes = 128 * BK * 2;
+  static constexpr int kBChunkBytes = BK * 64 * 2;              // one BK(k) x 64(n) box
+  static constexpr int kChunks = TILE_N / 64;
+  static constexpr int kStageBytes = kABytes + kBChunkBytes * kChunks;
+  static constexpr int kStages = (192 * 1024) / kStageBytes > 12 ? 12 : (192 * 1024) / kStageBytes;
+  static constexpr int kTmemCols = 2 * TILE_N;
+  static constexpr uint32_t kSwzK = BK == 64 ? 2 : 4;
+  static constexpr uint32_t kSboK = 8 * BK * 2;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiWarps * kStoreBufBytes + (int)sizeof(Ctl) + 1024;
+  static_assert(BK == 64 || BK == 32, "stage depth");
+  static_assert(TILE_N == 128 || TILE_N == 256, "stage width");
+};
+
+struct Tile {
+  int row0, rows;   // bucketed rows [row0, row0 + rows), all of type i; row0 < 0: no more tiles
+  int i, j;
+  int n0, cols;     // absolute first column, valid columns (<= tile_n)
+};
+
+// Tile t of the launch (uniform across the warp).  Type-major; inside a type: m-tile fastest, then
+// the column tile, then the output group.
+__device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, int t) {
+  Tile o;
+  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0;
+  if (t >= ctl->total) return o;
+  int i, rem, base, rows_i;
+  if (a.sched != 0) {
+    rows_i = a.rows_per_type;
+    const int per_type = ((rows_i + 127) >> 7) * a.q * a.nt_n;
+    i = t / per_type;
+    rem = t - i * per_type;
+    base = i * rows_i;
+  } else {
+    int lo = 0, hi = a.q;   // pre[lo] <= t < pre[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (ctl->pre[mid] <= t) lo = mid; else hi = mid;
+    }
+    i = lo;
+    rem = t - ctl->pre[i];
+    base = ctl->off[i];
+    rows_i = ctl->off[i + 1] - base;
+  }
+  const int mt_i = (rows_i + 127) >> 7;
+  const int u = rem / mt_i, mt = rem - u * mt_i;
+  const int j = u / a.nt_n, nt = u - j * a.nt_n;
+  o.row0 = base + (mt << 7);
+  o.rows = min(128, rows_i - (mt << 7));
+  o.i = i, o.j = j;
+  o.n0 = j * a.r + nt * a.tile_n;
+  o.cols = min(a.tile_n, a.r - nt * a.tile_n);
+  return o;
+}
+
+template <int TILE_N, int BK>
+__global__ void __launch_bounds__(kThreads, 1)
+proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const BigArgs a) {
+  using C = Cfg<TILE_N, BK>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t *store_buf = smem + C::kStages * C::kStageBytes;
+  Ctl *ctl = (Ctl *)(store_buf + kEpiWarps * kStoreBufBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = a.q;
+
+  if (warp == 0) {
+    if (lane < C::kStages) {
+      mbar_init(smem_u32(&ctl->full[lane]), 1);
+      mbar_init(smem_u32(&ctl->empty[lane]), 1);
+    } else if (lane < C::kStages + 2) {
+      mbar_init(smem_u32(&ctl->tmem_full[lane - C::kStages]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[lane - C::kStages]), kEpiWarps);
+    } else if (lane == 31) {
+      ctl->abort_flag = 0;
+      ctl->wait_limit = a.wait_limit;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  } else if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                 "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  } else if (warp == 3 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+  }
+  // Everything above touches only this CTA's own state and may overlap the previous kernel of the stream.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (warp == 2) {
+    // tile counts: one warp turns the bucket offsets into "tiles before type i"
+    if (a.sched != 0) {
+      if (lane == 0) ctl->total = q * ((a.rows_per_type + 127) >> 7) * q * a.nt_n;
+    } else {
+      int carry = 0;
+      for (int i0 = 0; i0 < q; i0 += 32) {
+        const int i = i0 + lane;
+        int v = 0;
+        if (i < q) {
+          const int lo = a.offsets[i], hi = a.offsets[i + 1];
+          ctl->off[i] = lo;
+          if (i == q - 1) ctl->off[q] = hi;
+          v = ((hi - lo + 127) >> 7) * q * a.nt_n;
+        }
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += n;
+        }
+        if (i < q) ctl->pre[i] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) ctl->pre[q] = carry, ctl->total = carry;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const int nkb_seg = (a.s + BK - 1) / BK;   // pipeline stages per reduction segment (the last one zero-padded)
+
+  if (warp == 0 || warp == kProducerWarpB) {
+    // ---------------- TMA producers (warp-uniform loops, one elected lane issues) ----------------
+    const bool loads_a = warp == 0;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    const uint32_t smem0 = smem_u32(smem);
+    for (int t = blockIdx.x; ok; t += gridDim.x) {
+      const Tile tl = decode_tile(a, ctl, t);
+      if (tl.row0 < 0) break;
+      const int n_seg = tl.i == tl.j ? 1 : 2;
+      const int a_row = a.sched == 2 ? tl.row0 - tl.i * a.rows_per_type : tl.row0;
+      for (int sg = 0; sg < n_seg && ok; ++sg) {
+        const int k = n_seg == 1 ? tl.i : (sg == 0 ? min(tl.i, tl.j) : max(tl.i, tl.j));
+        for (int kb = 0; kb < nkb_seg; ++kb) {
+          ok = __all_sync(0xffffffffu, wait_bar(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, a.status));
+          if (!ok) break;
+          const uint32_t bar = full0 + 8u * (uint32_t)stage;
+          const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
+          if (elect_one()) {
+            if (loads_a) {
+              mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+              if (a.sched == 2) tma_load_4d(sa, &tmA, bar, kb * BK, k, tl.i, a_row);
+              else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
+            } else {
+#pragma unroll
+              for (int c = 0; c < C::kChunks; ++c)
+                tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0 + c * 64, kb * BK, k);
+            }
+          }
+          __syncwarp();
+          if (++stage == C::kStages) stage = 0, phase ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    int stage = 0, acc = 0;
+    uint32_t phase = 0, acc_phase = 0;
+    bool ok = true;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
+    const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, C::kSboK, C::kSwzK);
+    const uint64_t db0 = make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
+    // instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, N = tile_n, M = 128
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(a.tile_n >> 3) << 17) |
+                           ((uint32_t)(128 >> 4) << 24);
+    for (int t = blockIdx.x; ok; t += gridDim.x) {
+      const Tile tl = decode_tile(a, ctl, t);
+      if (tl.row0 < 0) break;
+      const int n_kb = (tl.i == tl.j ? 1 : 2) * nkb_seg;
+      ok = __all_sync(0xffffffffu, wait_bar(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
+      for (int kb = 0; kb < n_kb; ++kb) {
+        ok = __all_sync(0xffffffffu, wait_bar(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        if (elect_one()) {
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk)
+            tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc, (kb | kk) ? 1u : 0u);
+          tc_commit(empty0 + 8u * (uint32_t)stage);
+        }
+        __syncwarp();
+        if (++stage == C::kStages) stage = 0, phase ^= 1u;
+      }
+      if (!ok) break;
+      if (elect_one()) tc_commit(tfull0 + 8u * (uint32_t)acc);
+      __syncwarp();
+      if (++acc == 2) acc = 0, acc_phase ^= 1u;
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int e = warp - 2;
+    const int quad = warp & 3;
+    const int half = e >> 2;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    uint8_t *buf = store_buf + e * kStoreBufBytes;
+    const uint32_t my_row = smem_u32(buf) + (uint32_t)lane * 64u;
+    const uint32_t sw = (uint32_t)((lane >> 1) & 3);
+    const int sub = lane >> 2, piece = lane & 3;
+    const uint32_t rd_base = smem_u32(buf) + (uint32_t)sub * 64u;
+    for (int t = blockIdx.x;; t += gridDim.x) {
+      const Tile tl = decode_tile(a, ctl, t);
+      if (tl.row0 < 0) break;
+      const int r = quad * 32 + lane;
+      int64_t out_row = -1;
+      if (r < tl.rows) {
+        if (a.sched == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
+        else if (a.sched == 0 && a.perm) out_row = __ldg(a.perm + tl.row0 + r);
+        else out_row = tl.row0 + r;
+        if (out_row >= a.M) out_row = -1;
+      }
+      bool ok = wait_bar(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TILE_N);
+      const int col_end = tl.n0 + tl.cols;
+      int64_t dst_row[4];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 8 + sub);
+#pragma unroll 1
+      for (int c0 = half * 32; c0 < tl.cols; c0 += 64) {
+        uint32_t v[32];
+        tc_ld_32x32(taddr + (uint32_t)c0, v);
+        tc_wait_ld();
+        const int col = tl.n0 + c0;
+        float f[32];
+#pragma unroll
+        for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+        if (a.bias) {
+          const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
+#pragma unroll
+          for (int x = 0; x < 32; ++x)
+            if (col + x < col_end) f[x] += __bfloat162float(__ldg(b + x));
+        }
+        if (a.act == ALG_ACT_GELU_ERF) {
+#pragma unroll
+          for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
+        } else if (a.act == ALG_ACT_GELU_TANH) {
+#pragma unroll
+          for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
+        }
+        if (a.y_bf16) {
+          // transpose through the warp's staging buffer: one store instruction then covers 8 rows x 64
+          // contiguous bytes; a 16-byte piece is stored when its 8 columns belong to the tile
+          uint32_t w[16];
+          pack_bf16_32(f, w);
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((((uint32_t)g) ^ sw) << 4)), "r"(w[g * 4]),
+                         "r"(w[g * 4 + 1]), "r"(w[g * 4 + 2]), "r"(w[g * 4 + 3])
+                         : "memory");
+          __syncwarp();
+          const bool piece_ok = col + piece * 8 < col_end;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int rr = g * 8 + sub;
+            const uint32_t rsw = (uint32_t)((rr >> 1) & 3);
+            uint4 val;
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                         : "r"(rd_base + (uint32_t)g * 512u + ((((uint32_t)piece) ^ rsw) << 4)));
+            if (dst_row[g] >= 0 && piece_ok)
+              *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col + piece * 8) = val;
+          }
+        } else if (out_row >= 0) {
+          float *dst = (float *)a.Y + out_row * a.ldy + col;
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if (col + g * 4 < col_end) ((float4 *)dst)[g] = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+      if (++acc == 2) acc = 0, acc_phase ^= 1u;
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  if (ctl->abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {   // copies still in flight land before shared memory is released
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+  }
+}
+
+template <int TILE_N, int BK>
+cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
+  using C = Cfg<TILE_N, BK>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(proj_big_kernel<TILE_N, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  static_assert(C::kSmemBytes <= 227 * 1024, "shared memory budget");
+  CUtensorMap tmA, tmB;
+  cudaError_t e;
+  if (a.sched == 2) {
+    // rows of type i are rows i, i + q, ...: {k in group, group, type, position in the type}
+    const uint64_t dims[4] = {(uint64_t)a.s, (uint64_t)a.q, (uint64_t)a.q, (uint64_t)a.rows_per_type};
+    const uint64_t str[3] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.q};
+    const uint32_t box[4] = {(uint32_t)BK, 1, 1, 128};
+    e = make_map_nd(&tmA, a.X, 4, dims, str, box, BK * 2);
+  } else {
+    const uint64_t dims[3] = {(uint64_t)a.s, (uint64_t)a.q, (uint64_t)a.M};
+    const uint64_t str[2] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2};
+    const uint32_t box[3] = {(uint32_t)BK, 1, 128};
+    e = make_map_nd(&tmA, a.X, 3, dims, str, box, BK * 2);
+  }
+  if (e != cudaSuccess) return e;
+  {
+    // the bank as {columns, k in group, group}: rows past the group's width read as zero
+    const uint64_t dims[3] = {(uint64_t)a.q * (uint64_t)a.r, (uint64_t)a.s, (uint64_t)a.q};
+    const uint64_t str[2] = {(uint64_t)a.ldw * 2, (uint64_t)a.ldw * 2 * (uint64_t)a.s};
+    const uint32_t box[3] = {64, (uint32_t)BK, 1};
+    e = make_map_nd(&tmB, a.W, 3, dims, str, box, 128);
+  }
+  if (e != cudaSuccess) return e;
+  long long tiles;
+  if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * a.q * a.nt_n;
+  else tiles = ((long long)a.M / 128 + a.q) * a.q * a.nt_n;   // upper bound: every type may end in a ragged tile
+  if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)std::min<long long>(num_sms, std::max<long long>(tiles, 1)), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, proj_big_kernel<TILE_N, BK>, tmA, tmB, a);
+  count_launch(1);
+  return e;
+}
+
+}  // namespace
+
+cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
+  cudaError_t e = tc_init();
+  if (e != cudaSuccess) return e;
+  if (a.q < 1 || a.q > kBigMaxQ || a.s % 8 || a.r % 8 || a.tile_n % 16 || a.tile_n < 16 || a.tile_n > 256) return cudaErrorInvalidValue;
+  if (a.nt_n != (a.r + a.tile_n - 1) / a.tile_n) return cudaErrorInvalidValue;
+  if (a.tile_n <= 128) return a.block_k == 64 ? launch_t<128, 64>(a, num_sms, st) : launch_t<128, 32>(a, num_sms, st);
+  return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);
+}
+
+}  // namespace algproj

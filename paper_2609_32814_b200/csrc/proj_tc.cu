@@ -34,8 +34,8 @@ ALG_TRACE_DEFINE(proj_tc)
 namespace {
 
 struct Ctl {
-  uint64_t full[8];
-  uint64_t empty[8];
+  uint64_t full[12];
+  uint64_t empty[12];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint32_t tmem_base;
@@ -81,14 +81,22 @@ constexpr int kThreads = 32 * (3 + kEpiWarps);
 // multiply-accumulate by a quarter against a 128 x 192 tile -- the layout for projections with a
 // long reduction and narrow output groups (TILE_N = 128 only, so that two tiles still fit the
 // 512 columns and the epilogue of one tile overlaps the main loop of the next).
-template <int TILE_N, int TILE_M>
+//
+// BK = reduction depth of one pipeline stage, 64 or 32.  The bytes a CTA has in flight are what its
+// operand fill rate hangs on (a freed stage is refilled one L2 round trip later); of S stages S - 1
+// are in flight while one is consumed, so twice as many stages of half the depth keep 7/8 instead of
+// 3/4 of the same shared memory busy.  BK = 32 rows of A are 64 bytes: 64-byte swizzle atoms there.
+template <int TILE_N, int TILE_M, int BK>
 struct Cfg {
   static constexpr int kHalves = TILE_M / 128;                  // accumulators (MMAs per K step) of a tile
-  static constexpr int kABytes = TILE_M * kTcBlockK * 2;        // 16 KB per 128 rows
-  static constexpr int kBChunkBytes = kTcBlockK * 64 * 2;       // one 64(k) x 64(n) box: 8 KB
+  static constexpr int kAHalfBytes = 128 * BK * 2;              // 128 rows of A: 16 KB (BK = 64) or 8 KB
+  static constexpr int kABytes = TILE_M * BK * 2;
+  static constexpr int kBChunkBytes = BK * 64 * 2;              // one BK(k) x 64(n) box: 8 KB or 4 KB
   static constexpr int kBBytes = kBChunkBytes * (TILE_N / 64);
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
+  static constexpr int kStages = (200 * 1024) / kStageBytes > 12 ? 12 : (200 * 1024) / kStageBytes;
+  static constexpr uint32_t kSwzK = BK == 64 ? 2 : 4;            // descriptor swizzle mode of a K-major operand
+  static constexpr uint32_t kSboK = 8 * BK * 2;                  // 8 rows of a K-major operand
   static constexpr int kAccStride = TILE_N * kHalves <= 128 ? 128 : 256;   // TMEM columns between the two tile buffers
   static constexpr int kTmemCols = 2 * kAccStride;
   static constexpr int kFixedSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + kSeqCap * 16 + 16 + 1024;  // + tile map
@@ -99,6 +107,7 @@ struct Cfg {
   // instruction descriptor: D=f32, A=B=bf16, A K-major, B MN-major, N, M=128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                      ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  static_assert(BK == 64 || BK == 32, "stage depth");
   static_assert(TILE_M == 128 || (TILE_M == 256 && TILE_N == 128), "256-row tiles are 128 columns wide");
   static_assert(kHalves == 1 || kEpiWarps == 8, "two accumulators need one epilogue warp group each");
 };
@@ -108,10 +117,10 @@ struct Cfg {
 // N = 256 MMA fills both halves of the accumulator, and the epilogue writes silu(gate) * up -- 128
 // output columns per tile, the hidden state is stored once and the two pre-activations never
 // leave the chip (the merged gate/up kernel of the appendix "Kernel Benchmark Details").
-template <int TILE_N, int TILE_M, bool GATED>
+template <int TILE_N, int TILE_M, bool GATED, int BK>
 __global__ void __launch_bounds__(kThreads, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
-  using C = Cfg<TILE_N, TILE_M>;
+  using C = Cfg<TILE_N, TILE_M, BK>;
   static_assert(!GATED || (TILE_N == 256 && TILE_M == 128), "the gated kernel pairs two 128-column halves");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -158,7 +167,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int k = 0; k < q; ++k)
         if ((mask >> k) & 1u)
           n += (a.dyn_so ? a.dyn_so[k + 1] - a.dyn_so[k] : a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k]) /
-               kTcBlockK;
+               BK;
       ctl->nkb[e] = (uint16_t)n;   // for tile records decoded after the precomputed ones
     }
   }
@@ -188,7 +197,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
       if (a.offsets || a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
       tile_plan_warp(tm, recs, kSeqCap, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom, blockIdx.x,
-                     gridDim.x, kTcBlockK, a.dyn_so);
+                     gridDim.x, BK, a.dyn_so);
     }
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -230,7 +239,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!((mask >> k) & 1u)) continue;
         const int k_begin = __shfl_sync(0xffffffffu, ctl->so[k], 0);
         const int k_end = __shfl_sync(0xffffffffu, ctl->so[k + 1], 0);
-        for (int k0 = k_begin; k0 < k_end; k0 += kTcBlockK) {
+        for (int k0 = k_begin; k0 < k_end; k0 += BK) {
           ok = __all_sync(0xffffffffu, wait_bar(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, a.status));
           if (!ok) break;
           const uint32_t bar = full0 + 8u * (uint32_t)stage;
@@ -269,10 +278,10 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
-    const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, 1024);
-    // B: the canonical bank lands MN-major (64-column chunks 8 KB apart, 16 k-rows = two 8-row groups
+    const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, C::kSboK, C::kSwzK);
+    // B: the canonical bank lands MN-major (64-column chunks one box apart, 16 k-rows = two 8-row groups
     // = 128 descriptor units per K step); used transposed it lands K-major like A (32 bytes per K step)
-    const uint64_t db0 = a.w_kmajor ? make_smem_desc(smem_u32(smem) + C::kABytes, 16, 1024)
+    const uint64_t db0 = a.w_kmajor ? make_smem_desc(smem_u32(smem) + C::kABytes, 16, C::kSboK, C::kSwzK)
                                     : make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
     const uint32_t idesc = a.w_kmajor ? (C::kIdesc & ~(1u << 16)) : C::kIdesc;
     const uint64_t db_step = a.w_kmajor ? 2 : 128;
@@ -297,13 +306,13 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         if (elect_one()) {
           // A: 16 k-elements = 32 bytes inside the swizzle atom; B: 16 k-rows = two 8-row groups;
-          // the second 128 rows of a 256-row tile sit 16 KB further in the stage and accumulate
+          // the second 128 rows of a 256-row tile sit behind the first in the stage and accumulate
           // TILE_N columns further in tensor memory
 #pragma unroll
-          for (int kk = 0; kk < kTcBlockK / 16; ++kk)
+          for (int kk = 0; kk < BK / 16; ++kk)
 #pragma unroll
             for (int h = 0; h < C::kHalves; ++h)
-              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * 1024), db + (uint64_t)kk * db_step,
+              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * (C::kAHalfBytes >> 4)), db + (uint64_t)kk * db_step,
                           idesc, (kb | kk) ? 1u : 0u);
           tc_commit(empty0 + 8u * (uint32_t)stage);
         }
@@ -462,12 +471,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
-template <int TILE_N, int TILE_M, bool GATED = false>
-cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
-  using C = Cfg<TILE_N, TILE_M>;
+template <int TILE_N, int TILE_M, bool GATED, int BK>
+cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
+  using C = Cfg<TILE_N, TILE_M, BK>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -480,14 +489,14 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   if (a.w_kmajor) {   // W is N x K here (rows = output columns, contiguous along the reduction): boxes of 64 x TILE_N
     if (GATED) return cudaErrorInvalidValue;
     b.b_3d = 0;
-    e = make_map_2d(&tmB, a.W, (uint64_t)a.K, (uint64_t)a.N, (uint64_t)a.ldw * 2, kTcBlockK, TILE_N);
+    e = make_map_2d_sw(&tmB, a.W, (uint64_t)a.K, (uint64_t)a.N, (uint64_t)a.ldw * 2, BK, TILE_N, BK * 2);
     if (e != cudaSuccess) return e;
   } else {
     b.b_3d = make_map_b3d(&tmB, a, GATED ? 2 : TILE_N / 64) == cudaSuccess;
   }
   if (GATED && !b.b_3d) return cudaErrorInvalidValue;
   if (!b.b_3d && !a.w_kmajor) {
-    e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, kTcBlockK);
+    e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, BK);
     if (e != cudaSuccess) return e;
   }
   // staging buffers for the transposing epilogue, when they fit and the output rows are 16-byte aligned
@@ -504,9 +513,16 @@ cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED, BK>, tmA, tmB, b);
   count_launch(1);
   return e;
+}
+
+template <int TILE_N, int TILE_M, bool GATED = false>
+cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
+  if (a.block_k == 32) return launch_bk<TILE_N, TILE_M, GATED, 32>(a, num_sms, st);
+  if (a.block_k == 64) return launch_bk<TILE_N, TILE_M, GATED, 64>(a, num_sms, st);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -525,6 +541,25 @@ cudaError_t make_map_2d_sw(CUtensorMap *map, const void *base, uint64_t inner, u
                                 : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                       : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t make_map_nd(CUtensorMap *map, const void *base, int rank, const uint64_t *dims, const uint64_t *stride_bytes,
+                        const uint32_t *box, int swizzle_bytes) {
+  cudaError_t e0 = tc_init();
+  if (e0 != cudaSuccess) return e0;
+  if (rank < 2 || rank > 5) return cudaErrorInvalidValue;
+  cuuint64_t d[5], st[4];
+  cuuint32_t b[5], estr[5];
+  for (int i = 0; i < rank; ++i) d[i] = dims[i], b[i] = box[i], estr[i] = 1;
+  for (int i = 0; i + 1 < rank; ++i) st[i] = stride_bytes[i];
+  const CUtensorMapSwizzle sw = swizzle_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                                      : CU_TENSOR_MAP_SWIZZLE_NONE;
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -550,7 +585,7 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
   if (w_cols % 64) return cudaErrorInvalidValue;
   cuuint64_t dims[3] = {64, (cuuint64_t)a.K, (cuuint64_t)(w_cols / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldw * 2, 128};
-  cuuint32_t box[3] = {64, kTcBlockK, (cuuint32_t)chunks};
+  cuuint32_t box[3] = {64, (cuuint32_t)a.block_k, (cuuint32_t)chunks};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.W), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -561,13 +596,14 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a) {
   const uint32_t box_rows = a.geom.tile_m == 256 && a.a_box_256 ? 256u : 128u;
   if (!a.a_cyclic_rows)
-    return make_map_2d(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, kTcBlockK, box_rows);
+    return make_map_2d_sw(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, (uint32_t)a.block_k, box_rows,
+                          a.block_k * 2);
   cuuint64_t dims[3] = {(cuuint64_t)a.K, (cuuint64_t)a.q, (cuuint64_t)a.a_cyclic_rows};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldx * 2, (cuuint64_t)a.ldx * 2 * (cuuint64_t)a.q};
-  cuuint32_t box[3] = {kTcBlockK, 1, box_rows};
+  cuuint32_t box[3] = {(cuuint32_t)a.block_k, 1, box_rows};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.X), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, a.block_k == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }

@@ -45,6 +45,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
       "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+          dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
 // One lane of the (converged) warp; the choice is uniform-friendly, unlike `lane == 0`.
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
@@ -100,13 +108,14 @@ __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bu
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
-// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// offsets (all >> 4), descriptor version 1, swizzle mode (2 = 128-byte, 4 = 64-byte atoms).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint64_t swizzle_mode = 2) {
   uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= 1ull << 46;
-  d |= 2ull << 61;
+  d |= swizzle_mode << 61;
   return d;
 }
 
@@ -210,6 +219,9 @@ cudaError_t make_map_2d(CUtensorMap *map, const void *base, uint64_t inner, uint
                         uint32_t box_inner, uint32_t box_outer);
 cudaError_t make_map_2d_sw(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld_bytes,
                            uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
+// General bf16 map of rank 2..5: dims[rank], byte strides of dims 1..rank-1, box[rank], swizzle 128 / 64 / 32 / 0.
+cudaError_t make_map_nd(CUtensorMap *map, const void *base, int rank, const uint64_t *dims, const uint64_t *stride_bytes,
+                        const uint32_t *box, int swizzle_bytes);
 // A operand of either kind: plain rows (2-D) or, for the cyclic schedule, the type-strided view
 // {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);

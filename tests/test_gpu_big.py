@@ -1,0 +1,138 @@
+"""GPU parity of the large-algebra path (q up to 256, equal group widths in multiples of 8 that need not
+fit the GPU tile; Section "Kernel Benchmarks", appendix "Large Projections and Square Products") against
+the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_32814_b200 import binding, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _types(schedule, M, q, seed):
+    if schedule == "cyclic":
+        return synth.cyclic_types(M, q)
+    if schedule == "interval":
+        return (np.arange(M) // (M // q)).astype(np.int32)
+    return synth.uniform_types(1000 + seed, M, q)
+
+
+def _workload(q, M, s_w, r_w, schedule, integer=True, seed=1):
+    return synth.make_workload("big", config=9, variant=seed, dtype="bf16", q=q, M=M, D=s_w * q, F=r_w * q,
+                               types=_types(schedule, M, q, seed), integer=integer, with_down=False)
+
+
+def _forward(wl, schedule, out_dtype, **kw):
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    assert proj.kernel_path(wl.M) == binding.ALG_PATH_TCGEN05
+    t = H.dev_types(wl.types) if schedule == "explicit" else None
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype, **kw)
+    assert proj.last_status() == 0
+    return Y, proj
+
+
+@pytest.mark.parametrize("q,M,s_w,r_w,schedule", [
+    (64, 64 * 48, 32, 64, "cyclic"),        # q > 32; 48 rows per type: every tile is ragged
+    (40, 40 * 130, 24, 40, "interval"),     # widths no multiple of 16: zero-padded stage, 8-column store masks; 128 + 2 rows
+    (256, 256 * 8, 8, 16, "cyclic"),        # the largest algebra, the narrowest groups
+    (128, 128 * 16, 40, 200, "interval"),   # 5120 -> 25600 at q = 128: blocks of 40 x 200
+    (48, 48 * 256, 64, 128, "interval"),    # 64-deep stages, two full m-tiles per type
+    (8, 1000, 160, 800, "explicit"),        # q <= 32 with widths off the tile grid: bucketing + gather, four 208-wide tiles
+    (4, 515, 80, 304, "explicit"),          # two 160-wide column tiles per group, the second one 144 wide
+    (2, 300, 72, 136, "cyclic"),            # equal buckets of 150 rows, 136 = 128 + 8 columns
+    (3, 301, 24, 40, "cyclic"),             # q does not divide M: counted buckets
+    (5, 640, 96, 264, "explicit"),          # two column tiles of 144 and 120
+])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
+    wl = _workload(q, M, s_w, r_w, schedule, seed=q + M % 13)
+    Y, proj = _forward(wl, schedule, out_dtype)
+    assert proj.gemm_count() == 2 * q * q - q
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+
+
+def test_big_is_the_square_product_of_two_algebra_elements():
+    """Eqs. q-product-diag / q-product-off: C = A * B for n x n arrays of b x b blocks equals the typed
+    projection of A's rows (block row i has type i) through B."""
+    n, b = 1024, 64
+    q = n // b
+    wl = _workload(q, n, b, b, "interval", seed=5)
+    Y, proj = _forward(wl, "interval", torch.float32)
+    ref = oracle.square(wl.X, wl.W_up, [b] * q, [b] * q, [b] * q)
+    assert np.array_equal(H.to_np(Y), ref)
+    rows = [n // q] * q
+    assert proj.macs(rows) == oracle.macs(oracle.support(q), [b] * q, [b] * q, rows)
+
+
+def test_big_counts_follow_the_law_at_large_q():
+    q = 96
+    proj = binding.Proj([16] * q, [24] * q, dtype="bf16", schedule="cyclic")
+    keep = oracle.support(q)
+    rows = list(range(1, q + 1))
+    assert proj.gemm_count() == oracle.gemm_count(keep) == 2 * q * q - q
+    assert proj.macs(rows) == oracle.macs(keep, [16] * q, [24] * q, rows)
+
+
+def test_big_bias_gelu_normal_data_and_strides():
+    q, M, s_w, r_w = 64, 64 * 40, 40, 104
+    wl = _workload(q, M, s_w, r_w, "cyclic", integer=False, seed=3)
+    bias = synth.bf16_round(synth.normal(77, (q * r_w,), 0.1))
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="cyclic")
+    # operands and result inside wider allocations
+    Xp = torch.zeros(M, q * s_w + 24, dtype=torch.bfloat16, device="cuda")
+    Xp[:, :q * s_w] = H.to_dev(wl.X, "bf16")
+    Wp = torch.zeros(q * s_w, q * r_w + 8, dtype=torch.bfloat16, device="cuda")
+    Wp[:, :q * r_w] = H.to_dev(wl.W_up, "bf16")
+    out = torch.full((M, q * r_w + 16), 7.0, dtype=torch.float32, device="cuda")
+    proj.forward(Xp[:, :q * s_w], None, Wp[:, :q * r_w], bias=H.to_dev(bias, "bf16"), act="gelu", out=out[:, :q * r_w])
+    assert proj.last_status() == 0
+    ref = oracle.gelu_array(oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, bias=bias))
+    got = out[:, :q * r_w].cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 5e-3
+    assert np.abs(got - ref).max() <= 2e-2
+    assert torch.all(out[:, q * r_w:] == 7.0)      # nothing is written past N
+
+
+def test_big_static_scratch_and_bad_type():
+    q, M, s_w, r_w = 4, 600, 40, 72
+    wl = _workload(q, M, s_w, r_w, "explicit", seed=11)
+    types = wl.types.copy()
+    types[17] = q + 3
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="explicit")
+    out = torch.empty(M, q * r_w, dtype=torch.float32, device="cuda")
+    proj.forward_static(H.to_dev(wl.X, "bf16"), H.dev_types(types), H.to_dev(wl.W_up, "bf16"), out)
+    assert proj.last_status() == 5
+    good = np.arange(M) != 17
+    ref = oracle.proj(wl.X[good], wl.types[good], wl.W_up, wl.d_widths, wl.f_widths)
+    got = out.cpu().numpy()
+    assert np.array_equal(got[good], ref)
+    assert not got[17].any()
+
+
+def test_big_refusals():
+    with pytest.raises(binding.AlgError):      # explicit types need the table-sized bucketing: q <= 32
+        binding.Proj([32] * 64, [64] * 64, dtype="bf16", schedule="explicit")
+    with pytest.raises(binding.AlgError):      # unequal widths at q > 32
+        binding.Proj([32] * 63 + [64], [64] * 64, dtype="bf16", schedule="cyclic")
+    with pytest.raises(binding.AlgError):      # widths that are no multiple of 8
+        binding.Proj([20] * 64, [100] * 64, dtype="bf16", schedule="cyclic")
+    with pytest.raises(binding.AlgError):
+        binding.Proj([32] * 64, [64] * 64, dtype="f32", schedule="cyclic")
+    with pytest.raises(binding.AlgError):
+        binding.Proj([32] * 64, [64] * 64, dtype="bf16", table="dense", schedule="cyclic")
+    with pytest.raises(binding.AlgError):
+        binding.Proj([8] * 257, [8] * 257, dtype="bf16", schedule="cyclic")
+    proj = binding.Proj([32] * 64, [64] * 64, dtype="bf16", schedule="interval")
+    X = torch.zeros(100, 64 * 32, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(64 * 32, 64 * 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.AlgError):      # q must divide M
+        proj.forward(X, None, W)
+    with pytest.raises(binding.AlgError):
+        proj.set_option("gemm_kernel", 2)

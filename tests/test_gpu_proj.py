@@ -240,6 +240,37 @@ def test_options_tile_width_and_in_kernel_plan():
     assert np.array_equal(H.to_np(Y8), ref[:8])
 
 
+@pytest.mark.parametrize("q,M,s_w,r_w,schedule,tile_n,kernel", [
+    (2, 1000, 384, 768, "explicit", 256, 1),   # 8 stages of 24 KB, ragged tiles, both endpoint products
+    (2, 1000, 384, 768, "explicit", 192, 1),
+    (2, 1026, 128, 384, "cyclic", 128, 1),     # twelve stages of 16 KB, type-strided A view
+    (2, 1337, 256, 384, "explicit", 0, 3),     # 256-row tiles: two A halves per stage
+    (3, 515, 64, 128, "explicit", 0, 1),       # two K blocks of 32 per group
+    (2, 2048, 1536, 384, "cyclic", 0, 3),      # long reduction through the ring many times over
+])
+def test_stage_depth_option_same_bits(q, M, s_w, r_w, schedule, tile_n, kernel):
+    """Stages of 32 and of 64 reduction steps (64- and 128-byte swizzle atoms of the K-major operand) are two
+    pipelines for the same arithmetic."""
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else None
+    wl = _tc_workload(q, M, s_w, r_w, types=types, seed=q * 41 + M % 17)
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    proj.set_option("gemm_kernel", kernel)
+    if tile_n:
+        proj.set_option("tile_n", tile_n)
+    t = None if schedule == "cyclic" else H.dev_types(wl.types)
+    for stage_k in (32, 64, 0):
+        proj.set_option("stage_k", stage_k)
+        for host_plan in (1, 0):
+            proj.set_option("host_plan", host_plan)
+            Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+            assert proj.last_status() == 0
+            bad = np.argwhere(H.to_np(Y) != ref)
+            assert bad.size == 0, f"stage_k {stage_k}: {len(bad)} mismatches, first at {bad[:5].tolist()}"
+    with pytest.raises(binding.AlgError):
+        proj.set_option("stage_k", 48)
+
+
 def test_tc_missing_type_and_single_row():
     wl = _tc_workload(2, 1, 128, 128, types=np.array([1], dtype=np.int32))
     Y, _ = _run_proj(wl, out_dtype=torch.float32)
