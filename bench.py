@@ -16,6 +16,9 @@ count only the block GEMMs the rule keeps.
     pilot              tensor-square law Q_2 (x) Q_2 at the paper's pilot shape (768 -> 1536 -> 768)
     gpilot g8b         gated (SwiGLU) FFN with merged gate/up bank: the pilot's FFN; 4096 -> 12288 at q=32
     train2 train8b     forward + both gradient maps of one projection (768 -> 3072 at q=2; 4096 -> 12288 at q=32)
+    sq4096 .. sq32768  square product of two n x n algebra elements with 128 x 128 blocks (q = n / 128 up to 256)
+    qwu<q>m<M> qwd<q>m<M>  one projection 5120 -> 25600 (u) or 25600 -> 5120 (d) cut into q in {32, 64, 128} equal
+                       groups (blocks 160 x 800 ... 40 x 200), M in {2048, 8192, 32768} rows, type = row block
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
 rank runs the same per-GPU batch (weak scaling), time = max over ranks.
@@ -42,6 +45,7 @@ import numpy as np
 
 METRIC = "star_q FFN kept-GEMM throughput (prefill)"
 UNIT = "TFLOP/s"
+BIG_METRIC = "star_q projection kept-GEMM throughput (large algebra, fixed blocks)"
 N_SETS = 6            # working sets of configuration 2
 L2_BYTES = 126e6
 
@@ -77,6 +81,30 @@ CONFIGS = {
     "4": dict(q=2, D=768, F=3072, M=64, law="qq", schedule="explicit",
               label="cfg4: KV-cached decode step, q=2 FFN 768->3072->768, M in {1,8,32,64}, type = position mod 2, bf16"),
 }
+
+
+def _large_algebra_configs():
+    """Fixed-block workloads of the paper's kernel study (appendix "Large Projections and Square Products");
+    paper_ms = the warm median the paper prints for its own kernel on an H200 NVL, kept for context."""
+    out = {}
+    for n, q, ms in ((4096, 32, 0.044), (8192, 64, 0.166), (16384, 128, 0.689), (32768, 256, 2.868)):
+        out[f"sq{n}"] = dict(big=True, q=q, s=128, r=128, M=n, schedule="interval", paper_ms=ms,
+                             label=f"square product of two n={n} algebra elements, 128x128 blocks (q={q}): typed projection "
+                                   f"{n}->{n} with type = block row, bf16")
+    paper = {("u", 32, 2048): 0.168, ("u", 64, 2048): 0.232, ("u", 128, 2048): 0.248, ("u", 32, 8192): 0.583,
+             ("u", 64, 8192): 0.523, ("u", 128, 8192): 0.401, ("u", 32, 32768): 2.335, ("u", 64, 32768): 2.055,
+             ("u", 128, 32768): 1.558, ("d", 32, 2048): 0.181, ("d", 64, 2048): 0.147, ("d", 128, 2048): 0.174,
+             ("d", 32, 8192): 0.576, ("d", 64, 8192): 0.396, ("d", 128, 8192): 0.411, ("d", 32, 32768): 2.354,
+             ("d", 64, 32768): 1.519, ("d", 128, 32768): 1.684}
+    for (way, q, M), ms in paper.items():
+        K, N = (5120, 25600) if way == "u" else (25600, 5120)
+        out[f"qw{way}{q}m{M}"] = dict(big=True, q=q, s=K // q, r=N // q, M=M, schedule="interval", paper_ms=ms,
+                                      label=f"projection {K}->{N} in q={q} equal groups, X as q x q blocks of {M // q}x{K // q}, "
+                                            f"W of {K // q}x{N // q}, M={M} rows, type = row block, bf16")
+    return out
+
+
+CONFIGS.update(_large_algebra_configs())
 WORKLOAD = CONFIGS["2"]["label"]
 
 
@@ -225,11 +253,47 @@ def oracle_ffn(name, wl, rows, keep):
     return oracle.ffn(wl.X[rows], wl.types[rows], wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
 
 
+def big_oracle_sample(cfg, budget_macs: float = 6.0e10):
+    """Sample of a large-algebra workload the CPU oracle can hold: the rows of the first q' types and the output
+    groups of the same types.  Because B(i,j) = {i,j}, that is the Q_q' projection over the same blocks, and its
+    outputs are outputs of the full problem.  Returns (callable, flops, description)."""
+    import oracle
+    from paper_2609_32814_b200 import synth
+    q, s, r, M = cfg["q"], cfg["s"], cfg["r"], cfg["M"]
+    qs = min(q, 32)
+    per_row = (2 * qs - 1) * s * r
+    n = int(max(qs, min(qs * (M // q), budget_macs // per_row)))
+    n -= n % qs
+    types = synth.cyclic_types(n, qs)
+    X = synth.bf16_round(synth.normal(synth.seed_for(9, 1), (n, qs * s), 1.0))
+    W = synth.bf16_round(synth.normal(synth.seed_for(9, 2), (qs * s, qs * r), 0.02))
+    flops = 2 * n * per_row
+    desc = f"{n} rows of {qs} of the {q} types, output groups of the same types (the Q_{qs} projection over the same {s}x{r} blocks), fp64"
+    return (lambda: oracle.proj(X, types, W, [s] * qs, [r] * qs)), flops, desc
+
+
 def run_reference(args):
     """The oracle as it stands, on the host cores, on a row sample of the same workload."""
     import oracle
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
+        return
+    if CONFIGS[args.config].get("big"):
+        fn, flops, sample = big_oracle_sample(CONFIGS[args.config], 3.0e10)
+        for _ in range(args.warmup):
+            fn()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            fn()
+        dt = (time.perf_counter() - t0) / args.steps
+        val = flops / dt / 1e12
+        print(json.dumps({"impl": "reference", "metric": BIG_METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": CONFIGS[args.config]["label"], "sample": sample},
+                          "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+                          "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
         return
     wl = make_workload(args.config)
     rows, keep, flops = oracle_sample(args.config, wl, 1.0e11)
@@ -279,6 +343,8 @@ def main():
     if args.steps is None:
         args.steps = {"2": 600, "3q4": 300, "3q8": 200, "pilot": 300, "gpilot": 300, "g8b": 100, "4": 20, "train2": 200,
                       "train8b": 100}.get(args.config, 20) if args.impl == "ours" else 3
+        if args.impl == "ours" and CONFIGS[args.config].get("big"):
+            args.steps = 200 if CONFIGS[args.config]["M"] <= 8192 else 50
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else min(args.warmup, 1)
     if args.impl == "reference":
         run_reference(args)
@@ -298,7 +364,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     binding.lib()  # fail loudly if the CUDA library is missing
     ctx = {"world": world, "rank": rank, "local_rank": local_rank, "dist": dist, "torch": torch, "binding": binding}
-    line = run_decode(args, ctx) if args.config == "4" else run_train(args, ctx) if CONFIGS[args.config].get("train") else run_prefill(args, ctx)
+    cfg = CONFIGS[args.config]
+    line = (run_decode(args, ctx) if args.config == "4" else run_train(args, ctx) if cfg.get("train") else
+            run_big(args, ctx) if cfg.get("big") else run_prefill(args, ctx))
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -660,6 +728,128 @@ def run_train(args, ctx):
             "clocks": dict(clocks.summary(), note="sampled during the timed region"),
             "e2e": {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                     "note": "gradients stay on the device in a training step; no host entry point is timed"},
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras}
+
+
+def run_big(args, ctx):
+    """--config sq* / qw*: a step = ONE projection of the large-algebra path (no pre-kernel: the schedules are
+    cyclic or interval with q | M)."""
+    torch, binding = ctx["torch"], ctx["binding"]
+    world, rank, local_rank = ctx["world"], ctx["rank"], ctx["local_rank"]
+    cfg = CONFIGS[args.config]
+    q, s, r, M = cfg["q"], cfg["s"], cfg["r"], cfg["M"]
+    K, N = q * s, q * r
+    stream = torch.cuda.current_stream()
+    proj = binding.Proj([s] * q, [r] * q, dtype="bf16", schedule=cfg["schedule"])
+    assert proj.kernel_path(M) == binding.ALG_PATH_TCGEN05
+    counts = [M // q] * q
+    flops = 2 * proj.macs(counts)
+    set_bytes = (M * K + K * N + M * N) * 2
+    n_sets = 1 if set_bytes > 2 * L2_BYTES else int(min(6, max(2, math.ceil(4 * L2_BYTES / set_bytes))))
+    gen = torch.Generator(device="cuda")
+    sets = []
+    for i in range(n_sets):
+        gen.manual_seed(20260932 + 900 + 16 * rank + i)
+        sets.append({"X": torch.randn((M, K), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16),
+                     "W": (torch.randn((K, N), generator=gen, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16),
+                     "Y": torch.empty((M, N), dtype=torch.bfloat16, device="cuda")})
+    ws = torch.empty(max(256, proj.workspace_bytes(M)), dtype=torch.uint8, device="cuda")
+
+    def step(i, h=proj):
+        s_ = sets[i % n_sets]
+        h.forward(s_["X"], None, s_["W"], out=s_["Y"], workspace=ws, stream=stream)
+
+    def time_steps(n, h=proj, clocks=None):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(n):
+            step(i, h)
+            if clocks is not None and i == 0:
+                clocks.arm()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert proj.last_status() == 0
+    launches0 = binding.launch_count()
+    with ClockSampler(local_rank) as clocks:
+        total_ms = time_steps(args.steps, clocks=clocks)
+    launches = binding.launch_count() - launches0
+    total_ms = max_over_ranks(total_ms, "cuda")
+    peaks = _peaks()
+    region_s = total_ms * 1e-3
+    peak_tf = peaks["bf16_tflops"] if region_s < 0.1 or not peaks["bf16_tflops_sustained"] else peaks["bf16_tflops_sustained"]
+    t_tensor, t_hbm = flops / (peak_tf * 1e12), set_bytes / (peaks["hbm_gbs"] * 1e9)
+    value = whole_job_value(flops, world, args.steps, total_ms)
+    if t_tensor >= t_hbm:
+        roofline = {"bound": "tensor", "achieved": value / world, "peak": peak_tf, "unit": "TFLOP/s", "frac": value / world / peak_tf,
+                    "peak_source": f"{peaks['source']} ({'burst' if peak_tf == peaks['bf16_tflops'] else 'sustained'})"}
+    else:
+        gbs = set_bytes * args.steps / region_s / 1e9
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                    "peak_source": peaks["source"]}
+    roofline.update({"kernel": "proj_big_kernel", "traffic": None, "tensor_time_us": t_tensor * 1e6, "hbm_time_us": t_hbm * 1e6,
+                     "algorithmic_bytes": set_bytes, "algorithmic_flops": flops})
+    ms_step = total_ms / args.steps
+    extras = {"paper": {"ms_per_step": cfg["paper_ms"], "hardware": "H200 NVL, the paper's own kernel, warm median",
+                        "time_ratio_paper_over_ours": cfg["paper_ms"] / ms_step}}
+    e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": M * K * 2, "d2h_bytes_per_step": M * N * 2}
+    if rank == 0 and not args.no_extras:
+        if K % 64 == 0 and N % 128 == 0:
+            dense = binding.Proj([K], [N], dtype="bf16", schedule="cyclic")    # q = 1: the ordinary product X W
+            wsd = torch.empty(max(256, dense.workspace_bytes(M)), dtype=torch.uint8, device="cuda")
+            def dstep(i):
+                s_ = sets[i % n_sets]
+                dense.forward(s_["X"], None, s_["W"], out=s_["Y"], workspace=wsd, stream=stream)
+            def dtime(n):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record(stream)
+                for i in range(n):
+                    dstep(i)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / n
+            dtime(2)
+            est = dtime(1)
+            dense_ms = dtime(int(max(2, min(20, 300.0 / max(est, 1e-3)))))
+            extras["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": ms_step, "time_ratio_star_over_dense": ms_step / dense_ms,
+                                  "control": "same library, q = 1 (ordinary X W on the table-driven tcgen05 kernel)",
+                                  "ideal_ratio": flops / (2.0 * M * K * N)}
+        # end to end through the C ABI's host entry point: pinned X in, Y out, copies inside the timing
+        Xh = sets[0]["X"].cpu().pin_memory()
+        Yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        wsh = torch.empty(proj.host_workspace_bytes(M, torch.bfloat16), dtype=torch.uint8, device="cuda")
+        n_e2e = int(max(2, min(20, 2000.0 / max(1.0, (M * K + M * N) * 2 / 25e6))))
+        for _ in range(2):
+            proj.forward_host(Xh, None, sets[0]["W"], Yh, workspace=wsh, stream=stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(n_e2e):
+            proj.forward_host(Xh, None, sets[0]["W"], Yh, workspace=wsh, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e["value"] = flops * n_e2e / (e0.elapsed_time(e1) * 1e-3) / 1e12
+        e2e["steps"] = n_e2e
+    cpu = None
+    if rank == 0:
+        fn, cflops, sample = big_oracle_sample(cfg)
+        t0 = time.perf_counter()
+        fn()
+        dt = time.perf_counter() - t0
+        cpu = {"value": cflops / dt / 1e12, "unit": UNIT, "cores": __import__("oracle").threads(), "kind": "oracle",
+               "sample": f"{sample}, {dt:.2f} s"}
+    return {"metric": BIG_METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic (generated on the device, seeded)",
+            "config": {"workload": cfg["label"], "rows_per_type": M // q, "tile": "128 rows x ceil16(r / ceil(r / 256)) columns",
+                       "l2": f"{n_sets} working set(s) of {set_bytes / 1e6:.0f} MB used round-robin, L2 is 126 MB"},
+            "clocks": dict(clocks.summary(), note="sampled during the timed region"), "e2e": e2e,
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras}
 
 

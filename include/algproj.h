@@ -298,6 +298,18 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
                                   size_t workspace_bytes, void *stream);
 alg_status_t alg_proj_grad_last_status(alg_proj_grad_t h, void *stream, alg_status_t *status);
 
+/* alg_proj_forward with X, types and Y in HOST memory (packed rows: ldx = K, ldy = N; pinned
+ * memory makes the copies asynchronous): copies X and types to device staging inside the
+ * workspace, runs the projection, copies Y back, all on `stream`; returns without
+ * synchronising.  W and bias stay device pointers.  Workspace size:
+ * alg_proj_host_workspace_bytes (device memory, 256-byte aligned). */
+alg_status_t alg_proj_host_workspace_bytes(alg_proj_t h, int64_t max_M, alg_dtype_t y_dtype,
+                                           size_t *bytes);
+alg_status_t alg_proj_forward_host(alg_proj_t h, const void *X_host, const int32_t *types_host,
+                                   int64_t M, const void *W, int64_t ldw, const void *bias,
+                                   alg_act_t act, void *Y_host, alg_dtype_t y_dtype,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
 /* Same computation with X, types and Y in HOST memory (pinned memory makes the copies
  * asynchronous).  Copies X and types to device staging inside the workspace, runs the
  * forward pass, copies Y back, all on `stream`; returns without synchronising.  Weights and

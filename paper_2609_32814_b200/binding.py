@@ -33,7 +33,7 @@ _SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC, "interval
 
 EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
-    "alg_proj_forward_static", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
+    "alg_proj_forward_static", "alg_proj_host_workspace_bytes", "alg_proj_forward_host", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
     "alg_ffn_gated_create", "alg_ffn_gated_forward", "alg_proj_grad_create", "alg_proj_grad_destroy",
     "alg_proj_grad_workspace_bytes", "alg_proj_grad_input", "alg_proj_grad_weight", "alg_proj_grad_last_status", "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.alg_proj_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
         L.alg_proj_forward.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp, ctypes.c_size_t, vp]
         L.alg_proj_forward_static.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp]
+        L.alg_proj_host_workspace_bytes.argtypes = [vp, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_proj_forward_host.argtypes = [vp, vp, vp, i64, vp, i64, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_proj_gemm_count.argtypes = [vp, ctypes.POINTER(i64)]
         L.alg_proj_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.alg_proj_kernel_path.argtypes = [vp, i64, ctypes.POINTER(i32)]
@@ -201,6 +203,22 @@ class Proj(_Handle):
                                              out.stride(0) if M else self.N, _DTYPES[out.dtype], _stream(stream)),
                "alg_proj_forward_static")
         return out
+
+    def host_workspace_bytes(self, max_M: int, out_dtype) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_proj_host_workspace_bytes(self._h, max_M, _DTYPES[out_dtype], ctypes.byref(out)),
+               "alg_proj_host_workspace_bytes")
+        return out.value
+
+    def forward_host(self, X_host, types_host, W, Y_host, bias=None, act=None, workspace=None, stream=None):
+        """alg_proj_forward_host: X_host / types_host / Y_host are packed CPU tensors (pinned for asynchronous copies)."""
+        M = X_host.shape[0]
+        need = self.host_workspace_bytes(M, Y_host.dtype)
+        ws = workspace if workspace is not None else self._workspace(need, W.device)
+        _check(lib().alg_proj_forward_host(self._h, _ptr(X_host), _ptr(types_host), M, _ptr(W), W.stride(0), _ptr(bias),
+                                           _ACTS[act], _ptr(Y_host), _DTYPES[Y_host.dtype], _ptr(ws), ws.numel(),
+                                           _stream(stream)), "alg_proj_forward_host")
+        return Y_host
 
     def gemm_count(self) -> int:
         n = ctypes.c_int64()

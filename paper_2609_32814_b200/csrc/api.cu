@@ -770,6 +770,40 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   return run_proj(*h, L, ws, X, ldx, false, W, ldw, bias, act, Y, ldy, y_dtype, false, M, st, nullptr, cyc);
 }
 
+alg_status_t alg_proj_host_workspace_bytes(alg_proj_t h, int64_t max_M, alg_dtype_t y_dtype, size_t *bytes) {
+  if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
+  const size_t dev = align_up(layout(*h, nullptr, max_M).total);
+  *bytes = dev + align_up((size_t)max_M * h->K * elem_bytes(h->dtype)) + align_up((size_t)max_M * sizeof(int32_t)) +
+           align_up((size_t)max_M * h->N * elem_bytes(y_dtype));
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_forward_host(alg_proj_t h, const void *X_host, const int32_t *types_host, int64_t M, const void *W,
+                                   int64_t ldw, const void *bias, alg_act_t act, void *Y_host, alg_dtype_t y_dtype,
+                                   void *workspace, size_t workspace_bytes, void *stream) {
+  if (!h || M < 0 || M > (1 << 30)) return ALG_ERR_INVALID_ARG;
+  if (M == 0) return ALG_OK;
+  if (!X_host || !Y_host || !workspace) return ALG_ERR_INVALID_ARG;
+  if (h->sched == ALG_SCHED_EXPLICIT && !types_host) return ALG_ERR_INVALID_ARG;
+  size_t need = 0;
+  alg_status_t s = alg_proj_host_workspace_bytes(h, M, y_dtype, &need);
+  if (s != ALG_OK) return s;
+  if (workspace_bytes < need) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)workspace;
+  const size_t dev = align_up(layout(*h, nullptr, M).total);
+  const size_t xb = (size_t)M * h->K * elem_bytes(h->dtype), tb = (size_t)M * sizeof(int32_t);
+  const size_t yb = (size_t)M * h->N * elem_bytes(y_dtype);
+  char *dX = ws + dev, *dT = dX + align_up(xb), *dY = dT + align_up(tb);
+  if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (types_host && cudaMemcpyAsync(dT, types_host, tb, cudaMemcpyHostToDevice, st) != cudaSuccess) return ALG_ERR_CUDA;
+  s = alg_proj_forward(h, dX, h->K, types_host ? (const int32_t *)dT : nullptr, M, W, ldw, bias, act, dY, h->N, y_dtype, ws, dev,
+                       st);
+  if (s != ALG_OK) return s;
+  return cuda_status(cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, st));
+}
+
 alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
   if (!h || !n) return ALG_ERR_INVALID_ARG;
   int64_t c = 0;

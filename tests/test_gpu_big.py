@@ -116,6 +116,19 @@ def test_big_static_scratch_and_bad_type():
     assert not got[17].any()
 
 
+def test_big_forward_host_matches_device_call():
+    q, M, s_w, r_w = 64, 64 * 20, 24, 56
+    wl = _workload(q, M, s_w, r_w, "interval", seed=21)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="interval")
+    W = H.to_dev(wl.W_up, "bf16")
+    Xh = torch.from_numpy(wl.X.astype(np.float32)).to(torch.bfloat16).pin_memory()
+    Yh = torch.empty(M, q * r_w, dtype=torch.float32).pin_memory()
+    proj.forward_host(Xh, None, W, Yh)
+    torch.cuda.synchronize()
+    assert proj.last_status() == 0
+    assert np.array_equal(Yh.numpy(), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+
+
 def test_big_refusals():
     with pytest.raises(binding.AlgError):      # explicit types need the table-sized bucketing: q <= 32
         binding.Proj([32] * 64, [64] * 64, dtype="bf16", schedule="explicit")
