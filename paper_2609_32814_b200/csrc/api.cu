@@ -209,7 +209,9 @@ void plan_big(alg_proj_s &p, int s, int r) {
   p.big.nt_n = (r + 255) / 256;
   p.big.tile_n = ((r + p.big.nt_n - 1) / p.big.nt_n + 15) / 16 * 16;
   p.big.nt_n = (r + p.big.tile_n - 1) / p.big.tile_n;
-  p.big.block_k = s % 64 == 0 ? 64 : 32;
+  // 64-deep stages whatever the group width: the copy engine is bound by row requests, and a 128-byte row of
+  // X costs one request whether or not part of it is zero fill
+  p.big.block_k = 64;
 }
 
 // Handle of the large-algebra path only (q > kMaxQ or the interval schedule): no interaction table.
@@ -566,7 +568,9 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
   a.M = (int)M, a.q = p.q;
   a.s = p.big.s, a.r = p.big.r;
   a.tile_n = p.big.tile_n, a.nt_n = p.big.nt_n;
-  a.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;   // 64-deep stages only when they divide the group width
+  a.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;
+  a.n_chunks = (a.tile_n + 63) / 64;
+  a.a_box_rows = 128;
   a.offsets = nullptr, a.perm = nullptr;
   a.rows_per_type = 0;
   a.status = p.d_status;
@@ -575,6 +579,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
   if (equal) {
     a.sched = p.sched == ALG_SCHED_INTERVAL ? 1 : 2;
     a.rows_per_type = (int)(M / p.q);
+    a.a_box_rows = (int)std::min<int64_t>(128, (a.rows_per_type + 7) / 8 * 8);   // no type has more rows than that
   } else {
     if (p.sched == ALG_SCHED_INTERVAL || p.q > kMaxQ) return ALG_ERR_INVALID_ARG;   // these need q | M
     BucketArgs b;

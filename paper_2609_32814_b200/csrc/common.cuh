@@ -179,6 +179,8 @@ struct BigArgs {
   int tile_n;             // columns per tile: multiple of 16, <= 256
   int nt_n;               // column tiles per output group = ceil(r / tile_n)
   int block_k;            // 64 or 32: reduction depth of a pipeline stage
+  int n_chunks;           // 64-column boxes of W fetched per stage = ceil(tile_n / 64)
+  int a_box_rows;         // rows of X fetched per stage: 128, or fewer when no type has that many rows
   int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
   const int *offsets;     // sched 0: device bucket offsets [q + 1]
   const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)

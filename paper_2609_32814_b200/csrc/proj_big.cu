@@ -22,6 +22,11 @@
 //    copies of X or W.  Everything stays 16-byte aligned because widths are multiples of 8.
 //  * The MMA width is a launch parameter (tile_n, a multiple of 16), stores are masked per 8
 //    columns.
+//  * What bounds operand fill on one SM is the number of row requests the copy engine makes (about one
+//    row of up to 128 bytes every two cycles), not their bytes.  So a stage is always fetched in rows of
+//    128 bytes (64-deep stages, even for groups narrower than 64: the rest of the row is zero fill), only
+//    the 64-column boxes of W the tile width needs are requested, and when no row type has 128 rows the box
+//    of X is cut to the rows there are (the MMA still spans 128 rows; the unused ones are never stored).
 // Warp roles as in proj_tc.cu: warp 0 = TMA producer of A, warp 10 = TMA producer of B, warp 1 =
 // TMEM allocator + MMA issuer, warps 2..9 = epilogue (TMEM lane quadrant = warp % 4; the two warps
 // of a quadrant alternate over the 32-column chunks).  Double-buffered accumulator; every wait is
@@ -35,6 +40,8 @@
 namespace algproj {
 
 using namespace tc;
+
+ALG_TRACE_DEFINE(proj_big)
 
 namespace {
 
@@ -142,6 +149,9 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   Ctl *ctl = (Ctl *)(store_buf + kEpiWarps * kStoreBufBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = a.q;
+  ALG_TRACE_VARS;
+  ALG_TRACE_CTA(0, 0);
+  if (threadIdx.x == 0) ALG_TRACE(0, 20);
 
   if (warp == 0) {
     if (lane < C::kStages) {
@@ -198,6 +208,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  if (threadIdx.x == 0) ALG_TRACE(0, 24);
   const int nkb_seg = (a.s + BK - 1) / BK;   // pipeline stages per reduction segment (the last one zero-padded)
 
   if (warp == 0 || warp == kProducerWarpB) {
@@ -208,9 +219,11 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     bool ok = true;
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     const uint32_t smem0 = smem_u32(smem);
+    const uint32_t stage_tx = (uint32_t)(a.a_box_rows * BK * 2 + a.n_chunks * C::kBChunkBytes);   // bytes the copies of a stage deliver
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
+      if (loads_a && lane == 0) ALG_TRACE(0, 1);
       const int n_seg = tl.i == tl.j ? 1 : 2;
       const int a_row = a.sched == 2 ? tl.row0 - tl.i * a.rows_per_type : tl.row0;
       for (int sg = 0; sg < n_seg && ok; ++sg) {
@@ -222,12 +235,11 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
           if (elect_one()) {
             if (loads_a) {
-              mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+              mbar_expect_tx(bar, stage_tx);
               if (a.sched == 2) tma_load_4d(sa, &tmA, bar, kb * BK, k, tl.i, a_row);
               else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
             } else {
-#pragma unroll
-              for (int c = 0; c < C::kChunks; ++c)
+              for (int c = 0; c < a.n_chunks; ++c)
                 tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0 + c * 64, kb * BK, k);
             }
           }
@@ -252,13 +264,16 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
       const int n_kb = (tl.i == tl.j ? 1 : 2) * nkb_seg;
+      if (lane == 0) ALG_TRACE(1, 1);
       ok = __all_sync(0xffffffffu, wait_bar(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
       if (!ok) break;
+      if (lane == 0) ALG_TRACE(1, 2);
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
       for (int kb = 0; kb < n_kb; ++kb) {
         ok = __all_sync(0xffffffffu, wait_bar(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
         if (!ok) break;
+        if (kb == 0 && lane == 0) ALG_TRACE(1, 3);
         tc_fence_after();
         const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
@@ -274,6 +289,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (!ok) break;
       if (elect_one()) tc_commit(tfull0 + 8u * (uint32_t)acc);
       __syncwarp();
+      if (lane == 0) ALG_TRACE(1, 4);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
     }
   } else {
@@ -283,11 +299,16 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int half = e >> 2;
     int acc = 0;
     uint32_t acc_phase = 0;
-    uint8_t *buf = store_buf + e * kStoreBufBytes;
-    const uint32_t my_row = smem_u32(buf) + (uint32_t)lane * 64u;
-    const uint32_t sw = (uint32_t)((lane >> 1) & 3);
-    const int sub = lane >> 2, piece = lane & 3;
-    const uint32_t rd_base = smem_u32(buf) + (uint32_t)sub * 64u;
+    // bf16 results leave through a 2 KB staging buffer per warp, 16 rows x 128 bytes at a time: every lane
+    // holds 64 columns of its own row (128 bytes); sixteen lanes write their rows (16-byte pieces
+    // XOR-swizzled by the row, conflict-free both ways), then eight lanes together store one whole row
+    // segment, so one store instruction covers 4 rows x 128 contiguous bytes -- full lines.  What bounds
+    // the store path of an SM is the number of line requests, not their bytes: rows of 64 bytes (32
+    // columns per pass) were measured at about half the store rate.
+    const uint32_t buf0 = smem_u32(store_buf + e * kStoreBufBytes);
+    const uint32_t wr_row = buf0 + (uint32_t)(lane & 15) * 128u;
+    const uint32_t wr_sw = (uint32_t)(lane & 7);
+    const int rd_r = lane >> 3, rd_p = lane & 7;     // row within a group of four, 16-byte piece of the row
     for (int t = blockIdx.x;; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
@@ -302,68 +323,111 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       bool ok = wait_bar(smem_u32(&ctl->tmem_full[acc]), acc_phase, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (e == 0 && lane == 0) ALG_TRACE(2, 1);
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TILE_N);
       const int col_end = tl.n0 + tl.cols;
-      int64_t dst_row[4];
+      // Tiles of this path have short reductions, so the epilogue is the longest chain of a tile: warps
+      // whose 32 rows lie past the tile's last row do nothing.
+      const int c_end = quad * 32 < tl.rows ? tl.cols : 0;
+      if (a.y_bf16) {
+        int64_t dst_row[8];   // rows this lane stores for: phase * 16 + g * 4 + rd_r
 #pragma unroll
-      for (int g = 0; g < 4; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 8 + sub);
+        for (int g = 0; g < 8; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 4 + rd_r);
+        // the two warps of a quadrant alternate over the 64-column chunks
 #pragma unroll 1
-      for (int c0 = half * 32; c0 < tl.cols; c0 += 64) {
-        uint32_t v[32];
-        tc_ld_32x32(taddr + (uint32_t)c0, v);
-        tc_wait_ld();
-        const int col = tl.n0 + c0;
-        float f[32];
+        for (int c0 = half * 64; c0 < c_end; c0 += 128) {
+          uint32_t v0[32], v1[32];
+          const bool second = c0 + 32 < c_end;
+          tc_ld_32x32(taddr + (uint32_t)c0, v0);
+          if (second) tc_ld_32x32(taddr + (uint32_t)(c0 + 32), v1);
+          tc_wait_ld();
+          const int col = tl.n0 + c0;
+          uint32_t w[32];
 #pragma unroll
-        for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
-        if (a.bias) {
-          const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
+          for (int hh = 0; hh < 2; ++hh) {
+            float f[32];
 #pragma unroll
-          for (int x = 0; x < 32; ++x)
-            if (col + x < col_end) f[x] += __bfloat162float(__ldg(b + x));
-        }
-        if (a.act == ALG_ACT_GELU_ERF) {
+            for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(hh ? v1[x] : v0[x]);
+            if (a.bias) {
+              const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col + hh * 32;
 #pragma unroll
-          for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
-        } else if (a.act == ALG_ACT_GELU_TANH) {
+              for (int x = 0; x < 32; ++x)
+                if (col + hh * 32 + x < col_end) f[x] += __bfloat162float(__ldg(b + x));
+            }
+            if (a.act == ALG_ACT_GELU_ERF) {
 #pragma unroll
-          for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
-        }
-        if (a.y_bf16) {
-          // transpose through the warp's staging buffer: one store instruction then covers 8 rows x 64
-          // contiguous bytes; a 16-byte piece is stored when its 8 columns belong to the tile
-          uint32_t w[16];
-          pack_bf16_32(f, w);
-          __syncwarp();
+              for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
+            } else if (a.act == ALG_ACT_GELU_TANH) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g)
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((((uint32_t)g) ^ sw) << 4)), "r"(w[g * 4]),
-                         "r"(w[g * 4 + 1]), "r"(w[g * 4 + 2]), "r"(w[g * 4 + 3])
-                         : "memory");
-          __syncwarp();
-          const bool piece_ok = col + piece * 8 < col_end;
+              for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
+            }
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int rr = g * 8 + sub;
-            const uint32_t rsw = (uint32_t)((rr >> 1) & 3);
-            uint4 val;
-            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
-                         : "r"(rd_base + (uint32_t)g * 512u + ((((uint32_t)piece) ^ rsw) << 4)));
-            if (dst_row[g] >= 0 && piece_ok)
-              *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col + piece * 8) = val;
+            for (int x = 0; x < 16; ++x) {
+              __nv_bfloat162 pk = __floats2bfloat162_rn(f[2 * x], f[2 * x + 1]);
+              w[hh * 16 + x] = *(uint32_t *)&pk;
+            }
           }
-        } else if (out_row >= 0) {
-          float *dst = (float *)a.Y + out_row * a.ldy + col;
+          const bool piece_ok = col + rd_p * 8 < col_end;
 #pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (col + g * 4 < col_end) ((float4 *)dst)[g] = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
+          for (int ph = 0; ph < 2; ++ph) {
+            __syncwarp();   // the previous rows have been read out of the buffer
+            if ((lane >> 4) == ph) {
+#pragma unroll
+              for (int pc = 0; pc < 8; ++pc)
+                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(wr_row + ((((uint32_t)pc) ^ wr_sw) << 4)),
+                             "r"(w[pc * 4]), "r"(w[pc * 4 + 1]), "r"(w[pc * 4 + 2]), "r"(w[pc * 4 + 3])
+                             : "memory");
+            }
+            __syncwarp();
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int rr = g * 4 + rd_r;     // row of the 16 staged ones
+              uint4 val;
+              asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                           : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                           : "r"(buf0 + (uint32_t)rr * 128u + ((((uint32_t)rd_p) ^ (uint32_t)(rr & 7)) << 4)));
+              const int64_t dr = dst_row[ph * 4 + g];
+              if (dr >= 0 && piece_ok) *(uint4 *)((__nv_bfloat16 *)a.Y + dr * a.ldy + col + rd_p * 8) = val;
+            }
+          }
+        }
+      } else {
+        // fp32 results: every lane stores its own row segment
+#pragma unroll 1
+        for (int c0 = half * 32; c0 < c_end; c0 += 64) {
+          uint32_t v[32];
+          tc_ld_32x32(taddr + (uint32_t)c0, v);
+          tc_wait_ld();
+          const int col = tl.n0 + c0;
+          float f[32];
+#pragma unroll
+          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          if (a.bias) {
+            const __nv_bfloat16 *b = (const __nv_bfloat16 *)a.bias + col;
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+              if (col + x < col_end) f[x] += __bfloat162float(__ldg(b + x));
+          }
+          if (a.act == ALG_ACT_GELU_ERF) {
+#pragma unroll
+            for (int x = 0; x < 32; x += 2) gelu_erf2(f[x], f[x + 1]);
+          } else if (a.act == ALG_ACT_GELU_TANH) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
+          }
+          if (out_row >= 0) {
+            float *dst = (float *)a.Y + out_row * a.ldy + col;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              if (col + g * 4 < col_end) ((float4 *)dst)[g] = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
+          }
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+      if (e == 0 && lane == 0) ALG_TRACE(2, 2);
       if (++acc == 2) acc = 0, acc_phase ^= 1u;
     }
   }
@@ -377,6 +441,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
+  ALG_TRACE_CTA(1, 0);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
@@ -400,12 +465,12 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
     // rows of type i are rows i, i + q, ...: {k in group, group, type, position in the type}
     const uint64_t dims[4] = {(uint64_t)a.s, (uint64_t)a.q, (uint64_t)a.q, (uint64_t)a.rows_per_type};
     const uint64_t str[3] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.q};
-    const uint32_t box[4] = {(uint32_t)BK, 1, 1, 128};
+    const uint32_t box[4] = {(uint32_t)BK, 1, 1, (uint32_t)a.a_box_rows};
     e = make_map_nd(&tmA, a.X, 4, dims, str, box, BK * 2);
   } else {
     const uint64_t dims[3] = {(uint64_t)a.s, (uint64_t)a.q, (uint64_t)a.M};
     const uint64_t str[2] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2};
-    const uint32_t box[3] = {(uint32_t)BK, 1, 128};
+    const uint32_t box[3] = {(uint32_t)BK, 1, (uint32_t)a.a_box_rows};
     e = make_map_nd(&tmA, a.X, 3, dims, str, box, BK * 2);
   }
   if (e != cudaSuccess) return e;
@@ -442,7 +507,8 @@ cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
   cudaError_t e = tc_init();
   if (e != cudaSuccess) return e;
   if (a.q < 1 || a.q > kBigMaxQ || a.s % 8 || a.r % 8 || a.tile_n % 16 || a.tile_n < 16 || a.tile_n > 256) return cudaErrorInvalidValue;
-  if (a.nt_n != (a.r + a.tile_n - 1) / a.tile_n) return cudaErrorInvalidValue;
+  if (a.nt_n != (a.r + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
+  if (a.a_box_rows < 8 || a.a_box_rows > 128 || a.a_box_rows % 8) return cudaErrorInvalidValue;
   if (a.tile_n <= 128) return a.block_k == 64 ? launch_t<128, 64>(a, num_sms, st) : launch_t<128, 32>(a, num_sms, st);
   return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);
 }

@@ -58,6 +58,22 @@ def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
 
 
+@pytest.mark.parametrize("q,M,s_w,r_w,schedule", [
+    (64, 64 * 48, 32, 64, "cyclic"),
+    (40, 40 * 130, 24, 40, "interval"),
+    (4, 515, 80, 304, "explicit"),
+])
+def test_big_stage_depth_32_same_bits(q, M, s_w, r_w, schedule):
+    """32-deep stages (64-byte rows of X, 64-byte swizzle atoms) are the other pipeline for the same sums."""
+    wl = _workload(q, M, s_w, r_w, schedule, seed=q + 3)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    proj.set_option("stage_k", 32)
+    t = H.dev_types(wl.types) if schedule == "explicit" else None
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert proj.last_status() == 0
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+
+
 def test_big_is_the_square_product_of_two_algebra_elements():
     """Eqs. q-product-diag / q-product-off: C = A * B for n x n arrays of b x b blocks equals the typed
     projection of A's rows (block row i has type i) through B."""
