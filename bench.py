@@ -186,6 +186,27 @@ class ClockSampler:
                 "reasons": [n for b, n in self.REASONS.items() if mask & b], "samples": len(live)}
 
 
+def extend_clock_record(clocks, step, local_rank, torch):
+    """When the timed region was too short for five clock samples, the same steps run on, untimed, under a
+    second sampler for a quarter of a second so that the clock record covers this load.  Returns the note
+    that goes beside the record."""
+    if len(clocks.armed_samples()) >= 5:
+        return "sampled during the timed region"
+    with ClockSampler(local_rank) as clocks2:
+        t_end = time.time() + 0.25
+        i = 0
+        while time.time() < t_end:
+            for _ in range(20):
+                step(i)
+                i += 1
+            clocks2.arm()
+            torch.cuda.synchronize()
+    clocks.samples = clocks.armed_samples() + clocks2.armed_samples()
+    clocks.t_arm = min([s[2] for s in clocks.samples], default=None)
+    clocks.max_mhz = clocks.max_mhz or clocks2.max_mhz
+    return "timed region too short for five samples: extended by 0.25 s of the same steps, untimed"
+
+
 def max_over_ranks(value: float, device=None) -> float:
     """Multi-rank timing rule: the job is as slow as its slowest rank (no-op without a process group)."""
     import torch
@@ -450,23 +471,7 @@ def run_prefill(args, ctx):
     with ClockSampler(local_rank) as clocks:
         total_ms = time_steps(args.steps, first=args.warmup, clocks=clocks)
     launches = binding.launch_count() - launches0
-    clock_note = "sampled during the timed region"
-    if len(clocks.armed_samples()) < 5:
-        # the timed region is too short for five samples: the same steps run on, untimed, under the
-        # sampler for a quarter of a second so that the clock record covers this load
-        with ClockSampler(local_rank) as clocks2:
-            t_end = time.time() + 0.25
-            i = 0
-            while time.time() < t_end:
-                for _ in range(20):
-                    step(i)
-                    i += 1
-                clocks2.arm()
-                torch.cuda.synchronize()
-        clocks.samples = clocks.armed_samples() + clocks2.armed_samples()
-        clocks.t_arm = min([s[2] for s in clocks.samples], default=None)
-        clocks.max_mhz = clocks.max_mhz or clocks2.max_mhz
-        clock_note = "timed region too short for five samples: extended by 0.25 s of the same steps, untimed"
+    clock_note = extend_clock_record(clocks, step, local_rank, torch)
     total_ms = max_over_ranks(total_ms, "cuda")
     ms_per_step = total_ms / args.steps
     value = whole_job_value(flops, world, args.steps, total_ms)
@@ -779,6 +784,7 @@ def run_big(args, ctx):
     with ClockSampler(local_rank) as clocks:
         total_ms = time_steps(args.steps, clocks=clocks)
     launches = binding.launch_count() - launches0
+    clock_note = extend_clock_record(clocks, step, local_rank, torch)
     total_ms = max_over_ranks(total_ms, "cuda")
     peaks = _peaks()
     region_s = total_ms * 1e-3
@@ -849,7 +855,7 @@ def run_big(args, ctx):
             "data": "synthetic (generated on the device, seeded)",
             "config": {"workload": cfg["label"], "rows_per_type": M // q, "tile": "128 rows x ceil16(r / ceil(r / 256)) columns",
                        "l2": f"{n_sets} working set(s) of {set_bytes / 1e6:.0f} MB used round-robin, L2 is 126 MB"},
-            "clocks": dict(clocks.summary(), note="sampled during the timed region"), "e2e": e2e,
+            "clocks": dict(clocks.summary(), note=clock_note), "e2e": e2e,
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras}
 
 
