@@ -16,6 +16,7 @@ count only the block GEMMs the rule keeps.
     pilot              tensor-square law Q_2 (x) Q_2 at the paper's pilot shape (768 -> 1536 -> 768)
     gpilot g8b         gated (SwiGLU) FFN with merged gate/up bank: the pilot's FFN; 4096 -> 12288 at q=32
     train2 train8b     forward + both gradient maps of one projection (768 -> 3072 at q=2; 4096 -> 12288 at q=32)
+    kp1p7b kp4b kp8b kp30b kpdsv3  the expansion projections of the paper's main kernel table (M = 2048)
     sq4096 .. sq32768  square product of two n x n algebra elements with 128 x 128 blocks (q = n / 128 up to 256)
     qwu<q>m<M> qwd<q>m<M>  one projection 5120 -> 25600 (u) or 25600 -> 5120 (d) cut into q in {32, 64, 128} equal
                        groups (blocks 160 x 800 ... 40 x 200), M in {2048, 8192, 32768} rows, type = row block
@@ -96,6 +97,13 @@ def _large_algebra_configs():
              ("u", 128, 32768): 1.558, ("d", 32, 2048): 0.181, ("d", 64, 2048): 0.147, ("d", 128, 2048): 0.174,
              ("d", 32, 8192): 0.576, ("d", 64, 8192): 0.396, ("d", 128, 8192): 0.411, ("d", 32, 32768): 2.354,
              ("d", 64, 32768): 1.519, ("d", 128, 32768): 1.684}
+    # the paper's main kernel table (M = 2048 rows, the q it selects): model shape -> (K, N, q, its kernel's ms)
+    for name, (K, N, q, ms) in {"kp1p7b": (2048, 6144, 32, 0.0249), "kp4b": (2560, 9728, 32, 0.0511),
+                                "kp8b": (4096, 12288, 32, 0.0636), "kp30b": (2048, 768, 16, 0.0084),
+                                "kpdsv3": (7168, 2048, 16, 0.0283)}.items():
+        out[name] = dict(big=True, q=q, s=K // q, r=N // q, M=2048, schedule="interval", paper_ms=ms,
+                         label=f"projection {K}->{N} in q={q} equal groups, X as q x q blocks of {2048 // q}x{K // q}, "
+                               f"W of {K // q}x{N // q}, M=2048 rows, type = row block, bf16")
     for (way, q, M), ms in paper.items():
         K, N = (5120, 25600) if way == "u" else (25600, 5120)
         out[f"qw{way}{q}m{M}"] = dict(big=True, q=q, s=K // q, r=N // q, M=M, schedule="interval", paper_ms=ms,
