@@ -148,9 +148,10 @@ typedef enum {
  * so a row panel W[S_i, :] is streamed once), the operands are fetched through per-group tensor
  * maps whose out-of-range elements read as zero (a group narrower than the 32- or 64-deep
  * pipeline stage, or a last column tile narrower than the tile, costs arithmetic on zeros but
- * no extra bytes), and stores are masked at 8-column granularity.  With q > ALG_MAX_Q only the
- * CYCLIC and INTERVAL schedules (q | M) are available; fp32 operands, other tables, unequal or
- * odd widths with q > ALG_MAX_Q are refused with ALG_ERR_UNSUPPORTED_SHAPE.  The FFN and gradient
+ * no extra bytes), and stores are masked at 8-column granularity.  All three schedules work
+ * (EXPLICIT and CYCLIC with q not dividing M go through bucketing and a row gather first;
+ * INTERVAL needs q | M); fp32 operands, other tables, unequal or odd widths with q > ALG_MAX_Q
+ * are refused with ALG_ERR_UNSUPPORTED_SHAPE.  The FFN and gradient
  * handles do not take this path.  */
 alg_status_t alg_proj_create(alg_proj_t *out, int q, const int32_t *in_widths,
                              const int32_t *out_widths, alg_dtype_t dtype, alg_table_t table,

@@ -247,7 +247,6 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   for (int g = 1; g < q && big_fits; ++g) big_fits = in_w[g] == in_w[0] && out_w[g] == out_w[0];
   if (q > kMaxQ || sched == ALG_SCHED_INTERVAL) {
     if (!big_fits || (int64_t)q * in_w[0] > (1 << 30) || (int64_t)q * out_w[0] > (1 << 30)) return ALG_ERR_UNSUPPORTED_SHAPE;
-    if (q > kMaxQ && sched == ALG_SCHED_EXPLICIT) return ALG_ERR_UNSUPPORTED_SHAPE;
     return init_big(p, q, in_w[0], out_w[0], sched);
   }
   if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
@@ -356,7 +355,7 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
   WsLayout L;
   size_t off = 0;
   L.hdr = off;
-  off = align_up(off + sizeof(WsHeader));
+  off = align_up(off + std::max(sizeof(WsHeader), (size_t)(first.q + 2) * sizeof(int)));   // more than kMaxQ types: a plain offset array
   L.chunks = off;
   off = align_up(off + (size_t)kMaxBucketChunks * (first.q + 1) * sizeof(int));
   L.perm = off;
@@ -581,13 +580,14 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
     a.rows_per_type = (int)(M / p.q);
     a.a_box_rows = (int)std::min<int64_t>(128, (a.rows_per_type + 7) / 8 * 8);   // no type has more rows than that
   } else {
-    if (p.sched == ALG_SCHED_INTERVAL || p.q > kMaxQ) return ALG_ERR_INVALID_ARG;   // these need q | M
+    if (p.sched == ALG_SCHED_INTERVAL) return ALG_ERR_INVALID_ARG;   // needs q | M
     BucketArgs b;
     b.types = p.sched == ALG_SCHED_CYCLIC ? nullptr : types;
     b.M = (int)M;
     b.q = p.q;
     b.chunk_rows = bucket_chunk_rows(M);
     b.hdr = (WsHeader *)(ws + L.hdr);
+    if (p.q > kMaxQ) b.big_offsets = (int *)(ws + L.hdr);
     b.chunk_counts = (int *)(ws + L.chunks);
     b.perm = (int *)(ws + L.perm);
     b.status = p.d_status;
@@ -601,7 +601,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
     if (launch_gather_rows(X, ldx, b.perm, (int)M, p.K, 2, ws + L.xb, st) != cudaSuccess) return ALG_ERR_CUDA;
     a.sched = 0;
     a.X = ws + L.xb, a.ldx = p.K;
-    a.offsets = b.hdr->offsets;
+    a.offsets = (const int *)(ws + L.hdr);   // WsHeader starts with its offsets
     a.perm = b.perm;
   }
   return cuda_status(launch_proj_big(a, p.num_sms, st));

@@ -31,12 +31,14 @@ __device__ __forceinline__ void write_pad_offsets(WsHeader *hdr, const int *offs
   hdr->pad_offsets[q] = run;
 }
 
-// Kernel 1: per-chunk histograms of the row types (pseudo-type q = out of range).
+// Kernel 1: per-chunk histograms of the row types (pseudo-type q = out of range).  CAP = largest q + 1
+// the instantiation serves: kMaxQ + 1 for table-driven handles, kBigMaxQ + 1 for the large-algebra path.
+template <int CAP>
 __global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
-  __shared__ int s_cnt[kMaxQ + 1];
+  __shared__ int s_cnt[CAP];
   const int tid = threadIdx.x;
   const int nt = a.q + 1;
-  if (tid < nt) s_cnt[tid] = 0;
+  for (int t = tid; t < nt; t += 256) s_cnt[t] = 0;
   __syncthreads();
   const int row_begin = blockIdx.x * a.chunk_rows;
   const int row_end = min(a.M, row_begin + a.chunk_rows);
@@ -46,17 +48,18 @@ __global__ void __launch_bounds__(256) bucket_count_kernel(const BucketArgs a) {
     atomicAdd(&s_cnt[t], 1);
   }
   __syncthreads();
-  if (tid < nt) a.chunk_counts[blockIdx.x * nt + tid] = s_cnt[tid];
+  for (int t = tid; t < nt; t += 256) a.chunk_counts[blockIdx.x * nt + t] = s_cnt[t];
 }
 
 // Kernel 2: every CTA scans the (at most 256) chunk histograms to find the bucket offsets and
 // its own base inside each bucket, then places its rows (stable inside a type).  CTA 0 also
 // publishes the offsets.
+template <int CAP>
 __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a) {
-  __shared__ int s_wcnt[8][kMaxQ + 1];
-  __shared__ int s_total[kMaxQ + 1];
-  __shared__ int s_base[kMaxQ + 1];     // rows of this type in earlier chunks (+ earlier sub-blocks)
-  __shared__ int s_offset[kMaxQ + 2];
+  __shared__ int s_wcnt[8][CAP];
+  __shared__ int s_total[CAP];
+  __shared__ int s_base[CAP];     // rows of this type in earlier chunks (+ earlier sub-blocks)
+  __shared__ int s_offset[CAP + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
   const int n_chunks = gridDim.x;
@@ -91,7 +94,7 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
   const int row_begin = blockIdx.x * a.chunk_rows;
   const int row_end = min(a.M, row_begin + a.chunk_rows);
   for (int r0 = row_begin; r0 < row_end; r0 += 256) {
-    for (int e = tid; e < 8 * (kMaxQ + 1); e += 256) (&s_wcnt[0][0])[e] = 0;
+    for (int e = tid; e < 8 * CAP; e += 256) (&s_wcnt[0][0])[e] = 0;
     __syncthreads();
     const int row = r0 + tid;
     const bool live = row < row_end;
@@ -110,17 +113,19 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
       }
     }
     __syncthreads();
-    if (tid < nt) {
+    for (int t2 = tid; t2 < nt; t2 += 256) {
       int add = 0;
-      for (int w = 0; w < 8; ++w) add += s_wcnt[w][tid];
-      s_base[tid] += add;
+      for (int w = 0; w < 8; ++w) add += s_wcnt[w][t2];
+      s_base[t2] += add;
     }
     __syncthreads();
   }
 
   if (blockIdx.x == 0) {
-    for (int t = tid; t <= nt; t += 256) a.hdr->offsets[t] = s_offset[t];
-    if (tid == 0) write_pad_offsets(a.hdr, s_offset, a.q);
+    // more than kMaxQ types: the offsets go to the caller's array (the fixed header has no room for them)
+    int *offsets = a.big_offsets ? a.big_offsets : a.hdr->offsets;
+    for (int t = tid; t <= nt; t += 256) offsets[t] = s_offset[t];
+    if (tid == 0 && !a.big_offsets) write_pad_offsets(a.hdr, s_offset, a.q);
   }
 }
 
@@ -320,13 +325,21 @@ cudaError_t launch_pdl(void (*kernel)(Args...), int grid, int block, cudaStream_
 }  // namespace
 
 cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
+  if (a.q > kMaxQ) {   // large-algebra path: two kernels, tables sized for kBigMaxQ types
+    if (a.q > kBigMaxQ || !a.big_offsets) return cudaErrorInvalidValue;
+    const int n_chunks = ceil_div(a.M, a.chunk_rows);
+    bucket_count_kernel<kBigMaxQ + 1><<<n_chunks, 256, 0, st>>>(a);
+    bucket_scatter_kernel<kBigMaxQ + 1><<<n_chunks, 256, 0, st>>>(a);
+    count_launch(2);
+    return cudaGetLastError();
+  }
   if (a.M <= 65536 && a.sync) {  // one kernel, every row type read once
     count_launch(1);
     return launch_pdl(bucket_onepass_kernel, ceil_div(a.M, kFusedThreads), kFusedThreads, st, a);
   }
   const int n_chunks = ceil_div(a.M, a.chunk_rows);
-  bucket_count_kernel<<<n_chunks, 256, 0, st>>>(a);
-  bucket_scatter_kernel<<<n_chunks, 256, 0, st>>>(a);
+  bucket_count_kernel<kMaxQ + 1><<<n_chunks, 256, 0, st>>>(a);
+  bucket_scatter_kernel<kMaxQ + 1><<<n_chunks, 256, 0, st>>>(a);
   count_launch(2);
   return cudaGetLastError();
 }

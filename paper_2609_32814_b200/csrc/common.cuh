@@ -72,6 +72,7 @@ struct BucketArgs {
   int q;
   int chunk_rows;        // bucket_chunk_rows(M)
   WsHeader *hdr;
+  int *big_offsets = nullptr;   // q > kMaxQ: bucket offsets [q + 2] go here instead of hdr->offsets
   int *chunk_counts;     // [n_chunks][q+1]
   int *perm;             // [M] bucketed position -> original row
   int *status;           // device status word of the handle

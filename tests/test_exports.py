@@ -36,7 +36,7 @@ def test_status_strings_and_argument_errors_need_no_gpu():
     assert L.alg_proj_create(ctypes.byref(h), 0, wp, wp, 1, 0, None, 0) == 1      # q < 1
     assert L.alg_proj_create(ctypes.byref(h), 257, wp, wp, 1, 0, None, 0) == 1    # q > ALG_MAX_Q_LARGE
     w33 = ctypes.cast((ctypes.c_int32 * 33)(*([128] * 33)), ctypes.c_void_p)
-    assert L.alg_proj_create(ctypes.byref(h), 33, w33, w33, 1, 0, None, 0) == 2   # q > ALG_MAX_Q needs a cyclic or interval schedule
+    assert L.alg_proj_create(ctypes.byref(h), 33, w33, w33, 0, 0, None, 0) == 2   # q > ALG_MAX_Q: bf16 operands only
     assert L.alg_proj_create(ctypes.byref(h), 2, None, wp, 1, 0, None, 0) == 1    # NULL widths
     assert L.alg_proj_create(ctypes.byref(h), 2, wp, wp, 7, 0, None, 0) == 1      # bad dtype
     assert L.alg_proj_create(ctypes.byref(h), 2, wp, wp, 1, 2, None, 0) == 1      # custom table without keep

@@ -45,6 +45,9 @@ def _forward(wl, schedule, out_dtype, **kw):
     (2, 300, 72, 136, "cyclic"),            # equal buckets of 150 rows, 136 = 128 + 8 columns
     (3, 301, 24, 40, "cyclic"),             # q does not divide M: counted buckets
     (5, 640, 96, 264, "explicit"),          # two column tiles of 144 and 120
+    (64, 3000, 32, 64, "explicit"),         # q > 32 with i.i.d. types: bucketing tables for 256 types, ragged buckets
+    (256, 4000, 8, 16, "explicit"),         # some types get a handful of rows
+    (40, 1003, 24, 40, "cyclic"),           # q > 32 and q does not divide M
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
@@ -116,8 +119,8 @@ def test_big_bias_gelu_normal_data_and_strides():
     assert torch.all(out[:, q * r_w:] == 7.0)      # nothing is written past N
 
 
-def test_big_static_scratch_and_bad_type():
-    q, M, s_w, r_w = 4, 600, 40, 72
+@pytest.mark.parametrize("q,M,s_w,r_w", [(4, 600, 40, 72), (48, 700, 16, 24)])
+def test_big_static_scratch_and_bad_type(q, M, s_w, r_w):
     wl = _workload(q, M, s_w, r_w, "explicit", seed=11)
     types = wl.types.copy()
     types[17] = q + 3
@@ -146,8 +149,6 @@ def test_big_forward_host_matches_device_call():
 
 
 def test_big_refusals():
-    with pytest.raises(binding.AlgError):      # explicit types need the table-sized bucketing: q <= 32
-        binding.Proj([32] * 64, [64] * 64, dtype="bf16", schedule="explicit")
     with pytest.raises(binding.AlgError):      # unequal widths at q > 32
         binding.Proj([32] * 63 + [64], [64] * 64, dtype="bf16", schedule="cyclic")
     with pytest.raises(binding.AlgError):      # widths that are no multiple of 8
