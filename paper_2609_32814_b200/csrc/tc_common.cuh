@@ -226,9 +226,6 @@ cudaError_t make_map_nd(CUtensorMap *map, const void *base, int rank, const uint
 // {K, q, M/q} of X with strides {ld, q*ld} and a box of 64 x 1 x 128 (same shared-memory image).
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a);
 cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks);
-// Output as the target of tiled stores of 32 columns x 32 rows (64-byte swizzle): plain rows, or
-// the type-strided view {N, q, M/q} for the cyclic schedule.  Fails when Y is not eligible.
-cudaError_t make_map_y(CUtensorMap *map, const ProjArgs &a);
 
 }  // namespace tc
 }  // namespace algproj
