@@ -77,6 +77,34 @@ def test_big_stage_depth_32_same_bits(q, M, s_w, r_w, schedule):
     assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
 
 
+def _random_case(k):
+    rng = np.random.default_rng(4242 + k)
+    q = int(rng.choice([1, 2, 3, 5, 7, 12, 24, 33, 47, 64, 96, 130, 200, 256]))
+    s_w = 8 * int(rng.integers(1, 13 if q < 100 else 5))
+    r_w = 8 * int(rng.integers(1, 41 if q < 40 else (13 if q < 100 else 5)))
+    schedule = str(rng.choice(["cyclic", "interval", "explicit"]))
+    rows = int(rng.integers(1, 300 if q < 40 else 40))
+    M = q * rows if schedule == "interval" or rng.random() < 0.5 else int(rng.integers(1, q * rows + 1))
+    return q, M, s_w, r_w, schedule
+
+
+@pytest.mark.parametrize("k", range(24))
+def test_big_random_shapes_integer_bit_exact(k):
+    """Seeded random algebra sizes, block shapes, row counts and schedules (whichever kernel the library picks)."""
+    q, M, s_w, r_w, schedule = _random_case(k)
+    wl = _workload(q, M, s_w, r_w, schedule, seed=100 + k)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    t = H.dev_types(wl.types) if schedule == "explicit" else None
+    out_dtype = torch.float32 if k % 2 else torch.bfloat16
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=out_dtype)
+    assert proj.last_status() == 0
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    bad = np.argwhere(H.to_np(Y) != ref)
+    assert bad.size == 0, f"case {(q, M, s_w, r_w, schedule)}: {len(bad)} mismatches, first at {bad[:5].tolist()}"
+
+
 def test_big_is_the_square_product_of_two_algebra_elements():
     """Eqs. q-product-diag / q-product-off: C = A * B for n x n arrays of b x b blocks equals the typed
     projection of A's rows (block row i has type i) through B."""
