@@ -17,9 +17,10 @@ count only the block GEMMs the rule keeps.
     gpilot g8b         gated (SwiGLU) FFN with merged gate/up bank: the pilot's FFN; 4096 -> 12288 at q=32
     train2 train8b     forward + both gradient maps of one projection (768 -> 3072 at q=2; 4096 -> 12288 at q=32)
     kp1p7b kp4b kp8b kp30b kpdsv3  the expansion projections of the paper's main kernel table (M = 2048)
-    sq4096 .. sq32768  square product of two n x n algebra elements with 128 x 128 blocks (q = n / 128 up to 256)
-    qwu<q>m<M> qwd<q>m<M>  one projection 5120 -> 25600 (u) or 25600 -> 5120 (d) cut into q in {32, 64, 128} equal
-                       groups (blocks 160 x 800 ... 40 x 200), M in {2048, 8192, 32768} rows, type = row block
+    sq4096 .. sq32768  square product of two n x n algebra elements with 128 x 128 blocks (q = n / 128 up to 256);
+                       sq<n>b256: the same with 256 x 256 blocks
+    qwu<q>m<M> qwd<q>m<M>  one projection 5120 -> 25600 (u) or 25600 -> 5120 (d) cut into q in {32, 64, 128, 256} equal
+                       groups (blocks 160 x 800 ... 20 x 100), M in {2048, 8192, 32768} rows, type = row block
 
 N > 1 (torchrun): rows shard across ranks, weights replicated, no data-path collective; every
 rank runs the same per-GPU batch (weak scaling), time = max over ranks.
@@ -92,11 +93,17 @@ def _large_algebra_configs():
         out[f"sq{n}"] = dict(big=True, q=q, s=128, r=128, M=n, schedule="interval", paper_ms=ms,
                              label=f"square product of two n={n} algebra elements, 128x128 blocks (q={q}): typed projection "
                                    f"{n}->{n} with type = block row, bf16")
+    for n, q, ms in ((4096, 16, 0.058), (8192, 32, 0.225), (16384, 64, 0.991), (32768, 128, 5.344)):
+        out[f"sq{n}b256"] = dict(big=True, q=q, s=256, r=256, M=n, schedule="interval", paper_ms=ms,
+                                 label=f"square product of two n={n} algebra elements, 256x256 blocks (q={q}): typed projection "
+                                       f"{n}->{n} with type = block row, bf16")
     paper = {("u", 32, 2048): 0.168, ("u", 64, 2048): 0.232, ("u", 128, 2048): 0.248, ("u", 32, 8192): 0.583,
              ("u", 64, 8192): 0.523, ("u", 128, 8192): 0.401, ("u", 32, 32768): 2.335, ("u", 64, 32768): 2.055,
              ("u", 128, 32768): 1.558, ("d", 32, 2048): 0.181, ("d", 64, 2048): 0.147, ("d", 128, 2048): 0.174,
              ("d", 32, 8192): 0.576, ("d", 64, 8192): 0.396, ("d", 128, 8192): 0.411, ("d", 32, 32768): 2.354,
-             ("d", 64, 32768): 1.519, ("d", 128, 32768): 1.684}
+             ("d", 64, 32768): 1.519, ("d", 128, 32768): 1.684,
+             ("u", 256, 2048): 0.266, ("u", 256, 8192): 0.414, ("u", 256, 32768): 1.169,
+             ("d", 256, 2048): 0.243, ("d", 256, 8192): 0.552, ("d", 256, 32768): 1.958}
     # the paper's main kernel table (M = 2048 rows, the q it selects): model shape -> (K, N, q, its kernel's ms)
     for name, (K, N, q, ms) in {"kp1p7b": (2048, 6144, 32, 0.0249), "kp4b": (2560, 9728, 32, 0.0511),
                                 "kp8b": (4096, 12288, 32, 0.0636), "kp30b": (2048, 768, 16, 0.0084),

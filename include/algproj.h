@@ -142,13 +142,16 @@ typedef enum {
  * Large-algebra path (the fixed-block regime of Section "Kernel Benchmarks" and of the appendix
  * "Large Projections and Square Products": q = n / b grows with the matrix, blocks such as
  * 160 x 800 or 40 x 200 that are no multiple of the GPU tile).  Taken for ALG_TABLE_QQ with
- * bf16 operands and EQUAL group widths s, r that are multiples of 8, when q > ALG_MAX_Q (up to
+ * bf16 operands and EQUAL group widths s, r that are multiples of 4, when q > ALG_MAX_Q (up to
  * ALG_MAX_Q_LARGE), when the widths do not fit the ordinary tensor-core path, or when the
  * schedule is INTERVAL.  Same tcgen05 pipeline; tiles are enumerated by arithmetic (type-major,
  * so a row panel W[S_i, :] is streamed once), the operands are fetched through per-group tensor
  * maps whose out-of-range elements read as zero (a group narrower than the 32- or 64-deep
  * pipeline stage, or a last column tile narrower than the tile, costs arithmetic on zeros but
- * no extra bytes), and stores are masked at 8-column granularity.  All three schedules work
+ * no extra bytes), and stores are masked at 8-column granularity.  Widths that are multiples of
+ * 4 but not of 8 (20 x 100) cannot be addressed by tensor maps: every call first repacks X and W
+ * into the workspace with each group widened to the next multiple of 8 (zeros), and stores Y in
+ * 4-column pieces; alg_proj_workspace_bytes accounts for the two repacked operands.  All three schedules work
  * (EXPLICIT and CYCLIC with q not dividing M go through bucketing and a row gather first;
  * INTERVAL needs q | M); fp32 operands, other tables, unequal or odd widths with q > ALG_MAX_Q
  * are refused with ALG_ERR_UNSUPPORTED_SHAPE.  The FFN and gradient

@@ -30,6 +30,8 @@ constexpr int kPlanSlots = 4;
 struct BigPlan {
   bool on = false;
   int s = 0, r = 0;       // width of every input / output group
+  int s_pad = 0, r_pad = 0;   // the same rounded up to multiples of 8: what the tensor maps can address
+  bool repack = false;    // widths that are multiples of 4 only: X and W are repacked with padded groups on every call
   int tile_n = 0, nt_n = 0, block_k = 0;
 };
 
@@ -206,6 +208,8 @@ alg_status_t pick_workers(alg_proj_s &p) {
 void plan_big(alg_proj_s &p, int s, int r) {
   p.big.on = true;
   p.big.s = s, p.big.r = r;
+  p.big.s_pad = (s + 7) / 8 * 8, p.big.r_pad = (r + 7) / 8 * 8;
+  p.big.repack = s % 8 != 0 || r % 8 != 0;
   p.big.nt_n = (r + 255) / 256;
   p.big.tile_n = ((r + p.big.nt_n - 1) / p.big.nt_n + 15) / 16 * 16;
   p.big.nt_n = (r + p.big.tile_n - 1) / p.big.tile_n;
@@ -243,7 +247,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   if (sched != ALG_SCHED_EXPLICIT && sched != ALG_SCHED_CYCLIC && sched != ALG_SCHED_INTERVAL) return ALG_ERR_INVALID_ARG;
   // large-algebra path: Q_q law, bf16, equal widths in multiples of 8
   bool big_fits = allow_big && table == ALG_TABLE_QQ && dtype == ALG_BF16 && in_w[0] > 0 && out_w[0] > 0 &&
-                  in_w[0] % 8 == 0 && out_w[0] % 8 == 0;
+                  in_w[0] % 4 == 0 && out_w[0] % 4 == 0;
   for (int g = 1; g < q && big_fits; ++g) big_fits = in_w[g] == in_w[0] && out_w[g] == out_w[0];
   if (q > kMaxQ || sched == ALG_SCHED_INTERVAL) {
     if (!big_fits || (int64_t)q * in_w[0] > (1 << 30) || (int64_t)q * out_w[0] > (1 << 30)) return ALG_ERR_UNSUPPORTED_SHAPE;
@@ -348,6 +352,7 @@ void free_proj(alg_proj_s &p) {
 
 struct WsLayout {
   size_t hdr = 0, chunks = 0, perm = 0, xb = 0, h = 0, total = 0;
+  size_t xp = 0, wp = 0;   // large-algebra path with widths that are multiples of 4 only: repacked X and W
 };
 
 // `second`: the down projection of an FFN (nullptr for a single projection).
@@ -363,6 +368,12 @@ WsLayout layout(const alg_proj_s &first, const alg_proj_s *second, int64_t M) {
   if (use_tc(first) || first.big.on) {
     L.xb = off;
     off = align_up(off + (size_t)M * first.K * 2, 1024);
+  }
+  if (first.big.on && first.big.repack) {
+    L.xp = off;
+    off = align_up(off + (size_t)M * first.q * first.big.s_pad * 2, 1024);
+    L.wp = off;
+    off = align_up(off + (size_t)first.q * first.big.s_pad * first.q * first.big.r_pad * 2, 1024);
   }
   if (second) {
     L.h = off;
@@ -566,6 +577,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
   a.y_bf16 = y_dtype == ALG_BF16;
   a.M = (int)M, a.q = p.q;
   a.s = p.big.s, a.r = p.big.r;
+  a.r_out = p.big.r;
   a.tile_n = p.big.tile_n, a.nt_n = p.big.nt_n;
   a.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;
   a.n_chunks = (a.tile_n + 63) / 64;
@@ -598,11 +610,25 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
     b.N = p.N;
     b.y_elem_bytes = elem_bytes(y_dtype);
     if (launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
-    if (launch_gather_rows(X, ldx, b.perm, (int)M, p.K, 2, ws + L.xb, st) != cudaSuccess) return ALG_ERR_CUDA;
     a.sched = 0;
-    a.X = ws + L.xb, a.ldx = p.K;
+    if (!p.big.repack) {   // (the repacking pass below gathers the rows itself)
+      if (launch_gather_rows(X, ldx, b.perm, (int)M, p.K, 2, ws + L.xb, st) != cudaSuccess) return ALG_ERR_CUDA;
+      a.X = ws + L.xb, a.ldx = p.K;
+    }
     a.offsets = (const int *)(ws + L.hdr);   // WsHeader starts with its offsets
     a.perm = b.perm;
+  }
+  if (p.big.repack) {
+    // groups widened to multiples of 8 with zeros: X (through the row permutation when there is one, straight from
+    // the caller's rows instead of the gathered copy) and the bank, both rewritten on every call
+    const bool permuted = a.sched == 0;
+    if (launch_pad_groups(X, ldx, permuted ? a.perm : nullptr, (int)M, p.q, p.big.s, p.big.s_pad, 0, 0, ws + L.xp, st) != cudaSuccess)
+      return ALG_ERR_CUDA;
+    if (launch_pad_groups(W, ldw, nullptr, p.K, p.q, p.big.r, p.big.r_pad, p.big.s, p.big.s_pad, ws + L.wp, st) != cudaSuccess)
+      return ALG_ERR_CUDA;
+    a.X = ws + L.xp, a.ldx = (int64_t)p.q * p.big.s_pad;
+    a.W = ws + L.wp, a.ldw = (int64_t)p.q * p.big.r_pad;
+    a.s = p.big.s_pad, a.r = p.big.r_pad;
   }
   return cuda_status(launch_proj_big(a, p.num_sms, st));
 }

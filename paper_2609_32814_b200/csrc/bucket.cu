@@ -10,6 +10,8 @@
 //                       then perm[offset[t] + base[t] + rank_in_chunk] = row  (stable); CTA 0
 //                       publishes the bucket offsets.
 //   kernel 3 (gather):  Xb[d,:] = X[perm[d],:]  -- every type becomes a contiguous M-slab.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace algproj {
@@ -322,7 +324,53 @@ cudaError_t launch_pdl(void (*kernel)(Args...), int grid, int block, cudaStream_
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
+// Column groups of c elements widened to c_pad (zeros), optionally row groups of rs rows widened to rs_pad (zero
+// rows); a thread moves 4 elements (8 bytes) of one destination row (blockIdx.y walks the rows).
+__global__ void __launch_bounds__(256) pad_groups_kernel(const uint2 *__restrict__ src, int64_t ld_src4, const int *__restrict__ perm,
+                                                         int rows_dst, int n_col_groups, int c4, int c_pad4, int rs, int rs_pad,
+                                                         uint2 *__restrict__ dst) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // perm may come from the previous kernel
+  const int w4 = n_col_groups * c_pad4;                 // 8-byte pieces per destination row
+  for (int R = blockIdx.y; R < rows_dst; R += gridDim.y) {
+    int64_t src_row = R;
+    bool row_live = true;
+    if (rs > 0) {
+      const int gr = R / rs_pad, kr = R - gr * rs_pad;
+      row_live = kr < rs;
+      src_row = (int64_t)gr * rs + kr;
+    } else if (perm) {
+      src_row = __ldg(perm + R);
+    }
+    const uint2 *srow = src + src_row * ld_src4;
+    uint2 *drow = dst + (int64_t)R * w4;
+    for (int x = blockIdx.x * 256 + threadIdx.x; x < w4; x += gridDim.x * 256) {
+      const int gc = x / c_pad4, cc = x - gc * c_pad4;
+      drow[x] = (row_live && cc < c4) ? __ldg(srow + gc * c4 + cc) : make_uint2(0u, 0u);
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_pad_groups(const void *src, int64_t ld_src, const int *perm, int rows_src, int n_col_groups, int c, int c_pad,
+                              int rs, int rs_pad, void *dst, cudaStream_t st) {
+  if (c % 4 || c_pad % 4 || ld_src % 4 || c_pad < c || (rs > 0 && (rs_pad < rs || rows_src % rs))) return cudaErrorInvalidValue;
+  const int rows_dst = rs > 0 ? rows_src / rs * rs_pad : rows_src;
+  const int w4 = n_col_groups * (c_pad / 4);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)std::max(1, std::min((w4 + 255) / 256, 8)), (unsigned)std::max(1, std::min(rows_dst, 148 * 8)), 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  count_launch(1);
+  return cudaLaunchKernelEx(&cfg, pad_groups_kernel, (const uint2 *)src, (int64_t)(ld_src / 4), perm, rows_dst, n_col_groups, c / 4,
+                            c_pad / 4, rs, rs_pad, (uint2 *)dst);
+}
 
 cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
   if (a.q > kMaxQ) {   // large-algebra path: two kernels, tables sized for kBigMaxQ types

@@ -176,7 +176,8 @@ struct BigArgs {
   int64_t ldy;
   int y_bf16;
   int M, q;
-  int s, r;               // width of every input / output group (multiples of 8)
+  int s, r;               // width of every input / output group as the operands hold them (multiples of 8)
+  int r_out;              // width of an output group in Y (a multiple of 4; < r when W was repacked with padding)
   int tile_n;             // columns per tile: multiple of 16, <= 256
   int nt_n;               // column tiles per output group = ceil(r / tile_n)
   int block_k;            // 64 or 32: reduction depth of a pipeline stage
@@ -190,6 +191,11 @@ struct BigArgs {
   long long wait_limit;
 };
 cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st);
+// dst[R, gc * c_pad + cc] = src[row(R), gc * c + cc] for cc < c, else 0 -- column groups of c elements widened to
+// c_pad; with rs > 0 the rows are grouped too (rs -> rs_pad, the extra rows zero).  perm (optional) maps a
+// destination row to its source row (rows without row groups only).  c, c_pad multiples of 4; bf16.
+cudaError_t launch_pad_groups(const void *src, int64_t ld_src, const int *perm, int rows_src, int n_col_groups, int c, int c_pad,
+                              int rs, int rs_pad, void *dst, cudaStream_t st);
 
 // tcgen05 paths.  One-CTA kernel: 128-row tiles, tile_n in {128, 192, 256}.  CTA-pair kernel
 // (cta_group::2): 256-row tiles, 256 columns wide with a 128-column remainder tile.

@@ -22,6 +22,12 @@
 //    copies of X or W.  Everything stays 16-byte aligned because widths are multiples of 8.
 //  * The MMA width is a launch parameter (tile_n, a multiple of 16), stores are masked per 8
 //    columns.
+//  * Group widths that are multiples of 4 but not of 8 (20 x 100: the q = 256 split of 5120 -> 25600) cannot be
+//    addressed by tensor maps (boxes start on 16 bytes).  For those the caller of this file repacks X and W with
+//    every group widened to the next multiple of 8 (zeros; pad_groups_kernel in bucket.cu) and passes the
+//    repacked widths as s, r and the width of Y's groups as r_out; stores then go in 8-byte pieces.  (Staging the
+//    unpadded operands with 8-byte asynchronous copies from two producer warps was built first: bit-exact, but
+//    each copy instruction took ~200 cycles to issue with the loads missing L2, 2-10 x slower than repacking.)
 //  * What bounds operand fill on one SM is the number of row requests the copy engine makes (about one
 //    row of up to 128 bytes every two cycles), not their bytes.  So a stage is always fetched in rows of
 //    128 bytes (64-deep stages, even for groups narrower than 64: the rest of the row is zero fill), only
@@ -101,14 +107,15 @@ struct Cfg {
 struct Tile {
   int row0, rows;   // bucketed rows [row0, row0 + rows), all of type i; row0 < 0: no more tiles
   int i, j;
-  int n0, cols;     // absolute first column, valid columns (<= tile_n)
+  int n0, cols;     // absolute first column in Y, valid columns (<= tile_n)
+  int n0_w;         // first column in the bank (differs from n0 when the bank's groups are padded)
 };
 
 // Tile t of the launch (uniform across the warp).  Type-major; inside a type: m-tile fastest, then
 // the column tile, then the output group.
 __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, int t) {
   Tile o;
-  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0;
+  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0;
   if (t >= ctl->total) return o;
   int i, rem, base, rows_i;
   if (a.sched != 0) {
@@ -134,8 +141,9 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   o.row0 = base + (mt << 7);
   o.rows = min(128, rows_i - (mt << 7));
   o.i = i, o.j = j;
-  o.n0 = j * a.r + nt * a.tile_n;
-  o.cols = min(a.tile_n, a.r - nt * a.tile_n);
+  o.n0 = j * a.r_out + nt * a.tile_n;
+  o.n0_w = j * a.r + nt * a.tile_n;
+  o.cols = min(a.tile_n, a.r_out - nt * a.tile_n);
   return o;
 }
 
@@ -240,7 +248,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
             } else {
               for (int c = 0; c < a.n_chunks; ++c)
-                tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0 + c * 64, kb * BK, k);
+                tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0_w + c * 64, kb * BK, k);
             }
           }
           __syncwarp();
@@ -309,6 +317,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t wr_row = buf0 + (uint32_t)(lane & 15) * 128u;
     const uint32_t wr_sw = (uint32_t)(lane & 7);
     const int rd_r = lane >> 3, rd_p = lane & 7;     // row within a group of four, 16-byte piece of the row
+    const bool store8 = (a.r_out & 7) != 0;
     for (int t = blockIdx.x;; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
@@ -388,7 +397,13 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                            : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
                            : "r"(buf0 + (uint32_t)rr * 128u + ((((uint32_t)rd_p) ^ (uint32_t)(rr & 7)) << 4)));
               const int64_t dr = dst_row[ph * 4 + g];
-              if (dr >= 0 && piece_ok) *(uint4 *)((__nv_bfloat16 *)a.Y + dr * a.ldy + col + rd_p * 8) = val;
+              if (store8) {   // output groups start on 8 bytes only: two 4-column pieces, each stored if it belongs to the tile
+                __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + dr * a.ldy + col + rd_p * 8;
+                if (dr >= 0 && piece_ok) *(uint2 *)dst = make_uint2(val.x, val.y);
+                if (dr >= 0 && col + rd_p * 8 + 4 < col_end) *(uint2 *)(dst + 4) = make_uint2(val.z, val.w);
+              } else if (dr >= 0 && piece_ok) {
+                *(uint4 *)((__nv_bfloat16 *)a.Y + dr * a.ldy + col + rd_p * 8) = val;
+              }
             }
           }
         }
@@ -507,7 +522,8 @@ cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
   cudaError_t e = tc_init();
   if (e != cudaSuccess) return e;
   if (a.q < 1 || a.q > kBigMaxQ || a.s % 8 || a.r % 8 || a.tile_n % 16 || a.tile_n < 16 || a.tile_n > 256) return cudaErrorInvalidValue;
-  if (a.nt_n != (a.r + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
+  if (a.r_out % 4 || a.r_out < 4 || a.r_out > a.r) return cudaErrorInvalidValue;
+  if (a.nt_n != (a.r_out + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
   if (a.a_box_rows < 8 || a.a_box_rows > 128 || a.a_box_rows % 8) return cudaErrorInvalidValue;
   if (a.tile_n <= 128) return a.block_k == 64 ? launch_t<128, 64>(a, num_sms, st) : launch_t<128, 32>(a, num_sms, st);
   return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);

@@ -48,6 +48,11 @@ def _forward(wl, schedule, out_dtype, **kw):
     (64, 3000, 32, 64, "explicit"),         # q > 32 with i.i.d. types: bucketing tables for 256 types, ragged buckets
     (256, 4000, 8, 16, "explicit"),         # some types get a handful of rows
     (40, 1003, 24, 40, "cyclic"),           # q > 32 and q does not divide M
+    (256, 256 * 16, 20, 100, "interval"),   # widths that are multiples of 4 only: the q = 256 split of 5120 -> 25600
+    (64, 64 * 130, 20, 100, "cyclic"),      # the same blocks, two m-tiles per type, type-strided rows
+    (12, 777, 100, 36, "explicit"),         # groups deeper than one stage (64 + 36): full and zero-padded stages share the ring
+    (4, 300, 132, 292, "explicit"),         # three stages per group, two column tiles (160 + 132)
+    (48, 48 * 8, 4, 4, "interval"),         # the narrowest groups there are
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
@@ -179,8 +184,8 @@ def test_big_forward_host_matches_device_call():
 def test_big_refusals():
     with pytest.raises(binding.AlgError):      # unequal widths at q > 32
         binding.Proj([32] * 63 + [64], [64] * 64, dtype="bf16", schedule="cyclic")
-    with pytest.raises(binding.AlgError):      # widths that are no multiple of 8
-        binding.Proj([20] * 64, [100] * 64, dtype="bf16", schedule="cyclic")
+    with pytest.raises(binding.AlgError):      # widths that are no multiple of 4
+        binding.Proj([18] * 64, [100] * 64, dtype="bf16", schedule="cyclic")
     with pytest.raises(binding.AlgError):
         binding.Proj([32] * 64, [64] * 64, dtype="f32", schedule="cyclic")
     with pytest.raises(binding.AlgError):
