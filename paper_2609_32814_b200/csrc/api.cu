@@ -582,6 +582,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
   a.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;
   a.n_chunks = (a.tile_n + 63) / 64;
   a.a_box_rows = 128;
+  a.pack = 1;
   a.offsets = nullptr, a.perm = nullptr;
   a.rows_per_type = 0;
   a.status = p.d_status;

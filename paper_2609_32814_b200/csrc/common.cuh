@@ -183,6 +183,7 @@ struct BigArgs {
   int block_k;            // 64 or 32: reduction depth of a pipeline stage
   int n_chunks;           // 64-column boxes of W fetched per stage = ceil(tile_n / 64)
   int a_box_rows;         // rows of X fetched per stage: 128, or fewer when no type has that many rows
+  int pack;               // set by the launcher: row types per tile (> 1 when a type has at most 64 rows; sched 1, 2)
   int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
   const int *offsets;     // sched 0: device bucket offsets [q + 1]
   const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)

@@ -28,6 +28,13 @@
 //    repacked widths as s, r and the width of Y's groups as r_out; stores then go in 8-byte pieces.  (Staging the
 //    unpadded operands with 8-byte asynchronous copies from two producer warps was built first: bit-exact, but
 //    each copy instruction took ~200 cycles to issue with the loads missing L2, 2-10 x slower than repacking.)
+//  * Types with at most 64 rows (large q at moderate M) would leave most of a 128-row tile empty, and every
+//    tile costs its epilogue and its hand-overs whatever it holds.  With equal buckets a tile then takes
+//    P = 128 / rows-per-type consecutive types: ONE diagonal segment x_j W_jj for all its rows (the map is the
+//    same for every type), then one panel segment x_i W_ij per type i != j whose A block is fetched through a
+//    view {s, group, row in type, type} with a 128-row box placed so that type i's rows land where they sit in
+//    the tile and every other row is out of range, i.e. zero: the product adds nothing to the other types'
+//    rows.  1 + P segments and one epilogue instead of 2 P segments and P epilogues.
 //  * What bounds operand fill on one SM is the number of row requests the copy engine makes (about one
 //    row of up to 128 bytes every two cycles), not their bytes.  So a stage is always fetched in rows of
 //    128 bytes (64-deep stages, even for groups narrower than 64: the rest of the row is zero fill), only
@@ -106,7 +113,8 @@ struct Cfg {
 
 struct Tile {
   int row0, rows;   // bucketed rows [row0, row0 + rows), all of type i; row0 < 0: no more tiles
-  int i, j;
+  int i, j;         // packed tiles: i = first of np consecutive types
+  int np;
   int n0, cols;     // absolute first column in Y, valid columns (<= tile_n)
   int n0_w;         // first column in the bank (differs from n0 when the bank's groups are padded)
 };
@@ -115,8 +123,21 @@ struct Tile {
 // the column tile, then the output group.
 __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, int t) {
   Tile o;
-  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0;
+  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0, o.np = 1;
   if (t >= ctl->total) return o;
+  if (a.pack > 1) {   // type-group major, then the output group, then the column tile
+    const int per_group = a.q * a.nt_n;
+    const int tg = t / per_group, rem = t - tg * per_group;
+    const int j = rem / a.nt_n, nt = rem - j * a.nt_n;
+    o.i = tg * a.pack, o.j = j;
+    o.np = min(a.pack, a.q - o.i);
+    o.row0 = o.i * a.rows_per_type;
+    o.rows = o.np * a.rows_per_type;
+    o.n0 = j * a.r_out + nt * a.tile_n;
+    o.n0_w = j * a.r + nt * a.tile_n;
+    o.cols = min(a.tile_n, a.r_out - nt * a.tile_n);
+    return o;
+  }
   int i, rem, base, rows_i;
   if (a.sched != 0) {
     rows_i = a.rows_per_type;
@@ -149,7 +170,8 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
 
 template <int TILE_N, int BK>
 __global__ void __launch_bounds__(kThreads, 1)
-proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const BigArgs a) {
+proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
+                const __grid_constant__ CUtensorMap tmB, const BigArgs a) {
   using C = Cfg<TILE_N, BK>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -181,13 +203,16 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   } else if (warp == 3 && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    if (a.pack > 1) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA2) : "memory");
   }
   // Everything above touches only this CTA's own state and may overlap the previous kernel of the stream.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 2) {
     // tile counts: one warp turns the bucket offsets into "tiles before type i"
-    if (a.sched != 0) {
+    if (a.pack > 1) {
+      if (lane == 0) ctl->total = ((q + a.pack - 1) / a.pack) * q * a.nt_n;
+    } else if (a.sched != 0) {
       if (lane == 0) ctl->total = q * ((a.rows_per_type + 127) >> 7) * q * a.nt_n;
     } else {
       int carry = 0;
@@ -232,17 +257,34 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
       if (loads_a && lane == 0) ALG_TRACE(0, 1);
-      const int n_seg = tl.i == tl.j ? 1 : 2;
+      const bool packed = a.pack > 1;
+      // packed tile: segment 0 is the diagonal one (group j), then one panel segment per type of the tile other than j
+      const int j_in = packed && tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0;
+      const int n_seg = packed ? 1 + tl.np - j_in : (tl.i == tl.j ? 1 : 2);
       const int a_row = a.sched == 2 ? tl.row0 - tl.i * a.rows_per_type : tl.row0;
       for (int sg = 0; sg < n_seg && ok; ++sg) {
-        const int k = n_seg == 1 ? tl.i : (sg == 0 ? min(tl.i, tl.j) : max(tl.i, tl.j));
+        int k;
+        if (packed) {
+          k = sg == 0 ? tl.j : tl.i + sg - 1;
+          if (sg > 0 && j_in && k >= tl.j) ++k;   // skip type j: its rows have their one product already
+        } else {
+          k = n_seg == 1 ? tl.i : (sg == 0 ? min(tl.i, tl.j) : max(tl.i, tl.j));
+        }
         for (int kb = 0; kb < nkb_seg; ++kb) {
           ok = __all_sync(0xffffffffu, wait_bar(empty0 + 8u * (uint32_t)stage, phase ^ 1u, ctl, a.status));
           if (!ok) break;
           const uint32_t bar = full0 + 8u * (uint32_t)stage;
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
           if (elect_one()) {
-            if (loads_a) {
+            if (loads_a && packed) {
+              if (sg == 0) {   // all rows of the tile: np types x rows_per_type rows, type-major
+                mbar_expect_tx(bar, (uint32_t)(a.pack * a.rows_per_type * BK * 2 + a.n_chunks * C::kBChunkBytes));
+                tma_load_4d(sa, &tmA, bar, kb * BK, k, 0, tl.i);
+              } else {         // the rows of type k where they sit in the tile, zeros everywhere else
+                mbar_expect_tx(bar, (uint32_t)(128 * BK * 2 + a.n_chunks * C::kBChunkBytes));
+                tma_load_4d(sa, &tmA2, bar, kb * BK, k, -(k - tl.i) * a.rows_per_type, k);
+              }
+            } else if (loads_a) {
               mbar_expect_tx(bar, stage_tx);
               if (a.sched == 2) tma_load_4d(sa, &tmA, bar, kb * BK, k, tl.i, a_row);
               else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
@@ -271,7 +313,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
-      const int n_kb = (tl.i == tl.j ? 1 : 2) * nkb_seg;
+      const int n_kb = (a.pack > 1 ? 1 + tl.np - (tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0) : (tl.i == tl.j ? 1 : 2)) * nkb_seg;
       if (lane == 0) ALG_TRACE(1, 1);
       ok = __all_sync(0xffffffffu, wait_bar(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
       if (!ok) break;
@@ -324,7 +366,10 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int r = quad * 32 + lane;
       int64_t out_row = -1;
       if (r < tl.rows) {
-        if (a.sched == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
+        if (a.sched == 2 && a.pack > 1) {   // rows of a packed tile are type-major: type tl.i + r / rows_per_type
+          const int ti = r / a.rows_per_type;
+          out_row = (int64_t)(r - ti * a.rows_per_type) * q + tl.i + ti;
+        } else if (a.sched == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
         else if (a.sched == 0 && a.perm) out_row = __ldg(a.perm + tl.row0 + r);
         else out_row = tl.row0 + r;
         if (out_row >= a.M) out_row = -1;
@@ -474,9 +519,22 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
     attr_set = true;
   }
   static_assert(C::kSmemBytes <= 227 * 1024, "shared memory budget");
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmA2, tmB;
   cudaError_t e;
-  if (a.sched == 2) {
+  BigArgs b = a;
+  // several types per tile when a type fills at most half of one (equal buckets only)
+  b.pack = a.sched != 0 && a.rows_per_type <= 64 ? std::min(a.q, 128 / a.rows_per_type) : 1;
+  if (b.pack > 1) {
+    // X as {k in group, group, row in type, type}: interval rows of a type are consecutive, cyclic ones q apart
+    const uint64_t rpt = (uint64_t)a.rows_per_type;
+    const uint64_t dims[4] = {(uint64_t)a.s, (uint64_t)a.q, rpt, (uint64_t)a.q};
+    const uint64_t str_i[3] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * rpt};
+    const uint64_t str_c[3] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.q, (uint64_t)a.ldx * 2};
+    const uint32_t box_d[4] = {(uint32_t)BK, 1, (uint32_t)a.rows_per_type, (uint32_t)b.pack};
+    const uint32_t box_p[4] = {(uint32_t)BK, 1, 128, 1};
+    e = make_map_nd(&tmA, a.X, 4, dims, a.sched == 2 ? str_c : str_i, box_d, BK * 2);
+    if (e == cudaSuccess) e = make_map_nd(&tmA2, a.X, 4, dims, a.sched == 2 ? str_c : str_i, box_p, BK * 2);
+  } else if (a.sched == 2) {
     // rows of type i are rows i, i + q, ...: {k in group, group, type, position in the type}
     const uint64_t dims[4] = {(uint64_t)a.s, (uint64_t)a.q, (uint64_t)a.q, (uint64_t)a.rows_per_type};
     const uint64_t str[3] = {(uint64_t)a.s * 2, (uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.q};
@@ -489,6 +547,7 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
     e = make_map_nd(&tmA, a.X, 3, dims, str, box, BK * 2);
   }
   if (e != cudaSuccess) return e;
+  if (b.pack <= 1) tmA2 = tmA;
   {
     // the bank as {columns, k in group, group}: rows past the group's width read as zero
     const uint64_t dims[3] = {(uint64_t)a.q * (uint64_t)a.r, (uint64_t)a.s, (uint64_t)a.q};
@@ -498,7 +557,8 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   }
   if (e != cudaSuccess) return e;
   long long tiles;
-  if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * a.q * a.nt_n;
+  if (b.pack > 1) tiles = (long long)((a.q + b.pack - 1) / b.pack) * a.q * a.nt_n;
+  else if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * a.q * a.nt_n;
   else tiles = ((long long)a.M / 128 + a.q) * a.q * a.nt_n;   // upper bound: every type may end in a ragged tile
   if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
@@ -511,7 +571,7 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_big_kernel<TILE_N, BK>, tmA, tmB, a);
+  e = cudaLaunchKernelEx(&cfg, proj_big_kernel<TILE_N, BK>, tmA, tmA2, tmB, b);
   count_launch(1);
   return e;
 }

@@ -53,6 +53,11 @@ def _forward(wl, schedule, out_dtype, **kw):
     (12, 777, 100, 36, "explicit"),         # groups deeper than one stage (64 + 36): full and zero-padded stages share the ring
     (4, 300, 132, 292, "explicit"),         # three stages per group, two column tiles (160 + 132)
     (48, 48 * 8, 4, 4, "interval"),         # the narrowest groups there are
+    (35, 35 * 40, 24, 40, "cyclic"),        # three types per tile, the last tile holds two; type-strided rows
+    (35, 35 * 40, 24, 40, "interval"),
+    (50, 50, 16, 24, "interval"),           # one row per type: fifty types in one tile
+    (7, 7 * 64, 64, 128, "interval"),       # two types per tile, the last one alone
+    (20, 20 * 33, 8, 264, "cyclic"),        # 33 rows per type (three per tile, boxes off the 8-row swizzle atom), two column tiles
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
