@@ -520,6 +520,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.gated_f = p.gated ? p.N : 0;
   a.w_kmajor = p.w_kmajor ? 1 : 0;
   a.dyn_so = nullptr;
+  a.seg_rows = 0;
   a.block_k = block_k_of(p);
   a.y_staged = 0;
   a.plan = nullptr;
@@ -1035,6 +1036,10 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   alg_proj_s &p = h->dw;
   const int mp = padded_rows(*h, M);
   WsHeader *hdr = (WsHeader *)(ws + L.hdr);
+  // Cyclic schedule with whole 64-row blocks per type: the buckets are rows t, t + q, ... of X and of G as they
+  // lie in memory, nothing is counted, permuted, transposed or copied (the kernel reads both through
+  // type-strided views and takes the X block as an MN-major A operand).
+  const bool in_place = h->sched == ALG_SCHED_CYCLIC && M > 0 && M % (64 * (int64_t)h->q) == 0 && block_k_of(p) == 64;
   // 1. row buckets of this batch (also for the cyclic schedule: the copies below need the permutation)
   BucketArgs b;
   b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
@@ -1049,14 +1054,16 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   b.wait_limit = p.wait_limit;
   b.Y = nullptr;   // nothing to zero: a row with an out-of-range type simply contributes to no block
   b.ldy = 0, b.N = 0, b.y_elem_bytes = 0;
-  if (M > 0 && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (M > 0 && !in_place && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (M == 0) {   // no rows: every block of dW is zero
     return cuda_status(cudaMemset2DAsync(dW, (size_t)lddw * elem_bytes(w_dtype), 0, (size_t)h->N * elem_bytes(w_dtype),
                                          (size_t)h->K, st));
   }
   // 2. padded, bucketed copies: X transposed (K x m_pad), G as it is (m_pad x N); pad rows are zero
-  if (launch_gather_transpose_padded(X, ldx, hdr, b.perm, h->q, mp, h->K, ws + L.xt, st) != cudaSuccess) return ALG_ERR_CUDA;
-  if (launch_gather_rows_padded(G, ldg, hdr, b.perm, h->q, mp, h->N, ws + L.gp, st) != cudaSuccess) return ALG_ERR_CUDA;
+  if (!in_place) {
+    if (launch_gather_transpose_padded(X, ldx, hdr, b.perm, h->q, mp, h->K, ws + L.xt, st) != cudaSuccess) return ALG_ERR_CUDA;
+    if (launch_gather_rows_padded(G, ldg, hdr, b.perm, h->q, mp, h->N, ws + L.gp, st) != cudaSuccess) return ALG_ERR_CUDA;
+  }
   // 3. the grouped GEMM: rows = input features (type = their group), reduction over the padded buckets
   ProjArgs a;
   const TcChoice tc = {tile_m_of(p), tile_n_of(p), &p.tab, p.d_tab};
@@ -1076,17 +1083,17 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   a.q = p.q;
   a.perm = nullptr;
   a.in_perm = nullptr;
-  a.X = ws + L.xt;
-  a.ldx = mp;
-  a.W = ws + L.gp;
-  a.ldw = h->N;
+  a.X = in_place ? X : (const void *)(ws + L.xt);
+  a.ldx = in_place ? ldx : mp;
+  a.W = in_place ? G : (const void *)(ws + L.gp);
+  a.ldw = in_place ? ldg : h->N;
   a.bias = nullptr;
   a.act = (int)ALG_ACT_NONE;
   a.Y = dW;
   a.ldy = lddw;
   a.y_bf16 = w_dtype == ALG_BF16;
   a.M = h->K;          // rows of this GEMM = input features
-  a.K = mp;            // reduction = padded rows of the batch
+  a.K = in_place ? (int)M : mp;   // reduction = (padded) rows of the batch
   a.N = h->N;
   a.status = p.d_status;
   a.a_cyclic_rows = 0;
@@ -1095,7 +1102,8 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   a.a_box_256 = 0;
   a.gated_f = 0;
   a.w_kmajor = 0;
-  a.dyn_so = hdr->pad_offsets;
+  a.dyn_so = in_place ? nullptr : hdr->pad_offsets;
+  a.seg_rows = in_place ? (int)(M / h->q) : 0;
   a.block_k = block_k_of(p);
   a.y_staged = 0;
   a.plan = nullptr;

@@ -144,6 +144,10 @@ struct ProjArgs {
   // reduction segments come from device memory (padded row buckets; dW = X^T G reduces over rows).
   int w_kmajor;
   const int *dyn_so;
+  // Weight-gradient pass with the cyclic schedule and M a multiple of 64 q: nothing is copied.  The reduction
+  // segment of type t is rows t, t + q, ... of X and of G read in place (type-strided views); the A operand is
+  // the X block as it lies in memory (features contiguous: MN-major A).  seg_rows = M / q; 0 = off.
+  int seg_rows;
   // Gated (SwiGLU) up projection: W is the merged bank [W_gate | W_up] with 2 * gated_f columns, a
   // tile accumulates 128 gate columns and the matching 128 up columns side by side, the epilogue
   // stores silu(gate) * up; N = gated_f is the width of the output.  0 = ordinary projection.

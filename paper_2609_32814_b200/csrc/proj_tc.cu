@@ -158,7 +158,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int e = lane; e < q * q; e += 32) ctl->keep[e] = a.st.valid ? a.st.keep[e] : tab->keep[e];
   } else if (warp == 4) {
     if (a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");   // segment offsets written by the bucketing kernel
-    for (int e = lane; e <= q; e += 32) ctl->so[e] = a.dyn_so ? a.dyn_so[e] : a.st.valid ? a.st.so[e] : tab->so[e];
+    for (int e = lane; e <= q; e += 32)
+      ctl->so[e] = a.seg_rows ? e * a.seg_rows : a.dyn_so ? a.dyn_so[e] : a.st.valid ? a.st.so[e] : tab->so[e];
   } else if (warp == 5) {
     if (a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int e = lane; e < q * q; e += 32) {
@@ -166,7 +167,10 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int n = 0;
       for (int k = 0; k < q; ++k)
         if ((mask >> k) & 1u)
-          n += (a.dyn_so ? a.dyn_so[k + 1] - a.dyn_so[k] : a.st.valid ? a.st.so[k + 1] - a.st.so[k] : tab->so[k + 1] - tab->so[k]) /
+          n += (a.seg_rows ? a.seg_rows
+                : a.dyn_so   ? a.dyn_so[k + 1] - a.dyn_so[k]
+                : a.st.valid ? a.st.so[k + 1] - a.st.so[k]
+                             : tab->so[k + 1] - tab->so[k]) /
                BK;
       ctl->nkb[e] = (uint16_t)n;   // for tile records decoded after the precomputed ones
     }
@@ -197,7 +201,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
       if (a.offsets || a.dyn_so) asm volatile("griddepcontrol.wait;" ::: "memory");  // bucket offsets come from the previous kernel
       tile_plan_warp(tm, recs, kSeqCap, tab, a.st, a.q, a.n_classes, a.offsets, a.cyclic_rows, a.M, a.geom, blockIdx.x,
-                     gridDim.x, BK, a.dyn_so);
+                     gridDim.x, BK, a.dyn_so, a.seg_rows);
     }
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -245,7 +249,20 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t bar = full0 + 8u * (uint32_t)stage;
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
           if (elect_one()) {
-            if (loads_a) {
+            if (a.seg_rows) {
+              // weight gradient, cyclic schedule: rows k, k + q, ... of X (A, features contiguous) and of G (B),
+              // 64 of them from position k0 - so[k] on, in boxes of 64 features / 64 output columns
+              const int pos0 = k0 - k_begin;
+              if (loads_a) {
+                mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+#pragma unroll
+                for (int c = 0; c < TILE_M / 64; ++c) tma_load_3d(sa + c * (64 * BK * 2), &tmA, bar, row0 + c * 64, k, pos0);
+              } else {
+#pragma unroll
+                for (int c = 0; c < TILE_N / 64; ++c)
+                  tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, n0 + c * 64, k, pos0);
+              }
+            } else if (loads_a) {
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
               else tma_load_2d(sa, &tmA, bar, k0, a_row);
@@ -278,12 +295,16 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     const uint32_t tfull0 = smem_u32(&ctl->tmem_full[0]), tempty0 = smem_u32(&ctl->tmem_empty[0]);
-    const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, C::kSboK, C::kSwzK);
+    // A: K-major rows of 128 (64) bytes; in the in-place weight-gradient pass the block lies MN-major like B
+    // (64-feature chunks one box apart, 16 reduction rows = 128 descriptor units per K step)
+    const uint64_t da0 = a.seg_rows ? make_smem_desc(smem_u32(smem), 64 * BK * 2, 1024)
+                                    : make_smem_desc(smem_u32(smem), 16, C::kSboK, C::kSwzK);
+    const uint64_t da_step = a.seg_rows ? 128 : 2;
     // B: the canonical bank lands MN-major (64-column chunks one box apart, 16 k-rows = two 8-row groups
     // = 128 descriptor units per K step); used transposed it lands K-major like A (32 bytes per K step)
     const uint64_t db0 = a.w_kmajor ? make_smem_desc(smem_u32(smem) + C::kABytes, 16, C::kSboK, C::kSwzK)
                                     : make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
-    const uint32_t idesc = a.w_kmajor ? (C::kIdesc & ~(1u << 16)) : C::kIdesc;
+    const uint32_t idesc = (a.w_kmajor ? (C::kIdesc & ~(1u << 16)) : C::kIdesc) | (a.seg_rows ? (1u << 15) : 0u);
     const uint64_t db_step = a.w_kmajor ? 2 : 128;
     TileRec rec = tile_seq_get(recs, tm, a.geom, 0, blockIdx.x, gridDim.x, ctl->nkb);
     while (ok && __shfl_sync(0xffffffffu, rec.row0, 0) >= 0) {
@@ -312,7 +333,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kk = 0; kk < BK / 16; ++kk)
 #pragma unroll
             for (int h = 0; h < C::kHalves; ++h)
-              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)(kk * 2 + h * (C::kAHalfBytes >> 4)), db + (uint64_t)kk * db_step,
+              tc_mma_bf16(d_tmem + (uint32_t)(h * TILE_N), da + (uint64_t)kk * da_step + (uint64_t)(h * (C::kAHalfBytes >> 4)), db + (uint64_t)kk * db_step,
                           idesc, (kb | kk) ? 1u : 0u);
           tc_commit(empty0 + 8u * (uint32_t)stage);
         }
@@ -483,9 +504,23 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   int smem_bytes = C::kFixedSmemBytes + (int)tile_map_bytes(a.n_classes);
   if (smem_bytes > 227 * 1024) return cudaErrorInvalidConfiguration;
   CUtensorMap tmA, tmB;
-  cudaError_t e = make_map_a(&tmA, a);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   ProjArgs b = a;
+  if (a.seg_rows) {
+    // X and G as {columns, type, position in the type}: rows t, t + q, ... are the reduction segment of type t
+    if (GATED || a.w_kmajor || TILE_M != 128 || BK != 64) return cudaErrorInvalidValue;
+    const uint64_t da[3] = {(uint64_t)a.M, (uint64_t)a.q, (uint64_t)a.seg_rows};
+    const uint64_t sa[2] = {(uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.q};
+    const uint64_t db[3] = {(uint64_t)a.N, (uint64_t)a.q, (uint64_t)a.seg_rows};
+    const uint64_t sb[2] = {(uint64_t)a.ldw * 2, (uint64_t)a.ldw * 2 * (uint64_t)a.q};
+    const uint32_t box[3] = {64, 1, 64};
+    e = make_map_nd(&tmA, a.X, 3, da, sa, box, 128);
+    if (e == cudaSuccess) e = make_map_nd(&tmB, a.W, 3, db, sb, box, 128);
+    if (e != cudaSuccess) return e;
+    b.b_3d = 0;
+  } else {
+  e = make_map_a(&tmA, a);
+  if (e != cudaSuccess) return e;
   if (a.w_kmajor) {   // W is N x K here (rows = output columns, contiguous along the reduction): boxes of 64 x TILE_N
     if (GATED) return cudaErrorInvalidValue;
     b.b_3d = 0;
@@ -498,6 +533,7 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   if (!b.b_3d && !a.w_kmajor) {
     e = make_map_2d(&tmB, a.W, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldw * 2, 64, BK);
     if (e != cudaSuccess) return e;
+  }
   }
   // staging buffers for the transposing epilogue, when they fit and the output rows are 16-byte aligned
   b.y_staged = !GATED && a.y_bf16 && smem_bytes + kEpiWarps * C::kStoreBufBytes <= 227 * 1024 && ((uintptr_t)a.Y & 15u) == 0 &&

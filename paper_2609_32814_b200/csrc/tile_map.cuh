@@ -142,11 +142,12 @@ __device__ __forceinline__ TileRec tile_seq_get(const TileRec *recs, TileMap *tm
 // included -- built by ONE warp with warp-level synchronisation only, so that the other warps of
 // the CTA can set up barriers and tensor memory meanwhile and a single CTA barrier ends the
 // prologue.  `keep` / `so` are read from the by-value table when it is valid, else from `tab`.
+// `seg_rows` (optional): every reduction segment has this many rows (weight-gradient pass, cyclic schedule).
 // `dyn_so` (optional, device memory): offsets of the reduction segments when they are not the
 // table's (weight-gradient pass: padded row buckets).
 __device__ inline void tile_plan_warp(TileMap *tm, TileRec *recs, int cap, const DevTable *tab, const SmallTable &st,
                                       int q, int nc, const int *offsets, int cyclic_rows, int M, const TileGeom &g,
-                                      int worker, int n_workers, int k_block, const int *dyn_so = nullptr) {
+                                      int worker, int n_workers, int k_block, const int *dyn_so = nullptr, int seg_rows = 0) {
   const int lane = threadIdx.x & 31;
   if (lane == 0) tm->n_classes = nc, tm->q = q;
   for (int t = lane; t <= q + 1; t += 32) tm->offsets[t] = offsets ? offsets[t] : (t <= q ? t * cyclic_rows : M);
@@ -186,7 +187,7 @@ __device__ inline void tile_plan_warp(TileMap *tm, TileRec *recs, int cap, const
       int n = 0;
       for (int k = 0; k < q; ++k)
         if ((mask >> k) & 1u)
-          n += (dyn_so ? dyn_so[k + 1] - dyn_so[k] : st.valid ? st.so[k + 1] - st.so[k] : tab->so[k + 1] - tab->so[k]) / k_block;
+          n += (seg_rows ? seg_rows : dyn_so ? dyn_so[k + 1] - dyn_so[k] : st.valid ? st.so[k + 1] - st.so[k] : tab->so[k + 1] - tab->so[k]) / k_block;
       rec.rows |= n << 16;
     }
     recs[r] = rec;

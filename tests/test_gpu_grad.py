@@ -26,7 +26,10 @@ def _problem(q, M, s_w, r_w, types=None, integer=True, seed=1):
     (3, 515, 128, 256, "explicit"),     # non-power-of-two q
     (4, 777, 128, 512, "explicit"),     # config-3 group shapes
     (1, 200, 256, 256, "explicit"),     # q = 1: the gradients of an ordinary GEMM
-    (2, 1024, 256, 128, "cyclic"),      # cyclic schedule
+    (2, 1024, 256, 128, "cyclic"),      # cyclic schedule, whole 64-row blocks per type: X and G read in place
+    (4, 4 * 192, 128, 384, "cyclic"),   # in place, three reduction blocks per type, four segments on the diagonal
+    (3, 3 * 64, 384, 128, "cyclic"),    # in place, one block per type, several feature tiles
+    (2, 1000, 128, 256, "cyclic"),      # 500 rows per type: not whole blocks, padded copies
 ])
 def test_grad_maps_integer_bit_exact(q, M, s_w, r_w, schedule):
     types = synth.cyclic_types(M, q) if schedule == "cyclic" else None
