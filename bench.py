@@ -715,7 +715,7 @@ def run_train(args, ctx):
         gbs = bytes_step * args.steps / region_s / 1e9
         roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": peaks["source"], "tensor_time_us": t_tensor * 1e6, "hbm_time_us": t_hbm * 1e6}
-    roofline.update({"kernel": "proj_tc_kernel (forward, dX with W used transposed, dW over padded row buckets)", "traffic": None,
+    roofline.update({"kernel": "proj_tc_kernel (forward, dX with W used transposed, dW over the row buckets: in place with the cyclic schedule, padded copies otherwise)", "traffic": None,
                      "parts": parts})
     extras = {}
     if rank == 0 and not args.no_extras:
