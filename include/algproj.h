@@ -102,7 +102,8 @@ typedef enum {
  *                     1 = one-CTA 128-row tiles (tcgen05 cta_group::1), 2 = CTA pairs
  *                     (cta_group::2), 3 = one-CTA 256-row x 128-column tiles (two accumulators
  *                     per tile, each B block feeds two MMAs).  2 and 3 need every output group
- *                     width to be a multiple of 128.
+ *                     width to be a multiple of 128.  4 = the large-algebra kernel (see
+ *                     alg_proj_create) for a projection handle whose law, dtype and widths fit it.
  *   TILE_N            tile width of the one-CTA kernel: 0 = automatic, or 128 / 192 / 256 when
  *                     that divides every output group width.
  *   STAGE_K           reduction depth of one pipeline stage of the one-CTA GEMM kernel: 0 =

@@ -29,6 +29,7 @@ constexpr int kPlanSlots = 4;
 // Large-algebra path (proj_big.cu): complete-graph law, equal group widths, q up to kBigMaxQ.
 struct BigPlan {
   bool on = false;
+  bool eligible = false;  // the handle's law, dtype and widths fit the large-algebra kernel (GEMM_KERNEL = 4 may select it)
   int s = 0, r = 0;       // width of every input / output group
   int s_pad = 0, r_pad = 0;   // the same rounded up to multiples of 8: what the tensor maps can address
   bool repack = false;    // widths that are multiples of 4 only: X and W are repacked with padded groups on every call
@@ -295,7 +296,11 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     }
   alg_status_t cs = configure_kernels(p);
   if (cs != ALG_OK) return cs;
-  if (big_fits && !p.tc_ok) plan_big(p, in_w[0], out_w[0]);   // widths the table-driven tensor path does not take
+  if (big_fits) {
+    plan_big(p, in_w[0], out_w[0]);
+    p.big.eligible = true;
+    p.big.on = !p.tc_ok;   // by default only for widths the table-driven tensor path does not take
+  }
 
   if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
   cudaDeviceProp prop;
@@ -481,10 +486,51 @@ const PlanSlot *prepare_cyclic_plan(alg_proj_s &p, const TcChoice &tc, int64_t M
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
+// Counted buckets (explicit types, or cyclic with q not dividing M) on the large-algebra kernel: always when the
+// handle has no other tensor-core kernel or asks for it; by the library's choice when the buckets are small
+// (at most two 128-row tiles per type on average) -- there the table-driven kernel spends its time on tile
+// records and half-empty tiles (4096 -> 12288 at q = 32, M = 2048: 95.7 -> 70.1 us; FFN 187.6 -> 139.0 us),
+// while with large buckets its tuned main loop and epilogue win (q = 8, M = 16384 FFN: 125.9 against 138.3 us).
+bool use_big_counted(const alg_proj_s &p, int64_t M) {
+  if (p.gated || p.big.repack) return false;
+  return p.big.on || (p.big.eligible && p.opt_kernel == 0 && M <= 256 * (int64_t)p.q);
+}
+
+
 alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
                       cudaEvent_t after_gather = nullptr, bool cyclic = false) {
+  if (!cyclic && use_big_counted(p, M)) {
+    // large-algebra kernel on counted buckets: X bucketed already or gathered here, rows of Y scattered back
+    // through the permutation unless the caller keeps the bucketed order
+    BigArgs g;
+    g.X = X, g.ldx = ldx;
+    if (!x_bucketed) {
+      if (launch_gather_rows(X, ldx, (const int *)(ws + L.perm), (int)M, p.K, 2, ws + L.xb, st) != cudaSuccess) return ALG_ERR_CUDA;
+      g.X = ws + L.xb, g.ldx = p.K;
+    }
+    if (after_gather) cudaEventRecord(after_gather, st);
+    g.W = W, g.ldw = ldw;
+    g.bias = bias;
+    g.act = (int)act;
+    g.Y = Y, g.ldy = ldy;
+    g.y_bf16 = y_dtype == ALG_BF16;
+    g.M = (int)M, g.q = p.q;
+    g.s = p.big.s, g.r = p.big.r, g.r_out = p.big.r;
+    g.tile_n = p.big.tile_n, g.nt_n = p.big.nt_n;
+    g.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;
+    g.n_chunks = (g.tile_n + 63) / 64;
+    g.a_box_rows = 128;
+    g.pack = 1;
+    g.sched = 0;
+    g.offsets = (const int *)(ws + L.hdr);
+    g.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
+    g.rows_per_type = 0;
+    g.status = p.d_status;
+    g.wait_limit = p.wait_limit;
+    return cuda_status(launch_proj_big(g, p.num_sms, st));
+  }
   ProjArgs a;
   const TcChoice tc = choose_tiling(p, M);
   const DevTable &tab = *tc.tab;
@@ -702,8 +748,14 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
   switch (option) {
     case ALG_OPT_GEMM_KERNEL:
     case ALG_OPT_TILE_N: {
-      if (no_table) return value == 0 ? ALG_OK : ALG_ERR_UNSUPPORTED_SHAPE;
-      if (option == ALG_OPT_GEMM_KERNEL && (value < 0 || value > 3)) return ALG_ERR_INVALID_ARG;
+      if (no_table) return value == 0 || (option == ALG_OPT_GEMM_KERNEL && value == 4) ? ALG_OK : ALG_ERR_UNSUPPORTED_SHAPE;
+      if (option == ALG_OPT_GEMM_KERNEL && (value < 0 || value > 4)) return ALG_ERR_INVALID_ARG;
+      if (option == ALG_OPT_GEMM_KERNEL && value == 4) {   // the large-algebra kernel, for handles that fit it
+        if (!p.big.eligible) return ALG_ERR_UNSUPPORTED_SHAPE;
+        p.big.on = true;
+        return ALG_OK;
+      }
+      if (option == ALG_OPT_GEMM_KERNEL && p.big.eligible) p.big.on = !p.tc_ok;
       if (option == ALG_OPT_TILE_N && value != 0 && value != 128 && value != 192 && value != 256) return ALG_ERR_INVALID_ARG;
       const int old_kernel = p.opt_kernel, old_tile = p.opt_tile_n;
       (option == ALG_OPT_GEMM_KERNEL ? p.opt_kernel : p.opt_tile_n) = (int)value;
@@ -780,7 +832,8 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
   if (use_decode(*h, M)) return run_decode(*h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
-  if (h->big.on) return run_big(*h, L, ws, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
+  if (h->big.on || (h->sched == ALG_SCHED_EXPLICIT && use_big_counted(*h, M)))
+    return run_big(*h, L, ws, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
 
   BucketArgs b;
   b.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
@@ -1126,8 +1179,13 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
   alg_ffn_s *f = new (std::nothrow) alg_ffn_s();
   if (!f) return ALG_ERR_INVALID_ARG;
   f->gated = gated;
-  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated);
-  if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status);
+  if (q > kMaxQ || schedule == ALG_SCHED_INTERVAL) {   // large-algebra handles are single projections
+    delete f;
+    return q > kBigMaxQ || q < 1 ? ALG_ERR_INVALID_ARG : ALG_ERR_UNSUPPORTED_SHAPE;
+  }
+  // (allow_big: with explicit types an FFN whose law and widths fit may run its projections on the large-algebra kernel)
+  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated, !gated);
+  if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status, false, !gated);
   if (s != ALG_OK) {
     free_proj(f->down);
     free_proj(f->up);

@@ -50,7 +50,8 @@ def test_ffn_f32_simt_small():
     assert H.rel_fro(got, ref) <= 1e-5 and H.max_abs(got, ref) <= 1e-4
 
 
-def test_ffn_integer_identity_activation_bit_exact():
+@pytest.mark.parametrize("kernel", [0, 1, 4])   # the library's choice, the table-driven kernel, the large-algebra kernel
+def test_ffn_integer_identity_activation_bit_exact(kernel):
     """With act = none both projections are exact integer arithmetic through the tensor cores
     (|H| <= 9*256 stays exactly representable in bf16 only if small: use entries in {-1,0,1})."""
     wl = synth.make_workload("ffnint", config=7, variant=2, dtype="bf16", q=2, M=600, D=128, F=256,
@@ -59,6 +60,7 @@ def test_ffn_integer_identity_activation_bit_exact():
     wl.W_up = np.sign(wl.W_up).astype(np.float32) * (np.abs(wl.W_up) > 2)
     wl.W_down = np.sign(wl.W_down).astype(np.float32)
     ffn = _ffn(wl)
+    ffn.set_option("gemm_kernel", kernel)
     Y = _run_ffn(wl, ffn, torch.float32, act=None)
     Hh = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
     assert np.abs(Hh).max() <= 256  # exactly representable in bf16

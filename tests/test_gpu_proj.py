@@ -11,10 +11,12 @@ pytestmark = pytest.mark.gpu
 
 
 def _run_proj(wl, *, table="qq", custom=None, bias=None, act=None, out_dtype=None, which="up", schedule="explicit",
-              expect_path=None):
+              expect_path=None, kernel=None):
     s, r = (wl.d_widths, wl.f_widths) if which == "up" else (wl.f_widths, wl.d_widths)
     W = wl.W_up if which == "up" else wl.W_down
     proj = binding.Proj(s, r, dtype=wl.dtype, table=table, custom_keep=custom, schedule=schedule)
+    if kernel is not None:
+        proj.set_option("gemm_kernel", kernel)
     if expect_path is not None:
         assert proj.kernel_path(wl.M) == expect_path
     X = H.to_dev(wl.X, wl.dtype)
@@ -89,9 +91,10 @@ def _tc_workload(q, M, s_w, r_w, types=None, integer=True, seed=1):
     (1, 520, 1024, 128),
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
-def test_tc_integer_bit_exact(q, M, s_w, r_w, out_dtype):
+@pytest.mark.parametrize("kernel", [0, 1, 4])   # the library's choice, the table-driven kernel, the large-algebra kernel
+def test_tc_integer_bit_exact(q, M, s_w, r_w, out_dtype, kernel):
     wl = _tc_workload(q, M, s_w, r_w, seed=q * 10 + M % 7)
-    Y, proj = _run_proj(wl, out_dtype=out_dtype, expect_path=binding.ALG_PATH_TCGEN05)
+    Y, proj = _run_proj(wl, out_dtype=out_dtype, expect_path=binding.ALG_PATH_TCGEN05, kernel=kernel)
     assert proj.gemm_count() == 2 * q * q - q
     ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
     if out_dtype == torch.bfloat16:
@@ -291,11 +294,12 @@ def test_tc_dense_and_custom_tables():
     assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, keep=keep))
 
 
-def test_tc_bias_and_gelu_normal_data():
+@pytest.mark.parametrize("kernel", [1, 4])   # the table-driven kernel, the large-algebra kernel
+def test_tc_bias_and_gelu_normal_data(kernel):
     wl = _tc_workload(2, 700, 384, 256, integer=False, seed=3)
     bias = synth.bf16_round(synth.normal(5, (wl.F,), 0.5))
     for act, out_dtype in (("gelu", torch.float32), ("gelu", torch.bfloat16), (None, torch.float32)):
-        Y, _ = _run_proj(wl, bias=bias, act=act, out_dtype=out_dtype)
+        Y, _ = _run_proj(wl, bias=bias, act=act, out_dtype=out_dtype, kernel=kernel)
         ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths, bias=bias)
         if act:
             ref = np.vectorize(oracle.gelu)(ref)
