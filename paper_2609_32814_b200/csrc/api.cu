@@ -495,12 +495,45 @@ bool use_big_counted(const alg_proj_s &p, int64_t M) {
   if (p.gated || p.big.repack) return false;
   return p.big.on || (p.big.eligible && p.opt_kernel == 0 && M <= 256 * (int64_t)p.q);
 }
+// Equal buckets (cyclic schedule, q | M): by the library's choice when a type has at most 128 rows -- the
+// large-algebra kernel then packs several types into a tile (FFN 4096 -> 12288 -> 4096 at q = 32, M = 2048:
+// 128.6 -> 71.1 us); with fuller buckets the table-driven kernel is faster (58.6 against 63.2 us on the q = 2
+// FFN at M = 8192).
+bool use_big_equal(const alg_proj_s &p, int64_t M) {
+  if (p.gated || p.big.repack) return false;
+  return p.big.on || (p.big.eligible && p.opt_kernel == 0 && M <= 128 * (int64_t)p.q);
+}
 
 
 alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
                       cudaEvent_t after_gather = nullptr, bool cyclic = false) {
+  if (cyclic && use_big_equal(p, M)) {
+    // equal buckets on the large-algebra kernel: the caller's rows are read / written in place (type-strided),
+    // a bucketed operand or result is the interval layout
+    BigArgs g;
+    g.X = X, g.ldx = ldx;
+    g.W = W, g.ldw = ldw;
+    g.bias = bias;
+    g.act = (int)act;
+    g.Y = Y, g.ldy = ldy;
+    g.y_bf16 = y_dtype == ALG_BF16;
+    g.M = (int)M, g.q = p.q;
+    g.s = p.big.s, g.r = p.big.r, g.r_out = p.big.r;
+    g.tile_n = p.big.tile_n, g.nt_n = p.big.nt_n;
+    g.block_k = p.opt_stage_k == 32 ? 32 : p.big.block_k;
+    g.n_chunks = (g.tile_n + 63) / 64;
+    g.rows_per_type = (int)(M / p.q);
+    g.a_box_rows = (int)std::min<int64_t>(128, (g.rows_per_type + 7) / 8 * 8);
+    g.pack = 1;
+    g.sched = x_bucketed ? 1 : 2, g.sched_out = y_bucketed ? 1 : 2;
+    g.offsets = nullptr, g.perm = nullptr;
+    g.status = p.d_status;
+    g.wait_limit = p.wait_limit;
+    if (after_gather) cudaEventRecord(after_gather, st);
+    return cuda_status(launch_proj_big(g, p.num_sms, st));
+  }
   if (!cyclic && use_big_counted(p, M)) {
     // large-algebra kernel on counted buckets: X bucketed already or gathered here, rows of Y scattered back
     // through the permutation unless the caller keeps the bucketed order
@@ -523,7 +556,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     g.n_chunks = (g.tile_n + 63) / 64;
     g.a_box_rows = 128;
     g.pack = 1;
-    g.sched = 0;
+    g.sched = 0, g.sched_out = 0;
     g.offsets = (const int *)(ws + L.hdr);
     g.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
     g.rows_per_type = 0;
@@ -678,6 +711,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
     a.W = ws + L.wp, a.ldw = (int64_t)p.q * p.big.r_pad;
     a.s = p.big.s_pad, a.r = p.big.r_pad;
   }
+  a.sched_out = a.sched;
   return cuda_status(launch_proj_big(a, p.num_sms, st));
 }
 
@@ -832,7 +866,8 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
   if (use_decode(*h, M)) return run_decode(*h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
-  if (h->big.on || (h->sched == ALG_SCHED_EXPLICIT && use_big_counted(*h, M)))
+  if (h->big.on || (h->sched == ALG_SCHED_EXPLICIT && use_big_counted(*h, M)) ||
+      (h->sched == ALG_SCHED_CYCLIC && M % h->q == 0 && use_big_equal(*h, M)))
     return run_big(*h, L, ws, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
 
   BucketArgs b;
@@ -1307,7 +1342,8 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   b.y_elem_bytes = elem_bytes(y_dtype);
   const bool tm = h->timing;
   if (tm) cudaEventRecord(h->ev[0], st);
-  const bool cyc = h->up.sched == ALG_SCHED_CYCLIC && use_tc(h->up) && use_tc(h->down) && M % h->up.q == 0;
+  const bool cyc = h->up.sched == ALG_SCHED_CYCLIC && M % h->up.q == 0 &&
+                   ((use_tc(h->up) && use_tc(h->down)) || (use_big_equal(h->up, M) && use_big_equal(h->down, M)));
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;

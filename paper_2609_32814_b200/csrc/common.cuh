@@ -189,6 +189,8 @@ struct BigArgs {
   int a_box_rows;         // rows of X fetched per stage: 128, or fewer when no type has that many rows
   int pack;               // set by the launcher: row types per tile (> 1 when a type has at most 64 rows; sched 1, 2)
   int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
+  int sched_out;          // how the rows of Y are addressed (same codes); differs from sched inside an FFN, whose
+                          // hidden state stays in bucketed (= interval) order between its two projections
   const int *offsets;     // sched 0: device bucket offsets [q + 1]
   const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)
   int rows_per_type;      // sched 1, 2: M / q

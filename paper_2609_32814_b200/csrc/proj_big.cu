@@ -366,11 +366,11 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int r = quad * 32 + lane;
       int64_t out_row = -1;
       if (r < tl.rows) {
-        if (a.sched == 2 && a.pack > 1) {   // rows of a packed tile are type-major: type tl.i + r / rows_per_type
+        if (a.sched_out == 2 && a.pack > 1) {   // rows of a packed tile are type-major: type tl.i + r / rows_per_type
           const int ti = r / a.rows_per_type;
           out_row = (int64_t)(r - ti * a.rows_per_type) * q + tl.i + ti;
-        } else if (a.sched == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
-        else if (a.sched == 0 && a.perm) out_row = __ldg(a.perm + tl.row0 + r);
+        } else if (a.sched_out == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
+        else if (a.sched_out == 0 && a.perm) out_row = __ldg(a.perm + tl.row0 + r);
         else out_row = tl.row0 + r;
         if (out_row >= a.M) out_row = -1;
       }
@@ -581,6 +581,7 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
 cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
   cudaError_t e = tc_init();
   if (e != cudaSuccess) return e;
+  if ((a.sched == 0) != (a.sched_out == 0)) return cudaErrorInvalidValue;   // counted buckets on both sides or on neither
   if (a.q < 1 || a.q > kBigMaxQ || a.s % 8 || a.r % 8 || a.tile_n % 16 || a.tile_n < 16 || a.tile_n > 256) return cudaErrorInvalidValue;
   if (a.r_out % 4 || a.r_out < 4 || a.r_out > a.r) return cudaErrorInvalidValue;
   if (a.nt_n != (a.r_out + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
