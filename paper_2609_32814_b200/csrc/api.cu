@@ -211,7 +211,8 @@ void plan_big(alg_proj_s &p, int s, int r) {
   p.big.s = s, p.big.r = r;
   p.big.s_pad = (s + 7) / 8 * 8, p.big.r_pad = (r + 7) / 8 * 8;
   p.big.repack = s % 8 != 0 || r % 8 != 0;
-  p.big.nt_n = (r + 255) / 256;
+  const int widest = p.gated ? 128 : 256;   // a gated tile holds its gate columns and as many up columns
+  p.big.nt_n = (r + widest - 1) / widest;
   p.big.tile_n = ((r + p.big.nt_n - 1) / p.big.nt_n + 15) / 16 * 16;
   p.big.nt_n = (r + p.big.tile_n - 1) / p.big.tile_n;
   // 64-deep stages whatever the group width: the copy engine is bound by row requests, and a 128-byte row of
@@ -492,7 +493,7 @@ bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 // records and half-empty tiles (4096 -> 12288 at q = 32, M = 2048: 95.7 -> 70.1 us; FFN 187.6 -> 139.0 us),
 // while with large buckets its tuned main loop and epilogue win (q = 8, M = 16384 FFN: 125.9 against 138.3 us).
 bool use_big_counted(const alg_proj_s &p, int64_t M) {
-  if (p.gated || p.big.repack) return false;
+  if (p.big.repack) return false;
   return p.big.on || (p.big.eligible && p.opt_kernel == 0 && M <= 256 * (int64_t)p.q);
 }
 // Equal buckets (cyclic schedule, q | M): by the library's choice when a type has at most 128 rows -- the
@@ -527,6 +528,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     g.rows_per_type = (int)(M / p.q);
     g.a_box_rows = (int)std::min<int64_t>(128, (g.rows_per_type + 7) / 8 * 8);
     g.pack = 1;
+    g.gated_f = 0;
     g.sched = x_bucketed ? 1 : 2, g.sched_out = y_bucketed ? 1 : 2;
     g.offsets = nullptr, g.perm = nullptr;
     g.status = p.d_status;
@@ -556,6 +558,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     g.n_chunks = (g.tile_n + 63) / 64;
     g.a_box_rows = 128;
     g.pack = 1;
+    g.gated_f = p.gated ? p.N : 0;
     g.sched = 0, g.sched_out = 0;
     g.offsets = (const int *)(ws + L.hdr);
     g.perm = y_bucketed ? nullptr : (const int *)(ws + L.perm);
@@ -663,6 +666,7 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
   a.n_chunks = (a.tile_n + 63) / 64;
   a.a_box_rows = 128;
   a.pack = 1;
+  a.gated_f = 0;
   a.offsets = nullptr, a.perm = nullptr;
   a.rows_per_type = 0;
   a.status = p.d_status;
@@ -1219,8 +1223,8 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
     return q > kBigMaxQ || q < 1 ? ALG_ERR_INVALID_ARG : ALG_ERR_UNSUPPORTED_SHAPE;
   }
   // (allow_big: with explicit types an FFN whose law and widths fit may run its projections on the large-algebra kernel)
-  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated, !gated);
-  if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status, false, !gated);
+  alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated, true);
+  if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status, false, true);
   if (s != ALG_OK) {
     free_proj(f->down);
     free_proj(f->up);

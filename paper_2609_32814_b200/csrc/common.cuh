@@ -187,6 +187,9 @@ struct BigArgs {
   int block_k;            // 64 or 32: reduction depth of a pipeline stage
   int n_chunks;           // 64-column boxes of W fetched per stage = ceil(tile_n / 64)
   int a_box_rows;         // rows of X fetched per stage: 128, or fewer when no type has that many rows
+  int gated_f;            // > 0: SwiGLU up projection over the merged bank [W_gate | W_up] (2 * gated_f columns): a tile
+                          // accumulates its gate columns and, n_chunks * 64 accumulator columns further, the matching
+                          // up columns; the epilogue stores silu(gate) * up (bf16).  tile_n <= 128.
   int pack;               // set by the launcher: row types per tile (> 1 when a type has at most 64 rows; sched 1, 2)
   int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
   int sched_out;          // how the rows of Y are addressed (same codes); differs from sched inside an FFN, whose

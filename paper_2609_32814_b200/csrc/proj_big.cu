@@ -252,7 +252,8 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     bool ok = true;
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     const uint32_t smem0 = smem_u32(smem);
-    const uint32_t stage_tx = (uint32_t)(a.a_box_rows * BK * 2 + a.n_chunks * C::kBChunkBytes);   // bytes the copies of a stage deliver
+    const int b_chunks = a.gated_f ? 2 * a.n_chunks : a.n_chunks;   // 64-column boxes of the bank per stage
+    const uint32_t stage_tx = (uint32_t)(a.a_box_rows * BK * 2 + b_chunks * C::kBChunkBytes);   // bytes the copies of a stage deliver
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
@@ -278,10 +279,10 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (elect_one()) {
             if (loads_a && packed) {
               if (sg == 0) {   // all rows of the tile: np types x rows_per_type rows, type-major
-                mbar_expect_tx(bar, (uint32_t)(a.pack * a.rows_per_type * BK * 2 + a.n_chunks * C::kBChunkBytes));
+                mbar_expect_tx(bar, (uint32_t)(a.pack * a.rows_per_type * BK * 2 + b_chunks * C::kBChunkBytes));
                 tma_load_4d(sa, &tmA, bar, kb * BK, k, 0, tl.i);
               } else {         // the rows of type k where they sit in the tile, zeros everywhere else
-                mbar_expect_tx(bar, (uint32_t)(128 * BK * 2 + a.n_chunks * C::kBChunkBytes));
+                mbar_expect_tx(bar, (uint32_t)(128 * BK * 2 + b_chunks * C::kBChunkBytes));
                 tma_load_4d(sa, &tmA2, bar, kb * BK, k, -(k - tl.i) * a.rows_per_type, k);
               }
             } else if (loads_a) {
@@ -291,6 +292,8 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             } else {
               for (int c = 0; c < a.n_chunks; ++c)
                 tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0_w + c * 64, kb * BK, k);
+              for (int c = 0; c < (a.gated_f ? a.n_chunks : 0); ++c)   // the matching up columns, behind the gate chunks
+                tma_load_3d(sa + C::kABytes + (a.n_chunks + c) * C::kBChunkBytes, &tmB, bar, a.gated_f + tl.n0_w + c * 64, kb * BK, k);
             }
           }
           __syncwarp();
@@ -308,7 +311,8 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint64_t da0 = make_smem_desc(smem_u32(smem), 16, C::kSboK, C::kSwzK);
     const uint64_t db0 = make_smem_desc(smem_u32(smem) + C::kABytes, C::kBChunkBytes, 1024);
     // instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, N = tile_n, M = 128
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(a.tile_n >> 3) << 17) |
+    const int mma_n = a.gated_f ? 2 * a.n_chunks * 64 : a.tile_n;   // gated: gate chunks and up chunks side by side
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(mma_n >> 3) << 17) |
                            ((uint32_t)(128 >> 4) << 24);
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
@@ -384,7 +388,60 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       // Tiles of this path have short reductions, so the epilogue is the longest chain of a tile: warps
       // whose 32 rows lie past the tile's last row do nothing.
       const int c_end = quad * 32 < tl.rows ? tl.cols : 0;
-      if (a.y_bf16) {
+      if (a.gated_f) {
+        // gate values sit in accumulator columns [0, cols), the matching up values n_chunks * 64 columns further;
+        // silu(g) * u with sigmoid(g) = (1 + tanh(g / 2)) / 2, then the 32 x 32 chunk goes through the warp's
+        // buffer as 64-byte rows (four lanes store one row segment, 8 rows per store instruction)
+        const uint32_t buf0 = smem_u32(store_buf + e * kStoreBufBytes);
+        const uint32_t my_row = buf0 + (uint32_t)lane * 64u;
+        const uint32_t sw = (uint32_t)((lane >> 1) & 3);
+        const int sub = lane >> 2, piece = lane & 3;
+        const uint32_t rd_base = buf0 + (uint32_t)sub * 64u;
+        const uint32_t up_off = (uint32_t)(a.n_chunks * 64);
+        int64_t dst_row[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 8 + sub);
+#pragma unroll 1
+        for (int c0 = half * 32; c0 < c_end; c0 += 64) {
+          uint32_t vg[32], vu[32];
+          tc_ld_32x32(taddr + (uint32_t)c0, vg);
+          tc_ld_32x32(taddr + up_off + (uint32_t)c0, vu);
+          tc_wait_ld();
+          const int col = tl.n0 + c0;
+          uint32_t w[16];
+#pragma unroll
+          for (int x = 0; x < 16; ++x) {
+            float o[2];
+#pragma unroll
+            for (int y = 0; y < 2; ++y) {
+              const float g = __uint_as_float(vg[2 * x + y]);
+              float th;
+              asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * g));
+              o[y] = g * fmaf(0.5f, th, 0.5f) * __uint_as_float(vu[2 * x + y]);
+            }
+            __nv_bfloat162 pk = __floats2bfloat162_rn(o[0], o[1]);
+            w[x] = *(uint32_t *)&pk;
+          }
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((((uint32_t)g) ^ sw) << 4)), "r"(w[g * 4]),
+                         "r"(w[g * 4 + 1]), "r"(w[g * 4 + 2]), "r"(w[g * 4 + 3])
+                         : "memory");
+          __syncwarp();
+          const bool piece_ok = col + piece * 8 < col_end;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int rr = g * 8 + sub;
+            const uint32_t rsw = (uint32_t)((rr >> 1) & 3);
+            uint4 val;
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                         : "r"(rd_base + (uint32_t)g * 512u + ((((uint32_t)piece) ^ rsw) << 4)));
+            if (dst_row[g] >= 0 && piece_ok) *(uint4 *)((__nv_bfloat16 *)a.Y + dst_row[g] * a.ldy + col + piece * 8) = val;
+          }
+        }
+      } else if (a.y_bf16) {
         int64_t dst_row[8];   // rows this lane stores for: phase * 16 + g * 4 + rd_r
 #pragma unroll
         for (int g = 0; g < 8; ++g) dst_row[g] = __shfl_sync(0xffffffffu, out_row, g * 4 + rd_r);
@@ -550,7 +607,7 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   if (b.pack <= 1) tmA2 = tmA;
   {
     // the bank as {columns, k in group, group}: rows past the group's width read as zero
-    const uint64_t dims[3] = {(uint64_t)a.q * (uint64_t)a.r, (uint64_t)a.s, (uint64_t)a.q};
+    const uint64_t dims[3] = {(uint64_t)a.q * (uint64_t)a.r * (a.gated_f ? 2 : 1), (uint64_t)a.s, (uint64_t)a.q};
     const uint64_t str[2] = {(uint64_t)a.ldw * 2, (uint64_t)a.ldw * 2 * (uint64_t)a.s};
     const uint32_t box[3] = {64, (uint32_t)BK, 1};
     e = make_map_nd(&tmB, a.W, 3, dims, str, box, 128);
@@ -586,6 +643,10 @@ cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
   if (a.r_out % 4 || a.r_out < 4 || a.r_out > a.r) return cudaErrorInvalidValue;
   if (a.nt_n != (a.r_out + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
   if (a.a_box_rows < 8 || a.a_box_rows > 128 || a.a_box_rows % 8) return cudaErrorInvalidValue;
+  if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
+    if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;
+    return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);
+  }
   if (a.tile_n <= 128) return a.block_k == 64 ? launch_t<128, 64>(a, num_sms, st) : launch_t<128, 32>(a, num_sms, st);
   return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);
 }

@@ -11,8 +11,10 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _run(wl, Wg, table="qq", schedule="explicit", out_dtype=torch.float32):
+def _run(wl, Wg, table="qq", schedule="explicit", out_dtype=torch.float32, kernel=None):
     ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16", table=table, schedule=schedule)
+    if kernel is not None:
+        ffn.set_option("gemm_kernel", kernel)
     Wgu = np.concatenate([Wg, wl.W_up], axis=1)          # the merged bank: [W_gate | W_up]
     Y = ffn.forward(H.to_dev(wl.X, "bf16"), None if schedule == "cyclic" else H.dev_types(wl.types),
                     H.to_dev(Wgu, "bf16"), H.to_dev(wl.W_down, "bf16"), out_dtype=out_dtype)
@@ -38,12 +40,13 @@ def _sample_rows(wl, per_type, seed=0):
     (1, 300, 128, 384, "explicit"),      # q = 1: an ordinary gated MLP
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
-def test_gated_ffn_small_shapes(q, M, D, F, schedule, out_dtype):
+@pytest.mark.parametrize("kernel", [1, 4])   # the table-driven kernel, the large-algebra kernel
+def test_gated_ffn_small_shapes(q, M, D, F, schedule, out_dtype, kernel):
     types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(600 + q, M, q)
     wl, Wg = synth.gated_ffn("gated", q, M, D, F, types, variant=q * 10 + M % 7)
     # weights of the test are scaled up so that the hidden state is of order one
     wl.W_up, Wg, wl.W_down = (synth.bf16_round(w * 4.0) for w in (wl.W_up, Wg, wl.W_down))
-    Y, ffn = _run(wl, Wg, schedule=schedule, out_dtype=out_dtype)
+    Y, ffn = _run(wl, Wg, schedule=schedule, out_dtype=out_dtype, kernel=kernel)
     ref = oracle.ffn_swiglu(wl.X, wl.types, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
     H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"gated q={q} M={M}")
     counts = np.bincount(wl.types, minlength=q).tolist()
