@@ -288,3 +288,39 @@ def test_pilot_tensor_square_law_and_interval_schedule():
     Yd = _run_ffn(d, ffn, torch.float32)
     refd = oracle.ffn(d.X, d.types, d.W_up, d.W_down, d.d_widths, d.f_widths, keep=keep)
     H.assert_bf16_close(H.to_np(Yd), refd, False, "pilot decode")
+
+
+def _random_ffn_case(k):
+    rng = np.random.default_rng(500 + k)
+    q = int(rng.choice([1, 2, 3, 4, 8, 16, 32]))
+    dw = int(rng.choice([8, 64, 128])) * int(rng.integers(1, 4))
+    fw = int(rng.choice([8, 64, 128])) * int(rng.integers(1, 4))
+    schedule = str(rng.choice(["cyclic", "explicit"]))
+    M = int(rng.integers(1, 40)) * q if rng.random() < 0.5 else int(rng.integers(1, 3000))
+    return q, M, dw, fw, schedule, int(rng.choice([0, 1, 4]))
+
+
+@pytest.mark.parametrize("k", range(24))
+def test_ffn_random_shapes_integer_bit_exact(k):
+    """Seeded random group counts, widths on and off the tile grid, row counts, schedules and kernel choices; with
+    act = none and entries in {-1, 0, 1} both projections are exact integer arithmetic."""
+    q, M, dw, fw, schedule, kernel = _random_ffn_case(k)
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(31 + k, M, q)
+    wl = synth.make_workload("ffnfz", config=7, variant=700 + k, dtype="bf16", q=q, M=M, D=dw * q, F=fw * q, types=types,
+                             integer=True)
+    wl.X = np.sign(wl.X).astype(np.float32)
+    wl.W_up = (np.sign(wl.W_up) * (np.abs(wl.W_up) > 2)).astype(np.float32)
+    wl.W_down = np.sign(wl.W_down).astype(np.float32)
+    Hh = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if np.abs(Hh).max() > 256:
+        pytest.skip("hidden state not exactly representable in bf16")
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    try:
+        ffn.set_option("gemm_kernel", kernel)
+    except binding.AlgError:
+        pass   # the handle's widths do not fit that kernel: the library's choice runs
+    t = None if schedule == "cyclic" else H.dev_types(wl.types)
+    Y = ffn.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"), act=None,
+                    out_dtype=torch.float32)
+    assert ffn.last_status() == 0
+    assert np.array_equal(H.to_np(Y), oracle.proj(Hh, wl.types, wl.W_down, wl.f_widths, wl.d_widths)), (q, M, dw, fw, schedule, kernel)
