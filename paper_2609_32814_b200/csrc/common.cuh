@@ -190,6 +190,9 @@ struct BigArgs {
   int gated_f;            // > 0: SwiGLU up projection over the merged bank [W_gate | W_up] (2 * gated_f columns): a tile
                           // accumulates its gate columns and, n_chunks * 64 accumulator columns further, the matching
                           // up columns; the epilogue stores silu(gate) * up (bf16).  tile_n <= 128.
+  int gpack;              // set by the launcher: output groups per tile (> 1 for narrow groups: one panel product over
+                          // all of the tile's columns, then one diagonal product per group); needs pack == 1
+  int col_units;          // set by the launcher: tiles per (row type, m-tile) = q * nt_n, or ceil(q / gpack)
   int pack;               // set by the launcher: row types per tile (> 1 when a type has at most 64 rows; sched 1, 2)
   int sched;              // 0: buckets from `offsets` (+ `perm` for the output rows), 1: interval, 2: cyclic
   int sched_out;          // how the rows of Y are addressed (same codes); differs from sched inside an FFN, whose

@@ -35,6 +35,12 @@
 //    view {s, group, row in type, type} with a 128-row box placed so that type i's rows land where they sit in
 //    the tile and every other row is out of range, i.e. zero: the product adds nothing to the other types'
 //    rows.  1 + P segments and one epilogue instead of 2 P segments and P epilogues.
+//  * Output groups of at most 128 columns (25600 -> 5120 in 64 ... 256 groups) make narrow tiles that cost their
+//    hand-overs and their A fetches like wide ones.  A tile then covers G = floor(256 / r) consecutive groups: the
+//    panel product x_i W[S_i, all its columns] is ONE segment, and each group g adds its diagonal product
+//    x_j W_jj as a full-width product whose B block is zero outside the group's columns -- fetched through a view of
+//    the bank by {column in group, column group, k, row group} with the box started at a negative column, so the
+//    out-of-range columns are the zeros.  1 + G segments for G groups instead of 2 G, and G times fewer tiles.
 //  * What bounds operand fill on one SM is the number of row requests the copy engine makes (about one
 //    row of up to 128 bytes every two cycles), not their bytes.  So a stage is always fetched in rows of
 //    128 bytes (64-deep stages, even for groups narrower than 64: the rest of the row is zero fill), only
@@ -113,8 +119,8 @@ struct Cfg {
 
 struct Tile {
   int row0, rows;   // bucketed rows [row0, row0 + rows), all of type i; row0 < 0: no more tiles
-  int i, j;         // packed tiles: i = first of np consecutive types
-  int np;
+  int i, j;         // packed tiles: i = first of np consecutive types; j = first of ng consecutive output groups
+  int np, ng;
   int n0, cols;     // absolute first column in Y, valid columns (<= tile_n)
   int n0_w;         // first column in the bank (differs from n0 when the bank's groups are padded)
 };
@@ -123,7 +129,7 @@ struct Tile {
 // the column tile, then the output group.
 __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, int t) {
   Tile o;
-  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0, o.np = 1;
+  o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0, o.np = 1, o.ng = 1;
   if (t >= ctl->total) return o;
   if (a.pack > 1) {   // type-group major, then the output group, then the column tile
     const int per_group = a.q * a.nt_n;
@@ -141,7 +147,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   int i, rem, base, rows_i;
   if (a.sched != 0) {
     rows_i = a.rows_per_type;
-    const int per_type = ((rows_i + 127) >> 7) * a.q * a.nt_n;
+    const int per_type = ((rows_i + 127) >> 7) * a.col_units;
     i = t / per_type;
     rem = t - i * per_type;
     base = i * rows_i;
@@ -158,9 +164,17 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   }
   const int mt_i = (rows_i + 127) >> 7;
   const int u = rem / mt_i, mt = rem - u * mt_i;
-  const int j = u / a.nt_n, nt = u - j * a.nt_n;
   o.row0 = base + (mt << 7);
   o.rows = min(128, rows_i - (mt << 7));
+  if (a.gpack > 1) {   // a tile of several whole output groups
+    o.i = i, o.j = u * a.gpack;
+    o.ng = min(a.gpack, a.q - o.j);
+    o.n0 = o.j * a.r_out;
+    o.n0_w = o.j * a.r;
+    o.cols = o.ng * a.r;   // columns of the accumulator in use (groups at their width in the bank)
+    return o;
+  }
+  const int j = u / a.nt_n, nt = u - j * a.nt_n;
   o.i = i, o.j = j;
   o.n0 = j * a.r_out + nt * a.tile_n;
   o.n0_w = j * a.r + nt * a.tile_n;
@@ -171,7 +185,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
 template <int TILE_N, int BK>
 __global__ void __launch_bounds__(kThreads, 1)
 proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
-                const __grid_constant__ CUtensorMap tmB, const BigArgs a) {
+                const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmB2, const BigArgs a) {
   using C = Cfg<TILE_N, BK>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -204,6 +218,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     if (a.pack > 1) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA2) : "memory");
+    if (a.gpack > 1) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB2) : "memory");
   }
   // Everything above touches only this CTA's own state and may overlap the previous kernel of the stream.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -213,7 +228,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (a.pack > 1) {
       if (lane == 0) ctl->total = ((q + a.pack - 1) / a.pack) * q * a.nt_n;
     } else if (a.sched != 0) {
-      if (lane == 0) ctl->total = q * ((a.rows_per_type + 127) >> 7) * q * a.nt_n;
+      if (lane == 0) ctl->total = q * ((a.rows_per_type + 127) >> 7) * a.col_units;
     } else {
       int carry = 0;
       for (int i0 = 0; i0 < q; i0 += 32) {
@@ -223,7 +238,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const int lo = a.offsets[i], hi = a.offsets[i + 1];
           ctl->off[i] = lo;
           if (i == q - 1) ctl->off[q] = hi;
-          v = ((hi - lo + 127) >> 7) * q * a.nt_n;
+          v = ((hi - lo + 127) >> 7) * a.col_units;
         }
         int incl = v;
 #pragma unroll
@@ -261,13 +276,19 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const bool packed = a.pack > 1;
       // packed tile: segment 0 is the diagonal one (group j), then one panel segment per type of the tile other than j
       const int j_in = packed && tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0;
-      const int n_seg = packed ? 1 + tl.np - j_in : (tl.i == tl.j ? 1 : 2);
+      // tile of several output groups: segment 0 is the panel product (k = i), then one diagonal product per group other than i
+      const bool gp = a.gpack > 1;
+      const int i_in = gp && tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0;
+      const int n_seg = packed ? 1 + tl.np - j_in : gp ? 1 + tl.ng - i_in : (tl.i == tl.j ? 1 : 2);
       const int a_row = a.sched == 2 ? tl.row0 - tl.i * a.rows_per_type : tl.row0;
       for (int sg = 0; sg < n_seg && ok; ++sg) {
         int k;
         if (packed) {
           k = sg == 0 ? tl.j : tl.i + sg - 1;
           if (sg > 0 && j_in && k >= tl.j) ++k;   // skip type j: its rows have their one product already
+        } else if (gp) {
+          k = sg == 0 ? tl.i : tl.j + sg - 1;
+          if (sg > 0 && i_in && k >= tl.i) ++k;   // group i: the panel product already holds x_i W_ii
         } else {
           k = n_seg == 1 ? tl.i : (sg == 0 ? min(tl.i, tl.j) : max(tl.i, tl.j));
         }
@@ -286,9 +307,18 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 tma_load_4d(sa, &tmA2, bar, kb * BK, k, -(k - tl.i) * a.rows_per_type, k);
               }
             } else if (loads_a) {
-              mbar_expect_tx(bar, stage_tx);
+              // (a diagonal segment of a multi-group tile fetches only the 64-column boxes its group touches)
+              const int goff = (k - tl.j) * a.r;
+              const int nb = gp && sg > 0 ? (goff + a.r - 1) / 64 - goff / 64 + 1 : b_chunks;
+              mbar_expect_tx(bar, (uint32_t)(a.a_box_rows * BK * 2 + nb * C::kBChunkBytes));
               if (a.sched == 2) tma_load_4d(sa, &tmA, bar, kb * BK, k, tl.i, a_row);
               else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
+            } else if (gp && sg > 0) {
+              // W_kk at the columns of its group inside the tile, zeros in the rest of the boxes it touches: column
+              // (64 c - offset of the group in the tile) of group k is out of range on both sides of the group
+              const int goff = (k - tl.j) * a.r;
+              for (int c = goff / 64; c <= (goff + a.r - 1) / 64; ++c)
+                tma_load_4d(sa + C::kABytes + c * C::kBChunkBytes, &tmB2, bar, c * 64 - goff, k, kb * BK, k);
             } else {
               for (int c = 0; c < a.n_chunks; ++c)
                 tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, tl.n0_w + c * 64, kb * BK, k);
@@ -317,24 +347,41 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
-      const int n_kb = (a.pack > 1 ? 1 + tl.np - (tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0) : (tl.i == tl.j ? 1 : 2)) * nkb_seg;
+      const int n_kb = (a.pack > 1    ? 1 + tl.np - (tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0)
+                        : a.gpack > 1 ? 1 + tl.ng - (tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0)
+                                      : (tl.i == tl.j ? 1 : 2)) *
+                       nkb_seg;
       if (lane == 0) ALG_TRACE(1, 1);
       ok = __all_sync(0xffffffffu, wait_bar(tempty0 + 8u * (uint32_t)acc, acc_phase ^ 1u, ctl, a.status));
       if (!ok) break;
       if (lane == 0) ALG_TRACE(1, 2);
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
+      const bool gp = a.gpack > 1;
+      const int i_in = gp && tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0;
       for (int kb = 0; kb < n_kb; ++kb) {
         ok = __all_sync(0xffffffffu, wait_bar(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
         if (!ok) break;
         if (kb == 0 && lane == 0) ALG_TRACE(1, 3);
         tc_fence_after();
         const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
-        const uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
+        uint32_t d_seg = d_tmem, idesc_seg = idesc;
+        if (gp && kb >= nkb_seg) {
+          // diagonal segment of a multi-group tile: only the 64-column boxes its group touches were fetched; the
+          // product covers exactly those accumulator columns (zeros outside the group add nothing)
+          int k = tl.j + kb / nkb_seg - 1;
+          if (i_in && k >= tl.i) ++k;
+          const int goff = (k - tl.j) * a.r;
+          const int c_lo = goff / 64, c_hi = (goff + a.r - 1) / 64;
+          db += (uint64_t)(c_lo * (C::kBChunkBytes >> 4));
+          d_seg += (uint32_t)(c_lo * 64);
+          idesc_seg = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(((c_hi - c_lo + 1) * 64) >> 3) << 17);
+        }
         if (elect_one()) {
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk)
-            tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc, (kb | kk) ? 1u : 0u);
+            tc_mma_bf16(d_seg, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 128), idesc_seg, (kb | kk) ? 1u : 0u);
           tc_commit(empty0 + 8u * (uint32_t)stage);
         }
         __syncwarp();
@@ -499,7 +546,18 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                            : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
                            : "r"(buf0 + (uint32_t)rr * 128u + ((((uint32_t)rd_p) ^ (uint32_t)(rr & 7)) << 4)));
               const int64_t dr = dst_row[ph * 4 + g];
-              if (store8) {   // output groups start on 8 bytes only: two 4-column pieces, each stored if it belongs to the tile
+              if (a.gpack > 1) {
+                // the piece's 8 accumulator columns lie in one group of the tile: group gi, column cg of it
+                const int tc = c0 + rd_p * 8, gi = tc / a.r, cg = tc - gi * a.r;
+                __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + dr * a.ldy + tl.n0 + gi * a.r_out + cg;
+                const bool in_tile = dr >= 0 && gi < tl.ng;
+                if (store8) {
+                  if (in_tile && cg < a.r_out) *(uint2 *)dst = make_uint2(val.x, val.y);
+                  if (in_tile && cg + 4 < a.r_out) *(uint2 *)(dst + 4) = make_uint2(val.z, val.w);
+                } else if (in_tile && cg < a.r_out) {
+                  *(uint4 *)dst = val;
+                }
+              } else if (store8) {   // output groups start on 8 bytes only: two 4-column pieces, each stored if it belongs to the tile
                 __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + dr * a.ldy + col + rd_p * 8;
                 if (dr >= 0 && piece_ok) *(uint2 *)dst = make_uint2(val.x, val.y);
                 if (dr >= 0 && col + rd_p * 8 + 4 < col_end) *(uint2 *)(dst + 4) = make_uint2(val.z, val.w);
@@ -533,7 +591,14 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
             for (int x = 0; x < 32; ++x) f[x] = gelu_tanh(f[x]);
           }
-          if (out_row >= 0) {
+          if (out_row >= 0 && a.gpack > 1) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {   // four accumulator columns lie in one group of the tile
+              const int tc = c0 + g * 4, gi = tc / a.r, cg = tc - gi * a.r;
+              if (gi < tl.ng && cg < a.r_out)
+                *(float4 *)((float *)a.Y + out_row * a.ldy + tl.n0 + gi * a.r_out + cg) = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
+            }
+          } else if (out_row >= 0) {
             float *dst = (float *)a.Y + out_row * a.ldy + col;
 #pragma unroll
             for (int g = 0; g < 8; ++g)
@@ -578,9 +643,7 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   static_assert(C::kSmemBytes <= 227 * 1024, "shared memory budget");
   CUtensorMap tmA, tmA2, tmB;
   cudaError_t e;
-  BigArgs b = a;
-  // several types per tile when a type fills at most half of one (equal buckets only)
-  b.pack = a.sched != 0 && a.rows_per_type <= 64 ? std::min(a.q, 128 / a.rows_per_type) : 1;
+  const BigArgs &b = a;
   if (b.pack > 1) {
     // X as {k in group, group, row in type, type}: interval rows of a type are consecutive, cyclic ones q apart
     const uint64_t rpt = (uint64_t)a.rows_per_type;
@@ -605,6 +668,15 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   }
   if (e != cudaSuccess) return e;
   if (b.pack <= 1) tmA2 = tmA;
+  CUtensorMap tmB2;
+  if (b.gpack > 1) {
+    // the bank by {column in group, column group, k in group, row group}
+    const uint64_t dims[4] = {(uint64_t)a.r, (uint64_t)a.q, (uint64_t)a.s, (uint64_t)a.q};
+    const uint64_t str[3] = {(uint64_t)a.r * 2, (uint64_t)a.ldw * 2, (uint64_t)a.ldw * 2 * (uint64_t)a.s};
+    const uint32_t box[4] = {64, 1, (uint32_t)BK, 1};
+    e = make_map_nd(&tmB2, a.W, 4, dims, str, box, 128);
+    if (e != cudaSuccess) return e;
+  }
   {
     // the bank as {columns, k in group, group}: rows past the group's width read as zero
     const uint64_t dims[3] = {(uint64_t)a.q * (uint64_t)a.r * (a.gated_f ? 2 : 1), (uint64_t)a.s, (uint64_t)a.q};
@@ -615,8 +687,8 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   long long tiles;
   if (b.pack > 1) tiles = (long long)((a.q + b.pack - 1) / b.pack) * a.q * a.nt_n;
-  else if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * a.q * a.nt_n;
-  else tiles = ((long long)a.M / 128 + a.q) * a.q * a.nt_n;   // upper bound: every type may end in a ragged tile
+  else if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * b.col_units;
+  else tiles = ((long long)a.M / 128 + a.q) * b.col_units;   // upper bound: every type may end in a ragged tile
   if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)std::min<long long>(num_sms, std::max<long long>(tiles, 1)), 1, 1);
@@ -628,21 +700,36 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_big_kernel<TILE_N, BK>, tmA, tmA2, tmB, b);
+  if (b.gpack <= 1) tmB2 = tmB;
+  e = cudaLaunchKernelEx(&cfg, proj_big_kernel<TILE_N, BK>, tmA, tmA2, tmB, tmB2, b);
   count_launch(1);
   return e;
 }
 
 }  // namespace
 
-cudaError_t launch_proj_big(const BigArgs &a, int num_sms, cudaStream_t st) {
+cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
   cudaError_t e = tc_init();
   if (e != cudaSuccess) return e;
+  BigArgs a = in;
   if ((a.sched == 0) != (a.sched_out == 0)) return cudaErrorInvalidValue;   // counted buckets on both sides or on neither
   if (a.q < 1 || a.q > kBigMaxQ || a.s % 8 || a.r % 8 || a.tile_n % 16 || a.tile_n < 16 || a.tile_n > 256) return cudaErrorInvalidValue;
   if (a.r_out % 4 || a.r_out < 4 || a.r_out > a.r) return cudaErrorInvalidValue;
   if (a.nt_n != (a.r_out + a.tile_n - 1) / a.tile_n || a.n_chunks != (a.tile_n + 63) / 64) return cudaErrorInvalidValue;
   if (a.a_box_rows < 8 || a.a_box_rows > 128 || a.a_box_rows % 8) return cudaErrorInvalidValue;
+  // several row types per tile when a type fills at most half of one (equal buckets only)
+  a.pack = a.sched != 0 && a.rows_per_type <= 64 ? std::min(a.q, 128 / a.rows_per_type) : 1;
+  // several whole output groups per tile when they are narrow (one type per tile, no bias, no gate).  Measured:
+  // 25600 -> 5120 at M = 32768: q = 64 (groups of 80) 0.557 -> 0.533 ms, q = 256 (24) 1.97 -> 1.57 ms; 5120 -> 25600 at
+  // q = 256 (104) 1.49 -> 1.39 ms; groups of 128 lose (square product n = 8192: 0.065 -> 0.088 ms) and stay one per tile
+  a.gpack = 1;
+  a.col_units = a.q * a.nt_n;
+  if (a.pack == 1 && a.nt_n == 1 && !a.gated_f && !a.bias && a.r <= 112 && a.q >= 2) {
+    a.gpack = std::min(a.q, 256 / a.r);
+    a.col_units = (a.q + a.gpack - 1) / a.gpack;
+    a.tile_n = (a.gpack * a.r + 15) / 16 * 16;
+    a.n_chunks = (a.tile_n + 63) / 64;
+  }
   if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
     if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;
     return a.block_k == 64 ? launch_t<256, 64>(a, num_sms, st) : launch_t<256, 32>(a, num_sms, st);
