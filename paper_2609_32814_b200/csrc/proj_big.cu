@@ -725,10 +725,17 @@ cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
   a.gpack = 1;
   a.col_units = a.q * a.nt_n;
   if (a.pack == 1 && a.nt_n == 1 && !a.gated_f && !a.bias && a.r <= 112 && a.q >= 2) {
-    a.gpack = std::min(a.q, 256 / a.r);
-    a.col_units = (a.q + a.gpack - 1) / a.gpack;
-    a.tile_n = (a.gpack * a.r + 15) / 16 * 16;
-    a.n_chunks = (a.tile_n + 63) / 64;
+    // ... as many as keep at least four tiles per SM (2048 -> 768 in 16 groups of 48 at M = 2048 has 256 tiles of one
+    // group: five groups per tile would leave 64 tiles for 148 SMs)
+    const long long m_tiles = a.sched != 0 ? (long long)a.q * ((a.rows_per_type + 127) / 128) : std::max<long long>(a.q, a.M / 128);
+    int g = std::min(a.q, 256 / a.r);
+    while (g > 1 && m_tiles * ((a.q + g - 1) / g) < 4ll * num_sms) --g;
+    if (g > 1) {
+      a.gpack = g;
+      a.col_units = (a.q + g - 1) / g;
+      a.tile_n = (g * a.r + 15) / 16 * 16;
+      a.n_chunks = (a.tile_n + 63) / 64;
+    }
   }
   if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
     if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;

@@ -58,10 +58,11 @@ def _forward(wl, schedule, out_dtype, **kw):
     (50, 50, 16, 24, "interval"),           # one row per type: fifty types in one tile
     (7, 7 * 64, 64, 128, "interval"),       # two types per tile, the last one alone
     (20, 20 * 33, 8, 264, "cyclic"),        # 33 rows per type (three per tile, boxes off the 8-row swizzle atom), two column tiles
-    (13, 13 * 150, 72, 40, "interval"),     # six output groups per tile (240 columns), the last tile holds one; 128 + 22 rows
-    (9, 1234, 136, 104, "explicit"),        # two groups per tile, the second one across three 64-column boxes; counted buckets
-    (21, 21 * 130, 24, 24, "cyclic"),       # ten groups per tile, the last tile one; groups straddle the 64-column boxes
-    (6, 6 * 200, 200, 88, "cyclic"),        # widths of 4 only in the reduction (repacked), two groups per tile
+    # several narrow output groups per tile (taken when at least four tiles per SM remain):
+    (40, 40 * 150, 72, 40, "cyclic"),       # five groups per tile (200 columns); 128 + 22 rows per type
+    (48, 4800, 136, 104, "explicit"),       # two groups per tile, the second one across three 64-column boxes; counted buckets
+    (64, 64 * 130, 24, 24, "interval"),     # ten groups per tile, the last tile four; groups straddle the 64-column boxes
+    (32, 32 * 200, 100, 88, "cyclic"),      # widths of 4 only in the reduction (repacked), two groups per tile
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
