@@ -238,7 +238,11 @@ alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *stat
  * and the same row types (the projection is row-local).  d_widths: q groups of d_model,
  * f_widths: q groups of d_ff.  X: M x D packed (ld = D), W_up: D x F packed, W_down: F x D
  * packed, Y: M x D packed.  The hidden state H = act(.) is kept in the workspace in the
- * handle's dtype (bf16: rounded to nearest even), rows in type-bucketed order. */
+ * handle's dtype (bf16: rounded to nearest even), rows in type-bucketed order.
+ * 1 <= q <= ALG_MAX_Q, schedule EXPLICIT or CYCLIC (larger algebras and the INTERVAL schedule
+ * exist for single projections only: ALG_ERR_UNSUPPORTED_SHAPE).  Which GEMM kernel runs the two
+ * projections is the library's choice per call (alg_ffn_set_option(GEMM_KERNEL) overrides it);
+ * kernels differ in the order of their fp32 sums, so results agree to rounding between them. */
 alg_status_t alg_ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths,
                             const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,
                             const uint8_t *custom_keep, alg_schedule_t schedule);
