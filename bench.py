@@ -66,9 +66,9 @@ CONFIGS = {
                 label="cfg5: q=8 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
     "5q16": dict(q=16, D=4096, F=16384, M=32768, law="qq", schedule="explicit",
                  label="cfg5: q=16 FFN 4096->16384->4096, M=32768 rows, i.i.d. row types, bf16"),
-    "pilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="explicit",
+    "pilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="interval", period=768,
                   label="pilot: Q_2 (x) Q_2 FFN 768->1536->768 (4 x 192 / 4 x 384), M=8x1536 rows, interval schedule, bf16"),
-    "gpilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="explicit", gated=True,
+    "gpilot": dict(q=4, D=768, F=1536, M=8 * 1536, law="q2pow", schedule="interval", period=768, gated=True,
                    label="gated pilot: bias-free SwiGLU FFN 768->1536->768 under Q_2 (x) Q_2 (4 x 192 / 4 x 384), merged gate/up "
                          "bank, M=8x1536 rows, interval schedule, bf16"),
     "g8b": dict(q=32, D=4096, F=12288, M=2048, law="qq", schedule="explicit", gated=True,
@@ -417,18 +417,25 @@ def run_prefill(args, ctx):
     name, cfg = args.config, CONFIGS[args.config]
     wl = make_workload(name)
     dev = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)
-    # configuration 2 fixes the schedule "type = position mod 2": its handle is created with that
-    # schedule (the per-call types array is then not needed); the explicit-types path of the same
+    # configuration 2 fixes the schedule "type = position mod 2" and the pilot shapes the interval typing
+    # of period 768: their handles are created with that schedule (the per-call types array is then not
+    # needed, rows are read and written in place); the explicit-types path of the same
     # workload is timed as a side measurement.  The other configurations draw i.i.d. row types.
     gated = bool(cfg.get("gated"))
     Handle = binding.GatedFFN if gated else binding.FFN
-    ffn = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"], schedule=cfg["schedule"])
+    def make_handle(table):
+        h = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table=table, schedule=cfg["schedule"])
+        if cfg.get("period"):       # interval typing that repeats: type = floor((position mod period) / (period / q))
+            h.set_option("interval_period", cfg["period"])
+        return h
+
+    ffn = make_handle(cfg["law"])
     w_up_host = np.concatenate([wl.meta["W_gate"], wl.W_up], axis=1) if gated else wl.W_up   # merged bank [W_gate | W_up]
     counts = np.bincount(wl.types, minlength=wl.q).tolist()
     flops = 2 * ffn.macs(counts)
     stream = torch.cuda.current_stream()
     types = torch.from_numpy(wl.types).cuda()
-    call_types = None if cfg["schedule"] == "cyclic" else types
+    call_types = types if cfg["schedule"] == "explicit" else None
     M, D, F = wl.M, wl.D, wl.F
 
     # ---- working sets: independent copies of (X, W_up, W_down, Y, workspace) used round-robin, so
@@ -559,8 +566,9 @@ def run_prefill(args, ctx):
         if gated:
             with torch.cuda.stream(sl["stream"]):
                 sl["Xd"].copy_(sl["X"], non_blocking=True)
-                sl["td"].copy_(sl["t"], non_blocking=True)
-                ffn.forward(sl["Xd"], sl["td"], sets[i % n_sets]["Wu"], sets[i % n_sets]["Wd"], out=sl["Yd"], workspace=sl["wsd"],
+                if sl["t"] is not None:
+                    sl["td"].copy_(sl["t"], non_blocking=True)
+                ffn.forward(sl["Xd"], None if sl["t"] is None else sl["td"], sets[i % n_sets]["Wu"], sets[i % n_sets]["Wd"], out=sl["Yd"], workspace=sl["wsd"],
                             stream=sl["stream"])
                 sl["Y"].copy_(sl["Yd"], non_blocking=True)
             return
@@ -592,7 +600,7 @@ def run_prefill(args, ctx):
     extras = {}
     if rank == 0 and not args.no_extras:
         n = min(24, args.steps)
-        dense = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table="dense", schedule=cfg["schedule"])
+        dense = make_handle("dense")
         time_steps(min(6, n), dense)
         dense_ms = time_steps(n, dense) / n
         star_ms = time_steps(n) / n
@@ -601,13 +609,14 @@ def run_prefill(args, ctx):
                               "control": "same library, ALG_TABLE_DENSE, same schedule, measured back to back with the star_q run",
                               "ideal_ratio": flops / (2.0 * (3 if gated else 2) * M * D * F)}
         del dense
-        if name == "2":
-            explicit = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+        if cfg["schedule"] != "explicit":
+            explicit = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"])
             time_steps(6, explicit, types)
             ex_ms = time_steps(n, explicit, types) / n
             extras["explicit_types"] = {"ms_per_step": ex_ms, "frac_of_roofline": (flops / (ex_ms * 1e-3) / 1e12) / peak_tf,
                                         "note": "same workload through ALG_SCHED_EXPLICIT (bucketing + row gather kernels run)"}
             del explicit
+        if name == "2":
             extras["decode"] = decode_measurements(binding)
 
     cpu = time_cpu_oracle(name, wl) if rank == 0 else None

@@ -81,7 +81,10 @@ typedef enum { ALG_ACT_NONE = 0, ALG_ACT_GELU_ERF = 1, ALG_ACT_GELU_TANH = 2 } a
  * INTERVAL: type of row b is b / (M/q), q | M: the rows of a type are contiguous -- the typing of
  *           the square product A * B of two algebra elements (Eqs. q-product-diag/off), where
  *           the rows of block row i of A carry type i; `types` may be NULL.  No permutation and
- *           no copy of X.  Large-algebra path only (see alg_proj_create). */
+ *           no copy of X.  Handles that fit the large-algebra path (see alg_proj_create) take it;
+ *           other bf16 handles with tensor-core widths read X in 64-row boxes inside the runs of
+ *           a type (M / q a multiple of 64) and may repeat the typing with a period
+ *           (ALG_OPT_INTERVAL_PERIOD); FFN handles of that kind accept INTERVAL too. */
 typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1, ALG_SCHED_INTERVAL = 2 } alg_schedule_t;
 
 /* Kernel families, reported by alg_proj_kernel_path(). */
@@ -108,7 +111,12 @@ typedef enum {
  *                     that divides every output group width.
  *   STAGE_K           reduction depth of one pipeline stage of the one-CTA GEMM kernel: 0 =
  *                     automatic, 32 (eight stages of 24 KB) or 64 (four stages of 48 KB).  Results
- *                     are identical; only the operand pipeline differs.
+ *                     are identical; only the operand pipeline differs.  A table-driven INTERVAL
+ *                     handle reads its runs with 64-deep stages only: 32 is ALG_ERR_UNSUPPORTED_SHAPE there.
+ *   INTERVAL_PERIOD   INTERVAL schedule of a table-driven handle: the typing repeats every P rows, type of
+ *                     row b = (b mod P) / (P / q) -- the pilot model's schedule
+ *                     floor((p mod 768) / 192) over a batch of sequences.  0 (default) = one period,
+ *                     P = M.  q must divide P, P must divide M, and P / q must be a multiple of 64.
  *   SMALL_M_KERNEL    1 (default): M <= 64 runs the weight-streaming kernels; 0: the prefill
  *                     kernels take every M.
  *   HOST_PLAN         1 (default): cyclic-schedule tile sequences are planned on the host;
@@ -127,7 +135,8 @@ typedef enum {
   ALG_OPT_HOST_PLAN = 4,
   ALG_OPT_WAIT_LIMIT_CYCLES = 5,
   ALG_OPT_TEST_STALL_BYTES = 6,
-  ALG_OPT_STAGE_K = 7
+  ALG_OPT_STAGE_K = 7,
+  ALG_OPT_INTERVAL_PERIOD = 8
 } alg_option_t;
 
 /* ---- projection handle ---------------------------------------------------------------------

@@ -29,6 +29,7 @@ constexpr int kPlanSlots = 4;
 // Large-algebra path (proj_big.cu): complete-graph law, equal group widths, q up to kBigMaxQ.
 struct BigPlan {
   bool on = false;
+  bool only = false;      // the handle has no interaction table: created for the large-algebra kernel alone
   bool eligible = false;  // the handle's law, dtype and widths fit the large-algebra kernel (GEMM_KERNEL = 4 may select it)
   int s = 0, r = 0;       // width of every input / output group
   int s_pad = 0, r_pad = 0;   // the same rounded up to multiples of 8: what the tensor maps can address
@@ -66,6 +67,7 @@ struct alg_proj_s {
   DecodePlan decode = {};
   // options (alg_proj_set_option)
   int opt_kernel = 0, opt_tile_n = 0, opt_stage_k = 0;
+  int64_t interval_period = 0;   // INTERVAL schedule of a table-driven handle: period of the typing (0 = the whole batch)
   bool opt_small_m = true, opt_host_plan = true;
   long long wait_limit = kDefaultWaitLimit;
   int test_extra_expect = 0;
@@ -171,6 +173,7 @@ alg_status_t configure_kernels(alg_proj_s &p) {
     p.pair_kernel = false;
   }
   if (p.w_kmajor || p.dyn_segments) p.pair_kernel = false;   // the gradient passes run on the one-CTA kernel
+  if (p.sched == ALG_SCHED_INTERVAL) p.pair_kernel = false;  // runs of a type are read in place by the one-CTA kernel only
   if (p.opt_kernel == 1) p.pair_kernel = false;
   if (p.opt_kernel == 2) {
     if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
@@ -228,6 +231,7 @@ alg_status_t init_big(alg_proj_s &p, int q, int s, int r, alg_schedule_t sched) 
   p.K = q * s;
   p.N = q * r;
   plan_big(p, s, r);
+  p.big.only = true;
   if (q <= kMaxQ)
     for (int g = 0; g < q; ++g) p.s[g] = s, p.r[g] = r;
   if (cudaGetDevice(&p.device) != cudaSuccess) return ALG_ERR_CUDA;
@@ -251,10 +255,11 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   bool big_fits = allow_big && table == ALG_TABLE_QQ && dtype == ALG_BF16 && in_w[0] > 0 && out_w[0] > 0 &&
                   in_w[0] % 4 == 0 && out_w[0] % 4 == 0;
   for (int g = 1; g < q && big_fits; ++g) big_fits = in_w[g] == in_w[0] && out_w[g] == out_w[0];
-  if (q > kMaxQ || sched == ALG_SCHED_INTERVAL) {
+  if (q > kMaxQ || (sched == ALG_SCHED_INTERVAL && big_fits)) {
     if (!big_fits || (int64_t)q * in_w[0] > (1 << 30) || (int64_t)q * out_w[0] > (1 << 30)) return ALG_ERR_UNSUPPORTED_SHAPE;
     return init_big(p, q, in_w[0], out_w[0], sched);
   }
+  // (an INTERVAL handle that does not fit the large-algebra path is a table-driven one: checked below)
   if (dtype != ALG_F32 && dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
   if (table != ALG_TABLE_QQ && table != ALG_TABLE_DENSE && table != ALG_TABLE_CUSTOM && table != ALG_TABLE_Q2POW)
     return ALG_ERR_INVALID_ARG;
@@ -297,6 +302,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
     }
   alg_status_t cs = configure_kernels(p);
   if (cs != ALG_OK) return cs;
+  if (sched == ALG_SCHED_INTERVAL && !use_tc(p)) return ALG_ERR_UNSUPPORTED_SHAPE;
   if (big_fits) {
     plan_big(p, in_w[0], out_w[0]);
     p.big.eligible = true;
@@ -333,7 +339,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
       if (cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming) != cudaSuccess) return ALG_ERR_CUDA;
     }
   }
-  if (dtype == ALG_BF16 && !p.gated && !p.w_kmajor && !p.dyn_segments) {
+  if (dtype == ALG_BF16 && !p.gated && !p.w_kmajor && !p.dyn_segments && sched != ALG_SCHED_INTERVAL) {
     p.decode_ok = decode_plan(q, p.s, p.K, p.N, p.num_sms, &p.decode);
     for (int g = 0; g < q && p.decode_ok; ++g)
       if (p.r[g] % p.decode.sn) p.decode_ok = false;
@@ -509,8 +515,8 @@ bool use_big_equal(const alg_proj_s &p, int64_t M) {
 alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, int64_t ldx,
                       bool x_bucketed, const void *W, int64_t ldw, const void *bias, alg_act_t act, void *Y,
                       int64_t ldy, alg_dtype_t y_dtype, bool y_bucketed, int64_t M, cudaStream_t st,
-                      cudaEvent_t after_gather = nullptr, bool cyclic = false) {
-  if (cyclic && use_big_equal(p, M)) {
+                      cudaEvent_t after_gather = nullptr, bool cyclic = false, int run_rows = 0, int64_t run_period = 0) {
+  if (cyclic && !run_rows && use_big_equal(p, M)) {
     // equal buckets on the large-algebra kernel: the caller's rows are read / written in place (type-strided),
     // a bucketed operand or result is the interval layout
     BigArgs g;
@@ -597,6 +603,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.status = p.d_status;
   a.a_cyclic_rows = (cyclic && !x_bucketed) ? (int)(M / p.q) : 0;
   a.out_cyclic_rows = (cyclic && !y_bucketed) ? (int)(M / p.q) : 0;
+  a.run_rows = run_rows, a.run_period = (int)run_period;
   a.b_3d = 0;
   a.a_box_256 = 0;
   a.gated_f = p.gated ? p.N : 0;
@@ -642,6 +649,15 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
   a.ldx = ldx;
   a.in_perm = x_bucketed ? nullptr : (const int *)(ws + L.perm);
   return cuda_status(launch_proj_simt(a, p.dtype == ALG_BF16, st));
+}
+
+// INTERVAL schedule of a table-driven handle: rows per run and period for a batch of M rows; false if the batch
+// does not split into whole periods of q runs of a multiple of 64 rows.
+bool interval_runs(const alg_proj_s &p, int64_t M, int *run_rows, int64_t *period) {
+  const int64_t P = p.interval_period ? p.interval_period : M;
+  if (P <= 0 || M % P || P % p.q || (P / p.q) % 64) return false;
+  *run_rows = (int)(P / p.q), *period = P;
+  return true;
 }
 
 bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && p.opt_small_m && M <= kDecodeMaxM; }
@@ -782,7 +798,7 @@ alg_status_t alg_proj_destroy(alg_proj_t h) {
 }
 
 static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value) {
-  const bool no_table = p.q > kMaxQ || p.sched == ALG_SCHED_INTERVAL;   // large-algebra handles have one kernel
+  const bool no_table = p.big.only;   // large-algebra handles have one kernel
   switch (option) {
     case ALG_OPT_GEMM_KERNEL:
     case ALG_OPT_TILE_N: {
@@ -815,8 +831,15 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
     }
     case ALG_OPT_STAGE_K:
       if (value != 0 && value != 32 && value != 64) return ALG_ERR_INVALID_ARG;
+      if (value == 32 && p.sched == ALG_SCHED_INTERVAL && !no_table) return ALG_ERR_UNSUPPORTED_SHAPE;  // runs: 64-deep only
       p.opt_stage_k = (int)value;
       for (PlanSlot &sl : p.plan) sl.M = -1;  // cached plans count K blocks of the old depth
+      return ALG_OK;
+    case ALG_OPT_INTERVAL_PERIOD:
+      if (value < 0 || value > (1 << 30)) return ALG_ERR_INVALID_ARG;
+      if (p.sched != ALG_SCHED_INTERVAL || (no_table && value != 0)) return ALG_ERR_UNSUPPORTED_SHAPE;
+      if (value % ((int64_t)64 * p.q)) return ALG_ERR_INVALID_ARG;   // q runs of a multiple of 64 rows
+      p.interval_period = value;
       return ALG_OK;
     case ALG_OPT_SMALL_M_KERNEL: p.opt_small_m = value != 0; return ALG_OK;
     case ALG_OPT_HOST_PLAN: p.opt_host_plan = value != 0; return ALG_OK;
@@ -889,6 +912,12 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   b.ldy = ldy;
   b.N = h->N;
   b.y_elem_bytes = elem_bytes(y_dtype);
+  if (h->sched == ALG_SCHED_INTERVAL) {   // runs of a type read and written in place
+    int run_rows = 0;
+    int64_t period = 0;
+    if (!interval_runs(*h, M, &run_rows, &period)) return ALG_ERR_INVALID_ARG;
+    return run_proj(*h, L, ws, X, ldx, false, W, ldw, bias, act, Y, ldy, y_dtype, false, M, st, nullptr, true, run_rows, period);
+  }
   // cyclic schedule with equal buckets: no counting, no permutation, no gather
   const bool cyc = h->sched == ALG_SCHED_CYCLIC && use_tc(*h) && M % h->q == 0;
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
@@ -932,7 +961,7 @@ alg_status_t alg_proj_forward_host(alg_proj_t h, const void *X_host, const int32
 alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
   if (!h || !n) return ALG_ERR_INVALID_ARG;
   int64_t c = 0;
-  if (h->q > kMaxQ || h->sched == ALG_SCHED_INTERVAL) c = 2 * (int64_t)h->q * h->q - h->q;   // no table: Q_q law (Eq. q-rank)
+  if (h->big.only) c = 2 * (int64_t)h->q * h->q - h->q;   // no table: Q_q law (Eq. q-rank)
   else for (int pr = 0; pr < h->q * h->q; ++pr) c += __builtin_popcount(h->tab.keep[pr]);
   *n = c;
   return ALG_OK;
@@ -941,7 +970,7 @@ alg_status_t alg_proj_gemm_count(alg_proj_t h, int64_t *n) {
 alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *macs) {
   if (!h || !rows_per_type || !macs) return ALG_ERR_INVALID_ARG;
   int64_t total = 0;
-  if (h->q > kMaxQ || h->sched == ALG_SCHED_INTERVAL) {   // no table: one product on the diagonal, two elsewhere
+  if (h->big.only) {   // no table: one product on the diagonal, two elsewhere
     for (int i = 0; i < h->q; ++i) {
       if (rows_per_type[i] < 0) return ALG_ERR_INVALID_ARG;
       total += rows_per_type[i] * (2 * (int64_t)h->q - 1) * h->big.s * h->big.r;
@@ -1190,6 +1219,7 @@ alg_status_t alg_proj_grad_weight(alg_proj_grad_t h, const void *X, int64_t ldx,
   a.status = p.d_status;
   a.a_cyclic_rows = 0;
   a.out_cyclic_rows = 0;
+  a.run_rows = 0, a.run_period = 0;
   a.b_3d = 0;
   a.a_box_256 = 0;
   a.gated_f = 0;
@@ -1218,13 +1248,14 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
   alg_ffn_s *f = new (std::nothrow) alg_ffn_s();
   if (!f) return ALG_ERR_INVALID_ARG;
   f->gated = gated;
-  if (q > kMaxQ || schedule == ALG_SCHED_INTERVAL) {   // large-algebra handles are single projections
+  if (q > kMaxQ) {   // large-algebra handles are single projections
     delete f;
     return q > kBigMaxQ || q < 1 ? ALG_ERR_INVALID_ARG : ALG_ERR_UNSUPPORTED_SHAPE;
   }
   // (allow_big: with explicit types an FFN whose law and widths fit may run its projections on the large-algebra kernel)
   alg_status_t s = init_proj(f->up, q, d_widths, f_widths, dtype, table, custom_keep, schedule, nullptr, gated, true);
   if (s == ALG_OK) s = init_proj(f->down, q, f_widths, d_widths, dtype, table, custom_keep, schedule, f->up.d_status, false, true);
+  if (s == ALG_OK && (f->up.big.only || f->down.big.only)) s = ALG_ERR_UNSUPPORTED_SHAPE;   // (interval schedule on the large-algebra path)
   if (s != ALG_OK) {
     free_proj(f->down);
     free_proj(f->up);
@@ -1233,7 +1264,8 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
   }
   f->D = f->up.K;
   f->F = f->up.N;
-  if (dtype == ALG_BF16 && !gated && ffn_decode_plan(q, f->up.s, f->down.s, f->D, f->F, f->up.num_sms, &f->fd)) {
+  if (dtype == ALG_BF16 && !gated && schedule != ALG_SCHED_INTERVAL &&
+      ffn_decode_plan(q, f->up.s, f->down.s, f->D, f->F, f->up.num_sms, &f->fd)) {
     f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
@@ -1346,18 +1378,22 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   b.y_elem_bytes = elem_bytes(y_dtype);
   const bool tm = h->timing;
   if (tm) cudaEventRecord(h->ev[0], st);
-  const bool cyc = h->up.sched == ALG_SCHED_CYCLIC && M % h->up.q == 0 &&
-                   ((use_tc(h->up) && use_tc(h->down)) || (use_big_equal(h->up, M) && use_big_equal(h->down, M)));
+  int run_rows = 0;
+  int64_t run_period = 0;
+  if (h->up.sched == ALG_SCHED_INTERVAL && !interval_runs(h->up, M, &run_rows, &run_period)) return ALG_ERR_INVALID_ARG;
+  const bool cyc = run_rows > 0 ||
+                   (h->up.sched == ALG_SCHED_CYCLIC && M % h->up.q == 0 &&
+                    ((use_tc(h->up) && use_tc(h->down)) || (use_big_equal(h->up, M) && use_big_equal(h->down, M))));
   if (!cyc && launch_bucket(b, st) != cudaSuccess) return ALG_ERR_CUDA;
   if (tm) cudaEventRecord(h->ev[1], st);
   void *H = ws + L.h;
   if (h->gated && (b_up || b_down || act != ALG_ACT_NONE)) return ALG_ERR_INVALID_ARG;   // bias-free, silu(gate) * up
   alg_status_t s = run_proj(h->up, L, ws, X, h->D, false, W_up, h->gated ? 2 * (int64_t)h->F : h->F, b_up, act, H, h->F,
-                            h->up.dtype, true, M, st, tm ? h->ev[2] : nullptr, cyc);
+                            h->up.dtype, true, M, st, tm ? h->ev[2] : nullptr, cyc, run_rows, run_period);
   if (s != ALG_OK) return s;
   if (tm) cudaEventRecord(h->ev[3], st);
   s = run_proj(h->down, L, ws, H, h->F, true, W_down, h->D, b_down, ALG_ACT_NONE, Y, h->D, y_dtype, false, M, st,
-               nullptr, cyc);
+               nullptr, cyc, run_rows, run_period);
   if (tm) cudaEventRecord(h->ev[4], st);
   return s;
 }

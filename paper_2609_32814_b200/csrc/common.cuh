@@ -137,6 +137,13 @@ struct ProjArgs {
   // original row = (bucketed row - i*M/q)*q + i.  0 = off.
   int a_cyclic_rows;
   int out_cyclic_rows;
+  // Interval schedule with a period (type of row b = (b mod run_period) / run_rows, run_rows = run_period / q):
+  // the rows of a type come in runs of run_rows consecutive rows, one run per period.  With run_rows > 0 the two
+  // fields above still switch the in-place views on, but the A operand is fetched in 64-row boxes from the view
+  // {K, row in run, type, period} (run_rows is a multiple of 64, so a box never leaves its run) and the epilogue
+  // computes original row = period * run_period + i * run_rows + row in run.  0 = cyclic addressing.
+  int run_rows;
+  int run_period;
   int b_3d;               // B tensor map is the 3-D chunked view (one copy per stage)
   int a_box_256;          // A tensor map carries 256-row boxes (one-CTA kernel with 256-row tiles)
   // Gradient passes.  w_kmajor: W is used transposed (B operand K-major; dX = G W^T): the reduction

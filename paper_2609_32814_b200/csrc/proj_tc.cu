@@ -117,7 +117,7 @@ struct Cfg {
 // N = 256 MMA fills both halves of the accumulator, and the epilogue writes silu(gate) * up -- 128
 // output columns per tile, the hidden state is stored once and the two pre-activations never
 // leave the chip (the merged gate/up kernel of the appendix "Kernel Benchmark Details").
-template <int TILE_N, int TILE_M, bool GATED, int BK>
+template <int TILE_N, int TILE_M, bool GATED, int BK, bool RUNS>
 __global__ void __launch_bounds__(kThreads, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
   using C = Cfg<TILE_N, TILE_M, BK>;
@@ -262,6 +262,14 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int c = 0; c < TILE_N / 64; ++c)
                   tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, n0 + c * 64, k, pos0);
               }
+            } else if (RUNS && loads_a && a.a_cyclic_rows) {
+              // runs of run_rows rows per period: 64-row boxes, each inside one run
+              mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+#pragma unroll
+              for (int h = 0; h < TILE_M / 64; ++h) {
+                const int b = a_row + 64 * h, per = b / a.run_rows;
+                tma_load_4d(sa + h * (64 * BK * 2), &tmA, bar, k0, b - per * a.run_rows, type_i, per);
+              }
             } else if (loads_a) {
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
               if (a.a_cyclic_rows) tma_load_3d(sa, &tmA, bar, k0, type_i, a_row);
@@ -364,7 +372,11 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // accumulated, its result is zero
       const bool empty_tile = ((uint32_t)rec.rows >> 16) == 0u;
       if (r < tile_rows) {
-        if (a.out_cyclic_rows) {
+        if (RUNS && a.out_cyclic_rows) {
+          const int i = (rec.pair & 0xFFFF) / q;
+          const int bt = rec.row0 + r - i * a.out_cyclic_rows, per = bt / a.run_rows;
+          out_row = (int64_t)per * a.run_period + i * a.run_rows + (bt - per * a.run_rows);
+        } else if (a.out_cyclic_rows) {
           const int i = (rec.pair & 0xFFFF) / q;
           out_row = (int64_t)(rec.row0 + r - i * a.out_cyclic_rows) * q + i;
         } else {
@@ -492,12 +504,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
-template <int TILE_N, int TILE_M, bool GATED, int BK>
+template <int TILE_N, int TILE_M, bool GATED, int BK, bool RUNS = false>
 cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   using C = Cfg<TILE_N, TILE_M, BK>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED, BK, RUNS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -549,13 +561,15 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED, BK>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED, BK, RUNS>, tmA, tmB, b);
   count_launch(1);
   return e;
 }
 
 template <int TILE_N, int TILE_M, bool GATED = false>
 cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
+  // the in-place view of an interval schedule (runs of a type) is a kernel variant of its own, 64-deep stages only
+  if (a.run_rows) return a.block_k == 64 ? launch_bk<TILE_N, TILE_M, GATED, 64, true>(a, num_sms, st) : cudaErrorInvalidValue;
   if (a.block_k == 32) return launch_bk<TILE_N, TILE_M, GATED, 32>(a, num_sms, st);
   if (a.block_k == 64) return launch_bk<TILE_N, TILE_M, GATED, 64>(a, num_sms, st);
   return cudaErrorInvalidValue;
@@ -634,6 +648,12 @@ cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a) {
   if (!a.a_cyclic_rows)
     return make_map_2d_sw(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, (uint32_t)a.block_k, box_rows,
                           a.block_k * 2);
+  if (a.run_rows) {   // {K, row in run, type, period}, boxes of 64 rows
+    const uint64_t dims[4] = {(uint64_t)a.K, (uint64_t)a.run_rows, (uint64_t)a.q, (uint64_t)(a.M / a.run_period)};
+    const uint64_t str[3] = {(uint64_t)a.ldx * 2, (uint64_t)a.ldx * 2 * (uint64_t)a.run_rows, (uint64_t)a.ldx * 2 * (uint64_t)a.run_period};
+    const uint32_t box[4] = {(uint32_t)a.block_k, 64, 1, 1};
+    return make_map_nd(map, a.X, 4, dims, str, box, a.block_k * 2);
+  }
   cuuint64_t dims[3] = {(cuuint64_t)a.K, (cuuint64_t)a.q, (cuuint64_t)a.a_cyclic_rows};
   cuuint64_t strides[2] = {(cuuint64_t)a.ldx * 2, (cuuint64_t)a.ldx * 2 * (cuuint64_t)a.q};
   cuuint32_t box[3] = {(cuuint32_t)a.block_k, 1, box_rows};

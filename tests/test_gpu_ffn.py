@@ -298,6 +298,51 @@ def test_pilot_tensor_square_law_and_interval_schedule():
     H.assert_bf16_close(H.to_np(Yd), refd, False, "pilot decode")
 
 
+@pytest.mark.parametrize("q,P,periods,dw,fw,table", [
+    (4, 768, 8, 192, 384, "q2pow"),     # the pilot's schedule floor((p mod 768) / 192): runs of 192 rows, eight sequences
+    (2, 256, 5, 128, 256, "qq_unequal"),  # runs of 128 rows; unequal widths keep the handle on the table-driven kernel
+    (4, 4096, 1, 128, 256, "q2pow"),    # one period: runs of 1024 rows (256-row tiles where the widths allow them)
+])
+def test_interval_schedule_with_period_reads_runs_in_place(q, P, periods, dw, fw, table):
+    """INTERVAL schedule of a table-driven handle: type = (row mod P) / (P / q).  No bucketing, no gather (two
+    launches per FFN); same bits as the explicit-types path on the same kernel, projection bit-exact on integers."""
+    M = P * periods
+    types = synth.interval_types(M, q, P)
+    d_w, f_w = [dw] * q, [fw] * q
+    law = "q2pow"
+    if table == "qq_unequal":
+        d_w, f_w, law = [dw, 2 * dw], [fw, 2 * fw], "qq"
+    wl = synth.make_workload("itv", config=7, variant=q * 100 + periods, dtype="bf16", q=q, M=M, D=sum(d_w), F=sum(f_w),
+                             types=types, integer=True, d_widths=d_w, f_widths=f_w)
+    keep = oracle.support(q, law)
+    proj = binding.Proj(d_w, f_w, dtype="bf16", table=law, schedule="interval")
+    if periods > 1:
+        proj.set_option("interval_period", P)
+    launches = binding.launch_count()
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), None, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+    assert proj.last_status() == 0 and binding.launch_count() - launches == 1
+    assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, wl.types, wl.W_up, d_w, f_w, keep=keep))
+    # the FFN on real data: interval schedule against explicit types on the same kernel, and against the oracle
+    wr = synth.make_workload("itvr", config=7, variant=q * 100 + periods + 1, dtype="bf16", q=q, M=M, D=sum(d_w), F=sum(f_w),
+                             types=types, d_widths=d_w, f_widths=f_w)
+    f_int = binding.FFN(d_w, f_w, dtype="bf16", table=law, schedule="interval")
+    if periods > 1:
+        f_int.set_option("interval_period", P)
+    f_exp = binding.FFN(d_w, f_w, dtype="bf16", table=law, schedule="explicit")
+    f_exp.set_option("gemm_kernel", 1)
+    launches = binding.launch_count()
+    Y_int = _run_ffn(wr, f_int, torch.float32, types=False)
+    assert binding.launch_count() - launches == 2
+    Y_exp = _run_ffn(wr, f_exp, torch.float32)
+    assert torch.equal(Y_int, Y_exp)
+    rows = _sample_rows(wr, 64, seed=5)
+    ref = oracle.ffn(wr.X[rows], wr.types[rows], wr.W_up, wr.W_down, d_w, f_w, keep=keep)
+    H.assert_bf16_close(H.to_np(Y_int[torch.from_numpy(rows).cuda()]), ref, False, "interval FFN")
+    # a batch that is no whole number of periods is refused
+    with pytest.raises(binding.AlgError):
+        proj.forward(H.to_dev(wl.X[:M - 64], "bf16"), None, H.to_dev(wl.W_up, "bf16"))
+
+
 def _random_ffn_case(k):
     rng = np.random.default_rng(500 + k)
     q = int(rng.choice([1, 2, 3, 4, 8, 16, 32]))

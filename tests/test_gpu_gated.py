@@ -90,6 +90,37 @@ def test_gated_pilot_shape_tensor_square_law():
     assert ffn.macs(counts) * 16 == 9 * 3 * M * 768 * 1536          # (3/4)^2 of the dense 3 M D F
 
 
+def test_gated_pilot_interval_schedule_in_place():
+    """The pilot's typing floor((p mod 768) / 192) as the handle's schedule: the merged gate/up kernel reads the runs
+    of a type in place and the down projection writes them back in place -- two launches, no types array, and the
+    same bits as the explicit-types path on the same kernel."""
+    M = 4 * 768
+    types = synth.interval_types(M, 4, 768)
+    wl, Wg = synth.gated_ffn("pilot-gated-itv", 4, M, 768, 1536, types, variant=3)
+    Wgu = H.to_dev(np.concatenate([Wg, wl.W_up], axis=1), "bf16")
+    Xd, Wd = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_down, "bf16")
+    f_int = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16", table="q2pow", schedule="interval")
+    f_int.set_option("interval_period", 768)
+    launches = binding.launch_count()
+    Y_int = f_int.forward(Xd, None, Wgu, Wd, out_dtype=torch.float32)
+    assert f_int.last_status() == 0 and binding.launch_count() - launches == 2
+    f_exp = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16", table="q2pow")
+    f_exp.set_option("gemm_kernel", 1)
+    Y_exp = f_exp.forward(Xd, H.dev_types(types), Wgu, Wd, out_dtype=torch.float32)
+    assert torch.equal(Y_int, Y_exp)
+    rows = _sample_rows(wl, 48, seed=6)
+    keep = oracle.support(4, "q2pow")
+    ref = oracle.ffn_swiglu(wl.X[rows], wl.types[rows], Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, keep=keep)
+    H.assert_bf16_close(H.to_np(Y_int[torch.from_numpy(rows).cuda()]), ref, False, "gated interval")
+    # options the run view does not have
+    with pytest.raises(binding.AlgError):
+        f_int.set_option("stage_k", 32)
+    with pytest.raises(binding.AlgError):
+        f_int.set_option("interval_period", 4 * 96)        # runs of 96 rows: no multiple of 64
+    with pytest.raises(binding.AlgError):
+        f_exp.set_option("interval_period", 768)           # not an interval handle
+
+
 def test_gated_kernel_table_shape_q32():
     """One shape of the paper's gated-FFN table: 4096 -> 12288 -> 4096 at q = 32 (group widths 128
     and 384), M = 2048 rows, i.i.d. row types."""
