@@ -113,6 +113,11 @@ typedef enum {
  *                     automatic, 32 (eight stages of 24 KB) or 64 (four stages of 48 KB).  Results
  *                     are identical; only the operand pipeline differs.  A table-driven INTERVAL
  *                     handle reads its runs with 64-deep stages only: 32 is ALG_ERR_UNSUPPORTED_SHAPE there.
+ *   ROW_GATHER        explicit row types on the one-CTA GEMM kernel: how the rows of a type reach the kernel.
+ *                     1 = a copy pass writes the type-bucketed copy of X into the workspace; 2 = the kernel's
+ *                     producer warps fetch the rows through the permutation themselves (four rows per copy
+ *                     instruction, X read in place, one launch fewer); 0 (default) = 1, which measures faster or
+ *                     equal on every benchmark step.  Results are identical.  Ignored by the other kernels.
  *   INTERVAL_PERIOD   INTERVAL schedule of a table-driven handle: the typing repeats every P rows, type of
  *                     row b = (b mod P) / (P / q) -- the pilot model's schedule
  *                     floor((p mod 768) / 192) over a batch of sequences.  0 (default) = one period,
@@ -136,7 +141,8 @@ typedef enum {
   ALG_OPT_WAIT_LIMIT_CYCLES = 5,
   ALG_OPT_TEST_STALL_BYTES = 6,
   ALG_OPT_STAGE_K = 7,
-  ALG_OPT_INTERVAL_PERIOD = 8
+  ALG_OPT_INTERVAL_PERIOD = 8,
+  ALG_OPT_ROW_GATHER = 9
 } alg_option_t;
 
 /* ---- projection handle ---------------------------------------------------------------------

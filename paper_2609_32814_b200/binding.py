@@ -23,7 +23,7 @@ ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
 ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC, ALG_SCHED_INTERVAL = 0, 1, 2
 ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
 OPTIONS = {"gemm_kernel": 1, "tile_n": 2, "small_m_kernel": 3, "host_plan": 4, "wait_limit_cycles": 5,
-           "test_stall_bytes": 6, "stage_k": 7, "interval_period": 8}
+           "test_stall_bytes": 6, "stage_k": 7, "interval_period": 8, "row_gather": 9}
 
 _DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
 _TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM, "q2pow": ALG_TABLE_Q2POW}

@@ -67,6 +67,7 @@ struct alg_proj_s {
   DecodePlan decode = {};
   // options (alg_proj_set_option)
   int opt_kernel = 0, opt_tile_n = 0, opt_stage_k = 0;
+  int opt_row_gather = 0;        // explicit types: 0 / 1 copy pass, 2 rows fetched by the GEMM's producer warps
   int64_t interval_period = 0;   // INTERVAL schedule of a table-driven handle: period of the typing (0 = the whole batch)
   bool opt_small_m = true, opt_host_plan = true;
   long long wait_limit = kDefaultWaitLimit;
@@ -628,6 +629,15 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     if (x_bucketed || cyclic) {
       a.X = X;
       a.ldx = ldx;
+    } else if (p.opt_row_gather == 2 && !p.pair_kernel && !p.w_kmajor && !p.dyn_segments && block_k_of(p) == 64) {
+      // explicit types: the producer warps of the one-CTA kernel fetch the rows of a tile through the permutation,
+      // four per copy instruction; X is read in place and no bucketed copy is written.  An option, not the
+      // default: the copy engine needs longer for gathered rows than for a box (reductions of 1024..2048 columns:
+      // 10 % slower), and where short reductions hide that (256 columns: a projection alone gains 10-13 % on
+      // L2-resident rows) the FFN step with its working set rotating through HBM measures even or 1-2 % slower
+      a.X = X;
+      a.ldx = ldx;
+      a.in_perm = (const int *)(ws + L.perm);
     } else {
       // explicit types: one pass writes the type-bucketed copy of X the tiled loads then read.  (Having
       // the GEMM's producer warps fetch the rows through the permutation themselves, with 16-byte
@@ -834,6 +844,10 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
       if (value == 32 && p.sched == ALG_SCHED_INTERVAL && !no_table) return ALG_ERR_UNSUPPORTED_SHAPE;  // runs: 64-deep only
       p.opt_stage_k = (int)value;
       for (PlanSlot &sl : p.plan) sl.M = -1;  // cached plans count K blocks of the old depth
+      return ALG_OK;
+    case ALG_OPT_ROW_GATHER:
+      if (value < 0 || value > 2) return ALG_ERR_INVALID_ARG;
+      p.opt_row_gather = (int)value;
       return ALG_OK;
     case ALG_OPT_INTERVAL_PERIOD:
       if (value < 0 || value > (1 << 30)) return ALG_ERR_INVALID_ARG;

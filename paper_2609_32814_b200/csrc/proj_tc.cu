@@ -117,8 +117,10 @@ struct Cfg {
 // N = 256 MMA fills both halves of the accumulator, and the epilogue writes silu(gate) * up -- 128
 // output columns per tile, the hidden state is stored once and the two pre-activations never
 // leave the chip (the merged gate/up kernel of the appendix "Kernel Benchmark Details").
-template <int TILE_N, int TILE_M, bool GATED, int BK, bool RUNS>
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int kGatherWarps = 6;   // AMODE 2: extra warps that only issue row gathers, after the B producer
+constexpr int kGatherLanes = 32 / (2 + kGatherWarps);   // lanes of a warp that issue gathers
+template <int TILE_N, int TILE_M, bool GATED, int BK, int AMODE>
+__global__ void __launch_bounds__(AMODE == 2 ? kThreads + 32 * kGatherWarps : kThreads, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a) {
   using C = Cfg<TILE_N, TILE_M, BK>;
   static_assert(!GATED || (TILE_N == 256 && TILE_M == 128), "the gated kernel pairs two 128-column halves");
@@ -218,7 +220,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // of a 128x256x64 block -- against ~290 cycles when the operands live in uniform registers.
   // Loop bounds read from shared memory are broadcast with a shuffle so that they count as
   // warp-uniform.
-  if (warp == 0 || warp == kProducerWarpB) {
+  if (warp == 0 || (AMODE == 2 ? warp >= kProducerWarpB : warp == kProducerWarpB)) {
     // ---------------- TMA producers: warp 0 loads A, the last warp loads B ----------------
     // Issuing a tiled load occupies the thread while the copy engine expands the box; with two
     // issuing warps a freed stage is refilled sooner, which shortens the
@@ -239,6 +241,20 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t mask = __shfl_sync(0xffffffffu, ctl->keep[pair], 0);
       const int type_i = pair / q;
       const int a_row = a.a_cyclic_rows ? row0 - type_i * a.a_cyclic_rows : row0;
+      // explicit types without a bucketed copy: a lane fetches four consecutive bucketed rows (and the same 128
+      // rows further for 256-row tiles) through the permutation; rows past the batch repeat its last row, they
+      // belong to no tile row that is stored
+      // Issuing a gather costs its thread ~56 cycles and the lanes of a warp issue one after the other, so the 32
+      // gathers of a 128-row stage are split between four warps (the two producers and two warps that do nothing
+      // else): eight lanes each, warp w of the four takes rows 32 w .. 32 w + 31.
+      int g_rows[TILE_M / 128][4];
+      const int g_slot = (loads_a ? 0 : warp - kProducerWarpB + 1) * kGatherLanes + (lane & (kGatherLanes - 1));
+      if (AMODE == 2) {
+#pragma unroll
+        for (int h = 0; h < TILE_M / 128; ++h)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) g_rows[h][j] = __ldg(a.in_perm + min(row0 + h * 128 + g_slot * 4 + j, a.M - 1));
+      }
       for (int k = 0; k < q && ok; ++k) {
         if (!((mask >> k) & 1u)) continue;
         const int k_begin = __shfl_sync(0xffffffffu, ctl->so[k], 0);
@@ -248,7 +264,32 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!ok) break;
           const uint32_t bar = full0 + 8u * (uint32_t)stage;
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
-          if (elect_one()) {
+          if (AMODE == 2) {
+            if (elect_one()) {
+              if (loads_a) {
+                mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
+              } else if (warp != kProducerWarpB) {
+                // a gather-only warp
+              } else if (GATED) {
+                tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
+                tma_load_3d(sa + C::kABytes + 2 * C::kBChunkBytes, &tmB, bar, 0, k0, (a.gated_f + n0) >> 6);
+              } else if (a.b_3d) {
+                tma_load_3d(sa + C::kABytes, &tmB, bar, 0, k0, n0 >> 6);
+              } else {
+#pragma unroll
+                for (int c = 0; c < TILE_N / 64; ++c)
+                  tma_load_2d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, n0 + c * 64, k0);
+              }
+            }
+            __syncwarp();
+            // one four-row gather per lane (and per 128 rows): 512 bytes each, 128-byte rows swizzled like a box
+            if (lane < kGatherLanes) {
+#pragma unroll
+              for (int h = 0; h < TILE_M / 128; ++h)
+                tma_gather4(sa + (uint32_t)(h * 128 * BK * 2 + g_slot * 4 * BK * 2), &tmA, bar, k0, g_rows[h][0], g_rows[h][1],
+                            g_rows[h][2], g_rows[h][3]);
+            }
+          } else if (elect_one()) {
             if (a.seg_rows) {
               // weight gradient, cyclic schedule: rows k, k + q, ... of X (A, features contiguous) and of G (B),
               // 64 of them from position k0 - so[k] on, in boxes of 64 features / 64 output columns
@@ -262,7 +303,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int c = 0; c < TILE_N / 64; ++c)
                   tma_load_3d(sa + C::kABytes + c * C::kBChunkBytes, &tmB, bar, n0 + c * 64, k, pos0);
               }
-            } else if (RUNS && loads_a && a.a_cyclic_rows) {
+            } else if (AMODE == 1 && loads_a && a.a_cyclic_rows) {
               // runs of run_rows rows per period: 64-row boxes, each inside one run
               mbar_expect_tx(bar, (uint32_t)C::kStageBytes);
 #pragma unroll
@@ -372,7 +413,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // accumulated, its result is zero
       const bool empty_tile = ((uint32_t)rec.rows >> 16) == 0u;
       if (r < tile_rows) {
-        if (RUNS && a.out_cyclic_rows) {
+        if (AMODE == 1 && a.out_cyclic_rows) {
           const int i = (rec.pair & 0xFFFF) / q;
           const int bt = rec.row0 + r - i * a.out_cyclic_rows, per = bt / a.run_rows;
           out_row = (int64_t)per * a.run_period + i * a.run_rows + (bt - per * a.run_rows);
@@ -504,12 +545,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
-template <int TILE_N, int TILE_M, bool GATED, int BK, bool RUNS = false>
+template <int TILE_N, int TILE_M, bool GATED, int BK, int AMODE = 0>
 cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   using C = Cfg<TILE_N, TILE_M, BK>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED, BK, RUNS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TILE_N, TILE_M, GATED, BK, AMODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -553,7 +594,7 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   if (b.y_staged) smem_bytes += kEpiWarps * C::kStoreBufBytes;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(num_sms, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3(AMODE == 2 ? kThreads + 32 * kGatherWarps : kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
@@ -561,7 +602,7 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED, BK, RUNS>, tmA, tmB, b);
+  e = cudaLaunchKernelEx(&cfg, proj_tc_kernel<TILE_N, TILE_M, GATED, BK, AMODE>, tmA, tmB, b);
   count_launch(1);
   return e;
 }
@@ -569,7 +610,9 @@ cudaError_t launch_bk(const ProjArgs &a, int num_sms, cudaStream_t st) {
 template <int TILE_N, int TILE_M, bool GATED = false>
 cudaError_t launch_t(const ProjArgs &a, int num_sms, cudaStream_t st) {
   // the in-place view of an interval schedule (runs of a type) is a kernel variant of its own, 64-deep stages only
-  if (a.run_rows) return a.block_k == 64 ? launch_bk<TILE_N, TILE_M, GATED, 64, true>(a, num_sms, st) : cudaErrorInvalidValue;
+  if (a.run_rows) return a.block_k == 64 ? launch_bk<TILE_N, TILE_M, GATED, 64, 1>(a, num_sms, st) : cudaErrorInvalidValue;
+  // so are the rows of explicit types fetched through the permutation by the A producer
+  if (a.in_perm) return a.block_k == 64 && !a.w_kmajor && !a.seg_rows ? launch_bk<TILE_N, TILE_M, GATED, 64, 2>(a, num_sms, st) : cudaErrorInvalidValue;
   if (a.block_k == 32) return launch_bk<TILE_N, TILE_M, GATED, 32>(a, num_sms, st);
   if (a.block_k == 64) return launch_bk<TILE_N, TILE_M, GATED, 64>(a, num_sms, st);
   return cudaErrorInvalidValue;
@@ -645,6 +688,8 @@ cudaError_t make_map_b3d(CUtensorMap *map, const ProjArgs &a, int chunks) {
 
 cudaError_t make_map_a(CUtensorMap *map, const ProjArgs &a) {
   const uint32_t box_rows = a.geom.tile_m == 256 && a.a_box_256 ? 256u : 128u;
+  if (a.in_perm)   // rows fetched four at a time through the permutation: boxes of one row
+    return make_map_2d_sw(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, (uint32_t)a.block_k, 1, a.block_k * 2);
   if (!a.a_cyclic_rows)
     return make_map_2d_sw(map, a.X, (uint64_t)a.K, (uint64_t)a.M, (uint64_t)a.ldx * 2, (uint32_t)a.block_k, box_rows,
                           a.block_k * 2);

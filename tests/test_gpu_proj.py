@@ -380,3 +380,31 @@ def test_gelu_epilogue_accuracy_on_a_dense_grid():
     assert err.max() <= 4e-7 + 2e-7 * np.abs(ref).max(), err.max()
     Yt = proj.forward(H.to_dev(X, "bf16"), t, W, act="gelu_tanh", out_dtype=torch.float32)
     assert np.abs(H.to_np(Yt) - ref).max() <= 2e-3      # the tanh form is a different function
+
+
+@pytest.mark.parametrize("q,M,dw,fw,kernel", [
+    (2, 128, 128, 128, 1),       # one tile
+    (4, 5000, 128, 512, 1),      # short reductions: the library's own choice is the in-kernel gather
+    (3, 777, 256, 384, 1),       # ragged buckets, 192-column tiles
+    (2, 4096, 384, 1536, 1),     # reductions of 384 and 768 columns
+    (2, 8192, 384, 384, 3),      # 256-row tiles: two gathers per lane and stage
+])
+def test_row_gather_in_the_kernel_matches_the_copy_pass(q, M, dw, fw, kernel):
+    """Explicit types, option ROW_GATHER: rows fetched through the permutation by the GEMM's producer warps (four rows
+    per copy instruction) against the bucketed copy -- same bits, one launch fewer, integers exact against the oracle."""
+    types = synth.uniform_types(900 + q, M, q)
+    wl = synth.make_workload("rowg", config=7, variant=q * 10 + kernel, dtype="bf16", q=q, M=M, D=q * dw, F=q * fw,
+                             types=types, integer=True, d_widths=[dw] * q, f_widths=[fw] * q)
+    X, W, t = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16"), H.dev_types(types)
+    out, launches = [], []
+    for mode in (1, 2):
+        proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+        proj.set_option("gemm_kernel", kernel)
+        proj.set_option("row_gather", mode)
+        n0 = binding.launch_count()
+        out.append(proj.forward(X, t, W, out_dtype=torch.float32))
+        launches.append(binding.launch_count() - n0)
+        assert proj.last_status() == 0
+    assert torch.equal(out[0], out[1])
+    assert launches[0] == launches[1] + 1
+    assert np.array_equal(H.to_np(out[1]), oracle.proj(wl.X, types, wl.W_up, wl.d_widths, wl.f_widths))
