@@ -167,8 +167,12 @@ alg_status_t configure_kernels(alg_proj_s &p) {
     min_klen = std::min(min_klen, len);
   }
   p.pair_kernel = p.tc_ok && all128 && min_klen >= 4096;
-  if (p.gated) {   // 128 output columns per tile (the MMA is 256 wide: gate and up halves)
-    if (!(p.tc_ok && all128)) return ALG_ERR_UNSUPPORTED_SHAPE;
+  if (p.gated && !(p.tc_ok && all128)) {
+    // hidden groups off the 128-column grid: only the large-algebra kernel has a gated form for them (the caller
+    // checks that the handle fits it)
+    p.tc_ok = false;
+    p.pair_kernel = false;
+  } else if (p.gated) {   // 128 output columns per tile (the MMA is 256 wide: gate and up halves)
     if (p.opt_kernel > 1 || (p.opt_tile_n != 0 && p.opt_tile_n != 128)) return ALG_ERR_UNSUPPORTED_SHAPE;
     p.tile_n = 128;
     p.pair_kernel = false;
@@ -304,6 +308,7 @@ alg_status_t init_proj(alg_proj_s &p, int q, const int32_t *in_w, const int32_t 
   alg_status_t cs = configure_kernels(p);
   if (cs != ALG_OK) return cs;
   if (sched == ALG_SCHED_INTERVAL && !use_tc(p)) return ALG_ERR_UNSUPPORTED_SHAPE;
+  if (gated && !p.tc_ok && !(big_fits && in_w[0] % 8 == 0 && out_w[0] % 8 == 0)) return ALG_ERR_UNSUPPORTED_SHAPE;
   if (big_fits) {
     plan_big(p, in_w[0], out_w[0]);
     p.big.eligible = true;

@@ -134,9 +134,31 @@ def test_gated_kernel_table_shape_q32():
     assert H.max_abs(got, ref) <= H.BF16_MAX_ABS
 
 
+@pytest.mark.parametrize("q,M,dw,fw", [
+    (32, 300, 64, 192),      # 2048 -> 6144 at q = 32: hidden groups of 192 columns, two 96-column tiles each
+    (32, 257, 80, 304),      # 2560 -> 9728: groups of 80 and 304 (reductions of 80 and 304 are no multiples of 64)
+    (32, 2048, 64, 24),      # 2048 -> 768 (an expert): hidden groups of 24 columns
+    (32, 333, 224, 64),      # 7168 -> 2048 (an expert)
+    (4, 1000, 64, 192),      # the same group widths at small q: several m-tiles per type
+    (3, 515, 80, 304),
+    (1, 1, 64, 24),          # one row
+])
+@pytest.mark.parametrize("schedule", ["explicit", "cyclic"])
+def test_gated_ffn_groups_off_the_tile_grid(q, M, dw, fw, schedule):
+    """Gated FFN whose groups are no multiples of 128 columns (the public model shapes of the paper's gated-FFN table
+    split 32 ways): both projections on the large-algebra kernel, hidden state in bucketed order."""
+    types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(700 + q + M, M, q)
+    wl, Wg = synth.gated_ffn("gated-off-grid", q, M, q * dw, q * fw, types, variant=q + dw + fw)
+    wl.W_up, Wg, wl.W_down = (synth.bf16_round(w * 2.0) for w in (wl.W_up, Wg, wl.W_down))
+    Y, ffn = _run(wl, Wg, schedule=schedule, out_dtype=torch.bfloat16)
+    rows = np.unique(np.concatenate([_sample_rows(wl, 6, seed=3), np.arange(min(M, 8))])) if M > 64 else np.arange(M)
+    ref = oracle.ffn_swiglu(wl.X[rows], wl.types[rows], Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, True, f"gated off-grid q={q} M={M}")
+
+
 def test_gated_refusals():
     with pytest.raises(binding.AlgError) as e:
-        binding.GatedFFN([64, 64], [192, 192], dtype="bf16")      # hidden groups are no multiples of 128
+        binding.GatedFFN([64, 128], [192, 320], dtype="bf16")     # hidden groups off the 128-column grid and unequal
     assert e.value.code == 2
     with pytest.raises(binding.AlgError):
         binding.GatedFFN([64, 64], [128, 128], dtype="f32")
