@@ -86,6 +86,7 @@ struct alg_ffn_s {
   // decode step of the whole FFN in one launch (M <= kFfnDecodeMaxM)
   bool gated = false;        // SwiGLU: up = merged gate/up projection with silu(gate) * up epilogue
   bool fd_ok = false;
+  bool gd_ok = false;        // gated decode step (M <= kGatedDecodeMaxM) in one launch
   FfnDecodePlan fd = {};
   unsigned int *d_counters = nullptr;
 };
@@ -1288,6 +1289,11 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
     f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
+  if (gated && schedule != ALG_SCHED_INTERVAL && f->up.big.eligible && f->down.big.eligible &&
+      gated_decode_fits(q, f->D, f->F)) {
+    f->gd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
+               cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
+  }
   *out = f;
   return ALG_OK;
 }
@@ -1371,6 +1377,24 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
       for (int e = 0; e < u.q * u.q; ++e) d.keep[e] = u.tab.keep[e];
     }
     return cuda_status(launch_ffn_decode(d, h->fd, st));
+  }
+  if (h->gd_ok && h->up.opt_small_m && M <= kGatedDecodeMaxM && !h->timing) {
+    // gated decode step of one row in one launch
+    if (b_up || b_down || act != ALG_ACT_NONE) return ALG_ERR_INVALID_ARG;
+    GatedDecodeArgs d = {};
+    d.X = X;
+    d.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;
+    d.M = (int)M;
+    d.W_gate_up = W_up, d.ldw_up = 2 * (int64_t)h->F;
+    d.W_down = W_down, d.ldw_dn = h->D;
+    d.H = ws + L.h;
+    d.Y = Y;
+    d.y_bf16 = y_dtype == ALG_BF16;
+    d.D = h->D, d.F = h->F, d.q = h->up.q;
+    d.counters = h->d_counters;
+    d.status = h->up.d_status;
+    d.wait_limit = h->up.wait_limit;
+    return cuda_status(launch_gated_decode(d, h->up.num_sms, st));
   }
   if (use_decode(h->up, M) && use_decode(h->down, M)) {
     // decode shapes: no bucketing, H stays in the original row order

@@ -187,8 +187,8 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
   __syncthreads();
   if (!s_go) return;
   if (tid == 0 && atomicAdd(a.sync + 1, 1u) == (unsigned)(n_chunks - 1)) a.sync[0] = 0u, a.sync[1] = 0u;
-  if (warp < 2) {   // lanes over the chunks (at most 64), one type after the other
-    for (int ty = warp; ty < nt; ty += 2) {
+  {   // lanes over the chunks (at most 64); the warps share the types, so that their round trips to L2 overlap
+    for (int ty = warp; ty < nt; ty += kFusedThreads / 32) {
       int before = 0, total = 0;
       for (int c = lane; c < n_chunks; c += 32) {
         const int v = __ldcg(a.chunk_counts + c * nt + ty);

@@ -307,6 +307,30 @@ struct FfnDecodeArgs {
 bool ffn_decode_plan(int q, const int *dw, const int *fw, int D, int F, int num_sms, FfnDecodePlan *plan);
 cudaError_t launch_ffn_decode(const FfnDecodeArgs &a, const FfnDecodePlan &plan, cudaStream_t st);
 
+// Decode step of one row of the gated FFN (complete-graph law, equal groups) in one launch (gated_decode.cu).
+constexpr int kGatedDecodeMaxM = 1;
+struct GatedDecodeArgs {
+  const void *X;            // [D] bf16
+  const int32_t *types;     // the row's type; nullptr => type 0 (row 0 of the cyclic schedule)
+  int M;                    // 1
+  const void *W_gate_up;    // [D][ldw_up] bf16: the merged bank [W_gate | W_up], 2 F columns
+  int64_t ldw_up;
+  const void *W_down;       // [F][ldw_dn] bf16
+  int64_t ldw_dn;
+  void *H;                  // [F] bf16 scratch in global memory, 16-byte aligned
+  void *Y;                  // [D]
+  int y_bf16;
+  int D, F, q;
+  int pc_up, pc_dn;         // columns of a warp's piece (8 or 16)                 (set by the launcher)
+  int ks_up, ks_dn;         // warps sharing the weight rows of a piece            (set by the launcher)
+  int units_up, units_dn;   // pieces x sharing warps                              (set by the launcher)
+  unsigned int *counters;   // [0] CTAs that finished phase 1, [1] CTAs past the wait; zero between launches
+  int *status;
+  long long wait_limit;
+};
+bool gated_decode_fits(int q, int D, int F);
+cudaError_t launch_gated_decode(const GatedDecodeArgs &a, int num_sms, cudaStream_t st);
+
 void count_launch(int n = 1);
 int handle_device(alg_proj_t h);  // device the handle was created on (-1 for a null handle)
 

@@ -1,0 +1,337 @@
+// Decode step of ONE row (M = 1) of the gated FFN  y = (silu(x * W_gate) .* (x * W_up)) * W_down  under the
+// complete-graph law with q equal groups, in ONE launch (the M = 1 rows of the paper's gated-FFN table, appendix
+// "Kernel Benchmark Details").
+//
+// A row of type i needs, for the output group j, the block W_ij of its row panel and the diagonal block W_jj
+// (Eqs. typed-diag / typed-off): 2 s of the q s weight rows above every output column.  The step is a pair of
+// matrix-vector products bound by memory LATENCY, so it runs on plain FMAs and is organised around the dependent
+// round trips.  A warp owns a piece of 8 or 16 output columns (and, while there are more warps than pieces, a
+// share of the weight rows); its lanes split the rows, every lane keeps up to 32 loads of 16 bytes in flight and
+// reads the activations it needs straight from global memory -- no staging, one CTA barrier per phase at most.
+// The first loads of W_gate_up are issued before the launch's dependency resolves (weights do not depend on the
+// previous kernel), those of W_down before the wait between the phases.  Phase 1 writes the hidden row h (bf16) to
+// global memory; all CTAs meet at a counter (bounded wait); phase 2 is the same routine on h and W_down.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+
+#include "common.cuh"
+#include "trace.cuh"
+
+namespace algproj {
+ALG_TRACE_DEFINE(gated_decode)
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kLoads = 32;   // 16-byte weight loads a lane keeps in flight
+
+// One matrix-vector phase as the kernel sees it.
+struct Phase {
+  const __nv_bfloat16 *W;   // weight bank, `ldw` elements per row
+  int64_t ldw;
+  int s;                    // rows of one input group
+  int group_w;              // columns of one output group
+  int n_cols;               // output columns (GATED: the up columns sit n_cols further in the bank)
+  int pc;                   // columns of a piece: 8 or 16
+  int ks;                   // warps that share the rows of a piece: 1, 2, 4 or 8
+};
+
+__device__ __forceinline__ void unpack8(const uint4 &v, float *f) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    f[2 * e] = __uint_as_float(w[e] << 16);
+    f[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+  }
+}
+
+// Where a lane stands in a piece: `sub` = which 8 columns, `lr` = which share of the rows.
+struct Lane {
+  int piece, part, sub, lr, rl, col, j;
+  bool on;
+};
+__device__ __forceinline__ Lane lane_of(const Phase &p, int unit) {
+  Lane l;
+  const int lane = threadIdx.x & 31, po = p.pc >> 3;
+  l.piece = unit / p.ks, l.part = unit - l.piece * p.ks;
+  l.sub = lane & (po - 1), l.lr = lane / po, l.rl = 32 / po;
+  l.col = l.piece * p.pc + 8 * l.sub;
+  l.on = l.col < p.n_cols;
+  l.j = l.on ? l.col / p.group_w : 0;
+  return l;
+}
+
+// Loads of one chunk: rows r0 .. of both segments (the diagonal block of group j, then -- unless the row's own type is
+// j -- its panel block), for the gate and, GATED, the up columns.  RC rows per segment and chunk.
+template <bool GATED>
+__device__ __forceinline__ void load_chunk(uint4 (&w)[kLoads], const Phase &p, const Lane &l, int type, int c0) {
+  constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
+  const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
+#pragma unroll
+  for (int sg = 0; sg < 2; ++sg) {
+    const int g = sg == 0 ? l.j : type;
+    const bool seg_on = l.on && (sg == 0 || type != l.j);
+    const __nv_bfloat16 *base = p.W + (int64_t)g * p.s * p.ldw + l.col;
+#pragma unroll
+    for (int u = 0; u < RC; ++u) {
+      const int kk = first + (c0 + u) * step;
+      const bool ok = seg_on && kk < p.s;
+      const __nv_bfloat16 *src = base + (int64_t)kk * p.ldw;
+      w[(sg * RC + u) * (GATED ? 2 : 1)] = ok ? __ldg((const uint4 *)src) : make_uint4(0, 0, 0, 0);
+      if (GATED) w[(sg * RC + u) * 2 + 1] = ok ? __ldg((const uint4 *)(src + p.n_cols)) : make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+// acc[0..8) (gate or plain) and acc[8..16) (up) += x[kk] * w[kk][...] for one chunk.  x is read from global memory
+// (FROM_L2: written by other CTAs of this launch).
+template <bool GATED, bool FROM_L2>
+__device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase &p, const Lane &l, int type, int c0,
+                                          const __nv_bfloat16 *x, float (&acc)[16]) {
+  constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
+  const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
+  float xv[2 * RC];
+#pragma unroll
+  for (int sg = 0; sg < 2; ++sg) {
+    const int g = sg == 0 ? l.j : type;
+    const bool seg_on = l.on && (sg == 0 || type != l.j);
+#pragma unroll
+    for (int u = 0; u < RC; ++u) {
+      const int kk = first + (c0 + u) * step;
+      unsigned short raw = 0;
+      if (seg_on && kk < p.s) {
+        const unsigned short *src = (const unsigned short *)(x + (int64_t)g * p.s + kk);
+        raw = FROM_L2 ? __ldcg(src) : __ldg(src);
+      }
+      xv[sg * RC + u] = __uint_as_float((uint32_t)raw << 16);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 2 * RC; ++e) {
+    float f[8];
+    unpack8(w[e * (GATED ? 2 : 1)], f);
+#pragma unroll
+    for (int cc = 0; cc < 8; ++cc) acc[cc] = fmaf(xv[e], f[cc], acc[cc]);
+    if (GATED) {
+      unpack8(w[e * 2 + 1], f);
+#pragma unroll
+      for (int cc = 0; cc < 8; ++cc) acc[8 + cc] = fmaf(xv[e], f[cc], acc[8 + cc]);
+    }
+  }
+}
+
+// One phase for the units of this warp.  `w` holds the first chunk of the first unit when have_first.  Results of a
+// piece: lanes with lr == 0 of the warp with part == 0 call `emit(col, acc)`.
+template <bool GATED, bool FROM_L2, typename Emit>
+__device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_bfloat16 *x, uint4 (&w)[kLoads], bool have_first,
+                                          int n_units, float *partial, Emit emit) {
+  constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_warps = gridDim.x * kWarps, po = p.pc >> 3;
+  const int rounds = (n_units + total_warps - 1) / total_warps;
+  for (int rd = 0; rd < rounds; ++rd) {
+    const int unit = rd * total_warps + blockIdx.x * kWarps + warp;
+    Lane l = lane_of(p, unit);
+    if (unit >= n_units) l.on = false;
+    float acc[16];
+#pragma unroll
+    for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
+    const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
+    for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
+      if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, type, c0);
+      fma_chunk<GATED, FROM_L2>(w, p, l, type, c0, x, acc);
+    }
+    // sum over the lanes that share the columns
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      if (d >= po) {
+#pragma unroll
+        for (int cc = 0; cc < (GATED ? 16 : 8); ++cc) acc[cc] += __shfl_xor_sync(0xffffffffu, acc[cc], d);
+      }
+    }
+    if (p.ks > 1) {   // the warps of a piece sit in one CTA
+      if (lane < po) {
+#pragma unroll
+        for (int cc = 0; cc < 16; ++cc) partial[(warp * 2 + lane) * 16 + cc] = acc[cc];
+      }
+      __syncthreads();
+      if (l.part == 0 && lane < po) {
+        for (int o = 1; o < p.ks; ++o)
+#pragma unroll
+          for (int cc = 0; cc < 16; ++cc) acc[cc] += partial[((warp + o) * 2 + lane) * 16 + cc];
+      }
+      __syncthreads();
+    }
+    if (l.on && l.part == 0 && lane < po) emit(l.col, acc);
+  }
+}
+
+__device__ __forceinline__ int read_type(const GatedDecodeArgs &a) {
+  const int t = a.types ? a.types[0] : 0;
+  return t < 0 || t >= a.q ? -1 : t;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gated_decode_kernel(const GatedDecodeArgs a) {
+  __shared__ float partial[kWarps * 2 * 16];
+  __shared__ int s_abort;
+  ALG_TRACE_VARS;
+  if (threadIdx.x == 0) ALG_TRACE(0, 1);
+  Phase up, dn;
+  up.W = (const __nv_bfloat16 *)a.W_gate_up, up.ldw = a.ldw_up, up.s = a.D / a.q, up.group_w = a.F / a.q, up.n_cols = a.F;
+  up.pc = a.pc_up, up.ks = a.ks_up;
+  dn.W = (const __nv_bfloat16 *)a.W_down, dn.ldw = a.ldw_dn, dn.s = a.F / a.q, dn.group_w = a.D / a.q, dn.n_cols = a.D;
+  dn.pc = a.pc_dn, dn.ks = a.ks_dn;
+  const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
+  __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
+  const int warp = threadIdx.x >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == 0) s_abort = 0;
+
+  // ---- before the dependency resolves: the row type as it stands now and the first W_gate_up loads it asks for
+  // (the type is read again after the wait) ----
+  const int t_early = read_type(a);
+  uint4 w[kLoads];
+  {
+    const int unit = blockIdx.x * kWarps + warp;
+    Lane l = lane_of(up, unit);
+    if (unit >= a.units_up || t_early < 0) l.on = false;
+    load_chunk<true>(w, up, l, max(t_early, 0), 0);
+  }
+  if (threadIdx.x == 0) ALG_TRACE(0, 2);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) ALG_TRACE(0, 3);
+  const int type = read_type(a);   // (in flight while phase 1 runs on the early value)
+
+  // ---- phase 1: h = silu(x * W_gate) .* (x * W_up); on the type read early, again if the type has changed since ----
+  for (int pass = 0; pass < 2; ++pass) {
+    const int t = pass == 0 ? t_early : type;
+    if (pass == 1 && type == t_early) break;
+    if (t < 0) continue;
+    run_phase<true, false>(up, t, X, w, pass == 0, a.units_up, partial, [&](int col, const float (&acc)[16]) {
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float g0 = acc[2 * e], g1 = acc[2 * e + 1];
+        __nv_bfloat162 pk = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * acc[8 + 2 * e], g1 / (1.f + __expf(-g1)) * acc[8 + 2 * e + 1]);
+        o[e] = *(uint32_t *)&pk;
+      }
+      *(uint4 *)(H + col) = make_uint4(o[0], o[1], o[2], o[3]);
+    });
+  }
+  if (type < 0 && threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);   // y = 0
+  if (threadIdx.x == 0) ALG_TRACE(0, 6);
+
+  // ---- the first W_down loads go out before the wait between the phases ----
+  {
+    const int unit = blockIdx.x * kWarps + warp;
+    Lane l = lane_of(dn, unit);
+    if (unit >= a.units_dn || type < 0) l.on = false;
+    load_chunk<false>(w, dn, l, max(type, 0), 0);
+  }
+
+  // ---- all of h is written before any of it is read: arrive, then wait (bounded) for the other CTAs ----
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ALG_TRACE(0, 8);
+    __threadfence();
+    atomicAdd(a.counters, 1u);
+    const long long t0 = clock64();
+    bool ok = false;
+    while (!ok) {
+      unsigned int seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters) : "memory");
+      ok = seen >= gridDim.x;
+      if (!ok && clock64() - t0 > a.wait_limit) break;
+    }
+    if (!ok) {
+      s_abort = 1;
+      atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+    }
+    __threadfence();
+    ALG_TRACE(0, 9);
+  }
+  __syncthreads();
+
+  // ---- phase 2: y = h * W_down ----
+  if (!s_abort) {
+    if (type >= 0) {
+      run_phase<false, true>(dn, type, H, w, true, a.units_dn, partial, [&](int col, const float (&acc)[16]) {
+        if (a.y_bf16) {
+          uint32_t o[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 pk = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+            o[e] = *(uint32_t *)&pk;
+          }
+          *(uint4 *)((__nv_bfloat16 *)a.Y + col) = make_uint4(o[0], o[1], o[2], o[3]);
+        } else {
+          float4 *dst = (float4 *)((float *)a.Y + col);
+          dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+          dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        }
+      });
+    } else {   // a row type outside [0, q): the row of Y is zero
+      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.D; c += gridDim.x * kThreads) {
+        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
+        else ((float *)a.Y)[c] = 0.f;
+      }
+    }
+  }
+  // the last CTA past the wait clears the counters for the next launch
+  if (threadIdx.x == 0) {
+    ALG_TRACE(0, 12);
+    const unsigned int left = atomicAdd(a.counters + 1, 1u);
+    if (left == gridDim.x - 1) {
+      a.counters[0] = 0;
+      a.counters[1] = 0;
+      __threadfence();
+    }
+  }
+}
+
+// warps per piece: as many (a power of two, at most the warps of a CTA) as the grid has warps for
+int pick_ks(int pieces, int grid) {
+  int ks = 1;
+  while (ks < kWarps && pieces * ks * 2 <= grid * kWarps) ks *= 2;
+  return ks;
+}
+
+}  // namespace
+
+bool gated_decode_fits(int q, int D, int F) {
+  if (q < 1 || D % q || F % q) return false;
+  return (D / q) % 8 == 0 && (F / q) % 8 == 0;
+}
+
+cudaError_t launch_gated_decode(const GatedDecodeArgs &in, int num_sms, cudaStream_t st) {
+  GatedDecodeArgs a = in;
+  if (a.M != 1 || !gated_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
+  const int s = a.D / a.q, r = a.F / a.q;
+  // every CTA must be resident for the wait between the phases: one CTA per SM at most
+  a.pc_up = r % 16 == 0 ? 16 : 8;
+  a.pc_dn = s % 16 == 0 ? 16 : 8;
+  const int pieces_up = a.F / a.pc_up, pieces_dn = a.D / a.pc_dn;
+  a.ks_up = pick_ks(pieces_up, num_sms);
+  a.ks_dn = pick_ks(pieces_dn, num_sms);
+  a.units_up = pieces_up * a.ks_up;
+  a.units_dn = pieces_dn * a.ks_dn;
+  const int grid = std::min(num_sms, (std::max(a.units_up, a.units_dn) + kWarps - 1) / kWarps);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gated_decode_kernel, a);
+  count_launch(1);
+  return e;
+}
+
+}  // namespace algproj

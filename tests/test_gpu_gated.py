@@ -156,6 +156,55 @@ def test_gated_ffn_groups_off_the_tile_grid(q, M, dw, fw, schedule):
     H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, True, f"gated off-grid q={q} M={M}")
 
 
+@pytest.mark.parametrize("q,dw,fw", [
+    (32, 64, 192),       # 2048 -> 6144
+    (32, 80, 304),       # 2560 -> 9728
+    (32, 128, 384),      # 4096 -> 12288
+    (32, 64, 24),        # 2048 -> 768
+    (32, 224, 64),       # 7168 -> 2048
+    (2, 128, 256),       # few wide groups: strips narrower than a group
+    (5, 40, 72),
+])
+@pytest.mark.parametrize("M", [1, 3, 8])
+def test_gated_decode_step_in_one_launch(q, dw, fw, M):
+    """Decode rows of the gated FFN against the oracle.  One row is one launch (two matrix-vector phases around a
+    bounded wait; twice in a row on the same handle: the counters are cleared by the kernel); a few rows go through
+    the prefill kernels.  Types explicit and cyclic."""
+    for schedule in ("explicit", "cyclic"):
+        types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(800 + q + M, M, q)
+        wl, Wg = synth.gated_ffn("gated-decode", q, M, q * dw, q * fw, types, variant=q + dw + M)
+        wl.W_up, Wg, wl.W_down = (synth.bf16_round(w * 2.0) for w in (wl.W_up, Wg, wl.W_down))
+        ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+        Wgu, Wd, X = H.to_dev(np.concatenate([Wg, wl.W_up], axis=1), "bf16"), H.to_dev(wl.W_down, "bf16"), H.to_dev(wl.X, "bf16")
+        t = None if schedule == "cyclic" else H.dev_types(types)
+        ref = oracle.ffn_swiglu(wl.X, wl.types, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+        for out_dtype in (torch.float32, torch.bfloat16):
+            n0 = binding.launch_count()
+            Y = ffn.forward(X, t, Wgu, Wd, out_dtype=out_dtype)
+            assert ffn.last_status() == 0 and (M > 1 or binding.launch_count() - n0 == 1)
+            H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"gated decode q={q} M={M} {schedule}")
+        # the prefill kernels on the same rows agree within the tolerance of two bf16 paths
+        ffn.set_option("small_m_kernel", 0)
+        Y2 = ffn.forward(X, t, Wgu, Wd, out_dtype=torch.float32)
+        H.assert_bf16_close(H.to_np(Y2), ref, False, "prefill kernels on decode rows")
+
+
+def test_gated_decode_row_type_out_of_range_gives_a_zero_row():
+    q, dw, fw = 4, 64, 128
+    wl, Wg = synth.gated_ffn("gated-decode-bad", q, 1, q * dw, q * fw, np.array([0], np.int32), variant=9)
+    ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    Wgu, Wd, X = H.to_dev(np.concatenate([Wg, wl.W_up], axis=1), "bf16"), H.to_dev(wl.W_down, "bf16"), H.to_dev(wl.X, "bf16")
+    for out_dtype in (torch.float32, torch.bfloat16):
+        Y = torch.full((1, q * dw), 3.0, dtype=out_dtype, device="cuda")
+        ffn.forward(X, H.dev_types(np.array([7], np.int32)), Wgu, Wd, out=Y)
+        assert ffn.last_status() == 5
+        assert np.all(H.to_np(Y) == 0)
+    # the handle is usable afterwards
+    Y = ffn.forward(X, H.dev_types(np.array([2], np.int32)), Wgu, Wd, out_dtype=torch.float32)
+    ref = oracle.ffn_swiglu(wl.X, np.array([2], np.int32), Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(Y), ref, False, "after a bad type")
+
+
 def test_gated_refusals():
     with pytest.raises(binding.AlgError) as e:
         binding.GatedFFN([64, 128], [192, 320], dtype="bf16")     # hidden groups off the 128-column grid and unequal
