@@ -646,6 +646,14 @@ def run_prefill(args, ctx):
             extras["paper_h200_us"] = {"M=1": cfg["paper_us"][0], "M=2048": cfg["paper_us"][1],
                                        "note": "the paper's own kernel on its H200 NVL (another machine: context)"}
             extras["decode_m1"] = gated_decode_chain(binding, cfg["q"], D, F)
+            cyc = Handle(wl.d_widths, wl.f_widths, dtype="bf16", table=cfg["law"], schedule="cyclic")
+            time_steps(6, cyc, None)
+            l0 = binding.launch_count()
+            cyc_ms = time_steps(n, cyc, None) / n
+            extras["cyclic_schedule"] = {"ms_per_step": cyc_ms, "launches_per_step": (binding.launch_count() - l0) // n,
+                                         "note": "same shapes and weights with type = position mod q as the handle's schedule: equal "
+                                                 "buckets, rows read and written in place (no bucketing, no gather)"}
+            del cyc
 
     cpu = time_cpu_oracle(name, wl) if rank == 0 else None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -276,10 +276,15 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
  * W_gate_up is the merged bank, D x 2F packed: columns [0, F) are W_gate, columns [F, 2F) are W_up,
  * each split into the q hidden groups f_widths; one kernel accumulates the gate and the up columns
  * of a tile side by side and stores silu(gate) * up, so the two pre-activations never reach memory.
- * W_down is F x D packed.  Create with alg_ffn_gated_create (bf16 only; every d width a multiple
- * of 64 and every f width a multiple of 128, else ALG_ERR_UNSUPPORTED_SHAPE); workspace size,
- * options, MAC count (three projections), status and destruction through the alg_ffn_* calls.
- * Every M runs the prefill kernels (there is no small-M kernel for the gated form yet). */
+ * W_down is F x D packed.  Create with alg_ffn_gated_create (bf16 only).  Shapes: every d width a
+ * multiple of 64 and every f width a multiple of 128 (any table); or, under ALG_TABLE_QQ, equal d
+ * widths and equal f widths that are multiples of 8 (the large-algebra kernel: e.g. 2048 -> 6144 or
+ * 2048 -> 768 split 32 ways); anything else is ALG_ERR_UNSUPPORTED_SHAPE.  Workspace size, options,
+ * MAC count (three projections), status and destruction through the alg_ffn_* calls.
+ * M = 1 under ALG_TABLE_QQ with equal widths is ONE launch (two matrix-vector phases on plain FMAs
+ * around a bounded wait; option SMALL_M_KERNEL = 0 sends it through the prefill kernels instead);
+ * every other M runs the prefill kernels.  With the CYCLIC schedule and q | M the rows are read and
+ * written in place (two launches); otherwise bucketing and the row gather run first. */
 alg_status_t alg_ffn_gated_create(alg_ffn_t *out, int q, const int32_t *d_widths,
                                   const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,
                                   const uint8_t *custom_keep, alg_schedule_t schedule);

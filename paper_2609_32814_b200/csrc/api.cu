@@ -514,7 +514,7 @@ bool use_big_counted(const alg_proj_s &p, int64_t M) {
 // 128.6 -> 71.1 us); with fuller buckets the table-driven kernel is faster (58.6 against 63.2 us on the q = 2
 // FFN at M = 8192).
 bool use_big_equal(const alg_proj_s &p, int64_t M) {
-  if (p.gated || p.big.repack) return false;
+  if (p.big.repack) return false;
   return p.big.on || (p.big.eligible && p.opt_kernel == 0 && M <= 128 * (int64_t)p.q);
 }
 
@@ -541,7 +541,7 @@ alg_status_t run_proj(alg_proj_s &p, const WsLayout &L, char *ws, const void *X,
     g.rows_per_type = (int)(M / p.q);
     g.a_box_rows = (int)std::min<int64_t>(128, (g.rows_per_type + 7) / 8 * 8);
     g.pack = 1;
-    g.gated_f = 0;
+    g.gated_f = p.gated ? p.N : 0;
     g.sched = x_bucketed ? 1 : 2, g.sched_out = y_bucketed ? 1 : 2;
     g.offsets = nullptr, g.perm = nullptr;
     g.status = p.d_status;

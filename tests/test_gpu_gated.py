@@ -137,7 +137,8 @@ def test_gated_kernel_table_shape_q32():
 @pytest.mark.parametrize("q,M,dw,fw", [
     (32, 300, 64, 192),      # 2048 -> 6144 at q = 32: hidden groups of 192 columns, two 96-column tiles each
     (32, 257, 80, 304),      # 2560 -> 9728: groups of 80 and 304 (reductions of 80 and 304 are no multiples of 64)
-    (32, 2048, 64, 24),      # 2048 -> 768 (an expert): hidden groups of 24 columns
+    (32, 2048, 64, 24),      # 2048 -> 768 (an expert): hidden groups of 24 columns; cyclic: two types per tile
+    (32, 32 * 200, 64, 192), # cyclic: 200 rows per type, two m-tiles each
     (32, 333, 224, 64),      # 7168 -> 2048 (an expert)
     (4, 1000, 64, 192),      # the same group widths at small q: several m-tiles per type
     (3, 515, 80, 304),
@@ -150,7 +151,10 @@ def test_gated_ffn_groups_off_the_tile_grid(q, M, dw, fw, schedule):
     types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(700 + q + M, M, q)
     wl, Wg = synth.gated_ffn("gated-off-grid", q, M, q * dw, q * fw, types, variant=q + dw + fw)
     wl.W_up, Wg, wl.W_down = (synth.bf16_round(w * 2.0) for w in (wl.W_up, Wg, wl.W_down))
+    n0 = binding.launch_count()
     Y, ffn = _run(wl, Wg, schedule=schedule, out_dtype=torch.bfloat16)
+    if schedule == "cyclic" and M % q == 0 and M > 1:
+        assert binding.launch_count() - n0 == 2      # equal buckets: rows read and written in place, no bucketing, no gather
     rows = np.unique(np.concatenate([_sample_rows(wl, 6, seed=3), np.arange(min(M, 8))])) if M > 64 else np.arange(M)
     ref = oracle.ffn_swiglu(wl.X[rows], wl.types[rows], Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
     H.assert_bf16_close(H.to_np(Y[torch.from_numpy(rows).cuda()]), ref, True, f"gated off-grid q={q} M={M}")
