@@ -1394,6 +1394,7 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
     d.counters = h->d_counters;
     d.status = h->up.d_status;
     d.wait_limit = h->up.wait_limit;
+    d.extra_arrivals = h->up.test_extra_expect ? 1 : 0;
     return cuda_status(launch_gated_decode(d, h->up.num_sms, st));
   }
   if (use_decode(h->up, M) && use_decode(h->down, M)) {

@@ -327,6 +327,7 @@ struct GatedDecodeArgs {
   unsigned int *counters;   // [0] CTAs that finished phase 1, [1] CTAs past the wait; zero between launches
   int *status;
   long long wait_limit;
+  int extra_arrivals;       // test hook: arrivals the wait between the phases expects beyond the grid's (never come)
 };
 bool gated_decode_fits(int q, int D, int F);
 cudaError_t launch_gated_decode(const GatedDecodeArgs &a, int num_sms, cudaStream_t st);

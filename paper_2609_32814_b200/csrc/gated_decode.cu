@@ -70,6 +70,7 @@ template <bool GATED>
 __device__ __forceinline__ void load_chunk(uint4 (&w)[kLoads], const Phase &p, const Lane &l, int type, int c0) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
+  const int nr = (p.s + step - 1) / step - c0;   // rows of this chunk some lane has (the same in every lane)
 #pragma unroll
   for (int sg = 0; sg < 2; ++sg) {
     const int g = sg == 0 ? l.j : type;
@@ -77,6 +78,7 @@ __device__ __forceinline__ void load_chunk(uint4 (&w)[kLoads], const Phase &p, c
     const __nv_bfloat16 *base = p.W + (int64_t)g * p.s * p.ldw + l.col;
 #pragma unroll
     for (int u = 0; u < RC; ++u) {
+      if (u >= nr) break;
       const int kk = first + (c0 + u) * step;
       const bool ok = seg_on && kk < p.s;
       const __nv_bfloat16 *src = base + (int64_t)kk * p.ldw;
@@ -93,6 +95,7 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
                                           const __nv_bfloat16 *x, float (&acc)[16]) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
+  const int nr = (p.s + step - 1) / step - c0;   // rows of this chunk some lane has (the same in every lane)
   float xv[2 * RC];
 #pragma unroll
   for (int sg = 0; sg < 2; ++sg) {
@@ -100,6 +103,7 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
     const bool seg_on = l.on && (sg == 0 || type != l.j);
 #pragma unroll
     for (int u = 0; u < RC; ++u) {
+      if (u >= nr) break;
       const int kk = first + (c0 + u) * step;
       unsigned short raw = 0;
       if (seg_on && kk < p.s) {
@@ -111,6 +115,7 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
   }
 #pragma unroll
   for (int e = 0; e < 2 * RC; ++e) {
+    if ((e % RC) >= nr) continue;
     float f[8];
     unpack8(w[e * (GATED ? 2 : 1)], f);
 #pragma unroll
@@ -243,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) gated_decode_kernel(const GatedDe
     while (!ok) {
       unsigned int seen;
       asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters) : "memory");
-      ok = seen >= gridDim.x;
+      ok = seen >= gridDim.x + (unsigned int)a.extra_arrivals;
       if (!ok && clock64() - t0 > a.wait_limit) break;
     }
     if (!ok) {

@@ -209,6 +209,28 @@ def test_gated_decode_row_type_out_of_range_gives_a_zero_row():
     H.assert_bf16_close(H.to_np(Y), ref, False, "after a bad type")
 
 
+def test_gated_decode_bounded_wait_expires_and_the_handle_recovers():
+    """The wait between the two phases of the one-launch decode step is bounded: made to expect an arrival that never
+    comes (nothing faults, every CTA leaves), it gives up after the limit, the status says so, and the next calls on
+    the same handle are right again."""
+    q, dw, fw = 32, 64, 192
+    wl, Wg = synth.gated_ffn("gated-decode-wait", q, 1, q * dw, q * fw, np.array([9], np.int32), variant=4)
+    ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    args = (H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(np.concatenate([Wg, wl.W_up], axis=1), "bf16"),
+            H.to_dev(wl.W_down, "bf16"))
+    ref = oracle.ffn_swiglu(wl.X, wl.types, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths)
+    H.assert_bf16_close(H.to_np(ffn.forward(*args, out_dtype=torch.float32)), ref, False, "before")
+    ffn.set_option("wait_limit_cycles", 6_000_000)       # about 3 ms
+    ffn.set_option("test_stall_bytes", 512)
+    ffn.forward(*args, out_dtype=torch.float32)
+    assert ffn.last_status() == 6
+    ffn.set_option("test_stall_bytes", 0)
+    ffn.set_option("wait_limit_cycles", 4_000_000_000)
+    for _ in range(2):
+        H.assert_bf16_close(H.to_np(ffn.forward(*args, out_dtype=torch.float32)), ref, False, "after")
+    assert ffn.last_status() == 0
+
+
 def test_gated_refusals():
     with pytest.raises(binding.AlgError) as e:
         binding.GatedFFN([64, 128], [192, 320], dtype="bf16")     # hidden groups off the 128-column grid and unequal
