@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libalgproj.so")
-SOURCES = ["api.cu", "bucket.cu", "proj_simt.cu", "proj_tc.cu", "proj_tc2.cu", "proj_big.cu", "decode.cu", "ffn_decode.cu", "gated_decode.cu", "static_ws.cu"]
+SOURCES = ["api.cu", "bucket.cu", "proj_simt.cu", "proj_tc.cu", "proj_tc2.cu", "proj_big.cu", "decode.cu", "ffn_decode.cu", "row_decode.cu", "static_ws.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -86,7 +86,7 @@ struct alg_ffn_s {
   // decode step of the whole FFN in one launch (M <= kFfnDecodeMaxM)
   bool gated = false;        // SwiGLU: up = merged gate/up projection with silu(gate) * up epilogue
   bool fd_ok = false;
-  bool gd_ok = false;        // gated decode step (M <= kGatedDecodeMaxM) in one launch
+  bool rd_ok = false;        // decode step of one row in one launch (row_decode.cu): gated, or plain without fd_ok
   FfnDecodePlan fd = {};
   unsigned int *d_counters = nullptr;
 };
@@ -677,6 +677,11 @@ bool interval_runs(const alg_proj_s &p, int64_t M, int *run_rows, int64_t *perio
 }
 
 bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && p.opt_small_m && M <= kDecodeMaxM; }
+// one row under the complete-graph law with equal groups: the one-launch FMA kernel of row_decode.cu
+bool use_row_decode(const alg_proj_s &p, int64_t M) {
+  return M == 1 && p.opt_small_m && p.dtype == ALG_BF16 && (p.big.eligible || p.big.only) && !p.big.repack && !p.gated &&
+         !p.w_kmajor && !p.dyn_segments && p.sched != ALG_SCHED_INTERVAL && row_decode_fits(p.q, p.K, p.N);
+}
 
 // Forward call on the large-algebra path.  Equal buckets (cyclic or interval schedule, q | M) need no
 // pre-kernel at all; explicit types (q <= kMaxQ) go through bucketing and the row gather first.
@@ -912,6 +917,22 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
+  if (use_row_decode(*h, M) && (!bias || aligned16(bias))) {
+    // one row: one launch of plain FMAs over the 2 / q of the bank the row's type needs
+    RowDecodeArgs d = {};
+    d.mode = 2;
+    d.X = X;
+    d.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
+    d.W1 = W, d.ldw1 = ldw;
+    d.b1 = bias;
+    d.act = (int)act;
+    d.Y = Y;
+    d.y_bf16 = y_dtype == ALG_BF16;
+    d.D = h->K, d.F = h->N, d.q = h->q;
+    d.status = h->d_status;
+    d.wait_limit = h->wait_limit;
+    return cuda_status(launch_row_decode(d, h->num_sms, st));
+  }
   if (use_decode(*h, M)) return run_decode(*h, X, ldx, types, M, W, ldw, bias, act, Y, ldy, y_dtype, st);
   if (h->big.on || (h->sched == ALG_SCHED_EXPLICIT && use_big_counted(*h, M)) ||
       (h->sched == ALG_SCHED_CYCLIC && M % h->q == 0 && use_big_equal(*h, M)))
@@ -1010,7 +1031,7 @@ alg_status_t alg_proj_macs(alg_proj_t h, const int64_t *rows_per_type, int64_t *
 
 alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path) {
   if (!h || !path || M < 0) return ALG_ERR_INVALID_ARG;
-  *path = use_decode(*h, M) ? ALG_PATH_DECODE : (use_tc(*h) || h->big.on) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
+  *path = use_row_decode(*h, M) || use_decode(*h, M) ? ALG_PATH_DECODE : (use_tc(*h) || h->big.on) ? ALG_PATH_TCGEN05 : ALG_PATH_SIMT;
   return ALG_OK;
 }
 
@@ -1289,9 +1310,9 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
     f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
-  if (gated && schedule != ALG_SCHED_INTERVAL && f->up.big.eligible && f->down.big.eligible &&
-      gated_decode_fits(q, f->D, f->F)) {
-    f->gd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
+  if (dtype == ALG_BF16 && !f->fd_ok && schedule != ALG_SCHED_INTERVAL && f->up.big.eligible && f->down.big.eligible &&
+      row_decode_fits(q, f->D, f->F)) {
+    f->rd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
   *out = f;
@@ -1378,15 +1399,17 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
     }
     return cuda_status(launch_ffn_decode(d, h->fd, st));
   }
-  if (h->gd_ok && h->up.opt_small_m && M <= kGatedDecodeMaxM && !h->timing) {
-    // gated decode step of one row in one launch
-    if (b_up || b_down || act != ALG_ACT_NONE) return ALG_ERR_INVALID_ARG;
-    GatedDecodeArgs d = {};
+  if (h->rd_ok && h->up.opt_small_m && M == 1 && !h->timing && (!b_up || aligned16(b_up)) && (!b_down || aligned16(b_down))) {
+    // decode step of one row in one launch
+    if (h->gated && (b_up || b_down || act != ALG_ACT_NONE)) return ALG_ERR_INVALID_ARG;   // bias-free, silu(gate) * up
+    RowDecodeArgs d = {};
+    d.mode = h->gated ? 0 : 1;
     d.X = X;
     d.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;
-    d.M = (int)M;
-    d.W_gate_up = W_up, d.ldw_up = 2 * (int64_t)h->F;
-    d.W_down = W_down, d.ldw_dn = h->D;
+    d.W1 = W_up, d.ldw1 = h->gated ? 2 * (int64_t)h->F : h->F;
+    d.W2 = W_down, d.ldw2 = h->D;
+    d.b1 = b_up, d.b2 = b_down;
+    d.act = (int)act;
     d.H = ws + L.h;
     d.Y = Y;
     d.y_bf16 = y_dtype == ALG_BF16;
@@ -1395,7 +1418,7 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
     d.status = h->up.d_status;
     d.wait_limit = h->up.wait_limit;
     d.extra_arrivals = h->up.test_extra_expect ? 1 : 0;
-    return cuda_status(launch_gated_decode(d, h->up.num_sms, st));
+    return cuda_status(launch_row_decode(d, h->up.num_sms, st));
   }
   if (use_decode(h->up, M) && use_decode(h->down, M)) {
     // decode shapes: no bucketing, H stays in the original row order

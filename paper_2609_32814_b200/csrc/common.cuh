@@ -307,30 +307,32 @@ struct FfnDecodeArgs {
 bool ffn_decode_plan(int q, const int *dw, const int *fw, int D, int F, int num_sms, FfnDecodePlan *plan);
 cudaError_t launch_ffn_decode(const FfnDecodeArgs &a, const FfnDecodePlan &plan, cudaStream_t st);
 
-// Decode step of one row of the gated FFN (complete-graph law, equal groups) in one launch (gated_decode.cu).
-constexpr int kGatedDecodeMaxM = 1;
-struct GatedDecodeArgs {
+// Decode step of one row (complete-graph law, equal groups) in one launch: projection, FFN or gated FFN
+// (row_decode.cu).
+struct RowDecodeArgs {
+  int mode;                 // 0 gated FFN, 1 FFN, 2 projection (W1, b1, act; F = its output width, D = its input width)
   const void *X;            // [D] bf16
   const int32_t *types;     // the row's type; nullptr => type 0 (row 0 of the cyclic schedule)
-  int M;                    // 1
-  const void *W_gate_up;    // [D][ldw_up] bf16: the merged bank [W_gate | W_up], 2 F columns
-  int64_t ldw_up;
-  const void *W_down;       // [F][ldw_dn] bf16
-  int64_t ldw_dn;
-  void *H;                  // [F] bf16 scratch in global memory, 16-byte aligned
-  void *Y;                  // [D]
+  const void *W1;           // [D][ldw1] bf16: W_up, the merged bank [W_gate | W_up] (2 F columns), or the projection's W
+  int64_t ldw1;
+  const void *W2;           // [F][ldw2] bf16: W_down
+  int64_t ldw2;
+  const void *b1, *b2;      // bf16 biases or nullptr (not gated)
+  int act;                  // activation of phase 1 (not gated)
+  void *H;                  // [F] bf16 scratch in global memory, 16-byte aligned (FFN modes)
+  void *Y;                  // [D] (projection: [F])
   int y_bf16;
   int D, F, q;
-  int pc_up, pc_dn;         // columns of a warp's piece (8 or 16)                 (set by the launcher)
-  int ks_up, ks_dn;         // warps sharing the weight rows of a piece            (set by the launcher)
-  int units_up, units_dn;   // pieces x sharing warps                              (set by the launcher)
-  unsigned int *counters;   // [0] CTAs that finished phase 1, [1] CTAs past the wait; zero between launches
+  int pc1, pc2;             // columns of a warp's piece (8 or 16)                 (set by the launcher)
+  int ks1, ks2;             // warps sharing the weight rows of a piece            (set by the launcher)
+  int units1, units2;       // pieces x sharing warps                              (set by the launcher)
+  unsigned int *counters;   // [0] CTAs that finished phase 1, [1] CTAs past the wait; zero between launches (FFN modes)
   int *status;
   long long wait_limit;
   int extra_arrivals;       // test hook: arrivals the wait between the phases expects beyond the grid's (never come)
 };
-bool gated_decode_fits(int q, int D, int F);
-cudaError_t launch_gated_decode(const GatedDecodeArgs &a, int num_sms, cudaStream_t st);
+bool row_decode_fits(int q, int D, int F);
+cudaError_t launch_row_decode(const RowDecodeArgs &a, int num_sms, cudaStream_t st);
 
 void count_launch(int n = 1);
 int handle_device(alg_proj_t h);  // device the handle was created on (-1 for a null handle)

@@ -1,6 +1,7 @@
-// Decode step of ONE row (M = 1) of the gated FFN  y = (silu(x * W_gate) .* (x * W_up)) * W_down  under the
-// complete-graph law with q equal groups, in ONE launch (the M = 1 rows of the paper's gated-FFN table, appendix
-// "Kernel Benchmark Details").
+// Decode step of ONE row (M = 1) under the complete-graph law with q equal groups, in ONE launch: a projection
+// y = act(x *_q W + b), the FFN  y = act(x *_q W_up + b_up) *_q W_down + b_down, or the gated FFN
+// y = (silu(x * W_gate) .* (x * W_up)) * W_down  (the M = 1 rows of the paper's kernel tables, appendix "Kernel
+// Benchmark Details").
 //
 // A row of type i needs, for the output group j, the block W_ij of its row panel and the diagonal block W_jj
 // (Eqs. typed-diag / typed-off): 2 s of the q s weight rows above every output column.  The step is a pair of
@@ -8,9 +9,9 @@
 // round trips.  A warp owns a piece of 8 or 16 output columns (and, while there are more warps than pieces, a
 // share of the weight rows); its lanes split the rows, every lane keeps up to 32 loads of 16 bytes in flight and
 // reads the activations it needs straight from global memory -- no staging, one CTA barrier per phase at most.
-// The first loads of W_gate_up are issued before the launch's dependency resolves (weights do not depend on the
-// previous kernel), those of W_down before the wait between the phases.  Phase 1 writes the hidden row h (bf16) to
-// global memory; all CTAs meet at a counter (bounded wait); phase 2 is the same routine on h and W_down.
+// The first weight loads are issued before the launch's dependency resolves (weights do not depend on the previous
+// kernel), those of W_down before the wait between the phases of an FFN.  Phase 1 of an FFN writes the hidden row h
+// (bf16) to global memory; all CTAs meet at a counter (bounded wait); phase 2 is the same routine on h and W_down.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -21,7 +22,7 @@
 #include "trace.cuh"
 
 namespace algproj {
-ALG_TRACE_DEFINE(gated_decode)
+ALG_TRACE_DEFINE(row_decode)
 namespace {
 
 constexpr int kThreads = 256;
@@ -174,67 +175,123 @@ __device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_b
   }
 }
 
-__device__ __forceinline__ int read_type(const GatedDecodeArgs &a) {
+__device__ __forceinline__ int read_type(const RowDecodeArgs &a) {
   const int t = a.types ? a.types[0] : 0;
   return t < 0 || t >= a.q ? -1 : t;
 }
 
-__global__ void __launch_bounds__(kThreads, 1) gated_decode_kernel(const GatedDecodeArgs a) {
+__device__ __forceinline__ float activate(float z, int act) {
+  if (act == ALG_ACT_GELU_ERF) return 0.5f * z * (1.f + erff(z * 0.70710678118654752f));
+  if (act == ALG_ACT_GELU_TANH) return 0.5f * z * (1.f + tanhf(0.79788456080286536f * (z + 0.044715f * z * z * z)));
+  return z;
+}
+
+// eight results of a piece: + bias, activation, stored as bf16 or fp32
+__device__ __forceinline__ void store8(const float (&acc)[16], int col, const void *bias, int act, void *out, bool out_bf16) {
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = acc[e];
+  if (bias) {
+    float b[8];
+    unpack8(__ldg((const uint4 *)((const __nv_bfloat16 *)bias + col)), b);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] += b[e];
+  }
+  if (act != ALG_ACT_NONE) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = activate(v[e], act);
+  }
+  if (out_bf16) {
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      __nv_bfloat162 pk = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+      o[e] = *(uint32_t *)&pk;
+    }
+    *(uint4 *)((__nv_bfloat16 *)out + col) = make_uint4(o[0], o[1], o[2], o[3]);
+  } else {
+    float4 *dst = (float4 *)((float *)out + col);
+    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+    dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// MODE 0: gated FFN, 1: FFN, 2: projection (W1 only)
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecodeArgs a) {
+  constexpr bool GATED = MODE == 0, FFN = MODE != 2;
   __shared__ float partial[kWarps * 2 * 16];
   __shared__ int s_abort;
   ALG_TRACE_VARS;
   if (threadIdx.x == 0) ALG_TRACE(0, 1);
-  Phase up, dn;
-  up.W = (const __nv_bfloat16 *)a.W_gate_up, up.ldw = a.ldw_up, up.s = a.D / a.q, up.group_w = a.F / a.q, up.n_cols = a.F;
-  up.pc = a.pc_up, up.ks = a.ks_up;
-  dn.W = (const __nv_bfloat16 *)a.W_down, dn.ldw = a.ldw_dn, dn.s = a.F / a.q, dn.group_w = a.D / a.q, dn.n_cols = a.D;
-  dn.pc = a.pc_dn, dn.ks = a.ks_dn;
+  // phase 1 maps the D (projection: K) inputs to F (N) columns of W1; phase 2 maps F back to D through W2
+  Phase p1, p2;
+  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.D / a.q, p1.group_w = a.F / a.q, p1.n_cols = a.F;
+  p1.pc = a.pc1, p1.ks = a.ks1;
+  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.F / a.q, p2.group_w = a.D / a.q, p2.n_cols = a.D;
+  p2.pc = a.pc2, p2.ks = a.ks2;
   const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
   __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
   const int warp = threadIdx.x >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) s_abort = 0;
 
-  // ---- before the dependency resolves: the row type as it stands now and the first W_gate_up loads it asks for
-  // (the type is read again after the wait) ----
+  // ---- before the dependency resolves: the row type as it stands now and the first W1 loads it asks for (the type
+  // is read again after the wait) ----
   const int t_early = read_type(a);
   uint4 w[kLoads];
   {
     const int unit = blockIdx.x * kWarps + warp;
-    Lane l = lane_of(up, unit);
-    if (unit >= a.units_up || t_early < 0) l.on = false;
-    load_chunk<true>(w, up, l, max(t_early, 0), 0);
+    Lane l = lane_of(p1, unit);
+    if (unit >= a.units1 || t_early < 0) l.on = false;
+    load_chunk<GATED>(w, p1, l, max(t_early, 0), 0);
   }
   if (threadIdx.x == 0) ALG_TRACE(0, 2);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) ALG_TRACE(0, 3);
   const int type = read_type(a);   // (in flight while phase 1 runs on the early value)
 
-  // ---- phase 1: h = silu(x * W_gate) .* (x * W_up); on the type read early, again if the type has changed since ----
+  // ---- phase 1 on the type read early, again if the type has changed since.  Gated: h = silu(x * W_gate) .*
+  // (x * W_up); FFN: h = act(x * W_up + b_up); projection: y = act(x * W + b) ----
   for (int pass = 0; pass < 2; ++pass) {
     const int t = pass == 0 ? t_early : type;
     if (pass == 1 && type == t_early) break;
     if (t < 0) continue;
-    run_phase<true, false>(up, t, X, w, pass == 0, a.units_up, partial, [&](int col, const float (&acc)[16]) {
-      uint32_t o[4];
+    run_phase<GATED, false>(p1, t, X, w, pass == 0, a.units1, partial, [&](int col, const float (&acc)[16]) {
+      if (GATED) {
+        uint32_t o[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float g0 = acc[2 * e], g1 = acc[2 * e + 1];
-        __nv_bfloat162 pk = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * acc[8 + 2 * e], g1 / (1.f + __expf(-g1)) * acc[8 + 2 * e + 1]);
-        o[e] = *(uint32_t *)&pk;
+        for (int e = 0; e < 4; ++e) {
+          const float g0 = acc[2 * e], g1 = acc[2 * e + 1];
+          __nv_bfloat162 pk = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * acc[8 + 2 * e], g1 / (1.f + __expf(-g1)) * acc[8 + 2 * e + 1]);
+          o[e] = *(uint32_t *)&pk;
+        }
+        *(uint4 *)(H + col) = make_uint4(o[0], o[1], o[2], o[3]);
+      } else if (FFN) {
+        store8(acc, col, a.b1, a.act, H, true);
+      } else {
+        store8(acc, col, a.b1, a.act, a.Y, a.y_bf16 != 0);
       }
-      *(uint4 *)(H + col) = make_uint4(o[0], o[1], o[2], o[3]);
     });
   }
   if (type < 0 && threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);   // y = 0
   if (threadIdx.x == 0) ALG_TRACE(0, 6);
+  if (!FFN) {
+    if (type < 0) {   // a row type outside [0, q): the row of Y is zero
+      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.F; c += gridDim.x * kThreads) {
+        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
+        else ((float *)a.Y)[c] = 0.f;
+      }
+    }
+    return;
+  }
 
   // ---- the first W_down loads go out before the wait between the phases ----
   {
     const int unit = blockIdx.x * kWarps + warp;
-    Lane l = lane_of(dn, unit);
-    if (unit >= a.units_dn || type < 0) l.on = false;
-    load_chunk<false>(w, dn, l, max(type, 0), 0);
+    Lane l = lane_of(p2, unit);
+    if (unit >= a.units2 || type < 0) l.on = false;
+    load_chunk<false>(w, p2, l, max(type, 0), 0);
   }
 
   // ---- all of h is written before any of it is read: arrive, then wait (bounded) for the other CTAs ----
@@ -260,24 +317,11 @@ __global__ void __launch_bounds__(kThreads, 1) gated_decode_kernel(const GatedDe
   }
   __syncthreads();
 
-  // ---- phase 2: y = h * W_down ----
+  // ---- phase 2: y = h * W_down (+ b_down) ----
   if (!s_abort) {
     if (type >= 0) {
-      run_phase<false, true>(dn, type, H, w, true, a.units_dn, partial, [&](int col, const float (&acc)[16]) {
-        if (a.y_bf16) {
-          uint32_t o[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 pk = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
-            o[e] = *(uint32_t *)&pk;
-          }
-          *(uint4 *)((__nv_bfloat16 *)a.Y + col) = make_uint4(o[0], o[1], o[2], o[3]);
-        } else {
-          float4 *dst = (float4 *)((float *)a.Y + col);
-          dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-          dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-        }
-      });
+      run_phase<false, true>(p2, type, H, w, true, a.units2, partial,
+                             [&](int col, const float (&acc)[16]) { store8(acc, col, a.b2, ALG_ACT_NONE, a.Y, a.y_bf16 != 0); });
     } else {   // a row type outside [0, q): the row of Y is zero
       for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.D; c += gridDim.x * kThreads) {
         if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
@@ -304,26 +348,8 @@ int pick_ks(int pieces, int grid) {
   return ks;
 }
 
-}  // namespace
-
-bool gated_decode_fits(int q, int D, int F) {
-  if (q < 1 || D % q || F % q) return false;
-  return (D / q) % 8 == 0 && (F / q) % 8 == 0;
-}
-
-cudaError_t launch_gated_decode(const GatedDecodeArgs &in, int num_sms, cudaStream_t st) {
-  GatedDecodeArgs a = in;
-  if (a.M != 1 || !gated_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
-  const int s = a.D / a.q, r = a.F / a.q;
-  // every CTA must be resident for the wait between the phases: one CTA per SM at most
-  a.pc_up = r % 16 == 0 ? 16 : 8;
-  a.pc_dn = s % 16 == 0 ? 16 : 8;
-  const int pieces_up = a.F / a.pc_up, pieces_dn = a.D / a.pc_dn;
-  a.ks_up = pick_ks(pieces_up, num_sms);
-  a.ks_dn = pick_ks(pieces_dn, num_sms);
-  a.units_up = pieces_up * a.ks_up;
-  a.units_dn = pieces_dn * a.ks_dn;
-  const int grid = std::min(num_sms, (std::max(a.units_up, a.units_dn) + kWarps - 1) / kWarps);
+template <int MODE>
+cudaError_t launch_mode(const RowDecodeArgs &a, int grid, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -334,9 +360,34 @@ cudaError_t launch_gated_decode(const GatedDecodeArgs &in, int num_sms, cudaStre
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, gated_decode_kernel, a);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, row_decode_kernel<MODE>, a);
   count_launch(1);
   return e;
+}
+
+}  // namespace
+
+bool row_decode_fits(int q, int D, int F) {
+  if (q < 1 || D % q || F % q) return false;
+  return (D / q) % 8 == 0 && (F / q) % 8 == 0;
+}
+
+cudaError_t launch_row_decode(const RowDecodeArgs &in, int num_sms, cudaStream_t st) {
+  RowDecodeArgs a = in;
+  if (a.mode < 0 || a.mode > 2 || !row_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
+  const int s = a.D / a.q, r = a.F / a.q;
+  a.pc1 = r % 16 == 0 ? 16 : 8;
+  a.pc2 = s % 16 == 0 ? 16 : 8;
+  const int pieces1 = a.F / a.pc1, pieces2 = a.mode == 2 ? 0 : a.D / a.pc2;
+  a.ks1 = pick_ks(pieces1, num_sms);
+  a.ks2 = pieces2 ? pick_ks(pieces2, num_sms) : 1;
+  a.units1 = pieces1 * a.ks1;
+  a.units2 = pieces2 * a.ks2;
+  // every CTA of an FFN must be resident for the wait between the phases: one CTA per SM at most
+  const int grid = std::min(num_sms, (std::max(a.units1, a.units2) + kWarps - 1) / kWarps);
+  if (a.mode == 0) return launch_mode<0>(a, grid, st);
+  if (a.mode == 1) return launch_mode<1>(a, grid, st);
+  return launch_mode<2>(a, grid, st);
 }
 
 }  // namespace algproj

@@ -299,3 +299,79 @@ def test_ffn_decode_bounded_waits_expire_and_the_handle_recovers():
     for _ in range(2):                                    # counters were reset with the status
         assert np.array_equal(H.to_np(ffn.forward(*args, act=None, out_dtype=torch.float32)), ref)
     assert ffn.last_status() == 0
+
+
+# ---- one row (M = 1) under the complete-graph law with equal groups: one launch of plain FMAs ----------------
+
+@pytest.mark.parametrize("q,s_w,r_w", [
+    (32, 64, 192), (32, 80, 304), (32, 128, 384), (32, 64, 24), (32, 224, 64),   # the public shapes of the paper's kernel tables
+    (64, 40, 200),      # an algebra beyond 32 groups (large-algebra handle)
+    (5, 24, 40),        # pieces of 8 columns on both sides
+    (1, 256, 512),      # q = 1: an ordinary matrix-vector product
+])
+def test_one_row_projection_in_one_launch(q, s_w, r_w):
+    """A projection of one row: one launch, integers exact against the oracle for both output types, bias and GELU
+    within the bf16 tolerance."""
+    wl = _wl(q, 1, s_w, r_w, types=np.array([(3 * q) // 4 % q], np.int32), seed=q + s_w)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    assert proj.kernel_path(1) == binding.ALG_PATH_DECODE
+    X, t, W = H.to_dev(wl.X, "bf16"), H.dev_types(wl.types), H.to_dev(wl.W_up, "bf16")
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    for out_dtype in (torch.float32, torch.bfloat16):
+        n0 = binding.launch_count()
+        Y = proj.forward(X, t, W, out_dtype=out_dtype)
+        assert binding.launch_count() - n0 == 1 and proj.last_status() == 0
+        assert np.array_equal(H.to_np(Y), ref if out_dtype == torch.float32 else H.bf16_rne(ref))
+    wr = _wl(q, 1, s_w, r_w, types=wl.types, integer=False, seed=q + s_w + 1)
+    bias = synth.bf16_round(synth.normal(6, (wr.F,), 0.5))
+    Xr, Wr = H.to_dev(wr.X, "bf16"), H.to_dev(wr.W_up, "bf16")
+    for act in (None, "gelu", "gelu_tanh"):
+        Y = proj.forward(Xr, t, Wr, bias=H.to_dev(bias, "bf16"), act=act, out_dtype=torch.float32)
+        z = oracle.proj(wr.X, wr.types, wr.W_up, wr.d_widths, wr.f_widths, bias=bias)
+        if act == "gelu":
+            z = np.vectorize(oracle.gelu)(z)
+        elif act == "gelu_tanh":
+            z = 0.5 * z * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (z + 0.044715 * z ** 3)))
+        H.assert_bf16_close(H.to_np(Y), z, False, f"one row act={act}")
+
+
+def test_one_row_type_written_just_before_and_out_of_range():
+    """The kernel reads the row type before its launch dependency resolves (to request weights early) and again
+    after: a type written on the device right before the call is the one that counts.  A type outside [0, q) gives a
+    zero row and status 5."""
+    q, s_w, r_w = 8, 64, 128
+    wl = _wl(q, 1, s_w, r_w, seed=77)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    buf = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.empty((1, wl.F), dtype=torch.float32, device="cuda")
+    for rep in range(5):
+        buf.fill_((rep * 5) % q)                  # stale: what the early read may see
+        buf.fill_((rep * 3 + 1) % q)              # the type of this step, written just before the call
+        proj.forward(X, buf, W, out=out)
+        t = np.array([(rep * 3 + 1) % q], np.int32)
+        assert np.array_equal(H.to_np(out), oracle.proj(wl.X, t, wl.W_up, wl.d_widths, wl.f_widths)), rep
+    assert proj.last_status() == 0
+    buf.fill_(q)
+    out.fill_(7.0)
+    proj.forward(X, buf, W, out=out)
+    assert proj.last_status() == 5 and np.all(H.to_np(out) == 0)
+
+
+@pytest.mark.parametrize("q,D,F", [(32, 4096, 12288), (32, 2048, 768), (4, 256, 1024)])
+def test_one_row_ffn_in_one_launch(q, D, F):
+    """FFN shapes the staged one-launch decode kernel does not hold in shared memory: one row is two matrix-vector
+    phases around a bounded wait, biases and GELU included; twice in a row (the counters are cleared by the kernel)."""
+    types = np.array([q // 2], np.int32)
+    wl = synth.make_workload("ffnrow", config=4, variant=q + D, dtype="bf16", q=q, M=1, D=D, F=F, types=types)
+    wl.W_up, wl.W_down = synth.bf16_round(wl.W_up * 2.0), synth.bf16_round(wl.W_down * 2.0)
+    b_up = synth.bf16_round(synth.normal(8, (F,), 0.3))
+    b_down = synth.bf16_round(synth.normal(9, (D,), 0.3))
+    ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    args = (H.to_dev(wl.X, "bf16"), H.dev_types(types), H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"))
+    ref = oracle.ffn(wl.X, types, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths, b_up=b_up, b_down=b_down)
+    for out_dtype in (torch.float32, torch.bfloat16):
+        n0 = binding.launch_count()
+        Y = ffn.forward(*args, b_up=H.to_dev(b_up, "bf16"), b_down=H.to_dev(b_down, "bf16"), act="gelu", out_dtype=out_dtype)
+        assert binding.launch_count() - n0 == 1 and ffn.last_status() == 0
+        H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"one-row FFN q={q}")
