@@ -105,10 +105,11 @@ def _large_algebra_configs():
              ("u", 256, 2048): 0.266, ("u", 256, 8192): 0.414, ("u", 256, 32768): 1.169,
              ("d", 256, 2048): 0.243, ("d", 256, 8192): 0.552, ("d", 256, 32768): 1.958}
     # the paper's main kernel table (M = 2048 rows, the q it selects): model shape -> (K, N, q, its kernel's ms)
-    for name, (K, N, q, ms) in {"kp1p7b": (2048, 6144, 32, 0.0249), "kp4b": (2560, 9728, 32, 0.0511),
-                                "kp8b": (4096, 12288, 32, 0.0636), "kp30b": (2048, 768, 16, 0.0084),
-                                "kpdsv3": (7168, 2048, 16, 0.0283)}.items():
-        out[name] = dict(big=True, q=q, s=K // q, r=N // q, M=2048, schedule="interval", paper_ms=ms,
+    # (the last figure: the paper's kernel at M = 1 with q = 32, its fixed-q table, in microseconds)
+    for name, (K, N, q, ms, m1_us) in {"kp1p7b": (2048, 6144, 32, 0.0249, 3.8), "kp4b": (2560, 9728, 32, 0.0511, 4.1),
+                                       "kp8b": (4096, 12288, 32, 0.0636, 4.4), "kp30b": (2048, 768, 16, 0.0084, 3.3),
+                                       "kpdsv3": (7168, 2048, 16, 0.0283, 3.8)}.items():
+        out[name] = dict(big=True, q=q, s=K // q, r=N // q, M=2048, schedule="interval", paper_ms=ms, paper_m1_us=m1_us,
                          label=f"projection {K}->{N} in q={q} equal groups, X as q x q blocks of {2048 // q}x{K // q}, "
                                f"W of {K // q}x{N // q}, M=2048 rows, type = row block, bf16")
     for (way, q, M), ms in paper.items():
@@ -886,6 +887,8 @@ def run_big(args, ctx):
             extras["vs_dense"] = {"dense_ms_per_step": dense_ms, "star_ms_per_step": ms_step, "time_ratio_star_over_dense": ms_step / dense_ms,
                                   "control": "same library, q = 1 (ordinary X W on the table-driven tcgen05 kernel)",
                                   "ideal_ratio": flops / (2.0 * M * K * N)}
+        if cfg.get("paper_m1_us"):
+            extras["decode_m1"] = dict(proj_decode_calls(binding, 32, K, N), paper_h200_us=cfg["paper_m1_us"])
         # end to end through the C ABI's host entry point: pinned X in, Y out, copies inside the timing
         Xh = sets[0]["X"].cpu().pin_memory()
         Yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
@@ -984,6 +987,49 @@ def decode_measurements(binding, layers=64, replays=20):
     return {"protocol": f"{layers}-layer dependent FFN chain with distinct weights in one CUDA graph, median of {replays} replays",
             "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res,
             "launches": binding.launch_count() - launches0}
+
+
+def proj_decode_calls(binding, q, K, N, calls=32, replays=20):
+    """One row (M = 1) through `calls` projections K -> N with distinct weight banks in one CUDA graph (independent
+    calls on one stream).  GB/s counts the 2/q of the bank the row's type needs plus x and y."""
+    import torch
+    peaks = _peaks()
+    g = torch.Generator(device="cuda").manual_seed(987)
+    Ws = [(torch.randn((K, N), device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(calls)]
+    X = torch.randn((1, K), device="cuda", generator=g).to(torch.bfloat16)
+    Ys = [torch.empty((1, N), dtype=torch.bfloat16, device="cuda") for _ in range(calls)]
+    types = torch.full((1,), 5 % q, dtype=torch.int32, device="cuda")
+    proj = binding.Proj([K // q] * q, [N // q] * q, dtype="bf16")
+    ws = torch.empty(max(256, proj.workspace_bytes(1)), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+
+    def chain():
+        for l in range(calls):
+            proj.forward(X, types, Ws[l], out=Ys[l], workspace=ws, stream=stream)
+
+    l0 = binding.launch_count()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        chain()
+        torch.cuda.synchronize()
+        per_call = (binding.launch_count() - l0) // calls
+        with torch.cuda.graph(gr, stream=stream):
+            chain()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts = []
+    for _ in range(replays):
+        e0.record()
+        gr.replay()
+        e1.record()
+        e1.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    assert proj.last_status() == 0
+    us = float(np.median(ts)) * 1e3 / calls
+    bytes_call = 2 * (K // q) * N * 2 + (K + N) * 2
+    gbs = bytes_call / (us * 1e-6) / 1e9
+    return {"protocol": f"{calls} projections {K}->{N} at q = {q}, M = 1, distinct weights, one CUDA graph, median of {replays} replays",
+            "us_per_call": us, "launches_per_call": per_call, "needed_mb_per_call": bytes_call / 1e6,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"]}}
 
 
 def gated_decode_chain(binding, q, D, F, layers=32, replays=20):

@@ -28,6 +28,8 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kLoads = 32;   // 16-byte weight loads a lane keeps in flight
+constexpr int kMaxPo = 8;
+constexpr int kPieceCols = 16;   // columns of a piece where the group width allows (32 and 64 measured the same or slower)    // a piece has at most 8 x 8 columns
 
 // One matrix-vector phase as the kernel sees it.
 struct Phase {
@@ -36,7 +38,7 @@ struct Phase {
   int s;                    // rows of one input group
   int group_w;              // columns of one output group
   int n_cols;               // output columns (GATED: the up columns sit n_cols further in the bank)
-  int pc;                   // columns of a piece: 8 or 16
+  int pc;                   // columns of a piece: 8, 16, 32 or 64
   int ks;                   // warps that share the rows of a piece: 1, 2, 4 or 8
 };
 
@@ -161,13 +163,13 @@ __device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_b
     if (p.ks > 1) {   // the warps of a piece sit in one CTA
       if (lane < po) {
 #pragma unroll
-        for (int cc = 0; cc < 16; ++cc) partial[(warp * 2 + lane) * 16 + cc] = acc[cc];
+        for (int cc = 0; cc < 16; ++cc) partial[(warp * kMaxPo + lane) * 16 + cc] = acc[cc];
       }
       __syncthreads();
       if (l.part == 0 && lane < po) {
         for (int o = 1; o < p.ks; ++o)
 #pragma unroll
-          for (int cc = 0; cc < 16; ++cc) acc[cc] += partial[((warp + o) * 2 + lane) * 16 + cc];
+          for (int cc = 0; cc < 16; ++cc) acc[cc] += partial[((warp + o) * kMaxPo + lane) * 16 + cc];
       }
       __syncthreads();
     }
@@ -220,7 +222,7 @@ __device__ __forceinline__ void store8(const float (&acc)[16], int col, const vo
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecodeArgs a) {
   constexpr bool GATED = MODE == 0, FFN = MODE != 2;
-  __shared__ float partial[kWarps * 2 * 16];
+  __shared__ float partial[kWarps * kMaxPo * 16];
   __shared__ int s_abort;
   ALG_TRACE_VARS;
   if (threadIdx.x == 0) ALG_TRACE(0, 1);
@@ -376,8 +378,9 @@ cudaError_t launch_row_decode(const RowDecodeArgs &in, int num_sms, cudaStream_t
   RowDecodeArgs a = in;
   if (a.mode < 0 || a.mode > 2 || !row_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
   const int s = a.D / a.q, r = a.F / a.q;
-  a.pc1 = r % 16 == 0 ? 16 : 8;
-  a.pc2 = s % 16 == 0 ? 16 : 8;
+  auto piece = [](int group_w) { return group_w % kPieceCols == 0 ? kPieceCols : group_w % 16 == 0 ? 16 : 8; };
+  a.pc1 = piece(r);
+  a.pc2 = piece(s);
   const int pieces1 = a.F / a.pc1, pieces2 = a.mode == 2 ? 0 : a.D / a.pc2;
   a.ks1 = pick_ks(pieces1, num_sms);
   a.ks2 = pieces2 ? pick_ks(pieces2, num_sms) : 1;
