@@ -91,7 +91,7 @@ typedef enum { ALG_SCHED_EXPLICIT = 0, ALG_SCHED_CYCLIC = 1, ALG_SCHED_INTERVAL 
 typedef enum {
   ALG_PATH_SIMT = 0,    /* fp32-FMA tiles, any widths                                    */
   ALG_PATH_TCGEN05 = 1, /* bf16 grouped tcgen05 GEMM, TMA-fed, TMEM accumulators         */
-  ALG_PATH_DECODE = 2   /* small-M weight-streaming kernel                               */
+  ALG_PATH_DECODE = 2   /* small-M kernels (one row: plain FMAs; up to 64 rows: weight streaming) */
 } alg_path_t;
 
 #define ALG_MAX_Q 32        /* general interaction tables (32-bit keep masks) */
@@ -122,8 +122,8 @@ typedef enum {
  *                     row b = (b mod P) / (P / q) -- the pilot model's schedule
  *                     floor((p mod 768) / 192) over a batch of sequences.  0 (default) = one period,
  *                     P = M.  q must divide P, P must divide M, and P / q must be a multiple of 64.
- *   SMALL_M_KERNEL    1 (default): M <= 64 runs the weight-streaming kernels; 0: the prefill
- *                     kernels take every M.
+ *   SMALL_M_KERNEL    1 (default): M = 1 and M <= 64 run the small-M kernels where they apply; 0: the
+ *                     prefill kernels take every M.
  *   HOST_PLAN         1 (default): cyclic-schedule tile sequences are planned on the host;
  *                     0: every CTA plans for itself.
  *   WAIT_LIMIT_CYCLES bound of every device-side wait (mbarrier, counter), in SM clock cycles;
@@ -190,8 +190,12 @@ alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes
  * workspace: >= alg_proj_workspace_bytes(h, M), 256-byte aligned.
  * bf16 pointers and leading dimensions must keep rows 16-byte aligned (multiples of 8
  * elements).  M = 0 is a successful no-op; a type with no rows is legal.
- * M <= 64 with bf16 runs the decode kernel (when its per-CTA weight slice fits shared memory),
- * larger M the prefill kernels.
+ * Small M with bf16: M = 1 under ALG_TABLE_QQ with equal widths in multiples of 8 is one launch of
+ * plain FMAs over the 2 / q of the bank the row's type needs (any q up to ALG_MAX_Q_LARGE); M <= 64
+ * runs the weight-streaming decode kernel when its per-CTA weight slice fits shared memory and the
+ * handle has at most 8 groups or a bank of at most 4 Mi elements; everything else the prefill
+ * kernels.  (The FFN calls: M = 1 likewise one launch -- both projections around a bounded wait --
+ * and M <= 16 for shapes whose weight slices fit shared memory.)
  * Kernels are launched with programmatic stream serialization: they may start while the
  * kernel before them on `stream` is finishing, and wait for it before they touch X, bias, Y or
  * the workspace.  The decode kernel requests W before that wait (weights do not change during
