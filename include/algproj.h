@@ -118,6 +118,9 @@ typedef enum {
  *                     producer warps fetch the rows through the permutation themselves (four rows per copy
  *                     instruction, X read in place, one launch fewer); 0 (default) = 1, which measures faster or
  *                     equal on every benchmark step.  Results are identical.  Ignored by the other kernels.
+ *   WEIGHT_PACKED     1: the W given to alg_proj_forward is the padded bank alg_proj_pack_weight wrote (ldw is
+ *                     ignored); 0 (default): the caller's K x N bank.  Only handles whose
+ *                     alg_proj_packed_weight_bytes is not 0 take 1 (else ALG_ERR_UNSUPPORTED_SHAPE).
  *   INTERVAL_PERIOD   INTERVAL schedule of a table-driven handle: the typing repeats every P rows, type of
  *                     row b = (b mod P) / (P / q) -- the pilot model's schedule
  *                     floor((p mod 768) / 192) over a batch of sequences.  0 (default) = one period,
@@ -142,7 +145,8 @@ typedef enum {
   ALG_OPT_TEST_STALL_BYTES = 6,
   ALG_OPT_STAGE_K = 7,
   ALG_OPT_INTERVAL_PERIOD = 8,
-  ALG_OPT_ROW_GATHER = 9
+  ALG_OPT_ROW_GATHER = 9,
+  ALG_OPT_WEIGHT_PACKED = 10
 } alg_option_t;
 
 /* ---- projection handle ---------------------------------------------------------------------
@@ -251,6 +255,19 @@ alg_status_t alg_proj_kernel_path(alg_proj_t h, int64_t M, alg_path_t *path);
  * ALG_ERR_DEVICE_TIMEOUT).  Synchronises `stream` first.  After ALG_ERR_DEVICE_TIMEOUT the
  * handle's internal counters are reset, so the next forward call starts clean. */
 alg_status_t alg_proj_last_status(alg_proj_t h, void *stream, alg_status_t *status);
+
+/* ---- weights packed once (large-algebra handles with group widths that are multiples of 4 only) ---
+ * Such a handle copies X and W with every group widened to a multiple of 8 by zeros on each forward
+ * call (tiled copies start on 16 bytes).  W does not change between calls: alg_proj_pack_weight
+ * writes the padded bank once -- (q * ceil8(s)) x (q * ceil8(r)) elements of the handle's dtype,
+ * row-major, device memory, 16-byte aligned -- and with option WEIGHT_PACKED = 1 alg_proj_forward
+ * reads it in place, so that only X is copied per call.  alg_proj_packed_weight_bytes: size of that
+ * buffer; 0 when the handle pads nothing (then there is nothing to pack: ALG_ERR_UNSUPPORTED_SHAPE
+ * from alg_proj_pack_weight).  The pack runs on `stream`; W: K x N, ldw >= N, as in
+ * alg_proj_forward. */
+alg_status_t alg_proj_packed_weight_bytes(alg_proj_t h, size_t *bytes);
+alg_status_t alg_proj_pack_weight(alg_proj_t h, const void *W, int64_t ldw, void *W_packed,
+                                  size_t packed_bytes, void *stream);
 
 /* ---- FFN handle: Y = act(X *_q W_up + b_up) *_q W_down + b_down  ---------------------------
  * The two-map MLP (g = 1 in Eq. icml-decode-total) with both projections under the same law

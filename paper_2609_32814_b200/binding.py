@@ -23,7 +23,7 @@ ALG_ACT_NONE, ALG_ACT_GELU_ERF, ALG_ACT_GELU_TANH = 0, 1, 2
 ALG_SCHED_EXPLICIT, ALG_SCHED_CYCLIC, ALG_SCHED_INTERVAL = 0, 1, 2
 ALG_PATH_SIMT, ALG_PATH_TCGEN05, ALG_PATH_DECODE = 0, 1, 2
 OPTIONS = {"gemm_kernel": 1, "tile_n": 2, "small_m_kernel": 3, "host_plan": 4, "wait_limit_cycles": 5,
-           "test_stall_bytes": 6, "stage_k": 7, "interval_period": 8, "row_gather": 9}
+           "test_stall_bytes": 6, "stage_k": 7, "interval_period": 8, "row_gather": 9, "weight_packed": 10}
 
 _DTYPES = {"f32": ALG_F32, "bf16": ALG_BF16, torch.float32: ALG_F32, torch.bfloat16: ALG_BF16}
 _TABLES = {"qq": ALG_TABLE_QQ, "dense": ALG_TABLE_DENSE, "custom": ALG_TABLE_CUSTOM, "q2pow": ALG_TABLE_Q2POW}
@@ -33,7 +33,7 @@ _SCHEDS = {"explicit": ALG_SCHED_EXPLICIT, "cyclic": ALG_SCHED_CYCLIC, "interval
 
 EXPORTS = [
     "alg_proj_create", "alg_proj_destroy", "alg_proj_set_option", "alg_ffn_set_option", "alg_proj_workspace_bytes", "alg_proj_forward", "alg_proj_gemm_count",
-    "alg_proj_forward_static", "alg_proj_host_workspace_bytes", "alg_proj_forward_host", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
+    "alg_proj_forward_static", "alg_proj_host_workspace_bytes", "alg_proj_forward_host", "alg_proj_packed_weight_bytes", "alg_proj_pack_weight", "alg_proj_macs", "alg_proj_kernel_path", "alg_proj_last_status", "alg_ffn_create", "alg_ffn_destroy",
     "alg_ffn_workspace_bytes", "alg_ffn_forward", "alg_ffn_host_workspace_bytes", "alg_ffn_forward_host",
     "alg_ffn_gated_create", "alg_ffn_gated_forward", "alg_proj_grad_create", "alg_proj_grad_destroy",
     "alg_proj_grad_workspace_bytes", "alg_proj_grad_input", "alg_proj_grad_weight", "alg_proj_grad_last_status", "alg_ffn_macs", "alg_ffn_last_status", "alg_ffn_set_timing", "alg_ffn_get_timing", "alg_status_string", "alg_launch_count",
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.alg_proj_forward.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp, ctypes.c_size_t, vp]
         L.alg_proj_forward_static.argtypes = [vp, vp, i64, vp, i64, vp, i64, vp, i32, vp, i64, i32, vp]
         L.alg_proj_host_workspace_bytes.argtypes = [vp, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_proj_packed_weight_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+        L.alg_proj_pack_weight.argtypes = [vp, vp, i64, vp, ctypes.c_size_t, vp]
         L.alg_proj_forward_host.argtypes = [vp, vp, vp, i64, vp, i64, vp, i32, vp, i32, vp, ctypes.c_size_t, vp]
         L.alg_proj_gemm_count.argtypes = [vp, ctypes.POINTER(i64)]
         L.alg_proj_macs.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -202,6 +204,18 @@ class Proj(_Handle):
                                              _ptr(W), W.stride(0), _ptr(bias), _ACTS[act], _ptr(out),
                                              out.stride(0) if M else self.N, _DTYPES[out.dtype], _stream(stream)),
                "alg_proj_forward_static")
+        return out
+
+    def packed_weight_bytes(self) -> int:
+        out = ctypes.c_size_t()
+        _check(lib().alg_proj_packed_weight_bytes(self._h, ctypes.byref(out)), "alg_proj_packed_weight_bytes")
+        return out.value
+
+    def pack_weight(self, W, stream=None):
+        """alg_proj_pack_weight: the padded bank as a flat bf16 tensor (pass it to forward with option weight_packed = 1)."""
+        out = torch.empty(self.packed_weight_bytes() // 2, dtype=torch.bfloat16, device=W.device)
+        _check(lib().alg_proj_pack_weight(self._h, _ptr(W), W.stride(0), _ptr(out), out.numel() * 2, _stream(stream)),
+               "alg_proj_pack_weight")
         return out
 
     def host_workspace_bytes(self, max_M: int, out_dtype) -> int:

@@ -67,6 +67,7 @@ struct alg_proj_s {
   DecodePlan decode = {};
   // options (alg_proj_set_option)
   int opt_kernel = 0, opt_tile_n = 0, opt_stage_k = 0;
+  bool opt_w_packed = false;     // large-algebra handle with padded groups: W arrives packed (alg_proj_pack_weight)
   int opt_row_gather = 0;        // explicit types: 0 / 1 copy pass, 2 rows fetched by the GEMM's producer warps
   int64_t interval_period = 0;   // INTERVAL schedule of a table-driven handle: period of the typing (0 = the whole batch)
   bool opt_small_m = true, opt_host_plan = true;
@@ -749,10 +750,11 @@ alg_status_t run_big(alg_proj_s &p, const WsLayout &L, char *ws, const void *X, 
     const bool permuted = a.sched == 0;
     if (launch_pad_groups(X, ldx, permuted ? a.perm : nullptr, (int)M, p.q, p.big.s, p.big.s_pad, 0, 0, ws + L.xp, st) != cudaSuccess)
       return ALG_ERR_CUDA;
-    if (launch_pad_groups(W, ldw, nullptr, p.K, p.q, p.big.r, p.big.r_pad, p.big.s, p.big.s_pad, ws + L.wp, st) != cudaSuccess)
+    if (!p.opt_w_packed &&
+        launch_pad_groups(W, ldw, nullptr, p.K, p.q, p.big.r, p.big.r_pad, p.big.s, p.big.s_pad, ws + L.wp, st) != cudaSuccess)
       return ALG_ERR_CUDA;
     a.X = ws + L.xp, a.ldx = (int64_t)p.q * p.big.s_pad;
-    a.W = ws + L.wp, a.ldw = (int64_t)p.q * p.big.r_pad;
+    a.W = p.opt_w_packed ? W : ws + L.wp, a.ldw = (int64_t)p.q * p.big.r_pad;
     a.s = p.big.s_pad, a.r = p.big.r_pad;
   }
   a.sched_out = a.sched;
@@ -859,6 +861,11 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
       p.opt_stage_k = (int)value;
       for (PlanSlot &sl : p.plan) sl.M = -1;  // cached plans count K blocks of the old depth
       return ALG_OK;
+    case ALG_OPT_WEIGHT_PACKED:
+      if (value != 0 && value != 1) return ALG_ERR_INVALID_ARG;
+      if (value == 1 && !(p.big.on && p.big.repack)) return ALG_ERR_UNSUPPORTED_SHAPE;
+      p.opt_w_packed = value == 1;
+      return ALG_OK;
     case ALG_OPT_ROW_GATHER:
       if (value < 0 || value > 2) return ALG_ERR_INVALID_ARG;
       p.opt_row_gather = (int)value;
@@ -895,6 +902,23 @@ alg_status_t alg_ffn_set_option(alg_ffn_t h, alg_option_t option, int64_t value)
   return set_option(h->down, option, value);
 }
 
+alg_status_t alg_proj_packed_weight_bytes(alg_proj_t h, size_t *bytes) {
+  if (!h || !bytes) return ALG_ERR_INVALID_ARG;
+  *bytes = h->big.on && h->big.repack ? (size_t)h->q * h->big.s_pad * (size_t)h->q * h->big.r_pad * 2 : 0;
+  return ALG_OK;
+}
+
+alg_status_t alg_proj_pack_weight(alg_proj_t h, const void *W, int64_t ldw, void *W_packed, size_t packed_bytes, void *stream) {
+  if (!h || !W || !W_packed) return ALG_ERR_INVALID_ARG;
+  if (!(h->big.on && h->big.repack)) return ALG_ERR_UNSUPPORTED_SHAPE;
+  size_t need = 0;
+  alg_proj_packed_weight_bytes(h, &need);
+  if (packed_bytes < need) return ALG_ERR_WORKSPACE_TOO_SMALL;
+  if (ldw < h->N || !aligned16(W_packed)) return ALG_ERR_INVALID_ARG;
+  return cuda_status(launch_pad_groups(W, ldw, nullptr, h->K, h->q, h->big.r, h->big.r_pad, h->big.s, h->big.s_pad, W_packed,
+                                       (cudaStream_t)stream));
+}
+
 alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes) {
   if (!h || !bytes || max_M < 0 || max_M > (1 << 30)) return ALG_ERR_INVALID_ARG;
   *bytes = layout(*h, nullptr, max_M).total;
@@ -908,6 +932,7 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
   if (M == 0) return ALG_OK;
   if (!X || !W || !Y || !workspace) return ALG_ERR_INVALID_ARG;
   if (h->sched == ALG_SCHED_EXPLICIT && !types) return ALG_ERR_INVALID_ARG;
+  if (h->opt_w_packed) ldw = (int64_t)h->q * h->big.r_pad;   // the packed bank has its own leading dimension
   if (ldx < h->K || ldw < (h->w_kmajor ? h->K : h->N) || ldy < h->N) return ALG_ERR_INVALID_ARG;
   if (y_dtype != ALG_F32 && y_dtype != ALG_BF16) return ALG_ERR_INVALID_ARG;
   if ((int)act < 0 || (int)act > 2) return ALG_ERR_INVALID_ARG;

@@ -131,6 +131,34 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   Tile o;
   o.row0 = -1, o.rows = 0, o.i = 0, o.j = 0, o.n0 = 0, o.cols = 0, o.n0_w = 0, o.np = 1, o.ng = 1;
   if (t >= ctl->total) return o;
+  if (a.pack > 1 && a.gpack > 1) {
+    // several types AND several output groups per tile.  Type-group major; inside a type group first the column
+    // units (a.gpack groups each) that hold none of its types, one tile each, then the groups of the other units
+    // one by one (a tile never holds a type together with other groups than its own: the diagonal product of
+    // group k and the panel product of type k would both carry x_k W_kk)
+    int lo = 0, hi = (a.q + a.pack - 1) / a.pack;   // pre[lo] <= t < pre[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (ctl->pre[mid] <= t) lo = mid; else hi = mid;
+    }
+    const int l = t - ctl->pre[lo], g = a.gpack;
+    o.i = lo * a.pack;
+    o.np = min(a.pack, a.q - o.i);
+    const int n_units = (a.q + g - 1) / g, ua = o.i / g, ub = (o.i + o.np - 1) / g, apart = n_units - (ub - ua + 1);
+    if (l < apart) {
+      o.j = (l < ua ? l : l + (ub - ua + 1)) * g;
+      o.ng = min(g, a.q - o.j);
+    } else {
+      o.j = ua * g + (l - apart);
+      o.ng = 1;
+    }
+    o.row0 = o.i * a.rows_per_type;
+    o.rows = o.np * a.rows_per_type;
+    o.n0 = o.j * a.r_out;
+    o.n0_w = o.j * a.r;
+    o.cols = o.ng * a.r;
+    return o;
+  }
   if (a.pack > 1) {   // type-group major, then the output group, then the column tile
     const int per_group = a.q * a.nt_n;
     const int tg = t / per_group, rem = t - tg * per_group;
@@ -225,7 +253,28 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 2) {
     // tile counts: one warp turns the bucket offsets into "tiles before type i"
-    if (a.pack > 1) {
+    if (a.pack > 1 && a.gpack > 1) {
+      // tiles before every type group (see decode_tile)
+      const int n_tg = (q + a.pack - 1) / a.pack, g = a.gpack, n_units = (q + g - 1) / g;
+      int carry = 0;
+      for (int t0 = 0; t0 < n_tg; t0 += 32) {
+        const int tg = t0 + lane;
+        int v = 0;
+        if (tg < n_tg) {
+          const int i0 = tg * a.pack, np = min(a.pack, q - i0), ua = i0 / g, ub = (i0 + np - 1) / g;
+          v = n_units - (ub - ua + 1) + (min(q, (ub + 1) * g) - ua * g);
+        }
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += n;
+        }
+        if (tg < n_tg) ctl->pre[tg] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) ctl->pre[n_tg] = carry, ctl->total = carry;
+    } else if (a.pack > 1) {
       if (lane == 0) ctl->total = ((q + a.pack - 1) / a.pack) * q * a.nt_n;
     } else if (a.sched != 0) {
       if (lane == 0) ctl->total = q * ((a.rows_per_type + 127) >> 7) * a.col_units;
@@ -275,15 +324,24 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (loads_a && lane == 0) ALG_TRACE(0, 1);
       const bool packed = a.pack > 1;
       // packed tile: segment 0 is the diagonal one (group j), then one panel segment per type of the tile other than j
-      const int j_in = packed && tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0;
+      const int j_in = packed && tl.ng == 1 && tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0;
       // tile of several output groups: segment 0 is the panel product (k = i), then one diagonal product per group other than i
       const bool gp = a.gpack > 1;
-      const int i_in = gp && tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0;
-      const int n_seg = packed ? 1 + tl.np - j_in : gp ? 1 + tl.ng - i_in : (tl.i == tl.j ? 1 : 2);
+      // several types and several groups: one panel segment per type, then one diagonal segment per group (all rows)
+      const bool pg = packed && gp;
+      const int i_in = gp && !packed && tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0;
+      const int n_seg = pg ? tl.ng + tl.np - j_in : packed ? 1 + tl.np - j_in : gp ? 1 + tl.ng - i_in : (tl.i == tl.j ? 1 : 2);
       const int a_row = a.sched == 2 ? tl.row0 - tl.i * a.rows_per_type : tl.row0;
       for (int sg = 0; sg < n_seg && ok; ++sg) {
         int k;
-        if (packed) {
+        // (packed tiles; with several groups the panel segments come first: they are as wide as the tile and the first
+        // product of a tile is the one that overwrites the accumulator)
+        const int n_panel = tl.np - j_in;
+        const bool diag_seg = pg ? sg >= n_panel : sg == 0;
+        if (pg) {
+          k = diag_seg ? tl.j + sg - n_panel : tl.i + sg;
+          if (!diag_seg && j_in && k >= tl.j) ++k;   // skip type j: its rows have their one product already
+        } else if (packed) {
           k = sg == 0 ? tl.j : tl.i + sg - 1;
           if (sg > 0 && j_in && k >= tl.j) ++k;   // skip type j: its rows have their one product already
         } else if (gp) {
@@ -299,8 +357,10 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const uint32_t sa = smem0 + (uint32_t)stage * (uint32_t)C::kStageBytes;
           if (elect_one()) {
             if (loads_a && packed) {
-              if (sg == 0) {   // all rows of the tile: np types x rows_per_type rows, type-major
-                mbar_expect_tx(bar, (uint32_t)(a.pack * a.rows_per_type * BK * 2 + b_chunks * C::kBChunkBytes));
+              if (diag_seg) {   // all rows of the tile: np types x rows_per_type rows, type-major
+                const int goff = (k - tl.j) * a.r;   // (with several groups only the 64-column boxes of group k are fetched)
+                const int nb = pg ? (goff + a.r - 1) / 64 - goff / 64 + 1 : b_chunks;
+                mbar_expect_tx(bar, (uint32_t)(a.pack * a.rows_per_type * BK * 2 + nb * C::kBChunkBytes));
                 tma_load_4d(sa, &tmA, bar, kb * BK, k, 0, tl.i);
               } else {         // the rows of type k where they sit in the tile, zeros everywhere else
                 mbar_expect_tx(bar, (uint32_t)(128 * BK * 2 + b_chunks * C::kBChunkBytes));
@@ -313,7 +373,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               mbar_expect_tx(bar, (uint32_t)(a.a_box_rows * BK * 2 + nb * C::kBChunkBytes));
               if (a.sched == 2) tma_load_4d(sa, &tmA, bar, kb * BK, k, tl.i, a_row);
               else tma_load_3d(sa, &tmA, bar, kb * BK, k, a_row);
-            } else if (gp && sg > 0) {
+            } else if (pg ? diag_seg : gp && sg > 0) {
               // W_kk at the columns of its group inside the tile, zeros in the rest of the boxes it touches: column
               // (64 c - offset of the group in the tile) of group k is out of range on both sides of the group
               const int goff = (k - tl.j) * a.r;
@@ -347,7 +407,10 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int t = blockIdx.x; ok; t += gridDim.x) {
       const Tile tl = decode_tile(a, ctl, t);
       if (tl.row0 < 0) break;
-      const int n_kb = (a.pack > 1    ? 1 + tl.np - (tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0)
+      const int j_in_t = tl.ng == 1 && tl.j >= tl.i && tl.j < tl.i + tl.np ? 1 : 0;
+      const bool pg = a.pack > 1 && a.gpack > 1;
+      const int n_kb = (pg            ? tl.ng + tl.np - j_in_t
+                        : a.pack > 1  ? 1 + tl.np - j_in_t
                         : a.gpack > 1 ? 1 + tl.ng - (tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0)
                                       : (tl.i == tl.j ? 1 : 2)) *
                        nkb_seg;
@@ -357,7 +420,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (lane == 0) ALG_TRACE(1, 2);
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
-      const bool gp = a.gpack > 1;
+      const bool gp = a.gpack > 1 && !pg;
       const int i_in = gp && tl.i >= tl.j && tl.i < tl.j + tl.ng ? 1 : 0;
       for (int kb = 0; kb < n_kb; ++kb) {
         ok = __all_sync(0xffffffffu, wait_bar(full0 + 8u * (uint32_t)stage, phase, ctl, a.status));
@@ -367,11 +430,11 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint64_t da = da0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         uint64_t db = db0 + (uint64_t)((uint32_t)stage * (uint32_t)(C::kStageBytes >> 4));
         uint32_t d_seg = d_tmem, idesc_seg = idesc;
-        if (gp && kb >= nkb_seg) {
+        if ((gp && kb >= nkb_seg) || (pg && kb >= (tl.np - j_in_t) * nkb_seg)) {
           // diagonal segment of a multi-group tile: only the 64-column boxes its group touches were fetched; the
           // product covers exactly those accumulator columns (zeros outside the group add nothing)
-          int k = tl.j + kb / nkb_seg - 1;
-          if (i_in && k >= tl.i) ++k;
+          int k = pg ? tl.j + kb / nkb_seg - (tl.np - j_in_t) : tl.j + kb / nkb_seg - 1;
+          if (!pg && i_in && k >= tl.i) ++k;
           const int goff = (k - tl.j) * a.r;
           const int c_lo = goff / 64, c_hi = (goff + a.r - 1) / 64;
           db += (uint64_t)(c_lo * (C::kBChunkBytes >> 4));
@@ -686,7 +749,14 @@ cudaError_t launch_t(const BigArgs &a, int num_sms, cudaStream_t st) {
   }
   if (e != cudaSuccess) return e;
   long long tiles;
-  if (b.pack > 1) tiles = (long long)((a.q + b.pack - 1) / b.pack) * a.q * a.nt_n;
+  if (b.pack > 1 && b.gpack > 1) {
+    tiles = 0;
+    const int g = b.gpack, n_units = (a.q + g - 1) / g;
+    for (int i0 = 0; i0 < a.q; i0 += b.pack) {
+      const int np = std::min(b.pack, a.q - i0), ua = i0 / g, ub = (i0 + np - 1) / g;
+      tiles += n_units - (ub - ua + 1) + (std::min(a.q, (ub + 1) * g) - ua * g);
+    }
+  } else if (b.pack > 1) tiles = (long long)((a.q + b.pack - 1) / b.pack) * a.q * a.nt_n;
   else if (a.sched != 0) tiles = (long long)a.q * ((a.rows_per_type + 127) / 128) * b.col_units;
   else tiles = ((long long)a.M / 128 + a.q) * b.col_units;   // upper bound: every type may end in a ragged tile
   if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
@@ -724,10 +794,14 @@ cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
   // q = 256 (104) 1.49 -> 1.39 ms; groups of 128 lose (square product n = 8192: 0.065 -> 0.088 ms) and stay one per tile
   a.gpack = 1;
   a.col_units = a.q * a.nt_n;
-  if (a.pack == 1 && a.nt_n == 1 && !a.gated_f && !a.bias && a.r <= 112 && a.q >= 2) {
+  if (a.nt_n == 1 && !a.gated_f && !a.bias && a.r <= 112 && a.q >= 2) {
     // ... as many as keep at least four tiles per SM (2048 -> 768 in 16 groups of 48 at M = 2048 has 256 tiles of one
-    // group: five groups per tile would leave 64 tiles for 148 SMs)
-    const long long m_tiles = a.sched != 0 ? (long long)a.q * ((a.rows_per_type + 127) / 128) : std::max<long long>(a.q, a.M / 128);
+    // group: five groups per tile would leave 64 tiles for 148 SMs).  Together with several types per tile: a tile of
+    // np types and ng groups runs np panel segments and ng diagonal segments instead of ng x (np + 1)
+    // (25600 -> 5120 at q = 256, M = 2048: 34 segments per 24 columns before)
+    const long long m_tiles = a.pack > 1    ? (a.q + a.pack - 1) / a.pack
+                              : a.sched != 0 ? (long long)a.q * ((a.rows_per_type + 127) / 128)
+                                             : std::max<long long>(a.q, a.M / 128);
     int g = std::min(a.q, 256 / a.r);
     while (g > 1 && m_tiles * ((a.q + g - 1) / g) < 4ll * num_sms) --g;
     if (g > 1) {

@@ -63,6 +63,12 @@ def _forward(wl, schedule, out_dtype, **kw):
     (48, 4800, 136, 104, "explicit"),       # two groups per tile, the second one across three 64-column boxes; counted buckets
     (64, 64 * 130, 24, 24, "interval"),     # ten groups per tile, the last tile four; groups straddle the 64-column boxes
     (32, 32 * 200, 100, 88, "cyclic"),      # widths of 4 only in the reduction (repacked), two groups per tile
+    # several types AND several groups per tile (panel segments of the types first, then one diagonal segment per group;
+    # groups that share a unit with the tile's own types come one by one):
+    (256, 256 * 8, 100, 20, "interval"),    # 25600 -> 5120 at q = 256, M = 2048: sixteen types x seven groups, repacked
+    (128, 128 * 16, 200, 40, "cyclic"),     # eight types x three groups, cyclic rows
+    (200, 200 * 8, 24, 24, "interval"),     # a last type group of eight types, a last unit of fewer groups
+    (160, 160 * 40, 16, 104, "interval"),   # three types of 40 rows x two groups of 104 columns (three boxes)
 ])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_big_integer_bit_exact(q, M, s_w, r_w, schedule, out_dtype):
@@ -209,3 +215,29 @@ def test_big_refusals():
         proj.forward(X, None, W)
     with pytest.raises(binding.AlgError):
         proj.set_option("gemm_kernel", 2)
+
+
+def test_weights_packed_once():
+    """Group widths that are multiples of 4 only: the bank padded once by alg_proj_pack_weight gives the same bits as the
+    per-call padding, with one launch fewer per call; handles that pad nothing have nothing to pack."""
+    q, M, s_w, r_w = 256, 256 * 8, 100, 20
+    wl = _workload(q, M, s_w, r_w, "interval", seed=77)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule="interval")
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    n0 = binding.launch_count()
+    Y0 = proj.forward(X, None, W, out_dtype=torch.float32)
+    per_call = binding.launch_count() - n0
+    assert proj.packed_weight_bytes() == (q * 104) * (q * 24) * 2
+    Wp = proj.pack_weight(W)
+    proj.set_option("weight_packed", 1)
+    n0 = binding.launch_count()
+    Y1 = proj.forward(X, None, Wp, out_dtype=torch.float32)
+    assert binding.launch_count() - n0 == per_call - 1 and proj.last_status() == 0
+    assert torch.equal(Y0, Y1)
+    assert np.array_equal(H.to_np(Y1), oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths))
+    plain = binding.Proj([64] * 40, [128] * 40, dtype="bf16", schedule="interval")
+    assert plain.packed_weight_bytes() == 0
+    with pytest.raises(binding.AlgError):
+        plain.set_option("weight_packed", 1)
+    with pytest.raises(binding.AlgError):
+        plain.pack_weight(torch.zeros((64 * 40, 128 * 40), dtype=torch.bfloat16, device="cuda"))
