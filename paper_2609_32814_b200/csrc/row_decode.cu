@@ -67,6 +67,16 @@ __device__ __forceinline__ Lane lane_of(const Phase &p, int unit) {
   return l;
 }
 
+// Unit (piece x share of its rows) of this warp in round rd.  The warps that share a piece sit in one CTA; the pieces
+// go round-robin over the CTAs, so that every SM carries the same number of busy warps (768 pieces on 148 SMs: five or
+// six warps each, not eight on 96 of them; measured equal to the blocked order -- the step is bound by the chain of
+// round trips, not by any one SM).
+__device__ __forceinline__ int unit_of(int rd, int ks) {
+  const int warp = threadIdx.x >> 5, slot = warp / ks, part = warp - slot * ks;
+  const int piece = (rd * (kWarps / ks) + slot) * gridDim.x + blockIdx.x;
+  return piece * ks + part;
+}
+
 // Loads of one chunk: rows r0 .. of both segments (the diagonal block of group j, then -- unless the row's own type is
 // j -- its panel block), for the gate and, GATED, the up columns.  RC rows per segment and chunk.
 template <bool GATED>
@@ -141,7 +151,7 @@ __device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_b
   const int total_warps = gridDim.x * kWarps, po = p.pc >> 3;
   const int rounds = (n_units + total_warps - 1) / total_warps;
   for (int rd = 0; rd < rounds; ++rd) {
-    const int unit = rd * total_warps + blockIdx.x * kWarps + warp;
+    const int unit = unit_of(rd, p.ks);
     Lane l = lane_of(p, unit);
     if (unit >= n_units) l.on = false;
     float acc[16];
@@ -243,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
   const int t_early = read_type(a);
   uint4 w[kLoads];
   {
-    const int unit = blockIdx.x * kWarps + warp;
+    const int unit = unit_of(0, p1.ks);
     Lane l = lane_of(p1, unit);
     if (unit >= a.units1 || t_early < 0) l.on = false;
     load_chunk<GATED>(w, p1, l, max(t_early, 0), 0);
@@ -290,7 +300,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
 
   // ---- the first W_down loads go out before the wait between the phases ----
   {
-    const int unit = blockIdx.x * kWarps + warp;
+    const int unit = unit_of(0, p2.ks);
     Lane l = lane_of(p2, unit);
     if (unit >= a.units2 || type < 0) l.on = false;
     load_chunk<false>(w, p2, l, max(type, 0), 0);
@@ -387,7 +397,7 @@ cudaError_t launch_row_decode(const RowDecodeArgs &in, int num_sms, cudaStream_t
   a.units1 = pieces1 * a.ks1;
   a.units2 = pieces2 * a.ks2;
   // every CTA of an FFN must be resident for the wait between the phases: one CTA per SM at most
-  const int grid = std::min(num_sms, (std::max(a.units1, a.units2) + kWarps - 1) / kWarps);
+  const int grid = std::min(num_sms, std::max(a.units1 / a.ks1, a.units2 / a.ks2));   // at most one piece group per CTA and slot
   if (a.mode == 0) return launch_mode<0>(a, grid, st);
   if (a.mode == 1) return launch_mode<1>(a, grid, st);
   return launch_mode<2>(a, grid, st);
