@@ -241,3 +241,29 @@ def test_weights_packed_once():
         plain.set_option("weight_packed", 1)
     with pytest.raises(binding.AlgError):
         plain.pack_weight(torch.zeros((64 * 40, 128 * 40), dtype=torch.bfloat16, device="cuda"))
+
+
+@pytest.mark.parametrize("k", range(16))
+def test_big_many_small_types_and_narrow_groups_random(k):
+    """Random shapes in the regime where a tile takes several types and several groups: many types of few rows, groups of
+    at most 112 columns, widths in multiples of 4 (padded per call or packed once); integers exact."""
+    rng = np.random.default_rng(31000 + k)
+    q = int(rng.choice([64, 96, 128, 160, 200, 256]))
+    rows = int(rng.choice([1, 2, 3, 5, 8, 12, 16, 24, 33, 40, 64]))
+    s_w, r_w = 4 * int(rng.integers(1, 17)), 4 * int(rng.integers(1, 29))
+    if (q * s_w) % 8 or (q * r_w) % 8:
+        s_w, r_w = 2 * s_w, 2 * r_w
+    schedule = str(rng.choice(["cyclic", "interval"]))
+    wl = _workload(q, q * rows, s_w, r_w, schedule, seed=700 + k)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+    W = H.to_dev(wl.W_up, "bf16")
+    if proj.packed_weight_bytes() and k % 2 == 0:
+        W = proj.pack_weight(W)
+        proj.set_option("weight_packed", 1)
+    out_dtype = torch.float32 if k % 2 else torch.bfloat16
+    Y = proj.forward(H.to_dev(wl.X, "bf16"), None, W, out_dtype=out_dtype)
+    assert proj.last_status() == 0
+    ref = oracle.proj(wl.X, wl.types, wl.W_up, wl.d_widths, wl.f_widths)
+    if out_dtype == torch.bfloat16:
+        ref = H.bf16_rne(ref)
+    assert np.array_equal(H.to_np(Y), ref), (q, rows, s_w, r_w, schedule)

@@ -375,3 +375,35 @@ def test_one_row_ffn_in_one_launch(q, D, F):
         Y = ffn.forward(*args, b_up=H.to_dev(b_up, "bf16"), b_down=H.to_dev(b_down, "bf16"), act="gelu", out_dtype=out_dtype)
         assert binding.launch_count() - n0 == 1 and ffn.last_status() == 0
         H.assert_bf16_close(H.to_np(Y), ref, out_dtype == torch.bfloat16, f"one-row FFN q={q}")
+
+
+@pytest.mark.parametrize("k", range(18))
+def test_one_row_random_shapes(k):
+    """Random group counts and widths for the one-row kernel: projection (integers exact), FFN and gated FFN (tolerance)."""
+    rng = np.random.default_rng(52000 + k)
+    q = int(rng.choice([1, 2, 3, 5, 8, 16, 32, 40, 64, 100, 256]))
+    s_w = 8 * int(rng.integers(1, 20 if q <= 40 else 5))
+    r_w = 8 * int(rng.integers(1, 40 if q <= 40 else 9))
+    t = np.array([int(rng.integers(0, q))], np.int32)
+    mode = k % 3 if q <= 32 else 0
+    if mode == 0:
+        wl = _wl(q, 1, s_w, r_w, types=t, seed=k)
+        proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+        Y = proj.forward(H.to_dev(wl.X, "bf16"), H.dev_types(t), H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+        assert proj.last_status() == 0
+        assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, t, wl.W_up, wl.d_widths, wl.f_widths))
+    elif mode == 1:
+        wl = synth.make_workload("row1", config=4, variant=k, dtype="bf16", q=q, M=1, D=s_w * q, F=r_w * q, types=t)
+        ffn = binding.FFN(wl.d_widths, wl.f_widths, dtype="bf16")
+        Y = ffn.forward(H.to_dev(wl.X, "bf16"), H.dev_types(t), H.to_dev(wl.W_up, "bf16"), H.to_dev(wl.W_down, "bf16"),
+                        act="gelu", out_dtype=torch.float32)
+        assert ffn.last_status() == 0
+        H.assert_bf16_close(H.to_np(Y), oracle.ffn(wl.X, t, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths), False, f"one-row FFN {k}")
+    else:
+        wl, Wg = synth.gated_ffn("row1g", q, 1, s_w * q, r_w * q, t, variant=k)
+        ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16")
+        Y = ffn.forward(H.to_dev(wl.X, "bf16"), H.dev_types(t), H.to_dev(np.concatenate([Wg, wl.W_up], axis=1), "bf16"),
+                        H.to_dev(wl.W_down, "bf16"), out_dtype=torch.float32)
+        assert ffn.last_status() == 0
+        H.assert_bf16_close(H.to_np(Y), oracle.ffn_swiglu(wl.X, t, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths), False,
+                            f"one-row gated FFN {k}")
