@@ -13,8 +13,10 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "trace.cuh"
 
 namespace algproj {
+ALG_TRACE_DEFINE(bucket)
 
 namespace {
 
@@ -146,8 +148,11 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
   const int n_chunks = gridDim.x;
+  ALG_TRACE_VARS;
+  if (tid == 0) ALG_TRACE(0, 1);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the row types may come from the previous kernel
+  if (tid == 0) ALG_TRACE(0, 2);
   for (int e = tid; e < 32 * (kMaxQ + 1); e += kFusedThreads) (&s_wcnt[0][0])[e] = 0;
   const int row = blockIdx.x * kFusedThreads + tid;
   const bool live = row < a.M;
@@ -155,21 +160,27 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
   if (live && t == a.q) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
   const unsigned peers = __match_any_sync(0xffffffffu, t);
   const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+  if (tid == 0) ALG_TRACE(0, 3);
   __syncthreads();
   if (live && rank_in_warp == 0) s_wcnt[warp][t] = __popc(peers);
   __syncthreads();
-  if (tid < nt) {   // exclusive prefix over the warps; the total goes to global memory
-    int run = 0;
-    for (int w = 0; w < 32; ++w) {
-      const int v = s_wcnt[w][tid];
-      s_wcnt[w][tid] = run;
-      run += v;
+  for (int ty = warp; ty < nt; ty += kFusedThreads / 32) {   // exclusive prefix over the warps (lane = warp); the total goes to global memory
+    const int v = s_wcnt[lane][ty];
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
     }
-    a.chunk_counts[blockIdx.x * nt + tid] = run;
-    __threadfence();
+    s_wcnt[lane][ty] = incl - v;
+    if (lane == 31) {
+      a.chunk_counts[blockIdx.x * nt + ty] = incl;
+      __threadfence();
+    }
   }
   __syncthreads();
   if (tid == 0) {
+    ALG_TRACE(0, 4);
     atomicAdd(a.sync, 1u);
     const long long t0 = clock64();
     int go = 1;
@@ -183,6 +194,7 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
       }
     } while (v < (unsigned)n_chunks);
     s_go = go;
+    ALG_TRACE(0, 5);
   }
   __syncthreads();
   if (!s_go) return;
@@ -204,14 +216,21 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
     }
   }
   __syncthreads();
-  if (tid == 0) {   // bucket offsets: exclusive prefix of the totals over the types
-    int run = 0;
-    for (int ty = 0; ty < nt; ++ty) {
-      const int v = s_offset[ty];
-      s_offset[ty] = run;
-      run += v;
+  if (tid == 0) ALG_TRACE(0, 6);
+  if (warp == 0) {   // bucket offsets: exclusive prefix of the totals over the types (nt <= 33: lane 0 takes two)
+    const int v0 = lane < nt ? s_offset[lane] : 0, v1 = lane == 0 && nt > 32 ? s_offset[32] : 0;
+    int incl = v0;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
     }
-    s_offset[nt] = run;  // == M
+    const int total32 = __shfl_sync(0xffffffffu, incl, 31);
+    if (lane < nt) s_offset[lane] = incl - v0;
+    if (lane == 0) {
+      if (nt > 32) s_offset[32] = total32, s_offset[33] = total32 + v1;
+      else s_offset[nt] = total32;   // == M
+    }
   }
   __syncthreads();
   if (live) {
@@ -221,34 +240,53 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
       for (int e = 0; e < a.N * a.y_elem_bytes; ++e) y[e] = 0;
     }
   }
+  if (tid == 0) ALG_TRACE(0, 7);
   if (blockIdx.x == 0) {
     for (int t2 = tid; t2 <= nt; t2 += kFusedThreads) a.hdr->offsets[t2] = s_offset[t2];
-    if (tid == 0) write_pad_offsets(a.hdr, s_offset, a.q);
+    if (warp == 1) {   // offsets of the buckets padded to multiples of 64 rows (q <= 32: one lane per type)
+      const int v = lane < a.q ? (s_offset[lane + 1] - s_offset[lane] + 63) & ~63 : 0;
+      int incl = v;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += o;
+      }
+      if (lane < a.q) a.hdr->pad_offsets[lane] = incl - v;
+      if (lane == 31) a.hdr->pad_offsets[a.q] = incl;
+    }
   }
+  if (tid == 0) ALG_TRACE(0, 8);
 }
 
+// U = 16-byte loads a lane keeps in flight: 4 for rows of up to 2 KB (more registers would cost occupancy there), 16
+// for wider rows (the copy of a wide row is bound by its round trips, one per batch of loads)
+template <int U>
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ X, int64_t ldx_v,
                                                           const int *__restrict__ perm, int M, int vecs,
                                                           uint4 *__restrict__ Xb) {
+  ALG_TRACE_VARS;
+  if (threadIdx.x == 0) ALG_TRACE(1, 1);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // perm comes from the bucketing kernel
-  // a warp copies one row at a time, four independent 16-byte loads per lane in flight
+  if (threadIdx.x == 0) ALG_TRACE(1, 2);
+  // a warp copies one row at a time, U independent 16-byte loads per lane in flight
   const int lane = threadIdx.x & 31;
   const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int n_warps = (gridDim.x * blockDim.x) >> 5;
   for (int d = warp_global; d < M; d += n_warps) {
     const uint4 *src = X + (int64_t)__ldg(perm + d) * ldx_v;
     uint4 *dst = Xb + (int64_t)d * vecs;
-    for (int v0 = lane; v0 < vecs; v0 += 128) {
-      uint4 r[4];
+    for (int v0 = lane; v0 < vecs; v0 += 32 * U) {
+      uint4 r[U];
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
+      for (int u = 0; u < U; ++u)
         if (v0 + u * 32 < vecs) r[u] = __ldg(src + v0 + u * 32);
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
+      for (int u = 0; u < U; ++u)
         if (v0 + u * 32 < vecs) dst[v0 + u * 32] = r[u];
     }
   }
+  if (threadIdx.x == 0) ALG_TRACE(1, 3);
 }
 
 // padded row p -> original row (or -1 for a pad row / beyond the last bucket)
@@ -398,7 +436,10 @@ cudaError_t launch_gather_rows(const void *X, int64_t ldx, const int *perm, int 
   int grid = ceil_div(M, 8);  // eight warps (rows) per CTA
   if (grid > 148 * 8) grid = 148 * 8;
   count_launch(1);
-  return launch_pdl(gather_rows_kernel, grid, 256, st, (const uint4 *)X, (int64_t)(ldx * elem_bytes / 16), perm, M, vecs,
+  if (vecs > 128)
+    return launch_pdl(gather_rows_kernel<16>, grid, 256, st, (const uint4 *)X, (int64_t)(ldx * elem_bytes / 16), perm, M, vecs,
+                      (uint4 *)Xb);
+  return launch_pdl(gather_rows_kernel<4>, grid, 256, st, (const uint4 *)X, (int64_t)(ldx * elem_bytes / 16), perm, M, vecs,
                     (uint4 *)Xb);
 }
 
