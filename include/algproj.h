@@ -125,8 +125,10 @@ typedef enum {
  *                     row b = (b mod P) / (P / q) -- the pilot model's schedule
  *                     floor((p mod 768) / 192) over a batch of sequences.  0 (default) = one period,
  *                     P = M.  q must divide P, P must divide M, and P / q must be a multiple of 64.
- *   SMALL_M_KERNEL    1 (default): M = 1 and M <= 64 run the small-M kernels where they apply; 0: the
- *                     prefill kernels take every M.
+ *   SMALL_M_KERNEL    1 (default): small batches run the small-M kernels where the library expects them to
+ *                     be faster; 0: the prefill kernels take every M; 2: only the weight-streaming /
+ *                     staged kernels (M <= 64 / M <= 16) besides the prefill kernels; 3: the row kernel
+ *                     (plain FMAs, M <= 8) wherever it fits.
  *   HOST_PLAN         1 (default): cyclic-schedule tile sequences are planned on the host;
  *                     0: every CTA plans for itself.
  *   WAIT_LIMIT_CYCLES bound of every device-side wait (mbarrier, counter), in SM clock cycles;
@@ -194,12 +196,13 @@ alg_status_t alg_proj_workspace_bytes(alg_proj_t h, int64_t max_M, size_t *bytes
  * workspace: >= alg_proj_workspace_bytes(h, M), 256-byte aligned.
  * bf16 pointers and leading dimensions must keep rows 16-byte aligned (multiples of 8
  * elements).  M = 0 is a successful no-op; a type with no rows is legal.
- * Small M with bf16: M = 1 under ALG_TABLE_QQ with equal widths in multiples of 8 is one launch of
- * plain FMAs over the 2 / q of the bank the row's type needs (any q up to ALG_MAX_Q_LARGE); M <= 64
+ * Small M with bf16: up to 8 rows under ALG_TABLE_QQ with equal widths in multiples of 8 are one launch
+ * of plain FMAs over the 2 / q of the bank each row's type needs (any q up to ALG_MAX_Q_LARGE), taken
+ * while the rows' weight segments stay below a measured break-even (always for one row); M <= 64
  * runs the weight-streaming decode kernel when its per-CTA weight slice fits shared memory and the
  * handle has at most 8 groups or a bank of at most 4 Mi elements; everything else the prefill
- * kernels.  (The FFN calls: M = 1 likewise one launch -- both projections around a bounded wait --
- * and M <= 16 for shapes whose weight slices fit shared memory.)
+ * kernels.  (The FFN calls: a few rows likewise one launch -- both projections around a bounded
+ * wait -- and M <= 16 for shapes whose weight slices fit shared memory.)
  * Kernels are launched with programmatic stream serialization: they may start while the
  * kernel before them on `stream` is finishing, and wait for it before they touch X, bias, Y or
  * the workspace.  The decode kernel requests W before that wait (weights do not change during
@@ -302,9 +305,9 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
  * widths and equal f widths that are multiples of 8 (the large-algebra kernel: e.g. 2048 -> 6144 or
  * 2048 -> 768 split 32 ways); anything else is ALG_ERR_UNSUPPORTED_SHAPE.  Workspace size, options,
  * MAC count (three projections), status and destruction through the alg_ffn_* calls.
- * M = 1 under ALG_TABLE_QQ with equal widths is ONE launch (two matrix-vector phases on plain FMAs
- * around a bounded wait; option SMALL_M_KERNEL = 0 sends it through the prefill kernels instead);
- * every other M runs the prefill kernels.  With the CYCLIC schedule and q | M the rows are read and
+ * A few rows (always M = 1) under ALG_TABLE_QQ with equal widths are ONE launch (two matrix-vector
+ * phases on plain FMAs around a bounded wait; option SMALL_M_KERNEL = 0 sends them through the prefill
+ * kernels instead); every other M runs the prefill kernels.  With the CYCLIC schedule and q | M the rows are read and
  * written in place (two launches); otherwise bucketing and the row gather run first. */
 alg_status_t alg_ffn_gated_create(alg_ffn_t *out, int q, const int32_t *d_widths,
                                   const int32_t *f_widths, alg_dtype_t dtype, alg_table_t table,

@@ -70,7 +70,8 @@ struct alg_proj_s {
   bool opt_w_packed = false;     // large-algebra handle with padded groups: W arrives packed (alg_proj_pack_weight)
   int opt_row_gather = 0;        // explicit types: 0 / 1 copy pass, 2 rows fetched by the GEMM's producer warps
   int64_t interval_period = 0;   // INTERVAL schedule of a table-driven handle: period of the typing (0 = the whole batch)
-  bool opt_small_m = true, opt_host_plan = true;
+  int opt_small_m = 1;           // 0 prefill kernels only, 1 the library's choice, 2 weight-streaming kernels only, 3 the row kernel wherever it fits
+  bool opt_host_plan = true;
   long long wait_limit = kDefaultWaitLimit;
   int test_extra_expect = 0;
   // cyclic schedule: per-worker tile sequences of the one-CTA kernel for the last few M, planned on the host
@@ -680,10 +681,24 @@ bool interval_runs(const alg_proj_s &p, int64_t M, int *run_rows, int64_t *perio
   return true;
 }
 
-bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && p.opt_small_m && M <= kDecodeMaxM; }
-// one row under the complete-graph law with equal groups: the one-launch FMA kernel of row_decode.cu
+bool use_decode(const alg_proj_s &p, int64_t M) { return p.decode_ok && p.opt_small_m != 0 && M <= kDecodeMaxM; }
+// a few rows under the complete-graph law with equal groups: the one-launch FMA kernel of row_decode.cu
+// Rows up to which the row kernel is the library's choice.  It reads the diagonal block and the panel block of every
+// row (2 M segments; repeats come from L2) and runs at about 2.5 us + 0.65 us per MB read, so it wins while that stays
+// below what the prefill kernels need for a handful of rows: measured break-even near 20 MB for a projection (15-19 us
+// through bucketing, gather and the GEMM) and 45 MB for an FFN (27-37 us).  Handles with a weight-streaming kernel
+// (few groups, small banks) keep that one: 768 -> 3072 at q = 2 takes 4.9 us there against 6.3 us here at M = 1.
+int row_decode_rows(const alg_proj_s &p) {
+  if (p.decode_ok) return 0;
+  const double per_row = 4.0 * p.K * (double)p.N / p.q;   // bytes: two segments of K / q rows of the bank
+  return (int)std::max(1.0, std::min((double)kRowDecodeMaxM, 20e6 / per_row));
+}
+int row_decode_rows_ffn(int q, int D, int F, bool gated) {
+  const double per_row = 4.0 * (gated ? 3 : 2) * D * (double)F / q;
+  return (int)std::max(1.0, std::min((double)kRowDecodeMaxM, 45e6 / per_row));
+}
 bool use_row_decode(const alg_proj_s &p, int64_t M) {
-  return M == 1 && p.opt_small_m && p.dtype == ALG_BF16 && (p.big.eligible || p.big.only) && !p.big.repack && !p.gated &&
+  return M >= 1 && M <= (p.opt_small_m == 3 ? kRowDecodeMaxM : row_decode_rows(p)) && p.opt_small_m != 0 && p.opt_small_m != 2 && p.dtype == ALG_BF16 && (p.big.eligible || p.big.only) && !p.big.repack && !p.gated &&
          !p.w_kmajor && !p.dyn_segments && p.sched != ALG_SCHED_INTERVAL && row_decode_fits(p.q, p.K, p.N);
 }
 
@@ -876,7 +891,10 @@ static alg_status_t set_option(alg_proj_s &p, alg_option_t option, int64_t value
       if (value % ((int64_t)64 * p.q)) return ALG_ERR_INVALID_ARG;   // q runs of a multiple of 64 rows
       p.interval_period = value;
       return ALG_OK;
-    case ALG_OPT_SMALL_M_KERNEL: p.opt_small_m = value != 0; return ALG_OK;
+    case ALG_OPT_SMALL_M_KERNEL:
+      if (value < 0 || value > 3) return ALG_ERR_INVALID_ARG;
+      p.opt_small_m = (int)value;
+      return ALG_OK;
     case ALG_OPT_HOST_PLAN: p.opt_host_plan = value != 0; return ALG_OK;
     case ALG_OPT_WAIT_LIMIT_CYCLES:
       if (value < 1000) return ALG_ERR_INVALID_ARG;
@@ -949,12 +967,13 @@ alg_status_t alg_proj_forward(alg_proj_t h, const void *X, int64_t ldx, const in
     // one row: one launch of plain FMAs over the 2 / q of the bank the row's type needs
     RowDecodeArgs d = {};
     d.mode = 2;
-    d.X = X;
+    d.M = (int)M;
+    d.X = X, d.ldx = ldx;
     d.types = h->sched == ALG_SCHED_CYCLIC ? nullptr : types;
     d.W1 = W, d.ldw1 = ldw;
     d.b1 = bias;
     d.act = (int)act;
-    d.Y = Y;
+    d.Y = Y, d.ldy = ldy;
     d.y_bf16 = y_dtype == ALG_BF16;
     d.D = h->K, d.F = h->N, d.q = h->q;
     d.status = h->d_status;
@@ -1338,10 +1357,11 @@ static alg_status_t ffn_create(alg_ffn_t *out, int q, const int32_t *d_widths, c
     f->fd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
                cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
   }
-  if (dtype == ALG_BF16 && !f->fd_ok && schedule != ALG_SCHED_INTERVAL && f->up.big.eligible && f->down.big.eligible &&
+  if (dtype == ALG_BF16 && schedule != ALG_SCHED_INTERVAL && f->up.big.eligible && f->down.big.eligible &&
       row_decode_fits(q, f->D, f->F)) {
-    f->rd_ok = cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
-               cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
+    // (the two one-launch decode kernels share the exchange counters: both leave them zero)
+    f->rd_ok = f->d_counters != nullptr || (cudaMalloc(&f->d_counters, 2 * sizeof(unsigned int)) == cudaSuccess &&
+                                            cudaMemset(f->d_counters, 0, 2 * sizeof(unsigned int)) == cudaSuccess);
   }
   *out = f;
   return ALG_OK;
@@ -1401,7 +1421,7 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
   if (workspace_bytes < L.total) return ALG_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)workspace;
-  if (h->fd_ok && h->up.opt_small_m && M <= kFfnDecodeMaxM && !h->timing) {
+  if (h->fd_ok && (h->up.opt_small_m == 1 || h->up.opt_small_m == 2 || (h->up.opt_small_m == 3 && !h->rd_ok)) && M <= kFfnDecodeMaxM && !h->timing) {
     // decode step in one launch: both projections, H exchanged through L2 inside the kernel
     const alg_proj_s &u = h->up;
     FfnDecodeArgs d = {};
@@ -1427,19 +1447,21 @@ alg_status_t alg_ffn_forward(alg_ffn_t h, const void *X, const int32_t *types, i
     }
     return cuda_status(launch_ffn_decode(d, h->fd, st));
   }
-  if (h->rd_ok && h->up.opt_small_m && M == 1 && !h->timing && (!b_up || aligned16(b_up)) && (!b_down || aligned16(b_down))) {
+  if (h->rd_ok && (h->up.opt_small_m == 1 || h->up.opt_small_m == 3) &&
+      M <= (h->up.opt_small_m == 3 ? kRowDecodeMaxM : row_decode_rows_ffn(h->up.q, h->D, h->F, h->gated)) && !h->timing && (!b_up || aligned16(b_up)) && (!b_down || aligned16(b_down))) {
     // decode step of one row in one launch
     if (h->gated && (b_up || b_down || act != ALG_ACT_NONE)) return ALG_ERR_INVALID_ARG;   // bias-free, silu(gate) * up
     RowDecodeArgs d = {};
     d.mode = h->gated ? 0 : 1;
-    d.X = X;
+    d.M = (int)M;
+    d.X = X, d.ldx = h->D;
     d.types = h->up.sched == ALG_SCHED_CYCLIC ? nullptr : types;
     d.W1 = W_up, d.ldw1 = h->gated ? 2 * (int64_t)h->F : h->F;
     d.W2 = W_down, d.ldw2 = h->D;
     d.b1 = b_up, d.b2 = b_down;
     d.act = (int)act;
     d.H = ws + L.h;
-    d.Y = Y;
+    d.Y = Y, d.ldy = h->D;
     d.y_bf16 = y_dtype == ALG_BF16;
     d.D = h->D, d.F = h->F, d.q = h->up.q;
     d.counters = h->d_counters;

@@ -307,20 +307,24 @@ struct FfnDecodeArgs {
 bool ffn_decode_plan(int q, const int *dw, const int *fw, int D, int F, int num_sms, FfnDecodePlan *plan);
 cudaError_t launch_ffn_decode(const FfnDecodeArgs &a, const FfnDecodePlan &plan, cudaStream_t st);
 
-// Decode step of one row (complete-graph law, equal groups) in one launch: projection, FFN or gated FFN
+// Decode step of a few rows (complete-graph law, equal groups) in one launch: projection, FFN or gated FFN
 // (row_decode.cu).
+constexpr int kRowDecodeMaxM = 8;
 struct RowDecodeArgs {
   int mode;                 // 0 gated FFN, 1 FFN, 2 projection (W1, b1, act; F = its output width, D = its input width)
-  const void *X;            // [D] bf16
-  const int32_t *types;     // the row's type; nullptr => type 0 (row 0 of the cyclic schedule)
+  int M;                    // rows, 1 .. kRowDecodeMaxM
+  const void *X;            // [M][ldx] bf16
+  int64_t ldx;
+  const int32_t *types;     // the rows' types; nullptr => row m has type m mod q (cyclic schedule)
   const void *W1;           // [D][ldw1] bf16: W_up, the merged bank [W_gate | W_up] (2 F columns), or the projection's W
   int64_t ldw1;
   const void *W2;           // [F][ldw2] bf16: W_down
   int64_t ldw2;
   const void *b1, *b2;      // bf16 biases or nullptr (not gated)
   int act;                  // activation of phase 1 (not gated)
-  void *H;                  // [F] bf16 scratch in global memory, 16-byte aligned (FFN modes)
-  void *Y;                  // [D] (projection: [F])
+  void *H;                  // [M][F] bf16 scratch in global memory, 16-byte aligned (FFN modes)
+  void *Y;                  // [M][ldy]: D columns (projection: F)
+  int64_t ldy;
   int y_bf16;
   int D, F, q;
   int pc1, pc2;             // columns of a warp's piece (8 or 16)                 (set by the launcher)

@@ -141,26 +141,36 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
   }
 }
 
-// One phase for the units of this warp.  `w` holds the first chunk of the first unit when have_first.  Results of a
-// piece: lanes with lr == 0 of the warp with part == 0 call `emit(col, acc)`.
+__device__ __forceinline__ int read_type(const RowDecodeArgs &a, int m) {
+  const int t = a.types ? a.types[m] : m % a.q;
+  return t < 0 || t >= a.q ? -1 : t;
+}
+
+// One phase for the units of this warp: unit = (row, piece, share of the piece's weight rows), rows outermost.  `w` holds
+// the first chunk of the first unit when have_first, fetched for row type t_first; the other units read their row's
+// type themselves.  Results of a piece: lanes with lr == 0 of the warp with part == 0 call `emit(row, col, acc)`.
 template <bool GATED, bool FROM_L2, typename Emit>
-__device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_bfloat16 *x, uint4 (&w)[kLoads], bool have_first,
-                                          int n_units, float *partial, Emit emit) {
+__device__ __forceinline__ void run_phase(const RowDecodeArgs &a, const Phase &p, const __nv_bfloat16 *x, int64_t ldx,
+                                          uint4 (&w)[kLoads], bool have_first, int t_first, int n_units, float *partial, Emit emit) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_warps = gridDim.x * kWarps, po = p.pc >> 3;
   const int rounds = (n_units + total_warps - 1) / total_warps;
+  const int per_row = n_units / a.M;
   for (int rd = 0; rd < rounds; ++rd) {
     const int unit = unit_of(rd, p.ks);
-    Lane l = lane_of(p, unit);
-    if (unit >= n_units) l.on = false;
+    const int m = min(unit / per_row, a.M - 1);
+    Lane l = lane_of(p, unit - m * per_row);
+    const int type = have_first && rd == 0 ? t_first : read_type(a, m);
+    if (unit >= n_units || type < 0) l.on = false;
+    const __nv_bfloat16 *xm = x + (int64_t)m * ldx;
     float acc[16];
 #pragma unroll
     for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
     const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
     for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
-      if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, type, c0);
-      fma_chunk<GATED, FROM_L2>(w, p, l, type, c0, x, acc);
+      if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, max(type, 0), c0);
+      fma_chunk<GATED, FROM_L2>(w, p, l, max(type, 0), c0, xm, acc);
     }
     // sum over the lanes that share the columns
 #pragma unroll
@@ -183,13 +193,8 @@ __device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_b
       }
       __syncthreads();
     }
-    if (l.on && l.part == 0 && lane < po) emit(l.col, acc);
+    if (l.on && l.part == 0 && lane < po) emit(m, l.col, acc);
   }
-}
-
-__device__ __forceinline__ int read_type(const RowDecodeArgs &a) {
-  const int t = a.types ? a.types[0] : 0;
-  return t < 0 || t >= a.q ? -1 : t;
 }
 
 __device__ __forceinline__ float activate(float z, int act) {
@@ -244,32 +249,31 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
   p2.pc = a.pc2, p2.ks = a.ks2;
   const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
   __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
-  const int warp = threadIdx.x >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) s_abort = 0;
 
-  // ---- before the dependency resolves: the row type as it stands now and the first W1 loads it asks for (the type
-  // is read again after the wait) ----
-  const int t_early = read_type(a);
+  // ---- before the dependency resolves: the type of this warp's first row as it stands now and the first W1 loads it
+  // asks for (the type is read again after the wait) ----
+  const int per_row1 = a.units1 / a.M;
+  const int unit1 = unit_of(0, p1.ks), m1 = min(unit1 / per_row1, a.M - 1);
+  const int t_early = read_type(a, m1);
   uint4 w[kLoads];
   {
-    const int unit = unit_of(0, p1.ks);
-    Lane l = lane_of(p1, unit);
-    if (unit >= a.units1 || t_early < 0) l.on = false;
+    Lane l = lane_of(p1, unit1 - m1 * per_row1);
+    if (unit1 >= a.units1 || t_early < 0) l.on = false;
     load_chunk<GATED>(w, p1, l, max(t_early, 0), 0);
   }
   if (threadIdx.x == 0) ALG_TRACE(0, 2);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) ALG_TRACE(0, 3);
-  const int type = read_type(a);   // (in flight while phase 1 runs on the early value)
+  const int type1 = read_type(a, m1);   // (in flight while phase 1 runs on the early value)
 
-  // ---- phase 1 on the type read early, again if the type has changed since.  Gated: h = silu(x * W_gate) .*
-  // (x * W_up); FFN: h = act(x * W_up + b_up); projection: y = act(x * W + b) ----
+  // ---- phase 1 with the early type for the first unit, again (all of it) if some warp of the CTA finds that its type
+  // has changed since.  Gated: h = silu(x * W_gate) .* (x * W_up); FFN: h = act(x * W_up + b_up); projection:
+  // y = act(x * W + b) ----
   for (int pass = 0; pass < 2; ++pass) {
-    const int t = pass == 0 ? t_early : type;
-    if (pass == 1 && type == t_early) break;
-    if (t < 0) continue;
-    run_phase<GATED, false>(p1, t, X, w, pass == 0, a.units1, partial, [&](int col, const float (&acc)[16]) {
+    if (pass == 1 && !__syncthreads_or(type1 != t_early)) break;
+    run_phase<GATED, false>(a, p1, X, a.ldx, w, pass == 0, t_early, a.units1, partial, [&](int m, int col, const float (&acc)[16]) {
       if (GATED) {
         uint32_t o[4];
 #pragma unroll
@@ -278,77 +282,78 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
           __nv_bfloat162 pk = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * acc[8 + 2 * e], g1 / (1.f + __expf(-g1)) * acc[8 + 2 * e + 1]);
           o[e] = *(uint32_t *)&pk;
         }
-        *(uint4 *)(H + col) = make_uint4(o[0], o[1], o[2], o[3]);
+        *(uint4 *)(H + (int64_t)m * a.F + col) = make_uint4(o[0], o[1], o[2], o[3]);
       } else if (FFN) {
-        store8(acc, col, a.b1, a.act, H, true);
+        store8(acc, col, a.b1, a.act, H + (int64_t)m * a.F, true);
       } else {
-        store8(acc, col, a.b1, a.act, a.Y, a.y_bf16 != 0);
+        store8(acc, col, a.b1, a.act, a.y_bf16 ? (void *)((__nv_bfloat16 *)a.Y + (int64_t)m * a.ldy) : (void *)((float *)a.Y + (int64_t)m * a.ldy),
+               a.y_bf16 != 0);
       }
     });
   }
-  if (type < 0 && threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);   // y = 0
   if (threadIdx.x == 0) ALG_TRACE(0, 6);
-  if (!FFN) {
-    if (type < 0) {   // a row type outside [0, q): the row of Y is zero
-      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.F; c += gridDim.x * kThreads) {
-        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
-        else ((float *)a.Y)[c] = 0.f;
-      }
-    }
-    return;
-  }
+  const int n_out = FFN ? a.D : a.F;   // width of Y
 
-  // ---- the first W_down loads go out before the wait between the phases ----
-  {
-    const int unit = unit_of(0, p2.ks);
-    Lane l = lane_of(p2, unit);
-    if (unit >= a.units2 || type < 0) l.on = false;
-    load_chunk<false>(w, p2, l, max(type, 0), 0);
-  }
+  if (FFN) {
+    // ---- the first W_down loads go out before the wait between the phases ----
+    const int per_row2 = a.units2 / a.M;
+    const int unit2 = unit_of(0, p2.ks), m2 = min(unit2 / per_row2, a.M - 1);
+    const int type2 = read_type(a, m2);
+    {
+      Lane l = lane_of(p2, unit2 - m2 * per_row2);
+      if (unit2 >= a.units2 || type2 < 0) l.on = false;
+      load_chunk<false>(w, p2, l, max(type2, 0), 0);
+    }
 
-  // ---- all of h is written before any of it is read: arrive, then wait (bounded) for the other CTAs ----
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    ALG_TRACE(0, 8);
-    __threadfence();
-    atomicAdd(a.counters, 1u);
-    const long long t0 = clock64();
-    bool ok = false;
-    while (!ok) {
-      unsigned int seen;
-      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters) : "memory");
-      ok = seen >= gridDim.x + (unsigned int)a.extra_arrivals;
-      if (!ok && clock64() - t0 > a.wait_limit) break;
-    }
-    if (!ok) {
-      s_abort = 1;
-      atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
-    }
-    __threadfence();
-    ALG_TRACE(0, 9);
-  }
-  __syncthreads();
-
-  // ---- phase 2: y = h * W_down (+ b_down) ----
-  if (!s_abort) {
-    if (type >= 0) {
-      run_phase<false, true>(p2, type, H, w, true, a.units2, partial,
-                             [&](int col, const float (&acc)[16]) { store8(acc, col, a.b2, ALG_ACT_NONE, a.Y, a.y_bf16 != 0); });
-    } else {   // a row type outside [0, q): the row of Y is zero
-      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.D; c += gridDim.x * kThreads) {
-        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
-        else ((float *)a.Y)[c] = 0.f;
-      }
-    }
-  }
-  // the last CTA past the wait clears the counters for the next launch
-  if (threadIdx.x == 0) {
-    ALG_TRACE(0, 12);
-    const unsigned int left = atomicAdd(a.counters + 1, 1u);
-    if (left == gridDim.x - 1) {
-      a.counters[0] = 0;
-      a.counters[1] = 0;
+    // ---- all of h is written before any of it is read: arrive, then wait (bounded) for the other CTAs ----
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      ALG_TRACE(0, 8);
       __threadfence();
+      atomicAdd(a.counters, 1u);
+      const long long t0 = clock64();
+      bool ok = false;
+      while (!ok) {
+        unsigned int seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters) : "memory");
+        ok = seen >= gridDim.x + (unsigned int)a.extra_arrivals;
+        if (!ok && clock64() - t0 > a.wait_limit) break;
+      }
+      if (!ok) {
+        s_abort = 1;
+        atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+      }
+      __threadfence();
+      ALG_TRACE(0, 9);
+    }
+    __syncthreads();
+
+    // ---- phase 2: y = h * W_down (+ b_down) ----
+    if (!s_abort) {
+      run_phase<false, true>(a, p2, H, a.F, w, true, type2, a.units2, partial, [&](int m, int col, const float (&acc)[16]) {
+        store8(acc, col, a.b2, ALG_ACT_NONE,
+               a.y_bf16 ? (void *)((__nv_bfloat16 *)a.Y + (int64_t)m * a.ldy) : (void *)((float *)a.Y + (int64_t)m * a.ldy), a.y_bf16 != 0);
+      });
+    }
+    // the last CTA past the wait clears the counters for the next launch
+    if (threadIdx.x == 0) {
+      ALG_TRACE(0, 12);
+      const unsigned int left = atomicAdd(a.counters + 1, 1u);
+      if (left == gridDim.x - 1) {
+        a.counters[0] = 0;
+        a.counters[1] = 0;
+        __threadfence();
+      }
+    }
+  }
+
+  // ---- rows whose type lies outside [0, q): zero, and the status says so ----
+  for (int m = 0; m < a.M; ++m) {
+    if (read_type(a, m) >= 0) continue;
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
+    for (int c = blockIdx.x * kThreads + threadIdx.x; c < n_out; c += gridDim.x * kThreads) {
+      if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[(int64_t)m * a.ldy + c] = __float2bfloat16_rn(0.f);
+      else ((float *)a.Y)[(int64_t)m * a.ldy + c] = 0.f;
     }
   }
 }
@@ -386,16 +391,16 @@ bool row_decode_fits(int q, int D, int F) {
 
 cudaError_t launch_row_decode(const RowDecodeArgs &in, int num_sms, cudaStream_t st) {
   RowDecodeArgs a = in;
-  if (a.mode < 0 || a.mode > 2 || !row_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
+  if (a.mode < 0 || a.mode > 2 || a.M < 1 || a.M > kRowDecodeMaxM || !row_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
   const int s = a.D / a.q, r = a.F / a.q;
   auto piece = [](int group_w) { return group_w % kPieceCols == 0 ? kPieceCols : group_w % 16 == 0 ? 16 : 8; };
   a.pc1 = piece(r);
   a.pc2 = piece(s);
   const int pieces1 = a.F / a.pc1, pieces2 = a.mode == 2 ? 0 : a.D / a.pc2;
-  a.ks1 = pick_ks(pieces1, num_sms);
-  a.ks2 = pieces2 ? pick_ks(pieces2, num_sms) : 1;
-  a.units1 = pieces1 * a.ks1;
-  a.units2 = pieces2 * a.ks2;
+  a.ks1 = pick_ks(pieces1 * a.M, num_sms);
+  a.ks2 = pieces2 ? pick_ks(pieces2 * a.M, num_sms) : 1;
+  a.units1 = a.M * pieces1 * a.ks1;
+  a.units2 = a.M * pieces2 * a.ks2;
   // every CTA of an FFN must be resident for the wait between the phases: one CTA per SM at most
   const int grid = std::min(num_sms, std::max(a.units1 / a.ks1, a.units2 / a.ks2));   // at most one piece group per CTA and slot
   if (a.mode == 0) return launch_mode<0>(a, grid, st);

@@ -407,3 +407,66 @@ def test_one_row_random_shapes(k):
         assert ffn.last_status() == 0
         H.assert_bf16_close(H.to_np(Y), oracle.ffn_swiglu(wl.X, t, Wg, wl.W_up, wl.W_down, wl.d_widths, wl.f_widths), False,
                             f"one-row gated FFN {k}")
+
+
+@pytest.mark.parametrize("q,s_w,r_w", [(32, 64, 192), (32, 128, 384), (5, 24, 40), (64, 40, 200)])
+@pytest.mark.parametrize("M", [2, 5, 8])
+def test_few_rows_on_the_row_kernel(q, s_w, r_w, M):
+    """Up to eight rows on the row kernel (forced with SMALL_M_KERNEL = 3; by its own choice the library takes it while
+    the rows' weight segments stay below the measured break-even): projection exact on integers, FFN and gated FFN within
+    tolerance, explicit and cyclic types, one launch each."""
+    for schedule in ("explicit", "cyclic"):
+        types = synth.cyclic_types(M, q) if schedule == "cyclic" else synth.uniform_types(5000 + q + M, M, q)
+        t = None if schedule == "cyclic" else H.dev_types(types)
+        wl = _wl(q, M, s_w, r_w, types=types, seed=q + M)
+        proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16", schedule=schedule)
+        proj.set_option("small_m_kernel", 3)
+        n0 = binding.launch_count()
+        Y = proj.forward(H.to_dev(wl.X, "bf16"), t, H.to_dev(wl.W_up, "bf16"), out_dtype=torch.float32)
+        assert binding.launch_count() - n0 == 1 and proj.last_status() == 0
+        assert np.array_equal(H.to_np(Y), oracle.proj(wl.X, types, wl.W_up, wl.d_widths, wl.f_widths))
+        if q > 32:
+            continue
+        wf = synth.make_workload("rows-ffn", config=4, variant=q + M, dtype="bf16", q=q, M=M, D=s_w * q, F=r_w * q, types=types)
+        ffn = binding.FFN(wf.d_widths, wf.f_widths, dtype="bf16", schedule=schedule)
+        ffn.set_option("small_m_kernel", 3)
+        n0 = binding.launch_count()
+        Y = ffn.forward(H.to_dev(wf.X, "bf16"), t, H.to_dev(wf.W_up, "bf16"), H.to_dev(wf.W_down, "bf16"), act="gelu",
+                        out_dtype=torch.bfloat16)
+        assert binding.launch_count() - n0 == 1 and ffn.last_status() == 0
+        H.assert_bf16_close(H.to_np(Y), oracle.ffn(wf.X, types, wf.W_up, wf.W_down, wf.d_widths, wf.f_widths), True, "rows FFN")
+        wg, Wg = synth.gated_ffn("rows-gated", q, M, s_w * q, r_w * q, types, variant=q + M)
+        gf = binding.GatedFFN(wg.d_widths, wg.f_widths, dtype="bf16", schedule=schedule)
+        gf.set_option("small_m_kernel", 3)
+        n0 = binding.launch_count()
+        Y = gf.forward(H.to_dev(wg.X, "bf16"), t, H.to_dev(np.concatenate([Wg, wg.W_up], axis=1), "bf16"), H.to_dev(wg.W_down, "bf16"),
+                       out_dtype=torch.float32)
+        assert binding.launch_count() - n0 == 1 and gf.last_status() == 0
+        H.assert_bf16_close(H.to_np(Y), oracle.ffn_swiglu(wg.X, types, Wg, wg.W_up, wg.W_down, wg.d_widths, wg.f_widths), False,
+                            "rows gated FFN")
+
+
+def test_few_rows_one_type_out_of_range_and_types_written_just_before():
+    q, s_w, r_w, M = 8, 64, 128, 6
+    wl = _wl(q, M, s_w, r_w, seed=91)
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    proj.set_option("small_m_kernel", 3)
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    buf = torch.zeros(M, dtype=torch.int32, device="cuda")
+    out = torch.empty((M, wl.F), dtype=torch.float32, device="cuda")
+    pos = torch.arange(M, dtype=torch.int32, device="cuda")
+    for rep in range(4):
+        buf.fill_(rep % q)                                  # stale: what the early read may see
+        torch.remainder(pos * 3 + rep, q, out=buf)          # the types of this step, written just before the call
+        proj.forward(X, buf, W, out=out)
+        t = ((np.arange(M) * 3 + rep) % q).astype(np.int32)
+        assert np.array_equal(H.to_np(out), oracle.proj(wl.X, t, wl.W_up, wl.d_widths, wl.f_widths)), rep
+    assert proj.last_status() == 0
+    t = np.array([1, 2, q + 3, 0, -1, 5], np.int32)
+    out.fill_(7.0)
+    proj.forward(X, H.dev_types(t), W, out=out)
+    assert proj.last_status() == 5
+    got = H.to_np(out)
+    good = [0, 1, 3, 5]
+    assert np.all(got[[2, 4]] == 0)
+    assert np.array_equal(got[good], oracle.proj(wl.X[good], t[good], wl.W_up, wl.d_widths, wl.f_widths))
