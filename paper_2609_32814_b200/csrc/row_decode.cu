@@ -141,36 +141,26 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
   }
 }
 
-__device__ __forceinline__ int read_type(const RowDecodeArgs &a, int m) {
-  const int t = a.types ? a.types[m] : m % a.q;
-  return t < 0 || t >= a.q ? -1 : t;
-}
-
-// One phase for the units of this warp: unit = (row, piece, share of the piece's weight rows), rows outermost.  `w` holds
-// the first chunk of the first unit when have_first, fetched for row type t_first; the other units read their row's
-// type themselves.  Results of a piece: lanes with lr == 0 of the warp with part == 0 call `emit(row, col, acc)`.
+// One phase for the units of this warp.  `w` holds the first chunk of the first unit when have_first.  Results of a
+// piece: lanes with lr == 0 of the warp with part == 0 call `emit(col, acc)`.
 template <bool GATED, bool FROM_L2, typename Emit>
-__device__ __forceinline__ void run_phase(const RowDecodeArgs &a, const Phase &p, const __nv_bfloat16 *x, int64_t ldx,
-                                          uint4 (&w)[kLoads], bool have_first, int t_first, int n_units, float *partial, Emit emit) {
+__device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_bfloat16 *x, uint4 (&w)[kLoads], bool have_first,
+                                          int n_units, float *partial, Emit emit) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_warps = gridDim.x * kWarps, po = p.pc >> 3;
   const int rounds = (n_units + total_warps - 1) / total_warps;
-  const int per_row = n_units / a.M;
   for (int rd = 0; rd < rounds; ++rd) {
     const int unit = unit_of(rd, p.ks);
-    const int m = min(unit / per_row, a.M - 1);
-    Lane l = lane_of(p, unit - m * per_row);
-    const int type = have_first && rd == 0 ? t_first : read_type(a, m);
-    if (unit >= n_units || type < 0) l.on = false;
-    const __nv_bfloat16 *xm = x + (int64_t)m * ldx;
+    Lane l = lane_of(p, unit);
+    if (unit >= n_units) l.on = false;
     float acc[16];
 #pragma unroll
     for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
     const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
     for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
-      if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, max(type, 0), c0);
-      fma_chunk<GATED, FROM_L2>(w, p, l, max(type, 0), c0, xm, acc);
+      if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, type, c0);
+      fma_chunk<GATED, FROM_L2>(w, p, l, type, c0, x, acc);
     }
     // sum over the lanes that share the columns
 #pragma unroll
@@ -193,8 +183,13 @@ __device__ __forceinline__ void run_phase(const RowDecodeArgs &a, const Phase &p
       }
       __syncthreads();
     }
-    if (l.on && l.part == 0 && lane < po) emit(m, l.col, acc);
+    if (l.on && l.part == 0 && lane < po) emit(l.col, acc);
   }
+}
+
+__device__ __forceinline__ int read_type(const RowDecodeArgs &a) {
+  const int t = a.types ? a.types[0] : 0;
+  return t < 0 || t >= a.q ? -1 : t;
 }
 
 __device__ __forceinline__ float activate(float z, int act) {
@@ -249,14 +244,227 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
   p2.pc = a.pc2, p2.ks = a.ks2;
   const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
   __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
+  const int warp = threadIdx.x >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == 0) s_abort = 0;
+
+  // ---- before the dependency resolves: the row type as it stands now and the first W1 loads it asks for (the type
+  // is read again after the wait) ----
+  const int t_early = read_type(a);
+  uint4 w[kLoads];
+  {
+    const int unit = unit_of(0, p1.ks);
+    Lane l = lane_of(p1, unit);
+    if (unit >= a.units1 || t_early < 0) l.on = false;
+    load_chunk<GATED>(w, p1, l, max(t_early, 0), 0);
+  }
+  if (threadIdx.x == 0) ALG_TRACE(0, 2);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) ALG_TRACE(0, 3);
+  const int type = read_type(a);   // (in flight while phase 1 runs on the early value)
+
+  // ---- phase 1 on the type read early, again if the type has changed since.  Gated: h = silu(x * W_gate) .*
+  // (x * W_up); FFN: h = act(x * W_up + b_up); projection: y = act(x * W + b) ----
+  for (int pass = 0; pass < 2; ++pass) {
+    const int t = pass == 0 ? t_early : type;
+    if (pass == 1 && type == t_early) break;
+    if (t < 0) continue;
+    run_phase<GATED, false>(p1, t, X, w, pass == 0, a.units1, partial, [&](int col, const float (&acc)[16]) {
+      if (GATED) {
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float g0 = acc[2 * e], g1 = acc[2 * e + 1];
+          __nv_bfloat162 pk = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * acc[8 + 2 * e], g1 / (1.f + __expf(-g1)) * acc[8 + 2 * e + 1]);
+          o[e] = *(uint32_t *)&pk;
+        }
+        *(uint4 *)(H + col) = make_uint4(o[0], o[1], o[2], o[3]);
+      } else if (FFN) {
+        store8(acc, col, a.b1, a.act, H, true);
+      } else {
+        store8(acc, col, a.b1, a.act, a.Y, a.y_bf16 != 0);
+      }
+    });
+  }
+  if (type < 0 && threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);   // y = 0
+  if (threadIdx.x == 0) ALG_TRACE(0, 6);
+  if (!FFN) {
+    if (type < 0) {   // a row type outside [0, q): the row of Y is zero
+      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.F; c += gridDim.x * kThreads) {
+        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
+        else ((float *)a.Y)[c] = 0.f;
+      }
+    }
+    return;
+  }
+
+  // ---- the first W_down loads go out before the wait between the phases ----
+  {
+    const int unit = unit_of(0, p2.ks);
+    Lane l = lane_of(p2, unit);
+    if (unit >= a.units2 || type < 0) l.on = false;
+    load_chunk<false>(w, p2, l, max(type, 0), 0);
+  }
+
+  // ---- all of h is written before any of it is read: arrive, then wait (bounded) for the other CTAs ----
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ALG_TRACE(0, 8);
+    __threadfence();
+    atomicAdd(a.counters, 1u);
+    const long long t0 = clock64();
+    bool ok = false;
+    while (!ok) {
+      unsigned int seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters) : "memory");
+      ok = seen >= gridDim.x + (unsigned int)a.extra_arrivals;
+      if (!ok && clock64() - t0 > a.wait_limit) break;
+    }
+    if (!ok) {
+      s_abort = 1;
+      atomicExch(a.status, (int)ALG_ERR_DEVICE_TIMEOUT);
+    }
+    __threadfence();
+    ALG_TRACE(0, 9);
+  }
+  __syncthreads();
+
+  // ---- phase 2: y = h * W_down (+ b_down) ----
+  if (!s_abort) {
+    if (type >= 0) {
+      run_phase<false, true>(p2, type, H, w, true, a.units2, partial,
+                             [&](int col, const float (&acc)[16]) { store8(acc, col, a.b2, ALG_ACT_NONE, a.Y, a.y_bf16 != 0); });
+    } else {   // a row type outside [0, q): the row of Y is zero
+      for (int c = blockIdx.x * kThreads + threadIdx.x; c < a.D; c += gridDim.x * kThreads) {
+        if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[c] = __float2bfloat16_rn(0.f);
+        else ((float *)a.Y)[c] = 0.f;
+      }
+    }
+  }
+  // the last CTA past the wait clears the counters for the next launch
+  if (threadIdx.x == 0) {
+    ALG_TRACE(0, 12);
+    const unsigned int left = atomicAdd(a.counters + 1, 1u);
+    if (left == gridDim.x - 1) {
+      a.counters[0] = 0;
+      a.counters[1] = 0;
+      __threadfence();
+    }
+  }
+}
+
+__device__ __forceinline__ int read_row_type(const RowDecodeArgs &a, int m) {
+  const int t = a.types ? a.types[m] : m % a.q;
+  return t < 0 || t >= a.q ? -1 : t;
+}
+
+// The same phase for several rows: unit = (row, piece, share of the piece's weight rows), rows outermost.  `w` holds
+// the first chunk of the first unit when have_first, fetched for row type t_first; the other units read their row's
+// type themselves.  Results of a piece: lanes with lr == 0 of the warp with part == 0 call `emit(row, col, acc)`.
+// Barrier of the warps that share a piece (2, 4 or 8 of them: at most four groups per CTA).  The ids are literals so
+// that the kernel reserves five hardware barriers, not all sixteen -- with sixteen a second CTA (the next launch's,
+// which starts early to request its weights) could not become resident beside this one.
+__device__ __forceinline__ void group_barrier(int id, int threads) {
+  switch (id) {
+    case 1: asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); break;
+    case 2: asm volatile("bar.sync 2, %0;" ::"r"(threads) : "memory"); break;
+    case 3: asm volatile("bar.sync 3, %0;" ::"r"(threads) : "memory"); break;
+    default: asm volatile("bar.sync 4, %0;" ::"r"(threads) : "memory"); break;
+  }
+}
+
+// A row whose type lies outside [0, q) reads nothing; with LAST (the phase that writes Y) its pieces are stored as zeros
+// and the status word says so.
+template <bool GATED, bool FROM_L2, bool LAST, typename Emit>
+__device__ __forceinline__ void run_rows_phase(const RowDecodeArgs &a, const Phase &p, const __nv_bfloat16 *x, int64_t ldx,
+                                          uint4 (&w)[kLoads], bool have_first, int t_first, int n_units, float *partial, Emit emit) {
+  constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_warps = gridDim.x * kWarps, po = p.pc >> 3;
+  const int rounds = (n_units + total_warps - 1) / total_warps;
+  const int per_row = a.M == 1 ? n_units : n_units / a.M;   // (one row: no division on the way to the first load)
+  for (int rd = 0; rd < rounds; ++rd) {
+    const int unit = unit_of(rd, p.ks);
+    const int m = a.M == 1 ? 0 : min(unit / per_row, a.M - 1);
+    const int real = read_row_type(a, m);   // (on its way while the first attempt below runs on the type read early)
+    int type = have_first && rd == 0 ? t_first : real;
+    const __nv_bfloat16 *xm = x + (int64_t)m * ldx;
+    // the first unit runs on the type read before the launch's dependency resolved; if the type has changed since, the
+    // warps of the piece (they share the row) do it again -- they meet at a barrier of their own, not the CTA's
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      Lane l = lane_of(p, unit - m * per_row);
+      if (unit >= n_units || type < 0) l.on = false;
+      float acc[16];
+#pragma unroll
+      for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
+      const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
+      for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
+        if (!(have_first && rd == 0 && attempt == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, max(type, 0), c0);
+        fma_chunk<GATED, FROM_L2>(w, p, l, max(type, 0), c0, xm, acc);
+      }
+      // sum over the lanes that share the columns
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        if (d >= po) {
+#pragma unroll
+          for (int cc = 0; cc < (GATED ? 16 : 8); ++cc) acc[cc] += __shfl_xor_sync(0xffffffffu, acc[cc], d);
+        }
+      }
+      if (p.ks > 1) {   // the warps of a piece sit side by side in one CTA
+        const int bar_id = 1 + warp / p.ks, bar_threads = 32 * p.ks;
+        if (lane < po) {
+#pragma unroll
+          for (int cc = 0; cc < 16; ++cc) partial[(warp * kMaxPo + lane) * 16 + cc] = acc[cc];
+        }
+        group_barrier(bar_id, bar_threads);
+        if (l.part == 0 && lane < po) {
+          for (int o = 1; o < p.ks; ++o)
+#pragma unroll
+            for (int cc = 0; cc < 16; ++cc) acc[cc] += partial[((warp + o) * kMaxPo + lane) * 16 + cc];
+        }
+        group_barrier(bar_id, bar_threads);
+      }
+      if (attempt == 0 && type != real) {
+        type = real;
+        continue;
+      }
+      if (l.on && l.part == 0 && lane < po) emit(m, l.col, acc);
+      if (LAST && type < 0 && unit < n_units && l.part == 0 && lane < po && l.col < p.n_cols) {
+        if (a.y_bf16) *(uint4 *)((__nv_bfloat16 *)a.Y + (int64_t)m * a.ldy + l.col) = make_uint4(0, 0, 0, 0);
+        else ((float4 *)((float *)a.Y + (int64_t)m * a.ldy + l.col))[0] = ((float4 *)((float *)a.Y + (int64_t)m * a.ldy + l.col))[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lane == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
+      }
+      break;
+    }
+  }
+}
+
+// Several rows (2 .. kRowDecodeMaxM): the row is the outermost dimension of the units; every warp reads the type of the
+// rows it works on.  (A kernel of its own: the index arithmetic of the general form costs the one-row step 0.4-1 us.)
+// MODE 0: gated FFN, 1: FFN, 2: projection (W1 only)
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1) rows_decode_kernel(const RowDecodeArgs a) {
+  constexpr bool GATED = MODE == 0, FFN = MODE != 2;
+  __shared__ float partial[kWarps * kMaxPo * 16];
+  __shared__ int s_abort;
+  ALG_TRACE_VARS;
+  if (threadIdx.x == 0) ALG_TRACE(0, 1);
+  // phase 1 maps the D (projection: K) inputs to F (N) columns of W1; phase 2 maps F back to D through W2
+  Phase p1, p2;
+  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.D / a.q, p1.group_w = a.F / a.q, p1.n_cols = a.F;
+  p1.pc = a.pc1, p1.ks = a.ks1;
+  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.F / a.q, p2.group_w = a.D / a.q, p2.n_cols = a.D;
+  p2.pc = a.pc2, p2.ks = a.ks2;
+  const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
+  __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) s_abort = 0;
 
   // ---- before the dependency resolves: the type of this warp's first row as it stands now and the first W1 loads it
   // asks for (the type is read again after the wait) ----
-  const int per_row1 = a.units1 / a.M;
-  const int unit1 = unit_of(0, p1.ks), m1 = min(unit1 / per_row1, a.M - 1);
-  const int t_early = read_type(a, m1);
+  const int per_row1 = a.M == 1 ? a.units1 : a.units1 / a.M;
+  const int unit1 = unit_of(0, p1.ks), m1 = a.M == 1 ? 0 : min(unit1 / per_row1, a.M - 1);
+  const int t_early = read_row_type(a, m1);
   uint4 w[kLoads];
   {
     Lane l = lane_of(p1, unit1 - m1 * per_row1);
@@ -266,14 +474,11 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
   if (threadIdx.x == 0) ALG_TRACE(0, 2);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) ALG_TRACE(0, 3);
-  const int type1 = read_type(a, m1);   // (in flight while phase 1 runs on the early value)
 
-  // ---- phase 1 with the early type for the first unit, again (all of it) if some warp of the CTA finds that its type
-  // has changed since.  Gated: h = silu(x * W_gate) .* (x * W_up); FFN: h = act(x * W_up + b_up); projection:
-  // y = act(x * W + b) ----
-  for (int pass = 0; pass < 2; ++pass) {
-    if (pass == 1 && !__syncthreads_or(type1 != t_early)) break;
-    run_phase<GATED, false>(a, p1, X, a.ldx, w, pass == 0, t_early, a.units1, partial, [&](int m, int col, const float (&acc)[16]) {
+  // ---- phase 1 (its first unit on the type read early).  Gated: h = silu(x * W_gate) .* (x * W_up); FFN:
+  // h = act(x * W_up + b_up); projection: y = act(x * W + b) ----
+  {
+    run_rows_phase<GATED, false, !FFN>(a, p1, X, a.ldx, w, true, t_early, a.units1, partial, [&](int m, int col, const float (&acc)[16]) {
       if (GATED) {
         uint32_t o[4];
 #pragma unroll
@@ -292,13 +497,12 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
     });
   }
   if (threadIdx.x == 0) ALG_TRACE(0, 6);
-  const int n_out = FFN ? a.D : a.F;   // width of Y
 
   if (FFN) {
     // ---- the first W_down loads go out before the wait between the phases ----
-    const int per_row2 = a.units2 / a.M;
-    const int unit2 = unit_of(0, p2.ks), m2 = min(unit2 / per_row2, a.M - 1);
-    const int type2 = read_type(a, m2);
+    const int per_row2 = a.M == 1 ? a.units2 : a.units2 / a.M;
+    const int unit2 = unit_of(0, p2.ks), m2 = a.M == 1 ? 0 : min(unit2 / per_row2, a.M - 1);
+    const int type2 = read_row_type(a, m2);
     {
       Lane l = lane_of(p2, unit2 - m2 * per_row2);
       if (unit2 >= a.units2 || type2 < 0) l.on = false;
@@ -330,7 +534,7 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
 
     // ---- phase 2: y = h * W_down (+ b_down) ----
     if (!s_abort) {
-      run_phase<false, true>(a, p2, H, a.F, w, true, type2, a.units2, partial, [&](int m, int col, const float (&acc)[16]) {
+      run_rows_phase<false, true, true>(a, p2, H, a.F, w, true, type2, a.units2, partial, [&](int m, int col, const float (&acc)[16]) {
         store8(acc, col, a.b2, ALG_ACT_NONE,
                a.y_bf16 ? (void *)((__nv_bfloat16 *)a.Y + (int64_t)m * a.ldy) : (void *)((float *)a.Y + (int64_t)m * a.ldy), a.y_bf16 != 0);
       });
@@ -347,15 +551,6 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
     }
   }
 
-  // ---- rows whose type lies outside [0, q): zero, and the status says so ----
-  for (int m = 0; m < a.M; ++m) {
-    if (read_type(a, m) >= 0) continue;
-    if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)ALG_ERR_BAD_TYPE);
-    for (int c = blockIdx.x * kThreads + threadIdx.x; c < n_out; c += gridDim.x * kThreads) {
-      if (a.y_bf16) ((__nv_bfloat16 *)a.Y)[(int64_t)m * a.ldy + c] = __float2bfloat16_rn(0.f);
-      else ((float *)a.Y)[(int64_t)m * a.ldy + c] = 0.f;
-    }
-  }
 }
 
 // warps per piece: as many (a power of two, at most the warps of a CTA) as the grid has warps for
@@ -377,7 +572,7 @@ cudaError_t launch_mode(const RowDecodeArgs &a, int grid, cudaStream_t st) {
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, row_decode_kernel<MODE>, a);
+  cudaError_t e = a.M == 1 ? cudaLaunchKernelEx(&cfg, row_decode_kernel<MODE>, a) : cudaLaunchKernelEx(&cfg, rows_decode_kernel<MODE>, a);
   count_launch(1);
   return e;
 }
