@@ -327,6 +327,8 @@ struct RowDecodeArgs {
   int64_t ldy;
   int y_bf16;
   int D, F, q;
+  int gs, gr;               // group widths D / q and F / q, and their reciprocals  (set by the launcher)
+  float inv_gs, inv_gr;
   int pc1, pc2;             // columns of a warp's piece (8 or 16)                 (set by the launcher)
   int ks1, ks2;             // warps sharing the weight rows of a piece            (set by the launcher)
   int units1, units2;       // pieces x sharing warps                              (set by the launcher)

@@ -28,8 +28,8 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kLoads = 32;   // 16-byte weight loads a lane keeps in flight
-constexpr int kMaxPo = 8;
-constexpr int kPieceCols = 16;   // columns of a piece where the group width allows (32 and 64 measured the same or slower)    // a piece has at most 8 x 8 columns
+constexpr int kMaxPo = 8;     // a piece has at most 8 x 8 columns
+constexpr int kPieceCols = 16;   // columns of a piece where the group width allows (32 and 64 measured the same or slower)
 
 // One matrix-vector phase as the kernel sees it.
 struct Phase {
@@ -37,6 +37,7 @@ struct Phase {
   int64_t ldw;
   int s;                    // rows of one input group
   int group_w;              // columns of one output group
+  float inv_group_w;
   int n_cols;               // output columns (GATED: the up columns sit n_cols further in the bank)
   int pc;                   // columns of a piece: 8, 16, 32 or 64
   int ks;                   // warps that share the rows of a piece: 1, 2, 4 or 8
@@ -56,14 +57,19 @@ struct Lane {
   int piece, part, sub, lr, rl, col, j;
   bool on;
 };
+// (ks and pc / 8 are powers of two: shifts, and the group of a column by a reciprocal -- the step is bound by latency,
+// and a handful of integer divisions on the way to the first load are a few hundred cycles of it)
 __device__ __forceinline__ Lane lane_of(const Phase &p, int unit) {
   Lane l;
-  const int lane = threadIdx.x & 31, po = p.pc >> 3;
-  l.piece = unit / p.ks, l.part = unit - l.piece * p.ks;
-  l.sub = lane & (po - 1), l.lr = lane / po, l.rl = 32 / po;
+  const int lane = threadIdx.x & 31, po = p.pc >> 3, po_sh = __ffs(po) - 1, ks_sh = __ffs(p.ks) - 1;
+  l.piece = unit >> ks_sh, l.part = unit & (p.ks - 1);
+  l.sub = lane & (po - 1), l.lr = lane >> po_sh, l.rl = 32 >> po_sh;
   l.col = l.piece * p.pc + 8 * l.sub;
   l.on = l.col < p.n_cols;
-  l.j = l.on ? l.col / p.group_w : 0;
+  int j = (int)(((float)l.col + 0.5f) * p.inv_group_w);   // exact below 2^22 columns up to one step, corrected here
+  if (j * p.group_w > l.col) --j;
+  if ((j + 1) * p.group_w <= l.col) ++j;
+  l.j = l.on ? j : 0;
   return l;
 }
 
@@ -72,8 +78,8 @@ __device__ __forceinline__ Lane lane_of(const Phase &p, int unit) {
 // six warps each, not eight on 96 of them; measured equal to the blocked order -- the step is bound by the chain of
 // round trips, not by any one SM).
 __device__ __forceinline__ int unit_of(int rd, int ks) {
-  const int warp = threadIdx.x >> 5, slot = warp / ks, part = warp - slot * ks;
-  const int piece = (rd * (kWarps / ks) + slot) * gridDim.x + blockIdx.x;
+  const int warp = threadIdx.x >> 5, ks_sh = __ffs(ks) - 1, slot = warp >> ks_sh, part = warp & (ks - 1);
+  const int piece = (rd * (kWarps >> ks_sh) + slot) * gridDim.x + blockIdx.x;
   return piece * ks + part;
 }
 
@@ -83,7 +89,7 @@ template <bool GATED>
 __device__ __forceinline__ void load_chunk(uint4 (&w)[kLoads], const Phase &p, const Lane &l, int type, int c0) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
-  const int nr = (p.s + step - 1) / step - c0;   // rows of this chunk some lane has (the same in every lane)
+  const int nr = ((p.s + step - 1) >> (__ffs(step) - 1)) - c0;   // rows of this chunk some lane has (the same in every lane)
 #pragma unroll
   for (int sg = 0; sg < 2; ++sg) {
     const int g = sg == 0 ? l.j : type;
@@ -108,7 +114,7 @@ __device__ __forceinline__ void fma_chunk(const uint4 (&w)[kLoads], const Phase 
                                           const __nv_bfloat16 *x, float (&acc)[16]) {
   constexpr int RC = GATED ? kLoads / 4 : kLoads / 2;
   const int step = p.ks * l.rl, first = l.part * l.rl + l.lr;
-  const int nr = (p.s + step - 1) / step - c0;   // rows of this chunk some lane has (the same in every lane)
+  const int nr = ((p.s + step - 1) >> (__ffs(step) - 1)) - c0;   // rows of this chunk some lane has (the same in every lane)
   float xv[2 * RC];
 #pragma unroll
   for (int sg = 0; sg < 2; ++sg) {
@@ -157,7 +163,7 @@ __device__ __forceinline__ void run_phase(const Phase &p, int type, const __nv_b
     float acc[16];
 #pragma unroll
     for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
-    const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
+    const int rows_per_lane = (p.s + p.ks * l.rl - 1) >> (__ffs(p.ks * l.rl) - 1);
     for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
       if (!(have_first && rd == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, type, c0);
       fma_chunk<GATED, FROM_L2>(w, p, l, type, c0, x, acc);
@@ -238,9 +244,9 @@ __global__ void __launch_bounds__(kThreads, 1) row_decode_kernel(const RowDecode
   if (threadIdx.x == 0) ALG_TRACE(0, 1);
   // phase 1 maps the D (projection: K) inputs to F (N) columns of W1; phase 2 maps F back to D through W2
   Phase p1, p2;
-  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.D / a.q, p1.group_w = a.F / a.q, p1.n_cols = a.F;
+  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.gs, p1.group_w = a.gr, p1.inv_group_w = a.inv_gr, p1.n_cols = a.F;
   p1.pc = a.pc1, p1.ks = a.ks1;
-  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.F / a.q, p2.group_w = a.D / a.q, p2.n_cols = a.D;
+  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.gr, p2.group_w = a.gs, p2.inv_group_w = a.inv_gs, p2.n_cols = a.D;
   p2.pc = a.pc2, p2.ks = a.ks2;
   const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
   __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
@@ -397,7 +403,7 @@ __device__ __forceinline__ void run_rows_phase(const RowDecodeArgs &a, const Pha
       float acc[16];
 #pragma unroll
       for (int cc = 0; cc < 16; ++cc) acc[cc] = 0.f;
-      const int rows_per_lane = (p.s + p.ks * l.rl - 1) / (p.ks * l.rl);
+      const int rows_per_lane = (p.s + p.ks * l.rl - 1) >> (__ffs(p.ks * l.rl) - 1);
       for (int c0 = 0; c0 < rows_per_lane; c0 += RC) {
         if (!(have_first && rd == 0 && attempt == 0 && c0 == 0)) load_chunk<GATED>(w, p, l, max(type, 0), c0);
         fma_chunk<GATED, FROM_L2>(w, p, l, max(type, 0), c0, xm, acc);
@@ -451,9 +457,9 @@ __global__ void __launch_bounds__(kThreads, 1) rows_decode_kernel(const RowDecod
   if (threadIdx.x == 0) ALG_TRACE(0, 1);
   // phase 1 maps the D (projection: K) inputs to F (N) columns of W1; phase 2 maps F back to D through W2
   Phase p1, p2;
-  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.D / a.q, p1.group_w = a.F / a.q, p1.n_cols = a.F;
+  p1.W = (const __nv_bfloat16 *)a.W1, p1.ldw = a.ldw1, p1.s = a.gs, p1.group_w = a.gr, p1.inv_group_w = a.inv_gr, p1.n_cols = a.F;
   p1.pc = a.pc1, p1.ks = a.ks1;
-  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.F / a.q, p2.group_w = a.D / a.q, p2.n_cols = a.D;
+  p2.W = (const __nv_bfloat16 *)a.W2, p2.ldw = a.ldw2, p2.s = a.gr, p2.group_w = a.gs, p2.inv_group_w = a.inv_gs, p2.n_cols = a.D;
   p2.pc = a.pc2, p2.ks = a.ks2;
   const __nv_bfloat16 *X = (const __nv_bfloat16 *)a.X;
   __nv_bfloat16 *H = (__nv_bfloat16 *)a.H;
@@ -588,6 +594,7 @@ cudaError_t launch_row_decode(const RowDecodeArgs &in, int num_sms, cudaStream_t
   RowDecodeArgs a = in;
   if (a.mode < 0 || a.mode > 2 || a.M < 1 || a.M > kRowDecodeMaxM || !row_decode_fits(a.q, a.D, a.F)) return cudaErrorInvalidValue;
   const int s = a.D / a.q, r = a.F / a.q;
+  a.gs = s, a.gr = r, a.inv_gs = 1.f / (float)s, a.inv_gr = 1.f / (float)r;
   auto piece = [](int group_w) { return group_w % kPieceCols == 0 ? kPieceCols : group_w % 16 == 0 ? 16 : 8; };
   a.pc1 = piece(r);
   a.pc2 = piece(s);
