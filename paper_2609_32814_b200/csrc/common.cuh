@@ -207,6 +207,7 @@ struct BigArgs {
   const int *offsets;     // sched 0: device bucket offsets [q + 1]
   const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)
   int rows_per_type;      // sched 1, 2: M / q
+  float inv_per_type;     // reciprocal of the tiles per type (or per type group) for the tile decode; 0 = divide  (set by the launcher)
   int *status;
   long long wait_limit;
 };

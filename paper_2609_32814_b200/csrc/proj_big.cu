@@ -125,6 +125,16 @@ struct Tile {
   int n0_w;         // first column in the bank (differs from n0 when the bank's groups are padded)
 };
 
+// t / d for 0 <= t < 2^22 with the reciprocal of d from the host: the tile decode runs once per tile in every role, and
+// tiles of this path are short -- an integer division is a few dozen dependent instructions
+__device__ __forceinline__ int fast_div(int t, int d, float inv_d) {
+  if (inv_d == 0.f) return t / d;
+  int qt = (int)(((float)t + 0.5f) * inv_d);
+  if (qt * d > t) --qt;
+  if ((qt + 1) * d <= t) ++qt;
+  return qt;
+}
+
 // Tile t of the launch (uniform across the warp).  Type-major; inside a type: m-tile fastest, then
 // the column tile, then the output group.
 __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, int t) {
@@ -161,8 +171,8 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   }
   if (a.pack > 1) {   // type-group major, then the output group, then the column tile
     const int per_group = a.q * a.nt_n;
-    const int tg = t / per_group, rem = t - tg * per_group;
-    const int j = rem / a.nt_n, nt = rem - j * a.nt_n;
+    const int tg = fast_div(t, per_group, a.inv_per_type), rem = t - tg * per_group;
+    const int j = a.nt_n == 1 ? rem : rem / a.nt_n, nt = rem - j * a.nt_n;
     o.i = tg * a.pack, o.j = j;
     o.np = min(a.pack, a.q - o.i);
     o.row0 = o.i * a.rows_per_type;
@@ -176,7 +186,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
   if (a.sched != 0) {
     rows_i = a.rows_per_type;
     const int per_type = ((rows_i + 127) >> 7) * a.col_units;
-    i = t / per_type;
+    i = fast_div(t, per_type, a.inv_per_type);
     rem = t - i * per_type;
     base = i * rows_i;
   } else {
@@ -191,7 +201,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
     rows_i = ctl->off[i + 1] - base;
   }
   const int mt_i = (rows_i + 127) >> 7;
-  const int u = rem / mt_i, mt = rem - u * mt_i;
+  const int u = mt_i == 1 ? rem : rem / mt_i, mt = rem - u * mt_i;
   o.row0 = base + (mt << 7);
   o.rows = min(128, rows_i - (mt << 7));
   if (a.gpack > 1) {   // a tile of several whole output groups
@@ -202,7 +212,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
     o.cols = o.ng * a.r;   // columns of the accumulator in use (groups at their width in the bank)
     return o;
   }
-  const int j = u / a.nt_n, nt = u - j * a.nt_n;
+  const int j = a.nt_n == 1 ? u : u / a.nt_n, nt = u - j * a.nt_n;
   o.i = i, o.j = j;
   o.n0 = j * a.r_out + nt * a.tile_n;
   o.n0_w = j * a.r + nt * a.tile_n;
@@ -810,6 +820,11 @@ cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
       a.tile_n = (g * a.r + 15) / 16 * 16;
       a.n_chunks = (a.tile_n + 63) / 64;
     }
+  }
+  {
+    const long long per = a.pack > 1 ? (long long)a.q * a.nt_n : a.sched != 0 ? (long long)((a.rows_per_type + 127) / 128) * a.col_units : 0;
+    const long long total = a.pack > 1 ? per * ((a.q + a.pack - 1) / a.pack) : per * a.q;
+    a.inv_per_type = per > 0 && total < (1 << 22) ? 1.f / (float)per : 0.f;
   }
   if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
     if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;
