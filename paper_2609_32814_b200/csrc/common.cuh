@@ -208,6 +208,7 @@ struct BigArgs {
   const int *perm;        // sched 0: bucketed row -> output row (nullptr = identity)
   int rows_per_type;      // sched 1, 2: M / q
   float inv_per_type;     // reciprocal of the tiles per type (or per type group) for the tile decode; 0 = divide  (set by the launcher)
+  float inv_r;            // 1 / r: group of an accumulator column in tiles of several groups                   (set by the launcher)
   int *status;
   long long wait_limit;
 };

@@ -621,7 +621,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               const int64_t dr = dst_row[ph * 4 + g];
               if (a.gpack > 1) {
                 // the piece's 8 accumulator columns lie in one group of the tile: group gi, column cg of it
-                const int tc = c0 + rd_p * 8, gi = tc / a.r, cg = tc - gi * a.r;
+                const int tc = c0 + rd_p * 8, gi = fast_div(tc, a.r, a.inv_r), cg = tc - gi * a.r;
                 __nv_bfloat16 *dst = (__nv_bfloat16 *)a.Y + dr * a.ldy + tl.n0 + gi * a.r_out + cg;
                 const bool in_tile = dr >= 0 && gi < tl.ng;
                 if (store8) {
@@ -667,7 +667,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (out_row >= 0 && a.gpack > 1) {
 #pragma unroll
             for (int g = 0; g < 8; ++g) {   // four accumulator columns lie in one group of the tile
-              const int tc = c0 + g * 4, gi = tc / a.r, cg = tc - gi * a.r;
+              const int tc = c0 + g * 4, gi = fast_div(tc, a.r, a.inv_r), cg = tc - gi * a.r;
               if (gi < tl.ng && cg < a.r_out)
                 *(float4 *)((float *)a.Y + out_row * a.ldy + tl.n0 + gi * a.r_out + cg) = make_float4(f[g * 4], f[g * 4 + 1], f[g * 4 + 2], f[g * 4 + 3]);
             }
@@ -825,6 +825,7 @@ cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
     const long long per = a.pack > 1 ? (long long)a.q * a.nt_n : a.sched != 0 ? (long long)((a.rows_per_type + 127) / 128) * a.col_units : 0;
     const long long total = a.pack > 1 ? per * ((a.q + a.pack - 1) / a.pack) : per * a.q;
     a.inv_per_type = per > 0 && total < (1 << 22) ? 1.f / (float)per : 0.f;
+    a.inv_r = 1.f / (float)a.r;
   }
   if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
     if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;
