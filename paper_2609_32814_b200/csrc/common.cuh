@@ -209,6 +209,8 @@ struct BigArgs {
   int rows_per_type;      // sched 1, 2: M / q
   float inv_per_type;     // reciprocal of the tiles per type (or per type group) for the tile decode; 0 = divide  (set by the launcher)
   float inv_r;            // 1 / r: group of an accumulator column in tiles of several groups                   (set by the launcher)
+  float inv_g, inv_rpt;   // 1 / gpack, 1 / rows_per_type                                                          (set by the launcher)
+  int n_tg, n_units;      // type groups ceil(q / pack), column units ceil(q / gpack)                              (set by the launcher)
   int *status;
   long long wait_limit;
 };

@@ -146,7 +146,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
     // units (a.gpack groups each) that hold none of its types, one tile each, then the groups of the other units
     // one by one (a tile never holds a type together with other groups than its own: the diagonal product of
     // group k and the panel product of type k would both carry x_k W_kk)
-    int lo = 0, hi = (a.q + a.pack - 1) / a.pack;   // pre[lo] <= t < pre[hi]
+    int lo = 0, hi = a.n_tg;   // pre[lo] <= t < pre[hi]
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
       if (ctl->pre[mid] <= t) lo = mid; else hi = mid;
@@ -154,7 +154,7 @@ __device__ __forceinline__ Tile decode_tile(const BigArgs &a, const Ctl *ctl, in
     const int l = t - ctl->pre[lo], g = a.gpack;
     o.i = lo * a.pack;
     o.np = min(a.pack, a.q - o.i);
-    const int n_units = (a.q + g - 1) / g, ua = o.i / g, ub = (o.i + o.np - 1) / g, apart = n_units - (ub - ua + 1);
+    const int n_units = a.n_units, ua = fast_div(o.i, g, a.inv_g), ub = fast_div(o.i + o.np - 1, g, a.inv_g), apart = n_units - (ub - ua + 1);
     if (l < apart) {
       o.j = (l < ua ? l : l + (ub - ua + 1)) * g;
       o.ng = min(g, a.q - o.j);
@@ -491,7 +491,7 @@ proj_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       int64_t out_row = -1;
       if (r < tl.rows) {
         if (a.sched_out == 2 && a.pack > 1) {   // rows of a packed tile are type-major: type tl.i + r / rows_per_type
-          const int ti = r / a.rows_per_type;
+          const int ti = fast_div(r, a.rows_per_type, a.inv_rpt);
           out_row = (int64_t)(r - ti * a.rows_per_type) * q + tl.i + ti;
         } else if (a.sched_out == 2) out_row = (int64_t)(tl.row0 + r - tl.i * a.rows_per_type) * q + tl.i;
         else if (a.sched_out == 0 && a.perm) out_row = __ldg(a.perm + tl.row0 + r);
@@ -826,6 +826,10 @@ cudaError_t launch_proj_big(const BigArgs &in, int num_sms, cudaStream_t st) {
     const long long total = a.pack > 1 ? per * ((a.q + a.pack - 1) / a.pack) : per * a.q;
     a.inv_per_type = per > 0 && total < (1 << 22) ? 1.f / (float)per : 0.f;
     a.inv_r = 1.f / (float)a.r;
+    a.inv_g = 1.f / (float)a.gpack;
+    a.inv_rpt = a.rows_per_type > 0 ? 1.f / (float)a.rows_per_type : 0.f;
+    a.n_tg = (a.q + a.pack - 1) / a.pack;
+    a.n_units = (a.q + a.gpack - 1) / a.gpack;
   }
   if (a.gated_f) {   // two accumulator halves of n_chunks * 64 columns each
     if (a.tile_n > 128 || !a.y_bf16 || a.r != a.r_out || a.gated_f != a.q * a.r || a.bias || a.act) return cudaErrorInvalidValue;
