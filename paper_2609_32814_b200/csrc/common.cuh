@@ -263,6 +263,7 @@ struct DecodeArgs {
   int K;
   int N;
   int splits;
+  uint32_t inv_splits;    // ceil(2^32 / splits): x / splits = umulhi(x, inv_splits) for x < 2^29, splits > 1 (set by the launcher)
   int box_rows;
   int w_smem_bytes;
   int x_smem_bytes;

@@ -113,6 +113,9 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   const int q = a.q;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int strip = blockIdx.x, split = blockIdx.y, splits = gridDim.y;
+  // x / splits = __umulhi(x, a.inv_splits) for every x the kernel divides (below 2^29): no integer division on the way
+  const uint32_t inv_splits = a.inv_splits;
+  auto div_splits = [&](int x) { return splits == 1 ? x : (int)__umulhi((uint32_t)x, inv_splits); };
   const int n0 = strip * SN;
   const int M = a.M;
   const int m_tiles = (M + 15) >> 4, m_pad = m_tiles << 4;
@@ -166,7 +169,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
       int len = 0;
       if (lane < q) {
         lo = s_rows32[lane][0], hi = s_rows32[lane][1];
-        if (lo | hi) len = (s_so[lane + 1] - s_so[lane]) / splits;  // nobody needs W_kj -> it is never read
+        if (lo | hi) len = div_splits(s_so[lane + 1] - s_so[lane]);  // nobody needs W_kj -> it is never read
       }
       const unsigned have = __ballot_sync(0xffffffffu, len > 0);
       int incl = len;
@@ -294,7 +297,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   }
   DTR();
   // ---- push the partial sums to the owners of the rows: row m -> CTA m % splits, slot m / splits ----
-  const int rows_owned_max = (m_pad + splits - 1) / splits;
+  const int rows_owned_max = div_splits(m_pad + splits - 1);
   {
     const uint32_t r_base = smem_u32(r_sm);
     const int g = lane >> 2, t4 = lane & 3;
@@ -304,8 +307,8 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const int m = mt * 16 + g + h * 8;
-          const uint32_t owner = (uint32_t)(m % splits);
-          const int slot = m / splits;
+          const int slot = div_splits(m);
+          const uint32_t owner = (uint32_t)(m - slot * splits);
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             const int col = warp * (SN / 4) + nt * 8 + t4 * 2;
@@ -324,7 +327,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   // ---- add the partial sums of my rows in split order, bias, activation, store ----
   {
     constexpr int kGroups = SN / 4;
-    const int my_rows = (M - split + splits - 1) / splits;  // rows m = split + splits * slot < M
+    const int my_rows = div_splits(M - split + splits - 1);  // rows m = split + splits * slot < M
     for (int e = tid; e < my_rows * kGroups; e += kThreads) {
       const int slot = e / kGroups, n = (e % kGroups) * 4;
       const int m = split + slot * splits;
@@ -436,6 +439,7 @@ bool decode_plan(int q, const int *s, int K, int N, int num_sms, DecodePlan *pla
 cudaError_t launch_decode(const DecodeArgs &a, const DecodePlan &plan, cudaStream_t st) {
   DecodeArgs b = a;
   b.splits = plan.splits;
+  b.inv_splits = (uint32_t)((0x100000000ull + (uint64_t)plan.splits - 1) / (uint64_t)plan.splits);
   b.box_rows = plan.box_rows;
   b.w_smem_bytes = plan.w_smem_bytes;
   b.x_smem_bytes = plan.x_smem_bytes;
