@@ -237,3 +237,53 @@ def test_gated_refusals():
     assert e.value.code == 2
     with pytest.raises(binding.AlgError):
         binding.GatedFFN([64, 64], [128, 128], dtype="f32")
+
+
+@pytest.mark.parametrize("M", [1, 3])
+def test_gated_decode_chain_in_a_graph_replays(M):
+    """Five dependent gated layers (distinct weights, layer l+1 reads layer l's output) captured in one CUDA graph, as
+    the benchmark's decode chain does: consecutive launches overlap through programmatic dependent launch (every launch
+    requests its weights before the one before it has finished) and share the handle's exchange counters.  Every replay
+    reproduces, bit for bit, the layers run one at a time with a device synchronisation between them; that result is
+    checked against the oracle layer by layer."""
+    q, dw, fw, L = 32, 64, 192, 5
+    types = synth.uniform_types(77, M, q)
+    wl, _ = synth.gated_ffn("gated-chain", q, M, q * dw, q * fw, types, variant=1)
+    D, F = q * dw, q * fw
+    ffn = binding.GatedFFN(wl.d_widths, wl.f_widths, dtype="bf16")
+    ffn.set_option("small_m_kernel", 3)
+    t = H.dev_types(types)
+    # (weights large enough that the activations do not die out along the chain: the gated map is quadratic in x)
+    Wgu_h = [synth.bf16_round(synth.normal(300 + l, (D, 2 * F), 0.12)) for l in range(L)]
+    Wd_h = [synth.bf16_round(synth.normal(400 + l, (F, D), 0.12)) for l in range(L)]
+    Wgu, Wd = [H.to_dev(w, "bf16") for w in Wgu_h], [H.to_dev(w, "bf16") for w in Wd_h]
+    acts = [H.to_dev(wl.X, "bf16")] + [torch.zeros((M, D), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    ws = torch.empty(ffn.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    want = [acts[0]]
+    for l in range(L):       # one layer at a time
+        n0 = binding.launch_count()
+        want.append(ffn.forward(want[l], t, Wgu[l], Wd[l], workspace=ws))
+        assert binding.launch_count() - n0 == 1
+        torch.cuda.synchronize()
+        ref = oracle.ffn_swiglu(H.to_np(want[l]), types, Wgu_h[l][:, :F], Wgu_h[l][:, F:], Wd_h[l], wl.d_widths, wl.f_widths)
+        assert H.rel_fro(H.to_np(want[l + 1]), ref) <= H.BF16_REL_FRO, f"layer {l}"    # (magnitudes grow along the chain)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        for l in range(L):   # back to back, overlapping
+            ffn.forward(acts[l], t, Wgu[l], Wd[l], out=acts[l + 1], workspace=ws, stream=stream)
+        stream.synchronize()
+        for l in range(L):
+            assert torch.equal(acts[l + 1], want[l + 1]), f"eager layer {l}"
+        with torch.cuda.graph(g, stream=stream):
+            for l in range(L):
+                ffn.forward(acts[l], t, Wgu[l], Wd[l], out=acts[l + 1], workspace=ws, stream=stream)
+    for rep in range(4):
+        for l in range(L):
+            acts[l + 1].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for l in range(L):
+            assert torch.equal(acts[l + 1], want[l + 1]), f"replay {rep} layer {l}"
+    assert ffn.last_status() == 0
