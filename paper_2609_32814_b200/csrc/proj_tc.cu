@@ -479,7 +479,11 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_wait_ld();
           float f[32];
 #pragma unroll
-          for (int x = 0; x < 32; ++x) f[x] = empty_tile ? 0.f : __uint_as_float(v[x]);
+          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          if (empty_tile) {   // (rare and the same for the whole tile: a branch, not 32 selects per chunk)
+#pragma unroll
+            for (int x = 0; x < 32; ++x) f[x] = 0.f;
+          }
           finish_32(f, a, col_base + c0);
           uint32_t w[16];
           pack_bf16_32(f, w);
