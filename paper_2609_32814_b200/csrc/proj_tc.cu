@@ -515,7 +515,11 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (out_row >= 0) {
           float f[32];
 #pragma unroll
-          for (int x = 0; x < 32; ++x) f[x] = empty_tile ? 0.f : __uint_as_float(v[x]);
+          for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
+          if (empty_tile) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) f[x] = 0.f;
+          }
           finish_and_store_32(f, a, out_row, col_base + c0);
         }
       }
