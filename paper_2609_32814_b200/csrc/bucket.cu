@@ -140,10 +140,20 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
 // and writes perm.  All CTAs are resident together: the grid is far smaller than the machine, and
 // the kernel launched after it starts only once every CTA of this one has.  The last CTA past the
 // wait clears the counter for the next launch.
+//
+// CLUSTER (M <= 8192): the CTAs form one thread-block cluster; the per-type counts stay in shared memory, the
+// cluster's hardware barrier replaces the counter and every CTA reads its peers' counts through the cluster's
+// shared-memory window -- no round trip to L2 between the ranking and the write of perm.
 constexpr int kFusedThreads = 1024;
+constexpr int kClusterRows = 8 * kFusedThreads;
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+template <bool CLUSTER>
 __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const BucketArgs a) {
   __shared__ int s_wcnt[32][kMaxQ + 1];   // rows of type t in warp w; then exclusive prefix over the warps
   __shared__ int s_base[kMaxQ + 1], s_offset[kMaxQ + 2];
+  __shared__ int s_tot[kMaxQ + 1];        // CLUSTER: rows of type t in this CTA, read by the peers
   __shared__ int s_go;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nt = a.q + 1;
@@ -174,10 +184,33 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
     }
     s_wcnt[lane][ty] = incl - v;
     if (lane == 31) {
-      a.chunk_counts[blockIdx.x * nt + ty] = incl;
-      __threadfence();
+      if (CLUSTER) {
+        s_tot[ty] = incl;
+      } else {
+        a.chunk_counts[blockIdx.x * nt + ty] = incl;
+        __threadfence();
+      }
     }
   }
+  if (CLUSTER) {
+    cluster_sync_all();   // (also orders the shared-memory writes above for this CTA's own threads)
+    for (int ty = warp; ty < nt; ty += kFusedThreads / 32) {   // lanes over the CTAs of the cluster (at most 8)
+      int v = 0;
+      if (lane < n_chunks) {
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(&s_tot[ty])), "r"(lane));
+        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+      }
+      int before = lane < (int)blockIdx.x ? v : 0, total = v;
+#pragma unroll
+      for (int d = 4; d > 0; d >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, d);
+        total += __shfl_xor_sync(0xffffffffu, total, d);
+      }
+      if (lane == 0) s_base[ty] = before, s_offset[ty] = total;
+    }
+    cluster_sync_all();   // no CTA leaves (or overwrites s_tot) while a peer may still read its counts
+  } else {
   __syncthreads();
   if (tid == 0) {
     ALG_TRACE(0, 4);
@@ -216,6 +249,7 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
     }
   }
   __syncthreads();
+  }
   if (tid == 0) ALG_TRACE(0, 6);
   if (warp == 0) {   // bucket offsets: exclusive prefix of the totals over the types (nt <= 33: lane 0 takes two)
     const int v0 = lane < nt ? s_offset[lane] : 0, v1 = lane == 0 && nt > 32 ? s_offset[32] : 0;
@@ -419,9 +453,26 @@ cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
     count_launch(2);
     return cudaGetLastError();
   }
+  if (a.M <= kClusterRows) {   // one kernel, one cluster of 1, 2, 4 or 8 CTAs (CTAs past the batch hold no row)
+    int n_cta = 1;
+    while (n_cta * kFusedThreads < a.M) n_cta *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_cta, 1, 1);
+    cfg.blockDim = dim3(kFusedThreads, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = n_cta, at[1].val.clusterDim.y = 1, at[1].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 2;
+    count_launch(1);
+    return cudaLaunchKernelEx(&cfg, bucket_onepass_kernel<true>, a);
+  }
   if (a.M <= 65536 && a.sync) {  // one kernel, every row type read once
     count_launch(1);
-    return launch_pdl(bucket_onepass_kernel, ceil_div(a.M, kFusedThreads), kFusedThreads, st, a);
+    return launch_pdl(bucket_onepass_kernel<false>, ceil_div(a.M, kFusedThreads), kFusedThreads, st, a);
   }
   const int n_chunks = ceil_div(a.M, a.chunk_rows);
   bucket_count_kernel<kMaxQ + 1><<<n_chunks, 256, 0, st>>>(a);

@@ -223,6 +223,28 @@ def test_bucketing_beyond_65536_rows():
     assert np.array_equal(got[good], ref[good])
 
 
+@pytest.mark.parametrize("M", [1, 1023, 1025, 2048, 2049, 4097, 8191, 8192, 8193])
+def test_bucketing_across_the_cluster_sizes(M):
+    """Up to 8192 rows the bucketing kernel is one cluster of 1, 2, 4 or 8 CTAs that exchange their counts
+    through shared memory; one row more takes the variant with the counter in global memory.  Skewed types
+    (one type absent, one holding half the rows), bit-exact on integer data, and an out-of-range type in the
+    last row."""
+    q = 4
+    wl = _tc_workload(q, M, 64, 128, seed=300 + M % 97)
+    rng = np.random.default_rng(M)
+    types = rng.choice(np.array([0, 2, 2, 3], np.int32), size=M)      # type 1 never occurs
+    proj = binding.Proj(wl.d_widths, wl.f_widths, dtype="bf16")
+    X, W = H.to_dev(wl.X, "bf16"), H.to_dev(wl.W_up, "bf16")
+    Y = proj.forward(X, H.dev_types(types), W, out_dtype=torch.float32)
+    assert proj.last_status() == 0
+    ref = oracle.proj(wl.X, types, wl.W_up, wl.d_widths, wl.f_widths)
+    assert np.array_equal(H.to_np(Y), ref)
+    types[M - 1] = q + 5
+    Yb = H.to_np(proj.forward(X, H.dev_types(types), W, out_dtype=torch.float32))
+    assert proj.last_status() == 5
+    assert not Yb[M - 1].any() and np.array_equal(Yb[:M - 1], ref[:M - 1])
+
+
 def test_options_tile_width_and_in_kernel_plan():
     """Every tile width that divides the groups, and both ways of planning the cyclic schedule,
     give the same bits."""
