@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(256) bucket_scatter_kernel(const BucketArgs a)
 // the kernel launched after it starts only once every CTA of this one has.  The last CTA past the
 // wait clears the counter for the next launch.
 //
-// CLUSTER (M <= 8192): the CTAs form one thread-block cluster; the per-type counts stay in shared memory, the
+// CLUSTER (M <= 8192, M <= 16384 where the device takes clusters of 16): the CTAs form one thread-block cluster; the per-type counts stay in shared memory, the
 // cluster's hardware barrier replaces the counter and every CTA reads its peers' counts through the cluster's
 // shared-memory window -- no round trip to L2 between the ranking and the write of perm.
 constexpr int kFusedThreads = 1024;
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
   }
   if (CLUSTER) {
     cluster_sync_all();   // (also orders the shared-memory writes above for this CTA's own threads)
-    for (int ty = warp; ty < nt; ty += kFusedThreads / 32) {   // lanes over the CTAs of the cluster (at most 8)
+    for (int ty = warp; ty < nt; ty += kFusedThreads / 32) {   // lanes over the CTAs of the cluster (at most 16)
       int v = 0;
       if (lane < n_chunks) {
         uint32_t remote;
@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(kFusedThreads) bucket_onepass_kernel(const Buc
       }
       int before = lane < (int)blockIdx.x ? v : 0, total = v;
 #pragma unroll
-      for (int d = 4; d > 0; d >>= 1) {
+      for (int d = 8; d > 0; d >>= 1) {
         before += __shfl_xor_sync(0xffffffffu, before, d);
         total += __shfl_xor_sync(0xffffffffu, total, d);
       }
@@ -453,7 +453,25 @@ cudaError_t launch_bucket(const BucketArgs &a, cudaStream_t st) {
     count_launch(2);
     return cudaGetLastError();
   }
-  if (a.M <= kClusterRows) {   // one kernel, one cluster of 1, 2, 4 or 8 CTAs (CTAs past the batch hold no row)
+  // clusters of 16 are not portable: asked for once, used where the device says one can be resident
+  static int rows16 = -1;
+  if (rows16 < 0) {
+    rows16 = 0;
+    if (cudaFuncSetAttribute(bucket_onepass_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t probe = {};
+      probe.gridDim = dim3(16, 1, 1);
+      probe.blockDim = dim3(kFusedThreads, 1, 1);
+      cudaLaunchAttribute pa[1];
+      pa[0].id = cudaLaunchAttributeClusterDimension;
+      pa[0].val.clusterDim.x = 16, pa[0].val.clusterDim.y = 1, pa[0].val.clusterDim.z = 1;
+      probe.attrs = pa;
+      probe.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, bucket_onepass_kernel<true>, &probe) == cudaSuccess && n > 0) rows16 = 16 * kFusedThreads;
+    }
+    (void)cudaGetLastError();
+  }
+  if (a.M <= std::max(kClusterRows, rows16)) {   // one kernel, one cluster of 1 ... 16 CTAs (CTAs past the batch hold no row)
     int n_cta = 1;
     while (n_cta * kFusedThreads < a.M) n_cta *= 2;
     cudaLaunchConfig_t cfg = {};

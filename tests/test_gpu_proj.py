@@ -223,10 +223,11 @@ def test_bucketing_beyond_65536_rows():
     assert np.array_equal(got[good], ref[good])
 
 
-@pytest.mark.parametrize("M", [1, 1023, 1025, 2048, 2049, 4097, 8191, 8192, 8193])
+@pytest.mark.parametrize("M", [1, 1023, 1025, 2048, 2049, 4097, 8191, 8192, 8193, 16384, 16385])
 def test_bucketing_across_the_cluster_sizes(M):
-    """Up to 8192 rows the bucketing kernel is one cluster of 1, 2, 4 or 8 CTAs that exchange their counts
-    through shared memory; one row more takes the variant with the counter in global memory.  Skewed types
+    """Up to 8192 rows (16384 where the device takes clusters of 16) the bucketing kernel is one cluster of
+    1 ... 16 CTAs that exchange their counts through shared memory; one row more takes the variant with the
+    counter in global memory.  Skewed types
     (one type absent, one holding half the rows), bit-exact on integer data, and an out-of-range type in the
     last row."""
     q = 4
